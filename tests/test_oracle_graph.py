@@ -1,0 +1,127 @@
+"""Pins for the oracle's graph evaluation: an independent float64 numpy evaluation of the same
+graph descriptions (sliding windows + einsum, no shared code), and fused == unfused."""
+import numpy as np
+import pytest
+from numpy.lib.stride_tricks import sliding_window_view
+
+from oracle import compile as oc
+from oracle import graph as og
+from paper_1907_01989_b200 import workloads as wl
+
+
+def np_eval(g, x):
+    """Evaluate the *unfused* graph in float64 with numpy only."""
+    val = {g.inputs[0]: x.astype(np.float64)}
+    for k, t in enumerate(g.inputs[1:], 1):
+        raise AssertionError("single-input graphs only")
+    for op in g.ops:
+        a = val[op.inputs[0]]
+        if op.kind in ("conv2d", "depthwise_conv2d"):
+            pt, pl, pb, pr = op.pads
+            ap = np.pad(a, ((0, 0), (pt, pb), (pl, pr), (0, 0)))
+            kh, kw = op.kh, op.kw
+            eh, ew = (kh - 1) * op.dilation[0] + 1, (kw - 1) * op.dilation[1] + 1
+            win = sliding_window_view(ap, (eh, ew), axis=(1, 2))          # B, H', W', C, eh, ew
+            win = win[:, ::op.stride[0], ::op.stride[1], :, ::op.dilation[0], ::op.dilation[1]]
+            w = op.weights.astype(np.float64)
+            if op.kind == "conv2d":
+                y = np.einsum("bhwcyx,oyxc->bhwo", win, w, optimize=True)
+            else:
+                y = np.einsum("bhwcyx,yxc->bhwc", win, w[0], optimize=True)
+            if op.bias is not None:
+                y = y + op.bias.astype(np.float64)
+        elif op.kind == "activation":
+            y = np.maximum(a, 0.0)
+            if op.act == "relu6":
+                y = np.minimum(y, 6.0)
+        elif op.kind == "add":
+            y = a + val[op.inputs[1]]
+        elif op.kind == "global_avg_pool":
+            y = a.mean(axis=(1, 2), keepdims=True)
+        elif op.kind == "resize_bilinear":
+            oh, ow = op.out_hw
+            assert op.align_corners
+            H, W = a.shape[1:3]
+            fy = np.arange(oh) * (H - 1) / (oh - 1)
+            fx = np.arange(ow) * (W - 1) / (ow - 1)
+            y0 = np.minimum(np.floor(fy).astype(int), H - 1)
+            x0 = np.minimum(np.floor(fx).astype(int), W - 1)
+            y1, x1 = np.minimum(y0 + 1, H - 1), np.minimum(x0 + 1, W - 1)
+            wy, wx = (fy - y0)[None, :, None, None], (fx - x0)[None, None, :, None]
+            rows0 = a[:, y0][:, :, x0] * (1 - wx) + a[:, y0][:, :, x1] * wx
+            rows1 = a[:, y1][:, :, x0] * (1 - wx) + a[:, y1][:, :, x1] * wx
+            y = rows0 * (1 - wy) + rows1 * wy
+        else:
+            raise ValueError(op.kind)
+        val[op.output] = y
+    return val
+
+
+NETS = [
+    ("separable_block", lambda: wl.separable_block(2)),
+    ("mobilenet_v1", lambda: wl.mobilenet_v1(1, size=96)),
+    ("mobilenet_v2", lambda: wl.mobilenet_v2(1, size=96)),
+    ("segmentation", lambda: wl.mobilenet_v2_segmentation(1, size=65)),
+]
+
+
+@pytest.mark.parametrize("name,make", NETS)
+def test_oracle_matches_float64_numpy_on_every_tensor(name, make):
+    g = make()
+    x = wl.make_input(g)
+    ref = np_eval(g, x)
+    got = og.run(g, [x], storage="f32", fused=False, keep_all=True)
+    assert set(got) == set(ref)
+    for t in got:
+        scale = max(1.0, float(np.abs(ref[t]).max()))
+        np.testing.assert_allclose(got[t], ref[t], rtol=0, atol=2e-5 * scale, err_msg=f"{name} tensor {t}")
+    # fused evaluation agrees with the same reference on the tensors that survive fusion
+    fused = og.run(g, [x], storage="f32", fused=True, keep_all=True)
+    for t in fused:
+        scale = max(1.0, float(np.abs(ref[t]).max()))
+        np.testing.assert_allclose(fused[t], ref[t], rtol=0, atol=2e-5 * scale)
+
+
+def test_full_size_mobilenet_v2_against_numpy():
+    g = wl.mobilenet_v2(1)
+    x = wl.make_input(g)
+    ref = np_eval(g, x)
+    got = og.run(g, [x], storage="f32", fused=True)
+    out = g.outputs[0]
+    assert got[out].shape == (1, 1, 1, 1001)
+    np.testing.assert_allclose(got[out], ref[out], rtol=0, atol=2e-5 * max(1.0, np.abs(ref[out]).max()))
+
+
+@pytest.mark.parametrize("name,make", NETS)
+def test_fused_equals_unfused(name, make):
+    g = make()
+    x = wl.make_input(g)
+    a = og.run(g, [x], storage="f32", fused=True)
+    b = og.run(g, [x], storage="f32", fused=False)
+    for t in g.outputs:
+        assert np.array_equal(a[t], b[t])  # same fp32 values through the same epilogue order: bit-exact
+    a = og.run(g, [x], storage="f16", fused=True, keep_all=True)
+    b = og.run(g, [x], storage="f16", fused=False, keep_all=True)
+    for t in a:
+        # fp16 storage: the unfused graph rounds between conv, activation and add; fusing removes
+        # roundings, so the two differ by a few fp16 ulps that then propagate
+        assert np.all(np.abs(a[t] - b[t]) <= 1e-2 + 1e-2 * np.abs(b[t])), (name, t)
+
+
+def test_f16_storage_values_are_representable():
+    g = wl.separable_block(1)
+    x = wl.make_input(g)
+    r = og.run(g, [x], storage="f16", keep_all=True)
+    for t, v in r.items():
+        assert np.array_equal(v, v.astype(np.float16).astype(np.float32))
+
+
+def test_input_generator_is_batch_independent():
+    g4, g2 = wl.mobilenet_v2(4, size=32), wl.mobilenet_v2(2, size=32)
+    x4 = wl.make_input(g4)
+    assert np.array_equal(wl.make_input(g2, images=[1, 3]), x4[[1, 3]])
+    assert np.array_equal(x4, x4.astype(np.float16).astype(np.float32))
+    assert x4.min() >= -1 and x4.max() <= 1
+    for a, b in zip(g4.ops, g2.ops):
+        if a.weights is not None:
+            assert np.array_equal(a.weights, b.weights) and np.array_equal(a.bias, b.bias)
