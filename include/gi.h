@@ -1,0 +1,233 @@
+/*
+ * gi - graph inference of fused convolutional networks on one NVIDIA B200 (sm_100a).
+ *
+ * The library implements the GPU inference path of "On-Device Neural Net Inference with
+ * Mobile GPUs" (arXiv 1907.01989): a sub-graph of supported operators is handed over once,
+ * initialised once, then run many times (Section 3, "General Architecture").
+ *
+ *   build    gi_graph_create / gi_graph_input / gi_add_op / gi_graph_output
+ *   compile  gi_compile   - topological order, fusion of element-wise operators into the
+ *                           convolution before them (Section 3.2), tensor lifetimes and the
+ *                           memory plan for intermediate tensors (Section 5), weight packing
+ *   run      gi_exec_bind, gi_run - enqueue every kernel on the caller's stream, no
+ *                           synchronisation with the CPU (Section 3.2, "Running Inference")
+ *
+ * All functions return a gi_status; none throws, aborts or prints.  A textual description
+ * of the last failure on the calling thread is available from gi_last_error().
+ *
+ * Memory.  The library owns only host memory.  Every device buffer - graph inputs and
+ * outputs, the arena that holds intermediate tensors, the packed-weight blob - is allocated
+ * and freed by the caller; the library never allocates or frees device memory.  Device
+ * pointers passed in must be 256-byte aligned.
+ *
+ * Layout.  Activations live in a channel-sliced layout (PHWC4, Section 4 "Data Layout"):
+ * a [H,W,C] tensor is cut into S = ceil(C/4) slices of 4 channels, missing channels are
+ * zero.  For a batch of B images the B planes of one slice are adjacent and the slices
+ * follow one another: element (b,h,w,c) is at element index
+ *     ((c/4 * B + b) * plane + h*W + w) * 4 + c%4,      plane = H*W rounded up to even.
+ * The extra pixel of an odd plane must hold finite values (the library writes zeros or
+ * finite values there).  Caller-visible tensors can instead be plain NHWC, in which case
+ * the executable starts / ends with a layout conversion kernel (Section 3, "Running
+ * Inference").
+ */
+#ifndef GI_H_
+#define GI_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define GI_API __attribute__((visibility("default")))
+#else
+#define GI_API
+#endif
+
+typedef int32_t gi_status;
+typedef int32_t gi_tensor; /* tensor id within one graph, >= 0 */
+typedef struct gi_graph gi_graph;
+typedef struct gi_exec gi_exec;
+
+enum {
+  GI_OK = 0,
+  GI_E_INVALID = -1,     /* bad argument: null pointer, unknown id or kind, shape mismatch */
+  GI_E_UNSUPPORTED = -2, /* a well-formed request this library has no kernel for */
+  GI_E_NOMEM = -3,       /* host allocation failed */
+  GI_E_CUDA = -4,        /* a CUDA call failed; gi_last_error() holds the CUDA error string */
+  GI_E_STATE = -5,       /* call out of order (e.g. gi_run before gi_exec_bind) */
+  GI_E_ARENA = -6        /* arena / weight buffer too small or misaligned */
+};
+
+enum { GI_F16 = 1, GI_F32 = 2 };   /* storage type of activations (and of NHWC inputs/outputs) */
+enum { GI_NHWC = 0, GI_PHWC4 = 1 }; /* layout of a caller-visible tensor */
+
+enum {
+  GI_OP_CONV2D = 1,           /* full convolution, kernel 1x1 or 3x3 */
+  GI_OP_DEPTHWISE_CONV2D = 2, /* depthwise 3x3, depth multiplier 1 */
+  GI_OP_ADD = 3,              /* element-wise sum of two tensors of the same shape */
+  GI_OP_ACTIVATION = 4,       /* ReLU or ReLU6 */
+  GI_OP_GLOBAL_AVG_POOL = 5,  /* mean over H*W */
+  GI_OP_RESIZE_BILINEAR = 6   /* bilinear up/down-sampling */
+};
+
+enum { GI_ACT_NONE = 0, GI_ACT_RELU = 1, GI_ACT_RELU6 = 2 };
+
+/* Memory planners for intermediate tensors (Section 5, "Memory Manager for Intermediate Tensors"). */
+enum {
+  GI_PLAN_GREEDY_BY_SIZE = 0,        /* offsets into one buffer, largest tensor first, best-fit gap (default) */
+  GI_PLAN_GREEDY_SHARED_OBJECTS = 1, /* Algorithm 1 of the paper, objects laid out in creation order */
+  GI_PLAN_NAIVE = 2                  /* every tensor its own memory (the paper's baseline) */
+};
+
+/* Pointwise (1x1 convolution) kernel choice. */
+enum {
+  GI_PW_AUTO = 0,      /* tensor-core kernel for fp16 storage, SIMT kernel for fp32 storage */
+  GI_PW_SIMT = 1       /* force the plain CUDA-core kernel (validation) */
+};
+
+/*
+ * One operator (Section 3.1: the operators of the delegated sub-graph).
+ * Convolutions compute, with out-of-range input reading as zero,
+ *   out[b,oy,ox,co] = bias[co] + sum_{ky,kx,ci} in[b, oy*stride_h - pad_t + ky*dilation_h,
+ *                                                ox*stride_w - pad_l + kx*dilation_w, ci] * w[co,ky,kx,ci]
+ * (Section 4, "For a 2D Convolution"); depthwise is the same sum with co = ci.
+ * Output extent: (in + pad_before + pad_after - ((k-1)*dilation + 1)) / stride + 1.
+ *
+ * weights: host pointer, [cout][kh][kw][cin] for CONV2D, [1][kh][kw][c] for DEPTHWISE_CONV2D,
+ * of type weight_dtype (GI_F32 or GI_F16); bias: host pointer to cout floats or NULL.  Both
+ * are copied by gi_add_op; the caller may free them as soon as it returns.
+ * Unused fields must be zero.  inputs[1] is used by GI_OP_ADD only (else -1 or 0).
+ */
+typedef struct gi_op_desc {
+  int32_t kind;
+  gi_tensor inputs[2];
+  int32_t kh, kw;
+  int32_t stride_h, stride_w;
+  int32_t dilation_h, dilation_w;
+  int32_t pad_t, pad_l, pad_b, pad_r;
+  int32_t cout;          /* CONV2D only */
+  int32_t act;           /* ACTIVATION only: GI_ACT_RELU | GI_ACT_RELU6 */
+  int32_t out_h, out_w;  /* RESIZE_BILINEAR only */
+  int32_t align_corners; /* RESIZE_BILINEAR only: 1 -> src = o*(in-1)/(out-1), 0 -> src = o*in/out */
+  int32_t weight_dtype;
+  const void* weights;
+  const float* bias;
+} gi_op_desc;
+
+typedef struct gi_compile_options {
+  int32_t planner;   /* GI_PLAN_* */
+  int32_t fuse;      /* 1: fold element-wise ops into convolutions (default), 0: one kernel per op */
+  int32_t align;     /* arena offset / tensor size granularity in bytes, power of two >= 256; 0 -> 256 */
+  int32_t pointwise; /* GI_PW_* */
+} gi_compile_options;
+
+typedef struct gi_exec_info {
+  int32_t n_ops;           /* executed ops: layout conversions + fused ops = kernel launches per gi_run */
+  int32_t n_fused_ops;     /* fused ops only */
+  int32_t n_tensors;       /* tensors of the graph (ids 0 .. n_tensors-1) */
+  int32_t batch, storage;
+  uint64_t arena_bytes;    /* bytes gi_run needs in dev_arena under the chosen planner */
+  uint64_t naive_bytes;    /* sum of all intermediate tensor sizes */
+  uint64_t lower_bound_bytes; /* max over ops of bytes alive at that op */
+  uint64_t weight_bytes;   /* bytes gi_exec_bind needs in dev_weights */
+} gi_exec_info;
+
+typedef struct gi_tensor_info {
+  int32_t h, w, c;
+  int32_t alive;        /* 0 if fusion removed the tensor */
+  int32_t intermediate; /* 1 if it lives in the arena */
+  int32_t first_op, last_op; /* executed-op indices, inclusive; -1 if not alive */
+  uint64_t bytes;       /* physical size under the size formula */
+  uint64_t offset;      /* arena offset (intermediate tensors only) */
+} gi_tensor_info;
+
+typedef struct gi_op_info {
+  int32_t kind;         /* GI_OP_* of the leading op; GI_EXEC_PACK / GI_EXEC_UNPACK for layout conversions */
+  int32_t graph_op;     /* index of the leading op in gi_add_op order; -1 for conversions */
+  gi_tensor inputs[2];  /* tensors the leading op reads (-1 = unused / caller buffer) */
+  gi_tensor residual;   /* tensor added in the epilogue, or -1 */
+  gi_tensor output;     /* tensor written (-1 = caller buffer) */
+  int32_t act_pre;      /* activation applied before the residual add */
+  int32_t act_post;     /* activation applied after the residual add */
+  int32_t kernel;       /* GI_KERNEL_* that runs this op */
+  uint64_t bytes;       /* algorithmic bytes: inputs + residual + output once, weights once */
+  uint64_t flops;       /* algorithmic flops (2 per multiply-add) */
+} gi_op_info;
+
+enum { GI_EXEC_PACK = 100, GI_EXEC_UNPACK = 101 };
+enum {
+  GI_KERNEL_PACK = 1, GI_KERNEL_UNPACK = 2, GI_KERNEL_CONV_SIMT = 3, GI_KERNEL_POINTWISE_TC = 4,
+  GI_KERNEL_DEPTHWISE = 5, GI_KERNEL_ELTWISE = 6, GI_KERNEL_POOL = 7, GI_KERNEL_RESIZE = 8
+};
+
+/* ---- graph construction (Section 3.1, "Initialization": the sub-graph given to the GPU backend) ---- */
+
+/* Create an empty graph for `batch` images whose activations are stored as `storage`
+ * (GI_F16: fp16 storage with fp32 accumulation; GI_F32: fp32 everywhere, for validation).
+ * *out is owned by the caller: release with gi_graph_destroy. */
+GI_API gi_status gi_graph_create(gi_graph** out, int32_t batch, int32_t storage);
+
+/* Declare a graph input of logical shape [batch,H,W,C]; `layout` says how the caller's device
+ * buffer handed to gi_run is laid out (GI_NHWC: batch*H*W*C storage elements; GI_PHWC4: the
+ * layout above).  Inputs are numbered in declaration order. */
+GI_API gi_status gi_graph_input(gi_graph* g, int32_t H, int32_t W, int32_t C, int32_t layout, gi_tensor* out);
+
+/* Append an operator; its inputs must already exist, so insertion order is a topological
+ * order (Section 5 sorts topologically; here the order is given and verified).  *out
+ * receives the id of its single output tensor.  GI_E_UNSUPPORTED for kernels other than
+ * 1x1 / 3x3 (full) or 3x3 (depthwise), GI_E_INVALID for shape or id errors. */
+GI_API gi_status gi_add_op(gi_graph* g, const gi_op_desc* desc, gi_tensor* out);
+
+/* Mark a tensor as graph output, delivered to the caller's buffer in `layout`.  Outputs are
+ * numbered in the order of these calls.  A graph input cannot be an output. */
+GI_API gi_status gi_graph_output(gi_graph* g, gi_tensor t, int32_t layout);
+
+GI_API void gi_graph_destroy(gi_graph* g);
+
+/* ---- compile (Sections 3.2 and 5) ---- */
+
+/* Build an executable: verify the order, fuse, compute lifetimes, plan memory, pack weights,
+ * choose a kernel and launch shape per fused op.  Host work only; no CUDA call is made.
+ * `opt` may be NULL for defaults.  The graph stays valid and may be compiled again. */
+GI_API gi_status gi_compile(const gi_graph* g, const gi_compile_options* opt, gi_exec** out);
+
+GI_API gi_status gi_exec_query(const gi_exec* e, gi_exec_info* info);
+GI_API gi_status gi_exec_tensor(const gi_exec* e, gi_tensor t, gi_tensor_info* info);
+GI_API gi_status gi_exec_op(const gi_exec* e, int32_t index, gi_op_info* info);
+
+/* Copy the packed weights (info.weight_bytes) into the caller's device buffer, asynchronously
+ * on `stream` (a cudaStream_t, NULL for the default stream).  Must precede gi_run; the buffer
+ * must stay alive and unmodified as long as the executable is used.  The host staging copy is
+ * kept, so binding again (another buffer or device) is allowed. */
+GI_API gi_status gi_exec_bind(gi_exec* e, void* dev_weights, size_t weight_bytes, void* stream);
+
+/* Enqueue one inference on `stream` and return without synchronising (Section 3.2: the GPU
+ * executes the queued programs without synchronisation with the CPU).  dev_inputs[i] /
+ * dev_outputs[i] are device pointers for input / output i in their declared layouts;
+ * dev_arena holds the intermediates (>= info.arena_bytes).  Nothing is launched if an
+ * argument check fails (GI_E_INVALID, GI_E_ARENA, GI_E_STATE).  Two runs of one executable
+ * may overlap only if they use different arenas and outputs.  Results are deterministic:
+ * the same inputs give bit-identical outputs. */
+GI_API gi_status gi_run(gi_exec* e, const void* const* dev_inputs, void* const* dev_outputs, void* dev_arena,
+                 size_t arena_bytes, void* stream);
+
+GI_API void gi_exec_destroy(gi_exec* e);
+
+/* ---- helpers ---- */
+GI_API const char* gi_status_str(gi_status s);
+GI_API const char* gi_last_error(void); /* thread-local, valid until the next failing call on this thread */
+
+/* Physical bytes of a [batch,H,W,C] tensor in the library's PHWC4 layout, rounded up to
+ * `align` (Section 4; C = 5 costs as much as C = 8). */
+GI_API uint64_t gi_tensor_bytes(int32_t batch, int32_t H, int32_t W, int32_t C, int32_t storage, int32_t align);
+
+/* Round n floats to fp16 bit patterns (round to nearest even) exactly as weight packing does. */
+GI_API void gi_f32_to_f16(const float* src, uint16_t* dst, size_t n);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GI_H_ */

@@ -1,0 +1,221 @@
+// Lowering: choose a kernel per executed op, pack its weights into the kernel's operand
+// layout (fp16 storage: weights rounded to fp16 once, biases stay fp32) and record the
+// launch geometry.  Host work only.
+#include <cstring>
+
+#include "gi_internal.h"
+#include "kernels.h"
+
+namespace gi {
+
+static float as_storage(float v, int storage) {
+  if (storage == GI_F32) return v;
+  // value the weight has after being stored as fp16
+  const uint16_t h = f32_to_f16_rne(v);
+  const uint32_t s = (h & 0x8000u) << 16, e = (h >> 10) & 0x1fu, m = h & 0x3ffu;
+  uint32_t u;
+  float r;
+  if (e == 0) {
+    r = static_cast<float>(m) * (1.0f / 16777216.0f);
+    std::memcpy(&u, &r, 4);
+  } else if (e == 31) {
+    u = 0x7f800000u | (m << 13);
+  } else {
+    u = ((e + 112u) << 23) | (m << 13);
+  }
+  u |= s;
+  std::memcpy(&r, &u, 4);
+  return r;
+}
+
+static uint64_t blob_reserve(std::vector<uint8_t>* blob, uint64_t bytes) {
+  const uint64_t off = round_up_u64(blob->size(), 256);
+  blob->resize(off + bytes, 0);
+  return off;
+}
+
+static Loc loc_of(const gi_exec* e, int t) {
+  Loc l;
+  if (t < 0) return l;
+  const TensorDesc& d = e->tensors[t];
+  if (d.input_index >= 0 && d.input_layout == GI_PHWC4) {
+    l.where = W_INPUT;
+    l.index = d.input_index;
+  } else if (d.output_index >= 0 && d.output_layout == GI_PHWC4) {
+    l.where = W_OUTPUT;
+    l.index = d.output_index;
+  } else {
+    l.where = W_ARENA;
+    l.offset = e->plan[t].offset;
+  }
+  return l;
+}
+
+// Weights of the CUDA-core convolution kernel: float W[group][tap][in_slice][OS*4 co][4 ci],
+// a group being OS consecutive output slices; entries beyond Cin / Cout are zero.
+static void pack_conv_simt(const OpNode& op, int cin, int storage, int os, std::vector<uint8_t>* blob, LaunchRec* r) {
+  const int taps = op.d.kh * op.d.kw, sin = slices(cin), sout = slices(op.d.cout);
+  const int groups = (sout + os - 1) / os, jn = os * 4;
+  const uint64_t nw = static_cast<uint64_t>(groups) * taps * sin * jn * 4;
+  const uint64_t woff = blob_reserve(blob, nw * sizeof(float));
+  const uint64_t boff = blob_reserve(blob, static_cast<uint64_t>(groups) * jn * sizeof(float));
+  float* w = reinterpret_cast<float*>(blob->data() + woff);
+  float* b = reinterpret_cast<float*>(blob->data() + boff);
+  for (int g = 0; g < groups; ++g)
+    for (int j = 0; j < jn; ++j) {
+      const int co = g * jn + j;
+      if (co >= op.d.cout) continue;
+      b[g * jn + j] = op.bias[co];
+      for (int tap = 0; tap < taps; ++tap)
+        for (int ci = 0; ci < cin; ++ci) {
+          const float v = op.weights[(static_cast<size_t>(co) * taps + tap) * cin + ci];
+          w[(((static_cast<size_t>(g) * taps + tap) * sin + ci / 4) * jn + j) * 4 + ci % 4] = as_storage(v, storage);
+        }
+    }
+  r->wts = Loc{W_WEIGHTS, 0, woff};
+  r->bias = Loc{W_WEIGHTS, 0, boff};
+  r->wts_bytes = nw * sizeof(float);
+}
+
+// Depthwise: float W[tap][C4], bias[C4].
+static void pack_depthwise(const OpNode& op, int c, int storage, std::vector<uint8_t>* blob, LaunchRec* r) {
+  const int taps = op.d.kh * op.d.kw, c4 = slices(c) * 4;
+  const uint64_t woff = blob_reserve(blob, static_cast<uint64_t>(taps) * c4 * sizeof(float));
+  const uint64_t boff = blob_reserve(blob, static_cast<uint64_t>(c4) * sizeof(float));
+  float* w = reinterpret_cast<float*>(blob->data() + woff);
+  float* b = reinterpret_cast<float*>(blob->data() + boff);
+  for (int ch = 0; ch < c; ++ch) {
+    b[ch] = op.bias[ch];
+    for (int tap = 0; tap < taps; ++tap) w[tap * c4 + ch] = as_storage(op.weights[static_cast<size_t>(tap) * c + ch], storage);
+  }
+  r->wts = Loc{W_WEIGHTS, 0, woff};
+  r->bias = Loc{W_WEIGHTS, 0, boff};
+  r->wts_bytes = static_cast<uint64_t>(taps) * c4 * sizeof(float);
+}
+
+gi_status lower(const gi_graph& g, gi_exec* e) {
+  const int eb = elem_bytes(e->storage);
+  const uint64_t B = static_cast<uint64_t>(e->batch);
+  for (size_t i = 0; i < e->ops.size(); ++i) {
+    const FusedOp& f = e->ops[i];
+    LaunchRec r;
+    gi_op_info info{};
+    info.kind = f.kind;
+    info.graph_op = f.graph_op;
+    info.inputs[0] = f.in0;
+    info.inputs[1] = f.in1;
+    info.residual = f.residual;
+    info.output = f.out;
+    info.act_pre = f.act_pre;
+    info.act_post = f.act_post;
+    r.B = e->batch;
+    r.ep.act_pre = f.act_pre;
+    r.ep.has_res = f.residual >= 0;
+    r.ep.act_post = f.act_post;
+    const TensorDesc* din = f.in0 >= 0 ? &e->tensors[f.in0] : nullptr;
+    const TensorDesc* dout = f.out >= 0 ? &e->tensors[f.out] : nullptr;
+    if (din) {
+      r.H = din->h;
+      r.W = din->w;
+      r.C = din->c;
+    }
+    if (dout) {
+      r.Ho = dout->h;
+      r.Wo = dout->w;
+      r.Co = dout->c;
+    }
+    r.in0 = loc_of(e, f.in0);
+    r.in1 = loc_of(e, f.in1);
+    r.res = loc_of(e, f.residual);
+    r.out = loc_of(e, f.out);
+    const uint64_t in_px = din ? B * din->h * din->w : 0, out_px = dout ? B * dout->h * dout->w : 0;
+    const uint64_t in_c4 = din ? slices(din->c) * 4 : 0, out_c4 = dout ? slices(dout->c) * 4 : 0;
+    switch (f.kind) {
+      case GI_EXEC_PACK: {
+        r.kernel = GI_KERNEL_PACK;
+        r.in0 = Loc{W_INPUT, f.io_index, 0};
+        r.H = dout->h;
+        r.W = dout->w;
+        r.C = dout->c;
+        info.bytes = out_px * dout->c * eb + out_px * out_c4 * eb;
+        break;
+      }
+      case GI_EXEC_UNPACK: {
+        r.kernel = GI_KERNEL_UNPACK;
+        r.out = Loc{W_OUTPUT, f.io_index, 0};
+        info.bytes = in_px * in_c4 * eb + in_px * din->c * eb;
+        break;
+      }
+      case GI_OP_CONV2D:
+      case GI_OP_DEPTHWISE_CONV2D: {
+        const OpNode& op = g.ops[f.graph_op];
+        r.kh = op.d.kh;
+        r.kw = op.d.kw;
+        r.sh = op.d.stride_h;
+        r.sw = op.d.stride_w;
+        r.dh = op.d.dilation_h;
+        r.dw = op.d.dilation_w;
+        r.pt = op.d.pad_t;
+        r.pl = op.d.pad_l;
+        const uint64_t taps = static_cast<uint64_t>(op.d.kh) * op.d.kw;
+        info.bytes = (in_px * in_c4 + out_px * out_c4 * (r.ep.has_res ? 2 : 1)) * eb;
+        if (f.kind == GI_OP_DEPTHWISE_CONV2D) {
+          r.kernel = GI_KERNEL_DEPTHWISE;
+          pack_depthwise(op, din->c, e->storage, &e->weight_blob, &r);
+          info.bytes += taps * din->c * eb;
+          info.flops = 2 * taps * out_px * din->c;
+        } else {
+          const bool pointwise = op.d.kh == 1 && op.d.stride_h == 1 && op.d.stride_w == 1 && op.d.pad_t == 0 &&
+                                 op.d.pad_l == 0 && op.d.pad_b == 0 && op.d.pad_r == 0;
+          if (pointwise && e->storage == GI_F16 && e->opt.pointwise == GI_PW_AUTO &&
+              pointwise_tc_supported(din->c, op.d.cout)) {
+            r.kernel = GI_KERNEL_POINTWISE_TC;
+            pointwise_tc_pack(op.weights.data(), op.bias.data(), din->c, op.d.cout, &e->weight_blob, &r);
+          } else {
+            r.kernel = GI_KERNEL_CONV_SIMT;
+            const int sout = slices(op.d.cout);
+            const int os = sout >= 8 ? 8 : sout >= 4 ? 4 : sout >= 2 ? 2 : 1;
+            r.tc_nt = os;
+            pack_conv_simt(op, din->c, e->storage, os, &e->weight_blob, &r);
+          }
+          info.bytes += taps * din->c * op.d.cout * eb;
+          info.flops = 2 * taps * out_px * din->c * op.d.cout;
+        }
+        break;
+      }
+      case GI_OP_ADD:
+      case GI_OP_ACTIVATION: {
+        r.kernel = GI_KERNEL_ELTWISE;
+        const OpNode& op = g.ops[f.graph_op];
+        if (f.kind == GI_OP_ACTIVATION) r.ep.act_pre = op.d.act;
+        info.act_pre = r.ep.act_pre;
+        r.ep.has_res = f.kind == GI_OP_ADD;
+        info.bytes = (in_px * in_c4 * (f.kind == GI_OP_ADD ? 2 : 1) + out_px * out_c4) * eb;
+        info.flops = out_px * dout->c;
+        break;
+      }
+      case GI_OP_GLOBAL_AVG_POOL:
+        r.kernel = GI_KERNEL_POOL;
+        info.bytes = (in_px * in_c4 + out_px * out_c4) * eb;
+        info.flops = in_px * din->c;
+        break;
+      case GI_OP_RESIZE_BILINEAR: {
+        r.kernel = GI_KERNEL_RESIZE;
+        r.align_corners = g.ops[f.graph_op].d.align_corners;
+        info.bytes = (in_px * in_c4 + out_px * out_c4) * eb;
+        info.flops = 8 * out_px * dout->c;
+        break;
+      }
+      default:
+        return fail(GI_E_INVALID, "gi_compile: unknown executed-op kind");
+    }
+    info.kernel = r.kernel;
+    e->launches.push_back(r);
+    e->op_info.push_back(info);
+  }
+  // keep the blob a whole number of 256-byte units so any tail read stays inside it
+  e->weight_blob.resize(round_up_u64(e->weight_blob.size() + 1, 256), 0);
+  return GI_OK;
+}
+
+}  // namespace gi

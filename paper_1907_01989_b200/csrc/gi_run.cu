@@ -1,0 +1,96 @@
+// Run half of the C ABI: weight upload and the launch loop.  gi_run only enqueues work on
+// the caller's stream; it never synchronises and never allocates device memory.
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <string>
+
+#include "gi_internal.h"
+#include "kernels.h"
+
+namespace gi {
+
+void release_run_state(gi_exec* e) {
+  if (e->tc_state) {
+    pointwise_tc_release(e->tc_state);
+    e->tc_state = nullptr;
+  }
+}
+
+static bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
+
+}  // namespace gi
+
+using namespace gi;
+
+extern "C" {
+
+gi_status gi_exec_bind(gi_exec* e, void* dev_weights, size_t weight_bytes, void* stream) {
+  if (!e || !dev_weights) return fail(GI_E_INVALID, "gi_exec_bind: null argument");
+  if (!aligned256(dev_weights)) return fail(GI_E_ARENA, "gi_exec_bind: dev_weights must be 256-byte aligned");
+  if (weight_bytes < e->weight_blob.size()) return fail(GI_E_ARENA, "gi_exec_bind: weight buffer too small");
+  const cudaError_t err = cudaMemcpyAsync(dev_weights, e->weight_blob.data(), e->weight_blob.size(), cudaMemcpyHostToDevice,
+                                          static_cast<cudaStream_t>(stream));
+  if (err != cudaSuccess) return fail(GI_E_CUDA, std::string("gi_exec_bind: ") + cudaGetErrorString(err));
+  if (e->dev_weights != dev_weights) release_run_state(e);  // cached tensor maps point at the old buffer
+  e->dev_weights = dev_weights;
+  return GI_OK;
+}
+
+gi_status gi_run(gi_exec* e, const void* const* dev_inputs, void* const* dev_outputs, void* dev_arena, size_t arena_bytes,
+                 void* stream) {
+  if (!e || !dev_inputs || !dev_outputs) return fail(GI_E_INVALID, "gi_run: null argument");
+  if (!e->dev_weights) return fail(GI_E_STATE, "gi_run: gi_exec_bind has not been called");
+  if (e->arena_bytes > 0) {
+    if (!dev_arena) return fail(GI_E_ARENA, "gi_run: null arena");
+    if (!aligned256(dev_arena)) return fail(GI_E_ARENA, "gi_run: arena must be 256-byte aligned");
+    if (arena_bytes < e->arena_bytes) return fail(GI_E_ARENA, "gi_run: arena smaller than gi_exec_info.arena_bytes");
+  }
+  for (int i = 0; i < e->n_inputs; ++i)
+    if (!dev_inputs[i] || !aligned256(dev_inputs[i])) return fail(GI_E_INVALID, "gi_run: input pointer null or not 256-byte aligned");
+  for (int i = 0; i < e->n_outputs; ++i)
+    if (!dev_outputs[i] || !aligned256(dev_outputs[i])) return fail(GI_E_INVALID, "gi_run: output pointer null or not 256-byte aligned");
+
+  auto resolve = [&](const Loc& l) -> void* {
+    switch (l.where) {
+      case W_ARENA: return static_cast<char*>(dev_arena) + l.offset;
+      case W_INPUT: return const_cast<void*>(dev_inputs[l.index]);
+      case W_OUTPUT: return dev_outputs[l.index];
+      case W_WEIGHTS: return static_cast<char*>(e->dev_weights) + l.offset;
+      default: return nullptr;
+    }
+  };
+
+  for (size_t i = 0; i < e->launches.size(); ++i) {
+    const LaunchRec& r = e->launches[i];
+    Ptrs p;
+    p.in0 = resolve(r.in0);
+    p.in1 = resolve(r.in1);
+    p.res = resolve(r.res);
+    p.out = resolve(r.out);
+    p.wts = resolve(r.wts);
+    p.bias = resolve(r.bias);
+    int err = 0;
+    switch (r.kernel) {
+      case GI_KERNEL_PACK: err = launch_pack(r, p, e->storage, stream); break;
+      case GI_KERNEL_UNPACK: err = launch_unpack(r, p, e->storage, stream); break;
+      case GI_KERNEL_CONV_SIMT: err = launch_conv_simt(r, p, e->storage, stream); break;
+      case GI_KERNEL_POINTWISE_TC: err = launch_pointwise_tc(r, p, &e->tc_state, static_cast<int>(i), stream); break;
+      case GI_KERNEL_DEPTHWISE: err = launch_depthwise(r, p, e->storage, stream); break;
+      case GI_KERNEL_ELTWISE:
+        if (r.ep.has_res && !p.in1) p.in1 = p.res;
+        err = launch_eltwise(r, p, e->storage, stream);
+        break;
+      case GI_KERNEL_POOL: err = launch_pool(r, p, e->storage, stream); break;
+      case GI_KERNEL_RESIZE: err = launch_resize(r, p, e->storage, stream); break;
+      default: return fail(GI_E_INVALID, "gi_run: corrupt launch table");
+    }
+    if (err != 0) {
+      return fail(GI_E_CUDA, "gi_run: launch " + std::to_string(i) + " failed: " +
+                                 cudaGetErrorString(static_cast<cudaError_t>(err)));
+    }
+  }
+  return GI_OK;
+}
+
+}  // extern "C"

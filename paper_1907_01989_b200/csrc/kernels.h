@@ -1,0 +1,36 @@
+// Launchers of the CUDA kernels.  Each takes resolved device pointers, enqueues on `stream`
+// and returns the cudaError_t of the launch (as int, so host-only files need no CUDA headers).
+#pragma once
+
+#include <cstdint>
+#include <vector>
+
+#include "gi_internal.h"
+
+namespace gi {
+
+struct Ptrs {
+  const void* in0 = nullptr;
+  const void* in1 = nullptr;
+  const void* res = nullptr;
+  void* out = nullptr;
+  const void* wts = nullptr;
+  const void* bias = nullptr;
+};
+
+int launch_pack(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
+int launch_unpack(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
+int launch_conv_simt(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
+int launch_depthwise(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
+int launch_eltwise(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
+int launch_pool(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
+int launch_resize(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
+
+// Tensor-core pointwise convolution (fp16 storage only).
+bool pointwise_tc_supported(int cin, int cout);
+void pointwise_tc_pack(const float* w, const float* bias, int cin, int cout, std::vector<uint8_t>* blob, LaunchRec* r);
+// tensor maps depend on device addresses; `state` caches them per executable
+int launch_pointwise_tc(const LaunchRec& r, const Ptrs& p, void** state, int launch_index, void* stream);
+void pointwise_tc_release(void* state);
+
+}  // namespace gi

@@ -1,0 +1,413 @@
+// CUDA-core kernels: layout conversion, depthwise 3x3, direct convolution, element-wise,
+// global average pool, bilinear resize.  All work on the channel-sliced layout
+//   element (b,h,w,c) -> ((c/4 * B + b) * P + h*W + w) * 4 + c%4,   P = H*W rounded up to even,
+// and move one pixel-slice (4 channels: 8 bytes fp16, 16 bytes fp32) per vector access, so a
+// warp touches 32 consecutive pixels of one plane = one contiguous 256 / 512-byte run.
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include "kernels.h"
+
+namespace gi {
+namespace {
+
+template <typename T>
+struct Px;  // one pixel-slice in storage type T
+
+template <>
+struct Px<__half> {
+  static __device__ __forceinline__ float4 load(const __half* p) {
+    const uint2 u = *reinterpret_cast<const uint2*>(p);
+    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&u.x));
+    const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&u.y));
+    return make_float4(a.x, a.y, b.x, b.y);
+  }
+  static __device__ __forceinline__ void store(__half* p, float4 v) {
+    const __half2 a = __floats2half2_rn(v.x, v.y), b = __floats2half2_rn(v.z, v.w);
+    uint2 u;
+    u.x = *reinterpret_cast<const unsigned*>(&a);
+    u.y = *reinterpret_cast<const unsigned*>(&b);
+    *reinterpret_cast<uint2*>(p) = u;
+  }
+  static __device__ __forceinline__ float get(const __half* p) { return __half2float(*p); }
+  static __device__ __forceinline__ void put(__half* p, float v) { *p = __float2half_rn(v); }
+};
+
+template <>
+struct Px<float> {
+  static __device__ __forceinline__ float4 load(const float* p) { return *reinterpret_cast<const float4*>(p); }
+  static __device__ __forceinline__ void store(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+  static __device__ __forceinline__ float get(const float* p) { return *p; }
+  static __device__ __forceinline__ void put(float* p, float v) { *p = v; }
+};
+
+__device__ __forceinline__ float act1(float v, int kind) {
+  if (kind == GI_ACT_RELU) return fmaxf(v, 0.0f);
+  if (kind == GI_ACT_RELU6) return fminf(fmaxf(v, 0.0f), 6.0f);
+  return v;
+}
+__device__ __forceinline__ float4 act4(float4 v, int kind) {
+  return make_float4(act1(v.x, kind), act1(v.y, kind), act1(v.z, kind), act1(v.w, kind));
+}
+
+// bias is already in v: activation, residual add, activation, in graph order
+template <typename T>
+__device__ __forceinline__ float4 epilogue(float4 v, const Epilogue& ep, const T* res, size_t idx) {
+  v = act4(v, ep.act_pre);
+  if (ep.has_res) {
+    const float4 r = Px<T>::load(res + idx);
+    v.x += r.x;
+    v.y += r.y;
+    v.z += r.z;
+    v.w += r.w;
+  }
+  return act4(v, ep.act_post);
+}
+
+// ------------------------------------------------------------------ layout conversion
+template <typename T>
+__global__ void pack_kernel(const T* __restrict__ nhwc, T* __restrict__ out, int B, int HW, int C, int P, int S) {
+  const size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x;
+  const size_t total = static_cast<size_t>(S) * B * P;
+  if (idx >= total) return;
+  const int pix = static_cast<int>(idx % P);
+  const int b = static_cast<int>((idx / P) % B);
+  const int s = static_cast<int>(idx / (static_cast<size_t>(P) * B));
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (pix < HW) {
+    const T* src = nhwc + (static_cast<size_t>(b) * HW + pix) * C + s * 4;
+    const int n = min(4, C - s * 4);
+    float t[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int j = 0; j < n; ++j) t[j] = Px<T>::get(src + j);
+    v = make_float4(t[0], t[1], t[2], t[3]);
+  }
+  Px<T>::store(out + idx * 4, v);
+}
+
+template <typename T>
+__global__ void unpack_kernel(const T* __restrict__ in, T* __restrict__ nhwc, int B, int HW, int C, int P, int S) {
+  const size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x;
+  const size_t total = static_cast<size_t>(B) * HW * S;
+  if (idx >= total) return;
+  const int s = static_cast<int>(idx % S);
+  const int pix = static_cast<int>((idx / S) % HW);
+  const int b = static_cast<int>(idx / (static_cast<size_t>(S) * HW));
+  const float4 v = Px<T>::load(in + ((static_cast<size_t>(s) * B + b) * P + pix) * 4);
+  const float t[4] = {v.x, v.y, v.z, v.w};
+  T* dst = nhwc + (static_cast<size_t>(b) * HW + pix) * C + s * 4;
+  const int n = min(4, C - s * 4);
+  for (int j = 0; j < n; ++j) Px<T>::put(dst + j, t[j]);
+}
+
+// ------------------------------------------------------------------ direct convolution
+struct ConvGeom {
+  int B, H, W, Sin, Pin, Ho, Wo, Sout, Pout;
+  int kh, kw, sh, sw, dh, dw, pt, pl;
+};
+
+// One thread = one output pixel x OS output slices.  Weights W[group][tap][in_slice][OS*4][4]
+// are read with warp-uniform addresses (one broadcast L1 transaction per float4).
+template <typename T, int OS>
+__global__ void __launch_bounds__(128) conv_simt_kernel(const T* __restrict__ in, const float4* __restrict__ w,
+                                                        const float* __restrict__ bias, const T* __restrict__ res,
+                                                        T* __restrict__ out, ConvGeom g, Epilogue ep) {
+  const int pix = blockIdx.x * 128 + threadIdx.x;
+  const int grp = blockIdx.y, b = blockIdx.z;
+  if (pix >= g.Pout) return;
+  constexpr int JN = OS * 4;
+  float acc[JN];
+#pragma unroll
+  for (int j = 0; j < JN; ++j) acc[j] = 0.f;
+  const bool real = pix < g.Ho * g.Wo;
+  if (real) {
+    const int oy = pix / g.Wo, ox = pix - oy * g.Wo;
+    const float4* wg = w + static_cast<size_t>(grp) * g.kh * g.kw * g.Sin * JN;
+    for (int ky = 0; ky < g.kh; ++ky) {
+      const int iy = oy * g.sh - g.pt + ky * g.dh;
+      if (iy < 0 || iy >= g.H) continue;
+      for (int kx = 0; kx < g.kw; ++kx) {
+        const int ix = ox * g.sw - g.pl + kx * g.dw;
+        if (ix < 0 || ix >= g.W) continue;
+        const float4* wt = wg + static_cast<size_t>(ky * g.kw + kx) * g.Sin * JN;
+        const T* ip = in + (static_cast<size_t>(b) * g.Pin + iy * g.W + ix) * 4;
+        for (int s = 0; s < g.Sin; ++s) {
+          const float4 x = Px<T>::load(ip + static_cast<size_t>(s) * g.B * g.Pin * 4);
+          const float4* ws = wt + s * JN;
+#pragma unroll
+          for (int j = 0; j < JN; ++j) {
+            const float4 wv = __ldg(ws + j);
+            acc[j] = fmaf(x.x, wv.x, acc[j]);
+            acc[j] = fmaf(x.y, wv.y, acc[j]);
+            acc[j] = fmaf(x.z, wv.z, acc[j]);
+            acc[j] = fmaf(x.w, wv.w, acc[j]);
+          }
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 0; o < OS; ++o) {
+    const int so = grp * OS + o;
+    if (so >= g.Sout) break;
+    const size_t idx = ((static_cast<size_t>(so) * g.B + b) * g.Pout + pix) * 4;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (real) {
+      const float4 bv = *reinterpret_cast<const float4*>(bias + (grp * OS + o) * 4);
+      v = make_float4(acc[o * 4] + bv.x, acc[o * 4 + 1] + bv.y, acc[o * 4 + 2] + bv.z, acc[o * 4 + 3] + bv.w);
+      v = epilogue<T>(v, ep, res, idx);
+    }
+    Px<T>::store(out + idx, v);
+  }
+}
+
+// ------------------------------------------------------------------ depthwise 3x3
+template <typename T>
+__global__ void __launch_bounds__(128) depthwise_kernel(const T* __restrict__ in, const float* __restrict__ w,
+                                                        const float* __restrict__ bias, const T* __restrict__ res,
+                                                        T* __restrict__ out, ConvGeom g, Epilogue ep) {
+  const int pix = blockIdx.x * 128 + threadIdx.x;
+  const int s = blockIdx.y, b = blockIdx.z;
+  if (pix >= g.Pout) return;
+  const size_t idx = ((static_cast<size_t>(s) * g.B + b) * g.Pout + pix) * 4;
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (pix < g.Ho * g.Wo) {
+    const int oy = pix / g.Wo, ox = pix - oy * g.Wo;
+    const int C4 = g.Sin * 4;
+    v = *reinterpret_cast<const float4*>(bias + s * 4);
+    const T* plane = in + (static_cast<size_t>(s) * g.B + b) * g.Pin * 4;
+#pragma unroll
+    for (int ky = 0; ky < 3; ++ky) {
+      const int iy = oy * g.sh - g.pt + ky * g.dh;
+      if (iy < 0 || iy >= g.H) continue;
+#pragma unroll
+      for (int kx = 0; kx < 3; ++kx) {
+        const int ix = ox * g.sw - g.pl + kx * g.dw;
+        if (ix < 0 || ix >= g.W) continue;
+        const float4 x = Px<T>::load(plane + (static_cast<size_t>(iy) * g.W + ix) * 4);
+        const float4 wv = __ldg(reinterpret_cast<const float4*>(w + (ky * 3 + kx) * C4 + s * 4));
+        v.x = fmaf(x.x, wv.x, v.x);
+        v.y = fmaf(x.y, wv.y, v.y);
+        v.z = fmaf(x.z, wv.z, v.z);
+        v.w = fmaf(x.w, wv.w, v.w);
+      }
+    }
+    v = epilogue<T>(v, ep, res, idx);
+  }
+  Px<T>::store(out + idx, v);
+}
+
+// ------------------------------------------------------------------ element-wise
+template <typename T>
+__global__ void eltwise_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restrict__ out, size_t n_px,
+                               Epilogue ep) {
+  const size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x;
+  if (i >= n_px) return;
+  const float4 v = epilogue<T>(Px<T>::load(a + i * 4), ep, b, i * 4);
+  Px<T>::store(out + i * 4, v);
+}
+
+// ------------------------------------------------------------------ global average pool
+// one warp per (slice, image): lanes stride over the pixels, shuffle reduction in a fixed order
+template <typename T>
+__global__ void pool_kernel(const T* __restrict__ in, T* __restrict__ out, int planes, int HW, int Pin, int Pout) {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, lane = threadIdx.x & 31;
+  if (warp >= planes) return;
+  const T* plane = in + static_cast<size_t>(warp) * Pin * 4;
+  float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int p = lane; p < HW; p += 32) {
+    const float4 x = Px<T>::load(plane + static_cast<size_t>(p) * 4);
+    s.x += x.x;
+    s.y += x.y;
+    s.z += x.z;
+    s.w += x.w;
+  }
+  for (int d = 16; d > 0; d >>= 1) {
+    s.x += __shfl_down_sync(0xffffffffu, s.x, d);
+    s.y += __shfl_down_sync(0xffffffffu, s.y, d);
+    s.z += __shfl_down_sync(0xffffffffu, s.z, d);
+    s.w += __shfl_down_sync(0xffffffffu, s.w, d);
+  }
+  if (lane < Pout) {
+    const float inv = 1.0f / static_cast<float>(HW);
+    const float4 v = lane == 0 ? make_float4(s.x * inv, s.y * inv, s.z * inv, s.w * inv) : make_float4(0.f, 0.f, 0.f, 0.f);
+    Px<T>::store(out + (static_cast<size_t>(warp) * Pout + lane) * 4, v);
+  }
+}
+
+// ------------------------------------------------------------------ bilinear resize
+// source coordinate as an exact fraction num/den so that floor() never depends on rounding
+template <typename T>
+__global__ void __launch_bounds__(128) resize_kernel(const T* __restrict__ in, T* __restrict__ out, int B, int H, int W,
+                                                     int Pin, int OH, int OW, int Pout, int ny, int dy, int nx, int dx) {
+  const int pix = blockIdx.x * 128 + threadIdx.x;
+  const int s = blockIdx.y, b = blockIdx.z;
+  if (pix >= Pout) return;
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (pix < OH * OW) {
+    const int oy = pix / OW, ox = pix - oy * OW;
+    const long long py = static_cast<long long>(oy) * ny, qx = static_cast<long long>(ox) * nx;
+    int y0 = static_cast<int>(py / dy), x0 = static_cast<int>(qx / dx);
+    float wy = static_cast<float>(py - static_cast<long long>(y0) * dy) / static_cast<float>(dy);
+    float wx = static_cast<float>(qx - static_cast<long long>(x0) * dx) / static_cast<float>(dx);
+    if (y0 > H - 1) { y0 = H - 1; wy = 0.f; }
+    if (x0 > W - 1) { x0 = W - 1; wx = 0.f; }
+    const int y1 = min(y0 + 1, H - 1), x1 = min(x0 + 1, W - 1);
+    const T* plane = in + (static_cast<size_t>(s) * B + b) * Pin * 4;
+    const float4 a = Px<T>::load(plane + (static_cast<size_t>(y0) * W + x0) * 4);
+    const float4 c = Px<T>::load(plane + (static_cast<size_t>(y0) * W + x1) * 4);
+    const float4 d = Px<T>::load(plane + (static_cast<size_t>(y1) * W + x0) * 4);
+    const float4 e = Px<T>::load(plane + (static_cast<size_t>(y1) * W + x1) * 4);
+    auto lerp2 = [&](float p00, float p01, float p10, float p11) {
+      const float top = fmaf(p01 - p00, wx, p00), bot = fmaf(p11 - p10, wx, p10);
+      return fmaf(bot - top, wy, top);
+    };
+    v = make_float4(lerp2(a.x, c.x, d.x, e.x), lerp2(a.y, c.y, d.y, e.y), lerp2(a.z, c.z, d.z, e.z),
+                    lerp2(a.w, c.w, d.w, e.w));
+  }
+  Px<T>::store(out + ((static_cast<size_t>(s) * B + b) * Pout + pix) * 4, v);
+}
+
+ConvGeom geom(const LaunchRec& r) {
+  ConvGeom g;
+  g.B = r.B;
+  g.H = r.H;
+  g.W = r.W;
+  g.Sin = slices(r.C);
+  g.Pin = plane_pixels(r.H, r.W);
+  g.Ho = r.Ho;
+  g.Wo = r.Wo;
+  g.Sout = slices(r.Co);
+  g.Pout = plane_pixels(r.Ho, r.Wo);
+  g.kh = r.kh;
+  g.kw = r.kw;
+  g.sh = r.sh;
+  g.sw = r.sw;
+  g.dh = r.dh;
+  g.dw = r.dw;
+  g.pt = r.pt;
+  g.pl = r.pl;
+  return g;
+}
+
+inline unsigned blocks_for(size_t n, unsigned per) { return static_cast<unsigned>((n + per - 1) / per); }
+
+}  // namespace
+
+#define GI_BY_STORAGE(call_h, call_f) \
+  do {                                \
+    if (storage == GI_F16) {          \
+      call_h;                         \
+    } else {                          \
+      call_f;                         \
+    }                                 \
+  } while (0)
+
+int launch_pack(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int S = slices(r.C), P = plane_pixels(r.H, r.W), HW = r.H * r.W;
+  const size_t total = static_cast<size_t>(S) * r.B * P;
+  GI_BY_STORAGE((pack_kernel<__half><<<blocks_for(total, 256), 256, 0, st>>>(static_cast<const __half*>(p.in0),
+                                                                             static_cast<__half*>(p.out), r.B, HW, r.C, P, S)),
+                (pack_kernel<float><<<blocks_for(total, 256), 256, 0, st>>>(static_cast<const float*>(p.in0),
+                                                                            static_cast<float*>(p.out), r.B, HW, r.C, P, S)));
+  return static_cast<int>(cudaGetLastError());
+}
+
+int launch_unpack(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int S = slices(r.C), P = plane_pixels(r.H, r.W), HW = r.H * r.W;
+  const size_t total = static_cast<size_t>(S) * r.B * HW;
+  GI_BY_STORAGE((unpack_kernel<__half><<<blocks_for(total, 256), 256, 0, st>>>(static_cast<const __half*>(p.in0),
+                                                                               static_cast<__half*>(p.out), r.B, HW, r.C, P, S)),
+                (unpack_kernel<float><<<blocks_for(total, 256), 256, 0, st>>>(static_cast<const float*>(p.in0),
+                                                                              static_cast<float*>(p.out), r.B, HW, r.C, P, S)));
+  return static_cast<int>(cudaGetLastError());
+}
+
+template <typename T>
+static void conv_dispatch(const LaunchRec& r, const Ptrs& p, cudaStream_t st) {
+  const ConvGeom g = geom(r);
+  const int os = r.tc_nt;
+  const dim3 grid(blocks_for(g.Pout, 128), (g.Sout + os - 1) / os, r.B);
+  const T* in = static_cast<const T*>(p.in0);
+  const float4* w = static_cast<const float4*>(p.wts);
+  const float* b = static_cast<const float*>(p.bias);
+  const T* res = static_cast<const T*>(p.res);
+  T* out = static_cast<T*>(p.out);
+  switch (os) {
+    case 8: conv_simt_kernel<T, 8><<<grid, 128, 0, st>>>(in, w, b, res, out, g, r.ep); break;
+    case 4: conv_simt_kernel<T, 4><<<grid, 128, 0, st>>>(in, w, b, res, out, g, r.ep); break;
+    case 2: conv_simt_kernel<T, 2><<<grid, 128, 0, st>>>(in, w, b, res, out, g, r.ep); break;
+    default: conv_simt_kernel<T, 1><<<grid, 128, 0, st>>>(in, w, b, res, out, g, r.ep); break;
+  }
+}
+
+int launch_conv_simt(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (r.B > 65535) return static_cast<int>(cudaErrorInvalidConfiguration);
+  GI_BY_STORAGE(conv_dispatch<__half>(r, p, st), conv_dispatch<float>(r, p, st));
+  return static_cast<int>(cudaGetLastError());
+}
+
+int launch_depthwise(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (r.B > 65535) return static_cast<int>(cudaErrorInvalidConfiguration);
+  const ConvGeom g = geom(r);
+  const dim3 grid(blocks_for(g.Pout, 128), g.Sout, r.B);
+  GI_BY_STORAGE((depthwise_kernel<__half><<<grid, 128, 0, st>>>(static_cast<const __half*>(p.in0), static_cast<const float*>(p.wts),
+                                                               static_cast<const float*>(p.bias), static_cast<const __half*>(p.res),
+                                                               static_cast<__half*>(p.out), g, r.ep)),
+                (depthwise_kernel<float><<<grid, 128, 0, st>>>(static_cast<const float*>(p.in0), static_cast<const float*>(p.wts),
+                                                              static_cast<const float*>(p.bias), static_cast<const float*>(p.res),
+                                                              static_cast<float*>(p.out), g, r.ep)));
+  return static_cast<int>(cudaGetLastError());
+}
+
+int launch_eltwise(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t n_px = static_cast<size_t>(slices(r.Co)) * r.B * plane_pixels(r.Ho, r.Wo);
+  GI_BY_STORAGE((eltwise_kernel<__half><<<blocks_for(n_px, 256), 256, 0, st>>>(static_cast<const __half*>(p.in0),
+                                                                               static_cast<const __half*>(p.in1),
+                                                                               static_cast<__half*>(p.out), n_px, r.ep)),
+                (eltwise_kernel<float><<<blocks_for(n_px, 256), 256, 0, st>>>(static_cast<const float*>(p.in0),
+                                                                              static_cast<const float*>(p.in1),
+                                                                              static_cast<float*>(p.out), n_px, r.ep)));
+  return static_cast<int>(cudaGetLastError());
+}
+
+int launch_pool(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int planes = slices(r.C) * r.B;
+  const unsigned blocks = blocks_for(static_cast<size_t>(planes) * 32, 256);
+  GI_BY_STORAGE((pool_kernel<__half><<<blocks, 256, 0, st>>>(static_cast<const __half*>(p.in0), static_cast<__half*>(p.out), planes,
+                                                            r.H * r.W, plane_pixels(r.H, r.W), plane_pixels(1, 1))),
+                (pool_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(p.in0), static_cast<float*>(p.out), planes,
+                                                           r.H * r.W, plane_pixels(r.H, r.W), plane_pixels(1, 1))));
+  return static_cast<int>(cudaGetLastError());
+}
+
+int launch_resize(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (r.B > 65535) return static_cast<int>(cudaErrorInvalidConfiguration);
+  int ny, dy, nx, dx;
+  if (r.align_corners) {
+    ny = r.Ho > 1 ? r.H - 1 : 0;
+    dy = r.Ho > 1 ? r.Ho - 1 : 1;
+    nx = r.Wo > 1 ? r.W - 1 : 0;
+    dx = r.Wo > 1 ? r.Wo - 1 : 1;
+  } else {
+    ny = r.H;
+    dy = r.Ho;
+    nx = r.W;
+    dx = r.Wo;
+  }
+  const int Pout = plane_pixels(r.Ho, r.Wo), Pin = plane_pixels(r.H, r.W);
+  const dim3 grid(blocks_for(Pout, 128), slices(r.C), r.B);
+  GI_BY_STORAGE((resize_kernel<__half><<<grid, 128, 0, st>>>(static_cast<const __half*>(p.in0), static_cast<__half*>(p.out), r.B, r.H,
+                                                            r.W, Pin, r.Ho, r.Wo, Pout, ny, dy, nx, dx)),
+                (resize_kernel<float><<<grid, 128, 0, st>>>(static_cast<const float*>(p.in0), static_cast<float*>(p.out), r.B, r.H,
+                                                           r.W, Pin, r.Ho, r.Wo, Pout, ny, dy, nx, dx)));
+  return static_cast<int>(cudaGetLastError());
+}
+
+}  // namespace gi

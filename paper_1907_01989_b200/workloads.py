@@ -267,11 +267,11 @@ def single_pointwise(batch: int, hw: int, cin: int, cout: int, residual: bool = 
     """1x1 conv + bias + activation (+ residual add read from a second graph input)."""
     b = GraphBuilder(f"pw_{batch}x{hw}x{cin}x{cout}", batch, 5)
     x = b.input(hw, hw, cin)
+    r = b.input(hw, hw, cout) if residual else None
     y = b.conv2d(x, cout, 1)
     if act != ACT_NONE:
         y = b.activation(y, act)
     if residual:
-        r = b.input(hw, hw, cout)
         y = b.add(r, y)
     b.output(y)
     return b.finish()
@@ -281,9 +281,10 @@ def single_depthwise(batch: int, hw: int, c: int, stride: int = 1, dilation: int
                      residual: bool = False) -> GraphSpec:
     b = GraphBuilder(f"dw_{batch}x{hw}x{c}_s{stride}d{dilation}", batch, 6)
     x = b.input(hw, hw, c)
+    ho = same_pads(hw, 3, stride, dilation)[0]
+    r = b.input(ho, ho, c) if residual else None
     y = b.activation(b.depthwise(x, 3, stride, dilation), ACT_RELU6)
     if residual:
-        r = b.input(*b.g.shapes[y])
         y = b.add(r, y)
     b.output(y)
     return b.finish()

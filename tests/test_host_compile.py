@@ -1,0 +1,268 @@
+"""Host-side tests of the C-ABI library (no GPU): exported symbols, error behaviour, and the
+compile step compared bit-exactly with the oracle's independent implementation."""
+import ctypes as C
+import os
+import random
+import re
+
+import numpy as np
+import pytest
+
+from oracle import compile as oc
+from paper_1907_01989_b200 import api
+from paper_1907_01989_b200 import workloads as wl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+KIND_NAME = {api.GI_OP_CONV2D: "conv2d", api.GI_OP_DEPTHWISE_CONV2D: "depthwise_conv2d", api.GI_OP_ADD: "add",
+             api.GI_OP_ACTIVATION: "activation", api.GI_OP_GLOBAL_AVG_POOL: "global_avg_pool",
+             api.GI_OP_RESIZE_BILINEAR: "resize_bilinear"}
+ACT_NAME = {api.GI_ACT_NONE: None, api.GI_ACT_RELU: "relu", api.GI_ACT_RELU6: "relu6"}
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "gi.h")).read()
+    declared = re.findall(r"^GI_API\s+[\w\s\*]+?\b(gi_\w+)\s*\(", header, flags=re.M)
+    assert sorted(declared) == sorted(api.EXPORTS)
+    L = api.lib()
+    for name in declared:
+        assert getattr(L, name) is not None
+
+
+def test_f32_to_f16_matches_numpy():
+    rng = np.random.default_rng(7)
+    pos = np.arange(0, 0x7bff, dtype=np.uint16)
+    lo = pos.view(np.float16).astype(np.float64)
+    hi = (pos + 1).astype(np.uint16).view(np.float16).astype(np.float64)
+    mid = ((lo + hi) / 2).astype(np.float32)
+    edge = np.array([65504.0, 65519.99, 65520.0, 65536.0, 1e10, -65520.0, 2.0 ** -24, 2.0 ** -25, 2.0 ** -26, 6.1e-5,
+                     2.0 ** -14, np.inf, -np.inf, 0.0, -0.0], dtype=np.float32)
+    r = (rng.standard_normal(500_000) * np.exp(rng.uniform(-20, 12, 500_000))).astype(np.float32)
+    allh = np.arange(65536, dtype=np.uint16).view(np.float16)
+    allh = allh[~np.isnan(allh)].astype(np.float32)
+    with np.errstate(over="ignore"):
+        for x in (mid, np.nextafter(mid, np.float32(np.inf)), np.nextafter(mid, np.float32(-np.inf)), -mid, edge, r, allh):
+            assert np.array_equal(api.gi_f32_to_f16(x), x.astype(np.float16).view(np.uint16))
+
+
+def test_tensor_bytes_matches_size_formula():
+    for batch, shape in [(1, (8, 6, 12)), (1, (7, 7, 5)), (3, (7, 7, 4)), (256, (112, 112, 96)), (2, (1, 1, 1001)),
+                         (16, (513, 513, 21))]:
+        for storage, eb in ((api.GI_F16, 2), (api.GI_F32, 4)):
+            for align in (256, 1024):
+                assert api.gi_tensor_bytes(batch, *shape, storage, align) == oc.tensor_bytes(batch, shape, eb, align)
+
+
+# ---------------------------------------------------------------------- compile step vs oracle
+def exec_records(ex):
+    """(ops, sizes, intermediates, lifetimes, offsets) as the library reports them."""
+    ops = ex.ops()
+    tensors = {t: ex.tensor(t) for t in range(ex.info.n_tensors)}
+    return ops, tensors
+
+
+def compare_with_oracle(spec, planner, fuse=True, storage=api.GI_F16, align=256):
+    g, ids = api.graph_from_spec(spec, storage)
+    assert all(ids[t] == t for t in ids)  # the builder and the library number tensors alike
+    ex = g.compile(planner=planner, fuse=fuse, align=align)
+    ops, tensors = exec_records(ex)
+    fused = oc.fuse(spec, enable=fuse)
+    n_in, n_out = len(spec.inputs), len(spec.outputs)
+    assert ex.info.n_fused_ops == len(fused)
+    assert ex.info.n_ops == len(fused) + n_in + n_out
+    for k in range(n_in):
+        assert ops[k].kind == api.GI_EXEC_PACK and ops[k].output == spec.inputs[k]
+    for k in range(n_out):
+        o = ops[n_in + len(fused) + k]
+        assert o.kind == api.GI_EXEC_UNPACK and o.inputs[0] == spec.outputs[k]
+    for f, o in zip(fused, ops[n_in:n_in + len(fused)]):
+        assert KIND_NAME[o.kind] == f.kind and o.graph_op == f.op_index and o.output == f.output
+        assert [t for t in (o.inputs[0], o.inputs[1]) if t >= 0] == f.inputs
+        adds = [a for k, a in f.epilogue if k == "add"]
+        assert (o.residual if o.residual >= 0 else None) == (adds[0] if adds else None)
+        if f.kind in oc.CONV_KINDS:
+            pre, post, seen_add = None, None, False
+            for k, a in f.epilogue:
+                if k == "add":
+                    seen_add = True
+                elif seen_add or pre is not None:
+                    post = a
+                else:
+                    pre = a
+            assert ACT_NAME[o.act_pre] == pre and ACT_NAME[o.act_post] == post
+    p = oc.plan_problem(spec, fused, 2 if storage == api.GI_F16 else 4, align, convert_io=True)
+    life = oc.lifetimes(p)
+    for t, ti in tensors.items():
+        assert bool(ti.alive) == (t in p.size)
+        assert (ti.h, ti.w, ti.c) == tuple(spec.shapes[t])
+        if t in p.size:
+            assert ti.intermediate == 1
+            assert ti.bytes == p.size[t]
+            assert (ti.first_op, ti.last_op) == life[t]
+    if planner == api.GI_PLAN_NAIVE:
+        off, total = oc.plan_naive(p)
+    elif planner == api.GI_PLAN_GREEDY_SHARED_OBJECTS:
+        off, total = oc.plan_greedy_shared_objects(p)[:2]
+    else:
+        off, total = oc.plan_greedy_by_size(p)
+    assert ex.info.arena_bytes == total
+    assert ex.info.naive_bytes == oc.plan_naive(p)[1]
+    assert ex.info.lower_bound_bytes == oc.lower_bound(p)
+    for t in p.intermediate:
+        assert tensors[t].offset == off[t], (t, tensors[t].offset, off[t])
+        assert tensors[t].offset % align == 0
+    oc.check_no_overlap(p, {t: tensors[t].offset for t in p.intermediate})
+    return ex
+
+
+PLANNERS = [api.GI_PLAN_GREEDY_BY_SIZE, api.GI_PLAN_GREEDY_SHARED_OBJECTS, api.GI_PLAN_NAIVE]
+NETS = [lambda: wl.separable_block(1), lambda: wl.mobilenet_v1(1), lambda: wl.mobilenet_v2(1),
+        lambda: wl.mobilenet_v2_segmentation(1), lambda: wl.mobilenet_v2(256), lambda: wl.mobilenet_v2_segmentation(16),
+        lambda: wl.single_pointwise(8, 14, 96, 576, residual=True), lambda: wl.single_depthwise(8, 7, 96, 2)]
+
+
+@pytest.mark.parametrize("planner", PLANNERS)
+@pytest.mark.parametrize("net", range(len(NETS)))
+def test_plan_offsets_bit_exact_on_workloads(net, planner):
+    spec = NETS[net]()
+    compare_with_oracle(spec, planner)
+    if net < 3:
+        compare_with_oracle(spec, planner, fuse=False)
+        compare_with_oracle(spec, planner, storage=api.GI_F32, align=1024)
+
+
+def random_spec(rnd: random.Random, n_ops: int) -> wl.GraphSpec:
+    b = wl.GraphBuilder("random", rnd.choice([1, 2, 3]), 99)
+    live = [b.input(rnd.choice([5, 8, 9]), rnd.choice([4, 7, 8]), rnd.choice([3, 4, 6, 8]))]
+    for _ in range(n_ops):
+        x = rnd.choice(live[-4:])
+        kind = rnd.choice(["conv1", "conv3", "dw", "act", "act", "add", "add", "pool"])
+        H, W, Cc = b.g.shapes[x]
+        if kind == "conv1":
+            y = b.conv2d(x, rnd.choice([4, 6, 8, Cc]), 1)
+        elif kind == "conv3":
+            y = b.conv2d(x, rnd.choice([4, 8, Cc]), 3, rnd.choice([1, 2]))
+        elif kind == "dw":
+            y = b.depthwise(x, 3, rnd.choice([1, 2]), rnd.choice([1, 2]))
+        elif kind == "act":
+            y = b.activation(x, rnd.choice([wl.ACT_RELU, wl.ACT_RELU6]))
+        elif kind == "add":
+            same = [t for t in live if b.g.shapes[t] == b.g.shapes[x]]
+            y = b.add(rnd.choice(same), x)
+        else:
+            if H * W == 1:
+                continue
+            y = b.global_avg_pool(x)
+        live.append(y)
+    used = {t for op in b.g.ops for t in op.inputs}
+    outs = [t for t in live[1:] if t not in used] or [live[-1]]
+    if live[-1] not in outs and live[-1] != live[0]:
+        outs.append(live[-1])
+    for t in outs:
+        if t != live[0]:
+            b.output(t)
+    if not b.g.outputs:
+        b.output(b.activation(live[0], wl.ACT_RELU))
+    return b.finish()
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_plan_offsets_bit_exact_on_random_graphs(seed):
+    rnd = random.Random(seed)
+    spec = random_spec(rnd, rnd.randint(1, 30))
+    for planner in PLANNERS:
+        compare_with_oracle(spec, planner)
+    compare_with_oracle(spec, api.GI_PLAN_GREEDY_BY_SIZE, fuse=False)
+
+
+def test_expected_fused_counts_and_arena():
+    for make, n_fused, mib in ((wl.mobilenet_v1, 29, 2.297), (wl.mobilenet_v2, 54, 2.871),
+                               (wl.mobilenet_v2_segmentation, 54, 15.14)):
+        g, _ = api.graph_from_spec(make(1))
+        ex = g.compile()
+        assert ex.info.n_fused_ops == n_fused and ex.info.n_ops == n_fused + 2
+        assert abs(ex.info.arena_bytes / 2 ** 20 - mib) < 2e-3
+        assert ex.info.arena_bytes == ex.info.lower_bound_bytes
+
+
+# ---------------------------------------------------------------------- error behaviour
+def _conv_desc(x, cout=8, k=1, **kw):
+    d = api.gi_op_desc()
+    d.kind = api.GI_OP_CONV2D
+    d.inputs[0] = x
+    d.inputs[1] = -1
+    d.kh = d.kw = k
+    d.stride_h = d.stride_w = d.dilation_h = d.dilation_w = 1
+    d.cout = cout
+    d.weight_dtype = api.GI_F32
+    for key, v in kw.items():
+        setattr(d, key, v)
+    return d
+
+
+def test_error_paths():
+    L = api.lib()
+    h = C.c_void_p()
+    assert L.gi_graph_create(C.byref(h), 0, api.GI_F16) == api.GI_E_INVALID
+    assert L.gi_graph_create(C.byref(h), 1, 7) == api.GI_E_INVALID
+    assert L.gi_graph_create(None, 1, api.GI_F16) == api.GI_E_INVALID
+    assert b"batch" in L.gi_last_error() or b"null" in L.gi_last_error()
+    g = api.Graph(2)
+    with pytest.raises(api.GiError):
+        g.input(0, 4, 4)
+    x = g.input(8, 8, 4)
+    w = np.zeros((8, 5, 5, 4), dtype=np.float32)
+    with pytest.raises(api.GiError) as ei:
+        g.add_op(_conv_desc(x, k=5, weights=w.ctypes.data))
+    assert ei.value.status == api.GI_E_UNSUPPORTED
+    with pytest.raises(api.GiError) as ei:
+        g.add_op(_conv_desc(x))  # no weights
+    assert ei.value.status == api.GI_E_INVALID
+    with pytest.raises(api.GiError):
+        g.add_op(_conv_desc(17, weights=w.ctypes.data))  # unknown tensor
+    with pytest.raises(api.GiError):
+        g.add_op(_conv_desc(x, weights=w.ctypes.data, stride_h=0))
+    with pytest.raises(api.GiError) as ei:
+        g.add_op(_conv_desc(x, weights=w.ctypes.data, stride_h=3, stride_w=3))
+    assert ei.value.status == api.GI_E_UNSUPPORTED
+    y = g.add_op(_conv_desc(x, cout=8, weights=w.ctypes.data))
+    d = api.gi_op_desc()
+    d.kind = api.GI_OP_ADD
+    d.inputs[0], d.inputs[1] = x, y  # 4 vs 8 channels
+    with pytest.raises(api.GiError):
+        g.add_op(d)
+    d = api.gi_op_desc()
+    d.kind = api.GI_OP_ACTIVATION
+    d.inputs[0] = y
+    with pytest.raises(api.GiError):
+        g.add_op(d)  # act missing
+    with pytest.raises(api.GiError):
+        g.output(x)  # an input cannot be an output
+    with pytest.raises(api.GiError):
+        g.compile()  # no outputs yet
+    g.output(y)
+    with pytest.raises(api.GiError):
+        g.output(y)
+    with pytest.raises(api.GiError):
+        g.compile(align=100)
+    with pytest.raises(api.GiError):
+        g.compile(planner=9)
+    ex = g.compile()
+    assert ex.info.n_ops == 3
+    with pytest.raises(api.GiError):
+        ex.tensor(99)
+    with pytest.raises(api.GiError):
+        ex.op(3)
+    # gi_run before gi_exec_bind is refused before anything touches the device
+    with pytest.raises(api.GiError) as ei:
+        ex.run_raw([256], [256], 256, 1 << 30, stream=0)
+    assert ei.value.status == api.GI_E_STATE
+
+
+def test_graph_reusable_after_compile_and_weights_copied():
+    spec = wl.separable_block(1)
+    g, _ = api.graph_from_spec(spec)
+    a = g.compile(planner=api.GI_PLAN_NAIVE)
+    b = g.compile(planner=api.GI_PLAN_GREEDY_BY_SIZE)
+    assert a.info.weight_bytes == b.info.weight_bytes > 0
+    assert a.info.arena_bytes >= b.info.arena_bytes
