@@ -1,0 +1,372 @@
+#!/usr/bin/env python
+"""Benchmark of the fused-CNN inference path: MobileNetV2-224, fp16 storage, batch 256 per GPU.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--net v2|v1|seg] [--batch B]
+
+One step = one gi_run of the whole network (layout conversion in, 54 fused ops, layout
+conversion out) on a batch of synthetic images.  Prints ONE JSON line on rank 0.
+
+* value        images/s with the input batch already resident in HBM (CUDA events on the run
+               stream around each gi_run, L2 flushed by an untimed 256 MiB memset between steps).
+* e2e          the same metric through the public call with HOST buffers: pinned fp16 NHWC images
+               copied to the device, gi_run, logits copied back, all inside the timed region.
+* roofline     the kernel family with the largest share of the step, from gi_run_timed (one CUDA
+               event pair per executed op, same stream): algorithmic bytes / measured time against
+               the measured HBM peak (or flops against the tensor peak where that binds).
+* cpu_baseline the CPU oracle as it stands on this machine's host cores, on a bounded sample of images.
+* batch1       latency of the same network at batch 1, plain launches and CUDA-graph replay.
+
+N > 1 runs independent replicas (one process per GPU, the batch is the only sharded axis and
+the path has no exchange step): weak scaling, no collective on the data path.
+--impl reference times the CPU oracle instead (rank 0 only).
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+NETS = {"v2": ("mobilenet_v2", "MobileNetV2-224"), "v1": ("mobilenet_v1", "MobileNetV1-224"),
+        "seg": ("mobilenet_v2_segmentation", "MobileNetV2-513-OS16-seg")}
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            p = json.load(fh)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi during the timed region (read-only query)."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for row in self.rows:
+            f = [x.strip() for x in row.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_images_per_s(spec_fn, budget_s=15.0):
+    """Time the CPU oracle on a bounded sample of the workload's images."""
+    from oracle import graph as og
+    from oracle import ops as oops
+    from paper_1907_01989_b200 import workloads as wl
+    spec1 = spec_fn(1)
+    x1 = wl.make_input(spec1, images=[0])
+    t0 = time.perf_counter()
+    og.run(spec1, [x1], storage="f16", fused=True)
+    t1 = time.perf_counter() - t0
+    cores = oops.num_threads()
+    n = int(max(1, min(64, budget_s / max(t1, 1e-3) * min(cores, 8) / 4)))
+    spec = spec_fn(n)
+    x = wl.make_input(spec, images=list(range(n)))
+    t0 = time.perf_counter()
+    og.run(spec, [x], storage="f16", fused=True)
+    dt = time.perf_counter() - t0
+    return n / dt, cores, f"{n} images of the workload, evaluated once as one batch of {n} ({dt:.1f} s)", n, dt
+
+
+def run_reference(args, spec_fn, label):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    sample = ""
+    for step in range(args.warmup + args.steps):
+        v, cores, sample, n, dt = oracle_images_per_s(spec_fn, budget_s=max(1.0, 100.0 / (args.warmup + args.steps)))
+        if step >= args.warmup:
+            vals.append((n, dt))
+    n_tot, t_tot = sum(n for n, _ in vals), sum(t for _, t in vals)
+    value = n_tot / t_tot
+    line = {"impl": "reference", "metric": f"{label} fp16 images/s (batch {args.batch})", "value": value,
+            "unit": "images/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * t_tot / len(vals), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f16", "data": "synthetic",
+            "config": {"workload": f"{NETS[args.net][0]}_batch{args.batch}", "note": "CPU oracle on host cores; "
+                       "each step is a bounded sample of the workload's images"},
+            "cpu_baseline": {"value": value, "unit": "images/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--net", default="v2", choices=sorted(NETS))
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--pointwise", default="auto", choices=["auto", "simt"])
+    ap.add_argument("--per-op", default=None, help="write the per-op timing table to this file")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.batch is None:
+        args.batch = 16 if args.net == "seg" else 256
+
+    from paper_1907_01989_b200 import workloads as wl
+    fn_name, label = NETS[args.net]
+    spec_fn = getattr(wl, fn_name)
+    if args.impl == "reference":
+        run_reference(args, spec_fn, label)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_1907_01989_b200 import api
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    spec = spec_fn(args.batch)
+    graph, _ = api.graph_from_spec(spec, api.GI_F16)
+    ex = graph.compile(pointwise=api.GI_PW_SIMT if args.pointwise == "simt" else api.GI_PW_AUTO)
+    ex.bind(dev)
+    ops = ex.ops()
+    # every rank draws its own images: rank r holds images [r*B, (r+1)*B) of the global batch
+    x_host = wl.make_input(spec, images=[rank * args.batch + i for i in range(args.batch)]).astype(np.float16)
+    x_pin = torch.from_numpy(x_host).pin_memory()
+    x_dev = x_pin.to(dev, non_blocking=False)
+    out_shape = (args.batch,) + tuple(spec.shapes[spec.outputs[0]])
+    out_dev = torch.empty(out_shape, dtype=torch.float16, device=dev)
+    out_pin = torch.empty(out_shape, dtype=torch.float16).pin_memory()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step_resident():
+        ex.run([x_dev], [out_dev], stream)
+
+    # ---- resident-input throughput -------------------------------------------------------
+    for _ in range(args.warmup):
+        flush.zero_()
+        step_resident()
+    sampler = ClockSampler(local)
+    barrier()
+    if rank == 0:
+        sampler.start()
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    wall0 = time.perf_counter()
+    for i in range(args.steps):
+        flush.zero_()
+        starts[i].record(stream)
+        step_resident()
+        ends[i].record(stream)
+    barrier()
+    wall = time.perf_counter() - wall0
+    clocks = sampler.stop() if rank == 0 else None
+    ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
+    t_steps = torch.tensor([sum(ms)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t_steps, op=dist.ReduceOp.MAX)
+    total_ms = float(t_steps.item())
+    ms_per_step = total_ms / args.steps
+    value = world * args.batch * args.steps / (total_ms * 1e-3)
+
+    # ---- end to end with host buffers ------------------------------------------------------
+    def step_e2e():
+        x_dev.copy_(x_pin, non_blocking=True)
+        ex.run([x_dev], [out_dev], stream)
+        out_pin.copy_(out_dev, non_blocking=True)
+
+    for _ in range(3):
+        step_e2e()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step_e2e()
+    e1.record(stream)
+    barrier()
+    t_e2e = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t_e2e, op=dist.ReduceOp.MAX)
+    e2e_value = world * args.batch * args.steps / (float(t_e2e.item()) * 1e-3)
+    logits_checksum = float(out_pin.float().abs().mean())
+
+    # ---- per-op times for the roofline (rank 0) ---------------------------------------------
+    line = None
+    if rank == 0:
+        peaks, peak_kind = load_peaks()
+        per_op = np.zeros(len(ops))
+        reps = max(3, min(args.steps, 10))
+        for _ in range(2):
+            ex.run_timed([x_dev], [out_dev], stream)
+        for _ in range(reps):
+            flush.zero_()
+            per_op += np.array(ex.run_timed([x_dev], [out_dev], stream))
+        per_op /= reps
+        fam = {}
+        for o, t in zip(ops, per_op):
+            name = api.KERNEL_NAMES[o.kernel]
+            f = fam.setdefault(name, {"launches": 0, "ms": 0.0, "bytes": 0, "flops": 0, "roof_ms": 0.0})
+            f["launches"] += 1
+            f["ms"] += float(t)
+            f["bytes"] += int(o.bytes)
+            f["flops"] += int(o.flops)
+            f["roof_ms"] += max(o.bytes / (peaks["hbm_gbs"] * 1e9), o.flops / (peaks["bf16_tflops_sustained"] * 1e12)) * 1e3
+        total_op_ms = sum(f["ms"] for f in fam.values())
+        kernels = []
+        for name, f in sorted(fam.items(), key=lambda kv: -kv[1]["ms"]):
+            kernels.append({"kernel": name, "launches": f["launches"], "ms": round(f["ms"], 4),
+                            "share": round(f["ms"] / total_op_ms, 4), "gbs": round(f["bytes"] / f["ms"] / 1e6, 1),
+                            "tflops": round(f["flops"] / f["ms"] / 1e9, 2),
+                            "frac_of_roofline": round(f["roof_ms"] / f["ms"], 4)})
+        top_name = kernels[0]["kernel"]
+        top = fam[top_name]
+        hbm_time = top["bytes"] / (peaks["hbm_gbs"] * 1e9)
+        tensor_time = top["flops"] / (peaks["bf16_tflops_sustained"] * 1e12)
+        if tensor_time > hbm_time:
+            roofline = {"bound": "tensor", "achieved": top["flops"] / top["ms"] / 1e9, "peak": peaks["bf16_tflops_sustained"],
+                        "unit": "TFLOP/s"}
+        else:
+            roofline = {"bound": "hbm", "achieved": top["bytes"] / top["ms"] / 1e6, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+        roofline["frac"] = roofline["achieved"] / roofline["peak"]
+        roofline.update({"traffic": None, "kernel": top_name, "launches_per_step": top["launches"],
+                         "bytes_per_step": top["bytes"], "ms_per_step": round(top["ms"], 4), "peak_source": peak_kind,
+                         "per_kernel": kernels})
+        if args.per_op:
+            with open(args.per_op, "w") as fh:
+                fh.write("# op kernel in_shape out_shape bytes flops ms GB/s TFLOP/s frac_of_roofline\n")
+                for i, (o, t) in enumerate(zip(ops, per_op)):
+                    ti = ex.tensor(o.inputs[0]) if o.inputs[0] >= 0 else None
+                    to = ex.tensor(o.output) if o.output >= 0 else None
+                    roof = max(o.bytes / (peaks["hbm_gbs"] * 1e9), o.flops / (peaks["bf16_tflops_sustained"] * 1e12)) * 1e3
+                    fh.write(f"{i} {api.KERNEL_NAMES[o.kernel]} "
+                             f"{(ti.h, ti.w, ti.c) if ti else '-'} {(to.h, to.w, to.c) if to else '-'} {o.bytes} {o.flops} "
+                             f"{t:.4f} {o.bytes / t / 1e6:.0f} {o.flops / t / 1e9:.1f} {roof / t:.3f}\n".replace(", ", ","))
+
+        # ---- batch-1 latency (the paper's protocol: 10 warm-up runs, mean of the next 100) ----
+        spec1 = spec_fn(1)
+        g1, _ = api.graph_from_spec(spec1, api.GI_F16)
+        ex1 = g1.compile(pointwise=api.GI_PW_SIMT if args.pointwise == "simt" else api.GI_PW_AUTO)
+        ex1.bind(dev)
+        x1 = torch.from_numpy(wl.make_input(spec1).astype(np.float16)).to(dev)
+        o1 = torch.empty((1,) + tuple(spec1.shapes[spec1.outputs[0]]), dtype=torch.float16, device=dev)
+        for _ in range(10):
+            ex1.run([x1], [o1], stream)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record(stream)
+        for _ in range(100):
+            ex1.run([x1], [o1], stream)
+        b.record(stream)
+        torch.cuda.synchronize()
+        b1_ms = a.elapsed_time(b) / 100
+        side = torch.cuda.Stream()
+        graph_ms = None
+        try:
+            with torch.cuda.stream(side):
+                ex1.run([x1], [o1], side)
+                side.synchronize()
+                cg = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(cg, stream=side):
+                    ex1.run([x1], [o1], torch.cuda.current_stream())
+                for _ in range(10):
+                    cg.replay()
+                side.synchronize()
+                a.record(side)
+                for _ in range(100):
+                    cg.replay()
+                b.record(side)
+                side.synchronize()
+                graph_ms = a.elapsed_time(b) / 100
+        except Exception as exc:  # graph capture is an extra, never the headline
+            graph_ms = f"capture failed: {type(exc).__name__}"
+
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            v, cores, sample, _, _ = oracle_images_per_s(spec_fn)
+            cpu = {"value": v, "unit": "images/s", "cores": cores, "kind": "oracle", "sample": sample}
+
+        line = {"metric": f"{label} fp16 images/s (batch {args.batch})", "value": value, "unit": "images/s",
+                "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+                "config": {"workload": f"{fn_name}_batch{args.batch}", "batch_per_gpu": args.batch,
+                           "launches_per_step": len(ops), "arena_mib": round(ex.info.arena_bytes / 2 ** 20, 1),
+                           "l2": "flushed between steps by an untimed 256 MiB memset; a step moves ~"
+                                 f"{sum(o.bytes for o in ops) / 1e9:.1f} GB", "parallelism": f"replicas x{world}",
+                           "pointwise": args.pointwise},
+                "roofline": roofline, "cpu_baseline": cpu,
+                "e2e": {"value": e2e_value, "unit": "images/s", "h2d_bytes_per_step": int(x_pin.numel() * 2),
+                        "d2h_bytes_per_step": int(out_pin.numel() * 2)},
+                "gpu_launches": args.steps * len(ops), "clocks": clocks,
+                "batch1": {"ms": b1_ms, "cuda_graph_ms": graph_ms, "launches": int(ex1.info.n_ops),
+                           "protocol": "10 warm-up runs, mean of the next 100"},
+                "step_ms_min_median_max": [min(ms), statistics.median(ms), max(ms)], "wall_s_timed_region": wall,
+                "logits_abs_mean": logits_checksum}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -214,6 +214,14 @@ GI_API gi_status gi_exec_bind(gi_exec* e, void* dev_weights, size_t weight_bytes
 GI_API gi_status gi_run(gi_exec* e, const void* const* dev_inputs, void* const* dev_outputs, void* dev_arena,
                  size_t arena_bytes, void* stream);
 
+/* Profiling aid: the same launches as gi_run, with a CUDA event recorded before each executed op
+ * and after the last one; synchronises `stream` before returning and writes the device time of
+ * op i, in milliseconds, to op_ms[i] (n_op_ms must be >= info.n_ops).  The paper's own protocol
+ * times whole inferences (Section 6); per-op times are what the per-kernel roofline needs.
+ * Creates and destroys CUDA events; not capturable; not for the production path. */
+GI_API gi_status gi_run_timed(gi_exec* e, const void* const* dev_inputs, void* const* dev_outputs, void* dev_arena,
+                              size_t arena_bytes, void* stream, float* op_ms, int32_t n_op_ms);
+
 GI_API void gi_exec_destroy(gi_exec* e);
 
 /* ---- helpers ---- */

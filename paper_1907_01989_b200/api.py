@@ -66,7 +66,7 @@ class gi_op_info(C.Structure):
 
 
 EXPORTS = ["gi_graph_create", "gi_graph_input", "gi_add_op", "gi_graph_output", "gi_graph_destroy", "gi_compile",
-           "gi_exec_query", "gi_exec_tensor", "gi_exec_op", "gi_exec_bind", "gi_run", "gi_exec_destroy",
+           "gi_exec_query", "gi_exec_tensor", "gi_exec_op", "gi_exec_bind", "gi_run", "gi_run_timed", "gi_exec_destroy",
            "gi_status_str", "gi_last_error", "gi_tensor_bytes", "gi_f32_to_f16"]
 
 _lib = None
@@ -100,6 +100,7 @@ def lib() -> C.CDLL:
     L.gi_exec_op.argtypes = [vp, C.c_int32, C.POINTER(gi_op_info)]
     L.gi_exec_bind.argtypes = [vp, vp, C.c_size_t, vp]
     L.gi_run.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp, C.c_size_t, vp]
+    L.gi_run_timed.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp, C.c_size_t, vp, C.POINTER(C.c_float), C.c_int32]
     L.gi_exec_destroy.argtypes = [vp]
     L.gi_exec_destroy.restype = None
     L.gi_status_str.argtypes = [C.c_int32]
@@ -111,7 +112,7 @@ def lib() -> C.CDLL:
     L.gi_f32_to_f16.argtypes = [vp, vp, C.c_size_t]
     L.gi_f32_to_f16.restype = None
     for name in ("gi_graph_create", "gi_graph_input", "gi_add_op", "gi_graph_output", "gi_compile", "gi_exec_query",
-                 "gi_exec_tensor", "gi_exec_op", "gi_exec_bind", "gi_run"):
+                 "gi_exec_tensor", "gi_exec_op", "gi_exec_bind", "gi_run", "gi_run_timed"):
         getattr(L, name).restype = C.c_int32
     _lib = L
     return L
@@ -256,6 +257,16 @@ class Executable:
         ins = (C.c_void_p * max(len(in_ptrs), 1))(*in_ptrs)
         outs = (C.c_void_p * max(len(out_ptrs), 1))(*out_ptrs)
         _check(lib().gi_run(self._h, ins, outs, arena_ptr, arena_bytes, _stream_ptr(stream)), "gi_run")
+
+    def run_timed(self, inputs, outputs, stream=None) -> List[float]:
+        """gi_run_timed: one run with an event around every executed op; returns per-op milliseconds."""
+        n = int(self.info.n_ops)
+        ms = (C.c_float * n)()
+        ins = (C.c_void_p * max(len(inputs), 1))(*[t.data_ptr() for t in inputs])
+        outs = (C.c_void_p * max(len(outputs), 1))(*[t.data_ptr() for t in outputs])
+        _check(lib().gi_run_timed(self._h, ins, outs, self._arena.data_ptr(), self._arena.numel(), _stream_ptr(stream),
+                                  ms, n), "gi_run_timed")
+        return list(ms)
 
     def run(self, inputs, outputs, stream=None) -> None:
         """inputs / outputs: torch CUDA tensors in the declared layouts (contiguous, storage dtype)."""

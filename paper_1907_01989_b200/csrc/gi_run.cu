@@ -4,6 +4,7 @@
 
 #include <cstdint>
 #include <string>
+#include <vector>
 
 #include "gi_internal.h"
 #include "kernels.h"
@@ -37,8 +38,8 @@ gi_status gi_exec_bind(gi_exec* e, void* dev_weights, size_t weight_bytes, void*
   return GI_OK;
 }
 
-gi_status gi_run(gi_exec* e, const void* const* dev_inputs, void* const* dev_outputs, void* dev_arena, size_t arena_bytes,
-                 void* stream) {
+static gi_status run_impl(gi_exec* e, const void* const* dev_inputs, void* const* dev_outputs, void* dev_arena,
+                          size_t arena_bytes, void* stream, cudaEvent_t* events) {
   if (!e || !dev_inputs || !dev_outputs) return fail(GI_E_INVALID, "gi_run: null argument");
   if (!e->dev_weights) return fail(GI_E_STATE, "gi_run: gi_exec_bind has not been called");
   if (e->arena_bytes > 0) {
@@ -63,6 +64,7 @@ gi_status gi_run(gi_exec* e, const void* const* dev_inputs, void* const* dev_out
 
   for (size_t i = 0; i < e->launches.size(); ++i) {
     const LaunchRec& r = e->launches[i];
+    if (events) cudaEventRecord(events[i], static_cast<cudaStream_t>(stream));
     Ptrs p;
     p.in0 = resolve(r.in0);
     p.in1 = resolve(r.in1);
@@ -90,7 +92,35 @@ gi_status gi_run(gi_exec* e, const void* const* dev_inputs, void* const* dev_out
                                  cudaGetErrorString(static_cast<cudaError_t>(err)));
     }
   }
+  if (events) cudaEventRecord(events[e->launches.size()], static_cast<cudaStream_t>(stream));
   return GI_OK;
+}
+
+gi_status gi_run(gi_exec* e, const void* const* dev_inputs, void* const* dev_outputs, void* dev_arena, size_t arena_bytes,
+                 void* stream) {
+  return run_impl(e, dev_inputs, dev_outputs, dev_arena, arena_bytes, stream, nullptr);
+}
+
+gi_status gi_run_timed(gi_exec* e, const void* const* dev_inputs, void* const* dev_outputs, void* dev_arena,
+                       size_t arena_bytes, void* stream, float* op_ms, int32_t n_op_ms) {
+  if (!e || !op_ms) return fail(GI_E_INVALID, "gi_run_timed: null argument");
+  const size_t n = e->launches.size();
+  if (n_op_ms < 0 || static_cast<size_t>(n_op_ms) < n) return fail(GI_E_INVALID, "gi_run_timed: op_ms too short");
+  std::vector<cudaEvent_t> ev(n + 1, nullptr);
+  gi_status st = GI_OK;
+  for (size_t i = 0; i <= n && st == GI_OK; ++i)
+    if (cudaEventCreate(&ev[i]) != cudaSuccess) st = fail(GI_E_CUDA, "gi_run_timed: cudaEventCreate failed");
+  if (st == GI_OK) st = run_impl(e, dev_inputs, dev_outputs, dev_arena, arena_bytes, stream, ev.data());
+  if (st == GI_OK) {
+    const cudaError_t err = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (err != cudaSuccess) st = fail(GI_E_CUDA, std::string("gi_run_timed: ") + cudaGetErrorString(err));
+  }
+  if (st == GI_OK)
+    for (size_t i = 0; i < n; ++i)
+      if (cudaEventElapsedTime(&op_ms[i], ev[i], ev[i + 1]) != cudaSuccess) op_ms[i] = -1.0f;
+  for (cudaEvent_t x : ev)
+    if (x) cudaEventDestroy(x);
+  return st;
 }
 
 }  // extern "C"
