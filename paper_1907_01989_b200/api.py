@@ -66,7 +66,7 @@ class gi_op_info(C.Structure):
 
 
 EXPORTS = ["gi_graph_create", "gi_graph_input", "gi_add_op", "gi_graph_output", "gi_graph_destroy", "gi_compile",
-           "gi_exec_query", "gi_exec_tensor", "gi_exec_op", "gi_exec_bind", "gi_run", "gi_run_timed", "gi_exec_destroy",
+           "gi_exec_query", "gi_exec_tensor", "gi_exec_op", "gi_exec_bind", "gi_run", "gi_run_timed", "gi_device_status", "gi_exec_destroy",
            "gi_status_str", "gi_last_error", "gi_tensor_bytes", "gi_f32_to_f16"]
 
 _lib = None
@@ -101,6 +101,8 @@ def lib() -> C.CDLL:
     L.gi_exec_bind.argtypes = [vp, vp, C.c_size_t, vp]
     L.gi_run.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp, C.c_size_t, vp]
     L.gi_run_timed.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp, C.c_size_t, vp, C.POINTER(C.c_float), C.c_int32]
+    L.gi_device_status.argtypes = [C.POINTER(C.c_uint32)]
+    L.gi_device_status.restype = C.c_int32
     L.gi_exec_destroy.argtypes = [vp]
     L.gi_exec_destroy.restype = None
     L.gi_status_str.argtypes = [C.c_int32]
@@ -133,6 +135,12 @@ def gi_f32_to_f16(x: np.ndarray) -> np.ndarray:
     out = np.empty(x.shape, dtype=np.uint16)
     lib().gi_f32_to_f16(x.ctypes.data, out.ctypes.data, x.size)
     return out
+
+
+def gi_device_status() -> int:
+    flags = C.c_uint32(0)
+    _check(lib().gi_device_status(C.byref(flags)), "gi_device_status")
+    return int(flags.value)
 
 
 class Graph:

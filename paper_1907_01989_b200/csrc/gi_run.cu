@@ -96,6 +96,14 @@ static gi_status run_impl(gi_exec* e, const void* const* dev_inputs, void* const
   return GI_OK;
 }
 
+gi_status gi_device_status(uint32_t* flags) {
+  if (!flags) return fail(GI_E_INVALID, "gi_device_status: null argument");
+  int err = 0;
+  *flags = pointwise_tc_error_word(&err);
+  if (err != 0) return fail(GI_E_CUDA, std::string("gi_device_status: ") + cudaGetErrorString(static_cast<cudaError_t>(err)));
+  return GI_OK;
+}
+
 gi_status gi_run(gi_exec* e, const void* const* dev_inputs, void* const* dev_outputs, void* dev_arena, size_t arena_bytes,
                  void* stream) {
   return run_impl(e, dev_inputs, dev_outputs, dev_arena, arena_bytes, stream, nullptr);

@@ -32,5 +32,6 @@ void pointwise_tc_pack(const float* w, const float* bias, int cin, int cout, std
 // tensor maps depend on device addresses; `state` caches them per executable
 int launch_pointwise_tc(const LaunchRec& r, const Ptrs& p, void** state, int launch_index, void* stream);
 void pointwise_tc_release(void* state);
+unsigned int pointwise_tc_error_word(int* cuda_err);
 
 }  // namespace gi

@@ -1,9 +1,556 @@
-// Tensor-core pointwise convolution (placeholder until the tcgen05 kernel lands).
+// Pointwise (1x1) convolution on the 5th-generation tensor cores: tcgen05.mma with the
+// accumulator in tensor memory, operands fed by TMA, fused bias / activation / residual
+// epilogue.  This is the "specialised 1x1 convolution" of Section 3.2, rebuilt for sm_100a.
+//
+// The channel-sliced layout stores 4 channels (8 bytes) per pixel-slice, while the tensor
+// core wants 16 contiguous bytes along K.  Two neighbouring pixels of one slice are 16
+// contiguous bytes, so a plane is read as rows of "pixel pairs":
+//     A'[r][s*8 + p*4 + c] = x[pixel 2r+p][channel 4s+c]           (r: pair, p: parity)
+// which is exactly the canonical K-major, no-swizzle operand layout (8 rows x 16 bytes per core
+// matrix) and can be copied by TMA with no repacking.  The weights are expanded at compile
+// time into B'[so*8 + p'*4 + j][s*8 + p*4 + c] = (p == p') ? w[4so+j][4s+c] : 0, so that
+//     D'[r][so*8 + p'*4 + j] = y[pixel 2r+p'][channel 4so+j],
+// i.e. 8 consecutive fp32 accumulator columns of one lane are the 16 output bytes of a pixel
+// pair in one output slice.  Half of the multiplies hit structural zeros; these layers are
+// bound by HBM bandwidth, not by the tensor pipe, so the pipe has the slack.
+//
+// One CTA per SM, persistent over (pixel tile, output-channel tile) units; warp 0 issues TMA,
+// warp 1 issues MMAs and owns tensor memory, warps 2-5 run the epilogue (one TMEM lane quarter
+// each).  Accumulators are double-buffered so the epilogue of a tile overlaps the next tile's
+// loads and MMAs.  Every wait is bounded: after about a second it raises an error word the
+// host can read, drains the copies in flight and leaves, so the context stays usable.
+#include <cuda.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <cstring>
+#include <mutex>
+#include <vector>
+
 #include "kernels.h"
 
 namespace gi {
-bool pointwise_tc_supported(int, int) { return false; }
-void pointwise_tc_pack(const float*, const float*, int, int, std::vector<uint8_t>*, LaunchRec*) {}
-int launch_pointwise_tc(const LaunchRec&, const Ptrs&, void**, int, void*) { return 1; }
-void pointwise_tc_release(void*) {}
+namespace {
+
+constexpr int kTileRows = 128;               // pixel pairs (TMEM lanes) per tile
+constexpr int kTilePx = 2 * kTileRows;       // pixels per tile
+constexpr int kSliceBytes = kTileRows * 16;  // one input slice of a tile in shared memory
+constexpr int kCoreBytes = 128;              // one 8x8 fp16 core matrix
+constexpr int kMaxStages = 8;
+constexpr int kMaxNts = 32;                  // output slices per tile: 32 * 8 = 256 accumulator columns
+constexpr int kSmemHeader = 1024;            // barriers, TMEM address, abort flag
+constexpr int kSmemBudget = 200 * 1024;
+constexpr int kThreads = 192;
+
+__device__ unsigned int g_tc_error = 0;  // sticky: non-zero once any wait in this module timed out
+
+struct TcParams {
+  const __half* res;
+  __half* out;
+  const float* bias;
+  const unsigned char* wts;
+  unsigned int m_total_px;  // batch * pixels per stored plane (even)
+  int s_out;                // real output slices
+  int nts, n_tiles;         // output slices per tile (even), number of such tiles
+  int kc, k_chunks;         // input slices per pipeline stage (even), stages per tile
+  int stages;
+  int m_tiles, groups;      // pixel tiles; each pixel tile is split over `groups` CTAs along n_tiles
+  int act_pre, has_res, act_post;
+  unsigned int tmem_cols;   // power of two >= 2 * nts * 8
+  unsigned int timeout_ns;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait.  Returns false if the CTA is aborting or the limit ran out (then it raises the
+// abort flag and the error word itself).
+__device__ __noinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile unsigned* abort_flag, unsigned timeout_ns,
+                                       unsigned code) {
+  unsigned long long t0 = 0;
+  for (unsigned spin = 0;; ++spin) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((spin & 255u) == 255u) {
+      if (*abort_flag) return false;
+      const unsigned long long now = global_timer_ns();
+      if (t0 == 0) {
+        t0 = now;
+      } else if (now - t0 > timeout_ns) {
+        *abort_flag = 1;
+        atomicOr(&g_tc_error, code);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(unsigned dst, const CUtensorMap* map, int x, int y, unsigned bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+               "l"(reinterpret_cast<unsigned long long>(map)), "r"(x), "r"(y), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_load(unsigned dst, const void* src, unsigned bytes, unsigned bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src),
+               "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(unsigned smem_dst, unsigned cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(unsigned taddr, unsigned cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem]^T, 128 x N x 16, fp16 operands, fp32 accumulate
+__device__ __forceinline__ void umma_f16(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc, unsigned idesc,
+                                         unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrive on an mbarrier once every MMA issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(unsigned bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// Shared-memory operand descriptor: K-major, no swizzle.  Core matrices are 8 rows x 16 bytes,
+// stored as 128 contiguous bytes; `lbo` is the byte distance between the two core matrices
+// an MMA reads along K, `sbo` the distance between consecutive 8-row groups.
+__device__ __forceinline__ unsigned long long smem_desc(unsigned addr, unsigned lbo, unsigned sbo) {
+  unsigned long long d = 0;
+  d |= static_cast<unsigned long long>((addr & 0x3ffffu) >> 4);
+  d |= static_cast<unsigned long long>((lbo >> 4) & 0x3fffu) << 16;
+  d |= static_cast<unsigned long long>((sbo >> 4) & 0x3fffu) << 32;
+  d |= 1ull << 46;  // descriptor version of this architecture
+  return d;         // base offset 0, layout type 0 (no swizzle)
+}
+
+// 32 lanes x 8 consecutive 32-bit columns: thread t of the warp receives lane (quarter*32 + t)
+__device__ __forceinline__ void tmem_ld8(unsigned taddr, unsigned* r) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr)
+               : "memory");
+}
+// wait for the loads above; the registers are operands so that no use can move above the wait
+__device__ __forceinline__ void tmem_ld_wait(unsigned* r) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                 "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]),
+                 "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),
+                 "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
+}
+
+__device__ __forceinline__ float act1(float v, int kind) {
+  if (kind == GI_ACT_RELU) return fmaxf(v, 0.0f);
+  if (kind == GI_ACT_RELU6) return fminf(fmaxf(v, 0.0f), 6.0f);
+  return v;
+}
+
+struct SmemHeader {
+  unsigned long long full[kMaxStages];
+  unsigned long long empty[kMaxStages];
+  unsigned long long acc_full[2];
+  unsigned long long acc_empty[2];
+  unsigned tmem_addr;
+  unsigned abort_flag;
+};
+static_assert(sizeof(SmemHeader) <= kSmemHeader, "header too large");
+
+enum : unsigned { kErrProducer = 1u, kErrMma = 2u, kErrEpilogue = 4u, kErrDrain = 8u };
+
+__global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const TcParams p) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  SmemHeader* hdr = reinterpret_cast<SmemHeader*>(smem);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned stage_a_bytes = static_cast<unsigned>(p.kc) * kSliceBytes;
+  const unsigned stage_b_bytes = static_cast<unsigned>(p.kc) * p.nts * kCoreBytes;
+  const unsigned stage_bytes = stage_a_bytes + stage_b_bytes;
+  const unsigned data0 = smem_u32(smem + kSmemHeader);
+  volatile unsigned* abort_flag = &hdr->abort_flag;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < p.stages; ++i) {
+      mbar_init(smem_u32(&hdr->full[i]), 1);
+      mbar_init(smem_u32(&hdr->empty[i]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&hdr->acc_full[i]), 1);
+      mbar_init(smem_u32(&hdr->acc_empty[i]), 4);
+    }
+    hdr->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32(&hdr->tmem_addr), p.tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const unsigned tmem_base = hdr->tmem_addr;
+  const int n_units = p.m_tiles * p.groups;
+  const unsigned acc_cols = static_cast<unsigned>(p.nts) * 8u;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      unsigned it = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+        const int m_tile = u / p.groups, grp = u - m_tile * p.groups;
+        for (int nt = grp; nt < p.n_tiles && ok; nt += p.groups) {
+          for (int kc_i = 0; kc_i < p.k_chunks; ++kc_i, ++it) {
+            const unsigned stage = it % p.stages, phase = (it / p.stages) & 1u;
+            if (!mbar_wait(smem_u32(&hdr->empty[stage]), phase ^ 1u, abort_flag, p.timeout_ns, kErrProducer)) {
+              ok = false;
+              break;
+            }
+            const unsigned full = smem_u32(&hdr->full[stage]);
+            mbar_expect_tx(full, stage_bytes);
+            const unsigned dst = data0 + stage * stage_bytes;
+            // pixels outside the tensor and slices beyond the last one arrive as zeros
+            tma_load_2d(dst, &tmap_a, m_tile * kTilePx, kc_i * p.kc, full);
+            bulk_load(dst + stage_a_bytes, p.wts + (static_cast<size_t>(nt) * p.k_chunks + kc_i) * stage_b_bytes, stage_b_bytes,
+                      full);
+          }
+        }
+      }
+      if (!ok) {
+        // copies already issued still land in shared memory: wait for them (bounded) before leaving
+        const unsigned first = it > static_cast<unsigned>(p.stages) ? it - p.stages : 0u;
+        for (unsigned j = first; j < it; ++j) {
+          unsigned long long t0 = global_timer_ns();
+          while (!mbar_try_wait(smem_u32(&hdr->full[j % p.stages]), (j / p.stages) & 1u)) {
+            if (global_timer_ns() - t0 > p.timeout_ns) {
+              atomicOr(&g_tc_error, kErrDrain);
+              break;
+            }
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      // instruction descriptor: fp32 accumulator, fp16 A and B, both K-major, M = 128, N = nts * 8
+      const unsigned idesc = (1u << 4) | ((acc_cols >> 3) << 17) | ((kTileRows >> 4) << 24);
+      const unsigned b_lbo = static_cast<unsigned>(p.nts) * kCoreBytes;
+      unsigned it = 0, tile = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+        const int m_tile = u / p.groups, grp = u - m_tile * p.groups;
+        for (int nt = grp; nt < p.n_tiles && ok; nt += p.groups, ++tile) {
+          const unsigned acc = tile & 1u, acc_phase = (tile >> 1) & 1u;
+          if (!mbar_wait(smem_u32(&hdr->acc_empty[acc]), acc_phase ^ 1u, abort_flag, p.timeout_ns, kErrMma)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const unsigned d_tmem = tmem_base + acc * acc_cols;
+          for (int kc_i = 0; kc_i < p.k_chunks; ++kc_i, ++it) {
+            const unsigned stage = it % p.stages, phase = (it / p.stages) & 1u;
+            if (!mbar_wait(smem_u32(&hdr->full[stage]), phase, abort_flag, p.timeout_ns, kErrMma)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after();
+            const unsigned a_base = data0 + stage * stage_bytes, b_base = a_base + stage_a_bytes;
+            for (int ks = 0; ks < p.kc / 2; ++ks) {
+              const unsigned long long ad = smem_desc(a_base + ks * 2 * kSliceBytes, kSliceBytes, kCoreBytes);
+              const unsigned long long bd = smem_desc(b_base + ks * 2 * b_lbo, b_lbo, kCoreBytes);
+              umma_f16(d_tmem, ad, bd, idesc, (kc_i > 0 || ks > 0) ? 1u : 0u);
+            }
+            umma_commit(smem_u32(&hdr->empty[stage]));  // the stage is free once these MMAs have read it
+          }
+          if (ok) umma_commit(smem_u32(&hdr->acc_full[acc]));
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5)
+    const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32) belong to this warp
+    const unsigned rows_total = p.m_total_px >> 1;
+    unsigned tile = 0;
+    bool ok = true;
+    for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+      const int m_tile = u / p.groups, grp = u - m_tile * p.groups;
+      const unsigned row = static_cast<unsigned>(m_tile) * kTileRows + quarter * 32 + lane;
+      const bool row_ok = row < rows_total;
+      for (int nt = grp; nt < p.n_tiles && ok; nt += p.groups, ++tile) {
+        const unsigned acc = tile & 1u, acc_phase = (tile >> 1) & 1u;
+        if (!mbar_wait(smem_u32(&hdr->acc_full[acc]), acc_phase, abort_flag, p.timeout_ns, kErrEpilogue)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        const unsigned t_addr = tmem_base + acc * acc_cols + (static_cast<unsigned>(quarter * 32) << 16);
+        for (int so_l = 0; so_l < p.nts; so_l += 4) {
+          unsigned r[32];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            // columns past this tile's accumulator are never read: clamp to the last valid slice
+            const int s = min(so_l + j, p.nts - 1);
+            tmem_ld8(t_addr + static_cast<unsigned>(s) * 8u, r + 8 * j);
+          }
+          tmem_ld_wait(r);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int so = nt * p.nts + so_l + j;
+            if (so_l + j >= p.nts || so >= p.s_out || !row_ok) continue;
+            const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias) + so);
+            float v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[8 * j + i]);
+            v[0] += b.x; v[1] += b.y; v[2] += b.z; v[3] += b.w;
+            v[4] += b.x; v[5] += b.y; v[6] += b.z; v[7] += b.w;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = act1(v[i], p.act_pre);
+            const size_t off = (static_cast<size_t>(so) * p.m_total_px + 2u * row) * 4u;  // in halves
+            if (p.has_res) {
+              const uint4 rr = __ldg(reinterpret_cast<const uint4*>(p.res + off));
+              const __half2* rh = reinterpret_cast<const __half2*>(&rr);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const float2 f = __half22float2(rh[i]);
+                v[2 * i] += f.x;
+                v[2 * i + 1] += f.y;
+              }
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = act1(v[i], p.act_post);
+            uint4 o;
+            __half2* oh = reinterpret_cast<__half2*>(&o);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) oh[i] = __floats2half2_rn(v[2 * i], v[2 * i + 1]);
+            *reinterpret_cast<uint4*>(p.out + off) = o;
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&hdr->acc_empty[acc]));
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, p.tmem_cols);
+  }
+}
+
+// ------------------------------------------------------------------ host side
+struct Tiling {
+  int s_in, s_out, kc, k_chunks, nts, n_tiles, stages;
+};
+
+Tiling choose_tiling(int cin, int cout) {
+  Tiling t;
+  t.s_in = slices(cin);
+  t.s_out = slices(cout);
+  const int s_in_even = (t.s_in + 1) / 2 * 2;
+  t.kc = s_in_even < 8 ? s_in_even : 8;
+  t.k_chunks = (s_in_even + t.kc - 1) / t.kc;
+  t.n_tiles = (t.s_out + kMaxNts - 1) / kMaxNts;
+  t.nts = (t.s_out + t.n_tiles - 1) / t.n_tiles;
+  t.nts = (t.nts + 1) / 2 * 2;  // N = nts * 8 must be a multiple of 16
+  const int stage_bytes = t.kc * (kSliceBytes + t.nts * kCoreBytes);
+  t.stages = kSmemBudget / stage_bytes;
+  if (t.stages > kMaxStages) t.stages = kMaxStages;
+  if (t.stages < 2) t.stages = 2;
+  return t;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(f);
+  });
+  return fn;
+}
+
+struct MapEntry {
+  const void* in = nullptr;
+  CUtensorMap map;
+};
+struct TcState {
+  std::vector<MapEntry> maps;
+};
+
+struct DeviceInfo {
+  int sms = 0;
+  bool attr_set = false;
+};
+DeviceInfo& device_info() {
+  static DeviceInfo info[64];
+  int dev = 0;
+  cudaGetDevice(&dev);
+  return info[dev & 63];
+}
+
+}  // namespace
+
+bool pointwise_tc_supported(int cin, int cout) { return cin > 0 && cout > 0; }
+
+// Expanded weights, per (output tile, K chunk): [kc input slices][nts output slices][8 rows x 8 halves],
+// row = parity' * 4 + output channel in slice, column = parity * 4 + input channel in slice.
+void pointwise_tc_pack(const float* w, const float* bias, int cin, int cout, std::vector<uint8_t>* blob, LaunchRec* r) {
+  const Tiling t = choose_tiling(cin, cout);
+  const size_t chunk_bytes = static_cast<size_t>(t.kc) * t.nts * kCoreBytes;
+  const size_t wbytes = static_cast<size_t>(t.n_tiles) * t.k_chunks * chunk_bytes;
+  const uint64_t woff = round_up_u64(blob->size(), 256);
+  blob->resize(woff + wbytes, 0);
+  const uint64_t boff = round_up_u64(blob->size(), 256);
+  blob->resize(boff + static_cast<size_t>(t.n_tiles) * t.nts * 4 * sizeof(float), 0);
+  uint16_t* wp = reinterpret_cast<uint16_t*>(blob->data() + woff);
+  float* bp = reinterpret_cast<float*>(blob->data() + boff);
+  for (int nt = 0; nt < t.n_tiles; ++nt)
+    for (int kc_i = 0; kc_i < t.k_chunks; ++kc_i)
+      for (int sl = 0; sl < t.kc; ++sl)
+        for (int ol = 0; ol < t.nts; ++ol) {
+          const int s = kc_i * t.kc + sl, so = nt * t.nts + ol;
+          uint16_t* core = wp + ((static_cast<size_t>(nt) * t.k_chunks + kc_i) * chunk_bytes +
+                                 (static_cast<size_t>(sl) * t.nts + ol) * kCoreBytes) / 2;
+          if (s >= t.s_in || so >= t.s_out) continue;
+          for (int j = 0; j < 4; ++j) {
+            const int co = so * 4 + j;
+            if (co >= cout) continue;
+            for (int c = 0; c < 4; ++c) {
+              const int ci = s * 4 + c;
+              if (ci >= cin) continue;
+              const uint16_t h = f32_to_f16_rne(w[static_cast<size_t>(co) * cin + ci]);
+              core[(0 * 4 + j) * 8 + 0 * 4 + c] = h;  // parity 0 block
+              core[(1 * 4 + j) * 8 + 1 * 4 + c] = h;  // parity 1 block
+            }
+          }
+        }
+  for (int co = 0; co < cout; ++co) bp[co] = bias[co];
+  r->wts = Loc{W_WEIGHTS, 0, woff};
+  r->bias = Loc{W_WEIGHTS, 0, boff};
+  r->wts_bytes = wbytes;
+  r->tc_nt = t.nts;
+  r->tc_kc = t.kc;
+  r->tc_stages = t.stages;
+}
+
+int launch_pointwise_tc(const LaunchRec& r, const Ptrs& p, void** state, int launch_index, void* stream) {
+  const Tiling t = choose_tiling(r.C, r.Co);
+  const unsigned m_total = static_cast<unsigned>(r.B) * static_cast<unsigned>(plane_pixels(r.H, r.W));
+  DeviceInfo& di = device_info();
+  if (di.sms == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&di.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || di.sms <= 0)
+      return static_cast<int>(cudaErrorInvalidDevice);
+  }
+  if (!di.attr_set) {
+    const cudaError_t e = cudaFuncSetAttribute(pointwise_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               kSmemHeader + kSmemBudget);
+    if (e != cudaSuccess) return static_cast<int>(e);
+    di.attr_set = true;
+  }
+  // tensor map over the input: pixels (8-byte elements) x slices; cached per launch and input address
+  if (!*state) *state = new TcState();
+  TcState* st = static_cast<TcState*>(*state);
+  if (st->maps.size() <= static_cast<size_t>(launch_index)) st->maps.resize(launch_index + 1);
+  MapEntry& me = st->maps[launch_index];
+  if (me.in != p.in0) {
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return static_cast<int>(cudaErrorNotSupported);
+    const cuuint64_t gdim[2] = {m_total, static_cast<cuuint64_t>(t.s_in)};
+    const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(m_total) * 8u};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(kTilePx), static_cast<cuuint32_t>(t.kc)};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult cr = enc(&me.map, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void*>(p.in0), gdim, gstride, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) return static_cast<int>(cudaErrorInvalidValue);
+    me.in = p.in0;
+  }
+  TcParams k;
+  k.res = static_cast<const __half*>(p.res);
+  k.out = static_cast<__half*>(p.out);
+  k.bias = static_cast<const float*>(p.bias);
+  k.wts = static_cast<const unsigned char*>(p.wts);
+  k.m_total_px = m_total;
+  k.s_out = t.s_out;
+  k.nts = t.nts;
+  k.n_tiles = t.n_tiles;
+  k.kc = t.kc;
+  k.k_chunks = t.k_chunks;
+  k.stages = t.stages;
+  k.m_tiles = static_cast<int>((m_total / 2 + kTileRows - 1) / kTileRows);
+  int groups = (di.sms + k.m_tiles - 1) / k.m_tiles;
+  if (groups > t.n_tiles) groups = t.n_tiles;
+  if (groups < 1) groups = 1;
+  k.groups = groups;
+  k.act_pre = r.ep.act_pre;
+  k.has_res = r.ep.has_res;
+  k.act_post = r.ep.act_post;
+  unsigned cols = 32;
+  while (cols < static_cast<unsigned>(2 * t.nts * 8)) cols <<= 1;
+  k.tmem_cols = cols;
+  k.timeout_ns = 1000000000u;
+  const long long units = static_cast<long long>(k.m_tiles) * groups;
+  const unsigned grid = static_cast<unsigned>(units < di.sms ? units : di.sms);
+  const size_t smem = kSmemHeader + static_cast<size_t>(t.stages) * t.kc * (kSliceBytes + t.nts * kCoreBytes);
+  pointwise_tc_kernel<<<grid, kThreads, smem, static_cast<cudaStream_t>(stream)>>>(me.map, k);
+  return static_cast<int>(cudaGetLastError());
+}
+
+void pointwise_tc_release(void* state) { delete static_cast<TcState*>(state); }
+
+unsigned int pointwise_tc_error_word(int* cuda_err) {
+  unsigned int v = 0;
+  const cudaError_t e = cudaMemcpyFromSymbol(&v, g_tc_error, sizeof v);
+  if (cuda_err) *cuda_err = static_cast<int>(e);
+  return v;
+}
+
 }  // namespace gi

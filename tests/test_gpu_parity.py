@@ -91,7 +91,12 @@ PW_CASES = [  # batch, hw, cin, cout, residual, act
 @pytest.mark.parametrize("case", PW_CASES)
 def test_pointwise(storage, case):
     batch, hw, cin, cout, residual, act = case
-    check_all_tensors(wl.single_pointwise(batch, hw, cin, cout, residual, act), storage)
+    spec = wl.single_pointwise(batch, hw, cin, cout, residual, act)
+    check_all_tensors(spec, storage)
+    # fp16 storage must take the tensor-core kernel, fp32 storage the CUDA-core one
+    kernels = [api.KERNEL_NAMES[o.kernel] for o in api.graph_from_spec(spec, storage)[0].compile().ops()]
+    assert ("pointwise_tc" in kernels) == (storage == api.GI_F16)
+    assert api.gi_device_status() == 0
 
 
 @pytest.mark.parametrize("case", PW_CASES[:6])
