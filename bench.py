@@ -143,6 +143,75 @@ def run_reference(args, spec_fn, label):
     print(json.dumps(line), flush=True)
 
 
+def run_sweep(args):
+    """Single fused operators (1x1 convolution, 3x3 depthwise) with PHWC4 buffers in and out, so
+    one kernel runs per call.  Each point is timed with a CUDA event pair per iteration on the run
+    stream, the L2 flushed by an untimed memset in between; prints one JSON line per point."""
+    import torch
+    from paper_1907_01989_b200 import api
+    from paper_1907_01989_b200 import workloads as wl
+    peaks, peak_kind = load_peaks()
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+    if args.points:
+        points = [tuple(int(v) for v in pt.split(",")) for pt in args.points.split(";") if pt]
+    elif args.sweep == "dw":
+        points = [(b, hw, c, s) for b in (64, 256) for hw, c in ((112, 32), (112, 96), (56, 144), (28, 192), (14, 384),
+                                                                 (14, 576), (7, 960)) for s in (1, 2)]
+    else:
+        points = [(256, 112, 16, 96), (256, 112, 32, 16), (256, 56, 24, 144), (256, 56, 144, 24), (256, 28, 32, 192),
+                  (256, 28, 192, 32), (256, 14, 64, 384), (256, 14, 384, 64), (256, 14, 96, 576), (256, 14, 576, 96),
+                  (256, 7, 160, 960), (256, 7, 960, 160), (256, 7, 320, 1280), (256, 14, 576, 576), (256, 14, 960, 960),
+                  (256, 14, 1280, 1280), (64, 56, 192, 192), (8, 28, 384, 384), (1, 14, 96, 576)]
+    rows = []
+    for pt in points:
+        if args.sweep == "dw":
+            b, hw, c, stride = pt
+            spec = wl.single_depthwise(b, hw, c, stride, 1, residual=args.residual)
+            name = f"dw3x3 b{b} {hw}x{hw}x{c} s{stride}"
+        else:
+            b, hw, cin, cout = pt
+            spec = wl.single_pointwise(b, hw, cin, cout, residual=args.residual)
+            name = f"pw1x1 b{b} {hw}x{hw} {cin}->{cout}"
+        g, _ = api.graph_from_spec(spec, api.GI_F16, io_layout=api.GI_PHWC4)
+        ex = g.compile()
+        ex.bind(dev)
+        ops = ex.ops()
+        assert len(ops) == 1
+        ins = [(torch.rand(api.gi_tensor_bytes(b, *spec.shapes[t]) // 2, device=dev) * 2 - 1).half() for t in spec.inputs]
+        outs = [torch.empty(api.gi_tensor_bytes(b, *spec.shapes[t]) // 2, dtype=torch.float16, device=dev)
+                for t in spec.outputs]
+        for _ in range(3):
+            ex.run(ins, outs, stream)
+        ms = []
+        for _ in range(args.iters):
+            flush.zero_()
+            a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            ex.run(ins, outs, stream)
+            z.record(stream)
+            z.synchronize()
+            ms.append(a.elapsed_time(z))
+        t = statistics.median(ms)
+        o = ops[0]
+        t_hbm = o.bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
+        t_tc = o.flops / (peaks["bf16_tflops"] * 1e12) * 1e3
+        row = {"op": name, "kernel": api.KERNEL_NAMES[o.kernel], "ms": round(t, 5), "bytes": int(o.bytes),
+               "flops": int(o.flops), "gbs": round(o.bytes / t / 1e6, 1), "tflops": round(o.flops / t / 1e9, 2),
+               "bound": "tensor" if t_tc > t_hbm else "hbm", "frac_of_roofline": round(max(t_hbm, t_tc) / t, 4),
+               "peak_source": peak_kind}
+        rows.append(row)
+        print(json.dumps(row), flush=True)
+    if args.out:
+        with open(args.out, "w") as fh:
+            fh.write("# op | kernel | ms | GB/s | TFLOP/s | bound | fraction of roofline (burst peaks, %s)\n" % peak_kind)
+            for r in rows:
+                fh.write(f"{r['op']} | {r['kernel']} | {r['ms']} | {r['gbs']} | {r['tflops']} | {r['bound']} | "
+                         f"{r['frac_of_roofline']}\n")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -154,11 +223,19 @@ def main():
     ap.add_argument("--pointwise", default="auto", choices=["auto", "simt"])
     ap.add_argument("--per-op", default=None, help="write the per-op timing table to this file")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", default=None, choices=["pw", "dw"], help="time single fused operators instead of a network")
+    ap.add_argument("--points", default=None, help="sweep points 'B,HW,Cin,Cout;...' (pw) or 'B,HW,C,stride;...' (dw)")
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--residual", action="store_true")
+    ap.add_argument("--out", default=None)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.batch is None:
         args.batch = 16 if args.net == "seg" else 256
 
+    if args.sweep:
+        run_sweep(args)
+        return
     from paper_1907_01989_b200 import workloads as wl
     fn_name, label = NETS[args.net]
     spec_fn = getattr(wl, fn_name)

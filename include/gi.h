@@ -224,7 +224,8 @@ GI_API gi_status gi_run_timed(gi_exec* e, const void* const* dev_inputs, void* c
 
 /* Health word of the device-side waits.  The tensor-core kernel waits on copy and MMA
  * completion with a limit of about one second per wait; a wait that runs out sets a bit here
- * (1 producer, 2 MMA issuer, 4 epilogue, 8 drain), lets the kernel finish without its results
+ * (1 producer, 2 MMA issuer, 4 epilogue, 8 drain; 0x10000 depthwise staging copy), lets the
+ * kernel finish without its results
  * and leaves the CUDA context usable.  Sticky until the process exits.  Synchronous: copies
  * the word from the current device. */
 GI_API gi_status gi_device_status(uint32_t* flags);

@@ -100,6 +100,7 @@ gi_status gi_device_status(uint32_t* flags) {
   if (!flags) return fail(GI_E_INVALID, "gi_device_status: null argument");
   int err = 0;
   *flags = pointwise_tc_error_word(&err);
+  if (err == 0) *flags |= depthwise_error_word(&err) << 16;
   if (err != 0) return fail(GI_E_CUDA, std::string("gi_device_status: ") + cudaGetErrorString(static_cast<cudaError_t>(err)));
   return GI_OK;
 }

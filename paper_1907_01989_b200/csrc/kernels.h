@@ -22,6 +22,9 @@ int launch_pack(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
 int launch_unpack(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
 int launch_conv_simt(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
 int launch_depthwise(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
+// fp16 storage, equal strides / dilations on both axes: shared-memory staged stencil
+int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream);
+unsigned int depthwise_error_word(int* cuda_err);
 int launch_eltwise(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
 int launch_pool(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
 int launch_resize(const LaunchRec& r, const Ptrs& p, int storage, void* stream);

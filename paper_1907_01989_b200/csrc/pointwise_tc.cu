@@ -15,8 +15,9 @@
 // bound by HBM bandwidth, not by the tensor pipe, so the pipe has the slack.
 //
 // One CTA per SM, persistent over (pixel tile, output-channel tile) units; warp 0 issues TMA,
-// warp 1 issues MMAs and owns tensor memory, warps 2-5 run the epilogue (one TMEM lane quarter
-// each).  Accumulators are double-buffered so the epilogue of a tile overlaps the next tile's
+// warp 1 issues MMAs and owns tensor memory, warps 2-17 run the epilogue: four warps per TMEM
+// lane quarter, each taking every fourth 16-column chunk and loading the next chunk from tensor
+// memory while it converts and stores the current one.  Accumulators are double-buffered so the epilogue of a tile overlaps the next tile's
 // loads and MMAs.  Every wait is bounded: after about a second it raises an error word the
 // host can read, drains the copies in flight and leaves, so the context stays usable.
 #include <cuda.h>
@@ -40,7 +41,9 @@ constexpr int kMaxStages = 8;
 constexpr int kMaxNts = 32;                  // output slices per tile: 32 * 8 = 256 accumulator columns
 constexpr int kSmemHeader = 1024;            // barriers, TMEM address, abort flag
 constexpr int kSmemBudget = 200 * 1024;
-constexpr int kThreads = 192;
+constexpr int kEpiWarpsPerQuarter = 4;       // epilogue warps sharing one TMEM lane quarter
+constexpr int kEpiWarps = 4 * kEpiWarpsPerQuarter;
+constexpr int kThreads = 64 + 32 * kEpiWarps;
 
 __device__ unsigned int g_tc_error = 0;  // sticky: non-zero once any wait in this module timed out
 
@@ -159,20 +162,21 @@ __device__ __forceinline__ unsigned long long smem_desc(unsigned addr, unsigned 
   return d;         // base offset 0, layout type 0 (no swizzle)
 }
 
-// 32 lanes x 8 consecutive 32-bit columns: thread t of the warp receives lane (quarter*32 + t)
-__device__ __forceinline__ void tmem_ld8(unsigned taddr, unsigned* r) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-               : "r"(taddr)
-               : "memory");
+// 32 lanes x 16 consecutive 32-bit columns: thread t of the warp receives lane (quarter*32 + t)
+__device__ __forceinline__ void tmem_ld16(unsigned taddr, unsigned* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
 }
-// wait for the loads above; the registers are operands so that no use can move above the wait
-__device__ __forceinline__ void tmem_ld_wait(unsigned* r) {
+// wait for every tensor-memory load issued so far; the registers of the chunk about to be used
+// are operands so that no use of them can be scheduled above the wait
+__device__ __forceinline__ void tmem_ld_wait16(unsigned* r) {
   asm volatile("tcgen05.wait::ld.sync.aligned;"
                : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
-                 "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]),
-                 "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),
-                 "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
                :
                : "memory");
 }
@@ -212,7 +216,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&hdr->acc_full[i]), 1);
-      mbar_init(smem_u32(&hdr->acc_empty[i]), 4);
+      mbar_init(smem_u32(&hdr->acc_empty[i]), kEpiWarps);
     }
     hdr->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -302,9 +306,11 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------ epilogue (warps 2..17)
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32) belong to this warp
+    const int sub = (warp - 2) >> 2;
     const unsigned rows_total = p.m_total_px >> 1;
+    const int n_chunks = p.nts >> 1;  // 2 output slices = 16 accumulator columns per chunk
     unsigned tile = 0;
     bool ok = true;
     for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
@@ -319,25 +325,23 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
         }
         tc_fence_after();
         const unsigned t_addr = tmem_base + acc * acc_cols + (static_cast<unsigned>(quarter * 32) << 16);
-        for (int so_l = 0; so_l < p.nts; so_l += 4) {
-          unsigned r[32];
+        const float4* bias4 = reinterpret_cast<const float4*>(p.bias) + static_cast<size_t>(nt) * p.nts;
+
+        auto issue = [&](unsigned* r, float4* b, int c) {
+          tmem_ld16(t_addr + static_cast<unsigned>(c) * 16u, r);
+          b[0] = __ldg(bias4 + 2 * c);
+          b[1] = __ldg(bias4 + 2 * c + 1);
+        };
+        auto finish = [&](const unsigned* r, const float4* b, int c) {
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            // columns past this tile's accumulator are never read: clamp to the last valid slice
-            const int s = min(so_l + j, p.nts - 1);
-            tmem_ld8(t_addr + static_cast<unsigned>(s) * 8u, r + 8 * j);
-          }
-          tmem_ld_wait(r);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int so = nt * p.nts + so_l + j;
-            if (so_l + j >= p.nts || so >= p.s_out || !row_ok) continue;
-            const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias) + so);
+          for (int j = 0; j < 2; ++j) {
+            const int so = nt * p.nts + 2 * c + j;
+            if (so >= p.s_out || !row_ok) continue;
             float v[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[8 * j + i]);
-            v[0] += b.x; v[1] += b.y; v[2] += b.z; v[3] += b.w;
-            v[4] += b.x; v[5] += b.y; v[6] += b.z; v[7] += b.w;
+            v[0] += b[j].x; v[1] += b[j].y; v[2] += b[j].z; v[3] += b[j].w;
+            v[4] += b[j].x; v[5] += b[j].y; v[6] += b[j].z; v[7] += b[j].w;
 #pragma unroll
             for (int i = 0; i < 8; ++i) v[i] = act1(v[i], p.act_pre);
             const size_t off = (static_cast<size_t>(so) * p.m_total_px + 2u * row) * 4u;  // in halves
@@ -358,6 +362,22 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
 #pragma unroll
             for (int i = 0; i < 4; ++i) oh[i] = __floats2half2_rn(v[2 * i], v[2 * i + 1]);
             *reinterpret_cast<uint4*>(p.out + off) = o;
+          }
+        };
+
+        unsigned ra[16], rb[16];
+        float4 ba[2], bb[2];
+        int c = sub;
+        if (c < n_chunks) issue(ra, ba, c);
+        for (; c < n_chunks; c += 2 * kEpiWarpsPerQuarter) {
+          const int c1 = c + kEpiWarpsPerQuarter, c2 = c + 2 * kEpiWarpsPerQuarter;
+          tmem_ld_wait16(ra);
+          if (c1 < n_chunks) issue(rb, bb, c1);
+          finish(ra, ba, c);
+          if (c1 < n_chunks) {
+            tmem_ld_wait16(rb);
+            if (c2 < n_chunks) issue(ra, ba, c2);
+            finish(rb, bb, c1);
           }
         }
         tc_fence_before();
@@ -526,9 +546,18 @@ int launch_pointwise_tc(const LaunchRec& r, const Ptrs& p, void** state, int lau
   k.k_chunks = t.k_chunks;
   k.stages = t.stages;
   k.m_tiles = static_cast<int>((m_total / 2 + kTileRows - 1) / kTileRows);
-  int groups = (di.sms + k.m_tiles - 1) / k.m_tiles;
-  if (groups > t.n_tiles) groups = t.n_tiles;
-  if (groups < 1) groups = 1;
+  // split the output tiles of one pixel tile over `groups` CTAs so that the busiest SM runs
+  // as few tiles as possible; ties go to fewer groups (the input tile is then re-read less)
+  int groups = 1;
+  long long best_rounds = -1;
+  for (int g = 1; g <= t.n_tiles; ++g) {
+    const long long units_g = static_cast<long long>(k.m_tiles) * g;
+    const long long rounds = ((units_g + di.sms - 1) / di.sms) * ((t.n_tiles + g - 1) / g);
+    if (best_rounds < 0 || rounds < best_rounds) {
+      best_rounds = rounds;
+      groups = g;
+    }
+  }
   k.groups = groups;
   k.act_pre = r.ep.act_pre;
   k.has_res = r.ep.has_res;
