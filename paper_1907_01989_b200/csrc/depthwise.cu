@@ -1,13 +1,15 @@
 // Depthwise 3x3 convolution for fp16 storage: a bandwidth-bound stencil.
 //
-// A CTA owns a band of output rows in a few planes (plane = one 4-channel slice of one image;
-// the planes of one slice are adjacent in memory, so they share the slice's 36 weights).  The
-// input rows the band needs - its halo included - are one contiguous run per plane and are staged
-// into shared memory by bulk asynchronous copies (16-byte aligned, one mbarrier).  Each thread then
-// walks down one output column, keeping a sliding window of input rows in registers, so every
-// input pixel-slice is read from HBM once, from shared memory three times, and is converted to
-// fp32 once per use; stores are 8 bytes per lane, contiguous across the warp.  Zero padding is
-// applied by predicates while the rows are fetched from shared memory.
+// A work item is a band of output rows in a few planes (plane = one 4-channel slice of one
+// image; the planes of one slice are adjacent in memory, so they share the slice's 36 weights).
+// The input rows a band needs - its halo included - are one contiguous run per plane and are
+// staged into shared memory by bulk asynchronous copies (16-byte aligned, one mbarrier per
+// buffer).  CTAs are persistent over a contiguous range of items and double-buffer the staging:
+// the copy for the next item is in flight while the current one is computed.  Each thread walks
+// down one output column; every input row it reads feeds three running accumulators (packed
+// two-wide fp32 FMAs), so an input pixel-slice is read from HBM once and from shared memory
+// three times; stores are 8 bytes per lane, contiguous across the warp.  Zero padding is applied
+// by predicates while the rows are fetched from shared memory.
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
@@ -21,23 +23,17 @@ __device__ unsigned int g_dw_error = 0;  // sticky: set if the staging copy did 
 struct DwGeom {
   int B, H, W, Pin, Ho, Wo, Pout, S;
   int stride, dil, pt, pl;
-  int nb;       // planes per CTA
-  int sub;      // sub-bands per CTA band (thread groups walking different rows of one plane)
+  int nb;       // planes per work item
+  int sub;      // sub-bands per band (thread groups walking different rows of one plane)
   int tr;       // output rows walked by one thread
-  int bands;    // CTA bands per plane
+  int bands;    // bands per plane
   int bchunks;  // ceil(B / nb)
-  int plane_stride_px;  // pixels reserved per plane in shared memory (even)
+  int plane_stride_px;  // pixels reserved per plane in one staging buffer (even)
+  int items;            // S * bchunks * bands
   unsigned timeout_ns;
 };
 
 __device__ __forceinline__ unsigned smem_u32(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ float4 ld_px(const __half* p) {
-  const uint2 u = *reinterpret_cast<const uint2*>(p);
-  const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&u.x));
-  const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&u.y));
-  return make_float4(a.x, a.y, b.x, b.y);
-}
 
 __device__ __forceinline__ float act1(float v, int kind) {
   if (kind == GI_ACT_RELU) return fmaxf(v, 0.0f);
@@ -45,166 +41,260 @@ __device__ __forceinline__ float act1(float v, int kind) {
   return v;
 }
 
-__device__ __forceinline__ void fma4(float4& acc, const float4& x, const float4& w) {
-  acc.x = fmaf(x.x, w.x, acc.x);
-  acc.y = fmaf(x.y, w.y, acc.y);
-  acc.z = fmaf(x.z, w.z, acc.z);
-  acc.w = fmaf(x.w, w.w, acc.w);
-}
-
+// three taps of one input row, 4 channels each, as packed pairs for the two-wide fp32 FMA
 struct Row {
-  float4 v[3];
+  float2 lo[3], hi[3];
+};
+struct Acc {
+  float2 lo, hi;
 };
 
-// MODE 0: stride 1, dilation 1 (one new input row per output row)
-// MODE 1: stride 2, dilation 1 (two new input rows per output row)
-// MODE 2: anything else (three rows fetched per output row)
-template <int MODE>
-__global__ void __launch_bounds__(512) depthwise_f16_kernel(const __half* __restrict__ in, const float* __restrict__ w,
-                                                             const float* __restrict__ bias, const __half* __restrict__ res,
-                                                             __half* __restrict__ out, const DwGeom g, const Epilogue ep) {
+__device__ __forceinline__ void fma_row(Acc& a, const Row& r, const float2* wlo, const float2* whi) {
+#pragma unroll
+  for (int k = 0; k < 3; ++k) {
+    a.lo = __ffma2_rn(r.lo[k], wlo[k], a.lo);
+    a.hi = __ffma2_rn(r.hi[k], whi[k], a.hi);
+  }
+}
+
+// MODE 0: stride 1, dilation 1 - every input row feeds three running accumulators
+// MODE 1: stride 2, dilation 1 - the last row of an output is the first row of the next
+// MODE 2: anything else        - three rows fetched per output row
+// ACT: activation applied right after the bias (the common fused case); a residual add or a
+// second activation takes the generic tail.
+template <int MODE, int ACT>
+__global__ void __launch_bounds__(256, 3) depthwise_f16_kernel(const __half* __restrict__ in, const float* __restrict__ w,
+                                                                const float* __restrict__ bias, const __half* __restrict__ res,
+                                                                __half* __restrict__ out, const DwGeom g, const Epilogue ep) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bar;
-  __half* tile = reinterpret_cast<__half*>(smem_raw);
+  __shared__ __align__(8) unsigned long long bars[2];
+  __shared__ unsigned timed_out;
+  const unsigned buf_bytes = static_cast<unsigned>(g.plane_stride_px) * 8u * g.nb;
 
-  const int band = blockIdx.x % g.bands;
-  const int bc = (blockIdx.x / g.bands) % g.bchunks;
-  const int s = blockIdx.x / (g.bands * g.bchunks);
-  const int b0 = bc * g.nb;
-  const int nbk = min(g.nb, g.B - b0);
+  // contiguous, balanced range of work items for this CTA: items of one slice stay together
+  const int per = g.items / gridDim.x, extra = g.items % gridDim.x;
+  const int first = blockIdx.x * per + min(static_cast<int>(blockIdx.x), extra);
+  const int count = per + (static_cast<int>(blockIdx.x) < extra ? 1 : 0);
   const int th = g.sub * g.tr;
-  const int oy0 = band * th, oy1 = min(g.Ho, oy0 + th);
-  const int in_y0 = max(0, oy0 * g.stride - g.pt);
-  const int in_y1 = min(g.H, (oy1 - 1) * g.stride - g.pt + 2 * g.dil + 1);
-  int start_px = in_y0 * g.W;
-  start_px -= start_px & 1;  // copies start on a 16-byte boundary: at most one pixel early
-  const int end_px = min((in_y1 * g.W + 1) & ~1, g.Pin);
-  const unsigned copy_bytes = static_cast<unsigned>(end_px - start_px) * 8u;
-  const unsigned bar_addr = smem_u32(&bar);
 
-  if (threadIdx.x == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_addr) : "memory");
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_addr), "r"(copy_bytes * nbk) : "memory");
+  auto item_rows = [&](int item, int& s, int& b0, int& nbk, int& oy0, int& oy1, int& start_px, unsigned& bytes, bool& last_band) {
+    const int band = item % g.bands;
+    const int bc = (item / g.bands) % g.bchunks;
+    s = item / (g.bands * g.bchunks);
+    b0 = bc * g.nb;
+    nbk = min(g.nb, g.B - b0);
+    oy0 = band * th;
+    oy1 = min(g.Ho, oy0 + th);
+    const int in_y0 = max(0, oy0 * g.stride - g.pt);
+    const int in_y1 = min(g.H, (oy1 - 1) * g.stride - g.pt + 2 * g.dil + 1);
+    start_px = in_y0 * g.W;
+    start_px -= start_px & 1;  // copies start on a 16-byte boundary: at most one pixel early
+    const int end_px = min((in_y1 * g.W + 1) & ~1, g.Pin);
+    bytes = static_cast<unsigned>(end_px - start_px) * 8u;
+    last_band = band == g.bands - 1;
+  };
+  auto issue = [&](int item, int buf) {  // thread 0 only
+    int s, b0, nbk, oy0, oy1, start_px;
+    unsigned bytes;
+    bool lb;
+    item_rows(item, s, b0, nbk, oy0, oy1, start_px, bytes, lb);
+    const unsigned bar = smem_u32(&bars[buf]);
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes * nbk) : "memory");
     for (int pi = 0; pi < nbk; ++pi) {
       const __half* src = in + ((static_cast<size_t>(s) * g.B + b0 + pi) * g.Pin + start_px) * 4;
-      const unsigned dst = smem_u32(tile + static_cast<size_t>(pi) * g.plane_stride_px * 4);
+      const unsigned dst = smem_u32(smem_raw) + buf * buf_bytes + static_cast<unsigned>(pi) * g.plane_stride_px * 8u;
       asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src),
-                   "r"(copy_bytes), "r"(bar_addr)
+                   "r"(bytes), "r"(bar)
                    : "memory");
     }
-  }
-  // weights of this slice: 9 taps x 4 channels, kept in registers
-  float4 wt[9];
-  const int C4 = g.S * 4;
-#pragma unroll
-  for (int t = 0; t < 9; ++t) wt[t] = __ldg(reinterpret_cast<const float4*>(w + t * C4 + s * 4));
-  const float4 bv = __ldg(reinterpret_cast<const float4*>(bias + s * 4));
-  __syncthreads();  // the barrier is initialised before anyone polls it
+  };
 
-  {  // bounded wait for the staged rows
-    unsigned ok = 0;
-    unsigned long long t0 = 0;
-    for (unsigned spin = 0; !ok; ++spin) {
-      asm volatile(
-          "{\n\t.reg .pred p;\n\t"
-          "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
-          "selp.u32 %0, 1, 0, p;\n\t}"
-          : "=r"(ok)
-          : "r"(bar_addr)
-          : "memory");
-      if (!ok && (spin & 255u) == 255u) {
-        unsigned long long now;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-        if (t0 == 0) {
-          t0 = now;
-        } else if (now - t0 > g.timeout_ns) {
-          atomicOr(&g_dw_error, 1u);
-          return;
+  if (threadIdx.x == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bars[0])) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bars[1])) : "memory");
+    timed_out = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    if (count > 0) issue(first, 0);
+  }
+  __syncthreads();
+
+  float2 wlo[9], whi[9];  // 9 taps x (channels 0-1, channels 2-3) of the current slice
+  float2 blo = make_float2(0.f, 0.f), bhi = blo;
+  int cur_s = -1;
+  const int C4 = g.S * 4;
+
+  for (int i = 0; i < count; ++i) {
+    const int buf = i & 1;
+    int s, b0, nbk, oy0, oy1, start_px;
+    unsigned bytes;
+    bool last_band;
+    item_rows(first + i, s, b0, nbk, oy0, oy1, start_px, bytes, last_band);
+    // the other buffer was last read in iteration i-1, which ended with a barrier: refill it now
+    if (threadIdx.x == 0 && i + 1 < count) issue(first + i + 1, buf ^ 1);
+    if (s != cur_s) {
+      cur_s = s;
+#pragma unroll
+      for (int t = 0; t < 9; ++t) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(w + t * C4 + s * 4));
+        wlo[t] = make_float2(v.x, v.y);
+        whi[t] = make_float2(v.z, v.w);
+      }
+      const float4 v = __ldg(reinterpret_cast<const float4*>(bias + s * 4));
+      blo = make_float2(v.x, v.y);
+      bhi = make_float2(v.z, v.w);
+    }
+    {  // bounded wait for this item's rows
+      const unsigned bar = smem_u32(&bars[buf]), parity = (i >> 1) & 1;
+      unsigned ok = 0;
+      unsigned long long t0 = 0;
+      for (unsigned spin = 0; !ok; ++spin) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (!ok && (spin & 255u) == 255u) {
+          unsigned long long now;
+          asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+          if (t0 == 0) {
+            t0 = now;
+          } else if (now - t0 > g.timeout_ns || *reinterpret_cast<volatile unsigned*>(&timed_out)) {
+            timed_out = 1;
+            atomicOr(&g_dw_error, 1u);
+            break;
+          }
         }
       }
     }
-  }
+    if (*reinterpret_cast<volatile unsigned*>(&timed_out)) break;  // give up; results of this launch are invalid
 
-  const int cols = nbk * g.sub * g.Wo;
-  for (int c = threadIdx.x; c < cols; c += blockDim.x) {
-    const int x = c % g.Wo, vp = c / g.Wo;
-    const int sb = vp % g.sub, pi = vp / g.sub;
-    const int ya = oy0 + sb * g.tr, yb = min(oy1, ya + g.tr);
-    if (ya >= yb) continue;
-    const int base_px = pi * g.plane_stride_px - start_px;  // pixel (iy, ix) is staged at base_px + iy*W + ix
-    // column offsets and validity of the three taps
-    int ix[3];
-    bool vx[3];
+    const __half* tile = reinterpret_cast<const __half*>(smem_raw + buf * buf_bytes);
+    const int cols = nbk * g.sub * g.Wo;
+    for (int c = threadIdx.x; c < cols; c += blockDim.x) {
+      const int x = c % g.Wo, vp = c / g.Wo;
+      const int sb = vp % g.sub, pi = vp / g.sub;
+      const int ya = oy0 + sb * g.tr, yb = min(oy1, ya + g.tr);
+      if (ya >= yb) continue;
+      // staged element offset of tap k in input row iy: col[k] + iy * row_stride (in halves)
+      int col[3];
+      bool vx[3];
 #pragma unroll
-    for (int k = 0; k < 3; ++k) {
-      ix[k] = x * g.stride - g.pl + k * g.dil;
-      vx[k] = ix[k] >= 0 && ix[k] < g.W;
+      for (int k = 0; k < 3; ++k) {
+        const int ix = x * g.stride - g.pl + k * g.dil;
+        vx[k] = ix >= 0 && ix < g.W;
+        col[k] = (pi * g.plane_stride_px - start_px + (vx[k] ? ix : 0)) * 4;
+      }
+      const int row_stride = g.W * 4;
+      auto fetch = [&](int iy) {
+        Row r;
+        if (iy >= 0 && iy < g.H) {
+          const __half* rowp = tile + iy * row_stride;
+#pragma unroll
+          for (int k = 0; k < 3; ++k) {
+            uint2 u = *reinterpret_cast<const uint2*>(rowp + col[k]);
+            if (!vx[k]) u = make_uint2(0u, 0u);
+            r.lo[k] = __half22float2(*reinterpret_cast<const __half2*>(&u.x));
+            r.hi[k] = __half22float2(*reinterpret_cast<const __half2*>(&u.y));
+          }
+        } else {
+#pragma unroll
+          for (int k = 0; k < 3; ++k) r.lo[k] = r.hi[k] = make_float2(0.f, 0.f);
+        }
+        return r;
+      };
+      __half* op = out + ((static_cast<size_t>(s) * g.B + b0 + pi) * g.Pout + static_cast<size_t>(ya) * g.Wo + x) * 4;
+      const __half* rp = res + ((static_cast<size_t>(s) * g.B + b0 + pi) * g.Pout + static_cast<size_t>(ya) * g.Wo + x) * 4;
+      const int out_stride = g.Wo * 4;
+      const bool tail = ep.has_res || ep.act_post != GI_ACT_NONE;
+      auto emit = [&](Acc a) {
+        float v[4] = {a.lo.x, a.lo.y, a.hi.x, a.hi.y};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) v[e] = act1(v[e], ACT);
+        if (tail) {
+          if (ep.has_res) {
+            const uint2 u = *reinterpret_cast<const uint2*>(rp);
+            const float2 r0 = __half22float2(*reinterpret_cast<const __half2*>(&u.x));
+            const float2 r1 = __half22float2(*reinterpret_cast<const __half2*>(&u.y));
+            v[0] += r0.x;
+            v[1] += r0.y;
+            v[2] += r1.x;
+            v[3] += r1.y;
+          }
+#pragma unroll
+          for (int e = 0; e < 4; ++e) v[e] = act1(v[e], ep.act_post);
+        }
+        const __half2 lo = __floats2half2_rn(v[0], v[1]), hi = __floats2half2_rn(v[2], v[3]);
+        uint2 u;
+        u.x = *reinterpret_cast<const unsigned*>(&lo);
+        u.y = *reinterpret_cast<const unsigned*>(&hi);
+        *reinterpret_cast<uint2*>(op) = u;
+        op += out_stride;
+        rp += out_stride;
+      };
+      const Acc zero_bias = {blo, bhi};
+      if (MODE == 0) {
+        const int iy0 = ya - g.pt;
+        Row r = fetch(iy0);
+        Acc b_acc = zero_bias;
+        fma_row(b_acc, r, wlo, whi);  // output ya, kernel row 0
+        r = fetch(iy0 + 1);
+        fma_row(b_acc, r, wlo + 3, whi + 3);  // output ya, kernel row 1
+        Acc c_acc = zero_bias;
+        fma_row(c_acc, r, wlo, whi);  // output ya+1, kernel row 0
+        for (int oy = ya; oy < yb; ++oy) {
+          r = fetch(oy - g.pt + 2);
+          Acc a_acc = b_acc;
+          fma_row(a_acc, r, wlo + 6, whi + 6);
+          emit(a_acc);
+          b_acc = c_acc;
+          fma_row(b_acc, r, wlo + 3, whi + 3);
+          c_acc = zero_bias;
+          fma_row(c_acc, r, wlo, whi);
+        }
+      } else if (MODE == 1) {
+        Acc carry = zero_bias;
+        fma_row(carry, fetch(ya * 2 - g.pt), wlo, whi);
+        for (int oy = ya; oy < yb; ++oy) {
+          Acc a_acc = carry;
+          fma_row(a_acc, fetch(oy * 2 - g.pt + 1), wlo + 3, whi + 3);
+          const Row r2 = fetch(oy * 2 - g.pt + 2);
+          fma_row(a_acc, r2, wlo + 6, whi + 6);
+          emit(a_acc);
+          carry = zero_bias;
+          fma_row(carry, r2, wlo, whi);
+        }
+      } else {
+        for (int oy = ya; oy < yb; ++oy) {
+          const int iy = oy * g.stride - g.pt;
+          Acc a_acc = zero_bias;
+          fma_row(a_acc, fetch(iy), wlo, whi);
+          fma_row(a_acc, fetch(iy + g.dil), wlo + 3, whi + 3);
+          fma_row(a_acc, fetch(iy + 2 * g.dil), wlo + 6, whi + 6);
+          emit(a_acc);
+        }
+      }
     }
-    auto fetch = [&](int iy) {
-      Row r;
-      const bool vy = iy >= 0 && iy < g.H;
-      const int row_px = base_px + iy * g.W;
-#pragma unroll
-      for (int k = 0; k < 3; ++k) r.v[k] = (vy && vx[k]) ? ld_px(tile + (row_px + ix[k]) * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-      return r;
-    };
-    const size_t out_plane = (static_cast<size_t>(s) * g.B + b0 + pi) * g.Pout;
-    auto emit = [&](int oy, const Row& r0, const Row& r1, const Row& r2) {
-      float4 acc = bv;
-#pragma unroll
-      for (int k = 0; k < 3; ++k) fma4(acc, r0.v[k], wt[k]);
-#pragma unroll
-      for (int k = 0; k < 3; ++k) fma4(acc, r1.v[k], wt[3 + k]);
-#pragma unroll
-      for (int k = 0; k < 3; ++k) fma4(acc, r2.v[k], wt[6 + k]);
-      acc = make_float4(act1(acc.x, ep.act_pre), act1(acc.y, ep.act_pre), act1(acc.z, ep.act_pre), act1(acc.w, ep.act_pre));
-      const size_t off = (out_plane + static_cast<size_t>(oy) * g.Wo + x) * 4;
-      if (ep.has_res) {
-        const float4 r = ld_px(res + off);
-        acc.x += r.x;
-        acc.y += r.y;
-        acc.z += r.z;
-        acc.w += r.w;
-      }
-      acc = make_float4(act1(acc.x, ep.act_post), act1(acc.y, ep.act_post), act1(acc.z, ep.act_post), act1(acc.w, ep.act_post));
-      const __half2 lo = __floats2half2_rn(acc.x, acc.y), hi = __floats2half2_rn(acc.z, acc.w);
-      uint2 u;
-      u.x = *reinterpret_cast<const unsigned*>(&lo);
-      u.y = *reinterpret_cast<const unsigned*>(&hi);
-      *reinterpret_cast<uint2*>(out + off) = u;
-    };
-    if (MODE == 0) {
-      Row r0 = fetch(ya - g.pt), r1 = fetch(ya - g.pt + 1);
-      for (int oy = ya; oy < yb; ++oy) {
-        const Row r2 = fetch(oy - g.pt + 2);
-        emit(oy, r0, r1, r2);
-        r0 = r1;
-        r1 = r2;
-      }
-    } else if (MODE == 1) {
-      Row r0 = fetch(ya * 2 - g.pt);
-      for (int oy = ya; oy < yb; ++oy) {
-        const Row r1 = fetch(oy * 2 - g.pt + 1), r2 = fetch(oy * 2 - g.pt + 2);
-        emit(oy, r0, r1, r2);
-        r0 = r2;
-      }
-    } else {
-      for (int oy = ya; oy < yb; ++oy) {
-        const int iy = oy * g.stride - g.pt;
-        emit(oy, fetch(iy), fetch(iy + g.dil), fetch(iy + 2 * g.dil));
-      }
+    // an odd plane carries one extra pixel: keep it zero
+    if (last_band && g.Pout > g.Ho * g.Wo && static_cast<int>(threadIdx.x) < nbk) {
+      const size_t off = ((static_cast<size_t>(s) * g.B + b0 + threadIdx.x) * g.Pout + g.Ho * g.Wo) * 4;
+      *reinterpret_cast<uint2*>(out + off) = make_uint2(0u, 0u);
     }
+    __syncthreads();  // everyone is done with this buffer before it is refilled
   }
-  // an odd plane carries one extra pixel: keep it zero
-  if (band == g.bands - 1 && g.Pout > g.Ho * g.Wo && threadIdx.x < nbk) {
-    const size_t off = ((static_cast<size_t>(s) * g.B + b0 + threadIdx.x) * g.Pout + g.Ho * g.Wo) * 4;
-    *reinterpret_cast<uint2*>(out + off) = make_uint2(0u, 0u);
+  if (*reinterpret_cast<volatile unsigned*>(&timed_out) && threadIdx.x == 0) {
+    // copies already issued may still land: give them the same bounded grace before leaving
+    unsigned long long t0, now;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    do {
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+    } while (now - t0 < g.timeout_ns);
   }
 }
 
-constexpr int kMaxSmem = 160 * 1024;
+constexpr int kMaxSmem = 200 * 1024;  // both staging buffers of one CTA
 
 }  // namespace
 
@@ -242,8 +332,8 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
     return (px + 1) & ~1;
   };
   g.plane_stride_px = smem_for(g);
-  // shrink until the staging buffer fits
-  while (static_cast<long long>(g.plane_stride_px) * 8 * g.nb > kMaxSmem && (g.nb > 1 || g.sub > 1 || g.tr > 1)) {
+  const long long budget = 64 * 1024;  // per staging buffer: two buffers per CTA, two or three CTAs per SM
+  while (static_cast<long long>(g.plane_stride_px) * 8 * g.nb > budget && (g.nb > 1 || g.sub > 1 || g.tr > 1)) {
     if (g.nb > 1) {
       g.nb = (g.nb + 1) / 2;
     } else if (g.sub > 1) {
@@ -255,39 +345,64 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
     g.bands = (total_sub + g.sub - 1) / g.sub;
     g.plane_stride_px = smem_for(g);
   }
-  const size_t smem = static_cast<size_t>(g.plane_stride_px) * 8 * g.nb;
+  const size_t smem = static_cast<size_t>(g.plane_stride_px) * 8 * g.nb * 2;
   if (smem > static_cast<size_t>(kMaxSmem)) return static_cast<int>(cudaErrorInvalidConfiguration);
   g.bchunks = (g.B + g.nb - 1) / g.nb;
-  const long long blocks = static_cast<long long>(g.S) * g.bchunks * g.bands;
-  if (blocks > 2147483647LL) return static_cast<int>(cudaErrorInvalidConfiguration);
+  const long long items = static_cast<long long>(g.S) * g.bchunks * g.bands;
+  if (items > 2147483647LL) return static_cast<int>(cudaErrorInvalidConfiguration);
+  g.items = static_cast<int>(items);
   int threads = (g.nb * g.sub * g.Wo + 31) / 32 * 32;
-  if (threads > 512) threads = 512;
+  if (threads > 256) threads = 256;
   if (threads < 32) threads = 32;
-  const int mode = (g.stride == 1 && g.dil == 1 && r.sw == 1 && r.dw == 1) ? 0
-                   : (g.stride == 2 && g.dil == 1 && r.sw == 2 && r.dw == 1) ? 1 : 2;
-  static bool attr_done[3] = {false, false, false};
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+  }
+  // persistent CTAs, a few per SM so that one CTA's copies overlap another's arithmetic
+  long long ctas_per_sm = static_cast<long long>(kMaxSmem) / static_cast<long long>(smem > 0 ? smem : 1);
+  if (ctas_per_sm > 2048 / threads) ctas_per_sm = 2048 / threads;
+  if (ctas_per_sm > 4) ctas_per_sm = 4;
+  if (ctas_per_sm < 1) ctas_per_sm = 1;
+  long long grid = static_cast<long long>(sms) * ctas_per_sm;
+  if (grid > items) grid = items;
+  const int mode = (g.stride == 1 && g.dil == 1) ? 0 : (g.stride == 2 && g.dil == 1) ? 1 : 2;
+  const int act = r.ep.act_pre;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const __half* in = static_cast<const __half*>(p.in0);
   const float* w = static_cast<const float*>(p.wts);
   const float* b = static_cast<const float*>(p.bias);
   const __half* res = static_cast<const __half*>(p.res);
   __half* out = static_cast<__half*>(p.out);
-#define GI_DW_LAUNCH(M)                                                                                                \
-  do {                                                                                                                 \
-    if (!attr_done[M]) {                                                                                               \
-      const cudaError_t e = cudaFuncSetAttribute(depthwise_f16_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem); \
-      if (e != cudaSuccess) return static_cast<int>(e);                                                                \
-      attr_done[M] = true;                                                                                             \
-    }                                                                                                                  \
-    depthwise_f16_kernel<M><<<static_cast<unsigned>(blocks), threads, smem, st>>>(in, w, b, res, out, g, r.ep);        \
+  static bool attr_done[3][3] = {};
+#define GI_DW_LAUNCH(M, A)                                                                                                       \
+  do {                                                                                                                           \
+    if (!attr_done[M][A]) {                                                                                                      \
+      const cudaError_t e = cudaFuncSetAttribute(depthwise_f16_kernel<M, A>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem); \
+      if (e != cudaSuccess) return static_cast<int>(e);                                                                          \
+      attr_done[M][A] = true;                                                                                                    \
+    }                                                                                                                            \
+    depthwise_f16_kernel<M, A><<<static_cast<unsigned>(grid), threads, smem, st>>>(in, w, b, res, out, g, r.ep);                 \
+  } while (0)
+#define GI_DW_MODE(M)                 \
+  do {                                \
+    if (act == GI_ACT_RELU6) {        \
+      GI_DW_LAUNCH(M, GI_ACT_RELU6);  \
+    } else if (act == GI_ACT_RELU) {  \
+      GI_DW_LAUNCH(M, GI_ACT_RELU);   \
+    } else {                          \
+      GI_DW_LAUNCH(M, GI_ACT_NONE);   \
+    }                                 \
   } while (0)
   if (mode == 0) {
-    GI_DW_LAUNCH(0);
+    GI_DW_MODE(0);
   } else if (mode == 1) {
-    GI_DW_LAUNCH(1);
+    GI_DW_MODE(1);
   } else {
-    GI_DW_LAUNCH(2);
+    GI_DW_MODE(2);
   }
+#undef GI_DW_MODE
 #undef GI_DW_LAUNCH
   return static_cast<int>(cudaGetLastError());
 }
