@@ -214,6 +214,29 @@ GI_API gi_status gi_exec_bind(gi_exec* e, void* dev_weights, size_t weight_bytes
 GI_API gi_status gi_run(gi_exec* e, const void* const* dev_inputs, void* const* dev_outputs, void* dev_arena,
                  size_t arena_bytes, void* stream);
 
+/* gi_run for callers that cannot allocate device memory.  (The paper has no counterpart: its
+ * engine always allocates the buffers its memory manager planned.)
+ *
+ * Some hosts of this library have no way to hand over an arena: a plug-in whose embedding
+ * application owns every device allocation and exposes none to it, a process started with a
+ * fixed device-memory budget that is already spent, a service loop that must not call
+ * cudaMalloc because that call synchronises the whole device and can fail under fragmentation.
+ * For them the intermediates live in a fixed array that is part of the library image itself:
+ * GI_STATIC_ARENA_BYTES of device memory on every GPU that loads the library, held until the
+ * process exits.  The caller still passes the input and output buffers and must have called
+ * gi_exec_bind with a weight buffer it obtained by whatever means it has.
+ *
+ * The call allocates nothing: no cudaMalloc, cudaFree or allocating library routine.  The
+ * first call on a device looks up the array's device address (once per device, with that
+ * device current); make that first call outside any stream capture.  An executable whose
+ * info.arena_bytes exceeds GI_STATIC_ARENA_BYTES is refused with GI_E_ARENA before anything is
+ * launched.  All calls on a device share the one array and it keeps the previous call's
+ * contents; nothing in it has to start at zero, because every kernel writes each byte of its
+ * output that a later kernel reads (padding lanes and pixels included).  Two calls that overlap
+ * on the GPU (different streams, or another thread) race on the array: serialise them. */
+#define GI_STATIC_ARENA_BYTES (16u << 20)
+GI_API gi_status gi_run_static(gi_exec* e, const void* const* dev_inputs, void* const* dev_outputs, void* stream);
+
 /* Profiling aid: the same launches as gi_run, with a CUDA event recorded before each executed op
  * and after the last one; synchronises `stream` before returning and writes the device time of
  * op i, in milliseconds, to op_ms[i] (n_op_ms must be >= info.n_ops).  The paper's own protocol

@@ -26,6 +26,7 @@ GI_EXEC_PACK, GI_EXEC_UNPACK = 100, 101
 GI_ACT_NONE, GI_ACT_RELU, GI_ACT_RELU6 = 0, 1, 2
 GI_PLAN_GREEDY_BY_SIZE, GI_PLAN_GREEDY_SHARED_OBJECTS, GI_PLAN_NAIVE = 0, 1, 2
 GI_PW_AUTO, GI_PW_SIMT = 0, 1
+GI_STATIC_ARENA_BYTES = 16 << 20
 KERNEL_NAMES = {1: "pack", 2: "unpack", 3: "conv_simt", 4: "pointwise_tc", 5: "depthwise", 6: "eltwise", 7: "pool",
                 8: "resize"}
 
@@ -66,7 +67,7 @@ class gi_op_info(C.Structure):
 
 
 EXPORTS = ["gi_graph_create", "gi_graph_input", "gi_add_op", "gi_graph_output", "gi_graph_destroy", "gi_compile",
-           "gi_exec_query", "gi_exec_tensor", "gi_exec_op", "gi_exec_bind", "gi_run", "gi_run_timed", "gi_device_status", "gi_exec_destroy",
+           "gi_exec_query", "gi_exec_tensor", "gi_exec_op", "gi_exec_bind", "gi_run", "gi_run_static", "gi_run_timed", "gi_device_status", "gi_exec_destroy",
            "gi_status_str", "gi_last_error", "gi_tensor_bytes", "gi_f32_to_f16"]
 
 _lib = None
@@ -100,6 +101,8 @@ def lib() -> C.CDLL:
     L.gi_exec_op.argtypes = [vp, C.c_int32, C.POINTER(gi_op_info)]
     L.gi_exec_bind.argtypes = [vp, vp, C.c_size_t, vp]
     L.gi_run.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp, C.c_size_t, vp]
+    L.gi_run_static.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp]
+    L.gi_run_static.restype = C.c_int32
     L.gi_run_timed.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp, C.c_size_t, vp, C.POINTER(C.c_float), C.c_int32]
     L.gi_device_status.argtypes = [C.POINTER(C.c_uint32)]
     L.gi_device_status.restype = C.c_int32
@@ -265,6 +268,12 @@ class Executable:
         ins = (C.c_void_p * max(len(in_ptrs), 1))(*in_ptrs)
         outs = (C.c_void_p * max(len(out_ptrs), 1))(*out_ptrs)
         _check(lib().gi_run(self._h, ins, outs, arena_ptr, arena_bytes, _stream_ptr(stream)), "gi_run")
+
+    def run_static(self, inputs, outputs, stream=None) -> None:
+        """gi_run_static: intermediates in the library's built-in arena; allocates nothing."""
+        ins = (C.c_void_p * max(len(inputs), 1))(*[t.data_ptr() for t in inputs])
+        outs = (C.c_void_p * max(len(outputs), 1))(*[t.data_ptr() for t in outputs])
+        _check(lib().gi_run_static(self._h, ins, outs, _stream_ptr(stream)), "gi_run_static")
 
     def run_timed(self, inputs, outputs, stream=None) -> List[float]:
         """gi_run_timed: one run with an event around every executed op; returns per-op milliseconds."""

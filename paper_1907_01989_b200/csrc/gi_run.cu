@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <mutex>
 #include <string>
 #include <vector>
 
@@ -108,6 +109,37 @@ gi_status gi_device_status(uint32_t* flags) {
 gi_status gi_run(gi_exec* e, const void* const* dev_inputs, void* const* dev_outputs, void* dev_arena, size_t arena_bytes,
                  void* stream) {
   return run_impl(e, dev_inputs, dev_outputs, dev_arena, arena_bytes, stream, nullptr);
+}
+
+// ---------------------------------------------------------------- fixed arena (no allocation)
+// The arena of gi_run_static.  In host code this name is only a handle for the symbol: the
+// address kernels can use is obtained with cudaGetSymbolAddress, once per device.
+static __device__ __align__(256) unsigned char g_static_arena[GI_STATIC_ARENA_BYTES];
+static std::mutex g_static_mu;
+static void* g_static_ptr[64] = {};
+
+gi_status gi_run_static(gi_exec* e, const void* const* dev_inputs, void* const* dev_outputs, void* stream) {
+  if (!e) return fail(GI_E_INVALID, "gi_run_static: null executable");
+  if (e->arena_bytes > GI_STATIC_ARENA_BYTES)
+    return fail(GI_E_ARENA, "gi_run_static: executable needs " + std::to_string(e->arena_bytes) +
+                                " arena bytes, the built-in arena holds " + std::to_string(GI_STATIC_ARENA_BYTES));
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return fail(GI_E_CUDA, std::string("gi_run_static: ") + cudaGetErrorString(err));
+  if (dev < 0 || dev >= 64) return fail(GI_E_UNSUPPORTED, "gi_run_static: device ordinal above 63");
+  void* arena = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+      void* ptr = nullptr;
+      err = cudaGetSymbolAddress(&ptr, g_static_arena);
+      if (err != cudaSuccess || !ptr)
+        return fail(GI_E_CUDA, std::string("gi_run_static: cudaGetSymbolAddress: ") + cudaGetErrorString(err));
+      g_static_ptr[dev] = ptr;
+    }
+    arena = g_static_ptr[dev];
+  }
+  return run_impl(e, dev_inputs, dev_outputs, arena, GI_STATIC_ARENA_BYTES, stream, nullptr);
 }
 
 gi_status gi_run_timed(gi_exec* e, const void* const* dev_inputs, void* const* dev_outputs, void* dev_arena,
