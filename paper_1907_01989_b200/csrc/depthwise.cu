@@ -28,6 +28,7 @@ struct DwGeom {
   int tr;       // output rows walked by one thread
   int bands;    // bands per plane
   int bchunks;  // ceil(B / nb)
+  int head_px;  // zeroed pixels in front of each plane's staged rows (even, >= W + 2)
   int plane_stride_px;  // pixels reserved per plane in one staging buffer (even)
   int items;            // S * bchunks * bands
   unsigned timeout_ns;
@@ -56,10 +57,24 @@ __device__ __forceinline__ void fma_row(Acc& a, const Row& r, const float2* wlo,
     a.hi = __ffma2_rn(r.hi[k], whi[k], a.hi);
   }
 }
+__device__ __forceinline__ Row widen(const uint2* u) {
+  Row r;
+#pragma unroll
+  for (int k = 0; k < 3; ++k) {
+    r.lo[k] = __half22float2(*reinterpret_cast<const __half2*>(&u[k].x));
+    r.hi[k] = __half22float2(*reinterpret_cast<const __half2*>(&u[k].y));
+  }
+  return r;
+}
 
-// MODE 0: stride 1, dilation 1 - every input row feeds three running accumulators
-// MODE 1: stride 2, dilation 1 - the last row of an output is the first row of the next
-// MODE 2: anything else        - three rows fetched per output row
+// Staging buffer of one plane: [head_px zeros][rows of the band, copied][W+1 zeros when the band
+// touches the bottom edge].  Row -1 and row H therefore read as zeros with no test in the loop.
+//
+// MODE 0: stride 1, dilation 1, at most one padding row above and below - every input row feeds
+//         three running accumulators
+// MODE 1: stride 2, dilation 1, same padding limit - the last row of an output is the first row
+//         of the next
+// MODE 2: anything else - three rows fetched per output row, each tap tested
 // ACT: activation applied right after the bias (the common fused case); a residual add or a
 // second activation takes the generic tail.
 template <int MODE, int ACT>
@@ -70,6 +85,7 @@ __global__ void __launch_bounds__(256, 3) depthwise_f16_kernel(const __half* __r
   __shared__ __align__(8) unsigned long long bars[2];
   __shared__ unsigned timed_out;
   const unsigned buf_bytes = static_cast<unsigned>(g.plane_stride_px) * 8u * g.nb;
+  const int W = g.W, H = g.H, Wo = g.Wo, stride = g.stride, pt = g.pt;
 
   // contiguous, balanced range of work items for this CTA: items of one slice stay together
   const int per = g.items / gridDim.x, extra = g.items % gridDim.x;
@@ -85,11 +101,11 @@ __global__ void __launch_bounds__(256, 3) depthwise_f16_kernel(const __half* __r
     nbk = min(g.nb, g.B - b0);
     oy0 = band * th;
     oy1 = min(g.Ho, oy0 + th);
-    const int in_y0 = max(0, oy0 * g.stride - g.pt);
-    const int in_y1 = min(g.H, (oy1 - 1) * g.stride - g.pt + 2 * g.dil + 1);
-    start_px = in_y0 * g.W;
+    const int in_y0 = max(0, oy0 * stride - pt);
+    const int in_y1 = min(H, (oy1 - 1) * stride - pt + 2 * g.dil + 1);
+    start_px = in_y0 * W;
     start_px -= start_px & 1;  // copies start on a 16-byte boundary: at most one pixel early
-    const int end_px = min((in_y1 * g.W + 1) & ~1, g.Pin);
+    const int end_px = min((in_y1 * W + 1) & ~1, g.Pin);
     bytes = static_cast<unsigned>(end_px - start_px) * 8u;
     last_band = band == g.bands - 1;
   };
@@ -99,22 +115,29 @@ __global__ void __launch_bounds__(256, 3) depthwise_f16_kernel(const __half* __r
     bool lb;
     item_rows(item, s, b0, nbk, oy0, oy1, start_px, bytes, lb);
     const unsigned bar = smem_u32(&bars[buf]);
+    // earlier generic-proxy writes to this buffer (the zeroed bottom row) precede the async writes
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes * nbk) : "memory");
     for (int pi = 0; pi < nbk; ++pi) {
       const __half* src = in + ((static_cast<size_t>(s) * g.B + b0 + pi) * g.Pin + start_px) * 4;
-      const unsigned dst = smem_u32(smem_raw) + buf * buf_bytes + static_cast<unsigned>(pi) * g.plane_stride_px * 8u;
+      const unsigned dst =
+          smem_u32(smem_raw) + buf * buf_bytes + (static_cast<unsigned>(pi) * g.plane_stride_px + g.head_px) * 8u;
       asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src),
                    "r"(bytes), "r"(bar)
                    : "memory");
     }
   };
 
+  // the zero heads are written once; copies never touch them
+  for (int i = threadIdx.x; i < 2 * g.nb * g.head_px; i += blockDim.x) {
+    const int plane = i / g.head_px, px = i - plane * g.head_px;
+    *reinterpret_cast<uint2*>(smem_raw + (static_cast<size_t>(plane) * g.plane_stride_px + px) * 8) = make_uint2(0u, 0u);
+  }
   if (threadIdx.x == 0) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bars[0])) : "memory");
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bars[1])) : "memory");
     timed_out = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     if (count > 0) issue(first, 0);
   }
   __syncthreads();
@@ -123,6 +146,7 @@ __global__ void __launch_bounds__(256, 3) depthwise_f16_kernel(const __half* __r
   float2 blo = make_float2(0.f, 0.f), bhi = blo;
   int cur_s = -1;
   const int C4 = g.S * 4;
+  const bool tail = ep.has_res || ep.act_post != GI_ACT_NONE;
 
   for (int i = 0; i < count; ++i) {
     const int buf = i & 1;
@@ -171,53 +195,57 @@ __global__ void __launch_bounds__(256, 3) depthwise_f16_kernel(const __half* __r
     }
     if (*reinterpret_cast<volatile unsigned*>(&timed_out)) break;  // give up; results of this launch are invalid
 
-    const __half* tile = reinterpret_cast<const __half*>(smem_raw + buf * buf_bytes);
-    const int cols = nbk * g.sub * g.Wo;
+    unsigned char* buf_base = smem_raw + buf * buf_bytes;
+    if (MODE != 2 && (oy1 - 1) * stride - pt + 2 >= H) {
+      // this band reads row H: W+1 zero pixels right after the last image row (they replace the
+      // plane's own padding pixel and whatever an earlier item left there)
+      const int z0 = H * W - start_px;
+      for (int j = threadIdx.x; j < nbk * (W + 1); j += blockDim.x) {
+        const int pi = j / (W + 1), px = j - pi * (W + 1);
+        *reinterpret_cast<uint2*>(buf_base + (static_cast<size_t>(pi) * g.plane_stride_px + g.head_px + z0 + px) * 8) =
+            make_uint2(0u, 0u);
+      }
+      __syncthreads();
+    }
+
+    const int cols = nbk * g.sub * Wo;
     for (int c = threadIdx.x; c < cols; c += blockDim.x) {
-      const int x = c % g.Wo, vp = c / g.Wo;
+      const int x = c % Wo, vp = c / Wo;
       const int sb = vp % g.sub, pi = vp / g.sub;
       const int ya = oy0 + sb * g.tr, yb = min(oy1, ya + g.tr);
       if (ya >= yb) continue;
-      // staged element offset of tap k in input row iy: col[k] + iy * row_stride (in halves)
-      int col[3];
-      bool vx[3];
-#pragma unroll
-      for (int k = 0; k < 3; ++k) {
-        const int ix = x * g.stride - g.pl + k * g.dil;
-        vx[k] = ix >= 0 && ix < g.W;
-        col[k] = (pi * g.plane_stride_px - start_px + (vx[k] ? ix : 0)) * 4;
-      }
-      const int row_stride = g.W * 4;
-      auto fetch = [&](int iy) {
-        Row r;
-        if (iy >= 0 && iy < g.H) {
-          const __half* rowp = tile + iy * row_stride;
-#pragma unroll
-          for (int k = 0; k < 3; ++k) {
-            uint2 u = *reinterpret_cast<const uint2*>(rowp + col[k]);
-            if (!vx[k]) u = make_uint2(0u, 0u);
-            r.lo[k] = __half22float2(*reinterpret_cast<const __half2*>(&u.x));
-            r.hi[k] = __half22float2(*reinterpret_cast<const __half2*>(&u.y));
+      // plane_zero: a pixel of the zero head; data: where pixel (0,0) of the plane would be staged
+      const __half* plane_zero = reinterpret_cast<const __half*>(buf_base) + static_cast<size_t>(pi) * g.plane_stride_px * 4;
+      const __half* data = plane_zero + (g.head_px - start_px) * 4;
+      const size_t out_off = ((static_cast<size_t>(s) * g.B + b0 + pi) * g.Pout + static_cast<size_t>(ya) * Wo + x) * 4;
+      __half* op = out + out_off;
+      const __half* rp = res + out_off;
+      const int out_stride = Wo * 4;
+      auto emit = [&](const Acc& a) {
+        uint2 u;
+        if (!tail) {
+          // clamping after the rounding equals rounding after the clamp: 0 and 6 are fp16 values
+          __half2 lo = __floats2half2_rn(a.lo.x, a.lo.y), hi = __floats2half2_rn(a.hi.x, a.hi.y);
+          if (ACT != GI_ACT_NONE) {
+            const __half2 z = __float2half2_rn(0.f);
+            lo = __hmax2(lo, z);
+            hi = __hmax2(hi, z);
           }
+          if (ACT == GI_ACT_RELU6) {
+            const __half2 six = __float2half2_rn(6.f);
+            lo = __hmin2(lo, six);
+            hi = __hmin2(hi, six);
+          }
+          u.x = *reinterpret_cast<const unsigned*>(&lo);
+          u.y = *reinterpret_cast<const unsigned*>(&hi);
         } else {
+          float v[4] = {a.lo.x, a.lo.y, a.hi.x, a.hi.y};
 #pragma unroll
-          for (int k = 0; k < 3; ++k) r.lo[k] = r.hi[k] = make_float2(0.f, 0.f);
-        }
-        return r;
-      };
-      __half* op = out + ((static_cast<size_t>(s) * g.B + b0 + pi) * g.Pout + static_cast<size_t>(ya) * g.Wo + x) * 4;
-      const __half* rp = res + ((static_cast<size_t>(s) * g.B + b0 + pi) * g.Pout + static_cast<size_t>(ya) * g.Wo + x) * 4;
-      const int out_stride = g.Wo * 4;
-      const bool tail = ep.has_res || ep.act_post != GI_ACT_NONE;
-      auto emit = [&](Acc a) {
-        float v[4] = {a.lo.x, a.lo.y, a.hi.x, a.hi.y};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) v[e] = act1(v[e], ACT);
-        if (tail) {
+          for (int e = 0; e < 4; ++e) v[e] = act1(v[e], ACT);
           if (ep.has_res) {
-            const uint2 u = *reinterpret_cast<const uint2*>(rp);
-            const float2 r0 = __half22float2(*reinterpret_cast<const __half2*>(&u.x));
-            const float2 r1 = __half22float2(*reinterpret_cast<const __half2*>(&u.y));
+            const uint2 q = *reinterpret_cast<const uint2*>(rp);
+            const float2 r0 = __half22float2(*reinterpret_cast<const __half2*>(&q.x));
+            const float2 r1 = __half22float2(*reinterpret_cast<const __half2*>(&q.y));
             v[0] += r0.x;
             v[1] += r0.y;
             v[2] += r1.x;
@@ -225,61 +253,108 @@ __global__ void __launch_bounds__(256, 3) depthwise_f16_kernel(const __half* __r
           }
 #pragma unroll
           for (int e = 0; e < 4; ++e) v[e] = act1(v[e], ep.act_post);
+          const __half2 lo = __floats2half2_rn(v[0], v[1]), hi = __floats2half2_rn(v[2], v[3]);
+          u.x = *reinterpret_cast<const unsigned*>(&lo);
+          u.y = *reinterpret_cast<const unsigned*>(&hi);
         }
-        const __half2 lo = __floats2half2_rn(v[0], v[1]), hi = __floats2half2_rn(v[2], v[3]);
-        uint2 u;
-        u.x = *reinterpret_cast<const unsigned*>(&lo);
-        u.y = *reinterpret_cast<const unsigned*>(&hi);
         *reinterpret_cast<uint2*>(op) = u;
         op += out_stride;
         rp += out_stride;
       };
-      const Acc zero_bias = {blo, bhi};
-      if (MODE == 0) {
-        const int iy0 = ya - g.pt;
-        Row r = fetch(iy0);
-        Acc b_acc = zero_bias;
-        fma_row(b_acc, r, wlo, whi);  // output ya, kernel row 0
-        r = fetch(iy0 + 1);
-        fma_row(b_acc, r, wlo + 3, whi + 3);  // output ya, kernel row 1
-        Acc c_acc = zero_bias;
-        fma_row(c_acc, r, wlo, whi);  // output ya+1, kernel row 0
-        for (int oy = ya; oy < yb; ++oy) {
-          r = fetch(oy - g.pt + 2);
-          Acc a_acc = b_acc;
-          fma_row(a_acc, r, wlo + 6, whi + 6);
-          emit(a_acc);
-          b_acc = c_acc;
-          fma_row(b_acc, r, wlo + 3, whi + 3);
-          c_acc = zero_bias;
-          fma_row(c_acc, r, wlo, whi);
+      const Acc bias_acc = {blo, bhi};
+
+      if (MODE != 2) {
+        // one pointer per tap column, walking down the staged rows; a column outside the image
+        // stays on a zero pixel
+        const __half* tp[3];
+        int step[3];
+        const int iy_first = ya * stride - pt;
+#pragma unroll
+        for (int k = 0; k < 3; ++k) {
+          const int ix = x * stride - g.pl + k;
+          const bool v = ix >= 0 && ix < W;
+          tp[k] = v ? data + (iy_first * W + ix) * 4 : plane_zero;
+          step[k] = v ? W * 4 : 0;
         }
-      } else if (MODE == 1) {
-        Acc carry = zero_bias;
-        fma_row(carry, fetch(ya * 2 - g.pt), wlo, whi);
-        for (int oy = ya; oy < yb; ++oy) {
-          Acc a_acc = carry;
-          fma_row(a_acc, fetch(oy * 2 - g.pt + 1), wlo + 3, whi + 3);
-          const Row r2 = fetch(oy * 2 - g.pt + 2);
-          fma_row(a_acc, r2, wlo + 6, whi + 6);
-          emit(a_acc);
-          carry = zero_bias;
-          fma_row(carry, r2, wlo, whi);
+        auto next_row = [&]() {
+          uint2 u[3];
+#pragma unroll
+          for (int k = 0; k < 3; ++k) {
+            u[k] = *reinterpret_cast<const uint2*>(tp[k]);
+            tp[k] += step[k];
+          }
+          return widen(u);
+        };
+        if (MODE == 0) {
+          Acc a0 = bias_acc, a1 = bias_acc, a2;
+          Row r = next_row();
+          fma_row(a0, r, wlo, whi);  // output ya, kernel row 0
+          r = next_row();
+          fma_row(a0, r, wlo + 3, whi + 3);  // output ya, kernel row 1
+          fma_row(a1, r, wlo, whi);          // output ya+1, kernel row 0
+          for (int oy = ya; oy < yb; oy += 3) {
+            r = next_row();
+            fma_row(a0, r, wlo + 6, whi + 6);
+            emit(a0);
+            fma_row(a1, r, wlo + 3, whi + 3);
+            a2 = bias_acc;
+            fma_row(a2, r, wlo, whi);
+            if (oy + 1 >= yb) break;
+            r = next_row();
+            fma_row(a1, r, wlo + 6, whi + 6);
+            emit(a1);
+            fma_row(a2, r, wlo + 3, whi + 3);
+            a0 = bias_acc;
+            fma_row(a0, r, wlo, whi);
+            if (oy + 2 >= yb) break;
+            r = next_row();
+            fma_row(a2, r, wlo + 6, whi + 6);
+            emit(a2);
+            fma_row(a0, r, wlo + 3, whi + 3);
+            a1 = bias_acc;
+            fma_row(a1, r, wlo, whi);
+          }
+        } else {
+          Acc carry = bias_acc;
+          fma_row(carry, next_row(), wlo, whi);
+          for (int oy = ya; oy < yb; ++oy) {
+            fma_row(carry, next_row(), wlo + 3, whi + 3);
+            const Row r2 = next_row();
+            fma_row(carry, r2, wlo + 6, whi + 6);
+            emit(carry);
+            carry = bias_acc;
+            fma_row(carry, r2, wlo, whi);
+          }
         }
       } else {
+        int ix[3];
+        bool vx[3];
+#pragma unroll
+        for (int k = 0; k < 3; ++k) {
+          ix[k] = x * stride - g.pl + k * g.dil;
+          vx[k] = ix[k] >= 0 && ix[k] < W;
+        }
+        auto fetch = [&](int iy) {
+          uint2 u[3];
+          const bool vy = iy >= 0 && iy < H;
+#pragma unroll
+          for (int k = 0; k < 3; ++k)
+            u[k] = (vy && vx[k]) ? *reinterpret_cast<const uint2*>(data + (iy * W + ix[k]) * 4) : make_uint2(0u, 0u);
+          return widen(u);
+        };
         for (int oy = ya; oy < yb; ++oy) {
-          const int iy = oy * g.stride - g.pt;
-          Acc a_acc = zero_bias;
-          fma_row(a_acc, fetch(iy), wlo, whi);
-          fma_row(a_acc, fetch(iy + g.dil), wlo + 3, whi + 3);
-          fma_row(a_acc, fetch(iy + 2 * g.dil), wlo + 6, whi + 6);
-          emit(a_acc);
+          const int iy = oy * stride - pt;
+          Acc a = bias_acc;
+          fma_row(a, fetch(iy), wlo, whi);
+          fma_row(a, fetch(iy + g.dil), wlo + 3, whi + 3);
+          fma_row(a, fetch(iy + 2 * g.dil), wlo + 6, whi + 6);
+          emit(a);
         }
       }
     }
     // an odd plane carries one extra pixel: keep it zero
-    if (last_band && g.Pout > g.Ho * g.Wo && static_cast<int>(threadIdx.x) < nbk) {
-      const size_t off = ((static_cast<size_t>(s) * g.B + b0 + threadIdx.x) * g.Pout + g.Ho * g.Wo) * 4;
+    if (last_band && g.Pout > g.Ho * Wo && static_cast<int>(threadIdx.x) < nbk) {
+      const size_t off = ((static_cast<size_t>(s) * g.B + b0 + threadIdx.x) * g.Pout + g.Ho * Wo) * 4;
       *reinterpret_cast<uint2*>(out + off) = make_uint2(0u, 0u);
     }
     __syncthreads();  // everyone is done with this buffer before it is refilled
@@ -313,6 +388,7 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
   g.pt = r.pt;
   g.pl = r.pl;
   g.timeout_ns = 1000000000u;
+  g.head_px = (g.W + 3) & ~1;
   // thread groups: as many "virtual planes" (plane x sub-band) as fit in ~256 threads
   int vp = 256 / g.Wo;
   if (vp < 1) vp = 1;
@@ -327,9 +403,9 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
   auto smem_for = [&](const DwGeom& q) {
     const int th = q.sub * q.tr;
     const int rows_in = (th - 1) * q.stride + 2 * q.dil + 1;
-    int px = (rows_in < q.H ? rows_in : q.H) * q.W + 2;
+    int px = (rows_in < q.H ? rows_in : q.H) * q.W + 2;  // + alignment pixel in front, rounding pixel behind
     if (px > q.Pin) px = q.Pin;
-    return (px + 1) & ~1;
+    return q.head_px + ((px + 1) & ~1) + ((q.W + 3) & ~1);  // zero head, staged rows, zero row behind
   };
   g.plane_stride_px = smem_for(g);
   const long long budget = 64 * 1024;  // per staging buffer: two buffers per CTA, two or three CTAs per SM
@@ -363,11 +439,14 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
   // persistent CTAs, a few per SM so that one CTA's copies overlap another's arithmetic
   long long ctas_per_sm = static_cast<long long>(kMaxSmem) / static_cast<long long>(smem > 0 ? smem : 1);
   if (ctas_per_sm > 2048 / threads) ctas_per_sm = 2048 / threads;
-  if (ctas_per_sm > 4) ctas_per_sm = 4;
+  if (ctas_per_sm > 3) ctas_per_sm = 3;
   if (ctas_per_sm < 1) ctas_per_sm = 1;
   long long grid = static_cast<long long>(sms) * ctas_per_sm;
   if (grid > items) grid = items;
-  const int mode = (g.stride == 1 && g.dil == 1) ? 0 : (g.stride == 2 && g.dil == 1) ? 1 : 2;
+  // the fast paths need the rows above and below the image to be at most one (zero rows in the buffer)
+  const int overshoot = (g.Ho - 1) * g.stride - g.pt + 2 - (g.H - 1);
+  const bool edge_ok = g.dil == 1 && g.pt <= 1 && overshoot <= 1;
+  const int mode = (edge_ok && g.stride == 1) ? 0 : (edge_ok && g.stride == 2) ? 1 : 2;
   const int act = r.ep.act_pre;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const __half* in = static_cast<const __half*>(p.in0);
