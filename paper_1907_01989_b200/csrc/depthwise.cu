@@ -57,6 +57,23 @@ __device__ __forceinline__ void fma_row(Acc& a, const Row& r, const float2* wlo,
     a.hi = __ffma2_rn(r.hi[k], whi[k], a.hi);
   }
 }
+// start of an accumulation: the bias is the addend of the first FMA
+__device__ __forceinline__ Acc fma_row_from(const Acc& bias, const Row& r, const float2* wlo, const float2* whi) {
+  Acc a;
+  a.lo = __ffma2_rn(r.lo[0], wlo[0], bias.lo);
+  a.hi = __ffma2_rn(r.hi[0], whi[0], bias.hi);
+#pragma unroll
+  for (int k = 1; k < 3; ++k) {
+    a.lo = __ffma2_rn(r.lo[k], wlo[k], a.lo);
+    a.hi = __ffma2_rn(r.hi[k], whi[k], a.hi);
+  }
+  return a;
+}
+__device__ __forceinline__ uint2 lds64(unsigned addr) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+  return v;
+}
 __device__ __forceinline__ Row widen(const uint2* u) {
   Row r;
 #pragma unroll
@@ -75,10 +92,10 @@ __device__ __forceinline__ Row widen(const uint2* u) {
 // MODE 1: stride 2, dilation 1, same padding limit - the last row of an output is the first row
 //         of the next
 // MODE 2: anything else - three rows fetched per output row, each tap tested
-// ACT: activation applied right after the bias (the common fused case); a residual add or a
-// second activation takes the generic tail.
-template <int MODE, int ACT>
-__global__ void __launch_bounds__(256, 3) depthwise_f16_kernel(const __half* __restrict__ in, const float* __restrict__ w,
+// ACT: activation applied right after the bias (the common fused case); TAIL: a residual add
+// and / or a second activation follow.
+template <int MODE, int ACT, bool TAIL>
+__global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __restrict__ in, const float* __restrict__ w,
                                                                 const float* __restrict__ bias, const __half* __restrict__ res,
                                                                 __half* __restrict__ out, const DwGeom g, const Epilogue ep) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -146,7 +163,6 @@ __global__ void __launch_bounds__(256, 3) depthwise_f16_kernel(const __half* __r
   float2 blo = make_float2(0.f, 0.f), bhi = blo;
   int cur_s = -1;
   const int C4 = g.S * 4;
-  const bool tail = ep.has_res || ep.act_post != GI_ACT_NONE;
 
   for (int i = 0; i < count; ++i) {
     const int buf = i & 1;
@@ -208,6 +224,7 @@ __global__ void __launch_bounds__(256, 3) depthwise_f16_kernel(const __half* __r
       __syncthreads();
     }
 
+    const unsigned buf_addr = smem_u32(buf_base);
     const int cols = nbk * g.sub * Wo;
     for (int c = threadIdx.x; c < cols; c += blockDim.x) {
       const int x = c % Wo, vp = c / Wo;
@@ -215,15 +232,15 @@ __global__ void __launch_bounds__(256, 3) depthwise_f16_kernel(const __half* __r
       const int ya = oy0 + sb * g.tr, yb = min(oy1, ya + g.tr);
       if (ya >= yb) continue;
       // plane_zero: a pixel of the zero head; data: where pixel (0,0) of the plane would be staged
-      const __half* plane_zero = reinterpret_cast<const __half*>(buf_base) + static_cast<size_t>(pi) * g.plane_stride_px * 4;
-      const __half* data = plane_zero + (g.head_px - start_px) * 4;
+      const unsigned plane_zero = buf_addr + static_cast<unsigned>(pi) * g.plane_stride_px * 8u;
+      const unsigned data = plane_zero + static_cast<unsigned>(g.head_px - start_px) * 8u;
       const size_t out_off = ((static_cast<size_t>(s) * g.B + b0 + pi) * g.Pout + static_cast<size_t>(ya) * Wo + x) * 4;
       __half* op = out + out_off;
-      const __half* rp = res + out_off;
+      const ptrdiff_t res_minus_out = res - out;  // only used when TAIL
       const int out_stride = Wo * 4;
       auto emit = [&](const Acc& a) {
         uint2 u;
-        if (!tail) {
+        if (!TAIL) {
           // clamping after the rounding equals rounding after the clamp: 0 and 6 are fp16 values
           __half2 lo = __floats2half2_rn(a.lo.x, a.lo.y), hi = __floats2half2_rn(a.hi.x, a.hi.y);
           if (ACT != GI_ACT_NONE) {
@@ -243,7 +260,7 @@ __global__ void __launch_bounds__(256, 3) depthwise_f16_kernel(const __half* __r
 #pragma unroll
           for (int e = 0; e < 4; ++e) v[e] = act1(v[e], ACT);
           if (ep.has_res) {
-            const uint2 q = *reinterpret_cast<const uint2*>(rp);
+            const uint2 q = *reinterpret_cast<const uint2*>(op + res_minus_out);
             const float2 r0 = __half22float2(*reinterpret_cast<const __half2*>(&q.x));
             const float2 r1 = __half22float2(*reinterpret_cast<const __half2*>(&q.y));
             v[0] += r0.x;
@@ -259,71 +276,64 @@ __global__ void __launch_bounds__(256, 3) depthwise_f16_kernel(const __half* __r
         }
         *reinterpret_cast<uint2*>(op) = u;
         op += out_stride;
-        rp += out_stride;
       };
       const Acc bias_acc = {blo, bhi};
 
       if (MODE != 2) {
         // one pointer per tap column, walking down the staged rows; a column outside the image
         // stays on a zero pixel
-        const __half* tp[3];
-        int step[3];
+        unsigned tp[3], step[3];
         const int iy_first = ya * stride - pt;
 #pragma unroll
         for (int k = 0; k < 3; ++k) {
           const int ix = x * stride - g.pl + k;
           const bool v = ix >= 0 && ix < W;
-          tp[k] = v ? data + (iy_first * W + ix) * 4 : plane_zero;
-          step[k] = v ? W * 4 : 0;
+          tp[k] = v ? data + static_cast<unsigned>((iy_first * W + ix) * 8) : plane_zero;
+          step[k] = v ? static_cast<unsigned>(W) * 8u : 0u;
         }
         auto next_row = [&]() {
           uint2 u[3];
 #pragma unroll
           for (int k = 0; k < 3; ++k) {
-            u[k] = *reinterpret_cast<const uint2*>(tp[k]);
+            u[k] = lds64(tp[k]);
             tp[k] += step[k];
           }
           return widen(u);
         };
         if (MODE == 0) {
-          Acc a0 = bias_acc, a1 = bias_acc, a2;
+          Acc a0, a1, a2;
           Row r = next_row();
-          fma_row(a0, r, wlo, whi);  // output ya, kernel row 0
+          a0 = fma_row_from(bias_acc, r, wlo, whi);  // output ya, kernel row 0
           r = next_row();
-          fma_row(a0, r, wlo + 3, whi + 3);  // output ya, kernel row 1
-          fma_row(a1, r, wlo, whi);          // output ya+1, kernel row 0
+          fma_row(a0, r, wlo + 3, whi + 3);          // output ya, kernel row 1
+          a1 = fma_row_from(bias_acc, r, wlo, whi);  // output ya+1, kernel row 0
           for (int oy = ya; oy < yb; oy += 3) {
             r = next_row();
             fma_row(a0, r, wlo + 6, whi + 6);
             emit(a0);
             fma_row(a1, r, wlo + 3, whi + 3);
-            a2 = bias_acc;
-            fma_row(a2, r, wlo, whi);
+            a2 = fma_row_from(bias_acc, r, wlo, whi);
             if (oy + 1 >= yb) break;
             r = next_row();
             fma_row(a1, r, wlo + 6, whi + 6);
             emit(a1);
             fma_row(a2, r, wlo + 3, whi + 3);
-            a0 = bias_acc;
-            fma_row(a0, r, wlo, whi);
+            a0 = fma_row_from(bias_acc, r, wlo, whi);
             if (oy + 2 >= yb) break;
             r = next_row();
             fma_row(a2, r, wlo + 6, whi + 6);
             emit(a2);
             fma_row(a0, r, wlo + 3, whi + 3);
-            a1 = bias_acc;
-            fma_row(a1, r, wlo, whi);
+            a1 = fma_row_from(bias_acc, r, wlo, whi);
           }
         } else {
-          Acc carry = bias_acc;
-          fma_row(carry, next_row(), wlo, whi);
+          Acc carry = fma_row_from(bias_acc, next_row(), wlo, whi);
           for (int oy = ya; oy < yb; ++oy) {
             fma_row(carry, next_row(), wlo + 3, whi + 3);
             const Row r2 = next_row();
             fma_row(carry, r2, wlo + 6, whi + 6);
             emit(carry);
-            carry = bias_acc;
-            fma_row(carry, r2, wlo, whi);
+            carry = fma_row_from(bias_acc, r2, wlo, whi);
           }
         }
       } else {
@@ -339,7 +349,7 @@ __global__ void __launch_bounds__(256, 3) depthwise_f16_kernel(const __half* __r
           const bool vy = iy >= 0 && iy < H;
 #pragma unroll
           for (int k = 0; k < 3; ++k)
-            u[k] = (vy && vx[k]) ? *reinterpret_cast<const uint2*>(data + (iy * W + ix[k]) * 4) : make_uint2(0u, 0u);
+            u[k] = (vy && vx[k]) ? lds64(data + static_cast<unsigned>((iy * W + ix[k]) * 8)) : make_uint2(0u, 0u);
           return widen(u);
         };
         for (int oy = ya; oy < yb; ++oy) {
@@ -439,7 +449,9 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
   // persistent CTAs, a few per SM so that one CTA's copies overlap another's arithmetic
   long long ctas_per_sm = static_cast<long long>(kMaxSmem) / static_cast<long long>(smem > 0 ? smem : 1);
   if (ctas_per_sm > 2048 / threads) ctas_per_sm = 2048 / threads;
-  if (ctas_per_sm > 3) ctas_per_sm = 3;
+  // the grid is oversubscribed 2x: the block scheduler then evens out the tail
+  ctas_per_sm *= 2;
+  if (ctas_per_sm > 6) ctas_per_sm = 6;
   if (ctas_per_sm < 1) ctas_per_sm = 1;
   long long grid = static_cast<long long>(sms) * ctas_per_sm;
   if (grid > items) grid = items;
@@ -454,25 +466,35 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
   const float* b = static_cast<const float*>(p.bias);
   const __half* res = static_cast<const __half*>(p.res);
   __half* out = static_cast<__half*>(p.out);
-  static bool attr_done[3][3] = {};
-#define GI_DW_LAUNCH(M, A)                                                                                                       \
-  do {                                                                                                                           \
-    if (!attr_done[M][A]) {                                                                                                      \
-      const cudaError_t e = cudaFuncSetAttribute(depthwise_f16_kernel<M, A>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem); \
-      if (e != cudaSuccess) return static_cast<int>(e);                                                                          \
-      attr_done[M][A] = true;                                                                                                    \
-    }                                                                                                                            \
-    depthwise_f16_kernel<M, A><<<static_cast<unsigned>(grid), threads, smem, st>>>(in, w, b, res, out, g, r.ep);                 \
+  static bool attr_done[3][3][2] = {};
+  const bool tail = r.ep.has_res || r.ep.act_post != GI_ACT_NONE;
+#define GI_DW_LAUNCH(M, A, T)                                                                                                 \
+  do {                                                                                                                        \
+    if (!attr_done[M][A][T]) {                                                                                                \
+      const cudaError_t e =                                                                                                   \
+          cudaFuncSetAttribute(depthwise_f16_kernel<M, A, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);         \
+      if (e != cudaSuccess) return static_cast<int>(e);                                                                       \
+      attr_done[M][A][T] = true;                                                                                              \
+    }                                                                                                                         \
+    depthwise_f16_kernel<M, A, T><<<static_cast<unsigned>(grid), threads, smem, st>>>(in, w, b, res, out, g, r.ep);           \
   } while (0)
-#define GI_DW_MODE(M)                 \
-  do {                                \
-    if (act == GI_ACT_RELU6) {        \
-      GI_DW_LAUNCH(M, GI_ACT_RELU6);  \
-    } else if (act == GI_ACT_RELU) {  \
-      GI_DW_LAUNCH(M, GI_ACT_RELU);   \
-    } else {                          \
-      GI_DW_LAUNCH(M, GI_ACT_NONE);   \
-    }                                 \
+#define GI_DW_ACT(M, A)       \
+  do {                        \
+    if (tail) {               \
+      GI_DW_LAUNCH(M, A, 1);  \
+    } else {                  \
+      GI_DW_LAUNCH(M, A, 0);  \
+    }                         \
+  } while (0)
+#define GI_DW_MODE(M)              \
+  do {                             \
+    if (act == GI_ACT_RELU6) {     \
+      GI_DW_ACT(M, GI_ACT_RELU6);  \
+    } else if (act == GI_ACT_RELU) { \
+      GI_DW_ACT(M, GI_ACT_RELU);   \
+    } else {                       \
+      GI_DW_ACT(M, GI_ACT_NONE);   \
+    }                              \
   } while (0)
   if (mode == 0) {
     GI_DW_MODE(0);
@@ -482,6 +504,7 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
     GI_DW_MODE(2);
   }
 #undef GI_DW_MODE
+#undef GI_DW_ACT
 #undef GI_DW_LAUNCH
   return static_cast<int>(cudaGetLastError());
 }
