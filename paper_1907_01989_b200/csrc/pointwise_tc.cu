@@ -199,6 +199,8 @@ static_assert(sizeof(SmemHeader) <= kSmemHeader, "header too large");
 
 enum : unsigned { kErrProducer = 1u, kErrMma = 2u, kErrEpilogue = 4u, kErrDrain = 8u };
 
+// ACT: activation right after the bias; TAIL: a residual add and / or a second activation follow
+template <int ACT, bool TAIL>
 __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const TcParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   SmemHeader* hdr = reinterpret_cast<SmemHeader*>(smem);
@@ -337,30 +339,37 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
           for (int j = 0; j < 2; ++j) {
             const int so = nt * p.nts + 2 * c + j;
             if (so >= p.s_out || !row_ok) continue;
-            float v[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[8 * j + i]);
-            v[0] += b[j].x; v[1] += b[j].y; v[2] += b[j].z; v[3] += b[j].w;
-            v[4] += b[j].x; v[5] += b[j].y; v[6] += b[j].z; v[7] += b[j].w;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = act1(v[i], p.act_pre);
             const size_t off = (static_cast<size_t>(so) * p.m_total_px + 2u * row) * 4u;  // in halves
-            if (p.has_res) {
-              const uint4 rr = __ldg(reinterpret_cast<const uint4*>(p.res + off));
+            // columns 8j..8j+7: channels 0-3 of the even pixel, then of the odd pixel; bias per channel
+            const float2 b01 = make_float2(b[j].x, b[j].y), b23 = make_float2(b[j].z, b[j].w);
+            float2 v[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              v[i] = __fadd2_rn(make_float2(__uint_as_float(r[8 * j + 2 * i]), __uint_as_float(r[8 * j + 2 * i + 1])),
+                                (i & 1) ? b23 : b01);
+            uint4 o;
+            __half2* oh = reinterpret_cast<__half2*>(&o);
+            if (!TAIL) {
+              // clamping after the rounding equals rounding after the clamp: 0 and 6 are fp16 values
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                __half2 h = __floats2half2_rn(v[i].x, v[i].y);
+                if (ACT != GI_ACT_NONE) h = __hmax2(h, __float2half2_rn(0.f));
+                if (ACT == GI_ACT_RELU6) h = __hmin2(h, __float2half2_rn(6.f));
+                oh[i] = h;
+              }
+            } else {
+              uint4 rr = make_uint4(0u, 0u, 0u, 0u);
+              if (p.has_res) rr = __ldg(reinterpret_cast<const uint4*>(p.res + off));
               const __half2* rh = reinterpret_cast<const __half2*>(&rr);
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
-                const float2 f = __half22float2(rh[i]);
-                v[2 * i] += f.x;
-                v[2 * i + 1] += f.y;
+                const float2 f = __half22float2(rh[i]);  // zero when there is no residual
+                const float x = act1(act1(v[i].x, ACT) + f.x, p.act_post);
+                const float y = act1(act1(v[i].y, ACT) + f.y, p.act_post);
+                oh[i] = __floats2half2_rn(x, y);
               }
             }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = act1(v[i], p.act_post);
-            uint4 o;
-            __half2* oh = reinterpret_cast<__half2*>(&o);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) oh[i] = __floats2half2_rn(v[2 * i], v[2 * i + 1]);
             *reinterpret_cast<uint4*>(p.out + off) = o;
           }
         };
@@ -510,8 +519,17 @@ int launch_pointwise_tc(const LaunchRec& r, const Ptrs& p, void** state, int lau
       return static_cast<int>(cudaErrorInvalidDevice);
   }
   if (!di.attr_set) {
-    const cudaError_t e = cudaFuncSetAttribute(pointwise_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               kSmemHeader + kSmemBudget);
+    cudaError_t e = cudaSuccess;
+    const int bytes = kSmemHeader + kSmemBudget;
+#define GI_TC_ATTR(A, T) \
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(pointwise_tc_kernel<A, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)
+    GI_TC_ATTR(GI_ACT_NONE, false);
+    GI_TC_ATTR(GI_ACT_RELU, false);
+    GI_TC_ATTR(GI_ACT_RELU6, false);
+    GI_TC_ATTR(GI_ACT_NONE, true);
+    GI_TC_ATTR(GI_ACT_RELU, true);
+    GI_TC_ATTR(GI_ACT_RELU6, true);
+#undef GI_TC_ATTR
     if (e != cudaSuccess) return static_cast<int>(e);
     di.attr_set = true;
   }
@@ -569,7 +587,19 @@ int launch_pointwise_tc(const LaunchRec& r, const Ptrs& p, void** state, int lau
   const long long units = static_cast<long long>(k.m_tiles) * groups;
   const unsigned grid = static_cast<unsigned>(units < di.sms ? units : di.sms);
   const size_t smem = kSmemHeader + static_cast<size_t>(t.stages) * t.kc * (kSliceBytes + t.nts * kCoreBytes);
-  pointwise_tc_kernel<<<grid, kThreads, smem, static_cast<cudaStream_t>(stream)>>>(me.map, k);
+  const bool tail = k.has_res || k.act_post != GI_ACT_NONE;
+  cudaStream_t cu_stream = static_cast<cudaStream_t>(stream);
+#define GI_TC_LAUNCH(A, T) pointwise_tc_kernel<A, T><<<grid, kThreads, smem, cu_stream>>>(me.map, k)
+  if (tail) {
+    if (k.act_pre == GI_ACT_RELU6) GI_TC_LAUNCH(GI_ACT_RELU6, true);
+    else if (k.act_pre == GI_ACT_RELU) GI_TC_LAUNCH(GI_ACT_RELU, true);
+    else GI_TC_LAUNCH(GI_ACT_NONE, true);
+  } else {
+    if (k.act_pre == GI_ACT_RELU6) GI_TC_LAUNCH(GI_ACT_RELU6, false);
+    else if (k.act_pre == GI_ACT_RELU) GI_TC_LAUNCH(GI_ACT_RELU, false);
+    else GI_TC_LAUNCH(GI_ACT_NONE, false);
+  }
+#undef GI_TC_LAUNCH
   return static_cast<int>(cudaGetLastError());
 }
 
