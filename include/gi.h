@@ -82,10 +82,10 @@ enum {
   GI_PLAN_NAIVE = 2                  /* every tensor its own memory (the paper's baseline) */
 };
 
-/* Pointwise (1x1 convolution) kernel choice. */
+/* Kernel choice for full convolutions (1x1, and 3x3 with at most 4 input channels). */
 enum {
-  GI_PW_AUTO = 0,      /* tensor-core kernel for fp16 storage, SIMT kernel for fp32 storage */
-  GI_PW_SIMT = 1       /* force the plain CUDA-core kernel (validation) */
+  GI_PW_AUTO = 0,      /* tensor-core kernels for fp16 storage, CUDA-core kernel for fp32 storage */
+  GI_PW_SIMT = 1       /* force the plain CUDA-core kernel for every full convolution (validation) */
 };
 
 /*
@@ -160,7 +160,7 @@ typedef struct gi_op_info {
 enum { GI_EXEC_PACK = 100, GI_EXEC_UNPACK = 101 };
 enum {
   GI_KERNEL_PACK = 1, GI_KERNEL_UNPACK = 2, GI_KERNEL_CONV_SIMT = 3, GI_KERNEL_POINTWISE_TC = 4,
-  GI_KERNEL_DEPTHWISE = 5, GI_KERNEL_ELTWISE = 6, GI_KERNEL_POOL = 7, GI_KERNEL_RESIZE = 8
+  GI_KERNEL_DEPTHWISE = 5, GI_KERNEL_ELTWISE = 6, GI_KERNEL_POOL = 7, GI_KERNEL_RESIZE = 8, GI_KERNEL_CONV3X3_TC = 9
 };
 
 /* ---- graph construction (Section 3.1, "Initialization": the sub-graph given to the GPU backend) ---- */
@@ -247,7 +247,8 @@ GI_API gi_status gi_run_timed(gi_exec* e, const void* const* dev_inputs, void* c
 
 /* Health word of the device-side waits.  The tensor-core kernel waits on copy and MMA
  * completion with a limit of about one second per wait; a wait that runs out sets a bit here
- * (1 producer, 2 MMA issuer, 4 epilogue, 8 drain; 0x10000 depthwise staging copy), lets the
+ * (1 producer, 2 MMA issuer, 4 epilogue, 8 drain; 0x10000 depthwise staging copy;
+ * 0x200000 / 0x400000 MMA issuer / epilogue of the 3x3 tensor-core kernel), lets the
  * kernel finish without its results
  * and leaves the CUDA context usable.  Sticky until the process exits.  Synchronous: copies
  * the word from the current device. */

@@ -171,6 +171,11 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
               pointwise_tc_supported(din->c, op.d.cout)) {
             r.kernel = GI_KERNEL_POINTWISE_TC;
             pointwise_tc_pack(op.weights.data(), op.bias.data(), din->c, op.d.cout, &e->weight_blob, &r);
+          } else if (e->storage == GI_F16 && e->opt.pointwise == GI_PW_AUTO &&
+                     conv3x3_tc_supported(din->c, op.d.cout, op.d.kh, op.d.kw, op.d.stride_h, op.d.stride_w,
+                                          op.d.dilation_h, op.d.dilation_w)) {
+            r.kernel = GI_KERNEL_CONV3X3_TC;
+            conv3x3_tc_pack(op.weights.data(), op.bias.data(), din->c, op.d.cout, &e->weight_blob, &r);
           } else {
             r.kernel = GI_KERNEL_CONV_SIMT;
             const int sout = slices(op.d.cout);

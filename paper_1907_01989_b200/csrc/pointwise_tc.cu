@@ -29,6 +29,7 @@
 #include <vector>
 
 #include "kernels.h"
+#include "sm100_ptx.cuh"
 
 namespace gi {
 namespace {
@@ -63,123 +64,7 @@ struct TcParams {
   unsigned int timeout_ns;
 };
 
-// ------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ unsigned smem_u32(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(unsigned bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
-  unsigned ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_timer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-
-// Bounded wait.  Returns false if the CTA is aborting or the limit ran out (then it raises the
-// abort flag and the error word itself).
-__device__ __noinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile unsigned* abort_flag, unsigned timeout_ns,
-                                       unsigned code) {
-  unsigned long long t0 = 0;
-  for (unsigned spin = 0;; ++spin) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((spin & 255u) == 255u) {
-      if (*abort_flag) return false;
-      const unsigned long long now = global_timer_ns();
-      if (t0 == 0) {
-        t0 = now;
-      } else if (now - t0 > timeout_ns) {
-        *abort_flag = 1;
-        atomicOr(&g_tc_error, code);
-        return false;
-      }
-    }
-  }
-}
-
-__device__ __forceinline__ void tma_load_2d(unsigned dst, const CUtensorMap* map, int x, int y, unsigned bar) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-               "l"(reinterpret_cast<unsigned long long>(map)), "r"(x), "r"(y), "r"(bar)
-               : "memory");
-}
-__device__ __forceinline__ void bulk_load(unsigned dst, const void* src, unsigned bytes, unsigned bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src),
-               "r"(bytes), "r"(bar)
-               : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc(unsigned smem_dst, unsigned cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(unsigned taddr, unsigned cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-
-// D[tmem] (+)= A[smem] * B[smem]^T, 128 x N x 16, fp16 operands, fp32 accumulate
-__device__ __forceinline__ void umma_f16(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc, unsigned idesc,
-                                         unsigned accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// arrive on an mbarrier once every MMA issued so far by this thread has completed
-__device__ __forceinline__ void umma_commit(unsigned bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-// Shared-memory operand descriptor: K-major, no swizzle.  Core matrices are 8 rows x 16 bytes,
-// stored as 128 contiguous bytes; `lbo` is the byte distance between the two core matrices
-// an MMA reads along K, `sbo` the distance between consecutive 8-row groups.
-__device__ __forceinline__ unsigned long long smem_desc(unsigned addr, unsigned lbo, unsigned sbo) {
-  unsigned long long d = 0;
-  d |= static_cast<unsigned long long>((addr & 0x3ffffu) >> 4);
-  d |= static_cast<unsigned long long>((lbo >> 4) & 0x3fffu) << 16;
-  d |= static_cast<unsigned long long>((sbo >> 4) & 0x3fffu) << 32;
-  d |= 1ull << 46;  // descriptor version of this architecture
-  return d;         // base offset 0, layout type 0 (no swizzle)
-}
-
-// 32 lanes x 16 consecutive 32-bit columns: thread t of the warp receives lane (quarter*32 + t)
-__device__ __forceinline__ void tmem_ld16(unsigned taddr, unsigned* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
-        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-}
-// wait for every tensor-memory load issued so far; the registers of the chunk about to be used
-// are operands so that no use of them can be scheduled above the wait
-__device__ __forceinline__ void tmem_ld_wait16(unsigned* r) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
-                 "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
-               :
-               : "memory");
-}
+using namespace ptx;
 
 __device__ __forceinline__ float act1(float v, int kind) {
   if (kind == GI_ACT_RELU) return fmaxf(v, 0.0f);
@@ -242,7 +127,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
         for (int nt = grp; nt < p.n_tiles && ok; nt += p.groups) {
           for (int kc_i = 0; kc_i < p.k_chunks; ++kc_i, ++it) {
             const unsigned stage = it % p.stages, phase = (it / p.stages) & 1u;
-            if (!mbar_wait(smem_u32(&hdr->empty[stage]), phase ^ 1u, abort_flag, p.timeout_ns, kErrProducer)) {
+            if (!mbar_wait(smem_u32(&hdr->empty[stage]), phase ^ 1u, abort_flag, p.timeout_ns, &g_tc_error, kErrProducer)) {
               ok = false;
               break;
             }
@@ -282,7 +167,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
         const int m_tile = u / p.groups, grp = u - m_tile * p.groups;
         for (int nt = grp; nt < p.n_tiles && ok; nt += p.groups, ++tile) {
           const unsigned acc = tile & 1u, acc_phase = (tile >> 1) & 1u;
-          if (!mbar_wait(smem_u32(&hdr->acc_empty[acc]), acc_phase ^ 1u, abort_flag, p.timeout_ns, kErrMma)) {
+          if (!mbar_wait(smem_u32(&hdr->acc_empty[acc]), acc_phase ^ 1u, abort_flag, p.timeout_ns, &g_tc_error, kErrMma)) {
             ok = false;
             break;
           }
@@ -290,7 +175,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
           const unsigned d_tmem = tmem_base + acc * acc_cols;
           for (int kc_i = 0; kc_i < p.k_chunks; ++kc_i, ++it) {
             const unsigned stage = it % p.stages, phase = (it / p.stages) & 1u;
-            if (!mbar_wait(smem_u32(&hdr->full[stage]), phase, abort_flag, p.timeout_ns, kErrMma)) {
+            if (!mbar_wait(smem_u32(&hdr->full[stage]), phase, abort_flag, p.timeout_ns, &g_tc_error, kErrMma)) {
               ok = false;
               break;
             }
@@ -321,7 +206,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
       const bool row_ok = row < rows_total;
       for (int nt = grp; nt < p.n_tiles && ok; nt += p.groups, ++tile) {
         const unsigned acc = tile & 1u, acc_phase = (tile >> 1) & 1u;
-        if (!mbar_wait(smem_u32(&hdr->acc_full[acc]), acc_phase, abort_flag, p.timeout_ns, kErrEpilogue)) {
+        if (!mbar_wait(smem_u32(&hdr->acc_full[acc]), acc_phase, abort_flag, p.timeout_ns, &g_tc_error, kErrEpilogue)) {
           ok = false;
           break;
         }
