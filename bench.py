@@ -62,7 +62,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                          "--format=csv,noheader,nounits", "-lms", "20"], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -157,6 +157,8 @@ def run_sweep(args):
     stream = torch.cuda.current_stream()
     if args.points:
         points = [tuple(int(v) for v in pt.split(",")) for pt in args.points.split(";") if pt]
+    elif args.sweep == "conv3":
+        points = [(256, 224, 3, 32, 2), (64, 224, 3, 32, 2), (16, 513, 3, 32, 2), (1, 224, 3, 32, 2)]
     elif args.sweep == "dw":
         points = [(b, hw, c, s) for b in (64, 256) for hw, c in ((112, 32), (112, 96), (56, 144), (28, 192), (14, 384),
                                                                  (14, 576), (7, 960)) for s in (1, 2)]
@@ -167,7 +169,11 @@ def run_sweep(args):
                   (256, 14, 1280, 1280), (64, 56, 192, 192), (8, 28, 384, 384), (1, 14, 96, 576)]
     rows = []
     for pt in points:
-        if args.sweep == "dw":
+        if args.sweep == "conv3":
+            b, hw, cin, cout, stride = pt
+            spec = wl.single_conv3x3(b, hw, cin, cout, stride)
+            name = f"conv3x3 b{b} {hw}x{hw} {cin}->{cout} s{stride}"
+        elif args.sweep == "dw":
             b, hw, c, stride = pt
             spec = wl.single_depthwise(b, hw, c, stride, 1, residual=args.residual)
             name = f"dw3x3 b{b} {hw}x{hw}x{c} s{stride}"
@@ -215,7 +221,7 @@ def run_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--net", default="v2", choices=sorted(NETS))
@@ -223,7 +229,9 @@ def main():
     ap.add_argument("--pointwise", default="auto", choices=["auto", "simt"])
     ap.add_argument("--per-op", default=None, help="write the per-op timing table to this file")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--sweep", default=None, choices=["pw", "dw"], help="time single fused operators instead of a network")
+    ap.add_argument("--no-batch1", action="store_true", help="skip the batch-1 latency leg (keeps profiler runs short)")
+    ap.add_argument("--sweep", default=None, choices=["pw", "dw", "conv3"],
+                    help="time single fused operators instead of a network")
     ap.add_argument("--points", default=None, help="sweep points 'B,HW,Cin,Cout;...' (pw) or 'B,HW,C,stride;...' (dw)")
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--residual", action="store_true")
@@ -381,42 +389,44 @@ def main():
                              f"{t:.4f} {o.bytes / t / 1e6:.0f} {o.flops / t / 1e9:.1f} {roof / t:.3f}\n".replace(", ", ","))
 
         # ---- batch-1 latency (the paper's protocol: 10 warm-up runs, mean of the next 100) ----
-        spec1 = spec_fn(1)
-        g1, _ = api.graph_from_spec(spec1, api.GI_F16)
-        ex1 = g1.compile(pointwise=api.GI_PW_SIMT if args.pointwise == "simt" else api.GI_PW_AUTO)
-        ex1.bind(dev)
-        x1 = torch.from_numpy(wl.make_input(spec1).astype(np.float16)).to(dev)
-        o1 = torch.empty((1,) + tuple(spec1.shapes[spec1.outputs[0]]), dtype=torch.float16, device=dev)
-        for _ in range(10):
-            ex1.run([x1], [o1], stream)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        a.record(stream)
-        for _ in range(100):
-            ex1.run([x1], [o1], stream)
-        b.record(stream)
-        torch.cuda.synchronize()
-        b1_ms = a.elapsed_time(b) / 100
-        side = torch.cuda.Stream()
-        graph_ms = None
-        try:
-            with torch.cuda.stream(side):
-                ex1.run([x1], [o1], side)
-                side.synchronize()
-                cg = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(cg, stream=side):
-                    ex1.run([x1], [o1], torch.cuda.current_stream())
-                for _ in range(10):
-                    cg.replay()
-                side.synchronize()
-                a.record(side)
-                for _ in range(100):
-                    cg.replay()
-                b.record(side)
-                side.synchronize()
-                graph_ms = a.elapsed_time(b) / 100
-        except Exception as exc:  # graph capture is an extra, never the headline
-            graph_ms = f"capture failed: {type(exc).__name__}"
+        b1_ms, graph_ms, b1_launches = None, None, None
+        if not args.no_batch1:
+            spec1 = spec_fn(1)
+            g1, _ = api.graph_from_spec(spec1, api.GI_F16)
+            ex1 = g1.compile(pointwise=api.GI_PW_SIMT if args.pointwise == "simt" else api.GI_PW_AUTO)
+            ex1.bind(dev)
+            x1 = torch.from_numpy(wl.make_input(spec1).astype(np.float16)).to(dev)
+            o1 = torch.empty((1,) + tuple(spec1.shapes[spec1.outputs[0]]), dtype=torch.float16, device=dev)
+            for _ in range(10):
+                ex1.run([x1], [o1], stream)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record(stream)
+            for _ in range(100):
+                ex1.run([x1], [o1], stream)
+            b.record(stream)
+            torch.cuda.synchronize()
+            b1_ms = a.elapsed_time(b) / 100
+            side = torch.cuda.Stream()
+            try:
+                with torch.cuda.stream(side):
+                    ex1.run([x1], [o1], side)
+                    side.synchronize()
+                    cg = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(cg, stream=side):
+                        ex1.run([x1], [o1], torch.cuda.current_stream())
+                    for _ in range(10):
+                        cg.replay()
+                    side.synchronize()
+                    a.record(side)
+                    for _ in range(100):
+                        cg.replay()
+                    b.record(side)
+                    side.synchronize()
+                    graph_ms = a.elapsed_time(b) / 100
+            except Exception as exc:  # graph capture is an extra, never the headline
+                graph_ms = f"capture failed: {type(exc).__name__}"
+            b1_launches = int(ex1.info.n_ops)
 
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
@@ -435,7 +445,7 @@ def main():
                 "e2e": {"value": e2e_value, "unit": "images/s", "h2d_bytes_per_step": int(x_pin.numel() * 2),
                         "d2h_bytes_per_step": int(out_pin.numel() * 2)},
                 "gpu_launches": args.steps * len(ops), "clocks": clocks,
-                "batch1": {"ms": b1_ms, "cuda_graph_ms": graph_ms, "launches": int(ex1.info.n_ops),
+                "batch1": {"ms": b1_ms, "cuda_graph_ms": graph_ms, "launches": b1_launches,
                            "protocol": "10 warm-up runs, mean of the next 100"},
                 "step_ms_min_median_max": [min(ms), statistics.median(ms), max(ms)], "wall_s_timed_region": wall,
                 "logits_abs_mean": logits_checksum}
