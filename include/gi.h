@@ -85,7 +85,9 @@ enum {
 /* Kernel choice for full convolutions (1x1, and 3x3 with at most 4 input channels). */
 enum {
   GI_PW_AUTO = 0,      /* tensor-core kernels for fp16 storage, CUDA-core kernel for fp32 storage */
-  GI_PW_SIMT = 1       /* force the plain CUDA-core kernel for every full convolution (validation) */
+  GI_PW_SIMT = 1,      /* force the plain CUDA-core kernel for every full convolution (validation) */
+  GI_PW_TC_PAIR = 2,   /* 1x1: always the pixel-pair tensor-core kernel (operands by TMA) */
+  GI_PW_TC_LANE = 3    /* 1x1: always the lane-per-pixel tensor-core kernel (activations through tensor memory) */
 };
 
 /*
@@ -160,7 +162,7 @@ typedef struct gi_op_info {
 enum { GI_EXEC_PACK = 100, GI_EXEC_UNPACK = 101 };
 enum {
   GI_KERNEL_PACK = 1, GI_KERNEL_UNPACK = 2, GI_KERNEL_CONV_SIMT = 3, GI_KERNEL_POINTWISE_TC = 4,
-  GI_KERNEL_DEPTHWISE = 5, GI_KERNEL_ELTWISE = 6, GI_KERNEL_POOL = 7, GI_KERNEL_RESIZE = 8, GI_KERNEL_CONV3X3_TC = 9
+  GI_KERNEL_DEPTHWISE = 5, GI_KERNEL_ELTWISE = 6, GI_KERNEL_POOL = 7, GI_KERNEL_RESIZE = 8, GI_KERNEL_CONV3X3_TC = 9, GI_KERNEL_POINTWISE_TS = 10
 };
 
 /* ---- graph construction (Section 3.1, "Initialization": the sub-graph given to the GPU backend) ---- */
@@ -248,7 +250,8 @@ GI_API gi_status gi_run_timed(gi_exec* e, const void* const* dev_inputs, void* c
 /* Health word of the device-side waits.  The tensor-core kernel waits on copy and MMA
  * completion with a limit of about one second per wait; a wait that runs out sets a bit here
  * (1 producer, 2 MMA issuer, 4 epilogue, 8 drain; 0x10000 depthwise staging copy;
- * 0x200000 / 0x400000 MMA issuer / epilogue of the 3x3 tensor-core kernel), lets the
+ * 0x200000 / 0x400000 MMA issuer / epilogue of the 3x3 tensor-core kernel; 0x1000000..0x8000000
+ * producer / MMA issuer / data warps / drain of the lane-per-pixel 1x1 kernel), lets the
  * kernel finish without its results
  * and leaves the CUDA context usable.  Sticky until the process exits.  Synchronous: copies
  * the word from the current device. */

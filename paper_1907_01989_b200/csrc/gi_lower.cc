@@ -167,12 +167,17 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
         } else {
           const bool pointwise = op.d.kh == 1 && op.d.stride_h == 1 && op.d.stride_w == 1 && op.d.pad_t == 0 &&
                                  op.d.pad_l == 0 && op.d.pad_b == 0 && op.d.pad_r == 0;
-          if (pointwise && e->storage == GI_F16 && e->opt.pointwise == GI_PW_AUTO &&
-              pointwise_tc_supported(din->c, op.d.cout)) {
+          const bool tc = e->storage == GI_F16 && e->opt.pointwise != GI_PW_SIMT;
+          // many input channels: the lane-per-pixel kernel (dense weight tile); few: the pixel-pair
+          // kernel (activations by TMA)
+          const bool lane_kernel = e->opt.pointwise == GI_PW_TC_LANE || (e->opt.pointwise == GI_PW_AUTO && din->c >= 64);
+          if (pointwise && tc && lane_kernel && pointwise_ts_supported(din->c, op.d.cout)) {
+            r.kernel = GI_KERNEL_POINTWISE_TS;
+            pointwise_ts_pack(op.weights.data(), op.bias.data(), din->c, op.d.cout, &e->weight_blob, &r);
+          } else if (pointwise && tc && pointwise_tc_supported(din->c, op.d.cout)) {
             r.kernel = GI_KERNEL_POINTWISE_TC;
             pointwise_tc_pack(op.weights.data(), op.bias.data(), din->c, op.d.cout, &e->weight_blob, &r);
-          } else if (e->storage == GI_F16 && e->opt.pointwise == GI_PW_AUTO &&
-                     conv3x3_tc_supported(din->c, op.d.cout, op.d.kh, op.d.kw, op.d.stride_h, op.d.stride_w,
+          } else if (tc && conv3x3_tc_supported(din->c, op.d.cout, op.d.kh, op.d.kw, op.d.stride_h, op.d.stride_w,
                                           op.d.dilation_h, op.d.dilation_w)) {
             r.kernel = GI_KERNEL_CONV3X3_TC;
             conv3x3_tc_pack(op.weights.data(), op.bias.data(), din->c, op.d.cout, &e->weight_blob, &r);

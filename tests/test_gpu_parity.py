@@ -87,15 +87,25 @@ PW_CASES = [  # batch, hw, cin, cout, residual, act
 ]
 
 
-@pytest.mark.parametrize("storage", STORAGES)
 @pytest.mark.parametrize("case", PW_CASES)
-def test_pointwise(storage, case):
+def test_pointwise_fp32(case):
     batch, hw, cin, cout, residual, act = case
     spec = wl.single_pointwise(batch, hw, cin, cout, residual, act)
-    check_all_tensors(spec, storage)
-    # fp16 storage must take the tensor-core kernel, fp32 storage the CUDA-core one
-    kernels = [api.KERNEL_NAMES[o.kernel] for o in api.graph_from_spec(spec, storage)[0].compile().ops()]
-    assert ("pointwise_tc" in kernels) == (storage == api.GI_F16)
+    check_all_tensors(spec, api.GI_F32)
+    kernels = [api.KERNEL_NAMES[o.kernel] for o in api.graph_from_spec(spec, api.GI_F32)[0].compile().ops()]
+    assert "conv_simt" in kernels  # fp32 storage always takes the CUDA-core kernel
+
+
+@pytest.mark.parametrize("mode,kernel", [(api.GI_PW_TC_PAIR, "pointwise_tc"), (api.GI_PW_TC_LANE, "pointwise_ts")],
+                         ids=["pair", "lane"])
+@pytest.mark.parametrize("case", PW_CASES)
+def test_pointwise_tensor_core(case, mode, kernel):
+    """Both tensor-core variants on every case: operands by TMA (pixel pairs) and through tensor memory."""
+    batch, hw, cin, cout, residual, act = case
+    spec = wl.single_pointwise(batch, hw, cin, cout, residual, act)
+    check_all_tensors(spec, api.GI_F16, pointwise=mode)
+    kernels = [api.KERNEL_NAMES[o.kernel] for o in api.graph_from_spec(spec, api.GI_F16)[0].compile(pointwise=mode).ops()]
+    assert kernel in kernels
     assert api.gi_device_status() == 0
 
 
@@ -120,9 +130,17 @@ def test_depthwise(storage, case):
 
 
 @pytest.mark.parametrize("storage", STORAGES)
-@pytest.mark.parametrize("case", [(1, 32, 3, 32, 2), (2, 17, 3, 32, 2), (1, 12, 8, 12, 1), (2, 9, 5, 6, 2)])
+@pytest.mark.parametrize("case", [(1, 32, 3, 32, 2), (2, 17, 3, 32, 2), (1, 12, 8, 12, 1), (2, 9, 5, 6, 2), (3, 21, 4, 21, 1),
+                                  (1, 40, 2, 200, 2)])
 def test_conv3x3(storage, case):
-    check_all_tensors(wl.single_conv3x3(*case), storage)
+    spec = wl.single_conv3x3(*case)
+    check_all_tensors(spec, storage)
+    kernels = [api.KERNEL_NAMES[o.kernel] for o in api.graph_from_spec(spec, storage)[0].compile().ops()]
+    # one input slice and fp16 storage: the tensor-core kernel; anything else: the CUDA-core kernel
+    assert ("conv3x3_tc" in kernels) == (storage == api.GI_F16 and case[2] <= 4)
+    if storage == api.GI_F16:
+        check_all_tensors(spec, storage, pointwise=api.GI_PW_SIMT)
+    assert api.gi_device_status() == 0
 
 
 @pytest.mark.parametrize("storage", STORAGES)
@@ -149,6 +167,11 @@ def test_standalone_elementwise_pool_resize(storage):
 @pytest.mark.parametrize("make", [wl.mobilenet_v1, wl.mobilenet_v2], ids=["v1", "v2"])
 def test_network_batch1_every_tensor(make, storage):
     check_all_tensors(make(1), storage)
+
+
+@pytest.mark.parametrize("mode", [api.GI_PW_TC_PAIR, api.GI_PW_TC_LANE], ids=["pair", "lane"])
+def test_network_with_one_pointwise_variant(mode):
+    check_all_tensors(wl.mobilenet_v2(3, size=160), api.GI_F16, pointwise=mode)
 
 
 def test_segmentation_batch1_every_tensor():
