@@ -80,7 +80,7 @@ static gi_status run_impl(gi_exec* e, const void* const* dev_inputs, void* const
       case GI_KERNEL_CONV_SIMT: err = launch_conv_simt(r, p, e->storage, stream); break;
       case GI_KERNEL_POINTWISE_TC: err = launch_pointwise_tc(r, p, &e->tc_state, static_cast<int>(i), stream); break;
       case GI_KERNEL_CONV3X3_TC: err = launch_conv3x3_tc(r, p, stream); break;
-      case GI_KERNEL_POINTWISE_TS: err = launch_pointwise_ts(r, p, stream); break;
+      case GI_KERNEL_POINTWISE_TS: err = launch_pointwise_ts(r, p, &e->tc_state, static_cast<int>(i), stream); break;
       case GI_KERNEL_DEPTHWISE: err = launch_depthwise(r, p, e->storage, stream); break;
       case GI_KERNEL_ELTWISE:
         if (r.ep.has_res && !p.in1) p.in1 = p.res;

@@ -47,7 +47,7 @@ unsigned int conv3x3_tc_error_word(int* cuda_err);
 // Pointwise convolution with the activation operand in tensor memory (fp16 storage).
 bool pointwise_ts_supported(int cin, int cout);
 void pointwise_ts_pack(const float* w, const float* bias, int cin, int cout, std::vector<uint8_t>* blob, LaunchRec* r);
-int launch_pointwise_ts(const LaunchRec& r, const Ptrs& p, void* stream);
+int launch_pointwise_ts(const LaunchRec& r, const Ptrs& p, void** state, int launch_index, void* stream);
 unsigned int pointwise_ts_error_word(int* cuda_err);
 
 }  // namespace gi

@@ -30,6 +30,7 @@
 
 #include "kernels.h"
 #include "sm100_ptx.cuh"
+#include "tma_host.h"
 
 namespace gi {
 namespace {
@@ -312,31 +313,6 @@ Tiling choose_tiling(int cin, int cout) {
   return t;
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    void* f = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(f);
-  });
-  return fn;
-}
-
-struct MapEntry {
-  const void* in = nullptr;
-  CUtensorMap map;
-};
-struct TcState {
-  std::vector<MapEntry> maps;
-};
-
 struct DeviceInfo {
   int sms = 0;
   bool attr_set = false;
@@ -419,21 +395,10 @@ int launch_pointwise_tc(const LaunchRec& r, const Ptrs& p, void** state, int lau
     di.attr_set = true;
   }
   // tensor map over the input: pixels (8-byte elements) x slices; cached per launch and input address
-  if (!*state) *state = new TcState();
-  TcState* st = static_cast<TcState*>(*state);
-  if (st->maps.size() <= static_cast<size_t>(launch_index)) st->maps.resize(launch_index + 1);
-  MapEntry& me = st->maps[launch_index];
+  MapEntry& me = map_cache_entry(state, launch_index);
   if (me.in != p.in0) {
-    EncodeTiledFn enc = encode_fn();
-    if (!enc) return static_cast<int>(cudaErrorNotSupported);
-    const cuuint64_t gdim[2] = {m_total, static_cast<cuuint64_t>(t.s_in)};
-    const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(m_total) * 8u};
-    const cuuint32_t box[2] = {static_cast<cuuint32_t>(kTilePx), static_cast<cuuint32_t>(t.kc)};
-    const cuuint32_t estr[2] = {1, 1};
-    const CUresult cr = enc(&me.map, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void*>(p.in0), gdim, gstride, box, estr,
-                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (cr != CUDA_SUCCESS) return static_cast<int>(cudaErrorInvalidValue);
+    const int err = encode_plane_map(&me.map, p.in0, m_total, t.s_in, kTilePx, t.kc);
+    if (err != 0) return err;
     me.in = p.in0;
   }
   TcParams k;
@@ -488,7 +453,7 @@ int launch_pointwise_tc(const LaunchRec& r, const Ptrs& p, void** state, int lau
   return static_cast<int>(cudaGetLastError());
 }
 
-void pointwise_tc_release(void* state) { delete static_cast<TcState*>(state); }
+void pointwise_tc_release(void* state) { map_cache_release(state); }
 
 unsigned int pointwise_tc_error_word(int* cuda_err) {
   unsigned int v = 0;

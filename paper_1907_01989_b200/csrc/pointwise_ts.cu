@@ -1,28 +1,31 @@
-// Pointwise (1x1) convolution, second tensor-core variant: the activation operand goes through
-// registers into TENSOR MEMORY and the MMA reads it from there (tcgen05.mma with A in TMEM), the
-// weights come from shared memory, filled by bulk TMA copies.
+// Pointwise (1x1) convolution, second tensor-core variant: weights stationary in shared memory,
+// the activation operand in TENSOR MEMORY (tcgen05.mma with A in TMEM).
 //
-// Why a second variant: a pixel-slice is 4 fp16 = two 32-bit words, and a TMEM lane holds the K
-// axis of an fp16 A operand two elements per 32-bit column - so "lane = pixel, columns 2s, 2s+1 =
-// slice s" IS the operand layout.  A thread loads the 8 bytes of its pixel for a run of slices
-// (coalesced: a warp reads 256 contiguous bytes per slice) and writes them to its lane with
-// tcgen05.st.  Nothing is padded or duplicated, so the tensor pipe does exactly 2*M*N*K flops and
-// the weight operand is the dense [Cout][Cin] matrix.  The pixel-pair variant (pointwise_tc.cu)
-// keeps its place for small Cin, where its fully asynchronous TMA feed wins; this one takes the
-// layers with many input channels, where the pair variant's 4x larger expanded weight tile made
-// the shared-memory fill, not HBM, the bound.
+// A pixel-slice is 4 fp16 = two 32-bit words, and a TMEM lane holds the K axis of an fp16 A
+// operand two elements per 32-bit column - so "lane = pixel, columns 2s, 2s+1 = slice s" IS the
+// operand layout, with nothing padded or duplicated: the tensor pipe does exactly 2*M*N*K flops
+// and the weight operand is the dense [Cout][Cin] matrix, small enough to stay in shared memory
+// for the whole kernel (each CTA keeps the rows of its share of the output channels).  What
+// streams is the activation only: TMA boxes of 128 pixels x ks slices land in a ring of shared
+// memory stages, four transfer warps move a stage into tensor memory (8-byte ld.shared per lane,
+// tcgen05.st), and every byte of shared memory that is not weights is activation in flight -
+// which is what a layer bound by HBM latency x bandwidth needs.  The pixel-pair variant
+// (pointwise_tc.cu) keeps the layers with few input channels and large planes; this one takes
+// the layers where that variant's 4x expanded weight tile crowded the activations out of shared
+// memory.
 //
-// CTA = 10 warps: warp 0 streams weight chunks (TMA, mbarrier ring), warp 1 issues MMAs and owns
-// tensor memory, warps 2-9 are the data warps: two per TMEM lane quarter, each loading half of a
-// K chunk of the next tile and then draining half of the accumulator columns of the previous
-// tile (bias, activation, residual, fp16 pack, 8-byte stores: 256 contiguous bytes per warp).
-// Accumulators and A chunks are double-buffered in the 512 TMEM columns.  Waits are bounded.
+// CTA = 22 warps: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-5 transfer
+// (one TMEM lane quarter each), warps 6-21 drain the accumulator (four per quarter: bias,
+// activation, residual, fp16 pack, 8-byte stores, 256 contiguous bytes per warp).  Accumulators
+// and A chunks are double-buffered in the 512 TMEM columns.  If a CTA's weight share does not
+// fit, the weights stream through the same stages instead.  All waits are bounded.
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 #include "kernels.h"
 #include "sm100_ptx.cuh"
+#include "tma_host.h"
 
 namespace gi {
 namespace {
@@ -30,25 +33,27 @@ namespace {
 using namespace ptx;
 
 constexpr int kRows = 128;
-constexpr int kDataWarps = 8;
-constexpr int kThreads = 64 + 32 * kDataWarps;
-constexpr int kMaxStages = 4;
+constexpr int kTransferWarps = 4;
+constexpr int kDrainWarps = 16;
+constexpr int kThreads = 32 * (2 + kTransferWarps + kDrainWarps);
+constexpr int kMaxStages = 8;
 constexpr int kSmemHeader = 1024;
-constexpr int kSmemBudget = 200 * 1024;
-constexpr int kMaxNt = 192;
+constexpr int kSmemBudget = 208 * 1024;        // stages + resident weights
+constexpr int kResidentLimit = 144 * 1024;     // weights larger than this stream through the stages
+constexpr int kMaxNcta = 192;
 
 __device__ unsigned int g_ts_error = 0;
 
 struct TsParams {
-  const __half* in;
   const __half* res;
   __half* out;
   const float* bias;
   const unsigned char* wts;
   unsigned int m_total_px;
-  int s_in, s_out;
-  int ks, n_chunks;      // input slices per K chunk (multiple of 4), chunks per tile
-  int n_t, n_tiles;      // output channels per tile (multiple of 16), tiles along N
+  int s_out;
+  int ks, n_chunks;      // input slices per A chunk (multiple of 8), chunks per pixel tile
+  int n_cta, n_parts;    // output channels per CTA (multiple of 16), CTAs sharing one pixel tile
+  int b_resident;        // 1: the CTA's weights are loaded once; 0: a weight chunk rides in every stage
   int stages;
   int m_tiles;
   int has_res, act_post;
@@ -56,15 +61,17 @@ struct TsParams {
 };
 
 struct Header {
-  unsigned long long b_full[kMaxStages];
-  unsigned long long b_empty[kMaxStages];
+  unsigned long long full[kMaxStages];
+  unsigned long long empty[kMaxStages];
   unsigned long long a_full[2];
   unsigned long long a_empty[2];
   unsigned long long acc_full[2];
   unsigned long long acc_empty[2];
+  unsigned long long b_ready;
   unsigned tmem_addr;
   unsigned abort_flag;
 };
+static_assert(sizeof(Header) <= kSmemHeader, "header too large");
 
 __device__ __forceinline__ void tmem_st16(unsigned taddr, const unsigned* r) {
   asm volatile(
@@ -74,6 +81,11 @@ __device__ __forceinline__ void tmem_st16(unsigned taddr, const unsigned* r) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ uint2 lds64(unsigned addr) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+  return v;
+}
 
 // D[tmem] (+)= A[tmem] * B[smem]^T, 128 x N x 16
 __device__ __forceinline__ void umma_f16_ts(unsigned d_tmem, unsigned a_tmem, unsigned long long b_desc, unsigned idesc,
@@ -96,28 +108,36 @@ enum : unsigned { kErrProducer = 1u, kErrMma = 2u, kErrData = 4u, kErrDrain = 8u
 
 // ACT: activation right after the bias; TAIL: a residual add and / or a second activation follow
 template <int ACT, bool TAIL>
-__global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const TsParams p) {
+__global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_constant__ CUtensorMap tmap_a, const TsParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   Header* hdr = reinterpret_cast<Header*>(smem);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile unsigned* abort_flag = &hdr->abort_flag;
-  const unsigned chunk_bytes = static_cast<unsigned>(p.ks) * p.n_t * 8u;  // ks/2 K units x n_t rows x 16 bytes
-  const unsigned data0 = smem_u32(smem + kSmemHeader);
-  const unsigned a_cols = static_cast<unsigned>(p.ks) * 2u;
-  const unsigned acc_cols = static_cast<unsigned>(p.n_t);
-  const int n_units = p.m_tiles * p.n_tiles;
+  const unsigned a_stage_bytes = static_cast<unsigned>(p.ks) * 1024u;             // ks slices x 128 pixels x 8 bytes
+  const unsigned b_chunk_bytes = static_cast<unsigned>(p.ks) * p.n_cta * 8u;      // ks/2 K units x n_cta rows x 16 bytes
+  const unsigned stage_bytes = a_stage_bytes + (p.b_resident ? 0u : b_chunk_bytes);
+  const unsigned b_res_bytes = p.b_resident ? b_chunk_bytes * p.n_chunks : 0u;
+  const unsigned b_res0 = smem_u32(smem + kSmemHeader);                          // resident weights first
+  const unsigned stage0 = b_res0 + b_res_bytes;
+  const unsigned a_cols = static_cast<unsigned>(p.ks) * 2u, acc_cols = static_cast<unsigned>(p.n_cta);
+  const unsigned a_col0 = 2u * acc_cols;  // TMEM columns: two accumulators, then two A chunk buffers
+
+  // this CTA's share of the output channels is fixed; it walks over pixel tiles
+  const int n_part = blockIdx.x % p.n_parts;
+  const int m_first = blockIdx.x / p.n_parts, m_step = gridDim.x / p.n_parts;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < p.stages; ++i) {
-      mbar_init(smem_u32(&hdr->b_full[i]), 1);
-      mbar_init(smem_u32(&hdr->b_empty[i]), 1);
+      mbar_init(smem_u32(&hdr->full[i]), 1);
+      mbar_init(smem_u32(&hdr->empty[i]), kTransferWarps + (p.b_resident ? 0 : 1));
     }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(smem_u32(&hdr->a_full[i]), kDataWarps);
+      mbar_init(smem_u32(&hdr->a_full[i]), kTransferWarps);
       mbar_init(smem_u32(&hdr->a_empty[i]), 1);
       mbar_init(smem_u32(&hdr->acc_full[i]), 1);
-      mbar_init(smem_u32(&hdr->acc_empty[i]), kDataWarps);
+      mbar_init(smem_u32(&hdr->acc_empty[i]), kDrainWarps);
     }
+    mbar_init(smem_u32(&hdr->b_ready), 1);
     hdr->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -127,33 +147,37 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const TsParam
   __syncthreads();
   tc_fence_after();
   const unsigned tmem_base = hdr->tmem_addr;
-  // TMEM columns: [0, 2*n_t) two accumulators, then two A chunk buffers of 2*ks columns
-  const unsigned a_col0 = 2u * acc_cols;
+  const unsigned char* w_part = p.wts + static_cast<size_t>(n_part) * p.n_chunks * b_chunk_bytes;
 
   if (warp == 0) {
-    // ------------------------------------------------------------ weight producer
+    // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
+      if (p.b_resident) {
+        const unsigned bar = smem_u32(&hdr->b_ready);
+        mbar_expect_tx(bar, b_res_bytes);
+        for (int c = 0; c < p.n_chunks; ++c) bulk_load(b_res0 + c * b_chunk_bytes, w_part + static_cast<size_t>(c) * b_chunk_bytes, b_chunk_bytes, bar);
+      }
       unsigned it = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-        const int n_tile = u % p.n_tiles;
+      for (int m = m_first; m < p.m_tiles && ok; m += m_step) {
         for (int c = 0; c < p.n_chunks; ++c, ++it) {
           const unsigned stage = it % p.stages, phase = (it / p.stages) & 1u;
-          if (!mbar_wait(smem_u32(&hdr->b_empty[stage]), phase ^ 1u, abort_flag, p.timeout_ns, &g_ts_error, kErrProducer)) {
+          if (!mbar_wait(smem_u32(&hdr->empty[stage]), phase ^ 1u, abort_flag, p.timeout_ns, &g_ts_error, kErrProducer)) {
             ok = false;
             break;
           }
-          const unsigned full = smem_u32(&hdr->b_full[stage]);
-          mbar_expect_tx(full, chunk_bytes);
-          bulk_load(data0 + stage * chunk_bytes, p.wts + (static_cast<size_t>(n_tile) * p.n_chunks + c) * chunk_bytes, chunk_bytes,
-                    full);
+          const unsigned full = smem_u32(&hdr->full[stage]);
+          mbar_expect_tx(full, stage_bytes);
+          const unsigned dst = stage0 + stage * stage_bytes;
+          tma_load_2d(dst, &tmap_a, m * kRows, c * p.ks, full);  // pixels / slices outside the tensor arrive as zeros
+          if (!p.b_resident) bulk_load(dst + a_stage_bytes, w_part + static_cast<size_t>(c) * b_chunk_bytes, b_chunk_bytes, full);
         }
       }
       if (!ok) {
         const unsigned first = it > static_cast<unsigned>(p.stages) ? it - p.stages : 0u;
         for (unsigned j = first; j < it; ++j) {
           unsigned long long t0 = global_timer_ns();
-          while (!mbar_try_wait(smem_u32(&hdr->b_full[j % p.stages]), (j / p.stages) & 1u)) {
+          while (!mbar_try_wait(smem_u32(&hdr->full[j % p.stages]), (j / p.stages) & 1u)) {
             if (global_timer_ns() - t0 > p.timeout_ns) {
               atomicOr(&g_ts_error, kErrDrain);
               break;
@@ -165,103 +189,108 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const TsParam
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      // instruction descriptor: fp32 accumulator, fp16 A and B, B K-major, M = 128, N = n_t
+      // instruction descriptor: fp32 accumulator, fp16 A and B, B K-major, M = 128, N = n_cta
       const unsigned idesc = (1u << 4) | ((acc_cols >> 3) << 17) | ((kRows >> 4) << 24);
       const unsigned b_lbo = acc_cols * 16u;  // distance between consecutive 8-element K units of the weight tile
       unsigned it = 0, tile = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++tile) {
+      if (p.b_resident) ok = mbar_wait(smem_u32(&hdr->b_ready), 0u, abort_flag, p.timeout_ns, &g_ts_error, kErrMma);
+      for (int m = m_first; m < p.m_tiles && ok; m += m_step, ++tile) {
         const unsigned acc = tile & 1u, acc_phase = (tile >> 1) & 1u;
         if (!mbar_wait(smem_u32(&hdr->acc_empty[acc]), acc_phase ^ 1u, abort_flag, p.timeout_ns, &g_ts_error, kErrMma)) break;
         const unsigned d_tmem = tmem_base + acc * acc_cols;
         for (int c = 0; c < p.n_chunks; ++c, ++it) {
-          const unsigned stage = it % p.stages, b_phase = (it / p.stages) & 1u;
+          const unsigned stage = it % p.stages, s_phase = (it / p.stages) & 1u;
           const unsigned abuf = it & 1u, a_phase = (it >> 1) & 1u;
-          if (!mbar_wait(smem_u32(&hdr->a_full[abuf]), a_phase, abort_flag, p.timeout_ns, &g_ts_error, kErrMma) ||
-              !mbar_wait(smem_u32(&hdr->b_full[stage]), b_phase, abort_flag, p.timeout_ns, &g_ts_error, kErrMma)) {
+          if (!p.b_resident && !mbar_wait(smem_u32(&hdr->full[stage]), s_phase, abort_flag, p.timeout_ns, &g_ts_error, kErrMma)) {
+            ok = false;
+            break;
+          }
+          if (!mbar_wait(smem_u32(&hdr->a_full[abuf]), a_phase, abort_flag, p.timeout_ns, &g_ts_error, kErrMma)) {
             ok = false;
             break;
           }
           tc_fence_after();
           const unsigned a_tmem = tmem_base + a_col0 + abuf * a_cols;
-          const unsigned b_base = data0 + stage * chunk_bytes;
+          const unsigned b_base = p.b_resident ? b_res0 + c * b_chunk_bytes : stage0 + stage * stage_bytes + a_stage_bytes;
           for (int ks = 0; ks < p.ks / 4; ++ks) {  // 16 channels = 4 slices = 8 TMEM columns = 2 K units per MMA
             const unsigned long long bd = smem_desc(b_base + ks * 2 * b_lbo, b_lbo, 128);
             umma_f16_ts(d_tmem, a_tmem + ks * 8, bd, idesc, (c > 0 || ks > 0) ? 1u : 0u);
           }
           umma_commit(smem_u32(&hdr->a_empty[abuf]));
-          umma_commit(smem_u32(&hdr->b_empty[stage]));
+          if (!p.b_resident) umma_commit(smem_u32(&hdr->empty[stage]));
         }
         if (ok) umma_commit(smem_u32(&hdr->acc_full[acc]));
       }
     }
-  } else {
-    // ------------------------------------------------------------ data warps: load A, drain D
-    const int quarter = warp & 3;          // TMEM lanes [32*quarter, +32)
-    const int half_id = (warp - 2) >> 2;   // which half of the chunk's slices / of the accumulator columns
+  } else if (warp < 2 + kTransferWarps) {
+    // ------------------------------------------------------------ transfer: shared memory -> tensor memory
+    const int quarter = warp & 3;  // TMEM lanes [32*quarter, +32)
     const unsigned lane_bits = static_cast<unsigned>(quarter * 32) << 16;
-    const int row_in_tile = quarter * 32 + lane;
-    const int ks_half = p.ks >> 1;         // slices this warp loads per chunk (multiple of 8)
+    const unsigned row_off = static_cast<unsigned>(quarter * 32 + lane) * 8u;
     unsigned it = 0;
     bool ok = true;
-
-    auto load_unit = [&](int u) -> bool {
-      const int m_tile = u / p.n_tiles;
-      const unsigned pixel = static_cast<unsigned>(m_tile) * kRows + row_in_tile;
-      const bool px_ok = pixel < p.m_total_px;
+    for (int m = m_first; m < p.m_tiles && ok; m += m_step) {
       for (int c = 0; c < p.n_chunks; ++c, ++it) {
+        const unsigned stage = it % p.stages, s_phase = (it / p.stages) & 1u;
         const unsigned abuf = it & 1u, a_phase = (it >> 1) & 1u;
-        if (!mbar_wait(smem_u32(&hdr->a_empty[abuf]), a_phase ^ 1u, abort_flag, p.timeout_ns, &g_ts_error, kErrData)) return false;
+        if (!mbar_wait(smem_u32(&hdr->full[stage]), s_phase, abort_flag, p.timeout_ns, &g_ts_error, kErrData) ||
+            !mbar_wait(smem_u32(&hdr->a_empty[abuf]), a_phase ^ 1u, abort_flag, p.timeout_ns, &g_ts_error, kErrData)) {
+          ok = false;
+          break;
+        }
         tc_fence_after();
-        const int s0 = c * p.ks + half_id * ks_half;
-        const unsigned t_addr = tmem_base + lane_bits + a_col0 + abuf * a_cols + static_cast<unsigned>(half_id * ks_half) * 2u;
-        const __half* src = p.in + (static_cast<size_t>(s0) * p.m_total_px + pixel) * 4;
-        const size_t slice_stride = static_cast<size_t>(p.m_total_px) * 4;
-        for (int j = 0; j < ks_half; j += 8) {
-          // up to 8 slices = 16 columns per store; all loads of a batch are issued before the store
+        const unsigned src = stage0 + stage * stage_bytes + row_off;
+        const unsigned t_addr = tmem_base + lane_bits + a_col0 + abuf * a_cols;
+        for (int j = 0; j < p.ks; j += 8) {
           unsigned r[16];
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
-            uint2 v = make_uint2(0u, 0u);
-            if (px_ok && j + q < ks_half && s0 + j + q < p.s_in) v = __ldg(reinterpret_cast<const uint2*>(src + (j + q) * slice_stride));
+            const uint2 v = lds64(src + static_cast<unsigned>(j + q) * 1024u);
             r[2 * q] = v.x;
             r[2 * q + 1] = v.y;
           }
-          tmem_st16(t_addr + j * 2, r);  // ks_half is a multiple of 8: always whole 16-column stores
+          tmem_st16(t_addr + j * 2, r);
         }
+        // the stage's activations are in registers / on their way to tensor memory: release it
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[stage]));
         tmem_st_wait();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&hdr->a_full[abuf]));
       }
-      return true;
-    };
-
-    auto drain_unit = [&](int u, unsigned tile) -> bool {
-      const int m_tile = u / p.n_tiles, n_tile = u - m_tile * p.n_tiles;
+    }
+  } else {
+    // ------------------------------------------------------------ drain: accumulator -> global memory
+    const int quarter = warp & 3;
+    constexpr int kParts = kDrainWarps / 4;                     // warps sharing one lane quarter
+    const int part_id = (warp - (2 + kTransferWarps)) >> 2;     // takes every kParts-th 16-column group
+    const unsigned lane_bits = static_cast<unsigned>(quarter * 32) << 16;
+    const int groups = p.n_cta >> 4;
+    unsigned tile = 0;
+    for (int m = m_first; m < p.m_tiles; m += m_step, ++tile) {
       const unsigned acc = tile & 1u, acc_phase = (tile >> 1) & 1u;
-      if (!mbar_wait(smem_u32(&hdr->acc_full[acc]), acc_phase, abort_flag, p.timeout_ns, &g_ts_error, kErrData)) return false;
+      if (!mbar_wait(smem_u32(&hdr->acc_full[acc]), acc_phase, abort_flag, p.timeout_ns, &g_ts_error, kErrData)) break;
       tc_fence_after();
-      const unsigned pixel = static_cast<unsigned>(m_tile) * kRows + row_in_tile;
+      const unsigned pixel = static_cast<unsigned>(m) * kRows + quarter * 32 + lane;
       const bool px_ok = pixel < p.m_total_px;
-      const int groups = p.n_t >> 4;                       // 16-column groups in the accumulator
-      const int g0 = half_id == 0 ? 0 : (groups + 1) >> 1; // first half takes the extra group
-      const int g1 = half_id == 0 ? (groups + 1) >> 1 : groups;
       const unsigned t_addr = tmem_base + lane_bits + acc * acc_cols;
-      for (int g = g0; g < g1; ++g) {
+      for (int g = part_id; g < groups; g += kParts) {
         unsigned r[16];
         tmem_ld16(t_addr + g * 16, r);
         tmem_ld_wait16(r);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          const int so = (n_tile * p.n_t) / 4 + g * 4 + j;
+          const int so = (n_part * p.n_cta) / 4 + g * 4 + j;
           if (so >= p.s_out || !px_ok) continue;
           const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias) + so);
           const size_t off = (static_cast<size_t>(so) * p.m_total_px + pixel) * 4;  // in halves
-          float2 v0 = __fadd2_rn(make_float2(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1])), make_float2(b.x, b.y));
-          float2 v1 = __fadd2_rn(make_float2(__uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3])), make_float2(b.z, b.w));
+          const float2 v0 = __fadd2_rn(make_float2(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1])), make_float2(b.x, b.y));
+          const float2 v1 = __fadd2_rn(make_float2(__uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3])), make_float2(b.z, b.w));
           __half2 h0, h1;
           if (!TAIL) {
+            // clamping after the rounding equals rounding after the clamp: 0 and 6 are fp16 values
             h0 = __floats2half2_rn(v0.x, v0.y);
             h1 = __floats2half2_rn(v1.x, v1.y);
             if (ACT != GI_ACT_NONE) {
@@ -289,21 +318,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const TsParam
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&hdr->acc_empty[acc]));
-      return true;
-    };
-
-    // software pipeline: the operand of unit i+1 is loaded before the accumulator of unit i is drained
-    int prev = -1;
-    unsigned tile = 0;
-    for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-      ok = load_unit(u);
-      if (ok && prev >= 0) {
-        ok = drain_unit(prev, tile);
-        ++tile;
-      }
-      prev = u;
     }
-    if (ok && prev >= 0) drain_unit(prev, tile);
   }
 
   tc_fence_before();
@@ -316,7 +331,8 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const TsParam
 }
 
 struct Tiling {
-  int s_in, s_out, ks, n_chunks, n_t, n_tiles, stages;
+  int s_in, s_out, ks, n_chunks, n_cta, n_parts, b_resident, stages;
+  size_t smem;
 };
 
 Tiling choose_tiling(int cin, int cout) {
@@ -324,69 +340,90 @@ Tiling choose_tiling(int cin, int cout) {
   t.s_in = slices(cin);
   t.s_out = slices(cout);
   const int n_pad = (cout + 15) / 16 * 16;
-  t.n_tiles = (n_pad + kMaxNt - 1) / kMaxNt;
-  t.n_t = ((n_pad + t.n_tiles - 1) / t.n_tiles + 15) / 16 * 16;
-  // TMEM: 2 accumulators of n_t columns, 2 A buffers of 2*ks columns, 512 in all
-  int ks_max = (512 - 2 * t.n_t) / 4;
-  ks_max = ks_max / 16 * 16;  // whole 16-column stores for both halves of a chunk
-  if (ks_max > 64) ks_max = 64;
-  const int s_pad = (t.s_in + 15) / 16 * 16;
-  t.n_chunks = (s_pad + ks_max - 1) / ks_max;
-  t.ks = ((s_pad + t.n_chunks - 1) / t.n_chunks + 15) / 16 * 16;
-  const int chunk_bytes = t.ks * t.n_t * 8;
-  t.stages = kSmemBudget / chunk_bytes;
-  if (t.stages > kMaxStages) t.stages = kMaxStages;
-  if (t.stages < 2) t.stages = 2;
+  t.n_parts = (n_pad + kMaxNcta - 1) / kMaxNcta;
+  const int s_pad = (t.s_in + 7) / 8 * 8;
+  for (;; ++t.n_parts) {
+    t.n_cta = ((n_pad + t.n_parts - 1) / t.n_parts + 15) / 16 * 16;
+    // TMEM: 2 accumulators of n_cta columns + 2 A buffers of 2*ks columns <= 512
+    int ks_max = (512 - 2 * t.n_cta) / 4 / 8 * 8;
+    if (ks_max > 64) ks_max = 64;
+    t.n_chunks = (s_pad + ks_max - 1) / ks_max;
+    t.ks = ((s_pad + t.n_chunks - 1) / t.n_chunks + 7) / 8 * 8;
+    const size_t b_all = static_cast<size_t>(t.n_chunks) * t.ks * t.n_cta * 8;
+    // prefer resident weights: split the output channels over more CTAs while that gets there and
+    // the share stays at least 64 channels wide
+    t.b_resident = b_all <= static_cast<size_t>(kResidentLimit);
+    if (t.b_resident || t.n_cta <= 64) break;
+  }
+  // two activation stages must fit beside the weights: shrink the chunk if they do not
+  for (;;) {
+    const size_t bc = static_cast<size_t>(t.ks) * t.n_cta * 8;
+    const size_t res = t.b_resident ? bc * t.n_chunks : 0;
+    const size_t st = static_cast<size_t>(t.ks) * 1024 + (t.b_resident ? 0 : bc);
+    if (t.ks <= 8 || res + 2 * st <= static_cast<size_t>(kSmemBudget)) break;
+    t.ks = (t.ks / 2 + 7) / 8 * 8;
+    t.n_chunks = (s_pad + t.ks - 1) / t.ks;
+  }
+  const size_t b_chunk = static_cast<size_t>(t.ks) * t.n_cta * 8;
+  const size_t resident = t.b_resident ? b_chunk * t.n_chunks : 0;
+  const size_t stage = static_cast<size_t>(t.ks) * 1024 + (t.b_resident ? 0 : b_chunk);
+  long long stages = (static_cast<long long>(kSmemBudget) - static_cast<long long>(resident)) / static_cast<long long>(stage);
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (stages < 2) stages = 2;
+  t.stages = static_cast<int>(stages);
+  t.smem = kSmemHeader + resident + stage * t.stages;
   return t;
 }
 
 }  // namespace
 
-bool pointwise_ts_supported(int cin, int cout) { return cin > 0 && cout > 0; }
+bool pointwise_ts_supported(int cin, int cout) {
+  if (cin <= 0 || cout <= 0) return false;
+  return choose_tiling(cin, cout).smem <= static_cast<size_t>(kSmemHeader + kSmemBudget + 16 * 1024);
+}
 
-// Dense weights as the B operand, per (output tile, K chunk): [ks/2 K units][n_t rows][8 halves].
+// Dense weights as the B operand, per (CTA share, K chunk): [ks/2 K units][n_cta rows][8 halves].
 void pointwise_ts_pack(const float* w, const float* bias, int cin, int cout, std::vector<uint8_t>* blob, LaunchRec* r) {
   const Tiling t = choose_tiling(cin, cout);
-  const size_t chunk_bytes = static_cast<size_t>(t.ks) * t.n_t * 8;
-  const size_t wbytes = static_cast<size_t>(t.n_tiles) * t.n_chunks * chunk_bytes;
+  const size_t chunk_bytes = static_cast<size_t>(t.ks) * t.n_cta * 8;
+  const size_t wbytes = static_cast<size_t>(t.n_parts) * t.n_chunks * chunk_bytes;
   const uint64_t woff = round_up_u64(blob->size(), 256);
   blob->resize(woff + wbytes, 0);
   const uint64_t boff = round_up_u64(blob->size(), 256);
-  blob->resize(boff + static_cast<size_t>(t.n_tiles) * t.n_t * sizeof(float), 0);
+  blob->resize(boff + static_cast<size_t>(t.n_parts) * t.n_cta * sizeof(float), 0);
   uint16_t* wp = reinterpret_cast<uint16_t*>(blob->data() + woff);
   float* bp = reinterpret_cast<float*>(blob->data() + boff);
   for (int co = 0; co < cout; ++co) {
-    const int nt = co / t.n_t, row = co % t.n_t;
+    const int part = co / t.n_cta, row = co % t.n_cta;
     bp[co] = bias[co];
     for (int ci = 0; ci < cin; ++ci) {
       const int chunk = ci / (t.ks * 4), k = ci % (t.ks * 4);
-      uint16_t* base = wp + (static_cast<size_t>(nt) * t.n_chunks + chunk) * (chunk_bytes / 2);
-      base[(static_cast<size_t>(k / 8) * t.n_t + row) * 8 + k % 8] = f32_to_f16_rne(w[static_cast<size_t>(co) * cin + ci]);
+      uint16_t* base = wp + (static_cast<size_t>(part) * t.n_chunks + chunk) * (chunk_bytes / 2);
+      base[(static_cast<size_t>(k / 8) * t.n_cta + row) * 8 + k % 8] = f32_to_f16_rne(w[static_cast<size_t>(co) * cin + ci]);
     }
   }
   r->wts = Loc{W_WEIGHTS, 0, woff};
   r->bias = Loc{W_WEIGHTS, 0, boff};
   r->wts_bytes = wbytes;
-  r->tc_nt = t.n_t;
+  r->tc_nt = t.n_cta;
   r->tc_kc = t.ks;
   r->tc_stages = t.stages;
 }
 
-int launch_pointwise_ts(const LaunchRec& r, const Ptrs& p, void* stream) {
+int launch_pointwise_ts(const LaunchRec& r, const Ptrs& p, void** state, int launch_index, void* stream) {
   const Tiling t = choose_tiling(r.C, r.Co);
   TsParams k;
-  k.in = static_cast<const __half*>(p.in0);
   k.res = static_cast<const __half*>(p.res);
   k.out = static_cast<__half*>(p.out);
   k.bias = static_cast<const float*>(p.bias);
   k.wts = static_cast<const unsigned char*>(p.wts);
   k.m_total_px = static_cast<unsigned>(r.B) * static_cast<unsigned>(plane_pixels(r.H, r.W));
-  k.s_in = t.s_in;
   k.s_out = t.s_out;
   k.ks = t.ks;
   k.n_chunks = t.n_chunks;
-  k.n_t = t.n_t;
-  k.n_tiles = t.n_tiles;
+  k.n_cta = t.n_cta;
+  k.n_parts = t.n_parts;
+  k.b_resident = t.b_resident;
   k.stages = t.stages;
   k.m_tiles = static_cast<int>((k.m_total_px + kRows - 1) / kRows);
   k.has_res = r.ep.has_res;
@@ -402,7 +439,7 @@ int launch_pointwise_ts(const LaunchRec& r, const Ptrs& p, void* stream) {
   const bool tail = k.has_res || k.act_post != GI_ACT_NONE;
   if (!attr_set) {
     cudaError_t e = cudaSuccess;
-    const int bytes = kSmemHeader + kSmemBudget;
+    const int bytes = kSmemHeader + kSmemBudget + 16 * 1024;
 #define GI_TS_ATTR(A, T) \
   if (e == cudaSuccess) e = cudaFuncSetAttribute(pointwise_ts_kernel<A, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)
     GI_TS_ATTR(GI_ACT_NONE, false);
@@ -415,15 +452,24 @@ int launch_pointwise_ts(const LaunchRec& r, const Ptrs& p, void* stream) {
     if (e != cudaSuccess) return static_cast<int>(e);
     attr_set = true;
   }
-  const long long units = static_cast<long long>(k.m_tiles) * k.n_tiles;
-  const unsigned grid = static_cast<unsigned>(units < sms ? units : sms);
+  MapEntry& me = map_cache_entry(state, launch_index);
+  if (me.in != p.in0) {
+    const int err = encode_plane_map(&me.map, p.in0, k.m_total_px, t.s_in, kRows, t.ks);
+    if (err != 0) return err;
+    me.in = p.in0;
+  }
+  // CTAs come in groups of n_parts (one per share of the output channels) that walk the pixel tiles together
+  long long groups = sms / t.n_parts;
+  if (groups < 1) groups = 1;
+  if (groups > k.m_tiles) groups = k.m_tiles;
+  const unsigned grid = static_cast<unsigned>(groups * t.n_parts);
   // the kernel reserves all of tensor memory, so exactly one CTA may live on an SM: ask for enough
   // shared memory that a second one cannot be co-resident
-  size_t smem = kSmemHeader + static_cast<size_t>(t.stages) * t.ks * t.n_t * 8;
+  size_t smem = t.smem;
   if (smem < 120 * 1024) smem = 120 * 1024;
   cudaStream_t cu_stream = static_cast<cudaStream_t>(stream);
   const int act = r.ep.act_pre;
-#define GI_TS_LAUNCH(A, T) pointwise_ts_kernel<A, T><<<grid, kThreads, smem, cu_stream>>>(k)
+#define GI_TS_LAUNCH(A, T) pointwise_ts_kernel<A, T><<<grid, kThreads, smem, cu_stream>>>(me.map, k)
   if (tail) {
     if (act == GI_ACT_RELU6) GI_TS_LAUNCH(GI_ACT_RELU6, true);
     else if (act == GI_ACT_RELU) GI_TS_LAUNCH(GI_ACT_RELU, true);
