@@ -52,8 +52,9 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi during the timed region (read-only query)."""
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    """Samples nvidia-smi (read-only query) from before the warm-up on; stop(t0, t1) keeps the
+    samples whose timestamp lies inside the timed region [t0, t1] (wall clock, seconds)."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
@@ -72,9 +73,9 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append(line.strip())
+            self.rows.append((time.time(), line.strip()))
 
-    def stop(self):
+    def stop(self, t0=None, t1=None):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -82,22 +83,44 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             pass
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for row in self.rows:
-            f = [x.strip() for x in row.split(",")]
-            if len(f) < 7:
-                continue
-            try:
-                sm.append(float(f[0]))
-                mx.append(float(f[1]))
-            except ValueError:
-                continue
-            for n, v in zip(names, f[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        return summarize_clock_rows(self.rows, t0, t1)
+
+
+def summarize_clock_rows(rows, t0=None, t1=None):
+    """rows: (arrival wall time, csv line).  A sample counts if it arrived inside [t0, t1 + 50 ms]."""
+    sm, mx, reasons = [], [], set()
+    names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+    for when, row in rows:
+        if t0 is not None and not (t0 <= when <= t1 + 0.05):
+            continue
+        f = [x.strip() for x in row.split(",")]
+        if len(f) < 8:
+            continue
+        try:
+            sm.append(float(f[1]))
+            mx.append(float(f[2]))
+        except ValueError:
+            continue
+        for n, v in zip(names, f[4:8]):
+            if v.lower().startswith("active"):
+                reasons.add(n)
+    return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+            "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def shard_images(rank: int, batch_per_gpu: int):
+    """Weak scaling by batch: rank r owns images [r*B, (r+1)*B) of the global batch; no exchange step."""
+    return [rank * batch_per_gpu + i for i in range(batch_per_gpu)]
+
+
+def job_throughput(local_ms: float, images_per_rank: int, steps: int, world: int, dist=None, device=None):
+    """Whole-job images/s: all ranks' images over the slowest rank's device time (max over ranks)."""
+    import torch
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    return world * images_per_rank * steps / (total_ms * 1e-3), total_ms
 
 
 def oracle_images_per_s(spec_fn, budget_s=15.0):
@@ -277,7 +300,7 @@ def main():
     ex.bind(dev)
     ops = ex.ops()
     # every rank draws its own images: rank r holds images [r*B, (r+1)*B) of the global batch
-    x_host = wl.make_input(spec, images=[rank * args.batch + i for i in range(args.batch)]).astype(np.float16)
+    x_host = wl.make_input(spec, images=shard_images(rank, args.batch)).astype(np.float16)
     x_pin = torch.from_numpy(x_host).pin_memory()
     x_dev = x_pin.to(dev, non_blocking=False)
     out_shape = (args.batch,) + tuple(spec.shapes[spec.outputs[0]])
@@ -290,31 +313,29 @@ def main():
         ex.run([x_dev], [out_dev], stream)
 
     # ---- resident-input throughput -------------------------------------------------------
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()  # started before the warm-up so that it is sampling when the timed region begins
     for _ in range(args.warmup):
         flush.zero_()
         step_resident()
-    sampler = ClockSampler(local)
     barrier()
-    if rank == 0:
-        sampler.start()
     starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     wall0 = time.perf_counter()
+    t_region0 = time.time()
     for i in range(args.steps):
         flush.zero_()
         starts[i].record(stream)
         step_resident()
         ends[i].record(stream)
     barrier()
+    t_region1 = time.time()
     wall = time.perf_counter() - wall0
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(t_region0, t_region1) if rank == 0 else None
     ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
-    t_steps = torch.tensor([sum(ms)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t_steps, op=dist.ReduceOp.MAX)
-    total_ms = float(t_steps.item())
+    value, total_ms = job_throughput(sum(ms), args.batch, args.steps, world, dist, dev)
     ms_per_step = total_ms / args.steps
-    value = world * args.batch * args.steps / (total_ms * 1e-3)
 
     # ---- end to end with host buffers ------------------------------------------------------
     def step_e2e():
@@ -331,10 +352,7 @@ def main():
         step_e2e()
     e1.record(stream)
     barrier()
-    t_e2e = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t_e2e, op=dist.ReduceOp.MAX)
-    e2e_value = world * args.batch * args.steps / (float(t_e2e.item()) * 1e-3)
+    e2e_value, _ = job_throughput(e0.elapsed_time(e1), args.batch, args.steps, world, dist, dev)
     logits_checksum = float(out_pin.float().abs().mean())
 
     # ---- per-op times for the roofline (rank 0) ---------------------------------------------
