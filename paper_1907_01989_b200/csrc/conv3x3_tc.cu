@@ -18,6 +18,7 @@
 #include <cuda_runtime.h>
 
 #include "kernels.h"
+#include "pdl.cuh"
 #include "sm100_ptx.cuh"
 
 namespace gi {
@@ -86,6 +87,9 @@ __global__ void __launch_bounds__(kThreads, 2) conv3x3_tc_kernel(const StemParam
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  // everything above touched only weights and on-chip state; the activations come after the wait
+  pdl_launch_dependents();
+  pdl_wait();
   const unsigned tmem_base = hdr->tmem_addr;
   const unsigned n_cols = static_cast<unsigned>(p.n_pad);
   const long long m_total = static_cast<long long>(p.B) * p.Pout;
@@ -302,7 +306,7 @@ int launch_conv3x3_tc(const LaunchRec& r, const Ptrs& p, void* stream) {
   if (per_sm < 1) per_sm = 1;
   long long grid = static_cast<long long>(sms) * per_sm;
   if (grid > tiles) grid = tiles;
-  conv3x3_tc_kernel<<<static_cast<unsigned>(grid), kThreads, smem, static_cast<cudaStream_t>(stream)>>>(k);
+  launch_pdl(conv3x3_tc_kernel, static_cast<unsigned>(grid), kThreads, smem, static_cast<cudaStream_t>(stream), k);
   return static_cast<int>(cudaGetLastError());
 }
 

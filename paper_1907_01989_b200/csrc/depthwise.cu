@@ -14,6 +14,7 @@
 #include <cuda_runtime.h>
 
 #include "kernels.h"
+#include "pdl.cuh"
 
 namespace gi {
 namespace {
@@ -145,11 +146,13 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
     }
   };
 
+  pdl_launch_dependents();
   // the zero heads are written once; copies never touch them
   for (int i = threadIdx.x; i < 2 * g.nb * g.head_px; i += blockDim.x) {
     const int plane = i / g.head_px, px = i - plane * g.head_px;
     *reinterpret_cast<uint2*>(smem_raw + (static_cast<size_t>(plane) * g.plane_stride_px + px) * 8) = make_uint2(0u, 0u);
   }
+  pdl_wait();  // the first staging copy below reads the previous kernel's output
   if (threadIdx.x == 0) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bars[0])) : "memory");
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bars[1])) : "memory");
@@ -476,7 +479,7 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
       if (e != cudaSuccess) return static_cast<int>(e);                                                                       \
       attr_done[M][A][T] = true;                                                                                              \
     }                                                                                                                         \
-    depthwise_f16_kernel<M, A, T><<<static_cast<unsigned>(grid), threads, smem, st>>>(in, w, b, res, out, g, r.ep);           \
+    launch_pdl(depthwise_f16_kernel<M, A, T>, static_cast<unsigned>(grid), threads, smem, st, in, w, b, res, out, g, r.ep);           \
   } while (0)
 #define GI_DW_ACT(M, A)       \
   do {                        \

@@ -7,6 +7,7 @@
 #include <cuda_runtime.h>
 
 #include "kernels.h"
+#include "pdl.cuh"
 
 namespace gi {
 namespace {
@@ -67,6 +68,8 @@ __device__ __forceinline__ float4 epilogue(float4 v, const Epilogue& ep, const T
 // ------------------------------------------------------------------ layout conversion
 template <typename T>
 __global__ void pack_kernel(const T* __restrict__ nhwc, T* __restrict__ out, int B, int HW, int C, int P, int S) {
+  pdl_launch_dependents();
+  pdl_wait();
   const size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x;
   const size_t total = static_cast<size_t>(S) * B * P;
   if (idx >= total) return;
@@ -86,6 +89,8 @@ __global__ void pack_kernel(const T* __restrict__ nhwc, T* __restrict__ out, int
 
 template <typename T>
 __global__ void unpack_kernel(const T* __restrict__ in, T* __restrict__ nhwc, int B, int HW, int C, int P, int S) {
+  pdl_launch_dependents();
+  pdl_wait();
   const size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x;
   const size_t total = static_cast<size_t>(B) * HW * S;
   if (idx >= total) return;
@@ -111,6 +116,8 @@ template <typename T, int OS>
 __global__ void __launch_bounds__(128) conv_simt_kernel(const T* __restrict__ in, const float4* __restrict__ w,
                                                         const float* __restrict__ bias, const T* __restrict__ res,
                                                         T* __restrict__ out, ConvGeom g, Epilogue ep) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int pix = blockIdx.x * 128 + threadIdx.x;
   const int grp = blockIdx.y, b = blockIdx.z;
   if (pix >= g.Pout) return;
@@ -165,6 +172,8 @@ template <typename T>
 __global__ void __launch_bounds__(128) depthwise_kernel(const T* __restrict__ in, const float* __restrict__ w,
                                                         const float* __restrict__ bias, const T* __restrict__ res,
                                                         T* __restrict__ out, ConvGeom g, Epilogue ep) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int pix = blockIdx.x * 128 + threadIdx.x;
   const int s = blockIdx.y, b = blockIdx.z;
   if (pix >= g.Pout) return;
@@ -200,6 +209,8 @@ __global__ void __launch_bounds__(128) depthwise_kernel(const T* __restrict__ in
 template <typename T>
 __global__ void eltwise_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restrict__ out, size_t n_px,
                                Epilogue ep) {
+  pdl_launch_dependents();
+  pdl_wait();
   const size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x;
   if (i >= n_px) return;
   const float4 v = epilogue<T>(Px<T>::load(a + i * 4), ep, b, i * 4);
@@ -210,6 +221,8 @@ __global__ void eltwise_kernel(const T* __restrict__ a, const T* __restrict__ b,
 // one warp per (slice, image): lanes stride over the pixels, shuffle reduction in a fixed order
 template <typename T>
 __global__ void pool_kernel(const T* __restrict__ in, T* __restrict__ out, int planes, int HW, int Pin, int Pout) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, lane = threadIdx.x & 31;
   if (warp >= planes) return;
   const T* plane = in + static_cast<size_t>(warp) * Pin * 4;
@@ -239,6 +252,8 @@ __global__ void pool_kernel(const T* __restrict__ in, T* __restrict__ out, int p
 template <typename T>
 __global__ void __launch_bounds__(128) resize_kernel(const T* __restrict__ in, T* __restrict__ out, int B, int H, int W,
                                                      int Pin, int OH, int OW, int Pout, int ny, int dy, int nx, int dx) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int pix = blockIdx.x * 128 + threadIdx.x;
   const int s = blockIdx.y, b = blockIdx.z;
   if (pix >= Pout) return;
@@ -306,9 +321,9 @@ int launch_pack(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int S = slices(r.C), P = plane_pixels(r.H, r.W), HW = r.H * r.W;
   const size_t total = static_cast<size_t>(S) * r.B * P;
-  GI_BY_STORAGE((pack_kernel<__half><<<blocks_for(total, 256), 256, 0, st>>>(static_cast<const __half*>(p.in0),
+  GI_BY_STORAGE((launch_pdl(pack_kernel<__half>, blocks_for(total, 256), 256, 0, st, static_cast<const __half*>(p.in0),
                                                                              static_cast<__half*>(p.out), r.B, HW, r.C, P, S)),
-                (pack_kernel<float><<<blocks_for(total, 256), 256, 0, st>>>(static_cast<const float*>(p.in0),
+                (launch_pdl(pack_kernel<float>, blocks_for(total, 256), 256, 0, st, static_cast<const float*>(p.in0),
                                                                             static_cast<float*>(p.out), r.B, HW, r.C, P, S)));
   return static_cast<int>(cudaGetLastError());
 }
@@ -317,9 +332,9 @@ int launch_unpack(const LaunchRec& r, const Ptrs& p, int storage, void* stream) 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int S = slices(r.C), P = plane_pixels(r.H, r.W), HW = r.H * r.W;
   const size_t total = static_cast<size_t>(S) * r.B * HW;
-  GI_BY_STORAGE((unpack_kernel<__half><<<blocks_for(total, 256), 256, 0, st>>>(static_cast<const __half*>(p.in0),
+  GI_BY_STORAGE((launch_pdl(unpack_kernel<__half>, blocks_for(total, 256), 256, 0, st, static_cast<const __half*>(p.in0),
                                                                                static_cast<__half*>(p.out), r.B, HW, r.C, P, S)),
-                (unpack_kernel<float><<<blocks_for(total, 256), 256, 0, st>>>(static_cast<const float*>(p.in0),
+                (launch_pdl(unpack_kernel<float>, blocks_for(total, 256), 256, 0, st, static_cast<const float*>(p.in0),
                                                                               static_cast<float*>(p.out), r.B, HW, r.C, P, S)));
   return static_cast<int>(cudaGetLastError());
 }
@@ -335,10 +350,10 @@ static void conv_dispatch(const LaunchRec& r, const Ptrs& p, cudaStream_t st) {
   const T* res = static_cast<const T*>(p.res);
   T* out = static_cast<T*>(p.out);
   switch (os) {
-    case 8: conv_simt_kernel<T, 8><<<grid, 128, 0, st>>>(in, w, b, res, out, g, r.ep); break;
-    case 4: conv_simt_kernel<T, 4><<<grid, 128, 0, st>>>(in, w, b, res, out, g, r.ep); break;
-    case 2: conv_simt_kernel<T, 2><<<grid, 128, 0, st>>>(in, w, b, res, out, g, r.ep); break;
-    default: conv_simt_kernel<T, 1><<<grid, 128, 0, st>>>(in, w, b, res, out, g, r.ep); break;
+    case 8: launch_pdl(conv_simt_kernel<T, 8>, grid, 128, 0, st, in, w, b, res, out, g, r.ep); break;
+    case 4: launch_pdl(conv_simt_kernel<T, 4>, grid, 128, 0, st, in, w, b, res, out, g, r.ep); break;
+    case 2: launch_pdl(conv_simt_kernel<T, 2>, grid, 128, 0, st, in, w, b, res, out, g, r.ep); break;
+    default: launch_pdl(conv_simt_kernel<T, 1>, grid, 128, 0, st, in, w, b, res, out, g, r.ep); break;
   }
 }
 
@@ -355,10 +370,10 @@ int launch_depthwise(const LaunchRec& r, const Ptrs& p, int storage, void* strea
   if (r.B > 65535) return static_cast<int>(cudaErrorInvalidConfiguration);
   const ConvGeom g = geom(r);
   const dim3 grid(blocks_for(g.Pout, 128), g.Sout, r.B);
-  GI_BY_STORAGE((depthwise_kernel<__half><<<grid, 128, 0, st>>>(static_cast<const __half*>(p.in0), static_cast<const float*>(p.wts),
+  GI_BY_STORAGE((launch_pdl(depthwise_kernel<__half>, grid, 128, 0, st, static_cast<const __half*>(p.in0), static_cast<const float*>(p.wts),
                                                                static_cast<const float*>(p.bias), static_cast<const __half*>(p.res),
                                                                static_cast<__half*>(p.out), g, r.ep)),
-                (depthwise_kernel<float><<<grid, 128, 0, st>>>(static_cast<const float*>(p.in0), static_cast<const float*>(p.wts),
+                (launch_pdl(depthwise_kernel<float>, grid, 128, 0, st, static_cast<const float*>(p.in0), static_cast<const float*>(p.wts),
                                                               static_cast<const float*>(p.bias), static_cast<const float*>(p.res),
                                                               static_cast<float*>(p.out), g, r.ep)));
   return static_cast<int>(cudaGetLastError());
@@ -367,10 +382,10 @@ int launch_depthwise(const LaunchRec& r, const Ptrs& p, int storage, void* strea
 int launch_eltwise(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t n_px = static_cast<size_t>(slices(r.Co)) * r.B * plane_pixels(r.Ho, r.Wo);
-  GI_BY_STORAGE((eltwise_kernel<__half><<<blocks_for(n_px, 256), 256, 0, st>>>(static_cast<const __half*>(p.in0),
+  GI_BY_STORAGE((launch_pdl(eltwise_kernel<__half>, blocks_for(n_px, 256), 256, 0, st, static_cast<const __half*>(p.in0),
                                                                                static_cast<const __half*>(p.in1),
                                                                                static_cast<__half*>(p.out), n_px, r.ep)),
-                (eltwise_kernel<float><<<blocks_for(n_px, 256), 256, 0, st>>>(static_cast<const float*>(p.in0),
+                (launch_pdl(eltwise_kernel<float>, blocks_for(n_px, 256), 256, 0, st, static_cast<const float*>(p.in0),
                                                                               static_cast<const float*>(p.in1),
                                                                               static_cast<float*>(p.out), n_px, r.ep)));
   return static_cast<int>(cudaGetLastError());
@@ -380,9 +395,9 @@ int launch_pool(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int planes = slices(r.C) * r.B;
   const unsigned blocks = blocks_for(static_cast<size_t>(planes) * 32, 256);
-  GI_BY_STORAGE((pool_kernel<__half><<<blocks, 256, 0, st>>>(static_cast<const __half*>(p.in0), static_cast<__half*>(p.out), planes,
+  GI_BY_STORAGE((launch_pdl(pool_kernel<__half>, blocks, 256, 0, st, static_cast<const __half*>(p.in0), static_cast<__half*>(p.out), planes,
                                                             r.H * r.W, plane_pixels(r.H, r.W), plane_pixels(1, 1))),
-                (pool_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(p.in0), static_cast<float*>(p.out), planes,
+                (launch_pdl(pool_kernel<float>, blocks, 256, 0, st, static_cast<const float*>(p.in0), static_cast<float*>(p.out), planes,
                                                            r.H * r.W, plane_pixels(r.H, r.W), plane_pixels(1, 1))));
   return static_cast<int>(cudaGetLastError());
 }
@@ -404,9 +419,9 @@ int launch_resize(const LaunchRec& r, const Ptrs& p, int storage, void* stream) 
   }
   const int Pout = plane_pixels(r.Ho, r.Wo), Pin = plane_pixels(r.H, r.W);
   const dim3 grid(blocks_for(Pout, 128), slices(r.C), r.B);
-  GI_BY_STORAGE((resize_kernel<__half><<<grid, 128, 0, st>>>(static_cast<const __half*>(p.in0), static_cast<__half*>(p.out), r.B, r.H,
+  GI_BY_STORAGE((launch_pdl(resize_kernel<__half>, grid, 128, 0, st, static_cast<const __half*>(p.in0), static_cast<__half*>(p.out), r.B, r.H,
                                                             r.W, Pin, r.Ho, r.Wo, Pout, ny, dy, nx, dx)),
-                (resize_kernel<float><<<grid, 128, 0, st>>>(static_cast<const float*>(p.in0), static_cast<float*>(p.out), r.B, r.H,
+                (launch_pdl(resize_kernel<float>, grid, 128, 0, st, static_cast<const float*>(p.in0), static_cast<float*>(p.out), r.B, r.H,
                                                            r.W, Pin, r.Ho, r.Wo, Pout, ny, dy, nx, dx)));
   return static_cast<int>(cudaGetLastError());
 }

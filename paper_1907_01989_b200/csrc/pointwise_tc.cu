@@ -29,6 +29,7 @@
 #include <vector>
 
 #include "kernels.h"
+#include "pdl.cuh"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"
 
@@ -114,6 +115,9 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  // the prologue above touched only on-chip state; activations are read and written after the wait
+  pdl_launch_dependents();
+  pdl_wait();
   const unsigned tmem_base = hdr->tmem_addr;
   const int n_units = p.m_tiles * p.groups;
   const unsigned acc_cols = static_cast<unsigned>(p.nts) * 8u;
@@ -439,7 +443,7 @@ int launch_pointwise_tc(const LaunchRec& r, const Ptrs& p, void** state, int lau
   const size_t smem = kSmemHeader + static_cast<size_t>(t.stages) * t.kc * (kSliceBytes + t.nts * kCoreBytes);
   const bool tail = k.has_res || k.act_post != GI_ACT_NONE;
   cudaStream_t cu_stream = static_cast<cudaStream_t>(stream);
-#define GI_TC_LAUNCH(A, T) pointwise_tc_kernel<A, T><<<grid, kThreads, smem, cu_stream>>>(me.map, k)
+#define GI_TC_LAUNCH(A, T) launch_pdl(pointwise_tc_kernel<A, T>, grid, kThreads, smem, cu_stream, me.map, k)
   if (tail) {
     if (k.act_pre == GI_ACT_RELU6) GI_TC_LAUNCH(GI_ACT_RELU6, true);
     else if (k.act_pre == GI_ACT_RELU) GI_TC_LAUNCH(GI_ACT_RELU, true);

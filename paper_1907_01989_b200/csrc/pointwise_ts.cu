@@ -24,6 +24,7 @@
 #include <cuda_runtime.h>
 
 #include "kernels.h"
+#include "pdl.cuh"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"
 
@@ -148,15 +149,19 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
   tc_fence_after();
   const unsigned tmem_base = hdr->tmem_addr;
   const unsigned char* w_part = p.wts + static_cast<size_t>(n_part) * p.n_chunks * b_chunk_bytes;
+  pdl_launch_dependents();
+  // the weights never change after binding: their copy starts while the previous kernel still runs
+  if (warp == 0 && lane == 0 && p.b_resident) {
+    const unsigned bar = smem_u32(&hdr->b_ready);
+    mbar_expect_tx(bar, b_res_bytes);
+    for (int c = 0; c < p.n_chunks; ++c)
+      bulk_load(b_res0 + c * b_chunk_bytes, w_part + static_cast<size_t>(c) * b_chunk_bytes, b_chunk_bytes, bar);
+  }
+  pdl_wait();  // activations are read and written only below
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      if (p.b_resident) {
-        const unsigned bar = smem_u32(&hdr->b_ready);
-        mbar_expect_tx(bar, b_res_bytes);
-        for (int c = 0; c < p.n_chunks; ++c) bulk_load(b_res0 + c * b_chunk_bytes, w_part + static_cast<size_t>(c) * b_chunk_bytes, b_chunk_bytes, bar);
-      }
       unsigned it = 0;
       bool ok = true;
       for (int m = m_first; m < p.m_tiles && ok; m += m_step) {
@@ -469,7 +474,7 @@ int launch_pointwise_ts(const LaunchRec& r, const Ptrs& p, void** state, int lau
   if (smem < 120 * 1024) smem = 120 * 1024;
   cudaStream_t cu_stream = static_cast<cudaStream_t>(stream);
   const int act = r.ep.act_pre;
-#define GI_TS_LAUNCH(A, T) pointwise_ts_kernel<A, T><<<grid, kThreads, smem, cu_stream>>>(me.map, k)
+#define GI_TS_LAUNCH(A, T) launch_pdl(pointwise_ts_kernel<A, T>, grid, kThreads, smem, cu_stream, me.map, k)
   if (tail) {
     if (act == GI_ACT_RELU6) GI_TS_LAUNCH(GI_ACT_RELU6, true);
     else if (act == GI_ACT_RELU) GI_TS_LAUNCH(GI_ACT_RELU, true);
