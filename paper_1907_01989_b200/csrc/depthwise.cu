@@ -32,6 +32,7 @@ struct DwGeom {
   int head_px;  // zeroed pixels in front of each plane's staged rows (even, >= W + 2)
   int plane_stride_px;  // pixels reserved per plane in one staging buffer (even)
   int items;            // S * bchunks * bands
+  int packed;           // 1: whole small planes, staged back to back by one copy per item
   unsigned timeout_ns;
 };
 
@@ -93,16 +94,20 @@ __device__ __forceinline__ Row widen(const uint2* u) {
 // MODE 1: stride 2, dilation 1, same padding limit - the last row of an output is the first row
 //         of the next
 // MODE 2: anything else - three rows fetched per output row, each tap tested
+// PACKED (modes 0/1, small planes): a work item is a run of whole planes, which are contiguous in
+//         memory, so ONE bulk copy stages them back to back (many small copies are slow); the
+//         rows above and below a plane are then its neighbours' rows, so row validity is tested
+//         (one compare per row) instead of relying on zero rows.
 // ACT: activation applied right after the bias (the common fused case); TAIL: a residual add
 // and / or a second activation follow.
-template <int MODE, int ACT, bool TAIL>
+template <int MODE, int ACT, bool TAIL, bool PACKED>
 __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __restrict__ in, const float* __restrict__ w,
                                                                 const float* __restrict__ bias, const __half* __restrict__ res,
                                                                 __half* __restrict__ out, const DwGeom g, const Epilogue ep) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ __align__(8) unsigned long long bars[2];
   __shared__ unsigned timed_out;
-  const unsigned buf_bytes = static_cast<unsigned>(g.plane_stride_px) * 8u * g.nb;
+  const unsigned buf_bytes = PACKED ? static_cast<unsigned>(g.Pin) * 8u * g.nb + 16u : static_cast<unsigned>(g.plane_stride_px) * 8u * g.nb;
   const int W = g.W, H = g.H, Wo = g.Wo, stride = g.stride, pt = g.pt;
 
   // contiguous, balanced range of work items for this CTA: items of one slice stay together
@@ -111,10 +116,24 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
   const int count = per + (static_cast<int>(blockIdx.x) < extra ? 1 : 0);
   const int th = g.sub * g.tr;
 
-  auto item_rows = [&](int item, int& s, int& b0, int& nbk, int& oy0, int& oy1, int& start_px, unsigned& bytes, bool& last_band) {
-    const int band = item % g.bands;
-    const int bc = (item / g.bands) % g.bchunks;
-    s = item / (g.bands * g.bchunks);
+  // work items are numbered band-fastest, then batch chunk, then slice; a CTA walks a contiguous
+  // range, so the triple is decoded once and then advanced without divisions
+  struct Item {
+    int s, bc, band;
+  };
+  auto advance = [&](Item it) {
+    if (++it.band == g.bands) {
+      it.band = 0;
+      if (++it.bc == g.bchunks) {
+        it.bc = 0;
+        ++it.s;
+      }
+    }
+    return it;
+  };
+  auto item_rows = [&](const Item& it, int& s, int& b0, int& nbk, int& oy0, int& oy1, int& start_px, unsigned& bytes, bool& last_band) {
+    const int band = it.band, bc = it.bc;
+    s = it.s;
     b0 = bc * g.nb;
     nbk = min(g.nb, g.B - b0);
     oy0 = band * th;
@@ -127,7 +146,7 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
     bytes = static_cast<unsigned>(end_px - start_px) * 8u;
     last_band = band == g.bands - 1;
   };
-  auto issue = [&](int item, int buf) {  // thread 0 only
+  auto issue = [&](const Item& item, int buf) {  // the 32 threads of warp 0: lane l copies planes l, l+32, ...
     int s, b0, nbk, oy0, oy1, start_px;
     unsigned bytes;
     bool lb;
@@ -135,8 +154,20 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
     const unsigned bar = smem_u32(&bars[buf]);
     // earlier generic-proxy writes to this buffer (the zeroed bottom row) precede the async writes
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes * nbk) : "memory");
-    for (int pi = 0; pi < nbk; ++pi) {
+    // the phase cannot complete before this arrival, whatever order the copies land in
+    if (threadIdx.x == 0)
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes * nbk) : "memory");
+    if (PACKED) {
+      if (threadIdx.x == 0) {
+        const __half* src = in + (static_cast<size_t>(s) * g.B + b0) * g.Pin * 4;
+        const unsigned dst = smem_u32(smem_raw) + buf * buf_bytes + 16u;  // one zero pixel pair in front
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                     "l"(src), "r"(bytes * nbk), "r"(bar)
+                     : "memory");
+      }
+      return;
+    }
+    for (int pi = threadIdx.x; pi < nbk; pi += 32) {
       const __half* src = in + ((static_cast<size_t>(s) * g.B + b0 + pi) * g.Pin + start_px) * 4;
       const unsigned dst =
           smem_u32(smem_raw) + buf * buf_bytes + (static_cast<unsigned>(pi) * g.plane_stride_px + g.head_px) * 8u;
@@ -148,9 +179,13 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
 
   pdl_launch_dependents();
   // the zero heads are written once; copies never touch them
-  for (int i = threadIdx.x; i < 2 * g.nb * g.head_px; i += blockDim.x) {
-    const int plane = i / g.head_px, px = i - plane * g.head_px;
-    *reinterpret_cast<uint2*>(smem_raw + (static_cast<size_t>(plane) * g.plane_stride_px + px) * 8) = make_uint2(0u, 0u);
+  if (PACKED) {
+    if (threadIdx.x < 4) *reinterpret_cast<uint2*>(smem_raw + (threadIdx.x >> 1) * buf_bytes + (threadIdx.x & 1) * 8) = make_uint2(0u, 0u);
+  } else {
+    for (int i = threadIdx.x; i < 2 * g.nb * g.head_px; i += blockDim.x) {
+      const int plane = i / g.head_px, px = i - plane * g.head_px;
+      *reinterpret_cast<uint2*>(smem_raw + (static_cast<size_t>(plane) * g.plane_stride_px + px) * 8) = make_uint2(0u, 0u);
+    }
   }
   pdl_wait();  // the first staging copy below reads the previous kernel's output
   if (threadIdx.x == 0) {
@@ -158,9 +193,14 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bars[1])) : "memory");
     timed_out = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    if (count > 0) issue(first, 0);
   }
   __syncthreads();
+  // column owned by this thread in the first pass over an item's columns: (plane, sub-band, x)
+  const int vp_first = static_cast<int>(threadIdx.x) / Wo;
+  const int x_first = static_cast<int>(threadIdx.x) - vp_first * Wo;
+  const int pi_first = vp_first / g.sub, sb_first = vp_first - pi_first * g.sub;
+  Item cur = {first / (g.bands * g.bchunks), (first / g.bands) % g.bchunks, first % g.bands};
+  if (threadIdx.x < 32 && count > 0) issue(cur, 0);
 
   float2 wlo[9], whi[9];  // 9 taps x (channels 0-1, channels 2-3) of the current slice
   float2 blo = make_float2(0.f, 0.f), bhi = blo;
@@ -172,9 +212,10 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
     int s, b0, nbk, oy0, oy1, start_px;
     unsigned bytes;
     bool last_band;
-    item_rows(first + i, s, b0, nbk, oy0, oy1, start_px, bytes, last_band);
+    item_rows(cur, s, b0, nbk, oy0, oy1, start_px, bytes, last_band);
+    cur = advance(cur);
     // the other buffer was last read in iteration i-1, which ended with a barrier: refill it now
-    if (threadIdx.x == 0 && i + 1 < count) issue(first + i + 1, buf ^ 1);
+    if (threadIdx.x < 32 && i + 1 < count) issue(cur, buf ^ 1);
     if (s != cur_s) {
       cur_s = s;
 #pragma unroll
@@ -215,7 +256,7 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
     if (*reinterpret_cast<volatile unsigned*>(&timed_out)) break;  // give up; results of this launch are invalid
 
     unsigned char* buf_base = smem_raw + buf * buf_bytes;
-    if (MODE != 2 && (oy1 - 1) * stride - pt + 2 >= H) {
+    if (MODE != 2 && !PACKED && (oy1 - 1) * stride - pt + 2 >= H) {
       // this band reads row H: W+1 zero pixels right after the last image row (they replace the
       // plane's own padding pixel and whatever an earlier item left there)
       const int z0 = H * W - start_px;
@@ -230,13 +271,19 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
     const unsigned buf_addr = smem_u32(buf_base);
     const int cols = nbk * g.sub * Wo;
     for (int c = threadIdx.x; c < cols; c += blockDim.x) {
-      const int x = c % Wo, vp = c / Wo;
-      const int sb = vp % g.sub, pi = vp / g.sub;
+      int x = x_first, sb = sb_first, pi = pi_first;  // the first pass uses the decomposition made once per CTA
+      if (c != static_cast<int>(threadIdx.x)) {
+        const int vp = c / Wo;
+        x = c - vp * Wo;
+        pi = vp / g.sub;
+        sb = vp - pi * g.sub;
+      }
       const int ya = oy0 + sb * g.tr, yb = min(oy1, ya + g.tr);
       if (ya >= yb) continue;
       // plane_zero: a pixel of the zero head; data: where pixel (0,0) of the plane would be staged
-      const unsigned plane_zero = buf_addr + static_cast<unsigned>(pi) * g.plane_stride_px * 8u;
-      const unsigned data = plane_zero + static_cast<unsigned>(g.head_px - start_px) * 8u;
+      const unsigned plane_zero = PACKED ? buf_addr : buf_addr + static_cast<unsigned>(pi) * g.plane_stride_px * 8u;
+      const unsigned data = PACKED ? buf_addr + 16u + static_cast<unsigned>(pi) * g.Pin * 8u
+                                   : plane_zero + static_cast<unsigned>(g.head_px - start_px) * 8u;
       const size_t out_off = ((static_cast<size_t>(s) * g.B + b0 + pi) * g.Pout + static_cast<size_t>(ya) * Wo + x) * 4;
       __half* op = out + out_off;
       const ptrdiff_t res_minus_out = res - out;  // only used when TAIL
@@ -287,6 +334,7 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
         // stays on a zero pixel
         unsigned tp[3], step[3];
         const int iy_first = ya * stride - pt;
+        int iy_cur = iy_first;
 #pragma unroll
         for (int k = 0; k < 3; ++k) {
           const int ix = x * stride - g.pl + k;
@@ -296,10 +344,21 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
         }
         auto next_row = [&]() {
           uint2 u[3];
+          if (PACKED) {
+            const bool vy = iy_cur >= 0 && iy_cur < H;  // outside the plane lie the neighbours' rows, not zeros
+            ++iy_cur;
 #pragma unroll
-          for (int k = 0; k < 3; ++k) {
-            u[k] = lds64(tp[k]);
-            tp[k] += step[k];
+            for (int k = 0; k < 3; ++k) {
+              u[k] = make_uint2(0u, 0u);
+              if (vy) u[k] = lds64(tp[k]);
+              tp[k] += step[k];
+            }
+          } else {
+#pragma unroll
+            for (int k = 0; k < 3; ++k) {
+              u[k] = lds64(tp[k]);
+              tp[k] += step[k];
+            }
           }
           return widen(u);
         };
@@ -434,7 +493,14 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
     g.bands = (total_sub + g.sub - 1) / g.sub;
     g.plane_stride_px = smem_for(g);
   }
-  const size_t smem = static_cast<size_t>(g.plane_stride_px) * 8 * g.nb * 2;
+  // the fast paths need the rows above and below the image to be at most one (zero rows in the buffer)
+  const int overshoot = (g.Ho - 1) * g.stride - g.pt + 2 - (g.H - 1);
+  const bool edge_ok = g.dil == 1 && g.pt <= 1 && overshoot <= 1;
+  const int mode = (edge_ok && g.stride == 1) ? 0 : (edge_ok && g.stride == 2) ? 1 : 2;
+  // small planes, several per item, each walked top to bottom by its threads: stage them with one copy
+  const bool packed = mode != 2 && g.bands == 1 && g.sub == 1 && g.nb > 4;
+  g.packed = packed ? 1 : 0;
+  const size_t smem = packed ? (static_cast<size_t>(g.Pin) * 8 * g.nb + 16) * 2 : static_cast<size_t>(g.plane_stride_px) * 8 * g.nb * 2;
   if (smem > static_cast<size_t>(kMaxSmem)) return static_cast<int>(cudaErrorInvalidConfiguration);
   g.bchunks = (g.B + g.nb - 1) / g.nb;
   const long long items = static_cast<long long>(g.S) * g.bchunks * g.bands;
@@ -458,10 +524,6 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
   if (ctas_per_sm < 1) ctas_per_sm = 1;
   long long grid = static_cast<long long>(sms) * ctas_per_sm;
   if (grid > items) grid = items;
-  // the fast paths need the rows above and below the image to be at most one (zero rows in the buffer)
-  const int overshoot = (g.Ho - 1) * g.stride - g.pt + 2 - (g.H - 1);
-  const bool edge_ok = g.dil == 1 && g.pt <= 1 && overshoot <= 1;
-  const int mode = (edge_ok && g.stride == 1) ? 0 : (edge_ok && g.stride == 2) ? 1 : 2;
   const int act = r.ep.act_pre;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const __half* in = static_cast<const __half*>(p.in0);
@@ -469,25 +531,29 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
   const float* b = static_cast<const float*>(p.bias);
   const __half* res = static_cast<const __half*>(p.res);
   __half* out = static_cast<__half*>(p.out);
-  static bool attr_done[3][3][2] = {};
+  static bool attr_done[3][3][2][2] = {};
   const bool tail = r.ep.has_res || r.ep.act_post != GI_ACT_NONE;
-#define GI_DW_LAUNCH(M, A, T)                                                                                                 \
+#define GI_DW_LAUNCH(M, A, T, P)                                                                                                 \
   do {                                                                                                                        \
-    if (!attr_done[M][A][T]) {                                                                                                \
+    if (!attr_done[M][A][T][P]) {                                                                                                \
       const cudaError_t e =                                                                                                   \
-          cudaFuncSetAttribute(depthwise_f16_kernel<M, A, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);         \
+          cudaFuncSetAttribute(depthwise_f16_kernel<M, A, T, P>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);         \
       if (e != cudaSuccess) return static_cast<int>(e);                                                                       \
-      attr_done[M][A][T] = true;                                                                                              \
+      attr_done[M][A][T][P] = true;                                                                                              \
     }                                                                                                                         \
-    launch_pdl(depthwise_f16_kernel<M, A, T>, static_cast<unsigned>(grid), threads, smem, st, in, w, b, res, out, g, r.ep);           \
+    launch_pdl(depthwise_f16_kernel<M, A, T, P>, static_cast<unsigned>(grid), threads, smem, st, in, w, b, res, out, g, r.ep);           \
   } while (0)
 #define GI_DW_ACT(M, A)       \
   do {                        \
-    if (tail) {               \
-      GI_DW_LAUNCH(M, A, 1);  \
-    } else {                  \
-      GI_DW_LAUNCH(M, A, 0);  \
-    }                         \
+    if (tail && packed) {        \
+      GI_DW_LAUNCH(M, A, 1, 1);  \
+    } else if (tail) {           \
+      GI_DW_LAUNCH(M, A, 1, 0);  \
+    } else if (packed) {         \
+      GI_DW_LAUNCH(M, A, 0, 1);  \
+    } else {                     \
+      GI_DW_LAUNCH(M, A, 0, 0);  \
+    }                            \
   } while (0)
 #define GI_DW_MODE(M)              \
   do {                             \
