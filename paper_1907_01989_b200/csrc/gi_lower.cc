@@ -170,9 +170,10 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
           const bool tc = e->storage == GI_F16 && e->opt.pointwise != GI_PW_SIMT;
           // many input channels: the lane-per-pixel kernel (dense weight tile); few: the pixel-pair
           // kernel (activations by TMA)
-          // (measured on MobileNetV2 at batch 256: the lane kernel wins from ~144 input channels on,
-          // except with a residual to read or a very deep, narrow projection)
-          const bool lane_auto = din->c >= 144 && !r.ep.has_res && !(din->c >= 768 && op.d.cout <= 192);
+          // (measured on MobileNetV2 at batch 256: the lane kernel wins from ~144 input channels on
+          // small planes and from 192 on everywhere, except for very deep, narrow projections)
+          const bool lane_auto = (din->c >= 192 || (din->c >= 144 && din->h * din->w < 2048)) &&
+                                 !(din->c >= 768 && op.d.cout <= 192);
           const bool lane_kernel = e->opt.pointwise == GI_PW_TC_LANE || (e->opt.pointwise == GI_PW_AUTO && lane_auto);
           if (pointwise && tc && lane_kernel && pointwise_ts_supported(din->c, op.d.cout)) {
             r.kernel = GI_KERNEL_POINTWISE_TS;

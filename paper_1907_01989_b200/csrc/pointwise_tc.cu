@@ -219,12 +219,22 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
         const unsigned t_addr = tmem_base + acc * acc_cols + (static_cast<unsigned>(quarter * 32) << 16);
         const float4* bias4 = reinterpret_cast<const float4*>(p.bias) + static_cast<size_t>(nt) * p.nts;
 
-        auto issue = [&](unsigned* r, float4* b, int c) {
+        // the chunk's bias and residual are fetched together with its accumulator columns, one chunk ahead
+        auto issue = [&](unsigned* r, float4* b, uint4* q, int c) {
           tmem_ld16(t_addr + static_cast<unsigned>(c) * 16u, r);
           b[0] = __ldg(bias4 + 2 * c);
           b[1] = __ldg(bias4 + 2 * c + 1);
+          if (TAIL) {
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+              const int so = nt * p.nts + 2 * c + j;
+              q[j] = make_uint4(0u, 0u, 0u, 0u);
+              if (p.has_res && so < p.s_out && row_ok)
+                q[j] = __ldg(reinterpret_cast<const uint4*>(p.res + (static_cast<size_t>(so) * p.m_total_px + 2u * row) * 4u));
+            }
+          }
         };
-        auto finish = [&](const unsigned* r, const float4* b, int c) {
+        auto finish = [&](const unsigned* r, const float4* b, const uint4* q, int c) {
 #pragma unroll
           for (int j = 0; j < 2; ++j) {
             const int so = nt * p.nts + 2 * c + j;
@@ -249,9 +259,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
                 oh[i] = h;
               }
             } else {
-              uint4 rr = make_uint4(0u, 0u, 0u, 0u);
-              if (p.has_res) rr = __ldg(reinterpret_cast<const uint4*>(p.res + off));
-              const __half2* rh = reinterpret_cast<const __half2*>(&rr);
+              const __half2* rh = reinterpret_cast<const __half2*>(&q[j]);
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
                 const float2 f = __half22float2(rh[i]);  // zero when there is no residual
@@ -266,17 +274,18 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
 
         unsigned ra[16], rb[16];
         float4 ba[2], bb[2];
+        uint4 qa[2], qb[2];
         int c = sub;
-        if (c < n_chunks) issue(ra, ba, c);
+        if (c < n_chunks) issue(ra, ba, qa, c);
         for (; c < n_chunks; c += 2 * kEpiWarpsPerQuarter) {
           const int c1 = c + kEpiWarpsPerQuarter, c2 = c + 2 * kEpiWarpsPerQuarter;
           tmem_ld_wait16(ra);
-          if (c1 < n_chunks) issue(rb, bb, c1);
-          finish(ra, ba, c);
+          if (c1 < n_chunks) issue(rb, bb, qb, c1);
+          finish(ra, ba, qa, c);
           if (c1 < n_chunks) {
             tmem_ld_wait16(rb);
-            if (c2 < n_chunks) issue(ra, ba, c2);
-            finish(rb, bb, c1);
+            if (c2 < n_chunks) issue(ra, ba, qa, c2);
+            finish(rb, bb, qb, c1);
           }
         }
         tc_fence_before();

@@ -276,12 +276,26 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
     unsigned tile = 0;
     for (int m = m_first; m < p.m_tiles; m += m_step, ++tile) {
       const unsigned acc = tile & 1u, acc_phase = (tile >> 1) & 1u;
-      if (!mbar_wait(smem_u32(&hdr->acc_full[acc]), acc_phase, abort_flag, p.timeout_ns, &g_ts_error, kErrData)) break;
-      tc_fence_after();
       const unsigned pixel = static_cast<unsigned>(m) * kRows + quarter * 32 + lane;
       const bool px_ok = pixel < p.m_total_px;
+      // the residual does not depend on the accumulator: the first group's is fetched before waiting
+      // for the MMAs, each further group's while the one before it is processed
+      auto fetch_res = [&](uint2* q, int g) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int so = (n_part * p.n_cta) / 4 + g * 4 + j;
+          q[j] = make_uint2(0u, 0u);
+          if (p.has_res && g < groups && so < p.s_out && px_ok)
+            q[j] = __ldg(reinterpret_cast<const uint2*>(p.res + (static_cast<size_t>(so) * p.m_total_px + pixel) * 4));
+        }
+      };
+      uint2 res_cur[4], res_next[4];
+      if (TAIL) fetch_res(res_cur, part_id);
+      if (!mbar_wait(smem_u32(&hdr->acc_full[acc]), acc_phase, abort_flag, p.timeout_ns, &g_ts_error, kErrData)) break;
+      tc_fence_after();
       const unsigned t_addr = tmem_base + lane_bits + acc * acc_cols;
       for (int g = part_id; g < groups; g += kParts) {
+        if (TAIL) fetch_res(res_next, g + kParts);
         unsigned r[16];
         tmem_ld16(t_addr + g * 16, r);
         tmem_ld_wait16(r);
@@ -307,8 +321,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
               h1 = __hmin2(h1, __float2half2_rn(6.f));
             }
           } else {
-            uint2 q = make_uint2(0u, 0u);
-            if (p.has_res) q = __ldg(reinterpret_cast<const uint2*>(p.res + off));
+            const uint2 q = res_cur[j];
             const float2 r0 = __half22float2(*reinterpret_cast<const __half2*>(&q.x));
             const float2 r1 = __half22float2(*reinterpret_cast<const __half2*>(&q.y));
             h0 = __floats2half2_rn(act1(act1(v0.x, ACT) + r0.x, p.act_post), act1(act1(v0.y, ACT) + r0.y, p.act_post));
@@ -318,6 +331,10 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
           o.x = *reinterpret_cast<const unsigned*>(&h0);
           o.y = *reinterpret_cast<const unsigned*>(&h1);
           *reinterpret_cast<uint2*>(p.out + off) = o;
+        }
+        if (TAIL) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) res_cur[j] = res_next[j];
         }
       }
       tc_fence_before();
