@@ -302,7 +302,7 @@ int launch_conv3x3_tc(const LaunchRec& r, const Ptrs& p, void* stream) {
   // a few CTAs per SM: one CTA's gather latency hides behind another's epilogue; tensor memory
   // allows 512 / tmem_cols of them
   int per_sm = static_cast<int>(512u / cols);
-  if (per_sm > 4) per_sm = 4;
+  if (per_sm > 8) per_sm = 8;
   if (per_sm < 1) per_sm = 1;
   long long grid = static_cast<long long>(sms) * per_sm;
   if (grid > tiles) grid = tiles;

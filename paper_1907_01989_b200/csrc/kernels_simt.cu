@@ -66,16 +66,15 @@ __device__ __forceinline__ float4 epilogue(float4 v, const Epilogue& ep, const T
 }
 
 // ------------------------------------------------------------------ layout conversion
+// grid: x over the pixels of a plane (padding pixel included), y over planes (slice * B + image)
 template <typename T>
 __global__ void pack_kernel(const T* __restrict__ nhwc, T* __restrict__ out, int B, int HW, int C, int P, int S) {
   pdl_launch_dependents();
   pdl_wait();
-  const size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x;
-  const size_t total = static_cast<size_t>(S) * B * P;
-  if (idx >= total) return;
-  const int pix = static_cast<int>(idx % P);
-  const int b = static_cast<int>((idx / P) % B);
-  const int s = static_cast<int>(idx / (static_cast<size_t>(P) * B));
+  const int pix = blockIdx.x * blockDim.x + threadIdx.x;
+  if (pix >= P) return;
+  const int plane = blockIdx.y;
+  const int s = plane / B, b = plane - s * B;
   float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
   if (pix < HW) {
     const T* src = nhwc + (static_cast<size_t>(b) * HW + pix) * C + s * 4;
@@ -84,7 +83,7 @@ __global__ void pack_kernel(const T* __restrict__ nhwc, T* __restrict__ out, int
     for (int j = 0; j < n; ++j) t[j] = Px<T>::get(src + j);
     v = make_float4(t[0], t[1], t[2], t[3]);
   }
-  Px<T>::store(out + idx * 4, v);
+  Px<T>::store(out + (static_cast<size_t>(plane) * P + pix) * 4, v);
 }
 
 template <typename T>
@@ -320,11 +319,12 @@ inline unsigned blocks_for(size_t n, unsigned per) { return static_cast<unsigned
 int launch_pack(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int S = slices(r.C), P = plane_pixels(r.H, r.W), HW = r.H * r.W;
-  const size_t total = static_cast<size_t>(S) * r.B * P;
-  GI_BY_STORAGE((launch_pdl(pack_kernel<__half>, blocks_for(total, 256), 256, 0, st, static_cast<const __half*>(p.in0),
-                                                                             static_cast<__half*>(p.out), r.B, HW, r.C, P, S)),
-                (launch_pdl(pack_kernel<float>, blocks_for(total, 256), 256, 0, st, static_cast<const float*>(p.in0),
-                                                                            static_cast<float*>(p.out), r.B, HW, r.C, P, S)));
+  if (static_cast<long long>(S) * r.B > 65535) return static_cast<int>(cudaErrorInvalidConfiguration);
+  const dim3 grid(blocks_for(P, 256), S * r.B);
+  GI_BY_STORAGE((launch_pdl(pack_kernel<__half>, grid, 256, 0, st, static_cast<const __half*>(p.in0), static_cast<__half*>(p.out),
+                            r.B, HW, r.C, P, S)),
+                (launch_pdl(pack_kernel<float>, grid, 256, 0, st, static_cast<const float*>(p.in0), static_cast<float*>(p.out), r.B,
+                            HW, r.C, P, S)));
   return static_cast<int>(cudaGetLastError());
 }
 
