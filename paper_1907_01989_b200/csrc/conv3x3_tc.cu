@@ -45,7 +45,9 @@ struct StemParams {
   int stride, dil, pt, pl;
   int s_out, n_pad;          // output slices; Cout rounded up to a multiple of 16
   int tiles;                 // ceil(B * Pout / 128)
-  int act_pre, has_res, act_post;
+  int step_b, step_q;        // gridDim.x * 128 pixels = step_b planes + step_q pixels
+  unsigned m_total;          // B * Pout (< 2^31)
+  int has_res, act_post;
   unsigned tmem_cols;
   unsigned timeout_ns;
 };
@@ -63,7 +65,9 @@ __device__ __forceinline__ float act1(float v, int kind) {
   return v;
 }
 
-__global__ void __launch_bounds__(kThreads, 2) conv3x3_tc_kernel(const StemParams p) {
+// ACT: activation right after the bias; TAIL: a residual add and / or a second activation follow
+template <int ACT, bool TAIL>
+__global__ void __launch_bounds__(kThreads, 6) conv3x3_tc_kernel(const StemParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   Header* hdr = reinterpret_cast<Header*>(smem);
   unsigned char* a_tiles = smem + 1024;                 // 2 x kABytes
@@ -83,6 +87,11 @@ __global__ void __launch_bounds__(kThreads, 2) conv3x3_tc_kernel(const StemParam
   // weights: plain copy into shared memory, then made visible to the tensor core's proxy
   for (int i = threadIdx.x; i < kKCores * p.n_pad; i += kThreads)
     reinterpret_cast<uint4*>(b_tile)[i] = __ldg(reinterpret_cast<const uint4*>(p.wts) + i);
+  // K elements 40..47 of both operand buffers are padding: zeroed once, never written again
+  if (threadIdx.x < kRows) {
+    reinterpret_cast<uint4*>(a_tiles)[5 * kRows + threadIdx.x] = make_uint4(0u, 0u, 0u, 0u);
+    reinterpret_cast<uint4*>(a_tiles + kABytes)[5 * kRows + threadIdx.x] = make_uint4(0u, 0u, 0u, 0u);
+  }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   tc_fence_before();
   __syncthreads();
@@ -92,29 +101,38 @@ __global__ void __launch_bounds__(kThreads, 2) conv3x3_tc_kernel(const StemParam
   pdl_wait();
   const unsigned tmem_base = hdr->tmem_addr;
   const unsigned n_cols = static_cast<unsigned>(p.n_pad);
-  const long long m_total = static_cast<long long>(p.B) * p.Pout;
 
   if (warp < 4) {
     const int t = threadIdx.x;  // row of the tile = TMEM lane
-    // ---- gather of one tile into operand buffer `buf`
-    auto gather = [&](int tile, int buf) {
-      const long long gp = static_cast<long long>(tile) * kRows + t;
+    const int real_px = p.Ho * p.Wo;
+    // ---- gather of one tile into operand buffer `buf`; this thread's pixel is q of image b
+    auto gather = [&](int buf, int b, int q, bool in_tensor) {
       uint2 tap[10];
 #pragma unroll
       for (int k = 0; k < 10; ++k) tap[k] = make_uint2(0u, 0u);
-      if (gp < m_total) {
-        const int b = static_cast<int>(gp / p.Pout), q = static_cast<int>(gp - static_cast<long long>(b) * p.Pout);
-        if (q < p.Ho * p.Wo) {
-          const int oy = q / p.Wo, ox = q - oy * p.Wo;
-          const __half* plane = p.in + static_cast<size_t>(b) * p.Pin * 4;
+      if (in_tensor && q < real_px) {
+        const int oy = q / p.Wo, ox = q - oy * p.Wo;
+        const int iy0 = oy * p.stride - p.pt, ix0 = ox * p.stride - p.pl;
+        const uint2* in8 = reinterpret_cast<const uint2*>(p.in);
+        const long long first = static_cast<long long>(b) * p.Pin + static_cast<long long>(iy0) * p.W + ix0;
+        if (iy0 >= 0 && ix0 >= 0 && iy0 + 2 * p.dil < p.H && ix0 + 2 * p.dil < p.W) {
+          // whole window inside the image (all but the border pixels): no per-tap tests
+          const uint2* row = in8 + first;
+          const int row_step = p.dil * p.W;
+#pragma unroll
+          for (int ky = 0; ky < 3; ++ky, row += row_step) {
+#pragma unroll
+            for (int kx = 0; kx < 3; ++kx) tap[ky * 3 + kx] = __ldg(row + kx * p.dil);
+          }
+        } else {
 #pragma unroll
           for (int ky = 0; ky < 3; ++ky) {
-            const int iy = oy * p.stride - p.pt + ky * p.dil;
+            const int iy = iy0 + ky * p.dil;
 #pragma unroll
             for (int kx = 0; kx < 3; ++kx) {
-              const int ix = ox * p.stride - p.pl + kx * p.dil;
+              const int ix = ix0 + kx * p.dil;
               if (iy >= 0 && iy < p.H && ix >= 0 && ix < p.W)
-                tap[ky * 3 + kx] = __ldg(reinterpret_cast<const uint2*>(plane + (static_cast<size_t>(iy) * p.W + ix) * 4));
+                tap[ky * 3 + kx] = __ldg(in8 + (first + static_cast<long long>(ky * p.dil) * p.W + kx * p.dil));
             }
           }
         }
@@ -122,75 +140,105 @@ __global__ void __launch_bounds__(kThreads, 2) conv3x3_tc_kernel(const StemParam
       uint4* dst = reinterpret_cast<uint4*>(a_tiles + buf * kABytes) + t;
 #pragma unroll
       for (int j = 0; j < 5; ++j) dst[j * kRows] = make_uint4(tap[2 * j].x, tap[2 * j].y, tap[2 * j + 1].x, tap[2 * j + 1].y);
-      dst[5 * kRows] = make_uint4(0u, 0u, 0u, 0u);
       // generic-proxy writes above must be visible to the MMA (async proxy) before the arrival
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       mbar_arrive(smem_u32(&hdr->a_full[buf]));
     };
-    // ---- epilogue of one tile from accumulator `buf`
-    auto epilogue = [&](int tile, int buf, unsigned phase) -> bool {
+    // ---- epilogue of one tile from accumulator `buf`; gp = this thread's pixel in the whole tensor
+    auto epilogue = [&](int buf, unsigned phase, unsigned gp, bool in_tensor, bool real) -> bool {
       if (!mbar_wait(smem_u32(&hdr->acc_full[buf]), phase, abort_flag, p.timeout_ns, &g_conv_tc_error, 4u)) return false;
       tc_fence_after();
-      const long long gp = static_cast<long long>(tile) * kRows + t;
-      const bool in_tensor = gp < m_total;
-      bool real = false;
-      if (in_tensor) {
-        const int b = static_cast<int>(gp / p.Pout);
-        real = static_cast<int>(gp - static_cast<long long>(b) * p.Pout) < p.Ho * p.Wo;
-      }
       const unsigned t_addr = tmem_base + buf * n_cols + (static_cast<unsigned>(warp * 32) << 16);
-      for (unsigned c0 = 0; c0 < n_cols; c0 += 16) {
-        unsigned r[16];
-        tmem_ld16(t_addr + c0, r);
-        tmem_ld_wait16(r);
+      auto finish = [&](const unsigned* r, unsigned c0) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int so = static_cast<int>(c0 / 4) + j;
           if (so >= p.s_out || !in_tensor) continue;
-          const size_t off = (static_cast<size_t>(so) * m_total + gp) * 4;  // in halves
+          const size_t off = (static_cast<size_t>(so) * p.m_total + gp) * 4;  // in halves
           uint2 o = make_uint2(0u, 0u);  // the padding pixel of an odd plane stays zero
           if (real) {
             const float4 bv = __ldg(reinterpret_cast<const float4*>(p.bias) + so);
-            float v[4] = {__uint_as_float(r[4 * j]) + bv.x, __uint_as_float(r[4 * j + 1]) + bv.y,
-                          __uint_as_float(r[4 * j + 2]) + bv.z, __uint_as_float(r[4 * j + 3]) + bv.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) v[e] = act1(v[e], p.act_pre);
-            if (p.has_res) {
-              const uint2 q = __ldg(reinterpret_cast<const uint2*>(p.res + off));
-              const float2 r0 = __half22float2(*reinterpret_cast<const __half2*>(&q.x));
-              const float2 r1 = __half22float2(*reinterpret_cast<const __half2*>(&q.y));
-              v[0] += r0.x;
-              v[1] += r0.y;
-              v[2] += r1.x;
-              v[3] += r1.y;
+            const float2 v0 = __fadd2_rn(make_float2(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1])), make_float2(bv.x, bv.y));
+            const float2 v1 = __fadd2_rn(make_float2(__uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3])), make_float2(bv.z, bv.w));
+            __half2 h0, h1;
+            if (!TAIL) {
+              // clamping after the rounding equals rounding after the clamp: 0 and 6 are fp16 values
+              h0 = __floats2half2_rn(v0.x, v0.y);
+              h1 = __floats2half2_rn(v1.x, v1.y);
+              if (ACT != GI_ACT_NONE) {
+                h0 = __hmax2(h0, __float2half2_rn(0.f));
+                h1 = __hmax2(h1, __float2half2_rn(0.f));
+              }
+              if (ACT == GI_ACT_RELU6) {
+                h0 = __hmin2(h0, __float2half2_rn(6.f));
+                h1 = __hmin2(h1, __float2half2_rn(6.f));
+              }
+            } else {
+              float2 r0 = make_float2(0.f, 0.f), r1 = make_float2(0.f, 0.f);
+              if (p.has_res) {
+                const uint2 q = __ldg(reinterpret_cast<const uint2*>(p.res + off));
+                r0 = __half22float2(*reinterpret_cast<const __half2*>(&q.x));
+                r1 = __half22float2(*reinterpret_cast<const __half2*>(&q.y));
+              }
+              h0 = __floats2half2_rn(act1(act1(v0.x, ACT) + r0.x, p.act_post), act1(act1(v0.y, ACT) + r0.y, p.act_post));
+              h1 = __floats2half2_rn(act1(act1(v1.x, ACT) + r1.x, p.act_post), act1(act1(v1.y, ACT) + r1.y, p.act_post));
             }
-#pragma unroll
-            for (int e = 0; e < 4; ++e) v[e] = act1(v[e], p.act_post);
-            const __half2 lo = __floats2half2_rn(v[0], v[1]), hi = __floats2half2_rn(v[2], v[3]);
-            o.x = *reinterpret_cast<const unsigned*>(&lo);
-            o.y = *reinterpret_cast<const unsigned*>(&hi);
+            o.x = *reinterpret_cast<const unsigned*>(&h0);
+            o.y = *reinterpret_cast<const unsigned*>(&h1);
           }
           *reinterpret_cast<uint2*>(p.out + off) = o;
+        }
+      };
+      // two 16-column reads in flight: the next one is issued before the current one is processed
+      unsigned ra[16], rb[16];
+      tmem_ld16(t_addr, ra);
+      for (unsigned c0 = 0; c0 < n_cols; c0 += 32) {
+        tmem_ld_wait16(ra);
+        if (c0 + 16 < n_cols) tmem_ld16(t_addr + c0 + 16, rb);
+        finish(ra, c0);
+        if (c0 + 16 < n_cols) {
+          tmem_ld_wait16(rb);
+          if (c0 + 32 < n_cols) tmem_ld16(t_addr + c0 + 32, ra);
+          finish(rb, c0 + 16);
         }
       }
       tc_fence_before();
       return true;
     };
 
-    // software pipeline over this CTA's tiles: gather(i+1) is issued before epilogue(i)
+    // software pipeline over this CTA's tiles: gather(i+1) is issued before epilogue(i).  The
+    // pixel of this thread advances by a fixed number of planes and pixels per step: no divisions
+    // by the plane size in the loop
+    const unsigned gp0 = static_cast<unsigned>(blockIdx.x) * kRows + t;
+    int b = static_cast<int>(gp0 / static_cast<unsigned>(p.Pout));
+    int q = static_cast<int>(gp0 - static_cast<unsigned>(b) * p.Pout);
+    unsigned gp = gp0;
+    const unsigned gp_step = gridDim.x * kRows;
     int n = 0;
-    int prev_tile = -1;
+    bool have_prev = false, prev_in = false, prev_real = false;
+    unsigned prev_gp = 0;
     for (int tile = blockIdx.x; tile < p.tiles; tile += gridDim.x, ++n) {
       // operand buffer n&1 was read by the MMAs of tile n-2, whose accumulator the epilogue of
       // tile n-2 has already waited for, so the buffer is free
-      gather(tile, n & 1);
-      if (prev_tile >= 0 && !epilogue(prev_tile, (n - 1) & 1, ((n - 1) >> 1) & 1)) {
-        prev_tile = -1;
+      const bool in_tensor = gp < p.m_total;
+      gather(n & 1, b, q, in_tensor);
+      if (have_prev && !epilogue((n - 1) & 1, ((n - 1) >> 1) & 1, prev_gp, prev_in, prev_real)) {
+        have_prev = false;
         break;
       }
-      prev_tile = tile;
+      have_prev = true;
+      prev_gp = gp;
+      prev_in = in_tensor;
+      prev_real = in_tensor && q < real_px;
+      gp += gp_step;
+      b += p.step_b;
+      q += p.step_q;
+      if (q >= p.Pout) {
+        q -= p.Pout;
+        ++b;
+      }
     }
-    if (prev_tile >= 0) epilogue(prev_tile, (n - 1) & 1, ((n - 1) >> 1) & 1);
+    if (have_prev) epilogue((n - 1) & 1, ((n - 1) >> 1) & 1, prev_gp, prev_in, prev_real);
   } else if (lane == 0) {
     // ---- MMA issuer
     // instruction descriptor: fp32 accumulator, fp16 A and B, both K-major, M = 128, N = n_pad
@@ -276,9 +324,10 @@ int launch_conv3x3_tc(const LaunchRec& r, const Ptrs& p, void* stream) {
   k.n_pad = r.tc_nt;
   const long long m_total = static_cast<long long>(r.B) * k.Pout;
   const long long tiles = (m_total + kRows - 1) / kRows;
-  if (tiles > 2147483647LL) return static_cast<int>(cudaErrorInvalidConfiguration);
+  // pixel indices are kept in 32 bits inside the kernel, with room for one step past the end
+  if (m_total > (1LL << 30)) return static_cast<int>(cudaErrorInvalidConfiguration);
   k.tiles = static_cast<int>(tiles);
-  k.act_pre = r.ep.act_pre;
+  k.m_total = static_cast<unsigned>(m_total);
   k.has_res = r.ep.has_res;
   k.act_post = r.ep.act_post;
   unsigned cols = 32;
@@ -294,19 +343,45 @@ int launch_conv3x3_tc(const LaunchRec& r, const Ptrs& p, void* stream) {
   }
   const size_t smem = 1024 + 2 * kABytes + static_cast<size_t>(kKCores) * k.n_pad * 16;
   if (!attr_set) {
-    const cudaError_t e = cudaFuncSetAttribute(conv3x3_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               1024 + 2 * kABytes + kKCores * kMaxN * 16);
+    cudaError_t e = cudaSuccess;
+    const int bytes = 1024 + 2 * kABytes + kKCores * kMaxN * 16;
+#define GI_C3_ATTR(A, T) \
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(conv3x3_tc_kernel<A, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)
+    GI_C3_ATTR(GI_ACT_NONE, false);
+    GI_C3_ATTR(GI_ACT_RELU, false);
+    GI_C3_ATTR(GI_ACT_RELU6, false);
+    GI_C3_ATTR(GI_ACT_NONE, true);
+    GI_C3_ATTR(GI_ACT_RELU, true);
+    GI_C3_ATTR(GI_ACT_RELU6, true);
+#undef GI_C3_ATTR
     if (e != cudaSuccess) return static_cast<int>(e);
     attr_set = true;
   }
   // a few CTAs per SM: one CTA's gather latency hides behind another's epilogue; tensor memory
-  // allows 512 / tmem_cols of them
+  // allows 512 / tmem_cols of them, the register file six
   int per_sm = static_cast<int>(512u / cols);
-  if (per_sm > 8) per_sm = 8;
+  if (per_sm > 6) per_sm = 6;
   if (per_sm < 1) per_sm = 1;
   long long grid = static_cast<long long>(sms) * per_sm;
   if (grid > tiles) grid = tiles;
-  launch_pdl(conv3x3_tc_kernel, static_cast<unsigned>(grid), kThreads, smem, static_cast<cudaStream_t>(stream), k);
+  const long long step = grid * kRows;
+  k.step_b = static_cast<int>(step / k.Pout);
+  k.step_q = static_cast<int>(step % k.Pout);
+  const unsigned g = static_cast<unsigned>(grid);
+  cudaStream_t cu_stream = static_cast<cudaStream_t>(stream);
+  const int act = r.ep.act_pre;
+  const bool tail = k.has_res || k.act_post != GI_ACT_NONE;
+#define GI_C3_LAUNCH(A, T) launch_pdl(conv3x3_tc_kernel<A, T>, g, kThreads, smem, cu_stream, k)
+  if (tail) {
+    if (act == GI_ACT_RELU6) GI_C3_LAUNCH(GI_ACT_RELU6, true);
+    else if (act == GI_ACT_RELU) GI_C3_LAUNCH(GI_ACT_RELU, true);
+    else GI_C3_LAUNCH(GI_ACT_NONE, true);
+  } else {
+    if (act == GI_ACT_RELU6) GI_C3_LAUNCH(GI_ACT_RELU6, false);
+    else if (act == GI_ACT_RELU) GI_C3_LAUNCH(GI_ACT_RELU, false);
+    else GI_C3_LAUNCH(GI_ACT_NONE, false);
+  }
+#undef GI_C3_LAUNCH
   return static_cast<int>(cudaGetLastError());
 }
 
