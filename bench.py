@@ -38,6 +38,7 @@ import numpy as np  # noqa: E402
 NETS = {"v2": ("mobilenet_v2", "MobileNetV2-224"), "v1": ("mobilenet_v1", "MobileNetV1-224"),
         "seg": ("mobilenet_v2_segmentation", "MobileNetV2-513-OS16-seg")}
 PW_MODES = {"auto": 0, "simt": 1, "pair": 2, "lane": 3}
+DW_MODES = {"auto": 0, "stencil": 1, "tc": 2}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -206,7 +207,7 @@ def run_sweep(args):
             spec = wl.single_pointwise(b, hw, cin, cout, residual=args.residual)
             name = f"pw1x1 b{b} {hw}x{hw} {cin}->{cout}"
         g, _ = api.graph_from_spec(spec, api.GI_F16, io_layout=api.GI_PHWC4)
-        ex = g.compile(pointwise=PW_MODES[args.pointwise])
+        ex = g.compile(pointwise=PW_MODES[args.pointwise], depthwise=DW_MODES[args.depthwise])
         ex.bind(dev)
         ops = ex.ops()
         assert len(ops) == 1
@@ -251,6 +252,7 @@ def main():
     ap.add_argument("--net", default="v2", choices=sorted(NETS))
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--pointwise", default="auto", choices=["auto", "simt", "pair", "lane"])
+    ap.add_argument("--depthwise", default="auto", choices=["auto", "stencil", "tc"])
     ap.add_argument("--per-op", default=None, help="write the per-op timing table to this file")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-batch1", action="store_true", help="skip the batch-1 latency leg (keeps profiler runs short)")
@@ -296,7 +298,7 @@ def main():
 
     spec = spec_fn(args.batch)
     graph, _ = api.graph_from_spec(spec, api.GI_F16)
-    ex = graph.compile(pointwise=PW_MODES[args.pointwise])
+    ex = graph.compile(pointwise=PW_MODES[args.pointwise], depthwise=DW_MODES[args.depthwise])
     ex.bind(dev)
     ops = ex.ops()
     # every rank draws its own images: rank r holds images [r*B, (r+1)*B) of the global batch
@@ -412,7 +414,7 @@ def main():
         if not args.no_batch1:
             spec1 = spec_fn(1)
             g1, _ = api.graph_from_spec(spec1, api.GI_F16)
-            ex1 = g1.compile(pointwise=PW_MODES[args.pointwise])
+            ex1 = g1.compile(pointwise=PW_MODES[args.pointwise], depthwise=DW_MODES[args.depthwise])
             ex1.bind(dev)
             x1 = torch.from_numpy(wl.make_input(spec1).astype(np.float16)).to(dev)
             o1 = torch.empty((1,) + tuple(spec1.shapes[spec1.outputs[0]]), dtype=torch.float16, device=dev)
@@ -459,7 +461,7 @@ def main():
                            "launches_per_step": len(ops), "arena_mib": round(ex.info.arena_bytes / 2 ** 20, 1),
                            "l2": "flushed between steps by an untimed 256 MiB memset; a step moves ~"
                                  f"{sum(o.bytes for o in ops) / 1e9:.1f} GB", "parallelism": f"replicas x{world}",
-                           "pointwise": args.pointwise},
+                           "pointwise": args.pointwise, "depthwise": args.depthwise},
                 "roofline": roofline, "cpu_baseline": cpu,
                 "e2e": {"value": e2e_value, "unit": "images/s", "h2d_bytes_per_step": int(x_pin.numel() * 2),
                         "d2h_bytes_per_step": int(out_pin.numel() * 2)},

@@ -17,11 +17,12 @@ STORAGES = [api.GI_F16, api.GI_F32]
 SNAME = {api.GI_F16: "f16", api.GI_F32: "f32"}
 
 
-def check_all_tensors(spec, storage, pointwise=api.GI_PW_AUTO, fuse=True):
+def check_all_tensors(spec, storage, pointwise=api.GI_PW_AUTO, fuse=True, depthwise=api.GI_DW_AUTO):
     """Naive planner keeps every intermediate, so each stored tensor is compared, not only the output."""
     xs = [wl.make_input(spec, index=i) for i in range(len(spec.inputs))]
     ref = og.run(spec, xs, storage=SNAME[storage], fused=fuse, keep_all=True)
-    run = GpuRun(spec, storage, planner=api.GI_PLAN_NAIVE, pointwise=pointwise, fuse=fuse, guard_bytes=4096)
+    run = GpuRun(spec, storage, planner=api.GI_PLAN_NAIVE, pointwise=pointwise, fuse=fuse, guard_bytes=4096,
+                 depthwise=depthwise)
     outs = run.run(xs)
     assert run.guard_intact()
     worst = 0.0
@@ -127,6 +128,49 @@ DW_CASES = [  # batch, hw, c, stride, dilation, residual
 def test_depthwise(storage, case):
     batch, hw, c, stride, dilation, residual = case
     check_all_tensors(wl.single_depthwise(batch, hw, c, stride, dilation, residual), storage)
+
+
+def depthwise_spec(batch, h, w, c, stride, residual, act=wl.ACT_RELU6):
+    b = wl.GraphBuilder(f"dwtc_{batch}x{h}x{w}x{c}_s{stride}", batch, 8)
+    x = b.input(h, w, c)
+    r = b.input(wl.same_pads(h, 3, stride, 1)[0], wl.same_pads(w, 3, stride, 1)[0], c) if residual else None
+    y = b.depthwise(x, 3, stride, 1)
+    if act is not None:
+        y = b.activation(y, act)
+    if residual:
+        y = b.add(r, y)
+    b.output(y)
+    return b.finish()
+
+
+DWTC_CASES = [  # batch, H, W, C, stride, residual: even planes, the shapes the tensor-core depthwise kernel takes
+    (1, 14, 14, 32, 1, False), (3, 14, 14, 20, 1, False), (2, 28, 28, 192, 1, True), (1, 56, 56, 24, 1, False),
+    (2, 112, 112, 8, 1, False), (5, 14, 14, 8, 1, False), (40, 4, 4, 8, 1, False), (1, 2, 2, 4, 1, False),
+    (1, 20, 36, 12, 1, False), (1, 6, 252, 4, 1, True), (2, 14, 14, 96, 2, False), (2, 112, 112, 32, 2, False),
+    (1, 56, 56, 144, 2, True), (2, 36, 20, 12, 2, False), (2, 2, 2, 4, 2, False), (37, 8, 8, 4, 2, False),
+]
+
+
+@pytest.mark.parametrize("case", DWTC_CASES)
+def test_depthwise_tensor_core(case):
+    batch, h, w, c, stride, residual = case
+    spec = depthwise_spec(batch, h, w, c, stride, residual)
+    forced = api.graph_from_spec(spec, api.GI_F16)[0].compile(depthwise=api.GI_DW_TC)
+    kernels = [api.KERNEL_NAMES[o.kernel] for o in forced.ops()]
+    assert "depthwise_tc" in kernels and "depthwise" not in kernels
+    check_all_tensors(spec, api.GI_F16, depthwise=api.GI_DW_TC)
+    # the same graph through the default (stencil) kernel
+    default = api.graph_from_spec(spec, api.GI_F16)[0].compile()
+    assert "depthwise_tc" not in [api.KERNEL_NAMES[o.kernel] for o in default.ops()]
+    check_all_tensors(spec, api.GI_F16)
+    assert api.gi_device_status() == 0
+
+
+@pytest.mark.parametrize("act", [None, wl.ACT_RELU])
+def test_depthwise_tensor_core_other_tails(act):
+    check_all_tensors(depthwise_spec(2, 28, 28, 12, 1, False, act), api.GI_F16, depthwise=api.GI_DW_TC)
+    check_all_tensors(depthwise_spec(2, 28, 28, 12, 2, True, act), api.GI_F16, depthwise=api.GI_DW_TC)
+    assert api.gi_device_status() == 0
 
 
 @pytest.mark.parametrize("storage", STORAGES)
