@@ -33,6 +33,7 @@ struct DwGeom {
   int plane_stride_px;  // pixels reserved per plane in one staging buffer (even)
   int items;            // S * bchunks * bands
   int packed;           // 1: whole small planes, staged back to back by one copy per item
+  int nbuf;             // staging buffers per CTA (2..4): nbuf - 1 items are in flight ahead of the one computed
   unsigned timeout_ns;
 };
 
@@ -105,7 +106,7 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
                                                                 const float* __restrict__ bias, const __half* __restrict__ res,
                                                                 __half* __restrict__ out, const DwGeom g, const Epilogue ep) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[2];
+  __shared__ __align__(8) unsigned long long bars[4];
   __shared__ unsigned timed_out;
   const unsigned buf_bytes = PACKED ? static_cast<unsigned>(g.Pin) * 8u * g.nb + 16u : static_cast<unsigned>(g.plane_stride_px) * 8u * g.nb;
   const int W = g.W, H = g.H, Wo = g.Wo, stride = g.stride, pt = g.pt;
@@ -180,17 +181,17 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
   pdl_launch_dependents();
   // the zero heads are written once; copies never touch them
   if (PACKED) {
-    if (threadIdx.x < 4) *reinterpret_cast<uint2*>(smem_raw + (threadIdx.x >> 1) * buf_bytes + (threadIdx.x & 1) * 8) = make_uint2(0u, 0u);
+    if (static_cast<int>(threadIdx.x) < 2 * g.nbuf)
+      *reinterpret_cast<uint2*>(smem_raw + (threadIdx.x >> 1) * buf_bytes + (threadIdx.x & 1) * 8) = make_uint2(0u, 0u);
   } else {
-    for (int i = threadIdx.x; i < 2 * g.nb * g.head_px; i += blockDim.x) {
+    for (int i = threadIdx.x; i < g.nbuf * g.nb * g.head_px; i += blockDim.x) {
       const int plane = i / g.head_px, px = i - plane * g.head_px;
       *reinterpret_cast<uint2*>(smem_raw + (static_cast<size_t>(plane) * g.plane_stride_px + px) * 8) = make_uint2(0u, 0u);
     }
   }
   pdl_wait();  // the first staging copy below reads the previous kernel's output
   if (threadIdx.x == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bars[0])) : "memory");
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bars[1])) : "memory");
+    for (int b = 0; b < g.nbuf; ++b) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bars[b])) : "memory");
     timed_out = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -200,22 +201,31 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
   const int x_first = static_cast<int>(threadIdx.x) - vp_first * Wo;
   const int pi_first = vp_first / g.sub, sb_first = vp_first - pi_first * g.sub;
   Item cur = {first / (g.bands * g.bchunks), (first / g.bands) % g.bchunks, first % g.bands};
-  if (threadIdx.x < 32 && count > 0) issue(cur, 0);
+  // the first nbuf - 1 items are requested up front; `ahead` is the next item to request
+  Item ahead = cur;
+  for (int j = 0; j < g.nbuf - 1 && j < count; ++j) {
+    if (threadIdx.x < 32) issue(ahead, j);
+    ahead = advance(ahead);
+  }
 
   float2 wlo[9], whi[9];  // 9 taps x (channels 0-1, channels 2-3) of the current slice
   float2 blo = make_float2(0.f, 0.f), bhi = blo;
   int cur_s = -1;
   const int C4 = g.S * 4;
 
+  int buf = 0, ahead_buf = g.nbuf - 1;
+  unsigned round = 0;  // how often the ring of buffers has wrapped: the parity of the wait
   for (int i = 0; i < count; ++i) {
-    const int buf = i & 1;
     int s, b0, nbk, oy0, oy1, start_px;
     unsigned bytes;
     bool last_band;
     item_rows(cur, s, b0, nbk, oy0, oy1, start_px, bytes, last_band);
     cur = advance(cur);
-    // the other buffer was last read in iteration i-1, which ended with a barrier: refill it now
-    if (threadIdx.x < 32 && i + 1 < count) issue(cur, buf ^ 1);
+    // the buffer nbuf - 1 ahead was last read in iteration i-1, which ended with a barrier: refill it now
+    if (i + g.nbuf - 1 < count) {
+      if (threadIdx.x < 32) issue(ahead, ahead_buf);
+      ahead = advance(ahead);
+    }
     if (s != cur_s) {
       cur_s = s;
 #pragma unroll
@@ -229,7 +239,7 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
       bhi = make_float2(v.z, v.w);
     }
     {  // bounded wait for this item's rows
-      const unsigned bar = smem_u32(&bars[buf]), parity = (i >> 1) & 1;
+      const unsigned bar = smem_u32(&bars[buf]), parity = round & 1u;
       unsigned ok = 0;
       unsigned long long t0 = 0;
       for (unsigned spin = 0; !ok; ++spin) {
@@ -292,19 +302,20 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
         uint2 u;
         if (!TAIL) {
           // clamping after the rounding equals rounding after the clamp: 0 and 6 are fp16 values
-          __half2 lo = __floats2half2_rn(a.lo.x, a.lo.y), hi = __floats2half2_rn(a.hi.x, a.hi.y);
-          if (ACT != GI_ACT_NONE) {
-            const __half2 z = __float2half2_rn(0.f);
-            lo = __hmax2(lo, z);
-            hi = __hmax2(hi, z);
-          }
-          if (ACT == GI_ACT_RELU6) {
-            const __half2 six = __float2half2_rn(6.f);
-            lo = __hmin2(lo, six);
-            hi = __hmin2(hi, six);
-          }
+          const __half2 lo = __floats2half2_rn(a.lo.x, a.lo.y), hi = __floats2half2_rn(a.hi.x, a.hi.y);
           u.x = *reinterpret_cast<const unsigned*>(&lo);
           u.y = *reinterpret_cast<const unsigned*>(&hi);
+          // the clamps as signed 16-bit integer min / max on the fp16 bit patterns (negative
+          // values have the sign bit set, non-negative ones order like integers): these run on
+          // the integer pipe, which this kernel leaves idle, instead of the busy fp16 / FMA pipe
+          if (ACT != GI_ACT_NONE) {
+            u.x = __vmaxs2(u.x, 0u);
+            u.y = __vmaxs2(u.y, 0u);
+          }
+          if (ACT == GI_ACT_RELU6) {
+            u.x = __vmins2(u.x, 0x46004600u);
+            u.y = __vmins2(u.y, 0x46004600u);
+          }
         } else {
           float v[4] = {a.lo.x, a.lo.y, a.hi.x, a.hi.y};
 #pragma unroll
@@ -430,6 +441,11 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
       *reinterpret_cast<uint2*>(out + off) = make_uint2(0u, 0u);
     }
     __syncthreads();  // everyone is done with this buffer before it is refilled
+    if (++buf == g.nbuf) {
+      buf = 0;
+      ++round;
+    }
+    if (++ahead_buf == g.nbuf) ahead_buf = 0;
   }
   if (*reinterpret_cast<volatile unsigned*>(&timed_out) && threadIdx.x == 0) {
     // copies already issued may still land: give them the same bounded grace before leaving
@@ -441,7 +457,9 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
   }
 }
 
-constexpr int kMaxSmem = 200 * 1024;  // both staging buffers of one CTA
+constexpr int kMaxSmem = 200 * 1024;    // all staging buffers of one CTA
+constexpr int kSmemPerCta = 110 * 1024; // target: two CTAs per SM
+constexpr int kSmemPerSm = 226 * 1024;
 
 }  // namespace
 
@@ -500,7 +518,12 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
   // small planes, several per item, each walked top to bottom by its threads: stage them with one copy
   const bool packed = mode != 2 && g.bands == 1 && g.sub == 1 && g.nb > 4;
   g.packed = packed ? 1 : 0;
-  const size_t smem = packed ? (static_cast<size_t>(g.Pin) * 8 * g.nb + 16) * 2 : static_cast<size_t>(g.plane_stride_px) * 8 * g.nb * 2;
+  const size_t buf_bytes = packed ? static_cast<size_t>(g.Pin) * 8 * g.nb + 16 : static_cast<size_t>(g.plane_stride_px) * 8 * g.nb;
+  // bytes in flight hide the HBM latency: two CTAs per SM (the register file allows no more),
+  // each with up to three items requested ahead of the one it computes
+  int nbuf = static_cast<int>(static_cast<size_t>(kSmemPerCta) / buf_bytes);
+  g.nbuf = nbuf > 4 ? 4 : nbuf < 2 ? 2 : nbuf;
+  const size_t smem = buf_bytes * g.nbuf;
   if (smem > static_cast<size_t>(kMaxSmem)) return static_cast<int>(cudaErrorInvalidConfiguration);
   g.bchunks = (g.B + g.nb - 1) / g.nb;
   const long long items = static_cast<long long>(g.S) * g.bchunks * g.bands;
@@ -516,7 +539,7 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
   }
   // persistent CTAs, a few per SM so that one CTA's copies overlap another's arithmetic
-  long long ctas_per_sm = static_cast<long long>(kMaxSmem) / static_cast<long long>(smem > 0 ? smem : 1);
+  long long ctas_per_sm = static_cast<long long>(kSmemPerSm) / static_cast<long long>(smem + 1024);
   if (ctas_per_sm > 2048 / threads) ctas_per_sm = 2048 / threads;
   // the grid is oversubscribed 2x: the block scheduler then evens out the tail
   ctas_per_sm *= 2;
