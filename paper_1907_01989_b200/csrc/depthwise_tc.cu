@@ -193,6 +193,7 @@ __global__ void __launch_bounds__(kThreads, 2) depthwise_tc_kernel(const __grid_
   const unsigned data0 = smem_u32(smem + kHeader + kLead);
 
   if (threadIdx.x == 0) {
+    prefetch_tensormap(&tmap);
     for (int i = 0; i < p.stages; ++i) {
       mbar_init(smem_u32(&hdr->full[i]), 1);
       mbar_init(smem_u32(&hdr->empty[i]), 1);

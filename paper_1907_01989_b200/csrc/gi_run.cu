@@ -171,3 +171,14 @@ gi_status gi_run_timed(gi_exec* e, const void* const* dev_inputs, void* const* d
 }
 
 }  // extern "C"
+
+#ifdef GI_TRACE
+namespace gi {
+int pointwise_ts_trace(unsigned long long* dst, int n);
+}
+// debug builds only: copy the timeline table of the lane-per-pixel kernel's last launch
+extern "C" GI_API int gi_debug_trace(int which, unsigned long long* dst, int n) {
+  (void)which;
+  return gi::pointwise_ts_trace(dst, n);
+}
+#endif

@@ -103,6 +103,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
   volatile unsigned* abort_flag = &hdr->abort_flag;
 
   if (threadIdx.x == 0) {
+    prefetch_tensormap(&tmap_a);
     for (int i = 0; i < p.stages; ++i) {
       mbar_init(smem_u32(&hdr->full[i]), 1);
       mbar_init(smem_u32(&hdr->empty[i]), 1);
@@ -465,12 +466,15 @@ int launch_pointwise_tc(const LaunchRec& r, const Ptrs& p, void** state, int lau
   k.epq = wide ? 4 : n_chunks >= 2 ? 2 : 1;
   int ctas_per_sm = wide ? 1 : 2;
   const size_t stage_bytes = static_cast<size_t>(t.kc) * (kSliceBytes + t.nts * kCoreBytes);
-  if (!wide) {
+  const long long units = static_cast<long long>(k.m_tiles) * groups;
+  // no more work units than SMs: a second CTA per SM would stay empty, so the one CTA keeps
+  // all of shared memory for stages in flight
+  if (units <= di.sms) ctas_per_sm = 1;
+  if (ctas_per_sm == 2) {
     const int st2 = static_cast<int>((108 * 1024 - kSmemHeader) / stage_bytes);
     if (st2 < 2) ctas_per_sm = 1;
     else if (st2 < k.stages) k.stages = st2;
   }
-  const long long units = static_cast<long long>(k.m_tiles) * groups;
   const long long slots = static_cast<long long>(di.sms) * ctas_per_sm;
   const unsigned grid = static_cast<unsigned>(units < slots ? units : slots);
   const size_t smem = kSmemHeader + static_cast<size_t>(k.stages) * stage_bytes;

@@ -27,6 +27,7 @@
 #include "pdl.cuh"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"
+#include "trace.cuh"
 
 namespace gi {
 namespace {
@@ -44,6 +45,7 @@ constexpr int kResidentLimit = 144 * 1024;     // weights larger than this strea
 constexpr int kMaxNcta = 192;
 
 __device__ unsigned int g_ts_error = 0;
+GI_TRACE_TABLE(g_ts_trace);
 
 struct TsParams {
   const __half* res;
@@ -128,6 +130,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
   const int m_first = blockIdx.x / p.n_parts, m_step = gridDim.x / p.n_parts;
 
   if (threadIdx.x == 0) {
+    prefetch_tensormap(&tmap_a);
     for (int i = 0; i < p.stages; ++i) {
       mbar_init(smem_u32(&hdr->full[i]), 1);
       mbar_init(smem_u32(&hdr->empty[i]), kTransferWarps + (p.b_resident ? 0 : 1));
@@ -149,6 +152,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
   tc_fence_after();
   const unsigned tmem_base = hdr->tmem_addr;
   const unsigned char* w_part = p.wts + static_cast<size_t>(n_part) * p.n_chunks * b_chunk_bytes;
+  if (threadIdx.x == 0) GI_TRACE_EVENT(g_ts_trace, 0);
   pdl_launch_dependents();
   // the weights never change after binding: their copy starts while the previous kernel still runs
   if (warp == 0 && lane == 0 && p.b_resident) {
@@ -158,6 +162,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
       bulk_load(b_res0 + c * b_chunk_bytes, w_part + static_cast<size_t>(c) * b_chunk_bytes, b_chunk_bytes, bar);
   }
   pdl_wait();  // activations are read and written only below
+  if (threadIdx.x == 0) GI_TRACE_EVENT(g_ts_trace, 1);
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -175,6 +180,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
           mbar_expect_tx(full, stage_bytes);
           const unsigned dst = stage0 + stage * stage_bytes;
           tma_load_2d(dst, &tmap_a, m * kRows, c * p.ks, full);  // pixels / slices outside the tensor arrive as zeros
+          if (it == 0) GI_TRACE_EVENT(g_ts_trace, 2);
           if (!p.b_resident) bulk_load(dst + a_stage_bytes, w_part + static_cast<size_t>(c) * b_chunk_bytes, b_chunk_bytes, full);
         }
       }
@@ -200,6 +206,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
       unsigned it = 0, tile = 0;
       bool ok = true;
       if (p.b_resident) ok = mbar_wait(smem_u32(&hdr->b_ready), 0u, abort_flag, p.timeout_ns, &g_ts_error, kErrMma);
+      GI_TRACE_EVENT(g_ts_trace, 3);
       for (int m = m_first; m < p.m_tiles && ok; m += m_step, ++tile) {
         const unsigned acc = tile & 1u, acc_phase = (tile >> 1) & 1u;
         if (!mbar_wait(smem_u32(&hdr->acc_empty[acc]), acc_phase ^ 1u, abort_flag, p.timeout_ns, &g_ts_error, kErrMma)) break;
@@ -216,6 +223,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
             break;
           }
           tc_fence_after();
+          if (it == 0) GI_TRACE_EVENT(g_ts_trace, 4);
           const unsigned a_tmem = tmem_base + a_col0 + abuf * a_cols;
           const unsigned b_base = p.b_resident ? b_res0 + c * b_chunk_bytes : stage0 + stage * stage_bytes + a_stage_bytes;
           for (int ks = 0; ks < p.ks / 4; ++ks) {  // 16 channels = 4 slices = 8 TMEM columns = 2 K units per MMA
@@ -226,7 +234,9 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
           if (!p.b_resident) umma_commit(smem_u32(&hdr->empty[stage]));
         }
         if (ok) umma_commit(smem_u32(&hdr->acc_full[acc]));
+        if (tile == 0) GI_TRACE_EVENT(g_ts_trace, 5);
       }
+      GI_TRACE_EVENT(g_ts_trace, 9);
     }
   } else if (warp < 2 + kTransferWarps) {
     // ------------------------------------------------------------ transfer: shared memory -> tensor memory
@@ -293,6 +303,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
       if (TAIL) fetch_res(res_cur, part_id);
       if (!mbar_wait(smem_u32(&hdr->acc_full[acc]), acc_phase, abort_flag, p.timeout_ns, &g_ts_error, kErrData)) break;
       tc_fence_after();
+      if (tile == 0 && threadIdx.x == 32 * (2 + kTransferWarps)) GI_TRACE_EVENT(g_ts_trace, 6);
       const unsigned t_addr = tmem_base + lane_bits + acc * acc_cols;
       for (int g = part_id; g < groups; g += kParts) {
         if (TAIL) fetch_res(res_next, g + kParts);
@@ -341,10 +352,12 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&hdr->acc_empty[acc]));
     }
+    if (threadIdx.x == 32 * (2 + kTransferWarps)) GI_TRACE_EVENT(g_ts_trace, 7);
   }
 
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) GI_TRACE_EVENT(g_ts_trace, 8);
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
@@ -504,6 +517,13 @@ int launch_pointwise_ts(const LaunchRec& r, const Ptrs& p, void** state, int lau
 #undef GI_TS_LAUNCH
   return static_cast<int>(cudaGetLastError());
 }
+
+#ifdef GI_TRACE
+int pointwise_ts_trace(unsigned long long* dst, int n) {
+  const size_t bytes = sizeof(unsigned long long) * (n < GI_TRACE_CTAS * GI_TRACE_EVENTS ? n : GI_TRACE_CTAS * GI_TRACE_EVENTS);
+  return static_cast<int>(cudaMemcpyFromSymbol(dst, g_ts_trace, bytes));
+}
+#endif
 
 unsigned int pointwise_ts_error_word(int* cuda_err) {
   unsigned int v = 0;
