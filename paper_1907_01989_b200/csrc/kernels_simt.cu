@@ -86,6 +86,30 @@ __global__ void pack_kernel(const T* __restrict__ nhwc, T* __restrict__ out, int
   Px<T>::store(out + (static_cast<size_t>(plane) * P + pix) * 4, v);
 }
 
+// fp16 images with 3 channels (the usual network input) whose pixel count is a multiple of 4:
+// a thread turns 4 pixels (24 contiguous bytes, three 8-byte loads) into 4 pixel-slices (two
+// 16-byte stores).  grid: x over quads of an image, y over images.
+__global__ void pack3_f16_kernel(const uint2* __restrict__ nhwc, uint4* __restrict__ out, int quads) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int q = blockIdx.x * blockDim.x + threadIdx.x;
+  if (q >= quads) return;
+  const size_t at = static_cast<size_t>(blockIdx.y) * quads + q;
+  const uint2 a = __ldg(nhwc + at * 3), c = __ldg(nhwc + at * 3 + 1), d = __ldg(nhwc + at * 3 + 2);
+  // halves h0..h11 = a.x, a.y, c.x, c.y, d.x, d.y (two per word); pixel i takes h[3i .. 3i+2] and a zero
+  uint4 lo, hi;
+  lo.x = a.x;
+  lo.y = a.y & 0xffffu;
+  lo.z = (a.y >> 16) | (c.x << 16);
+  lo.w = c.x >> 16;
+  hi.x = c.y;
+  hi.y = d.x & 0xffffu;
+  hi.z = (d.x >> 16) | (d.y << 16);
+  hi.w = d.y >> 16;
+  out[at * 2] = lo;
+  out[at * 2 + 1] = hi;
+}
+
 template <typename T>
 __global__ void unpack_kernel(const T* __restrict__ in, T* __restrict__ nhwc, int B, int HW, int C, int P, int S) {
   pdl_launch_dependents();
@@ -320,6 +344,13 @@ int launch_pack(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int S = slices(r.C), P = plane_pixels(r.H, r.W), HW = r.H * r.W;
   if (static_cast<long long>(S) * r.B > 65535) return static_cast<int>(cudaErrorInvalidConfiguration);
+  if (storage == GI_F16 && r.C == 3 && HW % 4 == 0 && r.B <= 65535) {
+    // P == HW here (no padding pixel), one slice: the planes of the images are back to back
+    const int quads = HW / 4;
+    launch_pdl(pack3_f16_kernel, dim3(blocks_for(quads, 256), r.B), 256, 0, st, static_cast<const uint2*>(p.in0),
+               static_cast<uint4*>(p.out), quads);
+    return static_cast<int>(cudaGetLastError());
+  }
   const dim3 grid(blocks_for(P, 256), S * r.B);
   GI_BY_STORAGE((launch_pdl(pack_kernel<__half>, grid, 256, 0, st, static_cast<const __half*>(p.in0), static_cast<__half*>(p.out),
                             r.B, HW, r.C, P, S)),
