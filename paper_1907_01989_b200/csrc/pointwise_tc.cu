@@ -255,13 +255,13 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
             uint4 o;
             __half2* oh = reinterpret_cast<__half2*>(&o);
             if (!TAIL) {
-              // clamping after the rounding equals rounding after the clamp: 0 and 6 are fp16 values
+              // the conversion instruction clamps at 0 itself; clamping at 6 after the rounding
+              // equals rounding after the clamp because 6 is an fp16 value
+              unsigned* ow = reinterpret_cast<unsigned*>(&o);
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
-                __half2 h = __floats2half2_rn(v[i].x, v[i].y);
-                if (ACT != GI_ACT_NONE) h = __hmax2(h, __float2half2_rn(0.f));
-                if (ACT == GI_ACT_RELU6) h = __hmin2(h, __float2half2_rn(6.f));
-                oh[i] = h;
+                ow[i] = pack_f16x2<ACT != GI_ACT_NONE>(v[i].x, v[i].y);
+                if (ACT == GI_ACT_RELU6) ow[i] = __vmins2(ow[i], 0x46004600u);  // non-negative fp16 order like integers
               }
             } else {
               const __half2* rh = reinterpret_cast<const __half2*>(&q[j]);
