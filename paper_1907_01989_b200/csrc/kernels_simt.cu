@@ -271,38 +271,72 @@ __global__ void pool_kernel(const T* __restrict__ in, T* __restrict__ out, int p
 }
 
 // ------------------------------------------------------------------ bilinear resize
-// source coordinate as an exact fraction num/den so that floor() never depends on rounding
-template <typename T>
-__global__ void __launch_bounds__(128) resize_kernel(const T* __restrict__ in, T* __restrict__ out, int B, int H, int W,
+// source coordinate as an exact fraction num/den so that floor() never depends on rounding.
+// grid: x over the columns of a row, y = SOURCE row y0, z = image.  All output rows whose upper
+// source row is y0 share the four source pixels of a column, so a thread interpolates along x once
+// per slice (top, bottom - top) and then emits every such output row with one FMA per channel;
+// the row weights are block-uniform and live in shared memory.  I is the integer type of the
+// coordinate products (32 bits whenever OH*ny and OW*nx fit: 64-bit divisions are emulated).
+constexpr int kResizeRows = 32;
+template <typename T, typename I>
+__global__ void __launch_bounds__(128) resize_kernel(const T* __restrict__ in, T* __restrict__ out, int B, int S, int H, int W,
                                                      int Pin, int OH, int OW, int Pout, int ny, int dy, int nx, int dx) {
+  __shared__ float wy_s[kResizeRows];
   pdl_launch_dependents();
   pdl_wait();
-  const int pix = blockIdx.x * 128 + threadIdx.x;
-  const int s = blockIdx.y, b = blockIdx.z;
-  if (pix >= Pout) return;
-  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (pix < OH * OW) {
-    const int oy = pix / OW, ox = pix - oy * OW;
-    const long long py = static_cast<long long>(oy) * ny, qx = static_cast<long long>(ox) * nx;
-    int y0 = static_cast<int>(py / dy), x0 = static_cast<int>(qx / dx);
-    float wy = static_cast<float>(py - static_cast<long long>(y0) * dy) / static_cast<float>(dy);
-    float wx = static_cast<float>(qx - static_cast<long long>(x0) * dx) / static_cast<float>(dx);
-    if (y0 > H - 1) { y0 = H - 1; wy = 0.f; }
-    if (x0 > W - 1) { x0 = W - 1; wx = 0.f; }
-    const int y1 = min(y0 + 1, H - 1), x1 = min(x0 + 1, W - 1);
-    const T* plane = in + (static_cast<size_t>(s) * B + b) * Pin * 4;
-    const float4 a = Px<T>::load(plane + (static_cast<size_t>(y0) * W + x0) * 4);
-    const float4 c = Px<T>::load(plane + (static_cast<size_t>(y0) * W + x1) * 4);
-    const float4 d = Px<T>::load(plane + (static_cast<size_t>(y1) * W + x0) * 4);
-    const float4 e = Px<T>::load(plane + (static_cast<size_t>(y1) * W + x1) * 4);
-    auto lerp2 = [&](float p00, float p01, float p10, float p11) {
-      const float top = fmaf(p01 - p00, wx, p00), bot = fmaf(p11 - p10, wx, p10);
-      return fmaf(bot - top, wy, top);
-    };
-    v = make_float4(lerp2(a.x, c.x, d.x, e.x), lerp2(a.y, c.y, d.y, e.y), lerp2(a.z, c.z, d.z, e.z),
-                    lerp2(a.w, c.w, d.w, e.w));
+  const int ox = blockIdx.x * 128 + threadIdx.x, y0 = blockIdx.y;
+  const bool active = ox < OW;
+  // output rows oy with floor(oy * ny / dy) == y0
+  int oy_lo, oy_hi;
+  if (ny == 0) {
+    oy_lo = 0;
+    oy_hi = y0 == 0 ? OH : 0;
+  } else {
+    oy_lo = static_cast<int>((static_cast<I>(y0) * static_cast<I>(dy) + static_cast<I>(ny - 1)) / static_cast<I>(ny));
+    const I hi = (static_cast<I>(y0 + 1) * static_cast<I>(dy) + static_cast<I>(ny - 1)) / static_cast<I>(ny);
+    oy_hi = hi > static_cast<I>(OH) ? OH : static_cast<int>(hi);
   }
-  Px<T>::store(out + ((static_cast<size_t>(s) * B + b) * Pout + pix) * 4, v);
+  const int y1 = min(y0 + 1, H - 1);
+  // column: source pixel pair and weight
+  int x0 = 0, x1 = 0;
+  float wx = 0.f;
+  if (active) {
+    const I qx = static_cast<I>(ox) * static_cast<I>(nx);
+    x0 = static_cast<int>(qx / static_cast<I>(dx));
+    wx = static_cast<float>(qx - static_cast<I>(x0) * static_cast<I>(dx)) / static_cast<float>(dx);
+    if (x0 > W - 1) {
+      x0 = W - 1;
+      wx = 0.f;
+    }
+    x1 = min(x0 + 1, W - 1);
+  }
+  const int o00 = (y0 * W + x0) * 4, o01 = (y0 * W + x1) * 4, o10 = (y1 * W + x0) * 4, o11 = (y1 * W + x1) * 4;
+  const size_t in_step = static_cast<size_t>(B) * Pin * 4, out_step = static_cast<size_t>(B) * Pout * 4;
+  const bool pad_col = ox == OW - 1 && Pout > OH * OW;  // an odd plane carries one extra pixel: keep it zero
+  for (int base = oy_lo; base < oy_hi; base += kResizeRows) {
+    const int cnt = min(kResizeRows, oy_hi - base);
+    __syncthreads();  // the previous chunk's weights are no longer needed
+    if (static_cast<int>(threadIdx.x) < cnt) {
+      const I py = static_cast<I>(base + threadIdx.x) * static_cast<I>(ny);
+      wy_s[threadIdx.x] = static_cast<float>(py - static_cast<I>(y0) * static_cast<I>(dy)) / static_cast<float>(dy);
+    }
+    __syncthreads();
+    if (!active) continue;
+    const T* plane = in + static_cast<size_t>(blockIdx.z) * Pin * 4;
+    T* orow = out + static_cast<size_t>(blockIdx.z) * Pout * 4 + (static_cast<size_t>(base) * OW + ox) * 4;
+    for (int s = 0; s < S; ++s, plane += in_step, orow += out_step) {
+      const float4 a = Px<T>::load(plane + o00), c = Px<T>::load(plane + o01), d = Px<T>::load(plane + o10), e = Px<T>::load(plane + o11);
+      const float4 top = make_float4(fmaf(c.x - a.x, wx, a.x), fmaf(c.y - a.y, wx, a.y), fmaf(c.z - a.z, wx, a.z), fmaf(c.w - a.w, wx, a.w));
+      const float4 bot = make_float4(fmaf(e.x - d.x, wx, d.x), fmaf(e.y - d.y, wx, d.y), fmaf(e.z - d.z, wx, d.z), fmaf(e.w - d.w, wx, d.w));
+      const float4 dif = make_float4(bot.x - top.x, bot.y - top.y, bot.z - top.z, bot.w - top.w);
+      T* o = orow;
+      for (int r = 0; r < cnt; ++r, o += static_cast<size_t>(OW) * 4) {
+        const float wy = wy_s[r];
+        Px<T>::store(o, make_float4(fmaf(dif.x, wy, top.x), fmaf(dif.y, wy, top.y), fmaf(dif.z, wy, top.z), fmaf(dif.w, wy, top.w)));
+      }
+      if (pad_col && base + cnt == OH) Px<T>::store(o - static_cast<size_t>(OW) * 4 + 4, make_float4(0.f, 0.f, 0.f, 0.f));
+    }
+  }
 }
 
 ConvGeom geom(const LaunchRec& r) {
@@ -435,7 +469,6 @@ int launch_pool(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
 
 int launch_resize(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (r.B > 65535) return static_cast<int>(cudaErrorInvalidConfiguration);
   int ny, dy, nx, dx;
   if (r.align_corners) {
     ny = r.Ho > 1 ? r.H - 1 : 0;
@@ -449,11 +482,19 @@ int launch_resize(const LaunchRec& r, const Ptrs& p, int storage, void* stream) 
     dx = r.Wo;
   }
   const int Pout = plane_pixels(r.Ho, r.Wo), Pin = plane_pixels(r.H, r.W);
-  const dim3 grid(blocks_for(Pout, 128), slices(r.C), r.B);
-  GI_BY_STORAGE((launch_pdl(resize_kernel<__half>, grid, 128, 0, st, static_cast<const __half*>(p.in0), static_cast<__half*>(p.out), r.B, r.H,
-                                                            r.W, Pin, r.Ho, r.Wo, Pout, ny, dy, nx, dx)),
-                (launch_pdl(resize_kernel<float>, grid, 128, 0, st, static_cast<const float*>(p.in0), static_cast<float*>(p.out), r.B, r.H,
-                                                           r.W, Pin, r.Ho, r.Wo, Pout, ny, dy, nx, dx)));
+  if (r.H > 65535 || r.B > 65535) return static_cast<int>(cudaErrorInvalidConfiguration);
+  const dim3 grid(blocks_for(r.Wo, 128), r.H, r.B);
+  const bool narrow = (static_cast<long long>(r.Ho) + 1) * ny + static_cast<long long>(r.H + 1) * dy < (1LL << 31) &&
+                      static_cast<long long>(r.Wo) * nx < (1LL << 31);
+#define GI_RESIZE(T, I)                                                                                                       \
+  launch_pdl(resize_kernel<T, I>, grid, 128, 0, st, static_cast<const T*>(p.in0), static_cast<T*>(p.out), r.B, slices(r.C), r.H, r.W, \
+             Pin, r.Ho, r.Wo, Pout, ny, dy, nx, dx)
+  if (narrow) {
+    GI_BY_STORAGE(GI_RESIZE(__half, unsigned), GI_RESIZE(float, unsigned));
+  } else {
+    GI_BY_STORAGE(GI_RESIZE(__half, unsigned long long), GI_RESIZE(float, unsigned long long));
+  }
+#undef GI_RESIZE
   return static_cast<int>(cudaGetLastError());
 }
 

@@ -317,3 +317,15 @@ def test_host_pipeline_matches_plain_runs():
     for w, o in zip(want, got):
         assert torch.equal(w, o)
     assert len({float(w.float().abs().sum()) for w in want}) == len(want)  # the batches really differ
+
+
+@pytest.mark.parametrize("storage", STORAGES)
+@pytest.mark.parametrize("case", [(3, 3, 200, 150, True), (3, 3, 200, 150, False), (9, 7, 1, 1, True), (9, 7, 9, 7, True),
+                                  (17, 5, 4, 40, False), (2, 33, 65, 513, True)])
+def test_resize_shapes(storage, case):
+    """Row intervals longer than one chunk of weights, a single output row, identity, mixed up / down scaling."""
+    h, w, oh, ow, align = case
+    b = wl.GraphBuilder(f"resize_{h}x{w}_{oh}x{ow}_{int(align)}", 2, 52)
+    x = b.input(h, w, 6)
+    b.output(b.resize_bilinear(b.conv2d(x, 6, 1), oh, ow, align))
+    check_all_tensors(b.finish(), storage)
