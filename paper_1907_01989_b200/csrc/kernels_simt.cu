@@ -127,6 +127,47 @@ __global__ void unpack_kernel(const T* __restrict__ in, T* __restrict__ nhwc, in
   for (int j = 0; j < n; ++j) Px<T>::put(dst + j, t[j]);
 }
 
+// fp16, any channel count: a block turns 128 consecutive pixels of one image into one contiguous
+// run of 128 * C halves.  The pixel-slices are read coalesced (8 bytes per lane and slice) into
+// shared memory in NHWC order; the run is then written with 4-byte stores (plus a 2-byte store at
+// a misaligned head / tail) instead of one 2-byte store per element.  grid: x over 128-pixel
+// chunks of an image, y over images; dynamic shared memory: 128 * C halves.
+__global__ void __launch_bounds__(128) unpack_f16_kernel(const __half* __restrict__ in, __half* __restrict__ nhwc, int B, int HW, int C,
+                                                         int P, int S) {
+  extern __shared__ __align__(16) unsigned char unpack_smem[];
+  unsigned short* tile = reinterpret_cast<unsigned short*>(unpack_smem);
+  pdl_launch_dependents();
+  pdl_wait();
+  const int pix0 = blockIdx.x * 128, b = blockIdx.y;
+  const int npx = min(128, HW - pix0);
+  const int t = threadIdx.x;
+  if (t < npx) {
+    const uint2* src = reinterpret_cast<const uint2*>(in) + static_cast<size_t>(b) * P + pix0 + t;
+    const size_t step = static_cast<size_t>(B) * P;
+    unsigned short* dst = tile + t * C;
+    for (int s = 0; s < S; ++s, src += step) {
+      const uint2 u = __ldg(src);
+      const unsigned short h[4] = {static_cast<unsigned short>(u.x & 0xffffu), static_cast<unsigned short>(u.x >> 16),
+                                   static_cast<unsigned short>(u.y & 0xffffu), static_cast<unsigned short>(u.y >> 16)};
+      const int n = min(4, C - s * 4);
+      for (int j = 0; j < n; ++j) dst[s * 4 + j] = h[j];
+    }
+  }
+  __syncthreads();
+  const size_t first = (static_cast<size_t>(b) * HW + pix0) * C;  // in halves
+  const int total = npx * C;
+  unsigned short* out = reinterpret_cast<unsigned short*>(nhwc) + first;
+  const int head = static_cast<int>(first & 1);  // halves before the first 4-byte boundary
+  if (t == 0 && head) out[0] = tile[0];
+  const int words = (total - head) / 2;
+  unsigned* out32 = reinterpret_cast<unsigned*>(out + head);
+  for (int w = t; w < words; w += 128) {
+    const int i = head + 2 * w;
+    out32[w] = static_cast<unsigned>(tile[i]) | (static_cast<unsigned>(tile[i + 1]) << 16);
+  }
+  if (t == 0 && ((total - head) & 1)) out[total - 1] = tile[total - 1];
+}
+
 // ------------------------------------------------------------------ direct convolution
 struct ConvGeom {
   int B, H, W, Sin, Pin, Ho, Wo, Sout, Pout;
@@ -397,6 +438,11 @@ int launch_unpack(const LaunchRec& r, const Ptrs& p, int storage, void* stream) 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int S = slices(r.C), P = plane_pixels(r.H, r.W), HW = r.H * r.W;
   const size_t total = static_cast<size_t>(S) * r.B * HW;
+  if (storage == GI_F16 && r.B <= 65535 && static_cast<size_t>(r.C) * 256 <= 48 * 1024) {
+    launch_pdl(unpack_f16_kernel, dim3(blocks_for(HW, 128), r.B), 128, static_cast<size_t>(r.C) * 256, st,
+               static_cast<const __half*>(p.in0), static_cast<__half*>(p.out), r.B, HW, r.C, P, S);
+    return static_cast<int>(cudaGetLastError());
+  }
   GI_BY_STORAGE((launch_pdl(unpack_kernel<__half>, blocks_for(total, 256), 256, 0, st, static_cast<const __half*>(p.in0),
                                                                                static_cast<__half*>(p.out), r.B, HW, r.C, P, S)),
                 (launch_pdl(unpack_kernel<float>, blocks_for(total, 256), 256, 0, st, static_cast<const float*>(p.in0),
