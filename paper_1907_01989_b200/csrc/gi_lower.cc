@@ -179,8 +179,11 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
           // kernel (activations by TMA)
           // (measured on MobileNetV2 at batch 256: the lane kernel wins from ~144 input channels on
           // small planes and from 192 on everywhere, except for very deep, narrow projections)
-          const bool lane_auto = (din->c >= 192 || (din->c >= 144 && din->h * din->w < 2048)) &&
-                                 !(din->c >= 768 && op.d.cout <= 192);
+          // (and whenever all pixels fit one wave of its 128-pixel tiles: latency-bound launches, where its
+          // shorter fill - dense weights, no expansion - wins: MobileNetV2 batch 1 0.296 -> 0.276 ms)
+          const bool one_wave = static_cast<long long>(e->batch) * din->h * din->w <= 148LL * 128;
+          const bool lane_auto = one_wave || ((din->c >= 192 || (din->c >= 144 && din->h * din->w < 2048)) &&
+                                              !(din->c >= 768 && op.d.cout <= 192));
           const bool lane_kernel = e->opt.pointwise == GI_PW_TC_LANE || (e->opt.pointwise == GI_PW_AUTO && lane_auto);
           if (pointwise && tc && lane_kernel && pointwise_ts_supported(din->c, op.d.cout)) {
             r.kernel = GI_KERNEL_POINTWISE_TS;

@@ -288,6 +288,9 @@ def test_kernel_choice_options():
     # fp32 storage never takes a tensor-core kernel
     ops32 = [api.KERNEL_NAMES[o.kernel] for o in api.graph_from_spec(even, api.GI_F32)[0].compile(depthwise=api.GI_DW_TC).ops()]
     assert "depthwise_tc" not in ops32
-    pw = wl.single_pointwise(2, 14, 64, 384)
+    pw = wl.single_pointwise(128, 14, 64, 384)
     assert "pointwise_tc" in kernels(pw) and "pointwise_ts" in kernels(pw, pointwise=api.GI_PW_TC_LANE)
     assert "conv_simt" in kernels(pw, pointwise=api.GI_PW_SIMT)
+    # all pixels in one wave of 128-pixel tiles: the lane-per-pixel kernel whatever the channel counts
+    small = wl.single_pointwise(2, 14, 64, 384)
+    assert "pointwise_ts" in kernels(small) and "pointwise_tc" in kernels(small, pointwise=api.GI_PW_TC_PAIR)
