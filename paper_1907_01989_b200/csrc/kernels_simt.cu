@@ -282,32 +282,46 @@ __global__ void eltwise_kernel(const T* __restrict__ a, const T* __restrict__ b,
 }
 
 // ------------------------------------------------------------------ global average pool
-// one warp per (slice, image): lanes stride over the pixels, shuffle reduction in a fixed order
+// eight lanes per (slice, image), four planes per warp: a lane strides over the pixels with all its
+// loads independent (many small planes are latency-bound otherwise), then a shuffle reduction over
+// the eight lanes in a fixed order
 template <typename T>
 __global__ void pool_kernel(const T* __restrict__ in, T* __restrict__ out, int planes, int HW, int Pin, int Pout) {
   pdl_launch_dependents();
   pdl_wait();
-  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, lane = threadIdx.x & 31;
-  if (warp >= planes) return;
-  const T* plane = in + static_cast<size_t>(warp) * Pin * 4;
+  const int lane = threadIdx.x & 31, sub = lane & 7;
+  const int plane_id = ((blockIdx.x * blockDim.x + threadIdx.x) >> 5) * 4 + (lane >> 3);
+  const bool live = plane_id < planes;
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int p = lane; p < HW; p += 32) {
-    const float4 x = Px<T>::load(plane + static_cast<size_t>(p) * 4);
-    s.x += x.x;
-    s.y += x.y;
-    s.z += x.z;
-    s.w += x.w;
+  if (live) {
+    const T* plane = in + static_cast<size_t>(plane_id) * Pin * 4;
+    int p = sub;
+    for (; p + 24 < HW; p += 32) {  // four loads in flight
+      const float4 x0 = Px<T>::load(plane + static_cast<size_t>(p) * 4), x1 = Px<T>::load(plane + static_cast<size_t>(p + 8) * 4);
+      const float4 x2 = Px<T>::load(plane + static_cast<size_t>(p + 16) * 4), x3 = Px<T>::load(plane + static_cast<size_t>(p + 24) * 4);
+      s.x += (x0.x + x1.x) + (x2.x + x3.x);
+      s.y += (x0.y + x1.y) + (x2.y + x3.y);
+      s.z += (x0.z + x1.z) + (x2.z + x3.z);
+      s.w += (x0.w + x1.w) + (x2.w + x3.w);
+    }
+    for (; p < HW; p += 8) {
+      const float4 x = Px<T>::load(plane + static_cast<size_t>(p) * 4);
+      s.x += x.x;
+      s.y += x.y;
+      s.z += x.z;
+      s.w += x.w;
+    }
   }
-  for (int d = 16; d > 0; d >>= 1) {
-    s.x += __shfl_down_sync(0xffffffffu, s.x, d);
-    s.y += __shfl_down_sync(0xffffffffu, s.y, d);
-    s.z += __shfl_down_sync(0xffffffffu, s.z, d);
-    s.w += __shfl_down_sync(0xffffffffu, s.w, d);
+  for (int d = 4; d > 0; d >>= 1) {
+    s.x += __shfl_down_sync(0xffffffffu, s.x, d, 8);
+    s.y += __shfl_down_sync(0xffffffffu, s.y, d, 8);
+    s.z += __shfl_down_sync(0xffffffffu, s.z, d, 8);
+    s.w += __shfl_down_sync(0xffffffffu, s.w, d, 8);
   }
-  if (lane < Pout) {
+  if (live && sub < Pout) {
     const float inv = 1.0f / static_cast<float>(HW);
-    const float4 v = lane == 0 ? make_float4(s.x * inv, s.y * inv, s.z * inv, s.w * inv) : make_float4(0.f, 0.f, 0.f, 0.f);
-    Px<T>::store(out + (static_cast<size_t>(warp) * Pout + lane) * 4, v);
+    const float4 v = sub == 0 ? make_float4(s.x * inv, s.y * inv, s.z * inv, s.w * inv) : make_float4(0.f, 0.f, 0.f, 0.f);
+    Px<T>::store(out + (static_cast<size_t>(plane_id) * Pout + sub) * 4, v);
   }
 }
 
@@ -505,7 +519,7 @@ int launch_eltwise(const LaunchRec& r, const Ptrs& p, int storage, void* stream)
 int launch_pool(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int planes = slices(r.C) * r.B;
-  const unsigned blocks = blocks_for(static_cast<size_t>(planes) * 32, 256);
+  const unsigned blocks = blocks_for(static_cast<size_t>(planes) * 8, 256);
   GI_BY_STORAGE((launch_pdl(pool_kernel<__half>, blocks, 256, 0, st, static_cast<const __half*>(p.in0), static_cast<__half*>(p.out), planes,
                                                             r.H * r.W, plane_pixels(r.H, r.W), plane_pixels(1, 1))),
                 (launch_pdl(pool_kernel<float>, blocks, 256, 0, st, static_cast<const float*>(p.in0), static_cast<float*>(p.out), planes,
