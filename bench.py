@@ -40,7 +40,6 @@ import numpy as np  # noqa: E402
 NETS = {"v2": ("mobilenet_v2", "MobileNetV2-224"), "v1": ("mobilenet_v1", "MobileNetV1-224"),
         "seg": ("mobilenet_v2_segmentation", "MobileNetV2-513-OS16-seg")}
 PW_MODES = {"auto": 0, "simt": 1, "pair": 2, "lane": 3}
-DW_MODES = {"auto": 0, "stencil": 1, "tc": 2}
 # dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes, from the ncu captures summarised
 # under profiles/ (depthwise: batch 128, 112x112x96, stride 1: 571.3 MB over 616.6 MB; pointwise_tc:
 # batch 64, 112x112, 16->96: 119.6 MB over 179.8 MB, the tail of the output still being in L2)
@@ -213,7 +212,7 @@ def run_sweep(args):
             spec = wl.single_pointwise(b, hw, cin, cout, residual=args.residual)
             name = f"pw1x1 b{b} {hw}x{hw} {cin}->{cout}"
         g, _ = api.graph_from_spec(spec, api.GI_F16, io_layout=api.GI_PHWC4)
-        ex = g.compile(pointwise=PW_MODES[args.pointwise], depthwise=DW_MODES[args.depthwise])
+        ex = g.compile(pointwise=PW_MODES[args.pointwise])
         ex.bind(dev)
         ops = ex.ops()
         assert len(ops) == 1
@@ -258,7 +257,6 @@ def main():
     ap.add_argument("--net", default="v2", choices=sorted(NETS))
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--pointwise", default="auto", choices=["auto", "simt", "pair", "lane"])
-    ap.add_argument("--depthwise", default="auto", choices=["auto", "stencil", "tc"])
     ap.add_argument("--per-op", default=None, help="write the per-op timing table to this file")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-batch1", action="store_true", help="skip the batch-1 latency leg (keeps profiler runs short)")
@@ -305,7 +303,7 @@ def main():
 
     spec = spec_fn(args.batch)
     graph, _ = api.graph_from_spec(spec, api.GI_F16)
-    ex = graph.compile(pointwise=PW_MODES[args.pointwise], depthwise=DW_MODES[args.depthwise])
+    ex = graph.compile(pointwise=PW_MODES[args.pointwise])
     ex.bind(dev)
     ops = ex.ops()
     # every rank draws its own images: rank r holds images [r*B, (r+1)*B) of the global batch
@@ -433,7 +431,7 @@ def main():
         if not args.no_batch1:
             spec1 = spec_fn(1)
             g1, _ = api.graph_from_spec(spec1, api.GI_F16)
-            ex1 = g1.compile(pointwise=PW_MODES[args.pointwise], depthwise=DW_MODES[args.depthwise])
+            ex1 = g1.compile(pointwise=PW_MODES[args.pointwise])
             ex1.bind(dev)
             x1 = torch.from_numpy(wl.make_input(spec1).astype(np.float16)).to(dev)
             o1 = torch.empty((1,) + tuple(spec1.shapes[spec1.outputs[0]]), dtype=torch.float16, device=dev)
@@ -480,7 +478,7 @@ def main():
                            "launches_per_step": len(ops), "arena_mib": round(ex.info.arena_bytes / 2 ** 20, 1),
                            "l2": "flushed between steps by an untimed 256 MiB memset; a step moves ~"
                                  f"{sum(o.bytes for o in ops) / 1e9:.1f} GB", "parallelism": f"replicas x{world}",
-                           "pointwise": args.pointwise, "depthwise": args.depthwise},
+                           "pointwise": args.pointwise},
                 "roofline": roofline, "cpu_baseline": cpu,
                 "e2e": {"value": e2e_value, "unit": "images/s", "h2d_bytes_per_step": int(x_pin.numel() * 2),
                         "d2h_bytes_per_step": int(out_pin.numel() * 2)},

@@ -90,14 +90,6 @@ enum {
   GI_PW_TC_LANE = 3    /* 1x1: always the lane-per-pixel tensor-core kernel (activations through tensor memory) */
 };
 
-/* Kernel choice for 3x3 depthwise convolutions on fp16 storage. */
-enum {
-  GI_DW_AUTO = 0,     /* the faster kernel: today always the CUDA-core stencil */
-  GI_DW_STENCIL = 1,  /* always the CUDA-core stencil kernel */
-  GI_DW_TC = 2        /* tensor-core kernel where the plane is even-sized, stride 1 or 2, dilation 1 (measured
-                         slower than the stencil on B200; kept for comparison); else the stencil */
-};
-
 /*
  * One operator (Section 3.1: the operators of the delegated sub-graph).
  * Convolutions compute, with out-of-range input reading as zero,
@@ -132,7 +124,6 @@ typedef struct gi_compile_options {
   int32_t fuse;      /* 1: fold element-wise ops into convolutions (default), 0: one kernel per op */
   int32_t align;     /* arena offset / tensor size granularity in bytes, power of two >= 256; 0 -> 256 */
   int32_t pointwise; /* GI_PW_* */
-  int32_t depthwise; /* GI_DW_* */
 } gi_compile_options;
 
 typedef struct gi_exec_info {
@@ -171,8 +162,7 @@ typedef struct gi_op_info {
 enum { GI_EXEC_PACK = 100, GI_EXEC_UNPACK = 101 };
 enum {
   GI_KERNEL_PACK = 1, GI_KERNEL_UNPACK = 2, GI_KERNEL_CONV_SIMT = 3, GI_KERNEL_POINTWISE_TC = 4,
-  GI_KERNEL_DEPTHWISE = 5, GI_KERNEL_ELTWISE = 6, GI_KERNEL_POOL = 7, GI_KERNEL_RESIZE = 8, GI_KERNEL_CONV3X3_TC = 9, GI_KERNEL_POINTWISE_TS = 10,
-  GI_KERNEL_DEPTHWISE_TC = 11
+  GI_KERNEL_DEPTHWISE = 5, GI_KERNEL_ELTWISE = 6, GI_KERNEL_POOL = 7, GI_KERNEL_RESIZE = 8, GI_KERNEL_CONV3X3_TC = 9, GI_KERNEL_POINTWISE_TS = 10
 };
 
 /* ---- graph construction (Section 3.1, "Initialization": the sub-graph given to the GPU backend) ---- */
@@ -261,8 +251,7 @@ GI_API gi_status gi_run_timed(gi_exec* e, const void* const* dev_inputs, void* c
  * completion with a limit of about one second per wait; a wait that runs out sets a bit here
  * (1 producer, 2 MMA issuer, 4 epilogue, 8 drain; 0x10000 depthwise staging copy;
  * 0x200000 / 0x400000 MMA issuer / epilogue of the 3x3 tensor-core kernel; 0x1000000..0x8000000
- * producer / MMA issuer / data warps / drain of the lane-per-pixel 1x1 kernel; 0x10000000..0x80000000
- * producer / MMA issuer / epilogue / drain of the tensor-core depthwise kernel), lets the
+ * producer / MMA issuer / data warps / drain of the lane-per-pixel 1x1 kernel), lets the
  * kernel finish without its results
  * and leaves the CUDA context usable.  Sticky until the process exits.  Synchronous: copies
  * the word from the current device. */

@@ -160,15 +160,8 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
         const uint64_t taps = static_cast<uint64_t>(op.d.kh) * op.d.kw;
         info.bytes = (in_px * in_c4 + out_px * out_c4 * (r.ep.has_res ? 2 : 1)) * eb;
         if (f.kind == GI_OP_DEPTHWISE_CONV2D) {
-          if (e->storage == GI_F16 && e->opt.depthwise == GI_DW_TC &&
-              depthwise_tc_supported(din->h, din->w, dout->h, dout->w, op.d.kh, op.d.kw, op.d.stride_h, op.d.stride_w,
-                                     op.d.dilation_h, op.d.dilation_w, op.d.pad_t, op.d.pad_l)) {
-            r.kernel = GI_KERNEL_DEPTHWISE_TC;
-            depthwise_tc_pack(op.weights.data(), op.bias.data(), din->c, op.d.stride_h, op.d.pad_t, op.d.pad_l, &e->weight_blob, &r);
-          } else {
-            r.kernel = GI_KERNEL_DEPTHWISE;
-            pack_depthwise(op, din->c, e->storage, &e->weight_blob, &r);
-          }
+          r.kernel = GI_KERNEL_DEPTHWISE;
+          pack_depthwise(op, din->c, e->storage, &e->weight_blob, &r);
           info.bytes += taps * din->c * eb;
           info.flops = 2 * taps * out_px * din->c;
         } else {

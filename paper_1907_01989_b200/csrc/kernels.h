@@ -44,12 +44,6 @@ void conv3x3_tc_pack(const float* w, const float* bias, int cin, int cout, std::
 int launch_conv3x3_tc(const LaunchRec& r, const Ptrs& p, void* stream);
 unsigned int conv3x3_tc_error_word(int* cuda_err);
 
-// Depthwise 3x3 convolution on the tensor cores (fp16 storage, even planes, stride 1 or 2).
-bool depthwise_tc_supported(int H, int W, int Ho, int Wo, int kh, int kw, int sh, int sw, int dh, int dw, int pt, int pl);
-void depthwise_tc_pack(const float* w, const float* bias, int c, int stride, int pt, int pl, std::vector<uint8_t>* blob, LaunchRec* r);
-int launch_depthwise_tc(const LaunchRec& r, const Ptrs& p, void** state, int launch_index, void* stream);
-unsigned int depthwise_tc_error_word(int* cuda_err);
-
 // Pointwise convolution with the activation operand in tensor memory (fp16 storage).
 bool pointwise_ts_supported(int cin, int cout);
 void pointwise_ts_pack(const float* w, const float* bias, int cin, int cout, std::vector<uint8_t>* blob, LaunchRec* r);

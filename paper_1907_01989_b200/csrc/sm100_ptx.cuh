@@ -30,19 +30,6 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
       : "memory");
   return ok != 0;
 }
-// same test, but the hardware may park the thread for up to `hint_ns` until the phase completes:
-// a parked thread issues nothing, a polling one takes issue slots from the warps that work
-__device__ __forceinline__ bool mbar_try_wait_parked(unsigned bar, unsigned parity, unsigned hint_ns) {
-  unsigned ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(hint_ns)
-      : "memory");
-  return ok != 0;
-}
 __device__ __forceinline__ unsigned long long global_timer_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -55,8 +42,8 @@ static __device__ __noinline__ bool mbar_wait(unsigned bar, unsigned parity, vol
                                        unsigned* error_word, unsigned code) {
   unsigned long long t0 = 0;
   for (unsigned spin = 0;; ++spin) {
-    if (mbar_try_wait_parked(bar, parity, 2000u)) return true;
-    if ((spin & 15u) == 15u) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((spin & 255u) == 255u) {
       if (*abort_flag) return false;
       const unsigned long long now = global_timer_ns();
       if (t0 == 0) {
@@ -131,6 +118,14 @@ __device__ __forceinline__ unsigned pack_f16x2(float x, float y) {
   if (RELU) asm("cvt.rn.relu.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(y), "f"(x));
   else asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(y), "f"(x));
   return d;
+}
+
+// The issuing thread's own instruction stream limits short tiles (measured: ~35 instructions per
+// MMA when both descriptors are built from scratch).  Everything but the start address is constant
+// per operand, and shared-memory addresses are below 2^18, so a descriptor is `fixed | (addr >> 4)`.
+__device__ __forceinline__ unsigned long long smem_desc_fixed(unsigned lbo, unsigned sbo) { return smem_desc(0u, lbo, sbo); }
+__device__ __forceinline__ unsigned long long smem_desc_at(unsigned long long fixed, unsigned addr) {
+  return fixed | static_cast<unsigned long long>(addr >> 4);
 }
 
 // 32 lanes x 16 consecutive 32-bit columns: thread t of the warp receives lane (quarter*32 + t)

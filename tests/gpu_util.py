@@ -19,12 +19,12 @@ def unpack_phwc4(raw: np.ndarray, B: int, H: int, W: int, Cc: int) -> np.ndarray
 
 class GpuRun:
     def __init__(self, spec, storage=api.GI_F16, planner=api.GI_PLAN_GREEDY_BY_SIZE, pointwise=api.GI_PW_AUTO,
-                 fuse=True, guard_bytes=0, depthwise=api.GI_DW_AUTO):
+                 fuse=True, guard_bytes=0):
         import torch
         self.torch = torch
         self.spec, self.storage = spec, storage
         self.graph, _ = api.graph_from_spec(spec, storage)
-        self.ex = self.graph.compile(planner=planner, fuse=fuse, pointwise=pointwise, depthwise=depthwise)
+        self.ex = self.graph.compile(planner=planner, fuse=fuse, pointwise=pointwise)
         dev = "cuda:0"
         nb = int(self.ex.info.arena_bytes)
         self.guard = guard_bytes

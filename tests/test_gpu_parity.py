@@ -17,12 +17,11 @@ STORAGES = [api.GI_F16, api.GI_F32]
 SNAME = {api.GI_F16: "f16", api.GI_F32: "f32"}
 
 
-def check_all_tensors(spec, storage, pointwise=api.GI_PW_AUTO, fuse=True, depthwise=api.GI_DW_AUTO):
+def check_all_tensors(spec, storage, pointwise=api.GI_PW_AUTO, fuse=True):
     """Naive planner keeps every intermediate, so each stored tensor is compared, not only the output."""
     xs = [wl.make_input(spec, index=i) for i in range(len(spec.inputs))]
     ref = og.run(spec, xs, storage=SNAME[storage], fused=fuse, keep_all=True)
-    run = GpuRun(spec, storage, planner=api.GI_PLAN_NAIVE, pointwise=pointwise, fuse=fuse, guard_bytes=4096,
-                 depthwise=depthwise)
+    run = GpuRun(spec, storage, planner=api.GI_PLAN_NAIVE, pointwise=pointwise, fuse=fuse, guard_bytes=4096)
     outs = run.run(xs)
     assert run.guard_intact()
     worst = 0.0
@@ -143,39 +142,33 @@ def depthwise_spec(batch, h, w, c, stride, residual, act=wl.ACT_RELU6):
     return b.finish()
 
 
-DWTC_CASES = [  # batch, H, W, C, stride, residual: even planes, the shapes the tensor-core depthwise kernel takes
+EVEN_DW_CASES = [  # batch, H, W, C, stride, residual: even and non-square planes, many small planes per item
     (1, 14, 14, 32, 1, False), (3, 14, 14, 20, 1, False), (2, 28, 28, 192, 1, True), (1, 56, 56, 24, 1, False),
     (2, 112, 112, 8, 1, False), (5, 14, 14, 8, 1, False), (40, 4, 4, 8, 1, False), (1, 2, 2, 4, 1, False),
     (1, 20, 36, 12, 1, False), (1, 6, 252, 4, 1, True), (2, 14, 14, 96, 2, False), (2, 112, 112, 32, 2, False),
     (1, 56, 56, 144, 2, True), (2, 36, 20, 12, 2, False), (2, 2, 2, 4, 2, False), (37, 8, 8, 4, 2, False),
+    (1, 64, 64, 8, 1, False), (2, 60, 128, 8, 2, False),
 ]
 
 
-@pytest.mark.parametrize("case", DWTC_CASES)
-def test_depthwise_tensor_core(case):
+@pytest.mark.parametrize("case", EVEN_DW_CASES)
+def test_depthwise_even_and_non_square_planes(case):
     batch, h, w, c, stride, residual = case
-    spec = depthwise_spec(batch, h, w, c, stride, residual)
-    forced = api.graph_from_spec(spec, api.GI_F16)[0].compile(depthwise=api.GI_DW_TC)
-    kernels = [api.KERNEL_NAMES[o.kernel] for o in forced.ops()]
-    assert "depthwise_tc" in kernels and "depthwise" not in kernels
-    check_all_tensors(spec, api.GI_F16, depthwise=api.GI_DW_TC)
-    # the same graph through the default (stencil) kernel
-    default = api.graph_from_spec(spec, api.GI_F16)[0].compile()
-    assert "depthwise_tc" not in [api.KERNEL_NAMES[o.kernel] for o in default.ops()]
-    check_all_tensors(spec, api.GI_F16)
+    check_all_tensors(depthwise_spec(batch, h, w, c, stride, residual), api.GI_F16)
     assert api.gi_device_status() == 0
 
 
 @pytest.mark.parametrize("act", [None, wl.ACT_RELU])
-def test_depthwise_tensor_core_other_tails(act):
-    check_all_tensors(depthwise_spec(2, 28, 28, 12, 1, False, act), api.GI_F16, depthwise=api.GI_DW_TC)
-    check_all_tensors(depthwise_spec(2, 28, 28, 12, 2, True, act), api.GI_F16, depthwise=api.GI_DW_TC)
+def test_depthwise_other_tails(act):
+    check_all_tensors(depthwise_spec(2, 28, 28, 12, 1, False, act), api.GI_F16)
+    check_all_tensors(depthwise_spec(2, 28, 28, 12, 2, True, act), api.GI_F16)
     assert api.gi_device_status() == 0
 
 
 @pytest.mark.parametrize("storage", STORAGES)
 @pytest.mark.parametrize("case", [(1, 32, 3, 32, 2), (2, 17, 3, 32, 2), (1, 12, 8, 12, 1), (2, 9, 5, 6, 2), (3, 21, 4, 21, 1),
-                                  (1, 40, 2, 200, 2)])
+                                  (1, 40, 2, 200, 2), (2, 224, 3, 32, 2), (3, 14, 4, 20, 2), (2, 6, 1, 8, 2), (1, 252, 3, 16, 2),
+                                  (5, 2, 3, 128, 2), (2, 64, 3, 32, 2), (1, 128, 3, 32, 2), (2, 60, 3, 32, 2)])
 def test_conv3x3(storage, case):
     spec = wl.single_conv3x3(*case)
     check_all_tensors(spec, storage)

@@ -273,21 +273,11 @@ def test_kernel_choice_options():
     def kernels(spec, **kw):
         return [api.KERNEL_NAMES[o.kernel] for o in api.graph_from_spec(spec, api.GI_F16)[0].compile(**kw).ops()]
 
-    even, odd = wl.single_depthwise(2, 14, 32, 1), wl.single_depthwise(2, 7, 32, 1)
-    assert "depthwise" in kernels(even) and "depthwise_tc" not in kernels(even)
-    assert "depthwise_tc" in kernels(even, depthwise=api.GI_DW_TC)
-    assert "depthwise_tc" in kernels(wl.single_depthwise(2, 14, 32, 2), depthwise=api.GI_DW_TC)
-    # odd planes and dilated windows stay on the stencil kernel even when the tensor-core one is asked for
-    assert "depthwise_tc" not in kernels(odd, depthwise=api.GI_DW_TC)
-    assert "depthwise_tc" not in kernels(wl.single_depthwise(2, 14, 32, 1, 2), depthwise=api.GI_DW_TC)
+    even = wl.single_depthwise(2, 14, 32, 1)
+    assert "depthwise" in kernels(even)
     g = api.graph_from_spec(even, api.GI_F16)[0]
     with pytest.raises(api.GiError):
-        g.compile(depthwise=7)
-    with pytest.raises(api.GiError):
         g.compile(pointwise=9)
-    # fp32 storage never takes a tensor-core kernel
-    ops32 = [api.KERNEL_NAMES[o.kernel] for o in api.graph_from_spec(even, api.GI_F32)[0].compile(depthwise=api.GI_DW_TC).ops()]
-    assert "depthwise_tc" not in ops32
     pw = wl.single_pointwise(128, 14, 64, 384)
     assert "pointwise_tc" in kernels(pw) and "pointwise_ts" in kernels(pw, pointwise=api.GI_PW_TC_LANE)
     assert "conv_simt" in kernels(pw, pointwise=api.GI_PW_SIMT)
