@@ -191,10 +191,16 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
             }
             tc_fence_after();
             const unsigned a_base = data0 + stage * stage_bytes, b_base = a_base + stage_a_bytes;
-            for (int ks = 0; ks < p.kc / 2; ++ks) {
-              const unsigned long long ad = smem_desc(a_base + ks * 2 * kSliceBytes, kSliceBytes, kCoreBytes);
-              const unsigned long long bd = smem_desc(b_base + ks * 2 * b_lbo, b_lbo, kCoreBytes);
-              umma_f16(d_tmem, ad, bd, idesc, (kc_i > 0 || ks > 0) ? 1u : 0u);
+            // descriptors built once per stage and advanced by adds: the issuing thread's own
+            // instruction stream is what bounds short tiles
+            unsigned long long ad = smem_desc(a_base, kSliceBytes, kCoreBytes), bd = smem_desc(b_base, b_lbo, kCoreBytes);
+            const unsigned long long ad_step = static_cast<unsigned long long>((2u * kSliceBytes) >> 4);
+            const unsigned long long bd_step = static_cast<unsigned long long>((2u * b_lbo) >> 4);
+            umma_f16(d_tmem, ad, bd, idesc, kc_i > 0 ? 1u : 0u);
+            for (int ks = 1; ks < p.kc / 2; ++ks) {
+              ad += ad_step;
+              bd += bd_step;
+              umma_f16(d_tmem, ad, bd, idesc, 1u);
             }
             umma_commit(smem_u32(&hdr->empty[stage]));  // the stage is free once these MMAs have read it
           }

@@ -226,9 +226,16 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
           if (it == 0) GI_TRACE_EVENT(g_ts_trace, 4);
           const unsigned a_tmem = tmem_base + a_col0 + abuf * a_cols;
           const unsigned b_base = p.b_resident ? b_res0 + c * b_chunk_bytes : stage0 + stage * stage_bytes + a_stage_bytes;
-          for (int ks = 0; ks < p.ks / 4; ++ks) {  // 16 channels = 4 slices = 8 TMEM columns = 2 K units per MMA
-            const unsigned long long bd = smem_desc(b_base + ks * 2 * b_lbo, b_lbo, 128);
-            umma_f16_ts(d_tmem, a_tmem + ks * 8, bd, idesc, (c > 0 || ks > 0) ? 1u : 0u);
+          // 16 channels = 4 slices = 8 TMEM columns = 2 K units per MMA.  The issuing thread's own
+          // instructions bound the tensor-heavy layers, so the descriptor is built once per chunk and
+          // advanced by an add (the address field counts 16-byte units and cannot carry out of its 14 bits)
+          unsigned long long bd = smem_desc(b_base, b_lbo, 128);
+          const unsigned long long bd_step = static_cast<unsigned long long>((2u * b_lbo) >> 4);
+          const int n_mma = p.ks / 4;
+          umma_f16_ts(d_tmem, a_tmem, bd, idesc, c > 0 ? 1u : 0u);
+          for (int ks = 1; ks < n_mma; ++ks) {
+            bd += bd_step;
+            umma_f16_ts(d_tmem, a_tmem + ks * 8, bd, idesc, 1u);
           }
           umma_commit(smem_u32(&hdr->a_empty[abuf]));
           if (!p.b_resident) umma_commit(smem_u32(&hdr->empty[stage]));
