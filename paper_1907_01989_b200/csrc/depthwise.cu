@@ -4,12 +4,14 @@
 // image; the planes of one slice are adjacent in memory, so they share the slice's 36 weights).
 // The input rows a band needs - its halo included - are one contiguous run per plane and are
 // staged into shared memory by bulk asynchronous copies (16-byte aligned, one mbarrier per
-// buffer).  CTAs are persistent over a contiguous range of items and double-buffer the staging:
-// the copy for the next item is in flight while the current one is computed.  Each thread walks
+// buffer).  CTAs are persistent over a contiguous range of items and stage into a ring of two to
+// four buffers: the copies for the next one to three items are in flight while the current one is
+// computed (bytes in flight are what hides the HBM latency).  Each thread walks
 // down one output column; every input row it reads feeds three running accumulators (packed
 // two-wide fp32 FMAs), so an input pixel-slice is read from HBM once and from shared memory
-// three times; stores are 8 bytes per lane, contiguous across the warp.  Zero padding is applied
-// by predicates while the rows are fetched from shared memory.
+// three times; stores are 8 bytes per lane, contiguous across the warp.  Zero padding: zero rows
+// staged above / below the band and a zero pixel that out-of-image columns point at (no tests in
+// the loop); the packed small-plane mode tests row validity instead.
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 

@@ -17,9 +17,11 @@
 // Two CTAs per SM, persistent over (pixel tile, output-channel tile) units; warp 0 issues TMA,
 // warp 1 issues MMAs and owns tensor memory, warps 2-9 run the epilogue: two warps per TMEM
 // lane quarter, each taking every second 16-column chunk and loading the next chunk from tensor
-// memory while it converts and stores the current one.  Two to eight accumulators live in tensor
-// memory (as many as fit), so the epilogue of a tile overlaps the loads and MMAs of the next ones.  Every wait is bounded: after about a second it raises an error word the
-// host can read, drains the copies in flight and leaves, so the context stays usable.
+// memory while it converts and stores the current one.  Two accumulators per CTA live in tensor
+// memory, so the epilogue of a tile overlaps the loads and MMAs of the next one.  (One layer
+// shape - very few input channels, 17-32 output slices - runs as one wide CTA per SM with four
+// epilogue warps per quarter instead.)  Every wait is bounded: after about a second it raises an
+// error word the host can read, drains the copies in flight and leaves, so the context stays usable.
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -209,7 +211,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..17)
+    // ------------------------------------------------------------ epilogue (warps 2 .. 1 + 4 * epq)
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32) belong to this warp
     const int sub = (warp - 2) >> 2;
     const unsigned rows_total = p.m_total_px >> 1;
