@@ -334,13 +334,9 @@ int launch_conv3x3_tc(const LaunchRec& r, const Ptrs& p, void* stream) {
   while (cols < static_cast<unsigned>(2 * k.n_pad)) cols <<= 1;
   k.tmem_cols = cols;
   k.timeout_ns = 1000000000u;
-  static int sms = 0;
-  static bool attr_set = false;
-  if (sms == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
-  }
+  static bool attr_set_dev[kMaxDevices] = {};
+  bool& attr_set = attr_set_dev[current_device_slot()];
+  const int sms = device_sm_count();
   const size_t smem = 1024 + 2 * kABytes + static_cast<size_t>(kKCores) * k.n_pad * 16;
   if (!attr_set) {
     cudaError_t e = cudaSuccess;

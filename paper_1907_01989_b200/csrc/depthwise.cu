@@ -534,12 +534,7 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
   int threads = (g.nb * g.sub * g.Wo + 31) / 32 * 32;
   if (threads > 256) threads = 256;
   if (threads < 32) threads = 32;
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
-  }
+  const int sms = device_sm_count();
   // persistent CTAs, a few per SM so that one CTA's copies overlap another's arithmetic
   long long ctas_per_sm = static_cast<long long>(kSmemPerSm) / static_cast<long long>(smem + 1024);
   if (ctas_per_sm > 2048 / threads) ctas_per_sm = 2048 / threads;
@@ -556,7 +551,8 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
   const float* b = static_cast<const float*>(p.bias);
   const __half* res = static_cast<const __half*>(p.res);
   __half* out = static_cast<__half*>(p.out);
-  static bool attr_done[3][3][2][2] = {};
+  static bool attr_done_dev[kMaxDevices][3][3][2][2] = {};
+  bool(&attr_done)[3][3][2][2] = attr_done_dev[current_device_slot()];
   const bool tail = r.ep.has_res || r.ep.act_post != GI_ACT_NONE;
 #define GI_DW_LAUNCH(M, A, T, P)                                                                                                 \
   do {                                                                                                                        \

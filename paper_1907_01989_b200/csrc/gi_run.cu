@@ -12,6 +12,24 @@
 
 namespace gi {
 
+int current_device_slot() {
+  int dev = 0;
+  cudaGetDevice(&dev);
+  return dev < 0 ? 0 : dev % kMaxDevices;
+}
+
+int device_sm_count() {
+  static int sms[kMaxDevices] = {};
+  const int slot = current_device_slot();
+  if (sms[slot] == 0) {
+    int dev = 0, n = 0;
+    cudaGetDevice(&dev);
+    sms[slot] = (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) ? n : 148;
+  }
+  return sms[slot];
+}
+
+
 void release_run_state(gi_exec* e) {
   if (e->tc_state) {
     pointwise_tc_release(e->tc_state);

@@ -9,6 +9,12 @@
 
 namespace gi {
 
+// Launch-side facts that belong to a device, not to the process (a process may drive several
+// GPUs): SM count and "shared-memory attribute already raised" flags, indexed by the current device.
+constexpr int kMaxDevices = 64;
+int current_device_slot();  // cudaGetDevice() folded into [0, kMaxDevices)
+int device_sm_count();      // of the current device (cached); 148 if the query fails
+
 struct Ptrs {
   const void* in0 = nullptr;
   const void* in1 = nullptr;

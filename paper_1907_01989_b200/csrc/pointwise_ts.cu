@@ -471,13 +471,9 @@ int launch_pointwise_ts(const LaunchRec& r, const Ptrs& p, void** state, int lau
   k.has_res = r.ep.has_res;
   k.act_post = r.ep.act_post;
   k.timeout_ns = 1000000000u;
-  static int sms = 0;
-  static bool attr_set = false;
-  if (sms == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
-  }
+  static bool attr_set_dev[kMaxDevices] = {};
+  bool& attr_set = attr_set_dev[current_device_slot()];
+  const int sms = device_sm_count();
   const bool tail = k.has_res || k.act_post != GI_ACT_NONE;
   if (!attr_set) {
     cudaError_t e = cudaSuccess;
