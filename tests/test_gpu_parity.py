@@ -322,3 +322,53 @@ def test_resize_shapes(storage, case):
     x = b.input(h, w, 6)
     b.output(b.resize_bilinear(b.conv2d(x, 6, 1), oh, ow, align))
     check_all_tensors(b.finish(), storage)
+
+
+# ---------------------------------------------------------------------- random graphs
+def _random_spec(rnd, n_ops):
+    """Random DAG of all operator kinds on small, ragged shapes (odd planes, C % 4 != 0)."""
+    b = wl.GraphBuilder("random_gpu", rnd.choice([1, 2, 5]), 98)
+    live = [b.input(rnd.choice([5, 8, 9, 16]), rnd.choice([4, 7, 8, 18]), rnd.choice([3, 4, 6, 8, 20]))]
+    for _ in range(n_ops):
+        x = rnd.choice(live[-4:])
+        kind = rnd.choice(["conv1", "conv1", "conv3", "dw", "dw", "act", "add", "pool", "resize"])
+        H, W, Cc = b.g.shapes[x]
+        if kind == "conv1":
+            y = b.conv2d(x, rnd.choice([4, 6, 8, 24, Cc]), 1)
+        elif kind == "conv3":
+            y = b.conv2d(x, rnd.choice([4, 8, Cc]), 3, rnd.choice([1, 2]))
+        elif kind == "dw":
+            y = b.depthwise(x, 3, rnd.choice([1, 2]), rnd.choice([1, 1, 2]))
+        elif kind == "act":
+            y = b.activation(x, rnd.choice([wl.ACT_RELU, wl.ACT_RELU6]))
+        elif kind == "add":
+            same = [t for t in live if b.g.shapes[t] == b.g.shapes[x]]
+            y = b.add(rnd.choice(same), x)
+        elif kind == "pool":
+            if H * W == 1:
+                continue
+            y = b.global_avg_pool(x)
+        else:
+            y = b.resize_bilinear(x, rnd.choice([1, 3, H, 2 * H + 1]), rnd.choice([2, W, 3 * W]), rnd.choice([True, False]))
+        live.append(y)
+    used = {t for op in b.g.ops for t in op.inputs}
+    outs = [t for t in live[1:] if t not in used] or [live[-1]]
+    for t in outs:
+        if t != live[0]:
+            b.output(t)
+    if not b.g.outputs:
+        b.output(b.activation(live[0], wl.ACT_RELU))
+    return b.finish()
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_graphs(seed):
+    """Every stored tensor of a random graph against the oracle, fp16 (tensor-core kernels) and fp32, fused."""
+    import random
+    rnd = random.Random(1000 + seed)
+    spec = _random_spec(rnd, rnd.randint(3, 14))
+    check_all_tensors(spec, api.GI_F16)  # small launches: every 1x1 takes the lane-per-pixel kernel
+    check_all_tensors(spec, api.GI_F16, pointwise=api.GI_PW_TC_PAIR)
+    check_all_tensors(spec, api.GI_F32)
+    check_outputs(spec, api.GI_F16)  # greedy-by-size arena: tensors share memory
+    assert api.gi_device_status() == 0
