@@ -120,14 +120,6 @@ __device__ __forceinline__ unsigned pack_f16x2(float x, float y) {
   return d;
 }
 
-// The issuing thread's own instruction stream limits short tiles (measured: ~35 instructions per
-// MMA when both descriptors are built from scratch).  Everything but the start address is constant
-// per operand, and shared-memory addresses are below 2^18, so a descriptor is `fixed | (addr >> 4)`.
-__device__ __forceinline__ unsigned long long smem_desc_fixed(unsigned lbo, unsigned sbo) { return smem_desc(0u, lbo, sbo); }
-__device__ __forceinline__ unsigned long long smem_desc_at(unsigned long long fixed, unsigned addr) {
-  return fixed | static_cast<unsigned long long>(addr >> 4);
-}
-
 // 32 lanes x 16 consecutive 32-bit columns: thread t of the warp receives lane (quarter*32 + t)
 __device__ __forceinline__ void tmem_ld16(unsigned taddr, unsigned* r) {
   asm volatile(
