@@ -35,6 +35,7 @@ struct DwGeom {
   int plane_stride_px;  // pixels reserved per plane in one staging buffer (even)
   int items;            // S * bchunks * bands
   int packed;           // 1: whole small planes, staged back to back by one copy per item
+  int in_dead;          // 1: the input tensor is not read again after this kernel
   int nbuf;             // staging buffers per CTA (2..4): nbuf - 1 items are in flight ahead of the one computed
   unsigned timeout_ns;
 };
@@ -155,6 +156,10 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
     bool lb;
     item_rows(item, s, b0, nbk, oy0, oy1, start_px, bytes, lb);
     const unsigned bar = smem_u32(&bars[buf]);
+    // an input nobody reads again leaves L2 first, so that the output written here stays for the next kernel
+    unsigned long long pol;
+    if (g.in_dead) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    else asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
     // earlier generic-proxy writes to this buffer (the zeroed bottom row) precede the async writes
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     // the phase cannot complete before this arrival, whatever order the copies land in
@@ -164,8 +169,8 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
       if (threadIdx.x == 0) {
         const __half* src = in + (static_cast<size_t>(s) * g.B + b0) * g.Pin * 4;
         const unsigned dst = smem_u32(smem_raw) + buf * buf_bytes + 16u;  // one zero pixel pair in front
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                     "l"(src), "r"(bytes * nbk), "r"(bar)
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst),
+                     "l"(src), "r"(bytes * nbk), "r"(bar), "l"(pol)
                      : "memory");
       }
       return;
@@ -174,8 +179,8 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
       const __half* src = in + ((static_cast<size_t>(s) * g.B + b0 + pi) * g.Pin + start_px) * 4;
       const unsigned dst =
           smem_u32(smem_raw) + buf * buf_bytes + (static_cast<unsigned>(pi) * g.plane_stride_px + g.head_px) * 8u;
-      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src),
-                   "r"(bytes), "r"(bar)
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst), "l"(src),
+                   "r"(bytes), "r"(bar), "l"(pol)
                    : "memory");
     }
   };
@@ -480,6 +485,7 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
   g.pt = r.pt;
   g.pl = r.pl;
   g.timeout_ns = 1000000000u;
+  g.in_dead = r.in0_dead;
   g.head_px = (g.W + 3) & ~1;
   // thread groups: as many "virtual planes" (plane x sub-band) as fit in ~256 threads
   int vp = 256 / g.Wo;

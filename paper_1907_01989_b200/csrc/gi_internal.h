@@ -65,6 +65,10 @@ struct LaunchRec {
   int tc_kc = 0;       // input slices per pipeline stage
   int tc_stages = 0;
   uint64_t wts_bytes = 0;
+  // no executed op reads the first input after this one (and it is not a graph output): it is read
+  // with the "evict first" L2 policy, which keeps this op's output - the next op's input - resident
+  // instead (MobileNetV2 at batch 256: 1.756 -> 1.728 ms, measured in one run on one GPU)
+  int in0_dead = 0;
 };
 
 struct FusedOp {

@@ -124,6 +124,8 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
       r.Wo = dout->w;
       r.Co = dout->c;
     }
+    if (f.in0 >= 0 && f.in0 != f.in1 && f.in0 != f.residual)
+      r.in0_dead = e->plan[f.in0].last == static_cast<int>(i) && e->tensors[f.in0].output_index < 0;
     r.in0 = loc_of(e, f.in0);
     r.in1 = loc_of(e, f.in1);
     r.res = loc_of(e, f.residual);

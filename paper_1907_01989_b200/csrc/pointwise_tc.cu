@@ -66,6 +66,7 @@ struct TcParams {
   int stages;
   int m_tiles, groups;      // pixel tiles; each pixel tile is split over `groups` CTAs along n_tiles
   int act_pre, has_res, act_post;
+  int in_dead;              // the input is not read again: its TMA loads carry the evict-first L2 hint
   unsigned int tmem_cols;   // power of two >= n_acc * nts * 8
   unsigned int n_acc;       // accumulator buffers in tensor memory (power of two, 2..8): tiles in flight
   int epq;                  // epilogue warps per TMEM lane quarter (1, 2 or 4); blockDim = 64 + 128 * epq
@@ -134,6 +135,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
     if (lane == 0) {
       unsigned it = 0;
       bool ok = true;
+      const unsigned long long evict_first = policy_evict_first();
       for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
         const int m_tile = u / p.groups, grp = u - m_tile * p.groups;
         for (int nt = grp; nt < p.n_tiles && ok; nt += p.groups) {
@@ -147,7 +149,8 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
             mbar_expect_tx(full, stage_bytes);
             const unsigned dst = data0 + stage * stage_bytes;
             // pixels outside the tensor and slices beyond the last one arrive as zeros
-            tma_load_2d(dst, &tmap_a, m_tile * kTilePx, kc_i * p.kc, full);
+            if (p.in_dead) tma_load_2d_hint(dst, &tmap_a, m_tile * kTilePx, kc_i * p.kc, full, evict_first);
+            else tma_load_2d(dst, &tmap_a, m_tile * kTilePx, kc_i * p.kc, full);
             bulk_load(dst + stage_a_bytes, p.wts + (static_cast<size_t>(nt) * p.k_chunks + kc_i) * stage_b_bytes, stage_b_bytes,
                       full);
           }
@@ -461,6 +464,7 @@ int launch_pointwise_tc(const LaunchRec& r, const Ptrs& p, void** state, int lau
   k.act_pre = r.ep.act_pre;
   k.has_res = r.ep.has_res;
   k.act_post = r.ep.act_post;
+  k.in_dead = r.in0_dead;
   // two buffers measured best on MobileNetV2 (four or eight were 4-8 % slower on the narrow layers)
   const unsigned n_acc = 2;
   k.n_acc = n_acc;

@@ -60,6 +60,7 @@ struct TsParams {
   int stages;
   int m_tiles;
   int has_res, act_post;
+  int in_dead;           // the input is not read again: its TMA loads carry the evict-first L2 hint
   unsigned int timeout_ns;
 };
 
@@ -169,6 +170,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
     if (lane == 0) {
       unsigned it = 0;
       bool ok = true;
+      const unsigned long long evict_first = policy_evict_first();
       for (int m = m_first; m < p.m_tiles && ok; m += m_step) {
         for (int c = 0; c < p.n_chunks; ++c, ++it) {
           const unsigned stage = it % p.stages, phase = (it / p.stages) & 1u;
@@ -179,7 +181,9 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
           const unsigned full = smem_u32(&hdr->full[stage]);
           mbar_expect_tx(full, stage_bytes);
           const unsigned dst = stage0 + stage * stage_bytes;
-          tma_load_2d(dst, &tmap_a, m * kRows, c * p.ks, full);  // pixels / slices outside the tensor arrive as zeros
+          // pixels / slices outside the tensor arrive as zeros
+          if (p.in_dead) tma_load_2d_hint(dst, &tmap_a, m * kRows, c * p.ks, full, evict_first);
+          else tma_load_2d(dst, &tmap_a, m * kRows, c * p.ks, full);
           if (it == 0) GI_TRACE_EVENT(g_ts_trace, 2);
           if (!p.b_resident) bulk_load(dst + a_stage_bytes, w_part + static_cast<size_t>(c) * b_chunk_bytes, b_chunk_bytes, full);
         }
@@ -470,6 +474,7 @@ int launch_pointwise_ts(const LaunchRec& r, const Ptrs& p, void** state, int lau
   k.m_tiles = static_cast<int>((k.m_total_px + kRows - 1) / kRows);
   k.has_res = r.ep.has_res;
   k.act_post = r.ep.act_post;
+  k.in_dead = r.in0_dead;
   k.timeout_ns = 1000000000u;
   static bool attr_set_dev[kMaxDevices] = {};
   bool& attr_set = attr_set_dev[current_device_slot()];
