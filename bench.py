@@ -237,7 +237,10 @@ def run_sweep(args):
         row = {"op": name, "kernel": api.KERNEL_NAMES[o.kernel], "ms": round(t, 5), "bytes": int(o.bytes),
                "flops": int(o.flops), "gbs": round(o.bytes / t / 1e6, 1), "tflops": round(o.flops / t / 1e9, 2),
                "bound": "tensor" if t_tc > t_hbm else "hbm", "frac_of_roofline": round(max(t_hbm, t_tc) / t, 4),
-               "peak_source": peak_kind}
+               "peak_source": peak_kind,
+               # the operator's tensors would fit in L2 (126 MB), but the untimed flush before each launch evicts
+               # them: the inputs of every timed launch come from DRAM, only the output may still sit in L2 at the end
+               "smaller_than_l2": bool(o.bytes < 126e6), "inputs_from": "dram (L2 flushed before each timed launch)"}
         rows.append(row)
         print(json.dumps(row), flush=True)
     if args.out:
