@@ -40,6 +40,7 @@ import numpy as np  # noqa: E402
 NETS = {"v2": ("mobilenet_v2", "MobileNetV2-224"), "v1": ("mobilenet_v1", "MobileNetV1-224"),
         "seg": ("mobilenet_v2_segmentation", "MobileNetV2-513-OS16-seg")}
 PW_MODES = {"auto": 0, "simt": 1, "pair": 2, "lane": 3}
+XOP_MODES = {"auto": 0, "off": 1, "on": 2}
 # dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes, from the ncu captures summarised
 # under profiles/ (depthwise: batch 128, 112x112x96, stride 1: 575.0 MB over 616.6 MB; pointwise_tc:
 # batch 64, 112x112, 16->96: 119.6 MB over 179.8 MB, the tail of the output still being in L2)
@@ -189,6 +190,9 @@ def run_sweep(args):
         points = [tuple(int(v) for v in pt.split(",")) for pt in args.points.split(";") if pt]
     elif args.sweep == "conv3":
         points = [(256, 224, 3, 32, 2), (64, 224, 3, 32, 2), (16, 513, 3, 32, 2), (1, 224, 3, 32, 2)]
+    elif args.sweep == "dwpw":  # the depthwise -> projection pairs of MobileNetV2 that have at least one tile per SM
+        points = [(256, 112, 32, 16, 1), (256, 112, 96, 24, 2), (256, 56, 144, 24, 1), (256, 56, 144, 32, 2), (256, 28, 192, 32, 1),
+                  (256, 28, 192, 64, 2), (256, 14, 384, 64, 1), (256, 14, 576, 96, 1)]
     elif args.sweep == "dw":
         points = [(b, hw, c, s) for b in (64, 256) for hw, c in ((112, 32), (112, 96), (56, 144), (28, 192), (14, 384),
                                                                  (14, 576), (7, 960)) for s in (1, 2)]
@@ -203,6 +207,10 @@ def run_sweep(args):
             b, hw, cin, cout, stride = pt
             spec = wl.single_conv3x3(b, hw, cin, cout, stride)
             name = f"conv3x3 b{b} {hw}x{hw} {cin}->{cout} s{stride}"
+        elif args.sweep == "dwpw":
+            b, hw, c, cout, stride = pt
+            spec = wl.depthwise_then_pointwise(b, hw, hw, c, cout, stride, residual=args.residual)
+            name = f"dw3x3+pw1x1 b{b} {hw}x{hw} {c}->{cout} s{stride}"
         elif args.sweep == "dw":
             b, hw, c, stride = pt
             spec = wl.single_depthwise(b, hw, c, stride, 1, residual=args.residual)
@@ -212,10 +220,10 @@ def run_sweep(args):
             spec = wl.single_pointwise(b, hw, cin, cout, residual=args.residual)
             name = f"pw1x1 b{b} {hw}x{hw} {cin}->{cout}"
         g, _ = api.graph_from_spec(spec, api.GI_F16, io_layout=api.GI_PHWC4)
-        ex = g.compile(pointwise=PW_MODES[args.pointwise])
+        ex = g.compile(pointwise=PW_MODES[args.pointwise], cross_op=XOP_MODES[args.cross_op])
         ex.bind(dev)
         ops = ex.ops()
-        assert len(ops) == 1
+        assert len(ops) == (2 if args.sweep == "dwpw" else 1)
         ins = [(torch.rand(api.gi_tensor_bytes(b, *spec.shapes[t]) // 2, device=dev) * 2 - 1).half() for t in spec.inputs]
         outs = [torch.empty(api.gi_tensor_bytes(b, *spec.shapes[t]) // 2, dtype=torch.float16, device=dev)
                 for t in spec.outputs]
@@ -231,10 +239,14 @@ def run_sweep(args):
             z.synchronize()
             ms.append(a.elapsed_time(z))
         t = statistics.median(ms)
-        o = ops[0]
+
+        class o:  # the graph's ops together (one op, or the depthwise + 1x1 pair: two kernels, or one for both)
+            bytes = sum(q.bytes for q in ops)
+            flops = sum(q.flops for q in ops)
+            kernel = "+".join(api.KERNEL_NAMES[q.kernel] for q in ops if api.KERNEL_NAMES[q.kernel] != "none")
         t_hbm = o.bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
         t_tc = o.flops / (peaks["bf16_tflops"] * 1e12) * 1e3
-        row = {"op": name, "kernel": api.KERNEL_NAMES[o.kernel], "ms": round(t, 5), "bytes": int(o.bytes),
+        row = {"op": name, "kernel": o.kernel, "ms": round(t, 5), "bytes": int(o.bytes),
                "flops": int(o.flops), "gbs": round(o.bytes / t / 1e6, 1), "tflops": round(o.flops / t / 1e9, 2),
                "bound": "tensor" if t_tc > t_hbm else "hbm", "frac_of_roofline": round(max(t_hbm, t_tc) / t, 4),
                "peak_source": peak_kind,
@@ -260,12 +272,15 @@ def main():
     ap.add_argument("--net", default="v2", choices=sorted(NETS))
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--pointwise", default="auto", choices=["auto", "simt", "pair", "lane"])
+    ap.add_argument("--cross-op", default="auto", choices=["auto", "off", "on"],
+                    help="depthwise + 1x1 convolution as one kernel: where the library chooses it, never, wherever supported")
     ap.add_argument("--per-op", default=None, help="write the per-op timing table to this file")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-batch1", action="store_true", help="skip the batch-1 latency leg (keeps profiler runs short)")
-    ap.add_argument("--sweep", default=None, choices=["pw", "dw", "conv3"],
+    ap.add_argument("--sweep", default=None, choices=["pw", "dw", "conv3", "dwpw"],
                     help="time single fused operators instead of a network")
-    ap.add_argument("--points", default=None, help="sweep points 'B,HW,Cin,Cout;...' (pw) or 'B,HW,C,stride;...' (dw)")
+    ap.add_argument("--points", default=None, help="sweep points 'B,HW,Cin,Cout;...' (pw), 'B,HW,C,stride;...' (dw), "
+                    "'B,HW,Cin,Cout,stride;...' (conv3), 'B,HW,C,Cout,stride;...' (dwpw: depthwise then 1x1, see --cross-op)")
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--residual", action="store_true")
     ap.add_argument("--out", default=None)
@@ -306,7 +321,7 @@ def main():
 
     spec = spec_fn(args.batch)
     graph, _ = api.graph_from_spec(spec, api.GI_F16)
-    ex = graph.compile(pointwise=PW_MODES[args.pointwise])
+    ex = graph.compile(pointwise=PW_MODES[args.pointwise], cross_op=XOP_MODES[args.cross_op])
     ex.bind(dev)
     ops = ex.ops()
     # every rank draws its own images: rank r holds images [r*B, (r+1)*B) of the global batch
@@ -463,7 +478,7 @@ def main():
         if not args.no_batch1:
             spec1 = spec_fn(1)
             g1, _ = api.graph_from_spec(spec1, api.GI_F16)
-            ex1 = g1.compile(pointwise=PW_MODES[args.pointwise])
+            ex1 = g1.compile(pointwise=PW_MODES[args.pointwise], cross_op=XOP_MODES[args.cross_op])
             ex1.bind(dev)
             x1 = torch.from_numpy(wl.make_input(spec1).astype(np.float16)).to(dev)
             o1 = torch.empty((1,) + tuple(spec1.shapes[spec1.outputs[0]]), dtype=torch.float16, device=dev)

@@ -90,6 +90,18 @@ enum {
   GI_PW_TC_LANE = 3    /* 1x1: always the lane-per-pixel tensor-core kernel (activations through tensor memory) */
 };
 
+/* Cross-operator kernels: a depthwise 3x3 convolution whose only consumer is a 1x1 convolution runs
+ * with it as one kernel, so the tensor between them never reaches memory (fp16 storage; Section 3.3
+ * folds element-wise operators into their producer, this folds a whole operator).  Results are
+ * those of the two operators run one after the other: the tensor between them is still rounded to
+ * fp16.  The memory plan is not affected: the tensor keeps its place in the arena, unused. */
+enum {
+  GI_XOP_AUTO = 0,  /* the library's choice: at present the same as GI_XOP_OFF, the single kernel has not measured
+                       faster than the two kernels on any layer of the benchmark networks (default) */
+  GI_XOP_OFF = 1,   /* one kernel per fused op */
+  GI_XOP_ON = 2     /* wherever the kernel supports the pair */
+};
+
 /*
  * One operator (Section 3.1: the operators of the delegated sub-graph).
  * Convolutions compute, with out-of-range input reading as zero,
@@ -124,6 +136,7 @@ typedef struct gi_compile_options {
   int32_t fuse;      /* 1: fold element-wise ops into convolutions (default), 0: one kernel per op */
   int32_t align;     /* arena offset / tensor size granularity in bytes, power of two >= 256; 0 -> 256 */
   int32_t pointwise; /* GI_PW_* */
+  int32_t cross_op;  /* GI_XOP_* */
 } gi_compile_options;
 
 typedef struct gi_exec_info {
@@ -162,7 +175,9 @@ typedef struct gi_op_info {
 enum { GI_EXEC_PACK = 100, GI_EXEC_UNPACK = 101 };
 enum {
   GI_KERNEL_PACK = 1, GI_KERNEL_UNPACK = 2, GI_KERNEL_CONV_SIMT = 3, GI_KERNEL_POINTWISE_TC = 4,
-  GI_KERNEL_DEPTHWISE = 5, GI_KERNEL_ELTWISE = 6, GI_KERNEL_POOL = 7, GI_KERNEL_RESIZE = 8, GI_KERNEL_CONV3X3_TC = 9, GI_KERNEL_POINTWISE_TS = 10
+  GI_KERNEL_DEPTHWISE = 5, GI_KERNEL_ELTWISE = 6, GI_KERNEL_POOL = 7, GI_KERNEL_RESIZE = 8, GI_KERNEL_CONV3X3_TC = 9, GI_KERNEL_POINTWISE_TS = 10,
+  GI_KERNEL_DEPTHWISE_POINTWISE = 11, /* this op and the next one, as one kernel */
+  GI_KERNEL_NONE = 12                 /* no launch: the op ran inside the previous op's kernel */
 };
 
 /* ---- graph construction (Section 3.1, "Initialization": the sub-graph given to the GPU backend) ---- */
@@ -251,7 +266,8 @@ GI_API gi_status gi_run_timed(gi_exec* e, const void* const* dev_inputs, void* c
  * completion with a limit of about one second per wait; a wait that runs out sets a bit here
  * (1 producer, 2 MMA issuer, 4 epilogue, 8 drain; 0x10000 depthwise staging copy;
  * 0x200000 / 0x400000 MMA issuer / epilogue of the 3x3 tensor-core kernel; 0x1000000..0x8000000
- * producer / MMA issuer / data warps / drain of the lane-per-pixel 1x1 kernel), lets the
+ * producer / MMA issuer / data warps / drain of the lane-per-pixel 1x1 kernel; 0x10000000..
+ * 0x80000000 copy warp / MMA issuer / compute warps / drain of the depthwise + pointwise kernel), lets the
  * kernel finish without its results
  * and leaves the CUDA context usable.  Sticky until the process exits.  Synchronous: copies
  * the word from the current device. */

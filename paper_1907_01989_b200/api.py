@@ -26,9 +26,10 @@ GI_EXEC_PACK, GI_EXEC_UNPACK = 100, 101
 GI_ACT_NONE, GI_ACT_RELU, GI_ACT_RELU6 = 0, 1, 2
 GI_PLAN_GREEDY_BY_SIZE, GI_PLAN_GREEDY_SHARED_OBJECTS, GI_PLAN_NAIVE = 0, 1, 2
 GI_PW_AUTO, GI_PW_SIMT, GI_PW_TC_PAIR, GI_PW_TC_LANE = 0, 1, 2, 3
+GI_XOP_AUTO, GI_XOP_OFF, GI_XOP_ON = 0, 1, 2
 GI_STATIC_ARENA_BYTES = 16 << 20
 KERNEL_NAMES = {1: "pack", 2: "unpack", 3: "conv_simt", 4: "pointwise_tc", 5: "depthwise", 6: "eltwise", 7: "pool",
-                8: "resize", 9: "conv3x3_tc", 10: "pointwise_ts"}
+                8: "resize", 9: "conv3x3_tc", 10: "pointwise_ts", 11: "depthwise_pointwise", 12: "none"}
 
 _KIND = {wl.CONV2D: GI_OP_CONV2D, wl.DEPTHWISE: GI_OP_DEPTHWISE_CONV2D, wl.ADD: GI_OP_ADD,
          wl.ACTIVATION: GI_OP_ACTIVATION, wl.GLOBAL_AVG_POOL: GI_OP_GLOBAL_AVG_POOL,
@@ -46,7 +47,8 @@ class gi_op_desc(C.Structure):
 
 
 class gi_compile_options(C.Structure):
-    _fields_ = [("planner", C.c_int32), ("fuse", C.c_int32), ("align", C.c_int32), ("pointwise", C.c_int32)]
+    _fields_ = [("planner", C.c_int32), ("fuse", C.c_int32), ("align", C.c_int32), ("pointwise", C.c_int32),
+                ("cross_op", C.c_int32)]
 
 
 class gi_exec_info(C.Structure):
@@ -173,8 +175,8 @@ class Graph:
         _check(lib().gi_graph_output(self._h, t, layout), "gi_graph_output")
 
     def compile(self, planner: int = GI_PLAN_GREEDY_BY_SIZE, fuse: bool = True, align: int = 256,
-                pointwise: int = GI_PW_AUTO) -> "Executable":
-        opt = gi_compile_options(planner, 1 if fuse else 0, align, pointwise)
+                pointwise: int = GI_PW_AUTO, cross_op: int = GI_XOP_AUTO) -> "Executable":
+        opt = gi_compile_options(planner, 1 if fuse else 0, align, pointwise, cross_op)
         h = C.c_void_p()
         _check(lib().gi_compile(self._h, C.byref(opt), C.byref(h)), "gi_compile")
         return Executable(h, self)

@@ -91,6 +91,8 @@ static gi_status run_impl(gi_exec* e, const void* const* dev_inputs, void* const
     p.out = resolve(r.out);
     p.wts = resolve(r.wts);
     p.bias = resolve(r.bias);
+    p.wts2 = resolve(r.wts2);
+    p.bias2 = resolve(r.bias2);
     int err = 0;
     switch (r.kernel) {
       case GI_KERNEL_PACK: err = launch_pack(r, p, e->storage, stream); break;
@@ -100,6 +102,8 @@ static gi_status run_impl(gi_exec* e, const void* const* dev_inputs, void* const
       case GI_KERNEL_CONV3X3_TC: err = launch_conv3x3_tc(r, p, stream); break;
       case GI_KERNEL_POINTWISE_TS: err = launch_pointwise_ts(r, p, &e->tc_state, static_cast<int>(i), stream); break;
       case GI_KERNEL_DEPTHWISE: err = launch_depthwise(r, p, e->storage, stream); break;
+      case GI_KERNEL_DEPTHWISE_POINTWISE: err = launch_depthwise_pointwise(r, p, stream); break;
+      case GI_KERNEL_NONE: break;  // computed by the previous launch
       case GI_KERNEL_ELTWISE:
         if (r.ep.has_res && !p.in1) p.in1 = p.res;
         err = launch_eltwise(r, p, e->storage, stream);
@@ -124,6 +128,7 @@ gi_status gi_device_status(uint32_t* flags) {
   if (err == 0) *flags |= depthwise_error_word(&err) << 16;
   if (err == 0) *flags |= conv3x3_tc_error_word(&err) << 20;
   if (err == 0) *flags |= pointwise_ts_error_word(&err) << 24;
+  if (err == 0) *flags |= depthwise_pointwise_error_word(&err) << 28;
   if (err != 0) return fail(GI_E_CUDA, std::string("gi_device_status: ") + cudaGetErrorString(static_cast<cudaError_t>(err)));
   return GI_OK;
 }
@@ -191,10 +196,10 @@ gi_status gi_run_timed(gi_exec* e, const void* const* dev_inputs, void* const* d
 #ifdef GI_TRACE
 namespace gi {
 int pointwise_ts_trace(unsigned long long* dst, int n);
+int depthwise_pointwise_trace(unsigned long long* dst, int n);
 }
 // debug builds only: copy the timeline table of the lane-per-pixel kernel's last launch
 extern "C" GI_API int gi_debug_trace(int which, unsigned long long* dst, int n) {
-  (void)which;
-  return gi::pointwise_ts_trace(dst, n);
+  return which == 1 ? gi::depthwise_pointwise_trace(dst, n) : gi::pointwise_ts_trace(dst, n);
 }
 #endif

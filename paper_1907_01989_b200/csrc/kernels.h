@@ -22,6 +22,8 @@ struct Ptrs {
   void* out = nullptr;
   const void* wts = nullptr;
   const void* bias = nullptr;
+  const void* wts2 = nullptr;   // second operator of a two-operator kernel
+  const void* bias2 = nullptr;
 };
 
 int launch_pack(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
@@ -55,5 +57,14 @@ bool pointwise_ts_supported(int cin, int cout);
 void pointwise_ts_pack(const float* w, const float* bias, int cin, int cout, std::vector<uint8_t>* blob, LaunchRec* r);
 int launch_pointwise_ts(const LaunchRec& r, const Ptrs& p, void** state, int launch_index, void* stream);
 unsigned int pointwise_ts_error_word(int* cuda_err);
+
+// Depthwise 3x3 followed by a pointwise convolution, as one kernel (fp16 storage): the depthwise
+// output stays on chip.  `dw` is the depthwise op's record; `tiles` receives the kernel's parallelism,
+// `lanes` how many of an MMA's 128 rows a pixel tile fills.
+bool depthwise_pointwise_supported(const LaunchRec& dw, int cout, long long* tiles, int* lanes);
+void depthwise_pointwise_pack(const float* w, const float* bias, int cin, int cout, int width, std::vector<uint8_t>* blob,
+                              LaunchRec* r);
+int launch_depthwise_pointwise(const LaunchRec& r, const Ptrs& p, void* stream);
+unsigned int depthwise_pointwise_error_word(int* cuda_err);
 
 }  // namespace gi

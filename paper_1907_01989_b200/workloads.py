@@ -290,6 +290,28 @@ def single_depthwise(batch: int, hw: int, c: int, stride: int = 1, dilation: int
     return b.finish()
 
 
+def depthwise_then_pointwise(batch: int, h: int, w: int, c: int, cout: int, stride: int = 1, residual: bool = False,
+                             dw_act=ACT_RELU6, pw_act=None, post_act=None) -> GraphSpec:
+    """Depthwise 3x3 (+ activation) feeding a 1x1 convolution (+ activation, + residual, + activation): the second
+    half of an inverted-residual block, the pattern one kernel can run without storing the tensor in between."""
+    b = GraphBuilder(f"dwpw_{batch}x{h}x{w}x{c}x{cout}_s{stride}", batch, 9)
+    x = b.input(h, w, c)
+    ho, wo = same_pads(h, 3, stride, 1)[0], same_pads(w, 3, stride, 1)[0]
+    r = b.input(ho, wo, cout) if residual else None
+    y = b.depthwise(x, 3, stride, 1)
+    if dw_act is not None:
+        y = b.activation(y, dw_act)
+    y = b.conv2d(y, cout, 1)
+    if pw_act is not None:
+        y = b.activation(y, pw_act)
+    if residual:
+        y = b.add(r, y)
+    if post_act is not None:
+        y = b.activation(y, post_act)
+    b.output(y)
+    return b.finish()
+
+
 def single_conv3x3(batch: int, hw: int, cin: int, cout: int, stride: int = 1) -> GraphSpec:
     b = GraphBuilder(f"conv3_{batch}x{hw}x{cin}x{cout}_s{stride}", batch, 7)
     x = b.input(hw, hw, cin)

@@ -19,12 +19,14 @@ def unpack_phwc4(raw: np.ndarray, B: int, H: int, W: int, Cc: int) -> np.ndarray
 
 class GpuRun:
     def __init__(self, spec, storage=api.GI_F16, planner=api.GI_PLAN_GREEDY_BY_SIZE, pointwise=api.GI_PW_AUTO,
-                 fuse=True, guard_bytes=0):
+                 fuse=True, guard_bytes=0, cross_op=api.GI_XOP_AUTO):
         import torch
         self.torch = torch
         self.spec, self.storage = spec, storage
         self.graph, _ = api.graph_from_spec(spec, storage)
-        self.ex = self.graph.compile(planner=planner, fuse=fuse, pointwise=pointwise)
+        self.ex = self.graph.compile(planner=planner, fuse=fuse, pointwise=pointwise, cross_op=cross_op)
+        # tensors that stay on chip: the input of an op that runs inside the previous op's kernel
+        self.on_chip = {o.inputs[0] for o in self.ex.ops() if api.KERNEL_NAMES[o.kernel] == "none"}
         dev = "cuda:0"
         nb = int(self.ex.info.arena_bytes)
         self.guard = guard_bytes

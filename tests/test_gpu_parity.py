@@ -17,15 +17,17 @@ STORAGES = [api.GI_F16, api.GI_F32]
 SNAME = {api.GI_F16: "f16", api.GI_F32: "f32"}
 
 
-def check_all_tensors(spec, storage, pointwise=api.GI_PW_AUTO, fuse=True):
+def check_all_tensors(spec, storage, pointwise=api.GI_PW_AUTO, fuse=True, cross_op=api.GI_XOP_AUTO):
     """Naive planner keeps every intermediate, so each stored tensor is compared, not only the output."""
     xs = [wl.make_input(spec, index=i) for i in range(len(spec.inputs))]
     ref = og.run(spec, xs, storage=SNAME[storage], fused=fuse, keep_all=True)
-    run = GpuRun(spec, storage, planner=api.GI_PLAN_NAIVE, pointwise=pointwise, fuse=fuse, guard_bytes=4096)
+    run = GpuRun(spec, storage, planner=api.GI_PLAN_NAIVE, pointwise=pointwise, fuse=fuse, guard_bytes=4096, cross_op=cross_op)
     outs = run.run(xs)
     assert run.guard_intact()
     worst = 0.0
     for t, r in ref.items():
+        if t in run.on_chip:  # never stored: covered through the tensor computed from it
+            continue
         got = outs[t] if t in outs else run.fetch(t)
         worst = max(worst, assert_close(got, r, storage, f"{spec.name} tensor {t}"))
     return worst
@@ -162,6 +164,42 @@ def test_depthwise_even_and_non_square_planes(case):
 def test_depthwise_other_tails(act):
     check_all_tensors(depthwise_spec(2, 28, 28, 12, 1, False, act), api.GI_F16)
     check_all_tensors(depthwise_spec(2, 28, 28, 12, 2, True, act), api.GI_F16)
+    assert api.gi_device_status() == 0
+
+
+def depthwise_pointwise_spec(batch, h, w, c, cout, stride, residual, dw_act=wl.ACT_RELU6, pw_act=None, post_act=None):
+    return wl.depthwise_then_pointwise(batch, h, w, c, cout, stride, residual, dw_act, pw_act, post_act)
+
+
+DWPW_CASES = [  # batch, H, W, C, Cout, stride, residual
+    (1, 32, 32, 32, 64, 1, False), (2, 112, 112, 32, 16, 1, False), (2, 56, 56, 144, 24, 1, True), (3, 28, 28, 192, 32, 1, True),
+    (5, 14, 14, 384, 64, 1, True), (3, 14, 14, 576, 96, 1, False), (2, 112, 112, 96, 24, 2, False), (2, 56, 56, 144, 32, 2, False),
+    (3, 28, 28, 192, 64, 2, False), (7, 7, 7, 64, 40, 1, True), (4, 14, 14, 48, 20, 2, False), (1, 20, 36, 16, 8, 1, False),
+    (2, 60, 128, 16, 3, 2, False), (40, 4, 4, 16, 16, 1, False), (1, 2, 2, 16, 250, 1, False), (2, 9, 5, 32, 17, 2, True),
+    (300, 14, 14, 32, 24, 1, False), (2, 64, 128, 16, 16, 1, False), (1200, 4, 4, 16, 16, 1, False), (1300, 6, 6, 16, 8, 2, True), (40, 56, 56, 16, 8, 1, True), (24, 112, 112, 16, 8, 1, False),
+    (40, 56, 56, 16, 24, 2, False), (150, 28, 28, 32, 40, 1, True),
+]
+
+
+@pytest.mark.parametrize("case", DWPW_CASES)
+def test_depthwise_pointwise_one_kernel(case):
+    """A depthwise op and the 1x1 convolution that consumes it, run by one kernel: same results as the two
+    operators one after the other (the tensor between them is rounded to fp16 on chip)."""
+    batch, h, w, c, cout, stride, residual = case
+    spec = depthwise_pointwise_spec(batch, h, w, c, cout, stride, residual)
+    graph, _ = api.graph_from_spec(spec, api.GI_F16)
+    names = [api.KERNEL_NAMES[o.kernel] for o in graph.compile(cross_op=api.GI_XOP_ON).ops()]
+    assert "depthwise_pointwise" in names and "none" in names, names
+    check_all_tensors(spec, api.GI_F16, cross_op=api.GI_XOP_ON)
+    assert api.gi_device_status() == 0
+
+
+@pytest.mark.parametrize("dw_act,pw_act,post_act", [(None, wl.ACT_RELU, None), (wl.ACT_RELU, wl.ACT_RELU6, wl.ACT_RELU),
+                                                    (wl.ACT_RELU6, None, wl.ACT_RELU6)])
+def test_depthwise_pointwise_epilogues(dw_act, pw_act, post_act):
+    for stride in (1, 2):
+        spec = depthwise_pointwise_spec(3, 28, 28, 32, 24, stride, True, dw_act, pw_act, post_act)
+        check_all_tensors(spec, api.GI_F16, cross_op=api.GI_XOP_ON)
     assert api.gi_device_status() == 0
 
 

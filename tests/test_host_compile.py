@@ -284,3 +284,35 @@ def test_kernel_choice_options():
     # all pixels in one wave of 128-pixel tiles: the lane-per-pixel kernel whatever the channel counts
     small = wl.single_pointwise(2, 14, 64, 384)
     assert "pointwise_ts" in kernels(small) and "pointwise_tc" in kernels(small, pointwise=api.GI_PW_TC_PAIR)
+
+
+def test_cross_op_option():
+    """Depthwise + 1x1 convolution as one kernel: chosen at compile time, only where the pattern and the kernel allow."""
+    def kernels(spec, storage=api.GI_F16, **kw):
+        return [api.KERNEL_NAMES[o.kernel] for o in api.graph_from_spec(spec, storage)[0].compile(**kw).ops()]
+
+    pair = wl.depthwise_then_pointwise(4, 28, 28, 32, 24, 1, residual=True)
+    assert "depthwise_pointwise" not in kernels(pair) and "depthwise_pointwise" not in kernels(pair, cross_op=api.GI_XOP_OFF)
+    on = kernels(pair, cross_op=api.GI_XOP_ON)
+    assert on.count("depthwise_pointwise") == 1 and on.count("none") == 1 and "depthwise" not in on
+    assert on.index("none") == on.index("depthwise_pointwise") + 1
+    # fp32 storage, channels not a multiple of 16, planes wider than 128 columns: two kernels
+    assert "depthwise_pointwise" not in kernels(pair, api.GI_F32, cross_op=api.GI_XOP_ON)
+    assert "depthwise_pointwise" not in kernels(wl.depthwise_then_pointwise(2, 14, 14, 24, 16), cross_op=api.GI_XOP_ON)
+    assert "depthwise_pointwise" not in kernels(wl.depthwise_then_pointwise(1, 8, 200, 16, 16), cross_op=api.GI_XOP_ON)
+    # the tensor between the two ops must have no other reader: a graph output stays a stored tensor
+    b = wl.GraphBuilder("dw_out_and_pw", 2, 11)
+    x = b.input(14, 14, 16)
+    y = b.activation(b.depthwise(x, 3, 1, 1), wl.ACT_RELU6)
+    b.output(y)
+    b.output(b.conv2d(y, 8, 1))
+    assert "depthwise_pointwise" not in kernels(b.finish(), cross_op=api.GI_XOP_ON)
+    # the plan is not affected: the tensor keeps its arena slot, the op count stays
+    g = api.graph_from_spec(pair, api.GI_F16)[0]
+    a, c = g.compile(cross_op=api.GI_XOP_OFF), g.compile(cross_op=api.GI_XOP_ON)
+    assert a.info.arena_bytes == c.info.arena_bytes and a.info.n_ops == c.info.n_ops
+    # whole network at batch 256: the pairs that qualify
+    v2 = kernels(wl.mobilenet_v2(256), cross_op=api.GI_XOP_ON)
+    assert v2.count("depthwise_pointwise") == v2.count("none") == 13
+    with pytest.raises(api.GiError):
+        g.compile(cross_op=7)
