@@ -150,6 +150,9 @@ EVEN_DW_CASES = [  # batch, H, W, C, stride, residual: even and non-square plane
     (1, 20, 36, 12, 1, False), (1, 6, 252, 4, 1, True), (2, 14, 14, 96, 2, False), (2, 112, 112, 32, 2, False),
     (1, 56, 56, 144, 2, True), (2, 36, 20, 12, 2, False), (2, 2, 2, 4, 2, False), (37, 8, 8, 4, 2, False),
     (1, 64, 64, 8, 1, False), (2, 60, 128, 8, 2, False),
+    # wide planes, stride 1: two output columns per thread
+    (3, 40, 96, 8, 1, True), (1, 33, 130, 12, 1, False), (2, 100, 200, 4, 1, False), (5, 7, 128, 8, 1, True),
+    (1, 1, 96, 4, 1, False), (2, 3, 254, 4, 1, True),
 ]
 
 
@@ -164,6 +167,8 @@ def test_depthwise_even_and_non_square_planes(case):
 def test_depthwise_other_tails(act):
     check_all_tensors(depthwise_spec(2, 28, 28, 12, 1, False, act), api.GI_F16)
     check_all_tensors(depthwise_spec(2, 28, 28, 12, 2, True, act), api.GI_F16)
+    check_all_tensors(depthwise_spec(2, 20, 112, 8, 1, False, act), api.GI_F16)
+    check_all_tensors(depthwise_spec(1, 20, 112, 8, 1, True, act), api.GI_F16)
     assert api.gi_device_status() == 0
 
 
