@@ -1,4 +1,5 @@
-"""Oracle for the compile step: operator fusion, tensor lifetimes, sizes, memory planners.
+"""Oracle for the compile step: operator fusion, tensor lifetimes, sizes, memory planners
+(naive, Algorithm 1, minimum-cost flow, greedy by size).
 
 TEST INFRASTRUCTURE ONLY (see oracle/__init__.py).  Every function follows its defining
 text step by step with plain Python containers; nothing here is tuned.
@@ -260,6 +261,110 @@ def plan_greedy_by_size(p: PlanProblem) -> Tuple[Dict[int, int], int]:
         offsets[t] = best_off if best_off is not None else cursor
     total = max((offsets[t] + p.size[t] for t in offsets), default=0)
     return offsets, total
+
+
+def plan_min_cost_flow(p: PlanProblem):
+    """The Minimum-Cost Flow Algorithm of Section 5, in the paper's steps and notation.
+
+    Tensors x = 1..N are the intermediate tensors in execution order (first use, then id).
+    Vertices: source s, sink t and two per tensor, l_x and r_x.  Edges, all of capacity 1:
+      1. s -> r_x, cost size_x: tensor x gets a new shared object;
+      2. l_x -> r_y, cost max(0, size_y - size_x), for every pair where the object of x can be
+         re-used for y - x is dead before y is born (last use of x < first use of y; an op's output
+         never shares with its input, as in Algorithm 1);
+      3. s -> l_x, cost 0;   4. r_x -> t, cost 0.
+    The minimum-cost flow (of value N) is found by successive shortest augmenting paths, each
+    found with the Shortest Path Faster Algorithm (queue-based Bellman-Ford), as the paper
+    names.  A saturated edge of type 1 creates a shared object for x; a saturated edge of type 2
+    gives y the object of x.  The size of an object is the largest tensor assigned to it.
+
+    Readings where the paper is silent: edges are inserted in the order 1, 2 (x ascending, then
+    y ascending), 3, 4; the queue is first-in first-out and a distance is replaced only by a
+    strictly smaller one; one arena, objects laid out in creation order (the order of the
+    tensors that open them), as for Algorithm 1.
+
+    Returns (offsets, total, object_of_tensor, object_sizes, flow_cost).
+    """
+    life = lifetimes(p)
+    ts = sorted(p.intermediate, key=lambda t: (life[t][0], t))
+    n = len(ts)
+    s_v, t_v = 0, 2 * n + 1
+
+    def l_v(i: int) -> int:
+        return 1 + i
+
+    def r_v(i: int) -> int:
+        return 1 + n + i
+
+    head: List[List[int]] = [[] for _ in range(2 * n + 2)]   # edge ids leaving each vertex
+    to: List[int] = []
+    cap: List[int] = []
+    cost: List[int] = []
+
+    def add_edge(u: int, v: int, c: int) -> None:  # edge 2k and its residual twin 2k+1
+        head[u].append(len(to)); to.append(v); cap.append(1); cost.append(c)
+        head[v].append(len(to)); to.append(u); cap.append(0); cost.append(-c)
+
+    for i, x in enumerate(ts):                       # type 1
+        add_edge(s_v, r_v(i), p.size[x])
+    for i, x in enumerate(ts):                       # type 2
+        for j, y in enumerate(ts):
+            if life[x][1] < life[y][0]:
+                add_edge(l_v(i), r_v(j), max(0, p.size[y] - p.size[x]))
+    for i in range(n):                               # type 3
+        add_edge(s_v, l_v(i), 0)
+    for i in range(n):                               # type 4
+        add_edge(r_v(i), t_v, 0)
+
+    flow, flow_cost = 0, 0
+    while True:
+        dist: List[Optional[int]] = [None] * (2 * n + 2)
+        via = [-1] * (2 * n + 2)
+        queued = [False] * (2 * n + 2)
+        dist[s_v] = 0
+        queue = [s_v]
+        while queue:
+            u = queue.pop(0)
+            queued[u] = False
+            for e in head[u]:
+                v = to[e]
+                if cap[e] > 0 and (dist[v] is None or dist[u] + cost[e] < dist[v]):
+                    dist[v] = dist[u] + cost[e]
+                    via[v] = e
+                    if not queued[v]:
+                        queued[v] = True
+                        queue.append(v)
+        if dist[t_v] is None:
+            break
+        v = t_v
+        while v != s_v:                              # push one unit along the shortest path
+            e = via[v]
+            cap[e] -= 1
+            cap[e ^ 1] += 1
+            v = to[e ^ 1]
+        flow += 1
+        flow_cost += dist[t_v]
+    assert flow == n
+    donor: Dict[int, int] = {}                       # y -> x for saturated edges of type 2
+    for i in range(n):
+        for e in head[l_v(i)]:
+            if e % 2 == 0 and cap[e] == 0:
+                donor[to[e] - 1 - n] = i
+    obj: Dict[int, int] = {}
+    sizes: List[int] = []
+    for j, y in enumerate(ts):                       # a donor is dead before y is born: it comes earlier
+        if j in donor:
+            obj[y] = obj[ts[donor[j]]]
+            sizes[obj[y]] = max(sizes[obj[y]], p.size[y])
+        else:
+            obj[y] = len(sizes)
+            sizes.append(p.size[y])
+    starts, total = [], 0
+    for sz in sizes:
+        starts.append(total)
+        total += sz
+    offsets = {t: starts[k] for t, k in obj.items()}
+    return offsets, total, obj, sizes, flow_cost
 
 
 def check_no_overlap(p: PlanProblem, offsets: Dict[int, int]) -> None:

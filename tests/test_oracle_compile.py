@@ -1,4 +1,4 @@
-"""Pins for the oracle's compile step: fusion, lifetimes and the three memory planners."""
+"""Pins for the oracle's compile step: fusion, lifetimes and the memory planners."""
 import itertools
 import os
 import random
@@ -50,6 +50,9 @@ def test_table4_memory_totals():
         greedy = oc.plan_greedy_shared_objects(p)[1] / MIB
         assert round(naive, 1) == t4["naive"][col]
         assert round(greedy, 1) == t4["greedy"][col]
+        # the minimum-cost flow strategy: larger than Algorithm 1 on MobileNet, smaller on MobileNetV2, as printed
+        mcfp = oc.plan_min_cost_flow(p)[1] / MIB
+        assert round(mcfp, 1) == t4["mcfp"][col]
 
 
 def test_release_before_allocate_would_not_match_table4():
@@ -116,6 +119,72 @@ def test_shared_object_size_is_max_of_its_tensors():
         _, _, obj, sizes = oc.plan_greedy_shared_objects(p)
         for k, s in enumerate(sizes):
             assert s == max(p.size[t] for t, o in obj.items() if o == k)
+
+
+# ---------------------------------------------------------------------- minimum-cost flow
+def cheapest_assignment(p):
+    """Brute force over the problem the flow network encodes: every tensor either opens an object (cost: its
+    size) or takes over the object of a tensor that is dead before it is born, each donor used once
+    (cost: the growth max(0, size_y - size_x))."""
+    life = oc.lifetimes(p)
+    ts = sorted(p.intermediate)
+    best = [None]
+
+    def rec(k, used, cost):
+        if best[0] is not None and cost >= best[0]:
+            return
+        if k == len(ts):
+            best[0] = cost
+            return
+        y = ts[k]
+        rec(k + 1, used, cost + p.size[y])
+        for x in ts:
+            if x not in used and life[x][1] < life[y][0]:
+                rec(k + 1, used | {x}, cost + max(0, p.size[y] - p.size[x]))
+
+    rec(0, frozenset(), 0)
+    return best[0]
+
+
+def test_mcfp_hand_example():
+    # t3 (20) may take over t0 (10, growth 10) or t1 (40, growth 0); t2 overlaps both: 10 + 40 + 3 + 0
+    p = hand_example()
+    off, total, obj, sizes, cost = oc.plan_min_cost_flow(p)
+    assert cost == 53 and total == 53 and sizes == [10, 40, 3]
+    assert obj[3] == obj[1] and off == {0: 0, 1: 10, 2: 50, 3: 10}
+    oc.check_no_overlap(p, off)
+
+
+def test_mcfp_chain_of_equal_tensors_uses_two_objects():
+    n = 9
+    p = problem([([X], [0])] + [([i - 1], [i]) for i in range(1, n)] + [([n - 1], [OUT])], {i: 7 for i in range(n)})
+    off, total, obj, sizes, cost = oc.plan_min_cost_flow(p)
+    assert cost == 14 and sizes == [7, 7]
+    assert all(obj[i] == i % 2 for i in range(n))
+
+
+def test_mcfp_flow_cost_is_the_minimum_and_bounds_the_total():
+    rnd = random.Random(5)
+    for trial in range(150):
+        p = random_problem(rnd, rnd.randint(2, 8))
+        off, total, obj, sizes, cost = oc.plan_min_cost_flow(p)
+        assert cost == cheapest_assignment(p)
+        # the growth charged per re-use is what the object grows by at most (the paper: "a good approximation")
+        assert oc.lower_bound(p) <= total <= cost <= oc.plan_naive(p)[1]
+        oc.check_no_overlap(p, off)
+        assert set(off) == p.intermediate
+        for t, k in obj.items():
+            assert p.size[t] <= sizes[k]
+
+
+def test_mcfp_invariants_larger_random_dags():
+    rnd = random.Random(6)
+    for trial in range(40):
+        p = random_problem(rnd, rnd.randint(10, 40))
+        off, total, obj, sizes, cost = oc.plan_min_cost_flow(p)
+        oc.check_no_overlap(p, off)
+        assert oc.lower_bound(p) <= total <= cost <= oc.plan_naive(p)[1]
+        assert total == sum(sizes)
 
 
 # ---------------------------------------------------------------------- greedy by size
