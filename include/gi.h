@@ -79,7 +79,9 @@ enum { GI_ACT_NONE = 0, GI_ACT_RELU = 1, GI_ACT_RELU6 = 2 };
 enum {
   GI_PLAN_GREEDY_BY_SIZE = 0,        /* offsets into one buffer, largest tensor first, best-fit gap (default) */
   GI_PLAN_GREEDY_SHARED_OBJECTS = 1, /* Algorithm 1 of the paper, objects laid out in creation order */
-  GI_PLAN_NAIVE = 2                  /* every tensor its own memory (the paper's baseline) */
+  GI_PLAN_NAIVE = 2,                 /* every tensor its own memory (the paper's baseline) */
+  GI_PLAN_MIN_COST_FLOW = 3          /* the paper's minimum-cost flow strategy (successive shortest paths, SPFA); shared
+                                        objects laid out in creation order; O(N^4) in the number of tensors */
 };
 
 /* Kernel choice for full convolutions (1x1, and 3x3 with at most 4 input channels). */

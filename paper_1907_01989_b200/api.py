@@ -24,7 +24,7 @@ GI_NHWC, GI_PHWC4 = 0, 1
 GI_OP_CONV2D, GI_OP_DEPTHWISE_CONV2D, GI_OP_ADD, GI_OP_ACTIVATION, GI_OP_GLOBAL_AVG_POOL, GI_OP_RESIZE_BILINEAR = 1, 2, 3, 4, 5, 6
 GI_EXEC_PACK, GI_EXEC_UNPACK = 100, 101
 GI_ACT_NONE, GI_ACT_RELU, GI_ACT_RELU6 = 0, 1, 2
-GI_PLAN_GREEDY_BY_SIZE, GI_PLAN_GREEDY_SHARED_OBJECTS, GI_PLAN_NAIVE = 0, 1, 2
+GI_PLAN_GREEDY_BY_SIZE, GI_PLAN_GREEDY_SHARED_OBJECTS, GI_PLAN_NAIVE, GI_PLAN_MIN_COST_FLOW = 0, 1, 2, 3
 GI_PW_AUTO, GI_PW_SIMT, GI_PW_TC_PAIR, GI_PW_TC_LANE = 0, 1, 2, 3
 GI_XOP_AUTO, GI_XOP_OFF, GI_XOP_ON = 0, 1, 2
 GI_STATIC_ARENA_BYTES = 16 << 20

@@ -2,6 +2,8 @@
 // for intermediate tensors (Section 5), plus the query half of the C ABI.
 #include <algorithm>
 #include <cstring>
+#include <deque>
+#include <limits>
 #include <map>
 #include <new>
 #include <set>
@@ -194,6 +196,105 @@ static uint64_t plan_shared_objects(gi_exec* e) {
   return total;
 }
 
+// The Minimum-Cost Flow Algorithm (Section 5).  Intermediate tensors in execution order (first use, then
+// id) are x = 1..N; the network has a source, a sink and vertices l_x, r_x; unit-capacity edges
+//   1. s -> r_x, cost size_x (x opens a shared object),
+//   2. l_x -> r_y, cost max(0, size_y - size_x), where x is dead before y is born (y takes over x's object),
+//   3. s -> l_x and 4. r_x -> t, cost 0.
+// The flow of value N and minimum cost is built one augmenting path at a time, each a shortest path found
+// by the queue-based Bellman-Ford the paper names (SPFA): first-in first-out queue, edges in the order they
+// were added (1, 2 by x then y, 3, 4), a distance replaced only by a strictly smaller one.  A saturated edge
+// of type 2 hands x's object to y; an object is as large as its largest tensor; objects are laid out in the
+// order their first tensors appear.
+static uint64_t plan_min_cost_flow(gi_exec* e) {
+  std::vector<int> ts;
+  for (size_t t = 0; t < e->plan.size(); ++t)
+    if (e->plan[t].intermediate) ts.push_back(static_cast<int>(t));
+  std::stable_sort(ts.begin(), ts.end(), [&](int a, int b) { return e->plan[a].first < e->plan[b].first; });
+  const int n = static_cast<int>(ts.size());
+  const int src = 0, sink = 2 * n + 1, nv = 2 * n + 2;
+  struct Edge {
+    int to, cap;
+    long long cost;
+  };
+  std::vector<Edge> edges;                  // edge 2k and its reverse 2k + 1
+  std::vector<std::vector<int>> out(static_cast<size_t>(nv));
+  auto add_edge = [&](int u, int v, long long c) {
+    out[static_cast<size_t>(u)].push_back(static_cast<int>(edges.size()));
+    edges.push_back({v, 1, c});
+    out[static_cast<size_t>(v)].push_back(static_cast<int>(edges.size()));
+    edges.push_back({u, 0, -c});
+  };
+  auto size_of = [&](int i) { return static_cast<long long>(e->plan[ts[static_cast<size_t>(i)]].bytes); };
+  for (int i = 0; i < n; ++i) add_edge(src, 1 + n + i, size_of(i));
+  for (int i = 0; i < n; ++i)
+    for (int j = 0; j < n; ++j)
+      if (e->plan[ts[static_cast<size_t>(i)]].last < e->plan[ts[static_cast<size_t>(j)]].first)
+        add_edge(1 + i, 1 + n + j, std::max<long long>(0, size_of(j) - size_of(i)));
+  for (int i = 0; i < n; ++i) add_edge(src, 1 + i, 0);
+  for (int i = 0; i < n; ++i) add_edge(1 + n + i, sink, 0);
+  const long long kInf = std::numeric_limits<long long>::max();
+  std::vector<long long> dist(static_cast<size_t>(nv));
+  std::vector<int> via(static_cast<size_t>(nv));
+  std::vector<char> queued(static_cast<size_t>(nv));
+  for (;;) {
+    std::fill(dist.begin(), dist.end(), kInf);
+    std::fill(via.begin(), via.end(), -1);
+    std::fill(queued.begin(), queued.end(), 0);
+    std::deque<int> queue;
+    dist[src] = 0;
+    queue.push_back(src);
+    while (!queue.empty()) {
+      const int u = queue.front();
+      queue.pop_front();
+      queued[static_cast<size_t>(u)] = 0;
+      for (int id : out[static_cast<size_t>(u)]) {
+        const Edge& ed = edges[static_cast<size_t>(id)];
+        if (ed.cap > 0 && dist[static_cast<size_t>(u)] + ed.cost < dist[static_cast<size_t>(ed.to)]) {
+          dist[static_cast<size_t>(ed.to)] = dist[static_cast<size_t>(u)] + ed.cost;
+          via[static_cast<size_t>(ed.to)] = id;
+          if (!queued[static_cast<size_t>(ed.to)]) {
+            queued[static_cast<size_t>(ed.to)] = 1;
+            queue.push_back(ed.to);
+          }
+        }
+      }
+    }
+    if (dist[static_cast<size_t>(sink)] == kInf) break;
+    for (int v = sink; v != src;) {
+      const int id = via[static_cast<size_t>(v)];
+      edges[static_cast<size_t>(id)].cap -= 1;
+      edges[static_cast<size_t>(id ^ 1)].cap += 1;
+      v = edges[static_cast<size_t>(id ^ 1)].to;
+    }
+  }
+  std::vector<int> donor(static_cast<size_t>(n), -1);
+  for (int i = 0; i < n; ++i)
+    for (int id : out[static_cast<size_t>(1 + i)])
+      if (id % 2 == 0 && edges[static_cast<size_t>(id)].cap == 0) donor[static_cast<size_t>(edges[static_cast<size_t>(id)].to - 1 - n)] = i;
+  std::vector<int> obj(static_cast<size_t>(n), -1);
+  std::vector<uint64_t> sizes;
+  for (int j = 0; j < n; ++j) {  // a donor is dead before its heir is born: it comes earlier in the order
+    const uint64_t need = e->plan[ts[static_cast<size_t>(j)]].bytes;
+    if (donor[static_cast<size_t>(j)] >= 0) {
+      obj[static_cast<size_t>(j)] = obj[static_cast<size_t>(donor[static_cast<size_t>(j)])];
+      uint64_t& sz = sizes[static_cast<size_t>(obj[static_cast<size_t>(j)])];
+      if (need > sz) sz = need;
+    } else {
+      obj[static_cast<size_t>(j)] = static_cast<int>(sizes.size());
+      sizes.push_back(need);
+    }
+  }
+  std::vector<uint64_t> start(sizes.size(), 0);
+  uint64_t total = 0;
+  for (size_t k = 0; k < sizes.size(); ++k) {
+    start[k] = total;
+    total += sizes[k];
+  }
+  for (int j = 0; j < n; ++j) e->plan[ts[static_cast<size_t>(j)]].offset = start[static_cast<size_t>(obj[static_cast<size_t>(j)])];
+  return total;
+}
+
 // Greedy by size: largest tensor first (ties: earlier first use, smaller id).  Among the
 // tensors already placed whose lifetime intersects, scan the free gaps from offset 0 upward
 // and take the smallest that fits (ties: lowest offset); otherwise append after them.
@@ -267,6 +368,7 @@ gi_status plan_memory(gi_exec* e) {
     case GI_PLAN_NAIVE: e->arena_bytes = plan_naive(e); break;
     case GI_PLAN_GREEDY_SHARED_OBJECTS: e->arena_bytes = plan_shared_objects(e); break;
     case GI_PLAN_GREEDY_BY_SIZE: e->arena_bytes = plan_by_size(e); break;
+    case GI_PLAN_MIN_COST_FLOW: e->arena_bytes = plan_min_cost_flow(e); break;
     default: return fail(GI_E_INVALID, "gi_compile: unknown planner");
   }
   return GI_OK;

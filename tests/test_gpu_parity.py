@@ -53,7 +53,8 @@ def test_separable_block(storage, pointwise):
     check_all_tensors(wl.separable_block(3, 9, 7, 10, 22), storage, pointwise)  # ragged: odd plane, C % 4 != 0
 
 
-@pytest.mark.parametrize("planner", [api.GI_PLAN_GREEDY_BY_SIZE, api.GI_PLAN_GREEDY_SHARED_OBJECTS, api.GI_PLAN_NAIVE])
+@pytest.mark.parametrize("planner", [api.GI_PLAN_GREEDY_BY_SIZE, api.GI_PLAN_GREEDY_SHARED_OBJECTS, api.GI_PLAN_NAIVE,
+                                     api.GI_PLAN_MIN_COST_FLOW])
 def test_planners_give_same_result(planner):
     spec = wl.mobilenet_v2(2, size=64)
     run, xs, outs = check_outputs(spec, api.GI_F16, planner=planner)

@@ -103,6 +103,8 @@ def compare_with_oracle(spec, planner, fuse=True, storage=api.GI_F16, align=256)
         off, total = oc.plan_naive(p)
     elif planner == api.GI_PLAN_GREEDY_SHARED_OBJECTS:
         off, total = oc.plan_greedy_shared_objects(p)[:2]
+    elif planner == api.GI_PLAN_MIN_COST_FLOW:
+        off, total = oc.plan_min_cost_flow(p)[:2]
     else:
         off, total = oc.plan_greedy_by_size(p)
     assert ex.info.arena_bytes == total
@@ -115,7 +117,7 @@ def compare_with_oracle(spec, planner, fuse=True, storage=api.GI_F16, align=256)
     return ex
 
 
-PLANNERS = [api.GI_PLAN_GREEDY_BY_SIZE, api.GI_PLAN_GREEDY_SHARED_OBJECTS, api.GI_PLAN_NAIVE]
+PLANNERS = [api.GI_PLAN_GREEDY_BY_SIZE, api.GI_PLAN_GREEDY_SHARED_OBJECTS, api.GI_PLAN_NAIVE, api.GI_PLAN_MIN_COST_FLOW]
 NETS = [lambda: wl.separable_block(1), lambda: wl.mobilenet_v1(1), lambda: wl.mobilenet_v2(1),
         lambda: wl.mobilenet_v2_segmentation(1), lambda: wl.mobilenet_v2(256), lambda: wl.mobilenet_v2_segmentation(16),
         lambda: wl.single_pointwise(8, 14, 96, 576, residual=True), lambda: wl.single_depthwise(8, 7, 96, 2)]
