@@ -96,7 +96,8 @@ enum {
  * with it as one kernel, so the tensor between them never reaches memory (fp16 storage; Section 3.3
  * folds element-wise operators into their producer, this folds a whole operator).  Results are
  * those of the two operators run one after the other: the tensor between them is still rounded to
- * fp16.  The memory plan is not affected: the tensor keeps its place in the arena, unused. */
+ * fp16.  The memory plan is not affected: the tensor keeps its place in the arena, unused; a pair whose input
+ * and output the planner placed on the same bytes (legal for two ops, not for one kernel) stays two kernels. */
 enum {
   GI_XOP_AUTO = 0,  /* the library's choice: at present the same as GI_XOP_OFF, the single kernel has not measured
                        faster than the two kernels on any layer of the benchmark networks (default) */

@@ -94,7 +94,8 @@ static void pack_depthwise(const OpNode& op, int c, int storage, std::vector<uin
 }
 
 // The executed op after depthwise op `i` is a 1x1 convolution that is the only reader of the depthwise
-// output, and that output is an arena tensor: the pair may run as one kernel.
+// output, that output is an arena tensor, and the pair's input and output do not share memory: the pair
+// may run as one kernel.
 static bool pointwise_follows(const gi_graph& g, const gi_exec* e, size_t i) {
   if (i + 1 >= e->ops.size()) return false;
   const FusedOp& f = e->ops[i];
@@ -105,6 +106,13 @@ static bool pointwise_follows(const gi_graph& g, const gi_exec* e, size_t i) {
   const TensorPlan& tp = e->plan[f.out];
   if (!tp.intermediate || tp.first != static_cast<int>(i) || tp.last != static_cast<int>(i + 1)) return false;
   if (e->tensors[f.out].output_index >= 0) return false;
+  // One kernel reads the depthwise input while it writes the 1x1 convolution's output.  As separate ops their
+  // lifetimes do not meet, so the planner may have given them the same arena bytes: then the pair stays two kernels.
+  const TensorPlan& pin = e->plan[f.in0];
+  const TensorPlan& pout = e->plan[n.out];
+  if (loc_of(e, f.in0).where == W_ARENA && loc_of(e, n.out).where == W_ARENA && pin.offset < pout.offset + pout.bytes &&
+      pout.offset < pin.offset + pin.bytes)
+    return false;
   const gi_op_desc& d = g.ops[n.graph_op].d;
   return d.kh == 1 && d.kw == 1 && d.stride_h == 1 && d.stride_w == 1 && d.pad_t == 0 && d.pad_l == 0 && d.pad_b == 0 &&
          d.pad_r == 0;

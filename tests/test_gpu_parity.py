@@ -194,7 +194,7 @@ def test_depthwise_pointwise_one_kernel(case):
     batch, h, w, c, cout, stride, residual = case
     spec = depthwise_pointwise_spec(batch, h, w, c, cout, stride, residual)
     graph, _ = api.graph_from_spec(spec, api.GI_F16)
-    names = [api.KERNEL_NAMES[o.kernel] for o in graph.compile(cross_op=api.GI_XOP_ON).ops()]
+    names = [api.KERNEL_NAMES[o.kernel] for o in graph.compile(cross_op=api.GI_XOP_ON, planner=api.GI_PLAN_NAIVE).ops()]
     assert "depthwise_pointwise" in names and "none" in names, names
     check_all_tensors(spec, api.GI_F16, cross_op=api.GI_XOP_ON)
     assert api.gi_device_status() == 0
@@ -273,6 +273,18 @@ def test_mobilenet_v2_batch256_sampled_images():
         assert np.array_equal(outs[t], again[t])
     # images are independent: the same image in another slot gives the same answer up to kernel tiling
     assert np.isfinite(outs[spec.outputs[0]]).all()
+
+
+def test_mobilenet_v2_batch64_one_kernel_pairs_sampled_images():
+    """The 13 depthwise -> projection pairs that qualify run as one kernel each (opt-in)."""
+    spec = wl.mobilenet_v2(64)
+    run, xs, outs = check_outputs(spec, api.GI_F16, images=[0, 33, 63], cross_op=api.GI_XOP_ON)
+    names = [api.KERNEL_NAMES[o.kernel] for o in run.ex.ops()]
+    assert names.count("depthwise_pointwise") >= 6
+    again = run.run(xs)
+    for t in spec.outputs:
+        assert np.array_equal(outs[t], again[t])
+    assert api.gi_device_status() == 0
 
 
 def test_mobilenet_v1_batch256_sampled_images():
@@ -415,4 +427,7 @@ def test_random_graphs(seed):
     check_all_tensors(spec, api.GI_F16, pointwise=api.GI_PW_TC_PAIR)
     check_all_tensors(spec, api.GI_F32)
     check_outputs(spec, api.GI_F16)  # greedy-by-size arena: tensors share memory
+    # depthwise -> 1x1 pairs as one kernel wherever the pattern occurs (the tensor in between is not stored)
+    check_all_tensors(spec, api.GI_F16, cross_op=api.GI_XOP_ON)
+    check_outputs(spec, api.GI_F16, cross_op=api.GI_XOP_ON)
     assert api.gi_device_status() == 0

@@ -295,7 +295,7 @@ def test_cross_op_option():
 
     pair = wl.depthwise_then_pointwise(4, 28, 28, 32, 24, 1, residual=True)
     assert "depthwise_pointwise" not in kernels(pair) and "depthwise_pointwise" not in kernels(pair, cross_op=api.GI_XOP_OFF)
-    on = kernels(pair, cross_op=api.GI_XOP_ON)
+    on = kernels(pair, cross_op=api.GI_XOP_ON, planner=api.GI_PLAN_NAIVE)
     assert on.count("depthwise_pointwise") == 1 and on.count("none") == 1 and "depthwise" not in on
     assert on.index("none") == on.index("depthwise_pointwise") + 1
     # fp32 storage, channels not a multiple of 16, planes wider than 128 columns: two kernels
@@ -311,10 +311,20 @@ def test_cross_op_option():
     assert "depthwise_pointwise" not in kernels(b.finish(), cross_op=api.GI_XOP_ON)
     # the plan is not affected: the tensor keeps its arena slot, the op count stays
     g = api.graph_from_spec(pair, api.GI_F16)[0]
-    a, c = g.compile(cross_op=api.GI_XOP_OFF), g.compile(cross_op=api.GI_XOP_ON)
+    a, c = g.compile(cross_op=api.GI_XOP_OFF, planner=api.GI_PLAN_NAIVE), g.compile(cross_op=api.GI_XOP_ON, planner=api.GI_PLAN_NAIVE)
     assert a.info.arena_bytes == c.info.arena_bytes and a.info.n_ops == c.info.n_ops
-    # whole network at batch 256: the pairs that qualify
-    v2 = kernels(wl.mobilenet_v2(256), cross_op=api.GI_XOP_ON)
+    # whole network at batch 256: 13 pairs qualify; one kernel reads the pair's input while it writes its output, so a
+    # pair whose input and output share arena bytes (legal for two ops: their lifetimes do not meet) stays two kernels
+    v2 = kernels(wl.mobilenet_v2(256), cross_op=api.GI_XOP_ON, planner=api.GI_PLAN_NAIVE)
     assert v2.count("depthwise_pointwise") == v2.count("none") == 13
+    gv2 = api.graph_from_spec(wl.mobilenet_v2(256), api.GI_F16)[0]
+    for planner in (api.GI_PLAN_GREEDY_BY_SIZE, api.GI_PLAN_GREEDY_SHARED_OBJECTS, api.GI_PLAN_MIN_COST_FLOW):
+        ex = gv2.compile(cross_op=api.GI_XOP_ON, planner=planner)
+        ops = ex.ops()
+        for i, o in enumerate(ops):
+            if api.KERNEL_NAMES[o.kernel] == "depthwise_pointwise":
+                tin, tout = ex.tensor(o.inputs[0]), ex.tensor(ops[i + 1].output)
+                assert tin.offset + tin.bytes <= tout.offset or tout.offset + tout.bytes <= tin.offset
+    assert [api.KERNEL_NAMES[o.kernel] for o in gv2.compile(cross_op=api.GI_XOP_ON).ops()].count("depthwise_pointwise") == 11
     with pytest.raises(api.GiError):
         g.compile(cross_op=7)
