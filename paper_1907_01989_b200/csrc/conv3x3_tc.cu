@@ -146,7 +146,7 @@ __global__ void __launch_bounds__(kThreads, 6) conv3x3_tc_kernel(const StemParam
     };
     // ---- epilogue of one tile from accumulator `buf`; gp = this thread's pixel in the whole tensor
     auto epilogue = [&](int buf, unsigned phase, unsigned gp, bool in_tensor, bool real) -> bool {
-      if (!mbar_wait(smem_u32(&hdr->acc_full[buf]), phase, abort_flag, p.timeout_ns, &g_conv_tc_error, 4u)) return false;
+      if (!mbar_wait_warp(smem_u32(&hdr->acc_full[buf]), phase, abort_flag, p.timeout_ns, &g_conv_tc_error, 4u)) return false;
       tc_fence_after();
       const unsigned t_addr = tmem_base + buf * n_cols + (static_cast<unsigned>(warp * 32) << 16);
       auto finish = [&](const unsigned* r, unsigned c0) {

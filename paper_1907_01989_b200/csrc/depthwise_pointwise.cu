@@ -366,14 +366,14 @@ __global__ void __launch_bounds__(kThreads, 1)  // 96 registers: one scheduler h
     const unsigned lane_bits = static_cast<unsigned>(quarter * 32) << 16;
     unsigned it = 0, ci = 0;
     // the weights of both operators arrive once, before the first tile
-    bool ok = mbar_wait(smem_u32(&hdr->b_ready), 0u, abort_flag, g.timeout_ns, &g_fu_error, kErrCompute);
+    bool ok = mbar_wait_warp(smem_u32(&hdr->b_ready), 0u, abort_flag, g.timeout_ns, &g_fu_error, kErrCompute);
     // a finished tile waiting for its drain: accumulator row j -> pixel pend_off + j * Wo of every output slice
     bool pend = false;
     int pend_t = 0;
     const bool plain = g.act_pre == GI_ACT_NONE && g.act_post == GI_ACT_NONE;
     const size_t slice_stride = static_cast<size_t>(g.B) * g.Pout;  // pixels between output slices
     auto drain = [&]() {
-      if (!mbar_wait(smem_u32(&hdr->acc_full), static_cast<unsigned>(pend_t) & 1u, abort_flag, g.timeout_ns, &g_fu_error, kErrCompute)) {
+      if (!mbar_wait_warp(smem_u32(&hdr->acc_full), static_cast<unsigned>(pend_t) & 1u, abort_flag, g.timeout_ns, &g_fu_error, kErrCompute)) {
         ok = false;
         return;
       }
@@ -476,13 +476,13 @@ __global__ void __launch_bounds__(kThreads, 1)  // 96 registers: one scheduler h
           bias_acc.lo = make_float2(v.x, v.y);
           bias_acc.hi = make_float2(v.z, v.w);
         }
-        if (!mbar_wait(smem_u32(&hdr->a_empty[abuf]), ((ci >> 1) & 1u) ^ 1u, abort_flag, g.timeout_ns, &g_fu_error, kErrCompute)) {
+        if (!mbar_wait_warp(smem_u32(&hdr->a_empty[abuf]), ((ci >> 1) & 1u) ^ 1u, abort_flag, g.timeout_ns, &g_fu_error, kErrCompute)) {
           ok = false;
           break;
         }
         tc_fence_after();
         const unsigned stage = it % g.nbuf;
-        if (!mbar_wait(smem_u32(&hdr->full[stage]), (it / g.nbuf) & 1u, abort_flag, g.timeout_ns, &g_fu_error, kErrCompute)) {
+        if (!mbar_wait_warp(smem_u32(&hdr->full[stage]), (it / g.nbuf) & 1u, abort_flag, g.timeout_ns, &g_fu_error, kErrCompute)) {
           ok = false;
           break;
         }

@@ -227,7 +227,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
       const bool row_ok = row < rows_total;
       for (int nt = grp; nt < p.n_tiles && ok; nt += p.groups, ++tile) {
         const unsigned acc = tile % p.n_acc, acc_phase = (tile / p.n_acc) & 1u;
-        if (!mbar_wait(smem_u32(&hdr->acc_full[acc]), acc_phase, abort_flag, p.timeout_ns, &g_tc_error, kErrEpilogue)) {
+        if (!mbar_wait_warp(smem_u32(&hdr->acc_full[acc]), acc_phase, abort_flag, p.timeout_ns, &g_tc_error, kErrEpilogue)) {
           ok = false;
           break;
         }

@@ -260,8 +260,8 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
       for (int c = 0; c < p.n_chunks; ++c, ++it) {
         const unsigned stage = it % p.stages, s_phase = (it / p.stages) & 1u;
         const unsigned abuf = it & 1u, a_phase = (it >> 1) & 1u;
-        if (!mbar_wait(smem_u32(&hdr->full[stage]), s_phase, abort_flag, p.timeout_ns, &g_ts_error, kErrData) ||
-            !mbar_wait(smem_u32(&hdr->a_empty[abuf]), a_phase ^ 1u, abort_flag, p.timeout_ns, &g_ts_error, kErrData)) {
+        if (!mbar_wait_warp(smem_u32(&hdr->full[stage]), s_phase, abort_flag, p.timeout_ns, &g_ts_error, kErrData) ||
+            !mbar_wait_warp(smem_u32(&hdr->a_empty[abuf]), a_phase ^ 1u, abort_flag, p.timeout_ns, &g_ts_error, kErrData)) {
           ok = false;
           break;
         }
@@ -312,7 +312,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
       };
       uint2 res_cur[4], res_next[4];
       if (TAIL) fetch_res(res_cur, part_id);
-      if (!mbar_wait(smem_u32(&hdr->acc_full[acc]), acc_phase, abort_flag, p.timeout_ns, &g_ts_error, kErrData)) break;
+      if (!mbar_wait_warp(smem_u32(&hdr->acc_full[acc]), acc_phase, abort_flag, p.timeout_ns, &g_ts_error, kErrData)) break;
       tc_fence_after();
       if (tile == 0 && threadIdx.x == 32 * (2 + kTransferWarps)) GI_TRACE_EVENT(g_ts_trace, 6);
       const unsigned t_addr = tmem_base + lane_bits + acc * acc_cols;

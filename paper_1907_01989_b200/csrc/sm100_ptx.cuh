@@ -57,6 +57,16 @@ static __device__ __noinline__ bool mbar_wait(unsigned bar, unsigned parity, vol
   }
 }
 
+// The same wait for a whole warp that goes on to warp-collective instructions (tcgen05.ld / .st / .wait are
+// .sync.aligned: all 32 lanes must execute them together).  Lanes leave the polling loop at different
+// iterations; the vote brings them back together and gives every lane the same answer, so that the warp
+// also gives up as one.
+__device__ __forceinline__ bool mbar_wait_warp(unsigned bar, unsigned parity, volatile unsigned* abort_flag, unsigned timeout_ns,
+                                               unsigned* error_word, unsigned code) {
+  const bool ok = mbar_wait(bar, parity, abort_flag, timeout_ns, error_word, code);
+  return __all_sync(0xffffffffu, ok) != 0;
+}
+
 __device__ __forceinline__ void tma_load_2d(unsigned dst, const CUtensorMap* map, int x, int y, unsigned bar) {
   asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
                "l"(reinterpret_cast<unsigned long long>(map)), "r"(x), "r"(y), "r"(bar)
