@@ -17,7 +17,7 @@ def unpack_phwc4(raw: np.ndarray, B: int, H: int, W: int, Cc: int) -> np.ndarray
     return np.ascontiguousarray(a.transpose(1, 2, 0, 3).reshape(B, H, W, S * 4)[..., :Cc])
 
 
-class GpuRun:
+class DeviceRun:
     def __init__(self, spec, storage=api.GI_F16, planner=api.GI_PLAN_GREEDY_BY_SIZE, pointwise=api.GI_PW_AUTO,
                  fuse=True, guard_bytes=0, cross_op=api.GI_XOP_AUTO):
         import torch

@@ -9,7 +9,7 @@ from oracle import ops as oops
 from paper_1907_01989_b200 import api
 from paper_1907_01989_b200 import workloads as wl
 
-from gpu_util import GpuRun, assert_close
+from gpu_util import DeviceRun, assert_close
 
 pytestmark = pytest.mark.gpu
 
@@ -21,7 +21,7 @@ def check_all_tensors(spec, storage, pointwise=api.GI_PW_AUTO, fuse=True, cross_
     """Naive planner keeps every intermediate, so each stored tensor is compared, not only the output."""
     xs = [wl.make_input(spec, index=i) for i in range(len(spec.inputs))]
     ref = og.run(spec, xs, storage=SNAME[storage], fused=fuse, keep_all=True)
-    run = GpuRun(spec, storage, planner=api.GI_PLAN_NAIVE, pointwise=pointwise, fuse=fuse, guard_bytes=4096, cross_op=cross_op)
+    run = DeviceRun(spec, storage, planner=api.GI_PLAN_NAIVE, pointwise=pointwise, fuse=fuse, guard_bytes=4096, cross_op=cross_op)
     outs = run.run(xs)
     assert run.guard_intact()
     worst = 0.0
@@ -35,7 +35,7 @@ def check_all_tensors(spec, storage, pointwise=api.GI_PW_AUTO, fuse=True, cross_
 
 def check_outputs(spec, storage, images=None, **kw):
     xs = [wl.make_input(spec, index=i) for i in range(len(spec.inputs))]
-    run = GpuRun(spec, storage, guard_bytes=4096, **kw)
+    run = DeviceRun(spec, storage, guard_bytes=4096, **kw)
     outs = run.run(xs)
     assert run.guard_intact()
     sel = list(range(spec.batch)) if images is None else images
@@ -58,7 +58,7 @@ def test_separable_block(storage, pointwise):
 def test_planners_give_same_result(planner):
     spec = wl.mobilenet_v2(2, size=64)
     run, xs, outs = check_outputs(spec, api.GI_F16, planner=planner)
-    base = GpuRun(spec, api.GI_F16, planner=api.GI_PLAN_NAIVE).run(xs)
+    base = DeviceRun(spec, api.GI_F16, planner=api.GI_PLAN_NAIVE).run(xs)
     for t in spec.outputs:
         assert np.array_equal(outs[t], base[t])
 
@@ -73,7 +73,7 @@ def test_pack_layout_bit_exact(storage, shape):
     b.output(b.activation(x, wl.ACT_RELU))
     spec = b.finish()
     xin = wl.make_input(spec)
-    run = GpuRun(spec, storage, planner=api.GI_PLAN_NAIVE)
+    run = DeviceRun(spec, storage, planner=api.GI_PLAN_NAIVE)
     outs = run.run([xin])
     phys = oops.phwc4_pack(xin).reshape(-1)
     got = run.fetch_raw(spec.inputs[0]).astype(np.float32)
@@ -299,7 +299,7 @@ def test_segmentation_batch16_sampled_images():
 def test_run_argument_checks():
     import torch
     spec = wl.separable_block(1)
-    run = GpuRun(spec, api.GI_F16)
+    run = DeviceRun(spec, api.GI_F16)
     x = torch.zeros((1, 32, 32, 32), dtype=torch.float16, device="cuda:0")
     out = run.outs[0]
     nb = int(run.ex.info.arena_bytes)
