@@ -209,7 +209,9 @@ GI_API void gi_graph_destroy(gi_graph* g);
 
 /* ---- compile (Sections 3.2 and 5) ---- */
 
-/* Build an executable: verify the order, fuse, compute lifetimes, plan memory, pack weights,
+/* Build an executable: verify the order, clean the graph (Section 3.1: an identity operator - a RESIZE to its
+ * input's own size - is dropped and its readers read its input, unless its output is a graph output; the
+ * dropped op's output tensor is then not alive), fuse, compute lifetimes, plan memory, pack weights,
  * choose a kernel and launch shape per fused op.  Host work only; no CUDA call is made.
  * `opt` may be NULL for defaults.  The graph stays valid and may be compiled again. */
 GI_API gi_status gi_compile(const gi_graph* g, const gi_compile_options* opt, gi_exec** out);

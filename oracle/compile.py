@@ -53,11 +53,26 @@ def fuse(g, enable: bool = True, fold_add: bool = True) -> List[FusedOp]:
     the other operand must be a different tensor of the same shape that exists before F runs
     (a graph input or the output of an earlier fused op); if both operands qualify the later
     fused op takes the add.  The folded op's output replaces x as F's output.
+
+    First the graph is cleaned (Section 3.1, "Graph transformation"): a superfluous identity operator -
+    here a resize to the size its input already has - is removed and what read its output reads its
+    input; it stays if its output is a graph output.
     """
+    alias: Dict[int, int] = {}
+
+    def src(t: int) -> int:
+        return alias.get(t, t)
+
+    dropped = set()
     uses: Dict[int, int] = {}
-    for op in g.ops:
+    for idx, op in enumerate(g.ops):
+        if (op.kind == "resize_bilinear" and tuple(g.shapes[op.output][:2]) == tuple(g.shapes[op.inputs[0]][:2])
+                and op.output not in set(g.outputs)):
+            alias[op.output] = src(op.inputs[0])
+            dropped.add(idx)
+            continue
         for t in op.inputs:
-            uses[t] = uses.get(t, 0) + 1
+            uses[src(t)] = uses.get(src(t), 0) + 1
     graph_outputs = set(g.outputs)
     graph_inputs = set(g.inputs)
     fused: List[FusedOp] = []
@@ -72,8 +87,11 @@ def fuse(g, enable: bool = True, fold_add: bool = True) -> List[FusedOp]:
         return None
 
     for idx, op in enumerate(g.ops):
+        if idx in dropped:
+            continue
+        ins = [src(t) for t in op.inputs]
         if enable and op.kind == "activation":
-            i = foldable_into(op.inputs[0])
+            i = foldable_into(ins[0])
             if i is not None and fused[i].can_take("act"):
                 fused[i].take("act")
                 fused[i].epilogue.append(("act", op.act))
@@ -82,7 +100,7 @@ def fuse(g, enable: bool = True, fold_add: bool = True) -> List[FusedOp]:
                 producer[op.output] = i
                 continue
         if enable and fold_add and op.kind == "add":
-            a, b = op.inputs
+            a, b = ins
             if a != b and g.shapes[a] == g.shapes[b]:
                 candidates = []
                 for x, other in ((a, b), (b, a)):
@@ -99,7 +117,7 @@ def fuse(g, enable: bool = True, fold_add: bool = True) -> List[FusedOp]:
                     fused[i].output = op.output
                     producer[op.output] = i
                     continue
-        fused.append(FusedOp(kind=op.kind, op_index=idx, inputs=list(op.inputs), output=op.output))
+        fused.append(FusedOp(kind=op.kind, op_index=idx, inputs=ins, output=op.output))
         producer[op.output] = len(fused) - 1
     return fused
 

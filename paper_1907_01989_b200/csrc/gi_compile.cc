@@ -28,17 +28,33 @@ static int next_slot(int slot, int what) {
 // fused op that produces its operand when that op leads with a convolution, the operand has
 // no other use and is not a graph output, and the chain stays inside [act][add][act]; the
 // other operand of a folded ADD must already exist when the convolution runs.
+//
+// Before that, the graph is cleaned as in Section 3.1: a superfluous identity operator - here a RESIZE whose
+// output has the size of its input - is dropped and its readers read its input instead (unless its output is
+// a graph output, which has to exist as a tensor of its own).
 gi_status fuse_graph(const gi_graph& g, bool enable, std::vector<FusedOp>* out) {
   const int nt = static_cast<int>(g.tensors.size());
+  std::vector<int> alias(nt);  // tensor -> the tensor that holds its values
+  for (int t = 0; t < nt; ++t) alias[t] = t;
+  std::vector<char> dropped(g.ops.size(), 0);
   std::vector<int> uses(nt, 0);
-  for (const OpNode& op : g.ops) {
+  for (size_t idx = 0; idx < g.ops.size(); ++idx) {
+    const OpNode& op = g.ops[idx];
     // insertion order must be topological: every input id is smaller than the output id
     for (int k = 0; k < 2; ++k) {
       const int t = op.d.inputs[k];
       if (k == 1 && op.d.kind != GI_OP_ADD) continue;
       if (t < 0 || t >= op.output) return fail(GI_E_INVALID, "gi_compile: operator reads a tensor defined after it");
-      ++uses[t];
     }
+    const int in0 = op.d.inputs[0];
+    if (op.d.kind == GI_OP_RESIZE_BILINEAR && g.tensors[op.output].h == g.tensors[in0].h &&
+        g.tensors[op.output].w == g.tensors[in0].w && g.tensors[op.output].output_index < 0) {
+      alias[op.output] = alias[in0];
+      dropped[idx] = 1;
+      continue;
+    }
+    ++uses[alias[in0]];
+    if (op.d.kind == GI_OP_ADD) ++uses[alias[op.d.inputs[1]]];
   }
   std::vector<FusedOp>& fused = *out;
   fused.clear();
@@ -53,8 +69,10 @@ gi_status fuse_graph(const gi_graph& g, bool enable, std::vector<FusedOp>* out) 
 
   for (size_t idx = 0; idx < g.ops.size(); ++idx) {
     const OpNode& op = g.ops[idx];
+    if (dropped[idx]) continue;
+    const int in_a = alias[op.d.inputs[0]], in_b = op.d.kind == GI_OP_ADD ? alias[op.d.inputs[1]] : -1;
     if (enable && op.d.kind == GI_OP_ACTIVATION) {
-      const int i = foldable(op.d.inputs[0]);
+      const int i = foldable(in_a);
       const int pos = i >= 0 ? next_slot(fused[i].slot, 0) : -1;
       if (pos >= 0) {
         FusedOp& f = fused[i];
@@ -67,7 +85,7 @@ gi_status fuse_graph(const gi_graph& g, bool enable, std::vector<FusedOp>* out) 
       }
     }
     if (enable && op.d.kind == GI_OP_ADD) {
-      const int a = op.d.inputs[0], b = op.d.inputs[1];
+      const int a = in_a, b = in_b;
       if (a != b) {
         int best = -1, best_x = -1, best_other = -1;
         const int pair[2][2] = {{a, b}, {b, a}};
@@ -96,8 +114,8 @@ gi_status fuse_graph(const gi_graph& g, bool enable, std::vector<FusedOp>* out) 
     FusedOp f;
     f.kind = op.d.kind;
     f.graph_op = static_cast<int>(idx);
-    f.in0 = op.d.inputs[0];
-    f.in1 = op.d.kind == GI_OP_ADD ? op.d.inputs[1] : -1;
+    f.in0 = in_a;
+    f.in1 = in_b;
     f.out = op.output;
     fused.push_back(f);
     producer[op.output] = static_cast<int>(fused.size()) - 1;

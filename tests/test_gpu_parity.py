@@ -431,3 +431,19 @@ def test_random_graphs(seed):
     check_all_tensors(spec, api.GI_F16, cross_op=api.GI_XOP_ON)
     check_outputs(spec, api.GI_F16, cross_op=api.GI_XOP_ON)
     assert api.gi_device_status() == 0
+
+
+def test_identity_resize_removed():
+    """A resize to the input's own size is dropped at compile time (Section 3.1); results are those of the oracle,
+    whose own clean-up is pinned to change nothing."""
+    b = wl.GraphBuilder("identity_ops", 3, 21)
+    x = b.input(10, 6, 8)
+    c = b.conv2d(x, 12, 1)
+    a = b.activation(b.resize_bilinear(c, 10, 6, True), wl.ACT_RELU6)
+    r2 = b.resize_bilinear(a, 10, 6, False)
+    b.output(r2)
+    b.output(b.resize_bilinear(b.depthwise(r2, 3, 1, 1), 20, 12, True))
+    spec = b.finish()
+    for storage in STORAGES:
+        check_all_tensors(spec, storage)
+        check_outputs(spec, storage)

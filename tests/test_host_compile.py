@@ -328,3 +328,21 @@ def test_cross_op_option():
     assert [api.KERNEL_NAMES[o.kernel] for o in gv2.compile(cross_op=api.GI_XOP_ON).ops()].count("depthwise_pointwise") == 11
     with pytest.raises(api.GiError):
         g.compile(cross_op=7)
+
+
+def test_identity_resize_removed_like_the_oracle():
+    """Graph clean-up (Section 3.1): the library drops the same identity ops as the oracle; plan and op list agree."""
+    for extra in (False, True):
+        b = wl.GraphBuilder("identity_ops", 2, 21)
+        x = b.input(6, 5, 8)
+        c = b.conv2d(x, 12, 1)
+        a = b.activation(b.resize_bilinear(c, 6, 5, True), wl.ACT_RELU)
+        r2 = b.resize_bilinear(a, 6, 5, False)
+        if extra:
+            b.output(r2)
+        b.output(b.resize_bilinear(r2, 12, 10, True))
+        spec = b.finish()
+        for planner in PLANNERS:
+            ex = compare_with_oracle(spec, planner)
+        assert ex.info.n_fused_ops == (3 if extra else 2)
+        compare_with_oracle(spec, api.GI_PLAN_GREEDY_BY_SIZE, fuse=False)

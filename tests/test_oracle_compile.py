@@ -355,3 +355,38 @@ def test_fusion_rules_small_cases():
            [("conv2d", [0], 1, None), ("add", [0, 1], 2, None), ("add", [0, 2], 3, None)])
     f = oc.fuse(g)
     assert len(f) == 2 and f[1].kind == "add"
+
+
+# ---------------------------------------------------------------------- identity removal (Section 3.1)
+def _identity_graph(extra_output=False):
+    """conv -> resize to the same size -> relu -> resize to the same size -> resize x2 -> output."""
+    b = wl.GraphBuilder("identity_ops", 2, 21)
+    x = b.input(6, 5, 8)
+    c = b.conv2d(x, 12, 1)
+    r1 = b.resize_bilinear(c, 6, 5, True)
+    a = b.activation(r1, wl.ACT_RELU)
+    r2 = b.resize_bilinear(a, 6, 5, False)
+    r3 = b.resize_bilinear(r2, 12, 10, True)
+    if extra_output:
+        b.output(r2)
+    b.output(r3)
+    return b.finish(), (c, r1, a, r2, r3)
+
+
+def test_identity_resize_is_removed_and_its_readers_read_its_input():
+    g, (c, r1, a, r2, r3) = _identity_graph()
+    f = oc.fuse(g)
+    # the activation folds into the convolution THROUGH the removed resize; the real resize reads the conv's result
+    assert [x.kind for x in f] == ["conv2d", "resize_bilinear"]
+    assert f[0].epilogue == [("act", "relu")] and f[0].output == a and f[1].inputs == [a] and f[1].output == r3
+    p = oc.plan_problem(g, f, convert_io=True)
+    assert r1 not in p.size and r2 not in p.size
+    # without fusion the identities are still removed
+    assert [x.kind for x in oc.fuse(g, enable=False)] == ["conv2d", "activation", "resize_bilinear"]
+
+
+def test_identity_resize_that_is_a_graph_output_stays():
+    g, (c, r1, a, r2, r3) = _identity_graph(extra_output=True)
+    f = oc.fuse(g)
+    assert [x.kind for x in f] == ["conv2d", "resize_bilinear", "resize_bilinear"]
+    assert f[1].output == r2 and f[1].inputs == [a] and f[2].inputs == [r2]

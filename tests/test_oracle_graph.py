@@ -125,3 +125,32 @@ def test_input_generator_is_batch_independent():
     for a, b in zip(g4.ops, g2.ops):
         if a.weights is not None:
             assert np.array_equal(a.weights, b.weights) and np.array_equal(a.bias, b.bias)
+
+
+def test_resize_to_the_same_size_is_the_identity_and_removing_it_changes_nothing():
+    """The premise of the identity-removal pass: bilinear resize to the input's own size returns the input
+    bit for bit (both corner conventions), so the cleaned graph computes exactly what the original does."""
+    from oracle import ops
+    rnd = np.random.default_rng(3)
+    x = rnd.standard_normal((2, 6, 5, 7)).astype(np.float32)
+    for ac in (True, False):
+        assert np.array_equal(ops.resize_bilinear(x, 6, 5, ac), x)
+    # the same network with and without the identity ops
+    def build(with_identities):
+        b = wl.GraphBuilder("identity_ops", 2, 21)
+        t = b.input(6, 5, 8)
+        y = b.conv2d(t, 12, 1)
+        if with_identities:
+            y = b.resize_bilinear(y, 6, 5, True)
+        y = b.activation(y, wl.ACT_RELU)
+        if with_identities:
+            y = b.resize_bilinear(y, 6, 5, False)
+        y = b.resize_bilinear(y, 12, 10, True)
+        b.output(y)
+        return b.finish()
+    ga, gb = build(True), build(False)
+    xs = [wl.make_input(ga, index=0)]
+    for storage in ("f16", "f32"):
+        ya = og.run(ga, xs, storage=storage)[ga.outputs[0]]
+        yb = og.run(gb, xs, storage=storage)[gb.outputs[0]]
+        assert np.array_equal(ya, yb)
