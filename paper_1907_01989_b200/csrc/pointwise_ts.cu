@@ -381,12 +381,22 @@ struct Tiling {
   size_t smem;
 };
 
-Tiling choose_tiling(int cin, int cout) {
+// `m_px`: pixels of the layer (batch x H x W; 0 = unknown).  A layer with few pixel tiles - batch 1, or the
+// classifier behind the global pool - is a handful of CTAs that each stream a wide share of the weights from
+// L2: there the output channels are split into narrower shares (down to 32 channels) until about half the
+// SMs take part, so that the weights arrive through many SMs at once.
+Tiling choose_tiling(int cin, int cout, long long m_px) {
   Tiling t;
   t.s_in = slices(cin);
   t.s_out = slices(cout);
   const int n_pad = (cout + 15) / 16 * 16;
   t.n_parts = (n_pad + kMaxNcta - 1) / kMaxNcta;
+  if (m_px > 0) {
+    const long long m_tiles = (m_px + kRows - 1) / kRows;
+    while (m_tiles * t.n_parts < 74 && ((n_pad + t.n_parts - 1) / t.n_parts + 15) / 16 * 16 > 32) ++t.n_parts;
+    const int n_cta = ((n_pad + t.n_parts - 1) / t.n_parts + 15) / 16 * 16;
+    t.n_parts = (n_pad + n_cta - 1) / n_cta;  // no share left empty by the rounding to 16 channels
+  }
   const int s_pad = (t.s_in + 7) / 8 * 8;
   for (;; ++t.n_parts) {
     t.n_cta = ((n_pad + t.n_parts - 1) / t.n_parts + 15) / 16 * 16;
@@ -425,12 +435,12 @@ Tiling choose_tiling(int cin, int cout) {
 
 bool pointwise_ts_supported(int cin, int cout) {
   if (cin <= 0 || cout <= 0) return false;
-  return choose_tiling(cin, cout).smem <= static_cast<size_t>(kSmemHeader + kSmemBudget + 16 * 1024);
+  return choose_tiling(cin, cout, 0).smem <= static_cast<size_t>(kSmemHeader + kSmemBudget + 16 * 1024);
 }
 
 // Dense weights as the B operand, per (CTA share, K chunk): [ks/2 K units][n_cta rows][8 halves].
 void pointwise_ts_pack(const float* w, const float* bias, int cin, int cout, std::vector<uint8_t>* blob, LaunchRec* r) {
-  const Tiling t = choose_tiling(cin, cout);
+  const Tiling t = choose_tiling(cin, cout, static_cast<long long>(r->B) * r->H * r->W);
   const size_t chunk_bytes = static_cast<size_t>(t.ks) * t.n_cta * 8;
   const size_t wbytes = static_cast<size_t>(t.n_parts) * t.n_chunks * chunk_bytes;
   const uint64_t woff = round_up_u64(blob->size(), 256);
@@ -457,7 +467,7 @@ void pointwise_ts_pack(const float* w, const float* bias, int cin, int cout, std
 }
 
 int launch_pointwise_ts(const LaunchRec& r, const Ptrs& p, void** state, int launch_index, void* stream) {
-  const Tiling t = choose_tiling(r.C, r.Co);
+  const Tiling t = choose_tiling(r.C, r.Co, static_cast<long long>(r.B) * r.H * r.W);
   TsParams k;
   k.res = static_cast<const __half*>(p.res);
   k.out = static_cast<__half*>(p.out);
