@@ -383,8 +383,9 @@ struct Tiling {
 
 // `m_px`: pixels of the layer (batch x H x W; 0 = unknown).  A layer with few pixel tiles - batch 1, or the
 // classifier behind the global pool - is a handful of CTAs that each stream a wide share of the weights from
-// L2: there the output channels are split into narrower shares (down to 32 channels) until about half the
-// SMs take part, so that the weights arrive through many SMs at once.
+// L2: there the output channels are split into narrower shares (down to 32 channels) until every SM
+// takes part (measured: better than half of them, and than 16- or 48-channel shares), so that the weights arrive
+// through many SMs at once.
 Tiling choose_tiling(int cin, int cout, long long m_px) {
   Tiling t;
   t.s_in = slices(cin);
@@ -393,7 +394,7 @@ Tiling choose_tiling(int cin, int cout, long long m_px) {
   t.n_parts = (n_pad + kMaxNcta - 1) / kMaxNcta;
   if (m_px > 0) {
     const long long m_tiles = (m_px + kRows - 1) / kRows;
-    while (m_tiles * t.n_parts < 74 && ((n_pad + t.n_parts - 1) / t.n_parts + 15) / 16 * 16 > 32) ++t.n_parts;
+    while (m_tiles * t.n_parts < 148 && ((n_pad + t.n_parts - 1) / t.n_parts + 15) / 16 * 16 > 32) ++t.n_parts;
     const int n_cta = ((n_pad + t.n_parts - 1) / t.n_parts + 15) / 16 * 16;
     t.n_parts = (n_pad + n_cta - 1) / n_cta;  // no share left empty by the rounding to 16 channels
   }
