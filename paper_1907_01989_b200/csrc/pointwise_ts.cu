@@ -59,6 +59,7 @@ struct TsParams {
   int b_resident;        // 1: the CTA's weights are loaded once; 0: a weight chunk rides in every stage
   int stages;
   int m_tiles;
+  int box_px;            // pixels per TMA box: 128, or 64 / 32 when the whole layer has no more (the rest of the tile is never fetched)
   int has_res, act_post;
   int in_dead;           // the input is not read again: its TMA loads carry the evict-first L2 hint
   unsigned int timeout_ns;
@@ -117,7 +118,8 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
   Header* hdr = reinterpret_cast<Header*>(smem);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile unsigned* abort_flag = &hdr->abort_flag;
-  const unsigned a_stage_bytes = static_cast<unsigned>(p.ks) * 1024u;             // ks slices x 128 pixels x 8 bytes
+  const unsigned slice_bytes = static_cast<unsigned>(p.box_px) * 8u;              // one slice of a box: box_px pixels x 8 bytes
+  const unsigned a_stage_bytes = static_cast<unsigned>(p.ks) * slice_bytes;       // ks slices
   const unsigned b_chunk_bytes = static_cast<unsigned>(p.ks) * p.n_cta * 8u;      // ks/2 K units x n_cta rows x 16 bytes
   const unsigned stage_bytes = a_stage_bytes + (p.b_resident ? 0u : b_chunk_bytes);
   const unsigned b_res_bytes = p.b_resident ? b_chunk_bytes * p.n_chunks : 0u;
@@ -268,11 +270,13 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
         tc_fence_after();
         const unsigned src = stage0 + stage * stage_bytes + row_off;
         const unsigned t_addr = tmem_base + lane_bits + a_col0 + abuf * a_cols;
-        for (int j = 0; j < p.ks; j += 8) {
+        // a box narrower than 128 pixels leaves the upper lane quarters without data: their rows of the
+        // accumulator are never stored, so their lanes of the A operand may hold anything
+        for (int j = 0; j < p.ks && quarter * 32 < p.box_px; j += 8) {
           unsigned r[16];
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
-            const uint2 v = lds64(src + static_cast<unsigned>(j + q) * 1024u);
+            const uint2 v = lds64(src + static_cast<unsigned>(j + q) * slice_bytes);
             r[2 * q] = v.x;
             r[2 * q + 1] = v.y;
           }
@@ -377,7 +381,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
 }
 
 struct Tiling {
-  int s_in, s_out, ks, n_chunks, n_cta, n_parts, b_resident, stages;
+  int s_in, s_out, ks, n_chunks, n_cta, n_parts, b_resident, stages, box_px;
   size_t smem;
 };
 
@@ -392,6 +396,10 @@ Tiling choose_tiling(int cin, int cout, long long m_px) {
   t.s_out = slices(cout);
   const int n_pad = (cout + 15) / 16 * 16;
   t.n_parts = (n_pad + kMaxNcta - 1) / kMaxNcta;
+  // a layer of at most 64 (32) pixels is fetched in boxes of 64 (32) pixels: less zero fill in shared memory,
+  // fewer lanes to move into tensor memory, and room for twice (four times) the slices per chunk
+  t.box_px = m_px > 0 && m_px <= 32 ? 32 : m_px > 0 && m_px <= 64 ? 64 : kRows;
+  const int slice_bytes = t.box_px * 8;
   if (m_px > 0) {
     const long long m_tiles = (m_px + kRows - 1) / kRows;
     while (m_tiles * t.n_parts < 148 && ((n_pad + t.n_parts - 1) / t.n_parts + 15) / 16 * 16 > 32) ++t.n_parts;
@@ -403,7 +411,7 @@ Tiling choose_tiling(int cin, int cout, long long m_px) {
     t.n_cta = ((n_pad + t.n_parts - 1) / t.n_parts + 15) / 16 * 16;
     // TMEM: 2 accumulators of n_cta columns + 2 A buffers of 2*ks columns <= 512
     int ks_max = (512 - 2 * t.n_cta) / 4 / 8 * 8;
-    if (ks_max > 64) ks_max = 64;
+    if (ks_max > 64 * (kRows / t.box_px)) ks_max = 64 * (kRows / t.box_px);
     t.n_chunks = (s_pad + ks_max - 1) / ks_max;
     t.ks = ((s_pad + t.n_chunks - 1) / t.n_chunks + 7) / 8 * 8;
     const size_t b_all = static_cast<size_t>(t.n_chunks) * t.ks * t.n_cta * 8;
@@ -416,14 +424,14 @@ Tiling choose_tiling(int cin, int cout, long long m_px) {
   for (;;) {
     const size_t bc = static_cast<size_t>(t.ks) * t.n_cta * 8;
     const size_t res = t.b_resident ? bc * t.n_chunks : 0;
-    const size_t st = static_cast<size_t>(t.ks) * 1024 + (t.b_resident ? 0 : bc);
+    const size_t st = static_cast<size_t>(t.ks) * slice_bytes + (t.b_resident ? 0 : bc);
     if (t.ks <= 8 || res + 2 * st <= static_cast<size_t>(kSmemBudget)) break;
     t.ks = (t.ks / 2 + 7) / 8 * 8;
     t.n_chunks = (s_pad + t.ks - 1) / t.ks;
   }
   const size_t b_chunk = static_cast<size_t>(t.ks) * t.n_cta * 8;
   const size_t resident = t.b_resident ? b_chunk * t.n_chunks : 0;
-  const size_t stage = static_cast<size_t>(t.ks) * 1024 + (t.b_resident ? 0 : b_chunk);
+  const size_t stage = static_cast<size_t>(t.ks) * slice_bytes + (t.b_resident ? 0 : b_chunk);
   long long stages = (static_cast<long long>(kSmemBudget) - static_cast<long long>(resident)) / static_cast<long long>(stage);
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages < 2) stages = 2;
@@ -441,7 +449,7 @@ bool pointwise_ts_supported(int cin, int cout) {
 
 // Dense weights as the B operand, per (CTA share, K chunk): [ks/2 K units][n_cta rows][8 halves].
 void pointwise_ts_pack(const float* w, const float* bias, int cin, int cout, std::vector<uint8_t>* blob, LaunchRec* r) {
-  const Tiling t = choose_tiling(cin, cout, static_cast<long long>(r->B) * r->H * r->W);
+  const Tiling t = choose_tiling(cin, cout, static_cast<long long>(r->B) * plane_pixels(r->H, r->W));
   const size_t chunk_bytes = static_cast<size_t>(t.ks) * t.n_cta * 8;
   const size_t wbytes = static_cast<size_t>(t.n_parts) * t.n_chunks * chunk_bytes;
   const uint64_t woff = round_up_u64(blob->size(), 256);
@@ -468,7 +476,7 @@ void pointwise_ts_pack(const float* w, const float* bias, int cin, int cout, std
 }
 
 int launch_pointwise_ts(const LaunchRec& r, const Ptrs& p, void** state, int launch_index, void* stream) {
-  const Tiling t = choose_tiling(r.C, r.Co, static_cast<long long>(r.B) * r.H * r.W);
+  const Tiling t = choose_tiling(r.C, r.Co, static_cast<long long>(r.B) * plane_pixels(r.H, r.W));
   TsParams k;
   k.res = static_cast<const __half*>(p.res);
   k.out = static_cast<__half*>(p.out);
@@ -483,6 +491,7 @@ int launch_pointwise_ts(const LaunchRec& r, const Ptrs& p, void** state, int lau
   k.b_resident = t.b_resident;
   k.stages = t.stages;
   k.m_tiles = static_cast<int>((k.m_total_px + kRows - 1) / kRows);
+  k.box_px = t.box_px;
   k.has_res = r.ep.has_res;
   k.act_post = r.ep.act_post;
   k.in_dead = r.in0_dead;
@@ -508,7 +517,7 @@ int launch_pointwise_ts(const LaunchRec& r, const Ptrs& p, void** state, int lau
   }
   MapEntry& me = map_cache_entry(state, launch_index);
   if (me.in != p.in0) {
-    const int err = encode_plane_map(&me.map, p.in0, k.m_total_px, t.s_in, kRows, t.ks);
+    const int err = encode_plane_map(&me.map, p.in0, k.m_total_px, t.s_in, t.box_px, t.ks);
     if (err != 0) return err;
     me.in = p.in0;
   }
