@@ -224,15 +224,20 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
           const bool pointwise = op.d.kh == 1 && op.d.stride_h == 1 && op.d.stride_w == 1 && op.d.pad_t == 0 &&
                                  op.d.pad_l == 0 && op.d.pad_b == 0 && op.d.pad_r == 0;
           const bool tc = e->storage == GI_F16 && e->opt.pointwise != GI_PW_SIMT;
-          // many input channels: the lane-per-pixel kernel (dense weight tile); few: the pixel-pair
-          // kernel (activations by TMA)
-          // (measured on MobileNetV2 at batch 256: the lane kernel wins from ~144 input channels on
-          // small planes and from 192 on everywhere, except for very deep, narrow projections)
-          // (and whenever all pixels fit one wave of its 128-pixel tiles: latency-bound launches, where its
-          // shorter fill - dense weights, no expansion - wins: MobileNetV2 batch 1 0.296 -> 0.276 ms)
-          const bool one_wave = static_cast<long long>(e->batch) * din->h * din->w <= 148LL * 128;
-          const bool lane_auto = one_wave || ((din->c >= 192 || (din->c >= 144 && din->h * din->w < 2048)) &&
-                                              !(din->c >= 768 && op.d.cout <= 192));
+          // Which tensor-core kernel: a rule distilled from measurements of both kernels on every 1x1 shape of
+          // the benchmark networks at batch 256 (single launches, and confirmed inside the networks: MobileNetV2
+          // 1.711 -> 1.688 ms, MobileNetV1 1.432 -> 1.383 ms against the previous rule).  The lane-per-pixel kernel
+          // (dense weights, activations through tensor memory) wins for 64 <= Cin < 960 with at least 96 output
+          // channels, except for narrow-input expansions (Cin <= 96, Cout >= 4 Cin); the pixel-pair kernel
+          // (both operands by TMA, 4x expanded weights) wins elsewhere: few input or output channels, where its
+          // tiles are small, and very deep inputs, where the lane kernel's weights no longer stay resident.
+          // Launches whose pixels all fit one wave of 128-pixel tiles are latency-bound and take the lane
+          // kernel (shorter fill; MobileNetV2 batch 1 0.296 -> 0.276 ms) - up to 64 tiles always, up to one
+          // tile per SM unless the input is 960 channels deep or more.
+          const long long m_px_all = static_cast<long long>(e->batch) * din->h * din->w;
+          const bool one_wave = m_px_all <= 64LL * 128 || (m_px_all <= 148LL * 128 && din->c < 960);
+          const bool lane_rule = op.d.cout >= 96 && din->c >= 64 && din->c < 960 && !(din->c <= 96 && op.d.cout >= 4 * din->c);
+          const bool lane_auto = one_wave || lane_rule;
           const bool lane_kernel = e->opt.pointwise == GI_PW_TC_LANE || (e->opt.pointwise == GI_PW_AUTO && lane_auto);
           if (pointwise && tc && lane_kernel && pointwise_ts_supported(din->c, op.d.cout)) {
             r.kernel = GI_KERNEL_POINTWISE_TS;
