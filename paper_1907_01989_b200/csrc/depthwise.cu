@@ -600,20 +600,28 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
   g.in_dead = r.in0_dead;
   g.head_px = (g.W + 3) & ~1;
   // two output columns per thread: stride 1, one padding column, rows of even length (16-byte aligned pixel
-  // pairs), wide planes (measured at batch 256: 112x112x32 0.1055 -> 0.0983 ms, 112x112x96 -6 %; 56x56 and
-  // smaller planes 2-12 % slower than one column per thread, so those keep it)
-  const bool pair = g.stride == 1 && g.dil == 1 && g.pl == 1 && g.pt <= 1 && g.W % 2 == 0 && g.Wo == g.W && g.W >= 96;
+  // pairs), planes at least 56 wide.  Measured at batch 256 against one column per thread: 112x112x32
+  // 0.1055 -> 0.0901 ms, 112x112x96 (batch 128) 0.1393 -> 0.1290 ms, 56x56x144 0.1208 -> 0.1024 ms; 28x28 and
+  // smaller planes are 2-12 % slower that way and keep one column per thread.
+  const bool pair = g.stride == 1 && g.dil == 1 && g.pl == 1 && g.pt <= 1 && g.W % 2 == 0 && g.Wo == g.W && g.W >= 56;
   const int wcols = pair ? g.Wo / 2 : g.Wo;
   // thread groups: as many "virtual planes" (plane x sub-band) as fit in ~256 threads
   int vp = 256 / wcols;
   if (vp < 1) vp = 1;
   g.nb = vp < g.B ? vp : g.B;
-  // (pairs: half of them as sub-bands of one plane rather than further planes - a sub-band shares its halo rows)
-  if (pair && g.nb >= 4 && g.Ho >= 32) g.nb /= 2;
   g.sub = vp / g.nb;
   if (g.sub < 1) g.sub = 1;
-  const int tr_target = g.stride == 1 ? (pair ? 8 : 16) : 8;
+  // rows walked by a thread: 16 (stride 1) or 8; pairs: 14, which divides the usual plane heights - bands of
+  // equal height measured better than taller ones with a short last band (16 rows: 10-20 % slower on 112 / 56)
+  const int tr_target = g.stride == 1 ? (pair ? 14 : 16) : 8;
   int total_sub = (g.Ho + tr_target - 1) / tr_target;
+  if (pair) {
+    // up to four sub-bands of one plane (they share halo rows), two passes of the threads per item; the
+    // staging budget below then decides how many planes go with them (56 rows of 112: one; of 56: two)
+    g.sub = total_sub < 4 ? total_sub : 4;
+    const int planes = 512 / (wcols * g.sub);
+    g.nb = planes < 1 ? 1 : planes < g.B ? planes : g.B;
+  }
   if (total_sub < g.sub) g.sub = total_sub;
   g.tr = (g.Ho + total_sub - 1) / total_sub;
   g.bands = (total_sub + g.sub - 1) / g.sub;
