@@ -65,12 +65,15 @@ enum { GI_F16 = 1, GI_F32 = 2 };   /* storage type of activations (and of NHWC i
 enum { GI_NHWC = 0, GI_PHWC4 = 1 }; /* layout of a caller-visible tensor */
 
 enum {
-  GI_OP_CONV2D = 1,           /* full convolution, kernel 1x1 or 3x3 */
-  GI_OP_DEPTHWISE_CONV2D = 2, /* depthwise 3x3, depth multiplier 1 */
-  GI_OP_ADD = 3,              /* element-wise sum of two tensors of the same shape */
+  GI_OP_CONV2D = 1,           /* full convolution, square kernel 1x1, 2x2 or 3x3, stride 1 to 3 (the sizes and
+                                 strides of the search space in Section 4, "Work Group: Choosing the Right Size") */
+  GI_OP_DEPTHWISE_CONV2D = 2, /* depthwise 3x3, stride 1 or 2, depth multiplier 1 */
+  GI_OP_ADD = 3,              /* element-wise sum of two tensors of the same shape; with inputs[1] = -1 the identity */
   GI_OP_ACTIVATION = 4,       /* ReLU or ReLU6 */
   GI_OP_GLOBAL_AVG_POOL = 5,  /* mean over H*W */
-  GI_OP_RESIZE_BILINEAR = 6   /* bilinear up/down-sampling */
+  GI_OP_RESIZE_BILINEAR = 6,  /* bilinear up/down-sampling */
+  GI_OP_CONCAT = 7            /* channel concatenation of two tensors of the same height and width: channels of
+                                 inputs[0], then those of inputs[1]; with inputs[1] = -1 the identity */
 };
 
 enum { GI_ACT_NONE = 0, GI_ACT_RELU = 1, GI_ACT_RELU6 = 2 };
@@ -116,7 +119,8 @@ enum {
  * weights: host pointer, [cout][kh][kw][cin] for CONV2D, [1][kh][kw][c] for DEPTHWISE_CONV2D,
  * of type weight_dtype (GI_F32 or GI_F16); bias: host pointer to cout floats or NULL.  Both
  * are copied by gi_add_op; the caller may free them as soon as it returns.
- * Unused fields must be zero.  inputs[1] is used by GI_OP_ADD only (else -1 or 0).
+ * Unused fields must be zero.  inputs[1] is used by GI_OP_ADD and GI_OP_CONCAT only (elsewhere -1 or 0); there -1
+ * means "no second input": the operator is then an identity, which gi_compile removes (Section 3.1).
  */
 typedef struct gi_op_desc {
   int32_t kind;
@@ -180,7 +184,8 @@ enum {
   GI_KERNEL_PACK = 1, GI_KERNEL_UNPACK = 2, GI_KERNEL_CONV_SIMT = 3, GI_KERNEL_POINTWISE_TC = 4,
   GI_KERNEL_DEPTHWISE = 5, GI_KERNEL_ELTWISE = 6, GI_KERNEL_POOL = 7, GI_KERNEL_RESIZE = 8, GI_KERNEL_CONV3X3_TC = 9, GI_KERNEL_POINTWISE_TS = 10,
   GI_KERNEL_DEPTHWISE_POINTWISE = 11, /* this op and the next one, as one kernel */
-  GI_KERNEL_NONE = 12                 /* no launch: the op ran inside the previous op's kernel */
+  GI_KERNEL_NONE = 12,                /* no launch: the op ran inside the previous op's kernel */
+  GI_KERNEL_CONCAT = 13
 };
 
 /* ---- graph construction (Section 3.1, "Initialization": the sub-graph given to the GPU backend) ---- */

@@ -6,7 +6,7 @@ import it, and it imports nothing from them.
 
   ops.c / ops.py  operator definitions (fp32 storage, double accumulation), PHWC4
                   indexing, fp16 rounding
-  compile.py      fusion pass, tensor lifetimes, size formula and the three memory
+  compile.py      graph clean-up, fusion pass, tensor lifetimes, size formula and the memory
                   planners, each written step by step from its defining text
   graph.py        evaluates a graph description (unfused or fused) with the operators
 """

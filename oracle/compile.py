@@ -55,8 +55,8 @@ def fuse(g, enable: bool = True, fold_add: bool = True) -> List[FusedOp]:
     fused op takes the add.  The folded op's output replaces x as F's output.
 
     First the graph is cleaned (Section 3.1, "Graph transformation"): a superfluous identity operator -
-    here a resize to the size its input already has - is removed and what read its output reads its
-    input; it stays if its output is a graph output.
+    a resize to the size its input already has, or an ADD / CONCAT with a single input - is removed and
+    what read its output reads its input; it stays if its output is a graph output.
     """
     alias: Dict[int, int] = {}
 
@@ -66,8 +66,9 @@ def fuse(g, enable: bool = True, fold_add: bool = True) -> List[FusedOp]:
     dropped = set()
     uses: Dict[int, int] = {}
     for idx, op in enumerate(g.ops):
-        if (op.kind == "resize_bilinear" and tuple(g.shapes[op.output][:2]) == tuple(g.shapes[op.inputs[0]][:2])
-                and op.output not in set(g.outputs)):
+        identity = ((op.kind == "resize_bilinear" and tuple(g.shapes[op.output][:2]) == tuple(g.shapes[op.inputs[0]][:2]))
+                    or (op.kind in ("add", "concat") and len(op.inputs) == 1))
+        if identity and op.output not in set(g.outputs):
             alias[op.output] = src(op.inputs[0])
             dropped.add(idx)
             continue
@@ -99,7 +100,7 @@ def fuse(g, enable: bool = True, fold_add: bool = True) -> List[FusedOp]:
                 fused[i].output = op.output
                 producer[op.output] = i
                 continue
-        if enable and fold_add and op.kind == "add":
+        if enable and fold_add and op.kind == "add" and len(ins) == 2:
             a, b = ins
             if a != b and g.shapes[a] == g.shapes[b]:
                 candidates = []

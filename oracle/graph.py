@@ -29,8 +29,12 @@ def _leading(op, x: Sequence[np.ndarray], f16: bool) -> np.ndarray:
         return fn(x[0], w, op.bias, op.stride, op.dilation, op.pads)
     if k == "activation":
         return ops.activation(x[0], op.act)
+    if k in ("add", "concat") and len(x) == 1:
+        return ops.activation(x[0], "none")  # a single-input ADD / CONCAT is the identity
     if k == "add":
         return ops.add(x[0], x[1])
+    if k == "concat":
+        return ops.concat(x[0], x[1])
     if k == "global_avg_pool":
         return ops.global_avg_pool(x[0])
     if k == "resize_bilinear":

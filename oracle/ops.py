@@ -104,6 +104,18 @@ def add(a, b):
     return out
 
 
+def concat(a, b):
+    """Channel concatenation (Section 3.1 lists CONCAT among the operators): out[..., :Ca] = a, out[..., Ca:] = b."""
+    a, b = _c(a), _c(b)
+    assert a.shape[:3] == b.shape[:3]
+    out = np.empty(a.shape[:3] + (a.shape[3] + b.shape[3],), dtype=np.float32)
+    for c in range(a.shape[3]):
+        out[..., c] = a[..., c]
+    for c in range(b.shape[3]):
+        out[..., a.shape[3] + c] = b[..., c]
+    return out
+
+
 def global_avg_pool(x):
     x = _c(x)
     B, H, W, Cc = x.shape

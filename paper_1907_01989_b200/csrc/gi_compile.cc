@@ -13,6 +13,8 @@
 namespace gi {
 
 static bool is_conv(int kind) { return kind == GI_OP_CONV2D || kind == GI_OP_DEPTHWISE_CONV2D; }
+// ADD and CONCAT read inputs[1] unless it is -1 (a single-input ADD / CONCAT is the identity)
+static bool two_inputs(const OpNode& op) { return (op.d.kind == GI_OP_ADD || op.d.kind == GI_OP_CONCAT) && op.d.inputs[1] >= 0; }
 
 // The folded chain must be a sub-sequence of [activation][add][activation].
 // `what`: 0 = activation, 1 = add.  Returns the pattern position it would occupy, or -1.
@@ -29,9 +31,9 @@ static int next_slot(int slot, int what) {
 // no other use and is not a graph output, and the chain stays inside [act][add][act]; the
 // other operand of a folded ADD must already exist when the convolution runs.
 //
-// Before that, the graph is cleaned as in Section 3.1: a superfluous identity operator - here a RESIZE whose
-// output has the size of its input - is dropped and its readers read its input instead (unless its output is
-// a graph output, which has to exist as a tensor of its own).
+// Before that, the graph is cleaned as in Section 3.1: a superfluous identity operator - a RESIZE whose
+// output has the size of its input, an ADD or CONCAT with a single input - is dropped and its readers read
+// its input instead (unless its output is a graph output, which has to exist as a tensor of its own).
 gi_status fuse_graph(const gi_graph& g, bool enable, std::vector<FusedOp>* out) {
   const int nt = static_cast<int>(g.tensors.size());
   std::vector<int> alias(nt);  // tensor -> the tensor that holds its values
@@ -43,18 +45,20 @@ gi_status fuse_graph(const gi_graph& g, bool enable, std::vector<FusedOp>* out) 
     // insertion order must be topological: every input id is smaller than the output id
     for (int k = 0; k < 2; ++k) {
       const int t = op.d.inputs[k];
-      if (k == 1 && op.d.kind != GI_OP_ADD) continue;
+      if (k == 1 && !two_inputs(op)) continue;
       if (t < 0 || t >= op.output) return fail(GI_E_INVALID, "gi_compile: operator reads a tensor defined after it");
     }
     const int in0 = op.d.inputs[0];
-    if (op.d.kind == GI_OP_RESIZE_BILINEAR && g.tensors[op.output].h == g.tensors[in0].h &&
-        g.tensors[op.output].w == g.tensors[in0].w && g.tensors[op.output].output_index < 0) {
+    const bool same_size_resize = op.d.kind == GI_OP_RESIZE_BILINEAR && g.tensors[op.output].h == g.tensors[in0].h &&
+                                  g.tensors[op.output].w == g.tensors[in0].w;
+    const bool single_input = (op.d.kind == GI_OP_ADD || op.d.kind == GI_OP_CONCAT) && !two_inputs(op);
+    if ((same_size_resize || single_input) && g.tensors[op.output].output_index < 0) {
       alias[op.output] = alias[in0];
       dropped[idx] = 1;
       continue;
     }
     ++uses[alias[in0]];
-    if (op.d.kind == GI_OP_ADD) ++uses[alias[op.d.inputs[1]]];
+    if (two_inputs(op)) ++uses[alias[op.d.inputs[1]]];
   }
   std::vector<FusedOp>& fused = *out;
   fused.clear();
@@ -70,7 +74,7 @@ gi_status fuse_graph(const gi_graph& g, bool enable, std::vector<FusedOp>* out) 
   for (size_t idx = 0; idx < g.ops.size(); ++idx) {
     const OpNode& op = g.ops[idx];
     if (dropped[idx]) continue;
-    const int in_a = alias[op.d.inputs[0]], in_b = op.d.kind == GI_OP_ADD ? alias[op.d.inputs[1]] : -1;
+    const int in_a = alias[op.d.inputs[0]], in_b = two_inputs(op) ? alias[op.d.inputs[1]] : -1;
     if (enable && op.d.kind == GI_OP_ACTIVATION) {
       const int i = foldable(in_a);
       const int pos = i >= 0 ? next_slot(fused[i].slot, 0) : -1;
@@ -84,7 +88,7 @@ gi_status fuse_graph(const gi_graph& g, bool enable, std::vector<FusedOp>* out) 
         continue;
       }
     }
-    if (enable && op.d.kind == GI_OP_ADD) {
+    if (enable && op.d.kind == GI_OP_ADD && in_b >= 0) {
       const int a = in_a, b = in_b;
       if (a != b) {
         int best = -1, best_x = -1, best_other = -1;

@@ -144,12 +144,12 @@ gi_status gi_add_op(gi_graph* g, const gi_op_desc* desc, gi_tensor* out) {
     case GI_OP_CONV2D:
     case GI_OP_DEPTHWISE_CONV2D: {
       const bool dwise = desc->kind == GI_OP_DEPTHWISE_CONV2D;
-      if (desc->kh != desc->kw || (desc->kh != 1 && desc->kh != 3) || (dwise && desc->kh != 3))
-        return fail(GI_E_UNSUPPORTED, "gi_add_op: kernel must be 1x1 or 3x3 (depthwise: 3x3)");
+      if (desc->kh != desc->kw || desc->kh < 1 || desc->kh > 3 || (dwise && desc->kh != 3))
+        return fail(GI_E_UNSUPPORTED, "gi_add_op: kernel must be 1x1, 2x2 or 3x3 (depthwise: 3x3)");
       if (desc->stride_h < 1 || desc->stride_w < 1 || desc->dilation_h < 1 || desc->dilation_w < 1)
         return fail(GI_E_INVALID, "gi_add_op: stride and dilation must be >= 1");
-      if (desc->stride_h > 2 || desc->stride_w > 2)
-        return fail(GI_E_UNSUPPORTED, "gi_add_op: stride above 2 is not supported");
+      if (desc->stride_h > (dwise ? 2 : 3) || desc->stride_w > (dwise ? 2 : 3))
+        return fail(GI_E_UNSUPPORTED, "gi_add_op: stride above 3 (depthwise: above 2) is not supported");
       if (desc->pad_t < 0 || desc->pad_l < 0 || desc->pad_b < 0 || desc->pad_r < 0)
         return fail(GI_E_INVALID, "gi_add_op: negative padding");
       if (!desc->weights) return fail(GI_E_INVALID, "gi_add_op: convolution without weights");
@@ -192,12 +192,25 @@ gi_status gi_add_op(gi_graph* g, const gi_op_desc* desc, gi_tensor* out) {
       break;
     }
     case GI_OP_ADD: {
-      if (!known(desc->inputs[1])) return fail(GI_E_INVALID, "gi_add_op: ADD needs two input tensors");
-      const TensorDesc& b = g->tensors[desc->inputs[1]];
-      if (b.h != in.h || b.w != in.w || b.c != in.c) return fail(GI_E_INVALID, "gi_add_op: ADD operands differ in shape");
       o.h = in.h;
       o.w = in.w;
       o.c = in.c;
+      if (desc->inputs[1] == -1) break;  // single input: the identity
+      if (!known(desc->inputs[1])) return fail(GI_E_INVALID, "gi_add_op: ADD: inputs[1] is neither a tensor of this graph nor -1");
+      const TensorDesc& b = g->tensors[desc->inputs[1]];
+      if (b.h != in.h || b.w != in.w || b.c != in.c) return fail(GI_E_INVALID, "gi_add_op: ADD operands differ in shape");
+      break;
+    }
+    case GI_OP_CONCAT: {
+      o.h = in.h;
+      o.w = in.w;
+      o.c = in.c;
+      if (desc->inputs[1] == -1) break;  // single input: the identity
+      if (!known(desc->inputs[1])) return fail(GI_E_INVALID, "gi_add_op: CONCAT: inputs[1] is neither a tensor of this graph nor -1");
+      const TensorDesc& b = g->tensors[desc->inputs[1]];
+      if (b.h != in.h || b.w != in.w) return fail(GI_E_INVALID, "gi_add_op: CONCAT operands differ in height or width");
+      if (static_cast<int64_t>(in.c) + b.c > (1 << 20)) return fail(GI_E_UNSUPPORTED, "gi_add_op: CONCAT: too many channels");
+      o.c = in.c + b.c;
       break;
     }
     case GI_OP_ACTIVATION:
@@ -221,7 +234,7 @@ gi_status gi_add_op(gi_graph* g, const gi_op_desc* desc, gi_tensor* out) {
     default:
       return fail(GI_E_INVALID, "gi_add_op: unknown operator kind");
   }
-  if (desc->kind != GI_OP_ADD) node.d.inputs[1] = -1;
+  if (desc->kind != GI_OP_ADD && desc->kind != GI_OP_CONCAT) node.d.inputs[1] = -1;
   if (static_cast<uint64_t>(o.h) * o.w > (1u << 28)) return fail(GI_E_UNSUPPORTED, "gi_add_op: output plane too large");
   g->tensors.push_back(o);
   node.output = static_cast<int>(g->tensors.size()) - 1;

@@ -261,15 +261,24 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
         }
         break;
       }
+      case GI_OP_CONCAT:
+        if (f.in1 >= 0) {
+          r.kernel = GI_KERNEL_CONCAT;
+          info.bytes = (in_px * (in_c4 + slices(e->tensors[f.in1].c) * 4) + out_px * out_c4) * eb;
+          break;
+        }
+        // a single-input CONCAT that survived the clean-up (its output is a graph output) is a copy
+        [[fallthrough]];
       case GI_OP_ADD:
       case GI_OP_ACTIVATION: {
         r.kernel = GI_KERNEL_ELTWISE;
         const OpNode& op = g.ops[f.graph_op];
         if (f.kind == GI_OP_ACTIVATION) r.ep.act_pre = op.d.act;
         info.act_pre = r.ep.act_pre;
-        r.ep.has_res = f.kind == GI_OP_ADD;
-        info.bytes = (in_px * in_c4 * (f.kind == GI_OP_ADD ? 2 : 1) + out_px * out_c4) * eb;
-        info.flops = out_px * dout->c;
+        const bool sum = f.kind == GI_OP_ADD && f.in1 >= 0;
+        r.ep.has_res = sum;
+        info.bytes = (in_px * in_c4 * (sum ? 2 : 1) + out_px * out_c4) * eb;
+        info.flops = f.kind == GI_OP_CONCAT || (f.kind == GI_OP_ADD && !sum) ? 0 : out_px * dout->c;
         break;
       }
       case GI_OP_GLOBAL_AVG_POOL:

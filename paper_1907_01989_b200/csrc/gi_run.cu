@@ -108,6 +108,7 @@ static gi_status run_impl(gi_exec* e, const void* const* dev_inputs, void* const
         if (r.ep.has_res && !p.in1) p.in1 = p.res;
         err = launch_eltwise(r, p, e->storage, stream);
         break;
+      case GI_KERNEL_CONCAT: err = launch_concat(r, p, e->storage, stream); break;
       case GI_KERNEL_POOL: err = launch_pool(r, p, e->storage, stream); break;
       case GI_KERNEL_RESIZE: err = launch_resize(r, p, e->storage, stream); break;
       default: return fail(GI_E_INVALID, "gi_run: corrupt launch table");

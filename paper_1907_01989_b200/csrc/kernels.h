@@ -34,6 +34,7 @@ int launch_depthwise(const LaunchRec& r, const Ptrs& p, int storage, void* strea
 int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream);
 unsigned int depthwise_error_word(int* cuda_err);
 int launch_eltwise(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
+int launch_concat(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
 int launch_pool(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
 int launch_resize(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
 

@@ -1,5 +1,5 @@
-// CUDA-core kernels: layout conversion, depthwise 3x3, direct convolution, element-wise,
-// global average pool, bilinear resize.  All work on the channel-sliced layout
+// CUDA-core kernels: layout conversion, depthwise 3x3, direct convolution, element-wise, channel
+// concatenation, global average pool, bilinear resize.  All work on the channel-sliced layout
 //   element (b,h,w,c) -> ((c/4 * B + b) * P + h*W + w) * 4 + c%4,   P = H*W rounded up to even,
 // and move one pixel-slice (4 channels: 8 bytes fp16, 16 bytes fp32) per vector access, so a
 // warp touches 32 consecutive pixels of one plane = one contiguous 256 / 512-byte run.
@@ -281,6 +281,44 @@ __global__ void eltwise_kernel(const T* __restrict__ a, const T* __restrict__ b,
   Px<T>::store(out + i * 4, v);
 }
 
+// ------------------------------------------------------------------ channel concatenation
+// grid: x over the pixels of all planes of one output slice (B * P), y over output slices.  Output channel c
+// is channel c of `a` for c < Ca and channel c - Ca of `b` after that; lanes beyond Ca + Cb and the padding
+// pixel of a plane are written as zeros.  With Ca a multiple of 4 every output slice is one whole input
+// slice (one vector load); otherwise each lane is fetched from the slice that holds it.
+template <typename T>
+__global__ void concat_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restrict__ out, size_t n_px, int P, int HW,
+                              int Ca, int Cb) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x;
+  if (i >= n_px) return;
+  const int so = blockIdx.y, c0 = so * 4;
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (static_cast<int>(i % P) < HW) {
+    if ((Ca & 3) == 0) {
+      const bool from_a = c0 < Ca;
+      const T* src = from_a ? a + (static_cast<size_t>(so) * n_px + i) * 4 : b + (static_cast<size_t>(so - Ca / 4) * n_px + i) * 4;
+      v = Px<T>::load(src);
+      const int valid = (from_a ? Ca : Ca + Cb) - c0;  // channels of this slice that exist
+      if (valid < 4) v.w = 0.f;
+      if (valid < 3) v.z = 0.f;
+      if (valid < 2) v.y = 0.f;
+    } else {
+      float lane[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int c = c0 + j;
+        lane[j] = 0.f;
+        if (c < Ca) lane[j] = Px<T>::get(a + (static_cast<size_t>(c >> 2) * n_px + i) * 4 + (c & 3));
+        else if (c < Ca + Cb) lane[j] = Px<T>::get(b + (static_cast<size_t>((c - Ca) >> 2) * n_px + i) * 4 + ((c - Ca) & 3));
+      }
+      v = make_float4(lane[0], lane[1], lane[2], lane[3]);
+    }
+  }
+  Px<T>::store(out + (static_cast<size_t>(so) * n_px + i) * 4, v);
+}
+
 // ------------------------------------------------------------------ global average pool
 // eight lanes per (slice, image), four planes per warp: a lane strides over the pixels with all its
 // loads independent (many small planes are latency-bound otherwise), then a shuffle reduction over
@@ -513,6 +551,20 @@ int launch_eltwise(const LaunchRec& r, const Ptrs& p, int storage, void* stream)
                 (launch_pdl(eltwise_kernel<float>, blocks_for(n_px, 256), 256, 0, st, static_cast<const float*>(p.in0),
                                                                               static_cast<const float*>(p.in1),
                                                                               static_cast<float*>(p.out), n_px, r.ep)));
+  return static_cast<int>(cudaGetLastError());
+}
+
+int launch_concat(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int P = plane_pixels(r.Ho, r.Wo), sout = slices(r.Co);
+  const size_t n_px = static_cast<size_t>(r.B) * P;
+  if (sout > 65535) return static_cast<int>(cudaErrorInvalidConfiguration);
+  const dim3 grid(blocks_for(n_px, 256), sout);
+  const int Ca = r.C, Cb = r.Co - r.C;
+  GI_BY_STORAGE((launch_pdl(concat_kernel<__half>, grid, 256, 0, st, static_cast<const __half*>(p.in0), static_cast<const __half*>(p.in1),
+                            static_cast<__half*>(p.out), n_px, P, r.Ho * r.Wo, Ca, Cb)),
+                (launch_pdl(concat_kernel<float>, grid, 256, 0, st, static_cast<const float*>(p.in0), static_cast<const float*>(p.in1),
+                            static_cast<float*>(p.out), n_px, P, r.Ho * r.Wo, Ca, Cb)));
   return static_cast<int>(cudaGetLastError());
 }
 

@@ -27,6 +27,7 @@ ADD = "add"
 ACTIVATION = "activation"
 GLOBAL_AVG_POOL = "global_avg_pool"
 RESIZE_BILINEAR = "resize_bilinear"
+CONCAT = "concat"
 
 ACT_NONE, ACT_RELU, ACT_RELU6 = "none", "relu", "relu6"
 
@@ -135,6 +136,20 @@ class GraphBuilder:
     def add(self, a: int, b: int) -> int:
         out = self._new(*self.g.shapes[a])
         self.g.ops.append(OpSpec(kind=ADD, inputs=[a, b], output=out))
+        return out
+
+    def concat(self, a: int, b: Optional[int] = None) -> int:
+        """Channels of `a`, then channels of `b`; with one input the identity."""
+        H, W, Ca = self.g.shapes[a]
+        Cb = 0 if b is None else self.g.shapes[b][2]
+        out = self._new(H, W, Ca + Cb)
+        self.g.ops.append(OpSpec(kind=CONCAT, inputs=[a] if b is None else [a, b], output=out))
+        return out
+
+    def identity_add(self, x: int) -> int:
+        """An ADD with a single input: the identity (graph clean-up removes it)."""
+        out = self._new(*self.g.shapes[x])
+        self.g.ops.append(OpSpec(kind=ADD, inputs=[x], output=out))
         return out
 
     def global_avg_pool(self, x: int) -> int:
@@ -308,6 +323,57 @@ def depthwise_then_pointwise(batch: int, h: int, w: int, c: int, cout: int, stri
         y = b.add(r, y)
     if post_act is not None:
         y = b.activation(y, post_act)
+    b.output(y)
+    return b.finish()
+
+
+# ----------------------------------------------------------------------------------------
+# Workload 10: a network of "fire" modules - squeeze 1x1, then a 1x1 and a 3x3 expansion whose outputs are
+# concatenated - with a 2x2 stride-2 stem and a 3x3 stride-3 reduction: the operators and the kernel sizes /
+# strides (1x1, 2x2, 3x3; 1 to 3) that the MobileNets do not use.  Channel counts are chosen so that one
+# concatenation joins whole 4-channel slices and the others do not.
+# ----------------------------------------------------------------------------------------
+def _fire(b: GraphBuilder, x: int, squeeze: int, e1: int, e3: int) -> int:
+    s = b.activation(b.conv2d(x, squeeze, 1), ACT_RELU)
+    left = b.activation(b.conv2d(s, e1, 1), ACT_RELU)
+    right = b.activation(b.conv2d(s, e3, 3), ACT_RELU)
+    return b.concat(left, right)
+
+
+def fire_network(batch: int = 1, size: int = 96, classes: int = 10) -> GraphSpec:
+    b = GraphBuilder("fire_network", batch, 10)
+    x = b.input(size, size, 3)
+    y = b.activation(b.conv2d(x, 24, 2, 2), ACT_RELU)
+    y = _fire(b, y, 8, 16, 16)
+    y = _fire(b, y, 8, 18, 14)
+    y = b.activation(b.conv2d(y, 48, 3, 3), ACT_RELU)
+    y = _fire(b, y, 12, 23, 25)
+    y = b.concat(y)
+    skip = y
+    y = _fire(b, y, 12, 24, 24)
+    y = b.add(skip, y)
+    y = b.identity_add(y)
+    y = b.activation(b.conv2d(y, 64, 2, 1), ACT_RELU6)
+    y = b.global_avg_pool(y)
+    y = b.conv2d(y, classes, 1)
+    b.output(y)
+    return b.finish()
+
+
+def single_concat(batch: int, h: int, w: int, ca: int, cb: int) -> GraphSpec:
+    b = GraphBuilder(f"concat_{batch}x{h}x{w}x{ca}+{cb}", batch, 11)
+    x = b.input(h, w, ca)
+    y = b.input(h, w, cb)
+    b.output(b.concat(x, y))
+    return b.finish()
+
+
+def single_conv(batch: int, h: int, w: int, cin: int, cout: int, k: int, stride: int, act: str = ACT_RELU) -> GraphSpec:
+    b = GraphBuilder(f"conv{k}_{batch}x{h}x{w}x{cin}x{cout}_s{stride}", batch, 12)
+    x = b.input(h, w, cin)
+    y = b.conv2d(x, cout, k, stride)
+    if act != ACT_NONE:
+        y = b.activation(y, act)
     b.output(y)
     return b.finish()
 

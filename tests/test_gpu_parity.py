@@ -387,7 +387,7 @@ def _random_spec(rnd, n_ops):
     live = [b.input(rnd.choice([5, 8, 9, 16]), rnd.choice([4, 7, 8, 18]), rnd.choice([3, 4, 6, 8, 20]))]
     for _ in range(n_ops):
         x = rnd.choice(live[-4:])
-        kind = rnd.choice(["conv1", "conv1", "conv3", "dw", "dw", "act", "add", "pool", "resize"])
+        kind = rnd.choice(["conv1", "conv1", "conv3", "dw", "dw", "act", "add", "pool", "resize", "conv2", "concat", "concat", "ident"])
         H, W, Cc = b.g.shapes[x]
         if kind == "conv1":
             y = b.conv2d(x, rnd.choice([4, 6, 8, 24, Cc]), 1)
@@ -400,6 +400,13 @@ def _random_spec(rnd, n_ops):
         elif kind == "add":
             same = [t for t in live if b.g.shapes[t] == b.g.shapes[x]]
             y = b.add(rnd.choice(same), x)
+        elif kind == "conv2":
+            y = b.conv2d(x, rnd.choice([4, 5, 8, 24]), rnd.choice([2, 3]), rnd.choice([1, 2, 3]))
+        elif kind == "concat":
+            same = [t for t in live if b.g.shapes[t][:2] == b.g.shapes[x][:2]]
+            y = b.concat(rnd.choice(same), x)
+        elif kind == "ident":
+            y = b.identity_add(x) if rnd.random() < 0.5 else b.concat(x)
         elif kind == "pool":
             if H * W == 1:
                 continue
@@ -417,7 +424,7 @@ def _random_spec(rnd, n_ops):
     return b.finish()
 
 
-@pytest.mark.parametrize("seed", range(16))
+@pytest.mark.parametrize("seed", range(24))
 def test_random_graphs(seed):
     """Every stored tensor of a random graph against the oracle, fp16 (tensor-core kernels) and fp32, fused."""
     import random
@@ -447,3 +454,88 @@ def test_identity_resize_removed():
     for storage in STORAGES:
         check_all_tensors(spec, storage)
         check_outputs(spec, storage)
+
+
+# ---------------------------------------------------------------------- second workload: CONCAT, 2x2 kernels, stride 3
+CONCAT_CASES = [  # batch, H, W, Ca, Cb: whole slices, ragged first input, ragged second input, odd planes, one channel each
+    (2, 8, 8, 8, 8), (3, 7, 5, 4, 6), (2, 9, 9, 6, 8), (1, 5, 3, 3, 3), (4, 1, 1, 1, 1), (2, 14, 14, 96, 32), (1, 33, 31, 5, 11),
+    (2, 6, 6, 7, 1), (300, 3, 3, 2, 9),
+]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("storage", STORAGES)
+@pytest.mark.parametrize("case", CONCAT_CASES)
+def test_concat_bit_exact(storage, case):
+    """CONCAT moves values without arithmetic: the result is the oracle's, bit for bit, and lanes beyond the last
+    channel and the padding pixel of an odd plane are zero in memory."""
+    spec = wl.single_concat(*case)
+    xs = [wl.make_input(spec, index=i) for i in range(2)]
+    ref = og.run(spec, xs, storage=SNAME[storage])[spec.outputs[0]]
+    run = DeviceRun(spec, storage, guard_bytes=4096)
+    got = run.run(xs)[spec.outputs[0]]
+    assert run.guard_intact()
+    assert np.array_equal(got, ref)
+    assert "concat" in [api.KERNEL_NAMES[o.kernel] for o in run.ex.ops()]
+    # the stored PHWC4 tensor (the unpack kernel reads it from the arena): padding is zero
+    t = spec.outputs[0]
+    B, H, W, Cc = (case[0], case[1], case[2], case[3] + case[4])
+    S, P = (Cc + 3) // 4, (H * W + 1) // 2 * 2
+    raw = run.fetch_raw(t)[: S * B * P * 4].reshape(S, B, P, 4).astype(np.float32)
+    assert not raw[:, :, H * W:, :].any()
+    if Cc % 4:
+        assert not raw[S - 1, :, :, Cc % 4:].any()
+    assert api.gi_device_status() == 0
+
+
+CONV_K_S_CASES = [  # batch, H, W, Cin, Cout, k, stride
+    (2, 8, 8, 3, 8, 2, 1), (2, 9, 7, 5, 6, 2, 2), (1, 16, 16, 8, 24, 2, 3), (3, 10, 11, 4, 5, 3, 3), (2, 7, 7, 6, 4, 1, 3),
+    (1, 96, 96, 3, 24, 2, 2), (2, 24, 24, 32, 48, 3, 3), (2, 5, 5, 12, 40, 2, 1), (1, 1, 1, 4, 4, 2, 3),
+]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("storage", STORAGES)
+@pytest.mark.parametrize("case", CONV_K_S_CASES)
+def test_conv_2x2_and_stride_3(storage, case):
+    """Kernel sizes and strides of the paper's search space that the MobileNets do not use (Section 4)."""
+    spec = wl.single_conv(*case)
+    check_all_tensors(spec, storage)
+    check_all_tensors(spec, storage, fuse=False)
+    assert api.gi_device_status() == 0
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("storage", STORAGES)
+def test_fire_network_every_tensor(storage):
+    for spec in (wl.fire_network(2), wl.fire_network(3, size=77)):
+        check_all_tensors(spec, storage)
+        for planner in (api.GI_PLAN_GREEDY_BY_SIZE, api.GI_PLAN_GREEDY_SHARED_OBJECTS, api.GI_PLAN_MIN_COST_FLOW):
+            check_outputs(spec, storage, planner=planner)
+    check_all_tensors(wl.fire_network(2), storage, fuse=False)
+    assert api.gi_device_status() == 0
+
+
+@pytest.mark.gpu
+def test_fire_network_batch64_sampled_images():
+    spec = wl.fire_network(64, size=192)
+    check_outputs(spec, api.GI_F16, images=[0, 31, 63])
+    assert api.gi_device_status() == 0
+
+
+@pytest.mark.gpu
+def test_single_input_add_and_concat():
+    """Removed at compile time unless they are graph outputs, where they run as copies (Section 3.1)."""
+    b = wl.GraphBuilder("ident_gpu", 3, 22)
+    x = b.input(7, 5, 6)
+    y = b.activation(b.conv2d(x, 10, 1), wl.ACT_RELU)
+    z = b.concat(b.identity_add(y))
+    out1 = b.activation(b.conv2d(z, 6, 3), wl.ACT_RELU6)
+    b.output(b.concat(out1))
+    b.output(b.identity_add(out1))
+    spec = b.finish()
+    for storage in STORAGES:
+        run, xs, outs = check_outputs(spec, storage)
+        names = [api.KERNEL_NAMES[o.kernel] for o in run.ex.ops()]
+        assert names.count("eltwise") == 2 and "concat" not in names
+        check_all_tensors(spec, storage)

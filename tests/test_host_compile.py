@@ -16,7 +16,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 KIND_NAME = {api.GI_OP_CONV2D: "conv2d", api.GI_OP_DEPTHWISE_CONV2D: "depthwise_conv2d", api.GI_OP_ADD: "add",
              api.GI_OP_ACTIVATION: "activation", api.GI_OP_GLOBAL_AVG_POOL: "global_avg_pool",
-             api.GI_OP_RESIZE_BILINEAR: "resize_bilinear"}
+             api.GI_OP_RESIZE_BILINEAR: "resize_bilinear", api.GI_OP_CONCAT: "concat"}
 ACT_NAME = {api.GI_ACT_NONE: None, api.GI_ACT_RELU: "relu", api.GI_ACT_RELU6: "relu6"}
 
 
@@ -120,7 +120,8 @@ def compare_with_oracle(spec, planner, fuse=True, storage=api.GI_F16, align=256)
 PLANNERS = [api.GI_PLAN_GREEDY_BY_SIZE, api.GI_PLAN_GREEDY_SHARED_OBJECTS, api.GI_PLAN_NAIVE, api.GI_PLAN_MIN_COST_FLOW]
 NETS = [lambda: wl.separable_block(1), lambda: wl.mobilenet_v1(1), lambda: wl.mobilenet_v2(1),
         lambda: wl.mobilenet_v2_segmentation(1), lambda: wl.mobilenet_v2(256), lambda: wl.mobilenet_v2_segmentation(16),
-        lambda: wl.single_pointwise(8, 14, 96, 576, residual=True), lambda: wl.single_depthwise(8, 7, 96, 2)]
+        lambda: wl.single_pointwise(8, 14, 96, 576, residual=True), lambda: wl.single_depthwise(8, 7, 96, 2),
+        lambda: wl.fire_network(4), lambda: wl.single_concat(3, 5, 5, 6, 7)]
 
 
 @pytest.mark.parametrize("planner", PLANNERS)
@@ -138,7 +139,7 @@ def random_spec(rnd: random.Random, n_ops: int) -> wl.GraphSpec:
     live = [b.input(rnd.choice([5, 8, 9]), rnd.choice([4, 7, 8]), rnd.choice([3, 4, 6, 8]))]
     for _ in range(n_ops):
         x = rnd.choice(live[-4:])
-        kind = rnd.choice(["conv1", "conv3", "dw", "act", "act", "add", "add", "pool"])
+        kind = rnd.choice(["conv1", "conv3", "dw", "act", "act", "add", "add", "pool", "conv2", "concat", "concat", "ident"])
         H, W, Cc = b.g.shapes[x]
         if kind == "conv1":
             y = b.conv2d(x, rnd.choice([4, 6, 8, Cc]), 1)
@@ -151,6 +152,13 @@ def random_spec(rnd: random.Random, n_ops: int) -> wl.GraphSpec:
         elif kind == "add":
             same = [t for t in live if b.g.shapes[t] == b.g.shapes[x]]
             y = b.add(rnd.choice(same), x)
+        elif kind == "conv2":
+            y = b.conv2d(x, rnd.choice([4, 5, 8]), rnd.choice([2, 3]), rnd.choice([1, 2, 3]))
+        elif kind == "concat":
+            same = [t for t in live if b.g.shapes[t][:2] == b.g.shapes[x][:2]]
+            y = b.concat(rnd.choice(same), x)
+        elif kind == "ident":
+            y = b.identity_add(x) if rnd.random() < 0.5 else b.concat(x)
         else:
             if H * W == 1:
                 continue
@@ -225,8 +233,18 @@ def test_error_paths():
     with pytest.raises(api.GiError):
         g.add_op(_conv_desc(x, weights=w.ctypes.data, stride_h=0))
     with pytest.raises(api.GiError) as ei:
-        g.add_op(_conv_desc(x, weights=w.ctypes.data, stride_h=3, stride_w=3))
+        g.add_op(_conv_desc(x, weights=w.ctypes.data, stride_h=4, stride_w=4))
     assert ei.value.status == api.GI_E_UNSUPPORTED
+    d = _conv_desc(x, k=3, weights=w.ctypes.data, stride_h=3, stride_w=3)
+    d.kind = api.GI_OP_DEPTHWISE_CONV2D
+    with pytest.raises(api.GiError) as ei:
+        g.add_op(d)  # depthwise: stride 3 has no kernel
+    assert ei.value.status == api.GI_E_UNSUPPORTED
+    d = api.gi_op_desc()
+    d.kind = api.GI_OP_CONCAT
+    d.inputs[0], d.inputs[1] = x, 17  # unknown second tensor
+    with pytest.raises(api.GiError):
+        g.add_op(d)
     y = g.add_op(_conv_desc(x, cout=8, weights=w.ctypes.data))
     d = api.gi_op_desc()
     d.kind = api.GI_OP_ADD

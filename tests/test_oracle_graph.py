@@ -34,8 +34,12 @@ def np_eval(g, x):
             y = np.maximum(a, 0.0)
             if op.act == "relu6":
                 y = np.minimum(y, 6.0)
+        elif op.kind in ("add", "concat") and len(op.inputs) == 1:
+            y = a
         elif op.kind == "add":
             y = a + val[op.inputs[1]]
+        elif op.kind == "concat":
+            y = np.concatenate([a, val[op.inputs[1]]], axis=3)
         elif op.kind == "global_avg_pool":
             y = a.mean(axis=(1, 2), keepdims=True)
         elif op.kind == "resize_bilinear":
@@ -62,6 +66,8 @@ NETS = [
     ("mobilenet_v1", lambda: wl.mobilenet_v1(1, size=96)),
     ("mobilenet_v2", lambda: wl.mobilenet_v2(1, size=96)),
     ("segmentation", lambda: wl.mobilenet_v2_segmentation(1, size=65)),
+    ("fire_network", lambda: wl.fire_network(2)),
+    ("fire_network_odd", lambda: wl.fire_network(1, size=77)),
 ]
 
 
@@ -71,7 +77,9 @@ def test_oracle_matches_float64_numpy_on_every_tensor(name, make):
     x = wl.make_input(g)
     ref = np_eval(g, x)
     got = og.run(g, [x], storage="f32", fused=False, keep_all=True)
-    assert set(got) == set(ref)
+    # the only tensors the oracle does not compute are the outputs of the identity operators its clean-up removes
+    removed = {op.output for op in g.ops if op.kind in ("add", "concat") and len(op.inputs) == 1 and op.output not in g.outputs}
+    assert set(ref) - set(got) == removed and set(got) <= set(ref)
     for t in got:
         scale = max(1.0, float(np.abs(ref[t]).max()))
         np.testing.assert_allclose(got[t], ref[t], rtol=0, atol=2e-5 * scale, err_msg=f"{name} tensor {t}")
@@ -154,3 +162,42 @@ def test_resize_to_the_same_size_is_the_identity_and_removing_it_changes_nothing
         ya = og.run(ga, xs, storage=storage)[ga.outputs[0]]
         yb = og.run(gb, xs, storage=storage)[gb.outputs[0]]
         assert np.array_equal(ya, yb)
+
+
+def test_concat_then_1x1_convolution_is_the_sum_of_the_convolutions_of_the_parts():
+    """Pins the channel order of CONCAT: a 1x1 convolution of concat(a, b) with weights [Wa | Wb] equals the
+    convolution of a with Wa plus that of b with Wb (bias counted once)."""
+    r = np.random.default_rng(5)
+    from oracle import ops
+    a = r.standard_normal((2, 5, 3, 6)).astype(np.float32)
+    b = r.standard_normal((2, 5, 3, 5)).astype(np.float32)
+    w = r.standard_normal((7, 1, 1, 11)).astype(np.float32)
+    bias = r.standard_normal(7).astype(np.float32)
+    whole = ops.conv2d(ops.concat(a, b), w, bias)
+    parts = (ops.conv2d(a, np.ascontiguousarray(w[..., :6]), bias).astype(np.float64)
+             + ops.conv2d(b, np.ascontiguousarray(w[..., 6:]), None).astype(np.float64))
+    np.testing.assert_allclose(whole, parts, rtol=0, atol=1e-5)
+    # and the values themselves: channel c of the result is channel c of a, then channel c - 6 of b
+    y = ops.concat(a, b)
+    assert y.shape == (2, 5, 3, 11)
+    assert np.array_equal(y[1, 4, 2], np.array(list(a[1, 4, 2]) + list(b[1, 4, 2]), dtype=np.float32))
+    swapped = ops.concat(b, a)
+    assert not np.array_equal(swapped, y) and np.array_equal(swapped[..., 5:], a)
+
+
+def test_single_input_add_and_concat_are_identities_and_removing_them_changes_nothing():
+    b = wl.GraphBuilder("ident", 2, 77)
+    x = b.input(6, 5, 7)
+    y = b.activation(b.conv2d(x, 10, 1), wl.ACT_RELU)
+    z = b.concat(b.identity_add(y))
+    out1 = b.activation(b.conv2d(z, 6, 3), wl.ACT_RELU6)
+    kept = b.concat(out1)  # a graph output: stays, as a copy
+    b.output(kept)
+    g = b.finish()
+    fused = oc.fuse(g)
+    assert [f.kind for f in fused] == ["conv2d", "conv2d", "concat"]
+    assert fused[1].inputs == [fused[0].output] and fused[2].inputs == [out1]
+    xin = wl.make_input(g)
+    a = og.run(g, [xin], storage="f32", fused=True)[kept]
+    ref = np_eval(g, xin)[kept]
+    np.testing.assert_allclose(a, ref, rtol=0, atol=2e-5)

@@ -47,6 +47,10 @@ CONV_CASES = [
     (6, 7, 5, 3, 1, (1, 1), (1, 1), (0, 0, 0, 0)),
     (8, 8, 1, 2, 3, (2, 1), (1, 2), (1, 2, 0, 2)),
     (4, 4, 3, 2, 2, (1, 1), (1, 1), (0, 0, 1, 1)),
+    (9, 7, 3, 2, 2, (2, 2), (1, 1), (0, 0, 1, 1)),
+    (10, 11, 2, 3, 3, (3, 3), (1, 1), (1, 0, 0, 1)),
+    (8, 8, 2, 2, 2, (3, 3), (1, 1), (0, 0, 0, 0)),
+    (7, 9, 4, 5, 1, (3, 2), (1, 1), (0, 0, 0, 0)),
 ]
 
 
