@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the fused-CNN inference path: MobileNetV2-224, fp16 storage, batch 256 per GPU.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--net v2|v1|seg] [--batch B]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--net v2|v1|seg|fire] [--batch B]
 
 One step = one gi_run of the whole network (layout conversion in, 54 fused ops, layout
 conversion out) on a batch of synthetic images.  Prints ONE JSON line on rank 0.
@@ -38,7 +38,7 @@ if ROOT not in sys.path:
 import numpy as np  # noqa: E402
 
 NETS = {"v2": ("mobilenet_v2", "MobileNetV2-224"), "v1": ("mobilenet_v1", "MobileNetV1-224"),
-        "seg": ("mobilenet_v2_segmentation", "MobileNetV2-513-OS16-seg")}
+        "seg": ("mobilenet_v2_segmentation", "MobileNetV2-513-OS16-seg"), "fire": ("fire_network", "fire-module-network-96")}
 PW_MODES = {"auto": 0, "simt": 1, "pair": 2, "lane": 3}
 XOP_MODES = {"auto": 0, "off": 1, "on": 2}
 # dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes, from the ncu captures summarised

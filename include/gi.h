@@ -87,7 +87,7 @@ enum {
                                         objects laid out in creation order; O(N^4) in the number of tensors */
 };
 
-/* Kernel choice for full convolutions (1x1, and 3x3 with at most 4 input channels). */
+/* Kernel choice for full convolutions. */
 enum {
   GI_PW_AUTO = 0,      /* tensor-core kernels for fp16 storage, CUDA-core kernel for fp32 storage */
   GI_PW_SIMT = 1,      /* force the plain CUDA-core kernel for every full convolution (validation) */
@@ -185,7 +185,8 @@ enum {
   GI_KERNEL_DEPTHWISE = 5, GI_KERNEL_ELTWISE = 6, GI_KERNEL_POOL = 7, GI_KERNEL_RESIZE = 8, GI_KERNEL_CONV3X3_TC = 9, GI_KERNEL_POINTWISE_TS = 10,
   GI_KERNEL_DEPTHWISE_POINTWISE = 11, /* this op and the next one, as one kernel */
   GI_KERNEL_NONE = 12,                /* no launch: the op ran inside the previous op's kernel */
-  GI_KERNEL_CONCAT = 13
+  GI_KERNEL_CONCAT = 13,
+  GI_KERNEL_CONV_TC = 14              /* k x k convolution, any number of input channels, on the tensor cores */
 };
 
 /* ---- graph construction (Section 3.1, "Initialization": the sub-graph given to the GPU backend) ---- */
@@ -275,7 +276,7 @@ GI_API gi_status gi_run_timed(gi_exec* e, const void* const* dev_inputs, void* c
 /* Health word of the device-side waits.  The tensor-core kernel waits on copy and MMA
  * completion with a limit of about one second per wait; a wait that runs out sets a bit here
  * (1 producer, 2 MMA issuer, 4 epilogue, 8 drain; 0x10000 depthwise staging copy;
- * 0x200000 / 0x400000 MMA issuer / epilogue of the 3x3 tensor-core kernel; 0x1000000..0x8000000
+ * 0x100000 / 0x200000 / 0x400000 gather / MMA issuer / epilogue of the k x k tensor-core kernels; 0x1000000..0x8000000
  * producer / MMA issuer / data warps / drain of the lane-per-pixel 1x1 kernel; 0x10000000..
  * 0x80000000 copy warp / MMA issuer / compute warps / drain of the depthwise + pointwise kernel), lets the
  * kernel finish without its results

@@ -1,0 +1,419 @@
+// Full k x k convolution (k = 1, 2, 3; any stride, dilation and padding) of a tensor with any number of
+// channels as an implicit GEMM on the tensor cores (Section 4, "For a 2D Convolution": each output iterates
+// over the window and the input slices under it - here window and slices are unrolled into the K axis).
+//
+//   D[pixel][co] = sum_k A[pixel][k] * B[co][k],   k = (tap * S_in + slice) * 4 + channel-in-slice
+//
+// The K axis is walked in chunks of 16 pixel-slices (64 values, four tcgen05.mma of K = 16).  A tile of 128
+// output pixels is one TMEM lane per pixel.  The 128 gather threads read the chunk's 8-byte pixel-slices of
+// their pixel from the channel-sliced input (zero outside the image; consecutive pixels of a row are
+// consecutive in memory, so a warp's loads coalesce) and write them, two per 16-byte unit, straight into the
+// canonical K-major shared-memory operand layout; the weights sit in shared memory for the whole kernel.
+// Operand buffers are double-buffered against the MMAs (a buffer is handed back by tcgen05.commit), the
+// accumulators against the epilogue: the gather of tile i+1 runs while the MMAs of tile i finish, and the
+// same 128 threads then drain tile i (bias, fused element-wise tail, 8 bytes per output slice).  Waits are
+// bounded like in the other tensor-core kernels.  The 3 x 3 kernel for a single input slice (the stem of the
+// MobileNets) is the special case with one chunk and no hand-back; it keeps its own file.
+#include <cuda.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include "kernels.h"
+#include "pdl.cuh"
+#include "sm100_ptx.cuh"
+
+namespace gi {
+namespace {
+
+using namespace ptx;
+
+constexpr int kRows = 128;             // output pixels per tile
+constexpr int kUnits = 16;             // pixel-slices (4 channels each) per K chunk
+constexpr int kKCores = kUnits / 2;    // 16-byte K units per row and chunk
+constexpr int kABytes = kKCores * kRows * 16;
+constexpr int kGatherThreads = 128;
+constexpr int kThreads = kGatherThreads + 32;
+constexpr int kMaxN = 256;
+constexpr int kHeaderBytes = 1024;
+constexpr int kMaxWeightBytes = 150 * 1024;
+
+__device__ unsigned int g_conv_kxk_error = 0;
+
+struct ConvParams {
+  const __half* in;
+  const __half* res;
+  __half* out;
+  const unsigned char* wts;  // [n_chunks * 8][n_pad][8] fp16
+  const float* bias;         // [n_pad]
+  int B, H, W, Pin, Ho, Wo, Pout;
+  int k, s_in, stride, dil, pt, pl;
+  int n_chunks;              // ceil(k * k * s_in / 16)
+  int s_out, n_pad;          // output slices; Cout rounded up to a multiple of 16
+  int tiles;                 // ceil(B * Pout / 128)
+  int step_b, step_q;        // gridDim.x * 128 pixels = step_b planes + step_q pixels
+  unsigned m_total;          // B * Pout (< 2^31)
+  int has_res, act_post;
+  unsigned tmem_cols;
+  unsigned timeout_ns;
+};
+
+struct Header {
+  unsigned long long a_full[2];
+  unsigned long long a_empty[2];
+  unsigned long long acc_full[2];
+  unsigned tmem_addr;
+  unsigned abort_flag;
+};
+
+__device__ __forceinline__ float act1(float v, int kind) {
+  if (kind == GI_ACT_RELU) return fmaxf(v, 0.0f);
+  if (kind == GI_ACT_RELU6) return fminf(fmaxf(v, 0.0f), 6.0f);
+  return v;
+}
+
+// ACT: activation right after the bias; TAIL: a residual add and / or a second activation follow
+template <int ACT, bool TAIL>
+__global__ void __launch_bounds__(kThreads, 4) conv_kxk_tc_kernel(const ConvParams p) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  Header* hdr = reinterpret_cast<Header*>(smem);
+  unsigned char* a_tiles = smem + kHeaderBytes;         // 2 x kABytes
+  unsigned char* b_tile = a_tiles + 2 * kABytes;        // n_chunks * 8 * n_pad * 16
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile unsigned* abort_flag = &hdr->abort_flag;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&hdr->a_full[i]), kGatherThreads);
+      mbar_init(smem_u32(&hdr->a_empty[i]), 1);
+      mbar_init(smem_u32(&hdr->acc_full[i]), 1);
+    }
+    hdr->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 4) tmem_alloc(smem_u32(&hdr->tmem_addr), p.tmem_cols);
+  // weights: plain copy into shared memory, then made visible to the tensor core's proxy
+  for (int i = threadIdx.x; i < p.n_chunks * kKCores * p.n_pad; i += kThreads)
+    reinterpret_cast<uint4*>(b_tile)[i] = __ldg(reinterpret_cast<const uint4*>(p.wts) + i);
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  // everything above touched only weights and on-chip state; the activations come after the wait
+  pdl_launch_dependents();
+  pdl_wait();
+  const unsigned tmem_base = hdr->tmem_addr;
+  const unsigned n_cols = static_cast<unsigned>(p.n_pad);
+
+  if (warp < 4) {
+    const int t = threadIdx.x;  // row of the tile = TMEM lane
+    const int real_px = p.Ho * p.Wo;
+    const uint2* in8 = reinterpret_cast<const uint2*>(p.in);
+    const long long slice_step = static_cast<long long>(p.B) * p.Pin;  // pixel-slices between two slices of one pixel
+    unsigned it = 0;  // K chunks gathered so far by this CTA
+    // ---- gather of all K chunks of one tile; this thread's pixel is q of image b.  Returns false on a timeout.
+    auto gather_tile = [&](int b, int q, bool in_tensor) -> bool {
+      const bool live = in_tensor && q < real_px;
+      int iy0 = 0, ix0 = 0;
+      if (live) {
+        const int oy = q / p.Wo, ox = q - oy * p.Wo;
+        iy0 = oy * p.stride - p.pt;
+        ix0 = ox * p.stride - p.pl;
+      }
+      // walk of the K axis: slice fastest, then the tap's column, then its row
+      int s = 0, kx = 0, ky = 0;
+      for (int c = 0; c < p.n_chunks; ++c, ++it) {
+        const int buf = static_cast<int>(it & 1u);
+        if (!mbar_wait_warp(smem_u32(&hdr->a_empty[buf]), ((it >> 1) & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_conv_kxk_error, 1u))
+          return false;
+        uint2 unit[kUnits];
+#pragma unroll
+        for (int j = 0; j < kUnits; ++j) {
+          unit[j] = make_uint2(0u, 0u);
+          if (ky < p.k) {
+            const int iy = iy0 + ky * p.dil, ix = ix0 + kx * p.dil;
+            if (live && iy >= 0 && iy < p.H && ix >= 0 && ix < p.W)
+              unit[j] = __ldg(in8 + (static_cast<long long>(s) * slice_step + static_cast<long long>(b) * p.Pin +
+                                     static_cast<long long>(iy) * p.W + ix));
+            if (++s == p.s_in) {
+              s = 0;
+              if (++kx == p.k) {
+                kx = 0;
+                ++ky;
+              }
+            }
+          }
+        }
+        uint4* dst = reinterpret_cast<uint4*>(a_tiles + buf * kABytes) + t;
+#pragma unroll
+        for (int j = 0; j < kKCores; ++j)
+          dst[j * kRows] = make_uint4(unit[2 * j].x, unit[2 * j].y, unit[2 * j + 1].x, unit[2 * j + 1].y);
+        // generic-proxy writes above must be visible to the MMA (async proxy) before the arrival
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(smem_u32(&hdr->a_full[buf]));
+      }
+      return true;
+    };
+    // ---- epilogue of one tile from accumulator `buf`; gp = this thread's pixel in the whole tensor
+    auto epilogue = [&](int buf, unsigned phase, unsigned gp, bool in_tensor, bool real) -> bool {
+      if (!mbar_wait_warp(smem_u32(&hdr->acc_full[buf]), phase, abort_flag, p.timeout_ns, &g_conv_kxk_error, 4u)) return false;
+      tc_fence_after();
+      const unsigned t_addr = tmem_base + buf * n_cols + (static_cast<unsigned>(warp * 32) << 16);
+      auto finish = [&](const unsigned* r, unsigned c0) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int so = static_cast<int>(c0 / 4) + j;
+          if (so >= p.s_out || !in_tensor) continue;
+          const size_t off = (static_cast<size_t>(so) * p.m_total + gp) * 4;  // in halves
+          uint2 o = make_uint2(0u, 0u);  // the padding pixel of an odd plane stays zero
+          if (real) {
+            const float4 bv = __ldg(reinterpret_cast<const float4*>(p.bias) + so);
+            float v[4] = {__uint_as_float(r[4 * j]) + bv.x, __uint_as_float(r[4 * j + 1]) + bv.y,
+                          __uint_as_float(r[4 * j + 2]) + bv.z, __uint_as_float(r[4 * j + 3]) + bv.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) v[e] = act1(v[e], ACT);
+            if (TAIL) {
+              if (p.has_res) {
+                const uint2 qv = __ldg(reinterpret_cast<const uint2*>(p.res + off));
+                const float2 r0 = __half22float2(*reinterpret_cast<const __half2*>(&qv.x));
+                const float2 r1 = __half22float2(*reinterpret_cast<const __half2*>(&qv.y));
+                v[0] += r0.x;
+                v[1] += r0.y;
+                v[2] += r1.x;
+                v[3] += r1.y;
+              }
+#pragma unroll
+              for (int e = 0; e < 4; ++e) v[e] = act1(v[e], p.act_post);
+            }
+            const __half2 h0 = __floats2half2_rn(v[0], v[1]), h1 = __floats2half2_rn(v[2], v[3]);
+            o.x = *reinterpret_cast<const unsigned*>(&h0);
+            o.y = *reinterpret_cast<const unsigned*>(&h1);
+          }
+          *reinterpret_cast<uint2*>(p.out + off) = o;
+        }
+      };
+      // two 16-column reads in flight: the next one is issued before the current one is processed
+      unsigned ra[16], rb[16];
+      tmem_ld16(t_addr, ra);
+      for (unsigned c0 = 0; c0 < n_cols; c0 += 32) {
+        tmem_ld_wait16(ra);
+        if (c0 + 16 < n_cols) tmem_ld16(t_addr + c0 + 16, rb);
+        finish(ra, c0);
+        if (c0 + 16 < n_cols) {
+          tmem_ld_wait16(rb);
+          if (c0 + 32 < n_cols) tmem_ld16(t_addr + c0 + 32, ra);
+          finish(rb, c0 + 16);
+        }
+      }
+      tc_fence_before();
+      return true;
+    };
+
+    // software pipeline over this CTA's tiles: the gather of tile n is issued before the epilogue of tile
+    // n - 1.  The pixel of this thread advances by a fixed number of planes and pixels per step: no
+    // divisions by the plane size in the loop
+    const unsigned gp0 = static_cast<unsigned>(blockIdx.x) * kRows + t;
+    int b = static_cast<int>(gp0 / static_cast<unsigned>(p.Pout));
+    int q = static_cast<int>(gp0 - static_cast<unsigned>(b) * p.Pout);
+    unsigned gp = gp0;
+    const unsigned gp_step = gridDim.x * kRows;
+    int n = 0;
+    bool have_prev = false, prev_in = false, prev_real = false;
+    unsigned prev_gp = 0;
+    for (int tile = blockIdx.x; tile < p.tiles; tile += gridDim.x, ++n) {
+      // accumulator n & 1 was drained by the epilogue of tile n - 2, which these threads ran before
+      // this gather: their arrivals for the first chunk also order the accumulator's reuse
+      const bool in_tensor = gp < p.m_total;
+      if (!gather_tile(b, q, in_tensor)) {
+        have_prev = false;
+        break;
+      }
+      if (have_prev && !epilogue((n - 1) & 1, ((n - 1) >> 1) & 1, prev_gp, prev_in, prev_real)) {
+        have_prev = false;
+        break;
+      }
+      have_prev = true;
+      prev_gp = gp;
+      prev_in = in_tensor;
+      prev_real = in_tensor && q < real_px;
+      gp += gp_step;
+      b += p.step_b;
+      q += p.step_q;
+      if (q >= p.Pout) {
+        q -= p.Pout;
+        ++b;
+      }
+    }
+    if (have_prev) epilogue((n - 1) & 1, ((n - 1) >> 1) & 1, prev_gp, prev_in, prev_real);
+  } else if (lane == 0) {
+    // ---- MMA issuer
+    // instruction descriptor: fp32 accumulator, fp16 A and B, both K-major, M = 128, N = n_pad
+    const unsigned idesc = (1u << 4) | ((n_cols >> 3) << 17) | ((kRows >> 4) << 24);
+    const unsigned b_base = smem_u32(b_tile), b_lbo = n_cols * 16u;
+    unsigned it = 0;
+    int n = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < p.tiles && ok; tile += gridDim.x, ++n) {
+      const unsigned d_tmem = tmem_base + static_cast<unsigned>(n & 1) * n_cols;
+      for (int c = 0; c < p.n_chunks; ++c, ++it) {
+        const int buf = static_cast<int>(it & 1u);
+        if (!mbar_wait(smem_u32(&hdr->a_full[buf]), (it >> 1) & 1u, abort_flag, p.timeout_ns, &g_conv_kxk_error, 2u)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        const unsigned a_base = smem_u32(a_tiles + buf * kABytes);
+        const unsigned bc_base = b_base + static_cast<unsigned>(c) * kKCores * b_lbo;
+#pragma unroll
+        for (int ks = 0; ks < kKCores / 2; ++ks) {
+          const unsigned long long ad = smem_desc(a_base + ks * 2 * kRows * 16, kRows * 16, 128);
+          const unsigned long long bd = smem_desc(bc_base + ks * 2 * b_lbo, b_lbo, 128);
+          umma_f16(d_tmem, ad, bd, idesc, (c > 0 || ks > 0) ? 1u : 0u);
+        }
+        if (c + 1 < p.n_chunks) umma_commit(smem_u32(&hdr->a_empty[buf]));  // the buffer is free once these MMAs have read it
+      }
+      if (ok) {
+        // the last chunk's buffer and the accumulator complete together; the accumulator's barrier, the
+        // one the epilogue waits on, is committed last
+        umma_commit(smem_u32(&hdr->a_empty[(it - 1u) & 1u]));
+        umma_commit(smem_u32(&hdr->acc_full[n & 1]));
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, p.tmem_cols);
+  }
+}
+
+int chunks_of(int k, int cin) { return (k * k * slices(cin) + kUnits - 1) / kUnits; }
+
+}  // namespace
+
+bool conv_kxk_tc_supported(int cin, int cout, int kh, int kw, int sh, int sw, int dh, int dw) {
+  if (kh != kw || kh < 1 || kh > 3 || sh != sw || dh != dw || cout < 1 || cout > kMaxN || cin < 1) return false;
+  const int n_pad = (cout + 15) / 16 * 16;
+  return static_cast<long long>(chunks_of(kh, cin)) * kKCores * n_pad * 16 <= kMaxWeightBytes;
+}
+
+// Weights as the B operand: [n_chunks * 8 K units][n_pad rows][8 halves], k = unit * 8 + e =
+// ((tap * S_in + slice) * 4 + channel-in-slice); entries of channels and units that do not exist are zero.
+void conv_kxk_tc_pack(const float* w, const float* bias, int cin, int cout, int k, std::vector<uint8_t>* blob, LaunchRec* r) {
+  const int n_pad = (cout + 15) / 16 * 16, s_in = slices(cin), taps = k * k;
+  const int cores = chunks_of(k, cin) * kKCores;
+  const size_t wbytes = static_cast<size_t>(cores) * n_pad * 16;
+  const uint64_t woff = round_up_u64(blob->size(), 256);
+  blob->resize(woff + wbytes, 0);
+  const uint64_t boff = round_up_u64(blob->size(), 256);
+  blob->resize(boff + static_cast<size_t>(n_pad) * sizeof(float), 0);
+  uint16_t* wp = reinterpret_cast<uint16_t*>(blob->data() + woff);
+  float* bp = reinterpret_cast<float*>(blob->data() + boff);
+  for (int co = 0; co < cout; ++co) {
+    bp[co] = bias[co];
+    for (int tap = 0; tap < taps; ++tap)
+      for (int ci = 0; ci < cin; ++ci) {
+        const int kk = (tap * s_in + ci / 4) * 4 + ci % 4;
+        wp[(static_cast<size_t>(kk / 8) * n_pad + co) * 8 + kk % 8] = f32_to_f16_rne(w[(static_cast<size_t>(co) * taps + tap) * cin + ci]);
+      }
+  }
+  r->wts = Loc{W_WEIGHTS, 0, woff};
+  r->bias = Loc{W_WEIGHTS, 0, boff};
+  r->wts_bytes = wbytes;
+  r->tc_nt = n_pad;
+}
+
+int launch_conv_kxk_tc(const LaunchRec& r, const Ptrs& p, void* stream) {
+  ConvParams k;
+  k.in = static_cast<const __half*>(p.in0);
+  k.res = static_cast<const __half*>(p.res);
+  k.out = static_cast<__half*>(p.out);
+  k.wts = static_cast<const unsigned char*>(p.wts);
+  k.bias = static_cast<const float*>(p.bias);
+  k.B = r.B;
+  k.H = r.H;
+  k.W = r.W;
+  k.Pin = plane_pixels(r.H, r.W);
+  k.Ho = r.Ho;
+  k.Wo = r.Wo;
+  k.Pout = plane_pixels(r.Ho, r.Wo);
+  k.k = r.kh;
+  k.s_in = slices(r.C);
+  k.stride = r.sh;
+  k.dil = r.dh;
+  k.pt = r.pt;
+  k.pl = r.pl;
+  k.n_chunks = chunks_of(r.kh, r.C);
+  k.s_out = slices(r.Co);
+  k.n_pad = r.tc_nt;
+  const long long m_total = static_cast<long long>(r.B) * k.Pout;
+  const long long tiles = (m_total + kRows - 1) / kRows;
+  // pixel indices are kept in 32 bits inside the kernel, with room for one step past the end
+  if (m_total > (1LL << 30)) return static_cast<int>(cudaErrorInvalidConfiguration);
+  k.tiles = static_cast<int>(tiles);
+  k.m_total = static_cast<unsigned>(m_total);
+  k.has_res = r.ep.has_res;
+  k.act_post = r.ep.act_post;
+  unsigned cols = 32;
+  while (cols < static_cast<unsigned>(2 * k.n_pad)) cols <<= 1;
+  k.tmem_cols = cols;
+  k.timeout_ns = 1000000000u;
+  static bool attr_set_dev[kMaxDevices] = {};
+  bool& attr_set = attr_set_dev[current_device_slot()];
+  const int sms = device_sm_count();
+  const size_t smem = kHeaderBytes + 2 * kABytes + static_cast<size_t>(k.n_chunks) * kKCores * k.n_pad * 16;
+  if (!attr_set) {
+    cudaError_t e = cudaSuccess;
+    const int bytes = kHeaderBytes + 2 * kABytes + kMaxWeightBytes;
+#define GI_CK_ATTR(A, T) \
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(conv_kxk_tc_kernel<A, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)
+    GI_CK_ATTR(GI_ACT_NONE, false);
+    GI_CK_ATTR(GI_ACT_RELU, false);
+    GI_CK_ATTR(GI_ACT_RELU6, false);
+    GI_CK_ATTR(GI_ACT_NONE, true);
+    GI_CK_ATTR(GI_ACT_RELU, true);
+    GI_CK_ATTR(GI_ACT_RELU6, true);
+#undef GI_CK_ATTR
+    if (e != cudaSuccess) return static_cast<int>(e);
+    attr_set = true;
+  }
+  // a few CTAs per SM: one CTA's gather latency hides behind another's epilogue; tensor memory allows
+  // 512 / tmem_cols of them, shared memory 227 KB / smem, the register file four
+  int per_sm = static_cast<int>(512u / cols);
+  const int by_smem = static_cast<int>((227 * 1024) / (smem + 1024));
+  if (per_sm > by_smem) per_sm = by_smem;
+  if (per_sm > 4) per_sm = 4;
+  if (per_sm < 1) per_sm = 1;
+  long long grid = static_cast<long long>(sms) * per_sm;
+  if (grid > tiles) grid = tiles;
+  const long long step = grid * kRows;
+  k.step_b = static_cast<int>(step / k.Pout);
+  k.step_q = static_cast<int>(step % k.Pout);
+  const unsigned g = static_cast<unsigned>(grid);
+  cudaStream_t cu_stream = static_cast<cudaStream_t>(stream);
+  const int act = r.ep.act_pre;
+  const bool tail = k.has_res || k.act_post != GI_ACT_NONE;
+#define GI_CK_LAUNCH(A, T) launch_pdl(conv_kxk_tc_kernel<A, T>, g, kThreads, smem, cu_stream, k)
+  if (tail) {
+    if (act == GI_ACT_RELU6) GI_CK_LAUNCH(GI_ACT_RELU6, true);
+    else if (act == GI_ACT_RELU) GI_CK_LAUNCH(GI_ACT_RELU, true);
+    else GI_CK_LAUNCH(GI_ACT_NONE, true);
+  } else {
+    if (act == GI_ACT_RELU6) GI_CK_LAUNCH(GI_ACT_RELU6, false);
+    else if (act == GI_ACT_RELU) GI_CK_LAUNCH(GI_ACT_RELU, false);
+    else GI_CK_LAUNCH(GI_ACT_NONE, false);
+  }
+#undef GI_CK_LAUNCH
+  return static_cast<int>(cudaGetLastError());
+}
+
+unsigned int conv_kxk_tc_error_word(int* cuda_err) {
+  unsigned int v = 0;
+  const cudaError_t e = cudaMemcpyFromSymbol(&v, g_conv_kxk_error, sizeof v);
+  if (cuda_err) *cuda_err = static_cast<int>(e);
+  return v;
+}
+
+}  // namespace gi

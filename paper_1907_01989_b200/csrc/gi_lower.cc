@@ -249,6 +249,11 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
                                           op.d.dilation_h, op.d.dilation_w)) {
             r.kernel = GI_KERNEL_CONV3X3_TC;
             conv3x3_tc_pack(op.weights.data(), op.bias.data(), din->c, op.d.cout, &e->weight_blob, &r);
+          } else if (tc && conv_kxk_tc_supported(din->c, op.d.cout, op.d.kh, op.d.kw, op.d.stride_h, op.d.stride_w,
+                                                  op.d.dilation_h, op.d.dilation_w)) {
+            // any other 1x1 (strided or padded), 2x2 or 3x3 convolution whose weights fit shared memory
+            r.kernel = GI_KERNEL_CONV_TC;
+            conv_kxk_tc_pack(op.weights.data(), op.bias.data(), din->c, op.d.cout, op.d.kh, &e->weight_blob, &r);
           } else {
             r.kernel = GI_KERNEL_CONV_SIMT;
             const int sout = slices(op.d.cout);

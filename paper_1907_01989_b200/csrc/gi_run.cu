@@ -108,6 +108,7 @@ static gi_status run_impl(gi_exec* e, const void* const* dev_inputs, void* const
         if (r.ep.has_res && !p.in1) p.in1 = p.res;
         err = launch_eltwise(r, p, e->storage, stream);
         break;
+      case GI_KERNEL_CONV_TC: err = launch_conv_kxk_tc(r, p, stream); break;
       case GI_KERNEL_CONCAT: err = launch_concat(r, p, e->storage, stream); break;
       case GI_KERNEL_POOL: err = launch_pool(r, p, e->storage, stream); break;
       case GI_KERNEL_RESIZE: err = launch_resize(r, p, e->storage, stream); break;
@@ -128,6 +129,7 @@ gi_status gi_device_status(uint32_t* flags) {
   *flags = pointwise_tc_error_word(&err);
   if (err == 0) *flags |= depthwise_error_word(&err) << 16;
   if (err == 0) *flags |= conv3x3_tc_error_word(&err) << 20;
+  if (err == 0) *flags |= conv_kxk_tc_error_word(&err) << 20;
   if (err == 0) *flags |= pointwise_ts_error_word(&err) << 24;
   if (err == 0) *flags |= depthwise_pointwise_error_word(&err) << 28;
   if (err != 0) return fail(GI_E_CUDA, std::string("gi_device_status: ") + cudaGetErrorString(static_cast<cudaError_t>(err)));

@@ -53,6 +53,12 @@ void conv3x3_tc_pack(const float* w, const float* bias, int cin, int cout, std::
 int launch_conv3x3_tc(const LaunchRec& r, const Ptrs& p, void* stream);
 unsigned int conv3x3_tc_error_word(int* cuda_err);
 
+// k x k convolution (k = 1..3) of any number of input channels on the tensor cores (conv_tc.cu)
+bool conv_kxk_tc_supported(int cin, int cout, int kh, int kw, int sh, int sw, int dh, int dw);
+void conv_kxk_tc_pack(const float* w, const float* bias, int cin, int cout, int k, std::vector<uint8_t>* blob, LaunchRec* r);
+int launch_conv_kxk_tc(const LaunchRec& r, const Ptrs& p, void* stream);
+unsigned int conv_kxk_tc_error_word(int* cuda_err);
+
 // Pointwise convolution with the activation operand in tensor memory (fp16 storage).
 bool pointwise_ts_supported(int cin, int cout);
 void pointwise_ts_pack(const float* w, const float* bias, int cin, int cout, std::vector<uint8_t>* blob, LaunchRec* r);

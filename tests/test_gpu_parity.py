@@ -539,3 +539,47 @@ def test_single_input_add_and_concat():
         names = [api.KERNEL_NAMES[o.kernel] for o in run.ex.ops()]
         assert names.count("eltwise") == 2 and "concat" not in names
         check_all_tensors(spec, storage)
+
+
+CONV_TC_CASES = [  # batch, H, W, Cin, Cout, k, stride, dilation, residual, act, post_act
+    (2, 12, 12, 8, 16, 3, 1, 1, False, wl.ACT_RELU, None),        # 5 chunks of 16 pixel-slices, the last one ragged
+    (3, 9, 7, 5, 6, 3, 2, 1, False, wl.ACT_RELU6, None),          # ragged channels both sides, odd planes
+    (2, 24, 24, 48, 64, 3, 1, 1, True, wl.ACT_NONE, wl.ACT_RELU),  # 7 chunks, residual then activation
+    (1, 20, 20, 64, 64, 3, 1, 2, False, wl.ACT_RELU, None),       # dilation 2, 9 chunks
+    (2, 16, 16, 16, 256, 3, 2, 1, False, wl.ACT_RELU6, None),     # all 512 accumulator columns
+    (2, 17, 15, 32, 48, 3, 3, 1, False, wl.ACT_RELU, None),       # stride 3
+    (2, 16, 16, 24, 40, 2, 2, 1, True, wl.ACT_RELU, wl.ACT_RELU6),  # 2x2
+    (4, 14, 14, 96, 24, 1, 2, 1, False, wl.ACT_NONE, None),       # strided 1x1
+    (70, 9, 9, 12, 20, 3, 1, 1, False, wl.ACT_RELU, None),        # many tiles: every CTA walks several
+    (1, 3, 3, 6, 4, 3, 1, 1, False, wl.ACT_NONE, None),           # a single, mostly empty tile
+]
+
+
+@pytest.mark.parametrize("case", CONV_TC_CASES)
+def test_conv_kxk_tensor_core(case):
+    B, H, W, cin, cout, k, stride, dil, residual, act, post = case
+    b = wl.GraphBuilder(f"convtc_{B}x{H}x{W}x{cin}x{cout}_k{k}s{stride}d{dil}", B, 13)
+    x = b.input(H, W, cin)
+    r = b.input(wl.same_pads(H, k, stride, dil)[0], wl.same_pads(W, k, stride, dil)[0], cout) if residual else None
+    y = b.conv2d(x, cout, k, stride, dil)
+    if act != wl.ACT_NONE:
+        y = b.activation(y, act)
+    if residual:
+        y = b.add(r, y)
+    if post is not None:
+        y = b.activation(y, post)
+    b.output(y)
+    spec = b.finish()
+    run = DeviceRun(spec, api.GI_F16)
+    assert [api.KERNEL_NAMES[o.kernel] for o in run.ex.ops()].count("conv_tc") == 1
+    check_all_tensors(spec, api.GI_F16)
+    check_outputs(spec, api.GI_F16)
+    check_all_tensors(spec, api.GI_F16, pointwise=api.GI_PW_SIMT)  # same graph on the CUDA-core kernel
+    assert api.gi_device_status() == 0
+
+
+def test_conv_kxk_weights_too_large_for_shared_memory_take_the_cuda_core_kernel():
+    spec = wl.single_conv(1, 6, 6, 256, 256, 3, 1)
+    run = DeviceRun(spec, api.GI_F16)
+    assert "conv_simt" in [api.KERNEL_NAMES[o.kernel] for o in run.ex.ops()]
+    check_all_tensors(spec, api.GI_F16)
