@@ -7,8 +7,10 @@
 // The K axis is walked in chunks of 16 pixel-slices (64 values, four tcgen05.mma of K = 16).  A tile of 128
 // output pixels is one TMEM lane per pixel.  The 128 gather threads read the chunk's 8-byte pixel-slices of
 // their pixel from the channel-sliced input (zero outside the image; consecutive pixels of a row are
-// consecutive in memory, so a warp's loads coalesce) and write them, two per 16-byte unit, straight into the
-// canonical K-major shared-memory operand layout; the weights sit in shared memory for the whole kernel.
+// consecutive in memory, so a warp's loads coalesce; where each pixel-slice of the K walk lies relative to the
+// window's first pixel is the same for every pixel and comes from a small table in shared memory) and write
+// them, two per 16-byte unit, straight into the canonical K-major shared-memory operand layout; the weights
+// sit in shared memory for the whole kernel.
 // Operand buffers are double-buffered against the MMAs (a buffer is handed back by tcgen05.commit), the
 // accumulators against the epilogue: the gather of tile i+1 runs while the MMAs of tile i finish, and the
 // same 128 threads then drain tile i (bias, fused element-wise tail, 8 bytes per output slice).  Waits are
@@ -28,9 +30,10 @@ namespace {
 using namespace ptx;
 
 constexpr int kRows = 128;             // output pixels per tile
-constexpr int kUnits = 16;             // pixel-slices (4 channels each) per K chunk
-constexpr int kKCores = kUnits / 2;    // 16-byte K units per row and chunk
-constexpr int kABytes = kKCores * kRows * 16;
+// pixel-slices (4 channels each) per K chunk: 16 (64 values, four MMAs), or 8 for a short K axis, where
+// the smaller operand buffers and register footprint let six CTAs instead of four share an SM (measured:
+// the fire network 0.296 -> 0.284 ms with 8, while 3x3 32 -> 32 and 64 -> 64 lose 8-18 % with 8)
+constexpr int kMaxUnits = 16;
 constexpr int kGatherThreads = 128;
 constexpr int kThreads = kGatherThreads + 32;
 constexpr int kMaxN = 256;
@@ -43,11 +46,12 @@ struct ConvParams {
   const __half* in;
   const __half* res;
   __half* out;
-  const unsigned char* wts;  // [n_chunks * 8][n_pad][8] fp16
+  const unsigned char* wts;  // [n_chunks * UNITS / 2][n_pad][8] fp16
   const float* bias;         // [n_pad]
   int B, H, W, Pin, Ho, Wo, Pout;
   int k, s_in, stride, dil, pt, pl;
-  int n_chunks;              // ceil(k * k * s_in / 16)
+  int slice_step;            // B * Pin: pixel-slices between two slices of one pixel (the whole input is < 2^31 pixel-slices)
+  int n_chunks;              // ceil(k * k * s_in / UNITS)
   int s_out, n_pad;          // output slices; Cout rounded up to a multiple of 16
   int tiles;                 // ceil(B * Pout / 128)
   int step_b, step_q;        // gridDim.x * 128 pixels = step_b planes + step_q pixels
@@ -71,9 +75,13 @@ __device__ __forceinline__ float act1(float v, int kind) {
   return v;
 }
 
-// ACT: activation right after the bias; TAIL: a residual add and / or a second activation follow
-template <int ACT, bool TAIL>
-__global__ void __launch_bounds__(kThreads, 4) conv_kxk_tc_kernel(const ConvParams p) {
+// UNITS: pixel-slices per K chunk; ACT: activation right after the bias; TAIL: a residual add and / or a second
+// activation follow
+template <int UNITS, int ACT, bool TAIL>
+__global__ void __launch_bounds__(kThreads, UNITS == 8 ? 6 : 4) conv_kxk_tc_kernel(const ConvParams p) {
+  constexpr int kUnits = UNITS;
+  constexpr int kKCores = kUnits / 2;  // 16-byte K units per row and chunk
+  constexpr int kABytes = kKCores * kRows * 16;
   extern __shared__ __align__(1024) unsigned char smem[];
   Header* hdr = reinterpret_cast<Header*>(smem);
   unsigned char* a_tiles = smem + kHeaderBytes;         // 2 x kABytes
@@ -94,6 +102,18 @@ __global__ void __launch_bounds__(kThreads, 4) conv_kxk_tc_kernel(const ConvPara
   // weights: plain copy into shared memory, then made visible to the tensor core's proxy
   for (int i = threadIdx.x; i < p.n_chunks * kKCores * p.n_pad; i += kThreads)
     reinterpret_cast<uint4*>(b_tile)[i] = __ldg(reinterpret_cast<const uint4*>(p.wts) + i);
+  // The K walk is the same for every pixel: per pixel-slice of the K axis, its distance (in pixel-slices) from
+  // slice 0 of the window's first pixel, and the tap's row / column offset for the border test.  -1 marks the
+  // padding behind the last pixel-slice.
+  int* unit_off = reinterpret_cast<int*>(b_tile + static_cast<size_t>(p.n_chunks) * kKCores * p.n_pad * 16);
+  int* unit_dyx = unit_off + p.n_chunks * kUnits;
+  for (int u = threadIdx.x; u < p.n_chunks * kUnits; u += kThreads) {
+    const int tap = u / p.s_in, sl = u - tap * p.s_in;
+    const int ky = tap / p.k, kx = tap - ky * p.k;
+    const bool exists = tap < p.k * p.k;
+    unit_off[u] = exists ? sl * p.slice_step + ky * p.dil * p.W + kx * p.dil : -1;
+    unit_dyx[u] = exists ? ((ky * p.dil) << 16) | (kx * p.dil) : 0;
+  }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   tc_fence_before();
   __syncthreads();
@@ -108,7 +128,7 @@ __global__ void __launch_bounds__(kThreads, 4) conv_kxk_tc_kernel(const ConvPara
     const int t = threadIdx.x;  // row of the tile = TMEM lane
     const int real_px = p.Ho * p.Wo;
     const uint2* in8 = reinterpret_cast<const uint2*>(p.in);
-    const long long slice_step = static_cast<long long>(p.B) * p.Pin;  // pixel-slices between two slices of one pixel
+    const int reach = (p.k - 1) * p.dil;  // last tap's row / column offset
     unsigned it = 0;  // K chunks gathered so far by this CTA
     // ---- gather of all K chunks of one tile; this thread's pixel is q of image b.  Returns false on a timeout.
     auto gather_tile = [&](int b, int q, bool in_tensor) -> bool {
@@ -119,27 +139,35 @@ __global__ void __launch_bounds__(kThreads, 4) conv_kxk_tc_kernel(const ConvPara
         iy0 = oy * p.stride - p.pt;
         ix0 = ox * p.stride - p.pl;
       }
-      // walk of the K axis: slice fastest, then the tap's column, then its row
-      int s = 0, kx = 0, ky = 0;
+      // slice 0 of the window's first pixel (outside the tensor for border pixels: only dereferenced where valid)
+      const uint2* base = in8 + (static_cast<long long>(b) * p.Pin + static_cast<long long>(iy0) * p.W + ix0);
+      // all but the border pixels have their whole window inside the image: no per-tap tests
+      const bool inside = live && iy0 >= 0 && ix0 >= 0 && iy0 + reach < p.H && ix0 + reach < p.W;
       for (int c = 0; c < p.n_chunks; ++c, ++it) {
         const int buf = static_cast<int>(it & 1u);
         if (!mbar_wait_warp(smem_u32(&hdr->a_empty[buf]), ((it >> 1) & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_conv_kxk_error, 1u))
           return false;
         uint2 unit[kUnits];
+        const int4* off4 = reinterpret_cast<const int4*>(unit_off + c * kUnits);
+        if (inside) {
 #pragma unroll
-        for (int j = 0; j < kUnits; ++j) {
-          unit[j] = make_uint2(0u, 0u);
-          if (ky < p.k) {
-            const int iy = iy0 + ky * p.dil, ix = ix0 + kx * p.dil;
-            if (live && iy >= 0 && iy < p.H && ix >= 0 && ix < p.W)
-              unit[j] = __ldg(in8 + (static_cast<long long>(s) * slice_step + static_cast<long long>(b) * p.Pin +
-                                     static_cast<long long>(iy) * p.W + ix));
-            if (++s == p.s_in) {
-              s = 0;
-              if (++kx == p.k) {
-                kx = 0;
-                ++ky;
-              }
+          for (int j4 = 0; j4 < kUnits / 4; ++j4) {
+            const int4 o = off4[j4];
+            const int of[4] = {o.x, o.y, o.z, o.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) unit[4 * j4 + e] = of[e] >= 0 ? __ldg(base + of[e]) : make_uint2(0u, 0u);
+          }
+        } else {
+          const int4* dyx4 = reinterpret_cast<const int4*>(unit_dyx + c * kUnits);
+#pragma unroll
+          for (int j4 = 0; j4 < kUnits / 4; ++j4) {
+            const int4 o = off4[j4], d = dyx4[j4];
+            const int of[4] = {o.x, o.y, o.z, o.w}, dd[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const unsigned iy = static_cast<unsigned>(iy0 + (dd[e] >> 16)), ix = static_cast<unsigned>(ix0 + (dd[e] & 0xffff));
+              const bool ok = live && of[e] >= 0 && iy < static_cast<unsigned>(p.H) && ix < static_cast<unsigned>(p.W);
+              unit[4 * j4 + e] = ok ? __ldg(base + of[e]) : make_uint2(0u, 0u);
             }
           }
         }
@@ -289,21 +317,24 @@ __global__ void __launch_bounds__(kThreads, 4) conv_kxk_tc_kernel(const ConvPara
   }
 }
 
-int chunks_of(int k, int cin) { return (k * k * slices(cin) + kUnits - 1) / kUnits; }
+int units_of(int k, int cin) { return k * k * slices(cin) <= 32 ? 8 : 16; }
+int chunks_of(int k, int cin) { return (k * k * slices(cin) + units_of(k, cin) - 1) / units_of(k, cin); }
+// 16-byte K units of the whole weight operand
+int cores_of(int k, int cin) { return chunks_of(k, cin) * units_of(k, cin) / 2; }
 
 }  // namespace
 
 bool conv_kxk_tc_supported(int cin, int cout, int kh, int kw, int sh, int sw, int dh, int dw) {
   if (kh != kw || kh < 1 || kh > 3 || sh != sw || dh != dw || cout < 1 || cout > kMaxN || cin < 1) return false;
   const int n_pad = (cout + 15) / 16 * 16;
-  return static_cast<long long>(chunks_of(kh, cin)) * kKCores * n_pad * 16 <= kMaxWeightBytes;
+  return static_cast<long long>(cores_of(kh, cin)) * n_pad * 16 <= kMaxWeightBytes;
 }
 
-// Weights as the B operand: [n_chunks * 8 K units][n_pad rows][8 halves], k = unit * 8 + e =
+// Weights as the B operand: [16-byte K units of all chunks][n_pad rows][8 halves], k = unit * 8 + e =
 // ((tap * S_in + slice) * 4 + channel-in-slice); entries of channels and units that do not exist are zero.
 void conv_kxk_tc_pack(const float* w, const float* bias, int cin, int cout, int k, std::vector<uint8_t>* blob, LaunchRec* r) {
   const int n_pad = (cout + 15) / 16 * 16, s_in = slices(cin), taps = k * k;
-  const int cores = chunks_of(k, cin) * kKCores;
+  const int cores = cores_of(k, cin);
   const size_t wbytes = static_cast<size_t>(cores) * n_pad * 16;
   const uint64_t woff = round_up_u64(blob->size(), 256);
   blob->resize(woff + wbytes, 0);
@@ -346,6 +377,9 @@ int launch_conv_kxk_tc(const LaunchRec& r, const Ptrs& p, void* stream) {
   k.pt = r.pt;
   k.pl = r.pl;
   k.n_chunks = chunks_of(r.kh, r.C);
+  // distances inside the input are kept in 32 bits
+  if (static_cast<long long>(k.s_in) * r.B * k.Pin >= (1LL << 31)) return static_cast<int>(cudaErrorInvalidConfiguration);
+  k.slice_step = r.B * k.Pin;
   k.s_out = slices(r.Co);
   k.n_pad = r.tc_nt;
   const long long m_total = static_cast<long long>(r.B) * k.Pout;
@@ -363,12 +397,18 @@ int launch_conv_kxk_tc(const LaunchRec& r, const Ptrs& p, void* stream) {
   static bool attr_set_dev[kMaxDevices] = {};
   bool& attr_set = attr_set_dev[current_device_slot()];
   const int sms = device_sm_count();
-  const size_t smem = kHeaderBytes + 2 * kABytes + static_cast<size_t>(k.n_chunks) * kKCores * k.n_pad * 16;
+  const int units = units_of(r.kh, r.C);
+  const size_t smem = kHeaderBytes + 2 * static_cast<size_t>(units / 2) * kRows * 16 + static_cast<size_t>(cores_of(r.kh, r.C)) * k.n_pad * 16 +
+                      static_cast<size_t>(k.n_chunks) * units * 8;  // + the two per-unit tables
   if (!attr_set) {
     cudaError_t e = cudaSuccess;
-    const int bytes = kHeaderBytes + 2 * kABytes + kMaxWeightBytes;
-#define GI_CK_ATTR(A, T) \
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(conv_kxk_tc_kernel<A, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)
+    // tables: at most 1/16 of the weights (n_pad >= 16)
+    const int bytes = kHeaderBytes + 2 * (kMaxUnits / 2) * kRows * 16 + kMaxWeightBytes + kMaxWeightBytes / 16;
+#define GI_CK_ATTR(A, T)                                                                                                             \
+  do {                                                                                                                               \
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv_kxk_tc_kernel<8, A, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);  \
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv_kxk_tc_kernel<16, A, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes); \
+  } while (0)
     GI_CK_ATTR(GI_ACT_NONE, false);
     GI_CK_ATTR(GI_ACT_RELU, false);
     GI_CK_ATTR(GI_ACT_RELU6, false);
@@ -380,11 +420,11 @@ int launch_conv_kxk_tc(const LaunchRec& r, const Ptrs& p, void* stream) {
     attr_set = true;
   }
   // a few CTAs per SM: one CTA's gather latency hides behind another's epilogue; tensor memory allows
-  // 512 / tmem_cols of them, shared memory 227 KB / smem, the register file four
+  // 512 / tmem_cols of them, shared memory 227 KB / smem, the register file four (six with 8-unit chunks)
   int per_sm = static_cast<int>(512u / cols);
   const int by_smem = static_cast<int>((227 * 1024) / (smem + 1024));
   if (per_sm > by_smem) per_sm = by_smem;
-  if (per_sm > 4) per_sm = 4;
+  if (per_sm > (units == 8 ? 6 : 4)) per_sm = units == 8 ? 6 : 4;
   if (per_sm < 1) per_sm = 1;
   long long grid = static_cast<long long>(sms) * per_sm;
   if (grid > tiles) grid = tiles;
@@ -395,7 +435,11 @@ int launch_conv_kxk_tc(const LaunchRec& r, const Ptrs& p, void* stream) {
   cudaStream_t cu_stream = static_cast<cudaStream_t>(stream);
   const int act = r.ep.act_pre;
   const bool tail = k.has_res || k.act_post != GI_ACT_NONE;
-#define GI_CK_LAUNCH(A, T) launch_pdl(conv_kxk_tc_kernel<A, T>, g, kThreads, smem, cu_stream, k)
+#define GI_CK_LAUNCH(A, T)                                                                      \
+  do {                                                                                          \
+    if (units == 8) launch_pdl(conv_kxk_tc_kernel<8, A, T>, g, kThreads, smem, cu_stream, k);   \
+    else launch_pdl(conv_kxk_tc_kernel<16, A, T>, g, kThreads, smem, cu_stream, k);             \
+  } while (0)
   if (tail) {
     if (act == GI_ACT_RELU6) GI_CK_LAUNCH(GI_ACT_RELU6, true);
     else if (act == GI_ACT_RELU) GI_CK_LAUNCH(GI_ACT_RELU, true);
