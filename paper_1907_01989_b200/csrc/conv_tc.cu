@@ -103,16 +103,16 @@ __global__ void __launch_bounds__(kThreads, UNITS == 8 ? 6 : 4) conv_kxk_tc_kern
   for (int i = threadIdx.x; i < p.n_chunks * kKCores * p.n_pad; i += kThreads)
     reinterpret_cast<uint4*>(b_tile)[i] = __ldg(reinterpret_cast<const uint4*>(p.wts) + i);
   // The K walk is the same for every pixel: per pixel-slice of the K axis, its distance (in pixel-slices) from
-  // slice 0 of the window's first pixel, and the tap's row / column offset for the border test.  -1 marks the
-  // padding behind the last pixel-slice.
+  // slice 0 of the window's first pixel, and the number of its tap (31 for the padding behind the last
+  // pixel-slice: a tap that is never valid).
   int* unit_off = reinterpret_cast<int*>(b_tile + static_cast<size_t>(p.n_chunks) * kKCores * p.n_pad * 16);
-  int* unit_dyx = unit_off + p.n_chunks * kUnits;
+  int* unit_tap = unit_off + p.n_chunks * kUnits;
   for (int u = threadIdx.x; u < p.n_chunks * kUnits; u += kThreads) {
     const int tap = u / p.s_in, sl = u - tap * p.s_in;
     const int ky = tap / p.k, kx = tap - ky * p.k;
     const bool exists = tap < p.k * p.k;
-    unit_off[u] = exists ? sl * p.slice_step + ky * p.dil * p.W + kx * p.dil : -1;
-    unit_dyx[u] = exists ? ((ky * p.dil) << 16) | (kx * p.dil) : 0;
+    unit_off[u] = exists ? sl * p.slice_step + ky * p.dil * p.W + kx * p.dil : 0;
+    unit_tap[u] = exists ? tap : 31;
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   tc_fence_before();
@@ -128,7 +128,6 @@ __global__ void __launch_bounds__(kThreads, UNITS == 8 ? 6 : 4) conv_kxk_tc_kern
     const int t = threadIdx.x;  // row of the tile = TMEM lane
     const int real_px = p.Ho * p.Wo;
     const uint2* in8 = reinterpret_cast<const uint2*>(p.in);
-    const int reach = (p.k - 1) * p.dil;  // last tap's row / column offset
     unsigned it = 0;  // K chunks gathered so far by this CTA
     // ---- gather of all K chunks of one tile; this thread's pixel is q of image b.  Returns false on a timeout.
     auto gather_tile = [&](int b, int q, bool in_tensor) -> bool {
@@ -141,35 +140,29 @@ __global__ void __launch_bounds__(kThreads, UNITS == 8 ? 6 : 4) conv_kxk_tc_kern
       }
       // slice 0 of the window's first pixel (outside the tensor for border pixels: only dereferenced where valid)
       const uint2* base = in8 + (static_cast<long long>(b) * p.Pin + static_cast<long long>(iy0) * p.W + ix0);
-      // all but the border pixels have their whole window inside the image: no per-tap tests
-      const bool inside = live && iy0 >= 0 && ix0 >= 0 && iy0 + reach < p.H && ix0 + reach < p.W;
+      // bit `tap` says whether that tap of this pixel's window lies inside the image: one test per tile and
+      // tap instead of one per gathered pixel-slice, and the same instructions for border and interior pixels
+      unsigned tap_ok = 0;
+      if (live) {
+        for (int ky = 0; ky < p.k; ++ky)
+          for (int kx = 0; kx < p.k; ++kx)
+            if (static_cast<unsigned>(iy0 + ky * p.dil) < static_cast<unsigned>(p.H) &&
+                static_cast<unsigned>(ix0 + kx * p.dil) < static_cast<unsigned>(p.W))
+              tap_ok |= 1u << (ky * p.k + kx);
+      }
       for (int c = 0; c < p.n_chunks; ++c, ++it) {
         const int buf = static_cast<int>(it & 1u);
         if (!mbar_wait_warp(smem_u32(&hdr->a_empty[buf]), ((it >> 1) & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_conv_kxk_error, 1u))
           return false;
         uint2 unit[kUnits];
         const int4* off4 = reinterpret_cast<const int4*>(unit_off + c * kUnits);
-        if (inside) {
+        const int4* tap4 = reinterpret_cast<const int4*>(unit_tap + c * kUnits);
 #pragma unroll
-          for (int j4 = 0; j4 < kUnits / 4; ++j4) {
-            const int4 o = off4[j4];
-            const int of[4] = {o.x, o.y, o.z, o.w};
+        for (int j4 = 0; j4 < kUnits / 4; ++j4) {
+          const int4 o = off4[j4], tp = tap4[j4];
+          const int of[4] = {o.x, o.y, o.z, o.w}, tn[4] = {tp.x, tp.y, tp.z, tp.w};
 #pragma unroll
-            for (int e = 0; e < 4; ++e) unit[4 * j4 + e] = of[e] >= 0 ? __ldg(base + of[e]) : make_uint2(0u, 0u);
-          }
-        } else {
-          const int4* dyx4 = reinterpret_cast<const int4*>(unit_dyx + c * kUnits);
-#pragma unroll
-          for (int j4 = 0; j4 < kUnits / 4; ++j4) {
-            const int4 o = off4[j4], d = dyx4[j4];
-            const int of[4] = {o.x, o.y, o.z, o.w}, dd[4] = {d.x, d.y, d.z, d.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const unsigned iy = static_cast<unsigned>(iy0 + (dd[e] >> 16)), ix = static_cast<unsigned>(ix0 + (dd[e] & 0xffff));
-              const bool ok = live && of[e] >= 0 && iy < static_cast<unsigned>(p.H) && ix < static_cast<unsigned>(p.W);
-              unit[4 * j4 + e] = ok ? __ldg(base + of[e]) : make_uint2(0u, 0u);
-            }
-          }
+          for (int e = 0; e < 4; ++e) unit[4 * j4 + e] = ((tap_ok >> tn[e]) & 1u) ? __ldg(base + of[e]) : make_uint2(0u, 0u);
         }
         uint4* dst = reinterpret_cast<uint4*>(a_tiles + buf * kABytes) + t;
 #pragma unroll
