@@ -147,36 +147,6 @@ __device__ __forceinline__ void umma_f16_ts(unsigned d_tmem, unsigned a_tmem, un
       : "memory");
 }
 
-// Bounded wait whose polls may sleep in hardware for up to a microsecond (they return as soon as the phase
-// completes): for the copy and MMA warps, which wait most of the time and must not take issue slots
-// from the compute warps.
-__device__ __forceinline__ bool mbar_wait_parked(unsigned bar, unsigned parity, volatile unsigned* abort_flag, unsigned timeout_ns,
-                                                 unsigned* error_word, unsigned code) {
-  unsigned long long t0 = 0;
-  for (unsigned spin = 0;; ++spin) {
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity), "r"(1000u)
-        : "memory");
-    if (ok) return true;
-    if ((spin & 15u) == 15u) {
-      if (*abort_flag) return false;
-      const unsigned long long now = global_timer_ns();
-      if (t0 == 0) {
-        t0 = now;
-      } else if (now - t0 > timeout_ns) {
-        *abort_flag = 1;
-        atomicOr(error_word, code);
-        return false;
-      }
-    }
-  }
-}
-
 // MODE 0: stride 1; MODE 1: stride 2 (both: dilation 1, at most one padding row / column on each
 // side).  Staging area of one plane: [head_px zeros][rows of the band][a zero row behind the image
 // when the band reaches its bottom]: the rows above and below the image read as zeros with no test

@@ -57,6 +57,37 @@ static __device__ __noinline__ bool mbar_wait(unsigned bar, unsigned parity, vol
   }
 }
 
+// The same bounded wait for a single thread that waits most of the time (a copy or MMA-issuing thread): each
+// poll may sleep in hardware for up to a microsecond and returns as soon as the phase completes, so the
+// waiting thread takes no issue slots from the warps that compute.  Used where the compute warps are bound by
+// instruction issue (the depthwise + 1x1 kernel); in the other tensor-core kernels it measured 0.3-0.7 %
+// slower than the plain poll on every network, so they keep mbar_wait.
+static __device__ __noinline__ bool mbar_wait_parked(unsigned bar, unsigned parity, volatile unsigned* abort_flag, unsigned timeout_ns,
+                                              unsigned* error_word, unsigned code) {
+  unsigned long long t0 = 0;
+  for (unsigned spin = 0;; ++spin) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(1000u)
+        : "memory");
+    if (ok) return true;
+    if ((spin & 15u) == 15u) {
+      if (*abort_flag) return false;
+      const unsigned long long now = global_timer_ns();
+      if (t0 == 0) {
+        t0 = now;
+      } else if (now - t0 > timeout_ns) {
+        *abort_flag = 1;
+        atomicOr(error_word, code);
+        return false;
+      }
+    }
+  }
+}
 // The same wait for a whole warp that goes on to warp-collective instructions (tcgen05.ld / .st / .wait are
 // .sync.aligned: all 32 lanes must execute them together).  Lanes leave the polling loop at different
 // iterations; the vote brings them back together and gives every lane the same answer, so that the warp
