@@ -46,15 +46,16 @@ struct ConvParams {
   const __half* in;
   const __half* res;
   __half* out;
-  const unsigned char* wts;  // [n_chunks * UNITS / 2][n_pad][8] fp16
-  const float* bias;         // [n_pad]
+  const unsigned char* wts;  // [n_groups][n_chunks * UNITS / 2][n_pad][8] fp16
+  const float* bias;         // [n_groups * n_pad]
   int B, H, W, Pin, Ho, Wo, Pout;
   int k, s_in, stride, dil, pt, pl;
   int slice_step;            // B * Pin: pixel-slices between two slices of one pixel (the whole input is < 2^31 pixel-slices)
   int n_chunks;              // ceil(k * k * s_in / UNITS)
-  int s_out, n_pad;          // output slices; Cout rounded up to a multiple of 16
+  int s_out, n_pad;          // output slices; output channels of one CTA group (a multiple of 16)
+  int n_groups;              // CTA groups over the output channels (weights of one group fit shared memory)
   int tiles;                 // ceil(B * Pout / 128)
-  int step_b, step_q;        // gridDim.x * 128 pixels = step_b planes + step_q pixels
+  int step_b, step_q;        // (gridDim.x / n_groups) * 128 pixels = step_b planes + step_q pixels
   unsigned m_total;          // B * Pout (< 2^31)
   int has_res, act_post;
   unsigned tmem_cols;
@@ -88,6 +89,13 @@ __global__ void __launch_bounds__(kThreads, UNITS == 8 ? 6 : 4) conv_kxk_tc_kern
   unsigned char* b_tile = a_tiles + 2 * kABytes;        // n_chunks * 8 * n_pad * 16
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile unsigned* abort_flag = &hdr->abort_flag;
+  // CTA group g computes output channels [g * n_pad, (g + 1) * n_pad) of every pixel tile it walks; the CTAs of
+  // one group share the tiles among themselves (one group unless the weights exceed shared memory)
+  // (the group's number is recomputed where it is needed rather than kept in a register across the tile loop)
+  const bool one_group = p.n_groups == 1;
+  const int cta = one_group ? static_cast<int>(blockIdx.x) : static_cast<int>(blockIdx.x) / p.n_groups;
+  const int ctas = one_group ? static_cast<int>(gridDim.x) : static_cast<int>(gridDim.x) / p.n_groups;
+  const unsigned char* wts = p.wts + (one_group ? 0 : static_cast<size_t>(blockIdx.x % p.n_groups) * p.n_chunks * kKCores * p.n_pad * 16);
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
@@ -101,7 +109,7 @@ __global__ void __launch_bounds__(kThreads, UNITS == 8 ? 6 : 4) conv_kxk_tc_kern
   if (warp == 4) tmem_alloc(smem_u32(&hdr->tmem_addr), p.tmem_cols);
   // weights: plain copy into shared memory, then made visible to the tensor core's proxy
   for (int i = threadIdx.x; i < p.n_chunks * kKCores * p.n_pad; i += kThreads)
-    reinterpret_cast<uint4*>(b_tile)[i] = __ldg(reinterpret_cast<const uint4*>(p.wts) + i);
+    reinterpret_cast<uint4*>(b_tile)[i] = __ldg(reinterpret_cast<const uint4*>(wts) + i);
   // The K walk is the same for every pixel: per pixel-slice of the K axis, its distance (in pixel-slices) from
   // slice 0 of the window's first pixel, and the number of its tap (31 for the padding behind the last
   // pixel-slice: a tap that is never valid).
@@ -179,15 +187,17 @@ __global__ void __launch_bounds__(kThreads, UNITS == 8 ? 6 : 4) conv_kxk_tc_kern
       if (!mbar_wait_warp(smem_u32(&hdr->acc_full[buf]), phase, abort_flag, p.timeout_ns, &g_conv_kxk_error, 4u)) return false;
       tc_fence_after();
       const unsigned t_addr = tmem_base + buf * n_cols + (static_cast<unsigned>(warp * 32) << 16);
+      const int grp = p.n_groups == 1 ? 0 : static_cast<int>(blockIdx.x) % p.n_groups, so0 = grp * (p.n_pad / 4);
+      const float* bias = p.bias + grp * p.n_pad;
       auto finish = [&](const unsigned* r, unsigned c0) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          const int so = static_cast<int>(c0 / 4) + j;
+          const int sg = static_cast<int>(c0 / 4) + j, so = so0 + sg;  // slice within the group, within the tensor
           if (so >= p.s_out || !in_tensor) continue;
           const size_t off = (static_cast<size_t>(so) * p.m_total + gp) * 4;  // in halves
           uint2 o = make_uint2(0u, 0u);  // the padding pixel of an odd plane stays zero
           if (real) {
-            const float4 bv = __ldg(reinterpret_cast<const float4*>(p.bias) + so);
+            const float4 bv = __ldg(reinterpret_cast<const float4*>(bias) + sg);
             float v[4] = {__uint_as_float(r[4 * j]) + bv.x, __uint_as_float(r[4 * j + 1]) + bv.y,
                           __uint_as_float(r[4 * j + 2]) + bv.z, __uint_as_float(r[4 * j + 3]) + bv.w};
 #pragma unroll
@@ -232,15 +242,15 @@ __global__ void __launch_bounds__(kThreads, UNITS == 8 ? 6 : 4) conv_kxk_tc_kern
     // software pipeline over this CTA's tiles: the gather of tile n is issued before the epilogue of tile
     // n - 1.  The pixel of this thread advances by a fixed number of planes and pixels per step: no
     // divisions by the plane size in the loop
-    const unsigned gp0 = static_cast<unsigned>(blockIdx.x) * kRows + t;
+    const unsigned gp0 = static_cast<unsigned>(cta) * kRows + t;
     int b = static_cast<int>(gp0 / static_cast<unsigned>(p.Pout));
     int q = static_cast<int>(gp0 - static_cast<unsigned>(b) * p.Pout);
     unsigned gp = gp0;
-    const unsigned gp_step = gridDim.x * kRows;
+    const unsigned gp_step = static_cast<unsigned>(ctas) * kRows;
     int n = 0;
     bool have_prev = false, prev_in = false, prev_real = false;
     unsigned prev_gp = 0;
-    for (int tile = blockIdx.x; tile < p.tiles; tile += gridDim.x, ++n) {
+    for (int tile = cta; tile < p.tiles; tile += ctas, ++n) {
       // accumulator n & 1 was drained by the epilogue of tile n - 2, which these threads ran before
       // this gather: their arrivals for the first chunk also order the accumulator's reuse
       const bool in_tensor = gp < p.m_total;
@@ -273,7 +283,7 @@ __global__ void __launch_bounds__(kThreads, UNITS == 8 ? 6 : 4) conv_kxk_tc_kern
     unsigned it = 0;
     int n = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < p.tiles && ok; tile += gridDim.x, ++n) {
+    for (int tile = cta; tile < p.tiles && ok; tile += ctas, ++n) {
       const unsigned d_tmem = tmem_base + static_cast<unsigned>(n & 1) * n_cols;
       for (int c = 0; c < p.n_chunks; ++c, ++it) {
         const int buf = static_cast<int>(it & 1u);
@@ -315,38 +325,58 @@ int chunks_of(int k, int cin) { return (k * k * slices(cin) + units_of(k, cin) -
 // 16-byte K units of the whole weight operand
 int cores_of(int k, int cin) { return chunks_of(k, cin) * units_of(k, cin) / 2; }
 
+// Output channels per CTA group: all of them (rounded up to 16) if their weights fit shared memory, else
+// the largest multiple of 16 whose weights do; 0 if not even 16 output channels fit.
+int group_channels(int k, int cin, int cout) {
+  const int n_pad = (cout + 15) / 16 * 16;
+  const long long per16 = static_cast<long long>(cores_of(k, cin)) * 16 * 16;  // weight bytes of 16 output channels
+  long long fit = kMaxWeightBytes / per16 * 16;
+  if (fit > kMaxN) fit = kMaxN;  // one MMA's N, and two accumulators in tensor memory
+  if (fit < 16) return 0;
+  if (fit >= n_pad) return n_pad;
+  const int groups = static_cast<int>((n_pad + fit - 1) / fit);
+  return ((n_pad / 16 + groups - 1) / groups) * 16;  // even split, rounded up to 16
+}
+
 }  // namespace
 
 bool conv_kxk_tc_supported(int cin, int cout, int kh, int kw, int sh, int sw, int dh, int dw) {
-  if (kh != kw || kh < 1 || kh > 3 || sh != sw || dh != dw || cout < 1 || cout > kMaxN || cin < 1) return false;
-  const int n_pad = (cout + 15) / 16 * 16;
-  return static_cast<long long>(cores_of(kh, cin)) * n_pad * 16 <= kMaxWeightBytes;
+  if (kh != kw || kh < 1 || kh > 3 || sh != sw || dh != dw || cout < 1 || cin < 1) return false;
+  const int ng = group_channels(kh, cin, cout);
+  if (ng == 0) return false;
+  // a group re-gathers the input: beyond eight groups the CUDA-core kernel's single pass is no worse
+  return ((cout + 15) / 16 * 16 + ng - 1) / ng <= 8;
 }
 
-// Weights as the B operand: [16-byte K units of all chunks][n_pad rows][8 halves], k = unit * 8 + e =
-// ((tap * S_in + slice) * 4 + channel-in-slice); entries of channels and units that do not exist are zero.
+// Weights as the B operand, per CTA group: [group][16-byte K units of all chunks][n_pad rows][8 halves],
+// k = unit * 8 + e = ((tap * S_in + slice) * 4 + channel-in-slice); entries of channels and units that do not
+// exist are zero.
 void conv_kxk_tc_pack(const float* w, const float* bias, int cin, int cout, int k, std::vector<uint8_t>* blob, LaunchRec* r) {
-  const int n_pad = (cout + 15) / 16 * 16, s_in = slices(cin), taps = k * k;
+  const int ng = group_channels(k, cin, cout), s_in = slices(cin), taps = k * k;
+  const int groups = ((cout + 15) / 16 * 16 + ng - 1) / ng;
   const int cores = cores_of(k, cin);
-  const size_t wbytes = static_cast<size_t>(cores) * n_pad * 16;
+  const size_t wbytes = static_cast<size_t>(groups) * cores * ng * 16;
   const uint64_t woff = round_up_u64(blob->size(), 256);
   blob->resize(woff + wbytes, 0);
   const uint64_t boff = round_up_u64(blob->size(), 256);
-  blob->resize(boff + static_cast<size_t>(n_pad) * sizeof(float), 0);
+  blob->resize(boff + static_cast<size_t>(groups) * ng * sizeof(float), 0);
   uint16_t* wp = reinterpret_cast<uint16_t*>(blob->data() + woff);
   float* bp = reinterpret_cast<float*>(blob->data() + boff);
   for (int co = 0; co < cout; ++co) {
-    bp[co] = bias[co];
+    bp[co] = bias[co];  // group g's biases start at g * ng: the same index
+    const int g = co / ng, cg = co - g * ng;
     for (int tap = 0; tap < taps; ++tap)
       for (int ci = 0; ci < cin; ++ci) {
         const int kk = (tap * s_in + ci / 4) * 4 + ci % 4;
-        wp[(static_cast<size_t>(kk / 8) * n_pad + co) * 8 + kk % 8] = f32_to_f16_rne(w[(static_cast<size_t>(co) * taps + tap) * cin + ci]);
+        wp[((static_cast<size_t>(g) * cores + kk / 8) * ng + cg) * 8 + kk % 8] =
+            f32_to_f16_rne(w[(static_cast<size_t>(co) * taps + tap) * cin + ci]);
       }
   }
   r->wts = Loc{W_WEIGHTS, 0, woff};
   r->bias = Loc{W_WEIGHTS, 0, boff};
   r->wts_bytes = wbytes;
-  r->tc_nt = n_pad;
+  r->tc_nt = ng;
+  r->tc_kc = groups;
 }
 
 int launch_conv_kxk_tc(const LaunchRec& r, const Ptrs& p, void* stream) {
@@ -375,6 +405,7 @@ int launch_conv_kxk_tc(const LaunchRec& r, const Ptrs& p, void* stream) {
   k.slice_step = r.B * k.Pin;
   k.s_out = slices(r.Co);
   k.n_pad = r.tc_nt;
+  k.n_groups = r.tc_kc;
   const long long m_total = static_cast<long long>(r.B) * k.Pout;
   const long long tiles = (m_total + kRows - 1) / kRows;
   // pixel indices are kept in 32 bits inside the kernel, with room for one step past the end
@@ -419,9 +450,12 @@ int launch_conv_kxk_tc(const LaunchRec& r, const Ptrs& p, void* stream) {
   if (per_sm > by_smem) per_sm = by_smem;
   if (per_sm > (units == 8 ? 6 : 4)) per_sm = units == 8 ? 6 : 4;
   if (per_sm < 1) per_sm = 1;
-  long long grid = static_cast<long long>(sms) * per_sm;
-  if (grid > tiles) grid = tiles;
-  const long long step = grid * kRows;
+  // the grid is a whole number of CTAs per group
+  long long per_group = static_cast<long long>(sms) * per_sm / k.n_groups;
+  if (per_group > tiles) per_group = tiles;
+  if (per_group < 1) per_group = 1;
+  const long long grid = per_group * k.n_groups;
+  const long long step = per_group * kRows;
   k.step_b = static_cast<int>(step / k.Pout);
   k.step_q = static_cast<int>(step % k.Pout);
   const unsigned g = static_cast<unsigned>(grid);

@@ -578,8 +578,19 @@ def test_conv_kxk_tensor_core(case):
     assert api.gi_device_status() == 0
 
 
-def test_conv_kxk_weights_too_large_for_shared_memory_take_the_cuda_core_kernel():
-    spec = wl.single_conv(1, 6, 6, 256, 256, 3, 1)
+@pytest.mark.parametrize("case", [(2, 14, 14, 96, 96, 3, 2), (1, 9, 9, 128, 144, 3, 1), (1, 6, 6, 256, 256, 3, 1), (3, 5, 5, 8, 300, 2, 1)])
+def test_conv_kxk_output_channels_split_over_cta_groups(case):
+    """Weights beyond the shared-memory budget (or more than 256 output channels): each CTA group computes a range
+    of output channels."""
+    spec = wl.single_conv(*case)
+    run = DeviceRun(spec, api.GI_F16)
+    assert "conv_tc" in [api.KERNEL_NAMES[o.kernel] for o in run.ex.ops()]
+    check_all_tensors(spec, api.GI_F16)
+    assert api.gi_device_status() == 0
+
+
+def test_conv_kxk_weights_far_too_large_take_the_cuda_core_kernel():
+    spec = wl.single_conv(1, 4, 4, 512, 512, 3, 1)
     run = DeviceRun(spec, api.GI_F16)
     assert "conv_simt" in [api.KERNEL_NAMES[o.kernel] for o in run.ex.ops()]
     check_all_tensors(spec, api.GI_F16)
