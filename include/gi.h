@@ -160,7 +160,8 @@ typedef struct gi_exec_info {
 typedef struct gi_tensor_info {
   int32_t h, w, c;
   int32_t alive;        /* 0 if fusion removed the tensor */
-  int32_t intermediate; /* 1 if it lives in the arena */
+  int32_t intermediate; /* 1 if it lives in the arena; 2 if it lives inside another arena tensor (an input of a CONCAT
+                           that needs no copy: `offset` then points into that tensor) */
   int32_t first_op, last_op; /* executed-op indices, inclusive; -1 if not alive */
   uint64_t bytes;       /* physical size under the size formula */
   uint64_t offset;      /* arena offset (intermediate tensors only) */
@@ -216,9 +217,13 @@ GI_API void gi_graph_destroy(gi_graph* g);
 /* ---- compile (Sections 3.2 and 5) ---- */
 
 /* Build an executable: verify the order, clean the graph (Section 3.1: an identity operator - a RESIZE to its
- * input's own size - is dropped and its readers read its input, unless its output is a graph output; the
- * dropped op's output tensor is then not alive), fuse, compute lifetimes, plan memory, pack weights,
- * choose a kernel and launch shape per fused op.  Host work only; no CUDA call is made.
+ * input's own size, an ADD or CONCAT with one input - is dropped and its readers read its input, unless its
+ * output is a graph output; the dropped op's output tensor is then not alive), fuse, compute lifetimes, plan
+ * memory, pack weights, choose a kernel and launch shape per fused op.  With `fuse` set, a CONCAT whose first
+ * input has a multiple of 4 channels, and whose inputs and output are neither graph inputs nor outputs, needs
+ * no copy: its inputs are placed inside its output (the slices of a tensor follow one another in memory,
+ * Section 4), their producers write there, and the CONCAT launches nothing (GI_KERNEL_NONE).
+ * Host work only; no CUDA call is made.
  * `opt` may be NULL for defaults.  The graph stays valid and may be compiled again. */
 GI_API gi_status gi_compile(const gi_graph* g, const gi_compile_options* opt, gi_exec** out);
 

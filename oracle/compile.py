@@ -148,19 +148,50 @@ class PlanProblem:
 EXTERNAL_BASE = 1 << 20  # ids of caller-owned NHWC buffers, outside the graph's tensor ids
 
 
+def concat_views(g, fused: Sequence[FusedOp]) -> Dict[int, Tuple[int, int]]:
+    """Concatenations that need no copy.  In the channel-sliced layout (Section 4) the slices of a tensor follow
+    one another, so concat(a, b) with C(a) a multiple of 4 is `a`'s slices followed by `b`'s: if a and b are
+    placed inside the result, their producers write the result directly.  Returns {a: (out, 0), b: (out, S(a))}
+    over all eligible CONCAT ops, walked in execution order.  Eligible: two different inputs, C(a) % 4 == 0,
+    none of a, b, out is a graph input or output, and neither a nor b is already placed inside another tensor
+    or has tensors placed inside it."""
+    views: Dict[int, Tuple[int, int]] = {}
+    roots: Set[int] = set()
+    io = set(g.inputs) | set(g.outputs)
+    for f in fused:
+        if f.kind != "concat" or len(f.inputs) != 2:
+            continue
+        a, b = f.inputs
+        out = f.output
+        if a == b or g.shapes[a][2] % 4 != 0 or {a, b, out} & io:
+            continue
+        if a in views or b in views or a in roots or b in roots:
+            continue
+        views[a] = (out, 0)
+        views[b] = (out, g.shapes[a][2] // 4)
+        roots.add(out)
+    return views
+
+
 def plan_problem(g, fused: Sequence[FusedOp], elem_bytes: int = 2, align: int = 256,
-                 convert_io: bool = True) -> PlanProblem:
+                 convert_io: bool = True, views: Optional[Dict[int, Tuple[int, int]]] = None) -> PlanProblem:
     """The executed op list and which tensors are intermediate (Section 5: neither a graph
     input nor a graph output, which the caller owns).  With convert_io, graph inputs and
     outputs are caller-owned NHWC buffers and a layout conversion op stands between each of
     them and the PHWC4 tensor the graph uses (Section 3, "Running Inference"), which makes
-    every tensor of the graph an intermediate."""
+    every tensor of the graph an intermediate.  With `views` (see concat_views) a tensor placed inside
+    another one is not planned: every use of it counts as a use of the tensor that holds it."""
+    views = views or {}
+
+    def root(t: int) -> int:
+        return views[t][0] if t in views else t
+
     ops: List[Tuple[List[int], List[int]]] = []
     if convert_io:
         for k, t in enumerate(g.inputs):
             ops.append(([EXTERNAL_BASE + k], [t]))
     for f in fused:
-        ops.append((f.reads(), [f.output]))
+        ops.append(([root(t) for t in f.reads()], [root(f.output)]))
     if convert_io:
         for k, t in enumerate(g.outputs):
             ops.append(([t], [EXTERNAL_BASE + len(g.inputs) + k]))
@@ -231,8 +262,8 @@ def plan_greedy_shared_objects(p: PlanProblem):
     obj: Dict[int, int] = {}
     for i, (reads, writes) in enumerate(p.ops):
         for t in writes:
-            if t not in p.intermediate:
-                continue
+            if t not in p.intermediate or t in obj:  # (a tensor that several ops write - see plan_problem's views -
+                continue                              # takes its object at the first of them)
             if not available:
                 sizes.append(p.size[t])
                 s = len(sizes) - 1

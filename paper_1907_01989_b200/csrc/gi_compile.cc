@@ -174,10 +174,14 @@ static uint64_t plan_shared_objects(gi_exec* e) {
   std::vector<Obj> objs;
   std::vector<int> pool;
   std::vector<int> obj_of(e->plan.size(), -1);
+  // a tensor placed inside another one (the input of a CONCAT that needs no copy) stands for that tensor,
+  // which takes its object at the first op that writes any part of it
+  auto holder = [&](int t) { return t >= 0 && e->plan[t].view_of >= 0 ? e->plan[t].view_of : t; };
   for (size_t i = 0; i < e->ops.size(); ++i) {
     const FusedOp& f = e->ops[i];
-    if (f.out >= 0 && e->plan[f.out].intermediate) {
-      const uint64_t need = e->plan[f.out].bytes;
+    const int out = holder(f.out);
+    if (out >= 0 && e->plan[out].intermediate && obj_of[out] < 0) {
+      const uint64_t need = e->plan[out].bytes;
       int s;
       if (pool.empty()) {
         objs.push_back({need});
@@ -195,10 +199,11 @@ static uint64_t plan_shared_objects(gi_exec* e) {
         pool.erase(pool.begin() + static_cast<long>(pick));
         if (need > objs[s].size) objs[s].size = need;
       }
-      obj_of[f.out] = s;
+      obj_of[out] = s;
     }
     int r[3];
     reads_of(f, r);
+    for (int k = 0; k < 3; ++k) r[k] = holder(r[k]);
     for (int k = 0; k < 3; ++k) {
       const int t = r[k];
       if (t < 0 || !e->plan[t].intermediate || e->plan[t].last != static_cast<int>(i)) continue;
@@ -361,20 +366,51 @@ static uint64_t plan_by_size(gi_exec* e) {
   return total;
 }
 
+// Concatenations that need no copy.  The slices of a tensor follow one another in memory (Section 4), so
+// concat(a, b) with C(a) a multiple of 4 is a's slices followed by b's: a and b are placed inside the result
+// and their producers write the result directly; the CONCAT itself launches nothing.  Eligible (walked in
+// execution order): two different inputs, C(a) % 4 == 0, none of a, b, out is a graph input or output, and
+// neither a nor b is already placed inside another tensor or holds tensors itself.
+static void find_concat_views(gi_exec* e) {
+  std::vector<char> is_root(e->tensors.size(), 0);
+  auto io = [&](int t) { return e->tensors[t].input_index >= 0 || e->tensors[t].output_index >= 0; };
+  for (const FusedOp& f : e->ops) {
+    if (f.kind != GI_OP_CONCAT || f.in1 < 0) continue;
+    const int a = f.in0, b = f.in1, out = f.out;
+    if (a == b || e->tensors[a].c % 4 != 0 || io(a) || io(b) || io(out)) continue;
+    if (e->plan[a].view_of >= 0 || e->plan[b].view_of >= 0 || is_root[a] || is_root[b]) continue;
+    e->plan[a].view_of = out;
+    e->plan[a].view_slice = 0;
+    e->plan[b].view_of = out;
+    e->plan[b].view_slice = e->tensors[a].c / 4;
+    is_root[out] = 1;
+  }
+}
+
 gi_status plan_memory(gi_exec* e) {
   const uint64_t align = static_cast<uint64_t>(e->opt.align);
   for (size_t t = 0; t < e->tensors.size(); ++t) {
     const TensorDesc& d = e->tensors[t];
     e->plan[t].bytes = gi_tensor_bytes(e->batch, d.h, d.w, d.c, e->storage, static_cast<int32_t>(align));
   }
+  if (e->opt.fuse) find_concat_views(e);
   compute_lifetimes(e);
+  // a tensor that holds others is in use whenever one of them is
+  for (size_t t = 0; t < e->tensors.size(); ++t) {
+    const TensorPlan& v = e->plan[t];
+    if (v.view_of < 0 || !v.alive) continue;
+    TensorPlan& r = e->plan[v.view_of];
+    r.first = std::min(r.first, v.first);
+    r.last = std::max(r.last, v.last);
+  }
   for (size_t t = 0; t < e->tensors.size(); ++t) {
     const TensorDesc& d = e->tensors[t];
     TensorPlan& p = e->plan[t];
-    // caller-owned PHWC4 inputs / outputs are not planned; everything else that is alive is
+    // caller-owned PHWC4 inputs / outputs are not planned, nor is a tensor placed inside another one;
+    // everything else that is alive is
     const bool callers = (d.input_index >= 0 && d.input_layout == GI_PHWC4) ||
                          (d.output_index >= 0 && d.output_layout == GI_PHWC4);
-    p.intermediate = p.alive && !callers;
+    p.intermediate = p.alive && !callers && p.view_of < 0;
   }
   e->naive_bytes = 0;
   for (const TensorPlan& p : e->plan)
@@ -392,6 +428,15 @@ gi_status plan_memory(gi_exec* e) {
     case GI_PLAN_GREEDY_BY_SIZE: e->arena_bytes = plan_by_size(e); break;
     case GI_PLAN_MIN_COST_FLOW: e->arena_bytes = plan_min_cost_flow(e); break;
     default: return fail(GI_E_INVALID, "gi_compile: unknown planner");
+  }
+  // tensors placed inside another one: their slices start `view_slice` slices into it
+  for (size_t t = 0; t < e->tensors.size(); ++t) {
+    TensorPlan& v = e->plan[t];
+    if (v.view_of < 0 || !v.alive) continue;
+    const TensorDesc& d = e->tensors[t];
+    const uint64_t slice_bytes = static_cast<uint64_t>(e->batch) * plane_pixels(d.h, d.w) * 4 * elem_bytes(e->storage);
+    v.offset = e->plan[v.view_of].offset + static_cast<uint64_t>(v.view_slice) * slice_bytes;
+    v.intermediate = 2;
   }
   return GI_OK;
 }

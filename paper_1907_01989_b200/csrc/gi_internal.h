@@ -86,8 +86,10 @@ struct FusedOp {
 };
 
 struct TensorPlan {
-  int alive = 0, intermediate = 0, first = -1, last = -1;
+  int alive = 0, intermediate = 0, first = -1, last = -1;  // intermediate: 1 planned, 2 placed inside `view_of`
   uint64_t bytes = 0, offset = 0;
+  int view_of = -1;    // the tensor whose memory holds this one (an input of a CONCAT that needs no copy), or -1
+  int view_slice = 0;  // first slice of `view_of` that this tensor occupies
 };
 
 }  // namespace gi

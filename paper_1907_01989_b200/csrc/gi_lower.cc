@@ -267,6 +267,12 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
         break;
       }
       case GI_OP_CONCAT:
+        if (f.in1 >= 0 && e->plan[f.in0].view_of == f.out && e->plan[f.in1].view_of == f.out) {
+          // both inputs were placed inside the output: their producers have already written it
+          r.kernel = GI_KERNEL_NONE;
+          info.bytes = 0;
+          break;
+        }
         if (f.in1 >= 0) {
           r.kernel = GI_KERNEL_CONCAT;
           info.bytes = (in_px * (in_c4 + slices(e->tensors[f.in1].c) * 4) + out_px * out_c4) * eb;

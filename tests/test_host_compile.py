@@ -90,11 +90,15 @@ def compare_with_oracle(spec, planner, fuse=True, storage=api.GI_F16, align=256)
                 else:
                     pre = a
             assert ACT_NAME[o.act_pre] == pre and ACT_NAME[o.act_post] == post
-    p = oc.plan_problem(spec, fused, 2 if storage == api.GI_F16 else 4, align, convert_io=True)
+    eb = 2 if storage == api.GI_F16 else 4
+    views = oc.concat_views(spec, fused) if fuse else {}
+    p = oc.plan_problem(spec, fused, eb, align, convert_io=True, views=views)
     life = oc.lifetimes(p)
     for t, ti in tensors.items():
-        assert bool(ti.alive) == (t in p.size)
+        assert bool(ti.alive) == (t in p.size or t in views)
         assert (ti.h, ti.w, ti.c) == tuple(spec.shapes[t])
+        if t in views:
+            assert ti.intermediate == 2 and t not in p.size
         if t in p.size:
             assert ti.intermediate == 1
             assert ti.bytes == p.size[t]
@@ -114,6 +118,9 @@ def compare_with_oracle(spec, planner, fuse=True, storage=api.GI_F16, align=256)
         assert tensors[t].offset == off[t], (t, tensors[t].offset, off[t])
         assert tensors[t].offset % align == 0
     oc.check_no_overlap(p, {t: tensors[t].offset for t in p.intermediate})
+    for t, (root, first_slice) in views.items():
+        H, W, _ = spec.shapes[t]
+        assert tensors[t].offset == off[root] + first_slice * spec.batch * ((H * W + 1) // 2 * 2) * 4 * eb
     return ex
 
 
@@ -364,3 +371,106 @@ def test_identity_resize_removed_like_the_oracle():
             ex = compare_with_oracle(spec, planner)
         assert ex.info.n_fused_ops == (3 if extra else 2)
         compare_with_oracle(spec, api.GI_PLAN_GREEDY_BY_SIZE, fuse=False)
+
+
+def _exact_bytes(spec, t, eb):
+    H, W, Cc = spec.shapes[t]
+    return ((Cc + 3) // 4) * spec.batch * ((H * W + 1) // 2 * 2) * 4 * eb
+
+
+@pytest.mark.parametrize("planner", PLANNERS)
+def test_concat_without_copy_memory_is_safe(planner):
+    """Inputs of a CONCAT that were placed inside its output: they tile the output's slices exactly, the CONCAT
+    launches nothing, and no two tensors that are in use at the same executed op share a byte - other than a
+    tensor and the tensor that holds it.  Checked on the fire network and on random graphs, from the
+    library's own answers (executed ops, offsets) with lifetimes recomputed here."""
+    specs = [wl.fire_network(2)]
+    for seed in range(60):
+        rnd = random.Random(500 + seed)
+        specs.append(random_spec(rnd, rnd.randint(4, 30)))
+    seen_views = 0
+    for spec in specs:
+        g, _ = api.graph_from_spec(spec, api.GI_F16)
+        ex = g.compile(planner=planner)
+        ops, tensors = exec_records(ex)
+        fused = oc.fuse(spec)
+        views = oc.concat_views(spec, fused)
+        seen_views += len(views)
+        # every eligible CONCAT launches nothing; its parts tile it
+        for f, o in zip(fused, ops[len(spec.inputs):]):
+            if f.kind == "concat" and len(f.inputs) == 2 and views.get(f.inputs[0], (None,))[0] == f.output:
+                a, b = f.inputs
+                assert api.KERNEL_NAMES[o.kernel] == "none"
+                assert tensors[a].offset == tensors[f.output].offset
+                assert tensors[b].offset == tensors[a].offset + _exact_bytes(spec, a, 2)
+                assert tensors[b].offset + _exact_bytes(spec, b, 2) == tensors[f.output].offset + _exact_bytes(spec, f.output, 2)
+            elif f.kind == "concat" and len(f.inputs) == 2:
+                assert api.KERNEL_NAMES[o.kernel] == "concat"
+        # own lifetimes from the executed list
+        life = {}
+        for i, o in enumerate(ops):
+            for t in (o.inputs[0], o.inputs[1], o.residual, o.output):
+                if t >= 0 and tensors[t].alive and tensors[t].intermediate:
+                    a, _ = life.get(t, (i, i))
+                    life[t] = (a, i)
+        ts = sorted(life)
+        for x in ts:
+            for y in ts:
+                if x >= y or life[x][1] < life[y][0] or life[y][1] < life[x][0]:
+                    continue
+                if views.get(x, (None,))[0] == y or views.get(y, (None,))[0] == x:
+                    continue
+                x0, x1 = tensors[x].offset, tensors[x].offset + _exact_bytes(spec, x, 2)
+                y0, y1 = tensors[y].offset, tensors[y].offset + _exact_bytes(spec, y, 2)
+                assert x1 <= y0 or y1 <= x0, (spec.name, x, y, life[x], life[y])
+        assert ex.info.arena_bytes >= max(tensors[t].offset + _exact_bytes(spec, t, 2) for t in ts)
+    assert seen_views >= 6  # the cases above do exercise it
+
+
+def test_concat_view_eligibility_rules():
+    def fused_and_views(build):
+        b = wl.GraphBuilder("views", 1, 60)
+        build(b)
+        spec = b.finish()
+        return spec, oc.concat_views(spec, oc.fuse(spec))
+
+    def ok(b):
+        x = b.input(6, 6, 4)
+        p, q = b.conv2d(x, 8, 1), b.conv2d(x, 6, 3)
+        b.output(b.conv2d(b.concat(p, q), 4, 1))
+    spec, v = fused_and_views(ok)
+    assert v == {1: (3, 0), 2: (3, 2)}
+
+    def ragged_first(b):
+        x = b.input(6, 6, 4)
+        p, q = b.conv2d(x, 6, 1), b.conv2d(x, 8, 3)
+        b.output(b.conv2d(b.concat(p, q), 4, 1))
+    assert fused_and_views(ragged_first)[1] == {}
+
+    def reads_graph_input(b):
+        x = b.input(6, 6, 4)
+        b.output(b.conv2d(b.concat(x, b.conv2d(x, 8, 1)), 4, 1))
+    assert fused_and_views(reads_graph_input)[1] == {}
+
+    def is_graph_output(b):
+        x = b.input(6, 6, 4)
+        b.output(b.concat(b.conv2d(x, 8, 1), b.conv2d(x, 8, 3)))
+    assert fused_and_views(is_graph_output)[1] == {}
+
+    def nested(b):
+        x = b.input(6, 6, 4)
+        inner = b.concat(b.conv2d(x, 8, 1), b.conv2d(x, 8, 3))   # tensors 1, 2 -> 3
+        outer = b.concat(inner, b.conv2d(x, 4, 1))                 # 3 holds tensors already: copied
+        b.output(b.conv2d(outer, 4, 1))
+    spec, v = fused_and_views(nested)
+    assert v == {1: (3, 0), 2: (3, 2)}
+
+    def same_twice_and_reused(b):
+        x = b.input(6, 6, 4)
+        p, q = b.conv2d(x, 8, 1), b.conv2d(x, 8, 3)
+        c1 = b.concat(p, p)          # one tensor twice: copied
+        c2 = b.concat(p, q)          # placed
+        c3 = b.concat(q, p)          # both already placed: copied
+        b.output(b.conv2d(b.add(b.add(c1, c2), c3), 4, 1))
+    spec, v = fused_and_views(same_twice_and_reused)
+    assert v == {1: (4, 0), 2: (4, 2)}
