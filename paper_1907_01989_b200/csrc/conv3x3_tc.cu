@@ -13,6 +13,13 @@
 // apply the fused element-wise tail and store 8 bytes per output slice (256 contiguous bytes per
 // warp).  Operand tiles and accumulators are double-buffered: the gather of tile i+1 runs while
 // the MMAs of tile i are in flight.  Waits are bounded like in the pointwise kernel.
+//
+// NHWC3: the input is the caller's NHWC tensor with 3 fp16 channels (stride 2, no padding above / left, even
+// H and W): the layout conversion in front of the convolution (Section 3, "Running Inference") disappears,
+// the image is read once, as 6 instead of 8 bytes per pixel.  The three pixels of a window row are 18
+// contiguous bytes (4-byte aligned because the first pixel's index is even): five 32-bit loads, whose last
+// half - the first channel of the next pixel - is masked off.  The K axis is then simply those 15 words + 1
+// zero word: k = 10 * ky + 3 * kx + ci, 32 values (two MMAs instead of three), the weights packed to match.
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -66,8 +73,9 @@ __device__ __forceinline__ float act1(float v, int kind) {
 }
 
 // ACT: activation right after the bias; TAIL: a residual add and / or a second activation follow
-template <int ACT, bool TAIL>
+template <int ACT, bool TAIL, bool NHWC3>
 __global__ void __launch_bounds__(kThreads, 6) conv3x3_tc_kernel(const StemParams p) {
+  constexpr int kCoresUsed = NHWC3 ? 4 : kKCores;  // 16-byte K units per row actually multiplied
   extern __shared__ __align__(1024) unsigned char smem[];
   Header* hdr = reinterpret_cast<Header*>(smem);
   unsigned char* a_tiles = smem + 1024;                 // 2 x kABytes
@@ -85,10 +93,10 @@ __global__ void __launch_bounds__(kThreads, 6) conv3x3_tc_kernel(const StemParam
   }
   if (warp == 4) tmem_alloc(smem_u32(&hdr->tmem_addr), p.tmem_cols);
   // weights: plain copy into shared memory, then made visible to the tensor core's proxy
-  for (int i = threadIdx.x; i < kKCores * p.n_pad; i += kThreads)
+  for (int i = threadIdx.x; i < kCoresUsed * p.n_pad; i += kThreads)
     reinterpret_cast<uint4*>(b_tile)[i] = __ldg(reinterpret_cast<const uint4*>(p.wts) + i);
   // K elements 40..47 of both operand buffers are padding: zeroed once, never written again
-  if (threadIdx.x < kRows) {
+  if (!NHWC3 && threadIdx.x < kRows) {
     reinterpret_cast<uint4*>(a_tiles)[5 * kRows + threadIdx.x] = make_uint4(0u, 0u, 0u, 0u);
     reinterpret_cast<uint4*>(a_tiles + kABytes)[5 * kRows + threadIdx.x] = make_uint4(0u, 0u, 0u, 0u);
   }
@@ -107,6 +115,37 @@ __global__ void __launch_bounds__(kThreads, 6) conv3x3_tc_kernel(const StemParam
     const int real_px = p.Ho * p.Wo;
     // ---- gather of one tile into operand buffer `buf`; this thread's pixel is q of image b
     auto gather = [&](int buf, int b, int q, bool in_tensor) {
+      if (NHWC3) {
+        unsigned w[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) w[k] = 0u;
+        if (in_tensor && q < real_px) {
+          const int oy = q / p.Wo, ox = q - oy * p.Wo;
+          const int iy0 = 2 * oy, ix0 = 2 * ox;  // even: the window's first pixel starts on a 4-byte boundary
+          // 32-bit words: a pixel is 1.5 words, a row p.W * 3 / 2 words (W is even)
+          const unsigned* row = reinterpret_cast<const unsigned*>(p.in) +
+                                ((static_cast<long long>(b) * p.H + iy0) * p.W + ix0) / 2 * 3;
+          const int row_words = p.W / 2 * 3;
+          const bool third = ix0 + 2 < p.W;  // the window's last column exists (else it is padding)
+#pragma unroll
+          for (int ky = 0; ky < 3; ++ky, row += row_words) {
+            if (iy0 + ky >= p.H) break;  // padding row below the image
+            w[5 * ky] = __ldg(row);
+            w[5 * ky + 1] = __ldg(row + 1);
+            w[5 * ky + 2] = __ldg(row + 2);
+            if (third) {
+              w[5 * ky + 3] = __ldg(row + 3);
+              w[5 * ky + 4] = __ldg(row + 4) & 0xffffu;  // upper half: first channel of the next pixel
+            }
+          }
+        }
+        uint4* dst = reinterpret_cast<uint4*>(a_tiles + buf * kABytes) + t;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) dst[j * kRows] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(smem_u32(&hdr->a_full[buf]));
+        return;
+      }
       uint2 tap[10];
 #pragma unroll
       for (int k = 0; k < 10; ++k) tap[k] = make_uint2(0u, 0u);
@@ -254,7 +293,7 @@ __global__ void __launch_bounds__(kThreads, 6) conv3x3_tc_kernel(const StemParam
       tc_fence_after();
       const unsigned a_base = smem_u32(a_tiles + buf * kABytes);
 #pragma unroll
-      for (int ks = 0; ks < 3; ++ks) {
+      for (int ks = 0; ks < kCoresUsed / 2; ++ks) {
         const unsigned long long ad = smem_desc(a_base + ks * 2 * kRows * 16, kRows * 16, 128);
         const unsigned long long bd = smem_desc(b_base + ks * 2 * b_lbo, b_lbo, 128);
         umma_f16(tmem_base + buf * n_cols, ad, bd, idesc, ks > 0 ? 1u : 0u);
@@ -278,7 +317,15 @@ bool conv3x3_tc_supported(int cin, int cout, int kh, int kw, int sh, int sw, int
   return kh == 3 && kw == 3 && cin <= 4 && cout >= 1 && cout <= kMaxN && sh == sw && dh == dw;
 }
 
-// Weights as the B operand: [6 K units][n_pad rows][8 halves], k = unit * 8 + e = tap * 4 + ci.
+// The convolution can read the caller's NHWC input itself (no layout conversion in front of it): three fp16
+// channels, stride 2 with no padding above / left, even H and W (the window's first pixel then starts on a
+// 4-byte boundary and the pixel after the window's last one always exists in the same row).
+bool conv3x3_tc_reads_nhwc(int cin, int H, int W, int stride, int dil, int pt, int pl) {
+  return cin == 3 && stride == 2 && dil == 1 && pt == 0 && pl == 0 && H % 2 == 0 && W % 2 == 0;
+}
+
+// Weights as the B operand: [6 K units][n_pad rows][8 halves], k = unit * 8 + e = tap * 4 + ci; for the
+// NHWC-reading variant (r->nhwc_in) [4 K units][n_pad rows][8 halves], k = 10 * ky + 3 * kx + ci.
 void conv3x3_tc_pack(const float* w, const float* bias, int cin, int cout, std::vector<uint8_t>* blob, LaunchRec* r) {
   const int n_pad = (cout + 15) / 16 * 16;
   const size_t wbytes = static_cast<size_t>(kKCores) * n_pad * 16;
@@ -292,7 +339,7 @@ void conv3x3_tc_pack(const float* w, const float* bias, int cin, int cout, std::
     bp[co] = bias[co];
     for (int tap = 0; tap < 9; ++tap)
       for (int ci = 0; ci < cin; ++ci) {
-        const int k = tap * 4 + ci;
+        const int k = r->nhwc_in ? 10 * (tap / 3) + 3 * (tap % 3) + ci : tap * 4 + ci;
         wp[(static_cast<size_t>(k / 8) * n_pad + co) * 8 + k % 8] = f32_to_f16_rne(w[(static_cast<size_t>(co) * 9 + tap) * cin + ci]);
       }
   }
@@ -341,8 +388,11 @@ int launch_conv3x3_tc(const LaunchRec& r, const Ptrs& p, void* stream) {
   if (!attr_set) {
     cudaError_t e = cudaSuccess;
     const int bytes = 1024 + 2 * kABytes + kKCores * kMaxN * 16;
-#define GI_C3_ATTR(A, T) \
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(conv3x3_tc_kernel<A, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)
+#define GI_C3_ATTR(A, T)                                                                                                               \
+  do {                                                                                                                                 \
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv3x3_tc_kernel<A, T, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes); \
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv3x3_tc_kernel<A, T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);  \
+  } while (0)
     GI_C3_ATTR(GI_ACT_NONE, false);
     GI_C3_ATTR(GI_ACT_RELU, false);
     GI_C3_ATTR(GI_ACT_RELU6, false);
@@ -367,7 +417,11 @@ int launch_conv3x3_tc(const LaunchRec& r, const Ptrs& p, void* stream) {
   cudaStream_t cu_stream = static_cast<cudaStream_t>(stream);
   const int act = r.ep.act_pre;
   const bool tail = k.has_res || k.act_post != GI_ACT_NONE;
-#define GI_C3_LAUNCH(A, T) launch_pdl(conv3x3_tc_kernel<A, T>, g, kThreads, smem, cu_stream, k)
+#define GI_C3_LAUNCH(A, T)                                                                              \
+  do {                                                                                                  \
+    if (r.nhwc_in) launch_pdl(conv3x3_tc_kernel<A, T, true>, g, kThreads, smem, cu_stream, k);          \
+    else launch_pdl(conv3x3_tc_kernel<A, T, false>, g, kThreads, smem, cu_stream, k);                   \
+  } while (0)
   if (tail) {
     if (act == GI_ACT_RELU6) GI_C3_LAUNCH(GI_ACT_RELU6, true);
     else if (act == GI_ACT_RELU) GI_C3_LAUNCH(GI_ACT_RELU, true);

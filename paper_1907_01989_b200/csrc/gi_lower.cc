@@ -118,6 +118,23 @@ static bool pointwise_follows(const gi_graph& g, const gi_exec* e, size_t i) {
          d.pad_r == 0;
 }
 
+// The executed op that converts graph input `t` from NHWC, if executed op `reader` is the only op that reads
+// the converted tensor (and it is not also a graph output); else -1.
+static int nhwc_pack_feeding_only(const gi_exec* e, int t, size_t reader) {
+  if (t < 0) return -1;
+  const TensorDesc& d = e->tensors[t];
+  if (d.input_index < 0 || d.input_layout != GI_NHWC || d.output_index >= 0) return -1;
+  int pack = -1;
+  for (size_t j = 0; j < e->ops.size(); ++j) {
+    const FusedOp& o = e->ops[j];
+    if (o.kind == GI_EXEC_PACK && o.out == t) pack = static_cast<int>(j);
+    if (j != reader && (o.in0 == t || o.in1 == t || o.residual == t)) return -1;
+  }
+  const FusedOp& r = e->ops[reader];
+  if (r.in1 == t || r.residual == t) return -1;
+  return pack;
+}
+
 gi_status lower(const gi_graph& g, gi_exec* e) {
   const int eb = elem_bytes(e->storage);
   const uint64_t B = static_cast<uint64_t>(e->batch);
@@ -248,6 +265,19 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
           } else if (tc && conv3x3_tc_supported(din->c, op.d.cout, op.d.kh, op.d.kw, op.d.stride_h, op.d.stride_w,
                                           op.d.dilation_h, op.d.dilation_w)) {
             r.kernel = GI_KERNEL_CONV3X3_TC;
+            // Section 3.2 folds cheap operators into the expensive one next to them; the layout conversion in
+            // front of the stem is such an operator: where the kernel can read the caller's NHWC tensor itself
+            // (and nothing else reads the converted tensor) the conversion launches nothing
+            const int pack_op = nhwc_pack_feeding_only(e, f.in0, i);
+            if (e->opt.fuse && pack_op >= 0 &&
+                conv3x3_tc_reads_nhwc(din->c, din->h, din->w, op.d.stride_h, op.d.dilation_h, op.d.pad_t, op.d.pad_l)) {
+              r.nhwc_in = 1;
+              r.in0 = Loc{W_INPUT, din->input_index, 0};
+              e->launches[pack_op].kernel = GI_KERNEL_NONE;
+              e->op_info[pack_op].kernel = GI_KERNEL_NONE;
+              e->op_info[pack_op].bytes = 0;
+              info.bytes = (in_px * din->c + out_px * out_c4 * (r.ep.has_res ? 2 : 1)) * eb;
+            }
             conv3x3_tc_pack(op.weights.data(), op.bias.data(), din->c, op.d.cout, &e->weight_blob, &r);
           } else if (tc && conv_kxk_tc_supported(din->c, op.d.cout, op.d.kh, op.d.kw, op.d.stride_h, op.d.stride_w,
                                                   op.d.dilation_h, op.d.dilation_w)) {

@@ -49,6 +49,7 @@ unsigned int pointwise_tc_error_word(int* cuda_err);
 
 // Full 3x3 convolution with one input slice (<= 4 channels) on the tensor cores (fp16 storage).
 bool conv3x3_tc_supported(int cin, int cout, int kh, int kw, int sh, int sw, int dh, int dw);
+bool conv3x3_tc_reads_nhwc(int cin, int H, int W, int stride, int dil, int pt, int pl);
 void conv3x3_tc_pack(const float* w, const float* bias, int cin, int cout, std::vector<uint8_t>* blob, LaunchRec* r);
 int launch_conv3x3_tc(const LaunchRec& r, const Ptrs& p, void* stream);
 unsigned int conv3x3_tc_error_word(int* cuda_err);

@@ -594,3 +594,52 @@ def test_conv_kxk_weights_far_too_large_take_the_cuda_core_kernel():
     run = DeviceRun(spec, api.GI_F16)
     assert "conv_simt" in [api.KERNEL_NAMES[o.kernel] for o in run.ex.ops()]
     check_all_tensors(spec, api.GI_F16)
+
+
+def _names(spec, **kw):
+    return [api.KERNEL_NAMES[o.kernel] for o in api.graph_from_spec(spec, api.GI_F16)[0].compile(**kw).ops()]
+
+
+@pytest.mark.parametrize("case", [(2, 32, 48, 16), (1, 224, 224, 32), (3, 6, 2, 24), (2, 2, 2, 8), (5, 62, 30, 40), (1, 130, 258, 16)])
+def test_stem_reads_nhwc_input_itself(case):
+    """3-channel NHWC fp16 input, 3x3 stride-2 convolution, even H and W: the layout conversion launches nothing and
+    the convolution gathers from the caller's tensor; results are those of the oracle (which knows no layouts)."""
+    B, H, W, cout = case
+    b = wl.GraphBuilder(f"stem_nhwc_{B}x{H}x{W}x{cout}", B, 14)
+    x = b.input(H, W, 3)
+    y = b.activation(b.conv2d(x, cout, 3, 2), wl.ACT_RELU6)
+    b.output(b.activation(b.depthwise(y, 3, 1), wl.ACT_RELU))
+    spec = b.finish()
+    assert _names(spec)[:2] == ["none", "conv3x3_tc"]
+    assert _names(spec, fuse=False)[0] == "pack"
+    check_all_tensors(spec, api.GI_F16)
+    check_outputs(spec, api.GI_F16)
+    assert api.gi_device_status() == 0
+
+
+def test_stem_keeps_the_layout_conversion_where_it_must():
+    def first_two(build, B=2):
+        b = wl.GraphBuilder("stem_pack", B, 15)
+        build(b)
+        spec = b.finish()
+        check_all_tensors(spec, api.GI_F16)
+        return _names(spec)[:2]
+
+    def odd(b):
+        b.output(b.activation(b.conv2d(b.input(33, 32, 3), 16, 3, 2), wl.ACT_RELU6))
+    assert first_two(odd) == ["pack", "conv3x3_tc"]
+
+    def stride1(b):
+        b.output(b.activation(b.conv2d(b.input(32, 32, 3), 16, 3, 1), wl.ACT_RELU6))
+    assert first_two(stride1) == ["pack", "conv3x3_tc"]
+
+    def four_channels(b):
+        b.output(b.activation(b.conv2d(b.input(32, 32, 4), 16, 3, 2), wl.ACT_RELU6))
+    assert first_two(four_channels) == ["pack", "conv3x3_tc"]
+
+    def second_reader(b):
+        x = b.input(32, 32, 3)
+        b.output(b.activation(b.conv2d(x, 16, 3, 2), wl.ACT_RELU6))
+        b.output(b.activation(b.depthwise(x, 3, 2), wl.ACT_RELU6))
+    assert first_two(second_reader) == ["pack", "conv3x3_tc"]
+    assert api.gi_device_status() == 0
