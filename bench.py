@@ -402,6 +402,8 @@ def main():
         fam = {}
         for o, t in zip(ops, per_op):
             name = api.KERNEL_NAMES[o.kernel]
+            if name == "none":  # nothing was launched for this op (it ran inside another op's kernel, or needs none)
+                continue
             f = fam.setdefault(name, {"launches": 0, "ms": 0.0, "bytes": 0, "flops": 0, "roof_ms": 0.0})
             f["launches"] += 1
             f["ms"] += float(t)
