@@ -190,6 +190,8 @@ def run_sweep(args):
         points = [tuple(int(v) for v in pt.split(",")) for pt in args.points.split(";") if pt]
     elif args.sweep == "conv3":
         points = [(256, 224, 3, 32, 2), (64, 224, 3, 32, 2), (16, 513, 3, 32, 2), (1, 224, 3, 32, 2)]
+    elif args.sweep == "stem":
+        points = [(256, 224, 32), (64, 224, 32), (1, 224, 32)]
     elif args.sweep == "dwpw":  # the depthwise -> projection pairs of MobileNetV2 that have at least one tile per SM
         points = [(256, 112, 32, 16, 1), (256, 112, 96, 24, 2), (256, 56, 144, 24, 1), (256, 56, 144, 32, 2), (256, 28, 192, 32, 1),
                   (256, 28, 192, 64, 2), (256, 14, 384, 64, 1), (256, 14, 576, 96, 1)]
@@ -203,7 +205,13 @@ def run_sweep(args):
                   (256, 14, 1280, 1280), (64, 56, 192, 192), (8, 28, 384, 384), (1, 14, 96, 576)]
     rows = []
     for pt in points:
-        if args.sweep == "conv3":
+        in_layout = api.GI_PHWC4
+        if args.sweep == "stem":
+            b, hw, cout = pt
+            spec = wl.single_conv3x3(b, hw, 3, cout, 2)
+            name = f"conv3x3 b{b} {hw}x{hw} 3->{cout} s2, NHWC input"
+            in_layout = api.GI_NHWC
+        elif args.sweep == "conv3":
             b, hw, cin, cout, stride = pt
             spec = wl.single_conv3x3(b, hw, cin, cout, stride)
             name = f"conv3x3 b{b} {hw}x{hw} {cin}->{cout} s{stride}"
@@ -219,12 +227,16 @@ def run_sweep(args):
             b, hw, cin, cout = pt
             spec = wl.single_pointwise(b, hw, cin, cout, residual=args.residual)
             name = f"pw1x1 b{b} {hw}x{hw} {cin}->{cout}"
-        g, _ = api.graph_from_spec(spec, api.GI_F16, io_layout=api.GI_PHWC4)
+        g, _ = api.graph_from_spec(spec, api.GI_F16, io_layout=in_layout, out_layout=api.GI_PHWC4)
         ex = g.compile(pointwise=PW_MODES[args.pointwise], cross_op=XOP_MODES[args.cross_op])
         ex.bind(dev)
         ops = ex.ops()
-        assert len(ops) == (2 if args.sweep == "dwpw" else 1)
-        ins = [(torch.rand(api.gi_tensor_bytes(b, *spec.shapes[t]) // 2, device=dev) * 2 - 1).half() for t in spec.inputs]
+        assert len(ops) == (2 if args.sweep in ("dwpw", "stem") else 1)
+        if args.sweep == "stem":  # the layout conversion must have been taken over by the convolution
+            assert [api.KERNEL_NAMES[q.kernel] for q in ops] == ["none", "conv3x3_tc"], "this shape keeps its layout conversion"
+            ins = [(torch.rand((b,) + tuple(spec.shapes[t]), device=dev) * 2 - 1).half() for t in spec.inputs]
+        else:
+            ins = [(torch.rand(api.gi_tensor_bytes(b, *spec.shapes[t]) // 2, device=dev) * 2 - 1).half() for t in spec.inputs]
         outs = [torch.empty(api.gi_tensor_bytes(b, *spec.shapes[t]) // 2, dtype=torch.float16, device=dev)
                 for t in spec.outputs]
         for _ in range(3):
@@ -277,10 +289,11 @@ def main():
     ap.add_argument("--per-op", default=None, help="write the per-op timing table to this file")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-batch1", action="store_true", help="skip the batch-1 latency leg (keeps profiler runs short)")
-    ap.add_argument("--sweep", default=None, choices=["pw", "dw", "conv3", "dwpw"],
+    ap.add_argument("--sweep", default=None, choices=["pw", "dw", "conv3", "dwpw", "stem"],
                     help="time single fused operators instead of a network")
     ap.add_argument("--points", default=None, help="sweep points 'B,HW,Cin,Cout;...' (pw), 'B,HW,C,stride;...' (dw), "
-                    "'B,HW,Cin,Cout,stride;...' (conv3), 'B,HW,C,Cout,stride;...' (dwpw: depthwise then 1x1, see --cross-op)")
+                    "'B,HW,Cin,Cout,stride;...' (conv3), 'B,HW,C,Cout,stride;...' (dwpw: depthwise then 1x1, see --cross-op), "
+                    "'B,HW,Cout;...' (stem: 3x3 stride-2 convolution of a 3-channel NHWC input, read in that layout)")
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--residual", action="store_true")
     ap.add_argument("--out", default=None)

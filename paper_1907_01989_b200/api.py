@@ -183,8 +183,10 @@ class Graph:
         return Executable(h, self)
 
 
-def graph_from_spec(spec: wl.GraphSpec, storage: int = GI_F16, io_layout: int = GI_NHWC):
-    """Build a gi graph from a workload description.  Returns (Graph, {spec tensor id -> gi tensor id})."""
+def graph_from_spec(spec: wl.GraphSpec, storage: int = GI_F16, io_layout: int = GI_NHWC, out_layout: int = None):
+    """Build a gi graph from a workload description.  Returns (Graph, {spec tensor id -> gi tensor id}).
+    `io_layout` is the layout of the graph's inputs and, unless `out_layout` is given, of its outputs."""
+    out_layout = io_layout if out_layout is None else out_layout
     g = Graph(spec.batch, storage)
     ids = {}
     for t in spec.inputs:
@@ -218,7 +220,7 @@ def graph_from_spec(spec: wl.GraphSpec, storage: int = GI_F16, io_layout: int = 
         ids[op.output] = g.add_op(d)
         del keep
     for t in spec.outputs:
-        g.output(ids[t], io_layout)
+        g.output(ids[t], out_layout)
     return g, ids
 
 
