@@ -643,3 +643,26 @@ def test_stem_keeps_the_layout_conversion_where_it_must():
         b.output(b.activation(b.depthwise(x, 3, 2), wl.ACT_RELU6))
     assert first_two(second_reader) == ["pack", "conv3x3_tc"]
     assert api.gi_device_status() == 0
+
+
+@pytest.mark.parametrize("cross_op", [api.GI_XOP_OFF, api.GI_XOP_ON])
+def test_fire_network_with_caller_owned_phwc4_buffers(cross_op):
+    """PHWC4 input and output (no layout conversions): the first convolution reads the caller's buffer, the
+    copy-free concatenations still apply (they are interior), the result is the oracle's."""
+    import torch
+    spec = wl.fire_network(3, size=64)
+    xin = wl.make_input(spec)
+    g, _ = api.graph_from_spec(spec, api.GI_F16, io_layout=api.GI_PHWC4)
+    ex = g.compile(cross_op=cross_op)
+    names = [api.KERNEL_NAMES[o.kernel] for o in ex.ops()]
+    assert names.count("none") == 2 and "pack" not in names and "unpack" not in names
+    ex.bind()
+    x = torch.from_numpy(oops.phwc4_pack(xin)).to("cuda:0").half().contiguous()
+    H, W, Cc = spec.shapes[spec.outputs[0]]
+    out = torch.zeros(api.gi_tensor_bytes(3, H, W, Cc) // 2, dtype=torch.float16, device="cuda:0")
+    for _ in range(2):  # a second run over the same arena gives the same answer
+        ex.run([x], [out])
+        torch.cuda.synchronize()
+        got = oops.phwc4_unpack(out.float().cpu().numpy(), 3, H, W, Cc)
+        assert_close(got, og.run(spec, [xin], storage="f16")[spec.outputs[0]], api.GI_F16, "fire network, phwc4 io")
+    assert api.gi_device_status() == 0
