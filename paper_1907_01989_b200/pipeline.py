@@ -15,7 +15,10 @@ class HostPipeline:
     """Two-slot software pipeline: H2D on a copy stream, gi_run + D2H on the compute stream."""
 
     def __init__(self, ex, input_shapes: Sequence[Sequence[int]], output_shapes: Sequence[Sequence[int]], dtype, device="cuda:0",
-                 slots: int = 2):
+                 slots: int = 2, graphs: bool = False):
+        """graphs: capture each slot's gi_run once as a CUDA graph (its device buffers never change) and replay
+        it per batch: one launch instead of one per kernel.  Falls back to plain launches if capture fails
+        (`self.graphs` then stays empty)."""
         import torch
         self.torch = torch
         self.ex = ex
@@ -28,6 +31,26 @@ class HostPipeline:
         self.free = [torch.cuda.Event() for _ in range(slots)]     # slot's kernels and read-back are done
         self.used = [False] * slots
         self.n = 0
+        self.graphs = []
+        if graphs:
+            try:
+                side = torch.cuda.Stream(device)
+                side.wait_stream(self.compute)
+                caught = []
+                with torch.cuda.stream(side):
+                    for s in range(slots):
+                        self.ex.run(self.ins[s], self.outs[s], side)  # warm-up: attributes, tensor maps
+                    side.synchronize()
+                    for s in range(slots):
+                        cg = torch.cuda.CUDAGraph()
+                        with torch.cuda.graph(cg, stream=side):
+                            self.ex.run(self.ins[s], self.outs[s], torch.cuda.current_stream(device))
+                        caught.append(cg)
+                self.compute.wait_stream(side)
+                torch.cuda.synchronize(device)
+                self.graphs = caught
+            except Exception:  # capture is an optimisation, never a requirement
+                self.graphs = []
 
     def submit(self, host_inputs: Sequence, host_outputs: Sequence) -> None:
         """Enqueue one batch: pinned host tensors in, pinned host tensors out.  Asynchronous; results are
@@ -43,7 +66,10 @@ class HostPipeline:
             self.loaded[s].record(self.copy)
         self.compute.wait_event(self.loaded[s])
         with torch.cuda.stream(self.compute):
-            self.ex.run(self.ins[s], self.outs[s], self.compute)
+            if self.graphs:
+                self.graphs[s].replay()
+            else:
+                self.ex.run(self.ins[s], self.outs[s], self.compute)
             for h, d in zip(host_outputs, self.outs[s]):
                 h.copy_(d, non_blocking=True)
             self.free[s].record(self.compute)

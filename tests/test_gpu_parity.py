@@ -341,7 +341,8 @@ def test_phwc4_io_layout_skips_conversions():
 
 
 @pytest.mark.gpu
-def test_host_pipeline_matches_plain_runs():
+@pytest.mark.parametrize("graphs", [False, True], ids=["launches", "cuda_graphs"])
+def test_host_pipeline_matches_plain_runs(graphs):
     """Batches submitted through the two-slot host pipeline come back in order and equal to plain runs."""
     import torch
     from paper_1907_01989_b200.pipeline import HostPipeline
@@ -358,7 +359,8 @@ def test_host_pipeline_matches_plain_runs():
         ex.run([x.to("cuda:0")], [out])
         torch.cuda.synchronize()
         want.append(out.cpu())
-    pipe = HostPipeline(ex, [shape_in], [shape_out], torch.float16, "cuda:0")
+    pipe = HostPipeline(ex, [shape_in], [shape_out], torch.float16, "cuda:0", graphs=graphs)
+    assert len(pipe.graphs) == (2 if graphs else 0)
     got = [torch.empty(shape_out, dtype=torch.float16).pin_memory() for _ in xs]
     for x, o in zip(xs, got):
         pipe.submit([x], [o])
