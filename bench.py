@@ -17,6 +17,11 @@ conversion out) on a batch of synthetic images.  Prints ONE JSON line on rank 0.
                the measured HBM peak (or flops against the tensor peak where that binds).
 * cpu_baseline the CPU oracle as it stands on this machine's host cores, on a bounded sample of images.
 * batch1       latency of the same network at batch 1, plain launches and CUDA-graph replay.
+* sustained    the same step (and the same host-buffer pipeline) repeated back to back for at least 3 s of
+               device time, with the SM clock sampled throughout: what the GPU holds under its power cap,
+               next to the 20-step burst the headline is.
+
+--gpus N without a torchrun environment starts the N ranks itself (re-executes under torch.distributed.run).
 
 N > 1 runs independent replicas (one process per GPU, the batch is the only sharded axis and
 the path has no exchange step): weak scaling, no collective on the data path.
@@ -150,6 +155,62 @@ def oracle_images_per_s(spec_fn, budget_s=15.0):
     return n / dt, cores, f"{n} images of the workload, evaluated once as one batch of {n} ({dt:.1f} s)", n, dt
 
 
+def respawn_under_torchrun(n: int) -> int:
+    """`python bench.py --gpus N` outside torchrun: start the N ranks (one per GPU) and return their exit code."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def clock_bins(chunks, rows):
+    """chunks: (wall start, wall end, device ms, images); rows: the sampler's (arrival time, csv line).  Each chunk gets
+    the median SM clock of the samples that arrived while it ran; returns images/s per 100 MHz clock bin."""
+    bins = {}
+    for w0, w1, ms, images in chunks:
+        mhz = []
+        for when, row in rows:
+            if w0 <= when <= w1:
+                try:
+                    mhz.append(float(row.split(",")[1]))
+                except (ValueError, IndexError):
+                    pass
+        if not mhz:
+            continue
+        key = int(statistics.median(mhz) // 100 * 100)
+        b = bins.setdefault(key, [0.0, 0])
+        b[0] += ms
+        b[1] += images
+    return {f"{k}-{k + 99} MHz": {"images_per_s": round(v[1] / v[0] * 1e3, 1), "seconds": round(v[0] * 1e-3, 3)}
+            for k, v in sorted(bins.items())}
+
+
+def sustained_leg(torch, stream, run_chunk, images_per_chunk, gpu_index, seconds=3.0):
+    """Repeat `run_chunk()` (which enqueues work and returns the device milliseconds it took, synchronised) until
+    at least `seconds` of device time have passed; SM clock sampled from before the first chunk."""
+    sampler = ClockSampler(gpu_index)
+    sampler.start()
+    time.sleep(0.1)
+    chunks, total_ms = [], 0.0
+    t0 = time.time()
+    while total_ms < seconds * 1e3 and len(chunks) < 100000:
+        w0 = time.time()
+        ms = run_chunk()
+        w1 = time.time()
+        chunks.append((w0, w1, ms, images_per_chunk))
+        total_ms += ms
+    t1 = time.time()
+    rows = list(sampler.rows)
+    clocks = sampler.stop(t0, t1)
+    images = images_per_chunk * len(chunks)
+    return {"images_per_s": images / total_ms * 1e3, "device_seconds": round(total_ms * 1e-3, 3), "wall_seconds": round(t1 - t0, 3),
+            "steps": None, "sm_mhz_median": clocks["sm_mhz"], "clock_samples": clocks.get("samples"),
+            "reasons": clocks["reasons"], "by_sm_clock": clock_bins(chunks, rows)}
+
+
 def run_reference(args, spec_fn, label):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -157,7 +218,8 @@ def run_reference(args, spec_fn, label):
     vals = []
     sample = ""
     for step in range(args.warmup + args.steps):
-        v, cores, sample, n, dt = oracle_images_per_s(spec_fn, budget_s=max(1.0, 100.0 / (args.warmup + args.steps)))
+        budget = args.budget_s if args.budget_s else max(1.0, 100.0 / (args.warmup + args.steps))
+        v, cores, sample, n, dt = oracle_images_per_s(spec_fn, budget_s=budget)
         if step >= args.warmup:
             vals.append((n, dt))
     n_tot, t_tot = sum(n for n, _ in vals), sum(t for _, t in vals)
@@ -172,6 +234,48 @@ def run_reference(args, spec_fn, label):
             "e2e": {"value": value, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
+
+
+def measure_fp16_peak():
+    """Dense fp16 matmul throughput of this GPU, measured the way the bf16 figure of MEASURED_PEAKS.json was:
+    torch.matmul 8192^3, best of 10 (burst) and back to back for 4 s (sustained).  A library GEMM as a yardstick
+    for the roofline denominators; nothing of the inference path runs here."""
+    import torch
+    torch.cuda.set_device(0)
+    out = {}
+    for name, dt in (("fp16", torch.float16), ("bf16", torch.bfloat16)):
+        a = torch.randn(8192, 8192, device="cuda", dtype=dt)
+        b = torch.randn(8192, 8192, device="cuda", dtype=dt)
+        flops = 2 * 8192 ** 3
+        for _ in range(3):
+            a @ b
+        best = 1e9
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            a @ b
+            e1.record()
+            e1.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        sampler = ClockSampler(0)
+        sampler.start()
+        t0 = time.time()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = 0
+        e0.record()
+        while time.time() - t0 < 4.0:
+            for _ in range(50):
+                a @ b
+            n += 50
+            torch.cuda.synchronize()
+        e1.record()
+        e1.synchronize()
+        t1 = time.time()
+        clocks = sampler.stop(t0, t1)
+        out[name] = {"tflops_burst": round(flops / best / 1e9, 1), "tflops_sustained": round(n * flops / e0.elapsed_time(e1) / 1e9, 1),
+                     "sm_mhz_median_sustained": clocks["sm_mhz"], "reasons": clocks["reasons"]}
+        time.sleep(2.0)
+    print(json.dumps({"fp16_peak": out, "how": "torch.matmul 8192^3: best of 10 (burst); back to back for 4 s (sustained)"}), flush=True)
 
 
 def run_sweep(args):
@@ -232,13 +336,51 @@ def run_sweep(args):
         ex.bind(dev)
         ops = ex.ops()
         assert len(ops) == (2 if args.sweep in ("dwpw", "stem") else 1)
+        # seeded images (the workload recipe), at most 8 distinct ones: image k of the batch is drawn image k % 8
+        n_img = min(b, 8)
+        xs_np = [wl.make_input(spec, images=list(range(n_img)), index=i) for i in range(len(spec.inputs))]
+
+        def to_device(x_np, layout):
+            x = torch.from_numpy(x_np).to(dev).half()
+            x = x.repeat((b + n_img - 1) // n_img, 1, 1, 1)[:b].contiguous()
+            return x if layout == api.GI_NHWC else to_phwc4(x)
+
+        def to_phwc4(x):  # layout only: [B,H,W,C] -> [S][B][plane][4], zero filled
+            B_, H_, W_, C_ = x.shape
+            S_, P_ = (C_ + 3) // 4, (H_ * W_ + 1) // 2 * 2
+            x = torch.nn.functional.pad(x.reshape(B_, H_ * W_, C_), (0, S_ * 4 - C_, 0, P_ - H_ * W_))
+            flat = x.reshape(B_, P_, S_, 4).permute(2, 0, 1, 3).contiguous().reshape(-1)
+            full = torch.zeros(api.gi_tensor_bytes(B_, H_, W_, C_) // 2, dtype=torch.float16, device=dev)
+            full[: flat.numel()] = flat
+            return full
+
+        def image_of(raw, t, img):  # one image of a PHWC4 tensor back as [1,H,W,C] fp32 on the host
+            H_, W_, C_ = spec.shapes[t]
+            S_, P_ = (C_ + 3) // 4, (H_ * W_ + 1) // 2 * 2
+            a = raw[: S_ * b * P_ * 4].reshape(S_, b, P_, 4)[:, img, : H_ * W_, :]
+            return a.permute(1, 0, 2).reshape(1, H_, W_, S_ * 4)[..., :C_].float().cpu().numpy()
+
         if args.sweep == "stem":  # the layout conversion must have been taken over by the convolution
             assert [api.KERNEL_NAMES[q.kernel] for q in ops] == ["none", "conv3x3_tc"], "this shape keeps its layout conversion"
-            ins = [(torch.rand((b,) + tuple(spec.shapes[t]), device=dev) * 2 - 1).half() for t in spec.inputs]
-        else:
-            ins = [(torch.rand(api.gi_tensor_bytes(b, *spec.shapes[t]) // 2, device=dev) * 2 - 1).half() for t in spec.inputs]
-        outs = [torch.empty(api.gi_tensor_bytes(b, *spec.shapes[t]) // 2, dtype=torch.float16, device=dev)
+        ins = [to_device(x, in_layout) for x in xs_np]
+        outs = [torch.full((api.gi_tensor_bytes(b, *spec.shapes[t]) // 2,), float("nan"), dtype=torch.float16, device=dev)
                 for t in spec.outputs]
+        checked, worst = False, None
+        if not args.no_check:
+            # what is timed below is first compared with the CPU oracle on sampled images (first and last of the batch)
+            from oracle import graph as og
+            ex.run(ins, outs, stream)
+            torch.cuda.synchronize()
+            sel = sorted({0, b - 1})
+            ref = og.run(spec, [x[[i % n_img for i in sel]] for x in xs_np], storage="f16", fused=True)
+            worst = 0.0
+            for t, o in zip(spec.outputs, outs):
+                for k, img in enumerate(sel):
+                    got, want = image_of(o, t, img), ref[t][k:k + 1]
+                    assert np.isfinite(got).all(), f"{name}: non-finite output"
+                    worst = max(worst, float((np.abs(got - want) / (1e-2 + 1e-2 * np.abs(want))).max()))
+            assert worst <= 1.0, f"{name}: disagrees with the oracle (normalised error {worst:.3f})"
+            checked = True
         for _ in range(3):
             ex.run(ins, outs, stream)
         ms = []
@@ -261,7 +403,8 @@ def run_sweep(args):
         row = {"op": name, "kernel": o.kernel, "ms": round(t, 5), "bytes": int(o.bytes),
                "flops": int(o.flops), "gbs": round(o.bytes / t / 1e6, 1), "tflops": round(o.flops / t / 1e9, 2),
                "bound": "tensor" if t_tc > t_hbm else "hbm", "frac_of_roofline": round(max(t_hbm, t_tc) / t, 4),
-               "peak_source": peak_kind,
+               "peak_source": peak_kind, "checked": checked,
+               "max_error_over_tolerance": None if worst is None else round(worst, 4),
                # the operator's tensors would fit in L2 (126 MB), but the untimed flush before each launch evicts
                # them: the inputs of every timed launch come from DRAM, only the output may still sit in L2 at the end
                "smaller_than_l2": bool(o.bytes < 126e6), "inputs_from": "dram (L2 flushed before each timed launch)"}
@@ -273,6 +416,29 @@ def run_sweep(args):
             for r in rows:
                 fh.write(f"{r['op']} | {r['kernel']} | {r['ms']} | {r['gbs']} | {r['tflops']} | {r['bound']} | "
                          f"{r['frac_of_roofline']}\n")
+
+
+def run_host_check(args):
+    """The multi-rank plumbing without a GPU: rank and world size from the launcher's environment, a gloo group,
+    the batch shard of this rank, and the whole-job throughput from the slowest rank's (synthetic) time."""
+    import torch.distributed as dist
+    from paper_1907_01989_b200 import workloads as wl
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    images = shard_images(rank, 3)
+    x = wl.make_input(wl.separable_block(3), images=images)
+    value, total_ms = job_throughput(100.0 + 10.0 * rank, 3, 4, world, dist, "cpu")
+    gathered = [None] * world
+    if world > 1:
+        dist.all_gather_object(gathered, (images, float(x.sum())))
+    else:
+        gathered = [(images, float(x.sum()))]
+    if rank == 0:
+        print(json.dumps({"host_check": True, "n_gpus": world, "value": value, "total_ms": total_ms, "shards": gathered}), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
 
 
 def main():
@@ -296,18 +462,36 @@ def main():
                     "'B,HW,Cout;...' (stem: 3x3 stride-2 convolution of a 3-channel NHWC input, read in that layout)")
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--residual", action="store_true")
+    ap.add_argument("--no-check", action="store_true", help="sweep: skip the comparison of sampled images with the CPU oracle")
+    ap.add_argument("--budget-s", type=float, default=None, help="--impl reference: seconds of oracle work per step")
+    ap.add_argument("--sustained-s", type=float, default=3.0, help="device seconds of the sustained legs (0: skip them)")
+    ap.add_argument("--host-check", action="store_true",
+                    help="no GPU work: every rank joins a gloo group, takes its shard of the batch and the ranks reduce a "
+                         "synthetic per-rank time with the same max-over-ranks code the timed run uses (tests the N > 1 plumbing)")
+    ap.add_argument("--fp16-peak", action="store_true", help="measure the dense fp16 matmul peak (burst and sustained) and exit")
     ap.add_argument("--out", default=None)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.batch is None:
         args.batch = 16 if args.net == "seg" else 256
 
+    if args.fp16_peak:
+        measure_fp16_peak()
+        return
     if args.sweep:
         run_sweep(args)
         return
+    # started as plain `python bench.py --gpus N`: start the N ranks here (one process per GPU)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(respawn_under_torchrun(args.gpus))
+    if "WORLD_SIZE" in os.environ and int(os.environ["WORLD_SIZE"]) != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={os.environ['WORLD_SIZE']}: launch one rank per GPU")
     from paper_1907_01989_b200 import workloads as wl
     fn_name, label = NETS[args.net]
     spec_fn = getattr(wl, fn_name)
+    if args.host_check:
+        run_host_check(args)
+        return
     if args.impl == "reference":
         run_reference(args, spec_fn, label)
         return
@@ -404,6 +588,55 @@ def main():
     e2e_graph_value = time_e2e(True) if world == 1 else None
     logits_checksum = float(out_pin.float().abs().mean())
 
+    # ---- sustained: the same step, and the same host pipeline, for seconds instead of a burst of K steps ----
+    sustained = None
+    if args.sustained_s > 0:
+        chunk = max(1, int(40.0 / max(ms_per_step, 0.05)))  # about 40 ms of device time between synchronisations
+
+        def chunk_back_to_back():
+            a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(chunk):
+                step_resident()
+            z.record(stream)
+            z.synchronize()
+            return a.elapsed_time(z)
+
+        def chunk_flushed():
+            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(chunk)]
+            for a, z in ev:
+                flush.zero_()
+                a.record(stream)
+                step_resident()
+                z.record(stream)
+            ev[-1][1].synchronize()
+            return sum(a.elapsed_time(z) for a, z in ev)
+
+        pipe_s = HostPipeline(ex, [tuple(x_dev.shape)], [tuple(out_dev.shape)], torch.float16, dev, graphs=False)
+        for _ in range(3):
+            pipe_s.submit([x_pin], [out_pin])
+        pipe_s.synchronize()
+
+        def chunk_e2e():
+            a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            pipe_s.copy.wait_event(a)
+            for _ in range(chunk):
+                pipe_s.submit([x_pin], [out_pin])
+            z.record(stream)
+            pipe_s.synchronize()
+            return a.elapsed_time(z)
+
+        barrier()
+        sustained = {"protocol": f"steps back to back in chunks of {chunk} (one synchronisation per chunk) until "
+                                 f"{args.sustained_s:g} s of device time; SM clock sampled every 20 ms; rank 0's replica",
+                     "back_to_back": sustained_leg(torch, stream, chunk_back_to_back, chunk * args.batch, local, args.sustained_s),
+                     "l2_flushed_between_steps": sustained_leg(torch, stream, chunk_flushed, chunk * args.batch, local, args.sustained_s),
+                     "e2e_host_buffers": sustained_leg(torch, stream, chunk_e2e, chunk * args.batch, local, args.sustained_s)}
+        for leg in ("back_to_back", "l2_flushed_between_steps", "e2e_host_buffers"):
+            sustained[leg]["steps"] = int(round(sustained[leg]["images_per_s"] * sustained[leg]["device_seconds"] / args.batch))
+        barrier()
+
     # ---- per-op times for the roofline (rank 0) ---------------------------------------------
     line = None
     if rank == 0:
@@ -449,6 +682,14 @@ def main():
         # to algorithmic bytes, see profiles/), which is valid because its traffic grows with the tensor
         ratio = NCU_DRAM_TO_ALGORITHMIC.get(top_name)
         traffic = None if ratio is None else ratio * top["bytes"] / top["launches"]
+        # the whole step against the sum of its ops' roofline times: free of the per-launch event overhead below
+        step_roof_ms = sum(f["roof_ms"] for f in fam.values())
+        roofline["step_frac"] = step_roof_ms / ms_per_step
+        roofline["step_roofline_ms"] = round(step_roof_ms, 4)
+        roofline["per_kernel_note"] = ("per-kernel times come from gi_run_timed, one event pair per launch: a launch then cannot "
+                                       "overlap its predecessor's tail as it does in the timed step, so they sum to "
+                                       f"{total_op_ms:.3f} ms against a {ms_per_step:.3f} ms step and the per-kernel fractions "
+                                       "are lower bounds; step_frac has neither problem")
         roofline.update({"traffic": traffic, "traffic_source": None if ratio is None else
                          f"ncu capture of a smaller case x {ratio} (dram bytes / algorithmic bytes), mean per launch",
                          "kernel": top_name, "launches_per_step": top["launches"],
@@ -552,7 +793,7 @@ def main():
                         "h2d_bytes_per_step": int(x_pin.numel() * 2),
                         "d2h_bytes_per_step": int(out_pin.numel() * 2)},
                 "gpu_launches": args.steps * n_launch, "clocks": clocks,
-                "cuda_graph_step": graph_step,
+                "cuda_graph_step": graph_step, "sustained": sustained,
                 "batch1": {"ms": b1_ms, "cuda_graph_ms": graph_ms, "launches": b1_launches,
                            "protocol": "10 warm-up runs, mean of the next 100"},
                 "step_ms_min_median_max": [min(ms), statistics.median(ms), max(ms)], "wall_s_timed_region": wall,

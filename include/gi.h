@@ -96,8 +96,8 @@ enum {
 };
 
 /* Cross-operator kernels: a depthwise 3x3 convolution whose only consumer is a 1x1 convolution runs
- * with it as one kernel, so the tensor between them never reaches memory (fp16 storage; Section 3.3
- * folds element-wise operators into their producer, this folds a whole operator).  Results are
+ * with it as one kernel, so the tensor between them never reaches memory (fp16 storage; the "Shader Program
+ * Optimization" paragraph of Section 3.2 folds element-wise operators into their producer, this folds a whole operator).  Results are
  * those of the two operators run one after the other: the tensor between them is still rounded to
  * fp16.  The memory plan is not affected: the tensor keeps its place in the arena, unused; a pair whose input
  * and output the planner placed on the same bytes (legal for two ops, not for one kernel) stays two kernels. */
@@ -204,8 +204,10 @@ GI_API gi_status gi_graph_input(gi_graph* g, int32_t H, int32_t W, int32_t C, in
 
 /* Append an operator; its inputs must already exist, so insertion order is a topological
  * order (Section 5 sorts topologically; here the order is given and verified).  *out
- * receives the id of its single output tensor.  GI_E_UNSUPPORTED for kernels other than
- * 1x1 / 3x3 (full) or 3x3 (depthwise), GI_E_INVALID for shape or id errors. */
+ * receives the id of its single output tensor.  GI_E_UNSUPPORTED for kernels other than square
+ * 1x1, 2x2 or 3x3 (full convolution, strides 1 to 3) or 3x3 (depthwise, strides 1 or 2), GI_E_INVALID
+ * for shape or id errors, GI_E_NOMEM if the copies of weights and bias cannot be allocated (the graph is
+ * then unchanged). */
 GI_API gi_status gi_add_op(gi_graph* g, const gi_op_desc* desc, gi_tensor* out);
 
 /* Mark a tensor as graph output, delivered to the caller's buffer in `layout`.  Outputs are
@@ -242,8 +244,12 @@ GI_API gi_status gi_exec_bind(gi_exec* e, void* dev_weights, size_t weight_bytes
  * dev_outputs[i] are device pointers for input / output i in their declared layouts;
  * dev_arena holds the intermediates (>= info.arena_bytes).  Nothing is launched if an
  * argument check fails (GI_E_INVALID, GI_E_ARENA, GI_E_STATE).  Two runs of one executable
- * may overlap only if they use different arenas and outputs.  Results are deterministic:
- * the same inputs give bit-identical outputs. */
+ * may overlap on the GPU only if they use different arenas and outputs; several host threads may then
+ * call gi_run on that executable at the same time (the per-executable cache of tensor maps is guarded,
+ * and keeps the maps of the last four distinct input addresses per launch, so alternating between a
+ * few arenas or input buffers re-encodes nothing).  gi_exec_bind and gi_exec_destroy must not run
+ * concurrently with gi_run on the same executable.  Results are deterministic: the same inputs give
+ * bit-identical outputs. */
 GI_API gi_status gi_run(gi_exec* e, const void* const* dev_inputs, void* const* dev_outputs, void* dev_arena,
                  size_t arena_bytes, void* stream);
 

@@ -582,7 +582,8 @@ constexpr int kSmemPerSm = 226 * 1024;
 
 }  // namespace
 
-int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
+// `dry_run`: stop after the geometry has been derived and checked, before anything that touches the device
+static int depthwise_f16_impl(const LaunchRec& r, const Ptrs& p, void* stream, bool dry_run) {
   DwGeom g;
   g.B = r.B;
   g.H = r.H;
@@ -664,6 +665,7 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
   const long long items = static_cast<long long>(g.S) * g.bchunks * g.bands;
   if (items > 2147483647LL) return static_cast<int>(cudaErrorInvalidConfiguration);
   g.items = static_cast<int>(items);
+  if (dry_run) return 0;
   int threads = (g.nb * g.sub * wcols + 31) / 32 * 32;
   if (threads > 256) threads = 256;
   if (threads < 32) threads = 32;
@@ -739,6 +741,16 @@ int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) {
 #undef GI_DW_LAUNCH
 #undef GI_DW_LAUNCH2
   return static_cast<int>(cudaGetLastError());
+}
+
+int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream) { return depthwise_f16_impl(r, p, stream, false); }
+
+// Host-only: the staged stencil can run this shape (its staging buffers fit shared memory, its work items an
+// int).  Decided once at compile time; shapes it cannot run (rows thousands of pixels wide) take the plain
+// one-thread-per-pixel kernel instead of failing in the middle of a run.
+bool depthwise_f16_supported(const LaunchRec& r) {
+  if (r.sh != r.sw || r.dh != r.dw) return false;
+  return depthwise_f16_impl(r, Ptrs{}, nullptr, true) == 0;
 }
 
 unsigned int depthwise_error_word(int* cuda_err) {

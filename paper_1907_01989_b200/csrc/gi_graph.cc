@@ -110,8 +110,14 @@ gi_status gi_graph_input(gi_graph* g, int32_t H, int32_t W, int32_t C, int32_t l
   t.c = C;
   t.input_index = static_cast<int>(g->inputs.size());
   t.input_layout = layout;
-  g->tensors.push_back(t);
-  g->inputs.push_back(static_cast<int>(g->tensors.size()) - 1);
+  const size_t nt = g->tensors.size();
+  try {
+    g->tensors.push_back(t);
+    g->inputs.push_back(static_cast<int>(nt));
+  } catch (const std::bad_alloc&) {
+    g->tensors.resize(nt);
+    return fail(GI_E_NOMEM, "gi_graph_input: out of host memory");
+  }
   *out = g->inputs.back();
   return GI_OK;
 }
@@ -123,14 +129,18 @@ gi_status gi_graph_output(gi_graph* g, gi_tensor t, int32_t layout) {
   TensorDesc& d = g->tensors[t];
   if (d.input_index >= 0) return fail(GI_E_INVALID, "gi_graph_output: a graph input cannot be an output");
   if (d.output_index >= 0) return fail(GI_E_INVALID, "gi_graph_output: tensor is already an output");
-  d.output_index = static_cast<int>(g->outputs.size());
+  try {
+    g->outputs.push_back(t);
+  } catch (const std::bad_alloc&) {
+    return fail(GI_E_NOMEM, "gi_graph_output: out of host memory");
+  }
+  d.output_index = static_cast<int>(g->outputs.size()) - 1;
   d.output_layout = layout;
-  g->outputs.push_back(t);
   return GI_OK;
 }
 
-gi_status gi_add_op(gi_graph* g, const gi_op_desc* desc, gi_tensor* out) {
-  if (!g || !desc || !out) return fail(GI_E_INVALID, "gi_add_op: null argument");
+// gi_add_op proper; may throw std::bad_alloc (the exported wrapper below turns that into GI_E_NOMEM)
+static gi_status add_op_checked(gi_graph* g, const gi_op_desc* desc, gi_tensor* out) {
   const int nt = static_cast<int>(g->tensors.size());
   auto known = [&](int t) { return t >= 0 && t < nt; };
   if (!known(desc->inputs[0])) return fail(GI_E_INVALID, "gi_add_op: inputs[0] is not a tensor of this graph");
@@ -238,14 +248,27 @@ gi_status gi_add_op(gi_graph* g, const gi_op_desc* desc, gi_tensor* out) {
   if (static_cast<uint64_t>(o.h) * o.w > (1u << 28)) return fail(GI_E_UNSUPPORTED, "gi_add_op: output plane too large");
   g->tensors.push_back(o);
   node.output = static_cast<int>(g->tensors.size()) - 1;
-  try {
-    g->ops.push_back(std::move(node));
-  } catch (const std::bad_alloc&) {
-    g->tensors.pop_back();
-    return fail(GI_E_NOMEM, "gi_add_op: out of host memory");
-  }
+  g->ops.push_back(std::move(node));
   *out = g->ops.back().output;
   return GI_OK;
+}
+
+gi_status gi_add_op(gi_graph* g, const gi_op_desc* desc, gi_tensor* out) {
+  if (!g || !desc || !out) return fail(GI_E_INVALID, "gi_add_op: null argument");
+  // no exception may cross the C boundary: whatever the copies of weights and bias or the growth of the
+  // graph's vectors throw, the graph is left as it was before the call
+  const size_t n_tensors = g->tensors.size(), n_ops = g->ops.size();
+  try {
+    return add_op_checked(g, desc, out);
+  } catch (const std::bad_alloc&) {
+    g->tensors.resize(n_tensors);
+    g->ops.resize(n_ops);
+    return fail(GI_E_NOMEM, "gi_add_op: out of host memory");
+  } catch (...) {
+    g->tensors.resize(n_tensors);
+    g->ops.resize(n_ops);
+    return fail(GI_E_NOMEM, "gi_add_op: unexpected host failure");
+  }
 }
 
 }  // extern "C"

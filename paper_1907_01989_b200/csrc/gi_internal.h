@@ -69,6 +69,8 @@ struct LaunchRec {
   // with the "evict first" L2 policy, which keeps this op's output - the next op's input - resident
   // instead (MobileNetV2 at batch 256: 1.756 -> 1.728 ms, measured in one run on one GPU)
   int in0_dead = 0;
+  // depthwise: 1 = the shared-memory staged fp16 stencil runs this op, 0 = the plain one-thread-per-pixel kernel
+  int dw_staged = 0;
   // the stem convolution reads the caller's NHWC input itself; the layout conversion in front of it launches nothing
   int nhwc_in = 0;
   // depthwise + pointwise as one kernel: the 1x1 convolution's weights, bias, output channels and epilogue

@@ -211,6 +211,10 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
           info.bytes = 0;
         } else if (f.kind == GI_OP_DEPTHWISE_CONV2D) {
           r.kernel = GI_KERNEL_DEPTHWISE;
+          r.C = din->c;
+          r.dw_staged = e->storage == GI_F16 && depthwise_f16_supported(r);
+          if (!r.dw_staged && e->batch > 65535)
+            return fail(GI_E_UNSUPPORTED, "gi_compile: depthwise convolution: batch above 65535 with a shape only the plain kernel runs");
           pack_depthwise(op, din->c, e->storage, &e->weight_blob, &r);
           info.bytes += taps * din->c * eb;
           info.flops = 2 * taps * out_px * din->c;

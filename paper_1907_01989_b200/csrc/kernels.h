@@ -32,6 +32,7 @@ int launch_conv_simt(const LaunchRec& r, const Ptrs& p, int storage, void* strea
 int launch_depthwise(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
 // fp16 storage, equal strides / dilations on both axes: shared-memory staged stencil
 int launch_depthwise_f16(const LaunchRec& r, const Ptrs& p, void* stream);
+bool depthwise_f16_supported(const LaunchRec& r);  // host-only check, used when the op is lowered
 unsigned int depthwise_error_word(int* cuda_err);
 int launch_eltwise(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
 int launch_concat(const LaunchRec& r, const Ptrs& p, int storage, void* stream);

@@ -529,7 +529,7 @@ int launch_conv_simt(const LaunchRec& r, const Ptrs& p, int storage, void* strea
 
 int launch_depthwise(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (storage == GI_F16 && r.sh == r.sw && r.dh == r.dw) return launch_depthwise_f16(r, p, stream);
+  if (r.dw_staged) return launch_depthwise_f16(r, p, stream);
   if (r.B > 65535) return static_cast<int>(cudaErrorInvalidConfiguration);
   const ConvGeom g = geom(r);
   const dim3 grid(blocks_for(g.Pout, 128), g.Sout, r.B);

@@ -427,11 +427,12 @@ int launch_pointwise_tc(const LaunchRec& r, const Ptrs& p, void** state, int lau
     di.attr_set = true;
   }
   // tensor map over the input: pixels (8-byte elements) x slices; cached per launch and input address
-  MapEntry& me = map_cache_entry(state, launch_index);
-  if (me.in != p.in0) {
-    const int err = encode_plane_map(&me.map, p.in0, m_total, t.s_in, kTilePx, t.kc);
+  CUtensorMap tmap;
+  {
+    const int err = map_cache_lookup(state, launch_index, p.in0, &tmap, [&](CUtensorMap* m) {
+      return encode_plane_map(m, p.in0, m_total, t.s_in, kTilePx, t.kc);
+    });
     if (err != 0) return err;
-    me.in = p.in0;
   }
   TcParams k;
   k.res = static_cast<const __half*>(p.res);
@@ -493,7 +494,7 @@ int launch_pointwise_tc(const LaunchRec& r, const Ptrs& p, void** state, int lau
   const unsigned threads = 64u + 128u * k.epq;
   const bool tail = k.has_res || k.act_post != GI_ACT_NONE;
   cudaStream_t cu_stream = static_cast<cudaStream_t>(stream);
-#define GI_TC_LAUNCH(A, T) launch_pdl(pointwise_tc_kernel<A, T>, grid, threads, smem, cu_stream, me.map, k)
+#define GI_TC_LAUNCH(A, T) launch_pdl(pointwise_tc_kernel<A, T>, grid, threads, smem, cu_stream, tmap, k)
   if (tail) {
     if (k.act_pre == GI_ACT_RELU6) GI_TC_LAUNCH(GI_ACT_RELU6, true);
     else if (k.act_pre == GI_ACT_RELU) GI_TC_LAUNCH(GI_ACT_RELU, true);

@@ -515,11 +515,12 @@ int launch_pointwise_ts(const LaunchRec& r, const Ptrs& p, void** state, int lau
     if (e != cudaSuccess) return static_cast<int>(e);
     attr_set = true;
   }
-  MapEntry& me = map_cache_entry(state, launch_index);
-  if (me.in != p.in0) {
-    const int err = encode_plane_map(&me.map, p.in0, k.m_total_px, t.s_in, t.box_px, t.ks);
+  CUtensorMap tmap;
+  {
+    const int err = map_cache_lookup(state, launch_index, p.in0, &tmap, [&](CUtensorMap* m) {
+      return encode_plane_map(m, p.in0, k.m_total_px, t.s_in, t.box_px, t.ks);
+    });
     if (err != 0) return err;
-    me.in = p.in0;
   }
   // CTAs come in groups of n_parts (one per share of the output channels) that walk the pixel tiles together
   long long groups = sms / t.n_parts;
@@ -532,7 +533,7 @@ int launch_pointwise_ts(const LaunchRec& r, const Ptrs& p, void** state, int lau
   if (smem < 120 * 1024) smem = 120 * 1024;
   cudaStream_t cu_stream = static_cast<cudaStream_t>(stream);
   const int act = r.ep.act_pre;
-#define GI_TS_LAUNCH(A, T) launch_pdl(pointwise_ts_kernel<A, T>, grid, kThreads, smem, cu_stream, me.map, k)
+#define GI_TS_LAUNCH(A, T) launch_pdl(pointwise_ts_kernel<A, T>, grid, kThreads, smem, cu_stream, tmap, k)
   if (tail) {
     if (act == GI_ACT_RELU6) GI_TS_LAUNCH(GI_ACT_RELU6, true);
     else if (act == GI_ACT_RELU) GI_TS_LAUNCH(GI_ACT_RELU, true);

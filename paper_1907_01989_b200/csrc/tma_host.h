@@ -45,20 +45,56 @@ inline int encode_plane_map(CUtensorMap* map, const void* base, unsigned long lo
   return cr == CUDA_SUCCESS ? 0 : static_cast<int>(cudaErrorInvalidValue);
 }
 
-// Tensor maps depend on device addresses: one cached entry per launch of an executable, kept in
-// a cache the executable owns through an opaque pointer.
-struct MapEntry {
-  const void* in = nullptr;
-  CUtensorMap map;
+// Tensor maps depend on device addresses.  The cache an executable owns (through an opaque pointer) keeps, per
+// launch, the maps of the last few distinct input addresses: a caller that alternates between two arenas or two
+// input buffers (a two-slot pipeline, gi_run followed by gi_run_static) encodes each map once, not on every call.
+// Host threads may run one executable at the same time (with different arenas): the cache is guarded by a
+// mutex and a launcher works on its own copy of the map, never on the cached one.
+constexpr int kMapWays = 4;
+struct MapSlot {
+  const void* in[kMapWays] = {};
+  CUtensorMap map[kMapWays];
+  int used = 0, next = 0;
 };
 struct MapCache {
-  std::vector<MapEntry> maps;
+  std::mutex mu;
+  std::vector<MapSlot> slots;
 };
-inline MapEntry& map_cache_entry(void** state, int launch_index) {
+inline MapCache* map_cache(void** state) {
+  static std::mutex create_mu;
+  std::lock_guard<std::mutex> lock(create_mu);
   if (!*state) *state = new MapCache();
-  MapCache* c = static_cast<MapCache*>(*state);
-  if (c->maps.size() <= static_cast<size_t>(launch_index)) c->maps.resize(launch_index + 1);
-  return c->maps[launch_index];
+  return static_cast<MapCache*>(*state);
+}
+// Copies the map for (launch, input address) into *out, encoding it with `encode(CUtensorMap*) -> int` (a
+// cudaError_t, 0 on success) if it is not cached.  Returns that error code.
+template <typename Encode>
+inline int map_cache_lookup(void** state, int launch_index, const void* in, CUtensorMap* out, Encode&& encode) {
+  MapCache* c = map_cache(state);
+  std::lock_guard<std::mutex> lock(c->mu);
+  if (c->slots.size() <= static_cast<size_t>(launch_index)) c->slots.resize(launch_index + 1);
+  MapSlot& s = c->slots[launch_index];
+  for (int i = 0; i < s.used; ++i)
+    if (s.in[i] == in) {
+      *out = s.map[i];
+      return 0;
+    }
+  int way;
+  if (s.used < kMapWays) {
+    way = s.used;
+  } else {
+    way = s.next;
+    s.next = (s.next + 1) % kMapWays;
+  }
+  const int err = encode(&s.map[way]);
+  if (err != 0) {
+    if (way < s.used) s.in[way] = nullptr;  // the overwritten entry is gone
+    return err;
+  }
+  if (way == s.used) ++s.used;
+  s.in[way] = in;
+  *out = s.map[way];
+  return 0;
 }
 inline void map_cache_release(void* state) { delete static_cast<MapCache*>(state); }
 

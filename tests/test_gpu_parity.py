@@ -668,3 +668,88 @@ def test_fire_network_with_caller_owned_phwc4_buffers(cross_op):
         got = oops.phwc4_unpack(out.float().cpu().numpy(), 3, H, W, Cc)
         assert_close(got, og.run(spec, [xin], storage="f16")[spec.outputs[0]], api.GI_F16, "fire network, phwc4 io")
     assert api.gi_device_status() == 0
+
+
+# ---------------------------------------------------------------------- the single-operator sweep at the sizes it is timed at
+# Corners of the single-operator grid that `bench.py --sweep` times: the tensor-bound 1x1 shapes (streamed weights, tens of
+# K chunks, many output tiles per pixel tile), the deep and narrow 7x7 layers, the widest plane with a residual, and the
+# depthwise shapes at batch 64 / 256.  Every image of the batch is drawn; three sampled images (first, middle, last: the
+# last one lies in the ragged tail tile) are compared element by element with the oracle.
+SWEEP_PW_CASES = [(256, 14, 576, 576, False), (256, 14, 960, 960, False), (256, 14, 1280, 1280, False), (256, 7, 960, 160, False),
+                  (256, 7, 320, 1280, False), (256, 112, 16, 96, True), (64, 56, 192, 192, True), (8, 28, 384, 384, False)]
+SWEEP_DW_CASES = [(256, 112, 96, 1), (256, 112, 96, 2), (256, 14, 576, 2), (64, 7, 960, 1), (256, 28, 192, 1), (64, 56, 144, 2)]
+
+
+@pytest.mark.parametrize("case", SWEEP_PW_CASES, ids=lambda c: "b%d_%dx%d_%dto%d%s" % (c[0], c[1], c[1], c[2], c[3], "_res" if c[4] else ""))
+def test_sweep_pointwise_points_at_full_size(case):
+    b, hw, cin, cout, res = case
+    spec = wl.single_pointwise(b, hw, cin, cout, residual=res)
+    run, _, _ = check_outputs(spec, api.GI_F16, images=[0, b // 2 + 1, b - 1])
+    assert any(api.KERNEL_NAMES[o.kernel] in ("pointwise_tc", "pointwise_ts") for o in run.ex.ops())
+    assert api.gi_device_status() == 0
+
+
+@pytest.mark.parametrize("mode", [api.GI_PW_TC_PAIR, api.GI_PW_TC_LANE], ids=["pair", "lane"])
+@pytest.mark.parametrize("case", [(256, 14, 576, 576), (64, 14, 1280, 1280)], ids=["576", "1280"])
+def test_sweep_tensor_bound_points_both_variants(case, mode):
+    b, hw, cin, cout = case
+    check_outputs(wl.single_pointwise(b, hw, cin, cout), api.GI_F16, images=[0, b - 1], pointwise=mode)
+
+
+@pytest.mark.parametrize("case", SWEEP_DW_CASES, ids=lambda c: "b%d_%dx%dx%d_s%d" % (c[0], c[1], c[1], c[2], c[3]))
+def test_sweep_depthwise_points_at_full_size(case):
+    b, hw, c, stride = case
+    spec = wl.single_depthwise(b, hw, c, stride, 1)
+    run, _, _ = check_outputs(spec, api.GI_F16, images=[0, b // 2 + 1, b - 1])
+    assert "depthwise" in [api.KERNEL_NAMES[o.kernel] for o in run.ex.ops()]
+    assert api.gi_device_status() == 0
+
+
+# ---------------------------------------------------------------------- one executable, several host threads / several arenas
+def test_two_threads_run_one_executable_with_their_own_arenas():
+    """gi_run may be called on one executable from several host threads as long as the runs use different arenas
+    and outputs; and a single thread that alternates between arenas gets the same answers every time."""
+    import threading
+    import torch
+    spec = wl.mobilenet_v2(2, size=96)
+    x_np = wl.make_input(spec)
+    ref = og.run(spec, [x_np], storage="f16")[spec.outputs[0]]
+    g, _ = api.graph_from_spec(spec, api.GI_F16)
+    ex = g.compile()
+    ex.bind("cuda:0")
+    nb = max(int(ex.info.arena_bytes), 256)
+    x = torch.from_numpy(x_np).to("cuda:0").half().contiguous()
+    out_shape = (spec.batch,) + tuple(spec.shapes[spec.outputs[0]])
+    n_threads, rounds = 3, 8
+    arenas = [torch.full((nb,), 0xFF, dtype=torch.uint8, device="cuda:0") for _ in range(n_threads)]
+    outs = [torch.zeros(out_shape, dtype=torch.float16, device="cuda:0") for _ in range(n_threads)]
+    streams = [torch.cuda.Stream() for _ in range(n_threads)]
+    torch.cuda.synchronize()
+    errors = []
+
+    def work(i):
+        try:
+            for _ in range(rounds):
+                ex.run_raw([x.data_ptr()], [outs[i].data_ptr()], arenas[i].data_ptr(), nb, streams[i])
+            streams[i].synchronize()
+        except Exception as exc:  # reported by the main thread
+            errors.append(exc)
+
+    threads = [threading.Thread(target=work, args=(i,)) for i in range(n_threads)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    torch.cuda.synchronize()
+    assert not errors, errors
+    first = outs[0].float().cpu().numpy()
+    assert_close(first, ref, api.GI_F16, "threaded run")
+    for o in outs[1:]:
+        assert np.array_equal(o.float().cpu().numpy(), first)
+    # one thread, alternating arenas
+    for k in range(6):
+        outs[k % 2].zero_()
+        ex.run_raw([x.data_ptr()], [outs[k % 2].data_ptr()], arenas[k % 3].data_ptr(), nb)
+        torch.cuda.synchronize()
+        assert np.array_equal(outs[k % 2].float().cpu().numpy(), first)
+    assert api.gi_device_status() == 0

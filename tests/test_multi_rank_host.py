@@ -62,6 +62,31 @@ def test_two_rank_sharding_and_max_reduction():
     assert np.isclose(gathered[0][1], float(full[:3].sum())) and np.isclose(gathered[1][1], float(full[3:].sum()))
 
 
+def test_bench_gpus_2_starts_its_own_ranks():
+    """`python bench.py --gpus 2` outside torchrun must start two ranks itself.  Run here without a GPU: each rank
+    joins a gloo group, takes its shard and the ranks reduce with the timed run's own max-over-ranks code."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--host-check"], env=env, cwd=ROOT,
+                       capture_output=True, text=True, timeout=300)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [json.loads(ln) for ln in p.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1                       # rank 0 alone prints
+    line = lines[0]
+    assert line["n_gpus"] == 2 and line["total_ms"] == 110.0
+    assert abs(line["value"] - 2 * 3 * 4 / 0.110) < 1e-6
+    assert [g[0] for g in line["shards"]] == [[0, 1, 2], [3, 4, 5]]
+
+
+def test_bench_refuses_a_world_size_that_contradicts_gpus():
+    import subprocess
+    env = dict(os.environ, WORLD_SIZE="2", RANK="0")
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "4", "--host-check"], env=env, cwd=ROOT,
+                       capture_output=True, text=True, timeout=120)
+    assert p.returncode != 0 and "WORLD_SIZE" in (p.stderr + p.stdout)
+
+
 def test_single_rank_needs_no_process_group():
     import bench
     value, total_ms = bench.job_throughput(50.0, 8, 2, 1, None, "cpu")

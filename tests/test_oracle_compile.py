@@ -27,10 +27,10 @@ def hand_example(t3=20):
     return problem(ops, {0: 10, 1: 40, 2: 3, 3: t3})
 
 
-# ---------------------------------------------------------------------- Table 4
-def _table4():
+# ---------------------------------------------------------------------- the memory table of Section 5
+def _memory_table():
     rows = {}
-    with open(os.path.join(GOLDEN, "table4_memory.txt")) as fh:
+    with open(os.path.join(GOLDEN, "section5_memory_table.txt")) as fh:
         for line in fh:
             if line.strip() and not line.startswith("#"):
                 k, v1, v2 = line.split()
@@ -38,11 +38,11 @@ def _table4():
     return rows
 
 
-def test_table4_memory_totals():
+def test_section5_memory_table_totals():
     """Algorithm 1 and the naive strategy reproduce the paper's printed totals for MobileNet v1 and
     MobileNetV2.  This pins 'outputs get their object before inputs are released' (the opposite
     order gives 1.53 for v1) and 'the pool is used whenever it is not empty, growing the object'."""
-    t4 = _table4()
+    t4 = _memory_table()
     for col, (g, fold_add) in enumerate(((wl.mobilenet_v1(1), True), (wl.mobilenet_v2(1), False))):
         fused = oc.fuse(g, fold_add=fold_add)
         p = oc.plan_problem(g, fused, elem_bytes=2, align=1, convert_io=False)
@@ -55,8 +55,8 @@ def test_table4_memory_totals():
         assert round(mcfp, 1) == t4["mcfp"][col]
 
 
-def test_release_before_allocate_would_not_match_table4():
-    # the other reading of Algorithm 1's order, kept here only to show Table 4 tells them apart
+def test_release_before_allocate_would_not_match_the_memory_table():
+    # the other reading of Algorithm 1's order, kept here only to show that the memory table of Section 5 tells them apart
     g = wl.mobilenet_v1(1)
     p = oc.plan_problem(g, oc.fuse(g), 2, 1, convert_io=False)
     life = oc.lifetimes(p)

@@ -44,10 +44,13 @@ def np_eval(g, x):
             y = a.mean(axis=(1, 2), keepdims=True)
         elif op.kind == "resize_bilinear":
             oh, ow = op.out_hw
-            assert op.align_corners
             H, W = a.shape[1:3]
-            fy = np.arange(oh) * (H - 1) / (oh - 1)
-            fx = np.arange(ow) * (W - 1) / (ow - 1)
+            if op.align_corners:  # the corner samples of input and output coincide
+                fy = np.linspace(0.0, H - 1.0, oh) if oh > 1 else np.zeros(1)
+                fx = np.linspace(0.0, W - 1.0, ow) if ow > 1 else np.zeros(1)
+            else:                 # output sample o sits at o / out of the way along the input's extent
+                fy = np.arange(oh) / oh * H
+                fx = np.arange(ow) / ow * W
             y0 = np.minimum(np.floor(fy).astype(int), H - 1)
             x0 = np.minimum(np.floor(fx).astype(int), W - 1)
             y1, x1 = np.minimum(y0 + 1, H - 1), np.minimum(x0 + 1, W - 1)
@@ -61,6 +64,20 @@ def np_eval(g, x):
     return val
 
 
+def resize_chain():
+    """Bilinear resizes in both corner conventions, up and down, with H != W and odd factors."""
+    b = wl.GraphBuilder("resize_chain", 2, 61)
+    x = b.input(9, 7, 5)
+    y = b.conv2d(x, 6, 1)
+    y = b.resize_bilinear(y, 23, 10, False)
+    y = b.activation(b.depthwise(y, 3, 1), wl.ACT_RELU6)
+    y = b.resize_bilinear(y, 7, 25, False)
+    y = b.resize_bilinear(y, 15, 9, True)
+    y = b.resize_bilinear(y, 30, 4, False)
+    b.output(y)
+    return b.finish()
+
+
 NETS = [
     ("separable_block", lambda: wl.separable_block(2)),
     ("mobilenet_v1", lambda: wl.mobilenet_v1(1, size=96)),
@@ -68,6 +85,7 @@ NETS = [
     ("segmentation", lambda: wl.mobilenet_v2_segmentation(1, size=65)),
     ("fire_network", lambda: wl.fire_network(2)),
     ("fire_network_odd", lambda: wl.fire_network(1, size=77)),
+    ("resize_both_corner_conventions", lambda: resize_chain()),
 ]
 
 

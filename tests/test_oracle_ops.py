@@ -218,6 +218,44 @@ def test_bilinear_constant_ramp_and_samples():
                                atol=1e-7)
 
 
+def test_bilinear_without_align_corners_closed_forms():
+    """Corner convention 0 (src = o * in / out, no half-pixel shift) against closed forms that do not
+    repeat that expression.  Each fails for the two plausible misreadings, a scale of (in-1)/(out-1)
+    and half-pixel centres."""
+    x = RNG.standard_normal(7).astype(np.float32)
+    # exact 2x up-sampling along W: even outputs are the samples, odd ones the mean of two neighbours,
+    # the last one repeats the last sample (its right neighbour is clamped)
+    col = x[None, None, :, None]
+    up = ops.resize_bilinear(col, 1, 14, False)[0, 0, :, 0]
+    assert np.array_equal(up[0::2], x)
+    np.testing.assert_allclose(up[1:-1:2], (x[:-1].astype(np.float64) + x[1:]) / 2, rtol=1e-6, atol=1e-7)
+    assert up[-1] == x[-1]
+    # the same along H (a transposed scale or axis would show here: H and W differ)
+    row = x[None, :, None, None]
+    up = ops.resize_bilinear(np.repeat(row, 3, axis=2), 14, 3, False)[0, :, :, 0]
+    for w in range(3):
+        assert np.array_equal(up[0::2, w], x)
+        np.testing.assert_allclose(up[1:-1:2, w], (x[:-1].astype(np.float64) + x[1:]) / 2, rtol=1e-6, atol=1e-7)
+        assert up[-1, w] == x[-1]
+    # exact 2x down-sampling picks every second sample
+    y = RNG.standard_normal((2, 8, 6, 3)).astype(np.float32)
+    assert np.array_equal(ops.resize_bilinear(y, 4, 3, False), y[:, ::2, ::2, :])
+    # a linear ramp of 5 samples resized to 13: the ramp evaluated at min(o * 5/13, 4)
+    ramp = (0.75 * np.arange(5, dtype=np.float64) - 1.5)
+    got = ops.resize_bilinear(ramp.astype(np.float32)[None, None, :, None], 1, 13, False)[0, 0, :, 0]
+    want = 0.75 * np.minimum(np.arange(13) * 5.0 / 13.0, 4.0) - 1.5
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-6)
+    got = ops.resize_bilinear(ramp.astype(np.float32)[None, :, None, None], 13, 1, False)[0, :, 0, 0]
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-6)
+    # and both axes at once, different sizes: 5x3 -> 13x4
+    yy, xx = np.meshgrid(np.arange(5, dtype=np.float64), np.arange(3, dtype=np.float64), indexing="ij")
+    plane = (0.5 * yy - 2.0 * xx + 0.25)
+    got = ops.resize_bilinear(plane.astype(np.float32)[None, :, :, None], 13, 4, False)[0, :, :, 0]
+    sy = np.minimum(np.arange(13) * 5.0 / 13.0, 4.0)[:, None]
+    sx = np.minimum(np.arange(4) * 3.0 / 4.0, 2.0)[None, :]
+    np.testing.assert_allclose(got, 0.5 * sy - 2.0 * sx + 0.25, rtol=0, atol=1e-6)
+
+
 # ---------------------------------------------------------------------- fp16 rounding
 def test_f16_rounding_matches_numpy_everywhere_it_matters():
     # all 65536 half patterns round-trip
