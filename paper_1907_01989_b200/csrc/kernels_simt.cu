@@ -66,24 +66,26 @@ __device__ __forceinline__ float4 epilogue(float4 v, const Epilogue& ep, const T
 }
 
 // ------------------------------------------------------------------ layout conversion
-// grid: x over the pixels of a plane (padding pixel included), y over planes (slice * B + image)
+// grid: x over the pixels of a plane (padding pixel included), y strides over planes (slice * B + image; a grid
+// dimension holds at most 65535, deep tensors at large batch have more planes than that)
 template <typename T>
 __global__ void pack_kernel(const T* __restrict__ nhwc, T* __restrict__ out, int B, int HW, int C, int P, int S) {
   pdl_launch_dependents();
   pdl_wait();
   const int pix = blockIdx.x * blockDim.x + threadIdx.x;
   if (pix >= P) return;
-  const int plane = blockIdx.y;
-  const int s = plane / B, b = plane - s * B;
-  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (pix < HW) {
-    const T* src = nhwc + (static_cast<size_t>(b) * HW + pix) * C + s * 4;
-    const int n = min(4, C - s * 4);
-    float t[4] = {0.f, 0.f, 0.f, 0.f};
-    for (int j = 0; j < n; ++j) t[j] = Px<T>::get(src + j);
-    v = make_float4(t[0], t[1], t[2], t[3]);
+  for (int plane = blockIdx.y; plane < S * B; plane += gridDim.y) {
+    const int s = plane / B, b = plane - s * B;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (pix < HW) {
+      const T* src = nhwc + (static_cast<size_t>(b) * HW + pix) * C + s * 4;
+      const int n = min(4, C - s * 4);
+      float t[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int j = 0; j < n; ++j) t[j] = Px<T>::get(src + j);
+      v = make_float4(t[0], t[1], t[2], t[3]);
+    }
+    Px<T>::store(out + (static_cast<size_t>(plane) * P + pix) * 4, v);
   }
-  Px<T>::store(out + (static_cast<size_t>(plane) * P + pix) * 4, v);
 }
 
 // fp16 images with 3 channels (the usual network input) whose pixel count is a multiple of 4:
@@ -470,7 +472,6 @@ inline unsigned blocks_for(size_t n, unsigned per) { return static_cast<unsigned
 int launch_pack(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int S = slices(r.C), P = plane_pixels(r.H, r.W), HW = r.H * r.W;
-  if (static_cast<long long>(S) * r.B > 65535) return static_cast<int>(cudaErrorInvalidConfiguration);
   if (storage == GI_F16 && r.C == 3 && HW % 4 == 0 && r.B <= 65535) {
     // P == HW here (no padding pixel), one slice: the planes of the images are back to back
     const int quads = HW / 4;
@@ -478,7 +479,9 @@ int launch_pack(const LaunchRec& r, const Ptrs& p, int storage, void* stream) {
                static_cast<uint4*>(p.out), quads);
     return static_cast<int>(cudaGetLastError());
   }
-  const dim3 grid(blocks_for(P, 256), S * r.B);
+  const long long planes = static_cast<long long>(S) * r.B;
+  if (planes > 2147483647LL) return static_cast<int>(cudaErrorInvalidConfiguration);
+  const dim3 grid(blocks_for(P, 256), static_cast<unsigned>(planes < 65535 ? planes : 65535));
   GI_BY_STORAGE((launch_pdl(pack_kernel<__half>, grid, 256, 0, st, static_cast<const __half*>(p.in0), static_cast<__half*>(p.out),
                             r.B, HW, r.C, P, S)),
                 (launch_pdl(pack_kernel<float>, grid, 256, 0, st, static_cast<const float*>(p.in0), static_cast<float*>(p.out), r.B,
