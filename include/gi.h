@@ -187,7 +187,8 @@ enum {
   GI_KERNEL_DEPTHWISE_POINTWISE = 11, /* this op and the next one, as one kernel */
   GI_KERNEL_NONE = 12,                /* no launch: the op ran inside the previous op's kernel */
   GI_KERNEL_CONCAT = 13,
-  GI_KERNEL_CONV_TC = 14              /* k x k convolution, any number of input channels, on the tensor cores */
+  GI_KERNEL_CONV_TC = 14,             /* k x k convolution, any number of input channels, on the tensor cores */
+  GI_KERNEL_INVERTED_RESIDUAL = 15    /* this op (1x1 expansion) and the next two (depthwise 3x3, 1x1 projection) as one kernel */
 };
 
 /* ---- graph construction (Section 3.1, "Initialization": the sub-graph given to the GPU backend) ---- */

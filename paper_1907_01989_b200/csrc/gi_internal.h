@@ -78,6 +78,10 @@ struct LaunchRec {
   Loc wts2, bias2;
   int Co2 = 0;
   Epilogue ep2;
+  // a whole inverted-residual block as one kernel: `ep` is the expansion's epilogue, `ep_mid` the depthwise op's,
+  // `ep2` the projection's; Cmid the hidden channels; the stride / pads are the depthwise op's, (Ho, Wo) its output
+  int Cmid = 0;
+  Epilogue ep_mid;
 };
 
 struct FusedOp {

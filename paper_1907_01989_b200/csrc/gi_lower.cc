@@ -118,6 +118,44 @@ static bool pointwise_follows(const gi_graph& g, const gi_exec* e, size_t i) {
          d.pad_r == 0;
 }
 
+static bool is_plain_pointwise(const gi_op_desc& d) {
+  return d.kh == 1 && d.kw == 1 && d.stride_h == 1 && d.stride_w == 1 && d.pad_t == 0 && d.pad_l == 0 && d.pad_b == 0 && d.pad_r == 0;
+}
+
+// A tensor written by executed op `i`, read by op `i + 1` and by nothing else, living in the arena: one that a kernel
+// running both ops never has to store.
+static bool private_between(const gi_exec* e, int t, size_t i) {
+  if (t < 0) return false;
+  const TensorPlan& tp = e->plan[t];
+  return tp.intermediate == 1 && tp.first == static_cast<int>(i) && tp.last == static_cast<int>(i + 1) &&
+         e->tensors[t].output_index < 0 && e->tensors[t].input_index < 0;
+}
+
+// Executed ops i, i + 1, i + 2 are the three convolutions of an inverted-residual block - 1x1 expansion, depthwise
+// 3x3, 1x1 projection (with or without the residual sum) - and the two tensors between them have no other reader, so
+// that one kernel may run all three and keep those tensors on chip.
+static bool block_follows(const gi_graph& g, const gi_exec* e, size_t i) {
+  if (i + 2 >= e->ops.size()) return false;
+  const FusedOp& a = e->ops[i];
+  const FusedOp& b = e->ops[i + 1];
+  const FusedOp& c = e->ops[i + 2];
+  if (a.kind != GI_OP_CONV2D || b.kind != GI_OP_DEPTHWISE_CONV2D || c.kind != GI_OP_CONV2D) return false;
+  if (a.residual >= 0 || a.act_post != GI_ACT_NONE || b.residual >= 0 || b.act_post != GI_ACT_NONE) return false;
+  if (b.in0 != a.out || c.in0 != b.out || c.residual == a.out || c.residual == b.out) return false;
+  if (!private_between(e, a.out, i) || !private_between(e, b.out, i + 1)) return false;
+  if (!is_plain_pointwise(g.ops[a.graph_op].d) || !is_plain_pointwise(g.ops[c.graph_op].d)) return false;
+  const gi_op_desc& d = g.ops[b.graph_op].d;
+  if (d.stride_h != d.stride_w || d.dilation_h != 1 || d.dilation_w != 1) return false;
+  // One kernel reads the block's input while it writes the block's output.  Without a residual the two never live
+  // at the same op, so the planner may have given them the same arena bytes: then the block stays three kernels.
+  const TensorPlan& pin = e->plan[a.in0];
+  const TensorPlan& pout = e->plan[c.out];
+  if (loc_of(e, a.in0).where == W_ARENA && loc_of(e, c.out).where == W_ARENA && pin.offset < pout.offset + pout.bytes &&
+      pout.offset < pin.offset + pin.bytes)
+    return false;
+  return true;
+}
+
 // The executed op that converts graph input `t` from NHWC, if executed op `reader` is the only op that reads
 // the converted tensor (and it is not also a graph output); else -1.
 static int nhwc_pack_feeding_only(const gi_exec* e, int t, size_t reader) {
@@ -138,7 +176,7 @@ static int nhwc_pack_feeding_only(const gi_exec* e, int t, size_t reader) {
 gi_status lower(const gi_graph& g, gi_exec* e) {
   const int eb = elem_bytes(e->storage);
   const uint64_t B = static_cast<uint64_t>(e->batch);
-  bool absorbed = false;  // this op runs inside the previous op's kernel
+  int absorbed = 0;  // this many following ops run inside the kernel of an op already lowered
   for (size_t i = 0; i < e->ops.size(); ++i) {
     const FusedOp& f = e->ops[i];
     LaunchRec r;
@@ -204,9 +242,9 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
         r.pl = op.d.pad_l;
         const uint64_t taps = static_cast<uint64_t>(op.d.kh) * op.d.kw;
         info.bytes = (in_px * in_c4 + out_px * out_c4 * (r.ep.has_res ? 2 : 1)) * eb;
-        if (absorbed) {
-          // the previous (depthwise) op's kernel computes this 1x1 convolution too; its bytes and flops are counted there
-          absorbed = false;
+        if (absorbed > 0) {
+          // an earlier op's kernel computes this convolution too; its bytes and flops are counted there
+          --absorbed;
           r.kernel = GI_KERNEL_NONE;
           info.bytes = 0;
         } else if (f.kind == GI_OP_DEPTHWISE_CONV2D) {
@@ -239,7 +277,7 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
             info.bytes = (in_px * in_c4 + px2 * c42 * (r.ep2.has_res ? 2 : 1) + taps * din->c +
                           static_cast<uint64_t>(din->c) * pw.d.cout) * eb;
             info.flops += 2 * px2 * din->c * pw.d.cout;
-            absorbed = true;
+            absorbed = 1;
           }
         } else {
           const bool pointwise = op.d.kh == 1 && op.d.stride_h == 1 && op.d.stride_w == 1 && op.d.pad_t == 0 &&
@@ -255,6 +293,47 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
           // Launches whose pixels all fit one wave of 128-pixel tiles are latency-bound and take the lane
           // kernel (shorter fill; MobileNetV2 batch 1 0.296 -> 0.276 ms) - up to 64 tiles always, up to one
           // tile per SM unless the input is 960 channels deep or more.
+          // Whole inverted-residual block as one kernel (small planes): chosen where the kernel has at least about one
+          // unit of work per SM - below that (batch 1) three kernels that each spread over all SMs are faster
+          long long ir_units = 0;
+          if (pointwise && tc && e->opt.fuse && e->opt.cross_op != GI_XOP_OFF && block_follows(g, e, i)) {
+            const FusedOp& fd = e->ops[i + 1];
+            const FusedOp& fp = e->ops[i + 2];
+            const OpNode& dwn = g.ops[fd.graph_op];
+            const OpNode& pwn = g.ops[fp.graph_op];
+            const TensorDesc& dd = e->tensors[fd.out];
+            if (inverted_residual_supported(e->batch, din->h, din->w, dd.h, dd.w, dwn.d.stride_h, dwn.d.dilation_h, dwn.d.pad_t,
+                                            dwn.d.pad_l, din->c, op.d.cout, pwn.d.cout, &ir_units) &&
+                (e->opt.cross_op == GI_XOP_ON || ir_units >= 96)) {
+              const TensorDesc& d2 = e->tensors[fp.out];
+              r.kernel = GI_KERNEL_INVERTED_RESIDUAL;
+              r.Ho = dd.h;
+              r.Wo = dd.w;
+              r.sh = r.sw = dwn.d.stride_h;
+              r.pt = dwn.d.pad_t;
+              r.pl = dwn.d.pad_l;
+              r.kh = r.kw = 3;
+              r.Cmid = op.d.cout;
+              r.Co2 = pwn.d.cout;
+              r.ep_mid.act_pre = fd.act_pre;
+              r.ep2.act_pre = fp.act_pre;
+              r.ep2.has_res = fp.residual >= 0;
+              r.ep2.act_post = fp.act_post;
+              r.out = loc_of(e, fp.out);
+              r.res = loc_of(e, fp.residual);
+              inverted_residual_pack(op.weights.data(), op.bias.data(), dwn.weights.data(), dwn.bias.data(), pwn.weights.data(),
+                                     pwn.bias.data(), din->c, op.d.cout, pwn.d.cout, &e->weight_blob, &r);
+              const uint64_t px2 = B * d2.h * d2.w, c42 = slices(d2.c) * 4;
+              info.bytes = (in_px * in_c4 + px2 * c42 * (r.ep2.has_res ? 2 : 1) + static_cast<uint64_t>(din->c) * op.d.cout +
+                            9ull * op.d.cout + static_cast<uint64_t>(op.d.cout) * pwn.d.cout) * eb;
+              info.flops = 2 * out_px * din->c * op.d.cout + 2 * 9 * px2 * op.d.cout + 2 * px2 * op.d.cout * pwn.d.cout;
+              absorbed = 2;
+              info.kernel = r.kernel;
+              e->launches.push_back(r);
+              e->op_info.push_back(info);
+              continue;
+            }
+          }
           const long long m_px_all = static_cast<long long>(e->batch) * din->h * din->w;
           const bool one_wave = m_px_all <= 64LL * 128 || (m_px_all <= 148LL * 128 && din->c < 960);
           const bool lane_rule = op.d.cout >= 96 && din->c >= 64 && din->c < 960 && !(din->c <= 96 && op.d.cout >= 4 * din->c);

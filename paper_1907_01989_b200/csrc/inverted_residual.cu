@@ -1,0 +1,705 @@
+// One inverted-residual block - expansion 1x1 -> activation -> depthwise 3x3 -> activation ->
+// projection 1x1 (-> + residual) - as ONE kernel (fp16 storage).  The paper's cure for an engine
+// bound by memory is fewer, fatter programs (Section 3.2, "Shader Program Optimization"); on the small
+// planes of a MobileNet (14x14, 7x7) three launches per block spend more time filling and draining
+// than computing, and the 6x expanded tensor makes four trips through L2 / HBM that exist only
+// because the block is three kernels.  Here it never leaves the SM.
+//
+// Work unit = `n_img` whole images (one 14x14 image, two 7x7 images), i.e. at most 256 input pixels =
+// one or two 128-row MMA tiles; row r of the tiles is pixel r of the unit.  One CTA per SM walks units.
+//   * The block input X is copied once per unit into shared memory in the canonical K-major operand
+//     layout (8 channels = 16 bytes per row and K group; 8-byte cp.async straight from the
+//     channel-sliced tensor, two slices interleaved).
+//   * The hidden channels are processed in chunks of 64:
+//       expansion     D1[rows x 64]   = X * We[chunk]^T                  tcgen05.mma, accumulator in TMEM (two buffers)
+//       drain         bias, activation, fp16 -> a zero-bordered tile in shared memory, one plane per (slice, image)
+//       depthwise     3x3 stencil from that tile (a thread walks down one column of one 4-channel slice, every
+//                     input row feeding three running accumulators), bias, activation, fp16 -> the A operand of
+//                     the projection, written into shared memory in the canonical layout
+//       projection    D2[rows x Cout] += A2 * Wp[:, chunk]^T             tcgen05.mma, accumulating over the chunks
+//     The chunk's weights (We rows, Wp columns, depthwise taps, both biases: one contiguous block, packed at
+//     compile time) stream from L2 through a ring of stages filled by bulk copies.
+//   * After the last chunk D2 is drained: bias, activation, residual, activation, fp16, 8-byte stores.
+// Results are those of the three operators run one after the other: both hidden tensors are rounded to fp16
+// exactly as the stored tensors would have been.
+//
+// Warps: 0 = weight copies, 1 = MMA issuer and TMEM owner, 2..17 = compute (drain, stencil, epilogue; they also
+// issue the cp.async copies of the next unit's X as soon as the last expansion of the current unit is done).
+// The MMA thread runs one chunk ahead: expansion(c+1) is in flight while the compute warps work on chunk c.
+// Every wait is bounded; a wait that runs out raises the abort flag, after which all roles skip their work but
+// still meet at every barrier, so the CTA leaves in order.
+#include <cuda.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <cstring>
+
+#include "kernels.h"
+#include "pdl.cuh"
+#include "sm100_ptx.cuh"
+
+namespace gi {
+namespace {
+
+using namespace ptx;
+
+constexpr int kNh = 64;  // hidden channels per chunk
+constexpr int kComputeWarps = 16;
+constexpr int kComputeThreads = 32 * kComputeWarps;
+constexpr int kThreads = 64 + kComputeThreads;
+constexpr int kMaxStages = 3;
+constexpr int kHeader = 1024;
+constexpr int kSmemMax = 227 * 1024;
+constexpr int kDwBytes = (9 * kNh + kNh + kNh) * 4;  // depthwise taps, depthwise bias, expansion bias of a chunk
+
+__device__ unsigned int g_ir_error = 0;
+enum : unsigned { kErrCopy = 1u, kErrMma = 2u, kErrCompute = 4u, kErrDrain = 8u };
+
+struct IrParams {
+  const __half* in;
+  const __half* res;
+  __half* out;
+  const unsigned char* wts;  // n_chunks blocks of stage_bytes
+  const float* bias2;        // cout_pad floats
+  int B, H, W, Pin, Ho, Wo, Pout;
+  int stride, pt, pl;
+  int s_in;                  // input slices (input channels are a multiple of 16)
+  int n_chunks;
+  int cout_pad, s_out;
+  int n_split, n_each;       // the projection's N per MMA: cout_pad = n_split * n_each, n_each <= 256
+  int n_img, r_in, r_out;    // images per unit, pixels per image on the input / output side
+  int mt_in, mt_out;         // 128-row tiles on the input / output side
+  int units;
+  int Wp, plane_words;       // padded hidden tile: row pitch and plane pitch in 8-byte words
+  int n_bands, band_rows;
+  int stages;
+  unsigned stage_bytes, we_bytes, wp_bytes;
+  unsigned x_bytes, a2_bytes, h_bytes;
+  unsigned d2_col0;
+  int act1, act2, act3, has_res, act4;  // after expansion, after depthwise, after projection, residual, after the sum
+  unsigned timeout_ns;
+};
+
+struct Header {
+  unsigned long long w_full[kMaxStages], w_empty[kMaxStages];
+  unsigned long long d1_full[2], d1_empty[2];
+  unsigned long long a2_full, a2_empty, d2_full, d2_empty, x_full;
+  unsigned tmem_addr, abort_flag;
+};
+static_assert(sizeof(Header) <= kHeader, "header too large");
+
+__device__ __forceinline__ float act1f(float v, int kind) {
+  if (kind == GI_ACT_RELU) return fmaxf(v, 0.0f);
+  if (kind == GI_ACT_RELU6) return fminf(fmaxf(v, 0.0f), 6.0f);
+  return v;
+}
+// two floats -> fp16 pair with the activation applied: clamping the rounded value equals rounding the clamped
+// one because 0 and 6 are fp16 values
+__device__ __forceinline__ unsigned pack_act(float x, float y, int kind) {
+  unsigned d = pack_f16x2<false>(x, y);
+  if (kind != GI_ACT_NONE) {
+    __half2 h = *reinterpret_cast<__half2*>(&d);
+    h = __hmax2(h, __float2half2_rn(0.f));
+    if (kind == GI_ACT_RELU6) h = __hmin2(h, __float2half2_rn(6.f));
+    d = *reinterpret_cast<unsigned*>(&h);
+  }
+  return d;
+}
+__device__ __forceinline__ uint2 lds64(unsigned addr) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float4 lds128f(unsigned addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void sts64(unsigned addr, unsigned x, unsigned y) {
+  asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void cp_async8(unsigned dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// barrier of the compute warps only (id 1); the copy and MMA warps never join it
+__device__ __forceinline__ void bar_compute() { asm volatile("bar.sync 1, %0;" ::"n"(kComputeThreads) : "memory"); }
+
+struct Tap {
+  float2 lo, hi;
+};
+__device__ __forceinline__ Tap tap_of(uint2 v) {
+  Tap t;
+  t.lo = __half22float2(*reinterpret_cast<const __half2*>(&v.x));
+  t.hi = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
+  return t;
+}
+
+template <int STRIDE>
+__global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const IrParams p) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  Header* hdr = reinterpret_cast<Header*>(smem);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile unsigned* abort_flag = &hdr->abort_flag;
+  const unsigned x0 = smem_u32(smem + kHeader);
+  const unsigned a20 = x0 + p.x_bytes;
+  const unsigned h0 = a20 + p.a2_bytes;
+  const unsigned st0 = h0 + p.h_bytes;
+  const unsigned d1_cols = static_cast<unsigned>(p.mt_in) * kNh;  // one D1 buffer
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < p.stages; ++i) {
+      mbar_init(smem_u32(&hdr->w_full[i]), 1);
+      mbar_init(smem_u32(&hdr->w_empty[i]), 1 + kComputeWarps);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&hdr->d1_full[i]), 1);
+      mbar_init(smem_u32(&hdr->d1_empty[i]), kComputeWarps);
+    }
+    mbar_init(smem_u32(&hdr->a2_full), 1);
+    mbar_init(smem_u32(&hdr->a2_empty), 1);
+    mbar_init(smem_u32(&hdr->d2_full), 1);
+    mbar_init(smem_u32(&hdr->d2_empty), kComputeWarps);
+    mbar_init(smem_u32(&hdr->x_full), 1);
+    hdr->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_proxy();
+  }
+  if (warp == 1) tmem_alloc(smem_u32(&hdr->tmem_addr), 512u);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const unsigned tmem_base = hdr->tmem_addr;
+  pdl_launch_dependents();
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ weight copies (weights never change: no wait
+    // for the previous kernel)
+    if (lane == 0) {
+      unsigned g = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
+        for (int c = 0; c < p.n_chunks; ++c, ++g) {
+          const unsigned stage = g % p.stages, phase = (g / p.stages) & 1u;
+          if (!mbar_wait(smem_u32(&hdr->w_empty[stage]), phase ^ 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCopy)) {
+            ok = false;
+            break;
+          }
+          const unsigned full = smem_u32(&hdr->w_full[stage]);
+          mbar_expect_tx(full, p.stage_bytes);
+          bulk_load(st0 + stage * p.stage_bytes, p.wts + static_cast<size_t>(c) * p.stage_bytes, p.stage_bytes, full);
+        }
+      }
+      if (!ok) {
+        // copies already issued still land in shared memory: give them a bounded grace before leaving
+        const unsigned first = g > static_cast<unsigned>(p.stages) ? g - p.stages : 0u;
+        for (unsigned j = first; j < g; ++j) {
+          const unsigned long long t0 = global_timer_ns();
+          while (!mbar_try_wait(smem_u32(&hdr->w_full[j % p.stages]), (j / p.stages) & 1u)) {
+            if (global_timer_ns() - t0 > p.timeout_ns) {
+              atomicOr(&g_ir_error, kErrDrain);
+              break;
+            }
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const unsigned idesc1 = (1u << 4) | ((static_cast<unsigned>(kNh) >> 3) << 17) | ((128u >> 4) << 24);
+      const unsigned idesc2 = (1u << 4) | ((static_cast<unsigned>(p.n_each) >> 3) << 17) | ((128u >> 4) << 24);
+      const unsigned x_lbo = static_cast<unsigned>(p.mt_in) * 2048u;    // K group pitch of X: rows x 16 bytes
+      const unsigned a2_lbo = static_cast<unsigned>(p.mt_out) * 2048u;  // of A2
+      const unsigned we_lbo = kNh * 16u, wp_lbo = static_cast<unsigned>(p.cout_pad) * 16u;
+      const int k_steps1 = p.s_in / 4;  // 16 input channels per MMA
+      unsigned g = 0, ul = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++ul) {
+        if (!mbar_wait(smem_u32(&hdr->x_full), ul & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma)) break;
+        tc_fence_after();
+        for (int c = 0; c <= p.n_chunks && ok; ++c) {
+          if (c < p.n_chunks) {
+            const unsigned gc = g + c, stage = gc % p.stages, buf = gc & 1u;
+            if (!mbar_wait(smem_u32(&hdr->w_full[stage]), (gc / p.stages) & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma) ||
+                !mbar_wait(smem_u32(&hdr->d1_empty[buf]), ((gc >> 1) & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after();
+            const unsigned we = st0 + stage * p.stage_bytes;
+            for (int t = 0; t < p.mt_in; ++t) {
+              const unsigned d = tmem_base + buf * d1_cols + static_cast<unsigned>(t) * kNh;
+              unsigned long long ad = smem_desc(x0 + static_cast<unsigned>(t) * 2048u, x_lbo, 128);
+              unsigned long long bd = smem_desc(we, we_lbo, 128);
+              const unsigned long long ad_step = static_cast<unsigned long long>((2u * x_lbo) >> 4);
+              const unsigned long long bd_step = static_cast<unsigned long long>((2u * we_lbo) >> 4);
+              for (int ks = 0; ks < k_steps1; ++ks) {
+                umma_f16(d, ad, bd, idesc1, ks > 0 ? 1u : 0u);
+                ad += ad_step;
+                bd += bd_step;
+              }
+            }
+            umma_commit(smem_u32(&hdr->d1_full[buf]));
+          }
+          if (c >= 1) {
+            const unsigned gp = g + c - 1, stage = gp % p.stages;
+            if (c == 1 && !mbar_wait(smem_u32(&hdr->d2_empty), (ul & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma)) {
+              ok = false;
+              break;
+            }
+            if (!mbar_wait(smem_u32(&hdr->a2_full), gp & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after();
+            const unsigned wp = st0 + stage * p.stage_bytes + p.we_bytes;
+            for (int t = 0; t < p.mt_out; ++t)
+              for (int h = 0; h < p.n_split; ++h) {
+                const unsigned d = tmem_base + p.d2_col0 + static_cast<unsigned>(t * p.cout_pad + h * p.n_each);
+                unsigned long long ad = smem_desc(a20 + static_cast<unsigned>(t) * 2048u, a2_lbo, 128);
+                unsigned long long bd = smem_desc(wp + static_cast<unsigned>(h * p.n_each) * 16u, wp_lbo, 128);
+                const unsigned long long ad_step = static_cast<unsigned long long>((2u * a2_lbo) >> 4);
+                const unsigned long long bd_step = static_cast<unsigned long long>((2u * wp_lbo) >> 4);
+                for (int ks = 0; ks < kNh / 16; ++ks) {
+                  umma_f16(d, ad, bd, idesc2, (c > 1 || ks > 0) ? 1u : 0u);
+                  ad += ad_step;
+                  bd += bd_step;
+                }
+              }
+            umma_commit(smem_u32(&hdr->a2_empty));
+            umma_commit(smem_u32(&hdr->w_empty[stage]));
+            if (c == p.n_chunks) umma_commit(smem_u32(&hdr->d2_full));
+          }
+        }
+        g += p.n_chunks;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ compute warps
+    const int cw = warp - 2, ctid = threadIdx.x - 64;
+    const int quarter = warp & 3, qsub = cw >> 2;  // TMEM lane quarter of this warp; its index among the four warps sharing it
+    const unsigned lane_bits = static_cast<unsigned>(quarter * 32) << 16;
+    const int rows_in = p.n_img * p.r_in, rows_out = p.n_img * p.r_out;
+
+    // copies of a unit's X: thread i takes (slice, row) pairs i, i + 512, ...; consecutive threads take consecutive
+    // pixels of one slice (coalesced 8-byte reads); rows of images beyond the batch are left as they are (their
+    // results are never stored)
+    auto issue_x = [&](int u) {
+      const int b0 = u * p.n_img;
+      const int total = p.s_in * rows_in;
+      for (int i = ctid; i < total; i += kComputeThreads) {
+        const int s = i / rows_in, r = i - s * rows_in;
+        const int img = r / p.r_in, q = r - img * p.r_in;
+        if (b0 + img >= p.B) continue;
+        const __half* src = p.in + ((static_cast<size_t>(s) * p.B + b0 + img) * p.Pin + q) * 4;
+        cp_async8(x0 + static_cast<unsigned>(s >> 1) * (static_cast<unsigned>(p.mt_in) * 2048u) + static_cast<unsigned>(r) * 16u +
+                      static_cast<unsigned>(s & 1) * 8u,
+                  src);
+      }
+    };
+
+    // the hidden tile's border is the zero padding of the depthwise convolution: cleared once, never written again
+    for (unsigned i = ctid; i < p.h_bytes / 16u; i += kComputeThreads)
+      asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(h0 + i * 16u), "r"(0u) : "memory");
+
+    // this thread's place in the stencil: (band, plane = slice of the chunk x image, output column)
+    const int planes = (kNh / 4) * p.n_img;
+    const int per_band = planes * p.Wo;
+    const int band = ctid / per_band;
+    const bool st_active = band < p.n_bands;
+    const int st_rem = ctid - band * per_band;
+    const int st_plane = st_rem / p.Wo, st_ox = st_rem - st_plane * p.Wo;
+    const int st_slice = st_plane / p.n_img, st_img = st_plane - st_slice * p.n_img;
+    const int st_r0 = band * p.band_rows, st_r1 = min(p.Ho, st_r0 + p.band_rows);
+    const unsigned st_h = h0 + static_cast<unsigned>(st_plane) * p.plane_words * 8u;
+    const unsigned st_a2 = a20 + static_cast<unsigned>(st_slice >> 1) * (static_cast<unsigned>(p.mt_out) * 2048u) +
+                           static_cast<unsigned>(st_img * p.r_out) * 16u + static_cast<unsigned>(st_slice & 1) * 8u;
+
+    pdl_wait();  // activations are read and written only below
+    bool ok = true;
+    if (static_cast<int>(blockIdx.x) < p.units) issue_x(blockIdx.x);
+    cp_async_wait_all();
+    fence_async_proxy();
+    bar_compute();
+    if (ctid == 0 && static_cast<int>(blockIdx.x) < p.units) mbar_arrive(smem_u32(&hdr->x_full));
+
+    unsigned g = 0, ul = 0;
+    for (int u = blockIdx.x; u < p.units; u += gridDim.x, ++ul) {
+      const int b0 = u * p.n_img;
+      for (int c = 0; c < p.n_chunks; ++c) {
+        const unsigned gc = g + c, stage = gc % p.stages, buf = gc & 1u;
+        const unsigned stg = st0 + stage * p.stage_bytes;
+        const unsigned dw0 = stg + p.we_bytes + p.wp_bytes;  // depthwise taps [9][64], depthwise bias [64], expansion bias [64]
+        ok = ok && mbar_wait_warp(smem_u32(&hdr->w_full[stage]), (gc / p.stages) & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
+        ok = ok && mbar_wait_warp(smem_u32(&hdr->d1_full[buf]), (gc >> 1) & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
+        if (ok) {
+          tc_fence_after();
+          // ---- drain D1: 16 hidden channels of one pixel per tcgen05.ld; bias, activation, fp16 -> hidden tile
+          for (int e = qsub; e < p.mt_in * 4; e += 4) {
+            const int t = e >> 2, j = e & 3;
+            unsigned r[16];
+            tmem_ld16(tmem_base + lane_bits + buf * d1_cols + static_cast<unsigned>(t * kNh + j * 16), r);
+            const int row = t * 128 + quarter * 32 + lane;
+            const int img = row / p.r_in, q = row - img * p.r_in;
+            const int y = q / p.W, x = q - y * p.W;
+            const bool valid = row < rows_in;
+            tmem_ld_wait16(r);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int sl = j * 4 + i;
+              const float4 b = lds128f(dw0 + (10 * kNh + sl * 4) * 4u);
+              const unsigned w0 = pack_act(__uint_as_float(r[4 * i]) + b.x, __uint_as_float(r[4 * i + 1]) + b.y, p.act1);
+              const unsigned w1 = pack_act(__uint_as_float(r[4 * i + 2]) + b.z, __uint_as_float(r[4 * i + 3]) + b.w, p.act1);
+              if (valid)
+                sts64(h0 + (static_cast<unsigned>(sl * p.n_img + img) * p.plane_words + static_cast<unsigned>((y + 1) * p.Wp + x + 1)) * 8u, w0, w1);
+            }
+          }
+          tc_fence_before();
+        }
+        __syncwarp();
+        if (lane == 0 && ok) mbar_arrive(smem_u32(&hdr->d1_empty[buf]));
+        // the last expansion of this unit is complete (its accumulator was just read): X may be overwritten
+        if (c == p.n_chunks - 1 && u + static_cast<int>(gridDim.x) < p.units && ok) issue_x(u + gridDim.x);
+        bar_compute();  // the hidden tile is complete
+
+        // ---- this thread's depthwise weights (its slice of the chunk) into registers, then the stage is released
+        float2 wlo[9], whi[9];
+        Tap bias;
+        if (ok && st_active) {
+#pragma unroll
+          for (int k = 0; k < 9; ++k) {
+            const float4 w = lds128f(dw0 + (k * kNh + st_slice * 4) * 4u);
+            wlo[k] = make_float2(w.x, w.y);
+            whi[k] = make_float2(w.z, w.w);
+          }
+          const float4 b = lds128f(dw0 + (9 * kNh + st_slice * 4) * 4u);
+          bias.lo = make_float2(b.x, b.y);
+          bias.hi = make_float2(b.z, b.w);
+        }
+        __syncwarp();
+        if (lane == 0 && ok) mbar_arrive(smem_u32(&hdr->w_empty[stage]));
+        ok = ok && mbar_wait_warp(smem_u32(&hdr->a2_empty), (gc & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
+
+        // ---- depthwise 3x3 from the hidden tile -> A operand of the projection
+        if (ok && st_active) {
+          auto emit = [&](const Tap& a, int oy) {
+            const unsigned w0 = pack_act(a.lo.x, a.lo.y, p.act2), w1 = pack_act(a.hi.x, a.hi.y, p.act2);
+            sts64(st_a2 + static_cast<unsigned>(oy * p.Wo + st_ox) * 16u, w0, w1);
+          };
+          if (STRIDE == 1) {
+            // padded row iy (image row iy - 1) is tap row 0 of output row iy, row 1 of iy - 1, row 2 of iy - 2
+            Tap a0 = bias, a1 = bias, a2 = bias;
+            auto step = [&](Tap& done, Tap& mid, Tap& fresh, int iy) {
+              const unsigned at = st_h + static_cast<unsigned>(iy * p.Wp + st_ox) * 8u;
+              const Tap t0 = tap_of(lds64(at)), t1 = tap_of(lds64(at + 8u)), t2 = tap_of(lds64(at + 16u));
+              done.lo = __ffma2_rn(t0.lo, wlo[6], done.lo);
+              done.hi = __ffma2_rn(t0.hi, whi[6], done.hi);
+              done.lo = __ffma2_rn(t1.lo, wlo[7], done.lo);
+              done.hi = __ffma2_rn(t1.hi, whi[7], done.hi);
+              done.lo = __ffma2_rn(t2.lo, wlo[8], done.lo);
+              done.hi = __ffma2_rn(t2.hi, whi[8], done.hi);
+              if (iy - 2 >= st_r0) emit(done, iy - 2);
+              mid.lo = __ffma2_rn(t0.lo, wlo[3], mid.lo);
+              mid.hi = __ffma2_rn(t0.hi, whi[3], mid.hi);
+              mid.lo = __ffma2_rn(t1.lo, wlo[4], mid.lo);
+              mid.hi = __ffma2_rn(t1.hi, whi[4], mid.hi);
+              mid.lo = __ffma2_rn(t2.lo, wlo[5], mid.lo);
+              mid.hi = __ffma2_rn(t2.hi, whi[5], mid.hi);
+              fresh.lo = __ffma2_rn(t0.lo, wlo[0], bias.lo);
+              fresh.hi = __ffma2_rn(t0.hi, whi[0], bias.hi);
+              fresh.lo = __ffma2_rn(t1.lo, wlo[1], fresh.lo);
+              fresh.hi = __ffma2_rn(t1.hi, whi[1], fresh.hi);
+              fresh.lo = __ffma2_rn(t2.lo, wlo[2], fresh.lo);
+              fresh.hi = __ffma2_rn(t2.hi, whi[2], fresh.hi);
+            };
+            // with one row of padding above, output row oy reads padded rows oy .. oy + 2
+            const int last = st_r1 + 1;
+            for (int iy = st_r0;;) {
+              step(a0, a1, a2, iy);
+              if (++iy > last) break;
+              step(a1, a2, a0, iy);
+              if (++iy > last) break;
+              step(a2, a0, a1, iy);
+              if (++iy > last) break;
+            }
+          } else {
+            for (int oy = st_r0; oy < st_r1; ++oy) {
+              Tap a = bias;
+#pragma unroll
+              for (int ky = 0; ky < 3; ++ky) {
+                const unsigned at = st_h + static_cast<unsigned>((oy * 2 - p.pt + ky + 1) * p.Wp + st_ox * 2 - p.pl + 1) * 8u;
+#pragma unroll
+                for (int kx = 0; kx < 3; ++kx) {
+                  const Tap t = tap_of(lds64(at + kx * 8u));
+                  a.lo = __ffma2_rn(t.lo, wlo[ky * 3 + kx], a.lo);
+                  a.hi = __ffma2_rn(t.hi, whi[ky * 3 + kx], a.hi);
+                }
+              }
+              emit(a, oy);
+            }
+          }
+        }
+        fence_async_proxy();  // the A operand was written with ordinary stores; the MMA reads it through the async proxy
+        bar_compute();        // A2 complete; nobody reads the hidden tile any more
+        if (ctid == 0 && ok) mbar_arrive(smem_u32(&hdr->a2_full));
+      }
+      g += p.n_chunks;
+
+      // ---- the next unit's X has been on its way since the last drain: publish it, then drain this unit's D2
+      const bool more = u + static_cast<int>(gridDim.x) < p.units;
+      if (more) {
+        cp_async_wait_all();
+        fence_async_proxy();
+        bar_compute();
+        if (ctid == 0 && ok) mbar_arrive(smem_u32(&hdr->x_full));
+      }
+      ok = ok && mbar_wait_warp(smem_u32(&hdr->d2_full), ul & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
+      if (ok) {
+        tc_fence_after();
+        const int groups = p.cout_pad >> 4;
+        for (int e = qsub; e < p.mt_out * groups; e += 4) {
+          const int t = e / groups, j = e - t * groups;
+          unsigned r[16];
+          tmem_ld16(tmem_base + lane_bits + p.d2_col0 + static_cast<unsigned>(t * p.cout_pad + j * 16), r);
+          const int row = t * 128 + quarter * 32 + lane;
+          const int img = row / p.r_out, q = row - img * p.r_out;
+          const bool valid = row < rows_out && b0 + img < p.B;
+          tmem_ld_wait16(r);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int so = j * 4 + i;
+            if (so >= p.s_out || !valid) continue;
+            const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias2) + so);
+            const size_t off = ((static_cast<size_t>(so) * p.B + b0 + img) * p.Pout + q) * 4;  // in halves
+            float v0 = act1f(__uint_as_float(r[4 * i]) + b.x, p.act3), v1 = act1f(__uint_as_float(r[4 * i + 1]) + b.y, p.act3);
+            float v2 = act1f(__uint_as_float(r[4 * i + 2]) + b.z, p.act3), v3 = act1f(__uint_as_float(r[4 * i + 3]) + b.w, p.act3);
+            if (p.has_res) {
+              const uint2 rq = __ldg(reinterpret_cast<const uint2*>(p.res + off));
+              const float2 r0 = __half22float2(*reinterpret_cast<const __half2*>(&rq.x));
+              const float2 r1 = __half22float2(*reinterpret_cast<const __half2*>(&rq.y));
+              v0 += r0.x;
+              v1 += r0.y;
+              v2 += r1.x;
+              v3 += r1.y;
+            }
+            uint2 o;
+            o.x = pack_f16x2<false>(act1f(v0, p.act4), act1f(v1, p.act4));
+            o.y = pack_f16x2<false>(act1f(v2, p.act4), act1f(v3, p.act4));
+            *reinterpret_cast<uint2*>(p.out + off) = o;
+            // an odd plane is stored with one extra pixel, which readers expect to be finite: zero it
+            if (q == p.r_out - 1 && p.Pout > p.r_out) *reinterpret_cast<uint2*>(p.out + off + 4) = make_uint2(0u, 0u);
+          }
+        }
+        tc_fence_before();
+      }
+      __syncwarp();
+      if (lane == 0 && ok) mbar_arrive(smem_u32(&hdr->d2_empty));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512u);
+  }
+}
+
+struct Shape {
+  int n_img, mt_in, mt_out, r_in, r_out, n_chunks, cout_pad, n_split, n_each, Wp, plane_words, n_bands, band_rows, stages;
+  unsigned we_bytes, wp_bytes, stage_bytes, x_bytes, a2_bytes, h_bytes;
+  size_t smem;
+  long long units;
+  bool ok;
+};
+
+Shape shape_of(int B, int H, int W, int Ho, int Wo, int stride, int cin, int chid, int cout) {
+  Shape s{};
+  s.ok = false;
+  if (cin <= 0 || cin % 16 != 0 || chid <= 0 || cout <= 0) return s;
+  s.r_in = H * W;
+  s.r_out = Ho * Wo;
+  if (s.r_in > 256 || s.r_in < 4) return s;
+  // as many whole images as fill one 128-row tile; a larger image takes two tiles by itself
+  s.n_img = s.r_in <= 128 ? 128 / s.r_in : 1;
+  if (s.n_img > B) s.n_img = B;
+  if (s.n_img > 2) s.n_img = 2;  // planes of the hidden tile: 16 slices x images; more images only shorten the columns walked
+  s.mt_in = (s.n_img * s.r_in + 127) / 128;
+  s.mt_out = (s.n_img * s.r_out + 127) / 128;
+  s.n_chunks = (chid + kNh - 1) / kNh;
+  s.cout_pad = (cout + 15) / 16 * 16;
+  s.n_split = (s.cout_pad + 255) / 256;
+  while (s.cout_pad % (16 * s.n_split) != 0) ++s.n_split;
+  s.n_each = s.cout_pad / s.n_split;
+  // tensor memory: two expansion accumulators and the projection accumulator
+  if (2 * s.mt_in * kNh + s.mt_out * s.cout_pad > 512) return s;
+  s.Wp = W + 2;
+  s.plane_words = (H + 2) * s.Wp;
+  while (s.plane_words % 16 != W % 16) ++s.plane_words;  // consecutive planes start W words apart (mod 16): no bank conflicts
+  const int planes = (kNh / 4) * s.n_img;
+  int bands = kComputeThreads / (planes * Wo);
+  if (bands < 1) return s;
+  if (bands > Ho) bands = Ho;
+  s.band_rows = (Ho + bands - 1) / bands;
+  s.n_bands = (Ho + s.band_rows - 1) / s.band_rows;
+  s.we_bytes = static_cast<unsigned>(kNh) * cin * 2u;
+  s.wp_bytes = static_cast<unsigned>(s.cout_pad) * kNh * 2u;
+  s.stage_bytes = s.we_bytes + s.wp_bytes + kDwBytes;
+  s.x_bytes = static_cast<unsigned>(cin / 8) * s.mt_in * 2048u;
+  s.a2_bytes = static_cast<unsigned>(kNh / 8) * s.mt_out * 2048u;
+  s.h_bytes = (static_cast<unsigned>(planes) * s.plane_words * 8u + 15u) / 16u * 16u;
+  const long long fixed = kHeader + static_cast<long long>(s.x_bytes) + s.a2_bytes + s.h_bytes;
+  long long stages = (kSmemMax - fixed) / s.stage_bytes;
+  if (stages < 2) return s;
+  s.stages = stages > kMaxStages ? kMaxStages : static_cast<int>(stages);
+  s.smem = static_cast<size_t>(fixed) + static_cast<size_t>(s.stages) * s.stage_bytes;
+  s.units = (static_cast<long long>(B) + s.n_img - 1) / s.n_img;
+  (void)stride;
+  s.ok = true;
+  return s;
+}
+
+}  // namespace
+
+bool inverted_residual_supported(int B, int H, int W, int Ho, int Wo, int stride, int dil, int pt, int pl, int cin, int chid,
+                                 int cout, long long* units) {
+  if (stride < 1 || stride > 2 || dil != 1 || pt < 0 || pt > 1 || pl < 0 || pl > 1) return false;
+  // every tap must stay inside the padded hidden tile (one zero row / column on each side)
+  if ((Ho - 1) * stride - pt + 2 > H || (Wo - 1) * stride - pl + 2 > W) return false;
+  if (stride == 1 && (pt != 1 || pl != 1 || Ho != H || Wo != W)) return false;
+  const Shape s = shape_of(B, H, W, Ho, Wo, stride, cin, chid, cout);
+  if (!s.ok) return false;
+  if (units) *units = s.units;
+  return true;
+}
+
+// Per chunk of 64 hidden channels one contiguous block: We[cin/8][64][8] (expansion rows of the chunk, K-major core
+// matrices), Wp[8][cout_pad][8] (projection columns of the chunk), depthwise taps [9][64], depthwise bias [64],
+// expansion bias [64] (floats).  Hidden channels beyond `chid` are zero throughout, so they contribute nothing.
+void inverted_residual_pack(const float* we, const float* be, const float* wd, const float* bd, const float* wp, const float* bp,
+                            int cin, int chid, int cout, std::vector<uint8_t>* blob, LaunchRec* r) {
+  const Shape s = shape_of(r->B, r->H, r->W, r->Ho, r->Wo, r->sh, cin, chid, cout);
+  const uint64_t woff = round_up_u64(blob->size(), 256);
+  blob->resize(woff + static_cast<size_t>(s.n_chunks) * s.stage_bytes, 0);
+  const uint64_t boff = round_up_u64(blob->size(), 256);
+  blob->resize(boff + static_cast<size_t>(s.cout_pad) * sizeof(float), 0);
+  for (int c = 0; c < s.n_chunks; ++c) {
+    uint8_t* base = blob->data() + woff + static_cast<size_t>(c) * s.stage_bytes;
+    uint16_t* pe = reinterpret_cast<uint16_t*>(base);
+    uint16_t* pp = reinterpret_cast<uint16_t*>(base + s.we_bytes);
+    float* pd = reinterpret_cast<float*>(base + s.we_bytes + s.wp_bytes);
+    for (int n = 0; n < kNh; ++n) {
+      const int hch = c * kNh + n;
+      if (hch >= chid) continue;
+      for (int ci = 0; ci < cin; ++ci)
+        pe[(static_cast<size_t>(ci / 8) * kNh + n) * 8 + ci % 8] = f32_to_f16_rne(we[static_cast<size_t>(hch) * cin + ci]);
+      for (int co = 0; co < cout; ++co)
+        pp[(static_cast<size_t>(n / 8) * s.cout_pad + co) * 8 + n % 8] = f32_to_f16_rne(wp[static_cast<size_t>(co) * chid + hch]);
+      for (int k = 0; k < 9; ++k) {
+        // the depthwise taps take part in the arithmetic as the fp16 values the stored weights would have
+        const uint16_t hb = f32_to_f16_rne(wd[static_cast<size_t>(k) * chid + hch]);
+        const uint32_t sg = (hb & 0x8000u) << 16, ex = (hb >> 10) & 0x1fu, m = hb & 0x3ffu;
+        float v;
+        uint32_t bits;
+        if (ex == 0) {
+          v = static_cast<float>(m) * (1.0f / 16777216.0f);
+          std::memcpy(&bits, &v, 4);
+        } else if (ex == 31) {
+          bits = 0x7f800000u | (m << 13);
+        } else {
+          bits = ((ex + 112u) << 23) | (m << 13);
+        }
+        bits |= sg;
+        std::memcpy(&v, &bits, 4);
+        pd[k * kNh + n] = v;
+      }
+      pd[9 * kNh + n] = bd[hch];
+      pd[10 * kNh + n] = be[hch];
+    }
+  }
+  float* b2 = reinterpret_cast<float*>(blob->data() + boff);
+  for (int co = 0; co < cout; ++co) b2[co] = bp[co];
+  r->wts = Loc{W_WEIGHTS, 0, woff};
+  r->bias2 = Loc{W_WEIGHTS, 0, boff};
+  r->wts_bytes = static_cast<uint64_t>(s.n_chunks) * s.stage_bytes;
+}
+
+int launch_inverted_residual(const LaunchRec& r, const Ptrs& p, void* stream) {
+  const Shape s = shape_of(r.B, r.H, r.W, r.Ho, r.Wo, r.sh, r.C, r.Cmid, r.Co2);
+  if (!s.ok) return static_cast<int>(cudaErrorInvalidConfiguration);
+  IrParams k{};
+  k.in = static_cast<const __half*>(p.in0);
+  k.res = static_cast<const __half*>(p.res);
+  k.out = static_cast<__half*>(p.out);
+  k.wts = static_cast<const unsigned char*>(p.wts);
+  k.bias2 = static_cast<const float*>(p.bias2);
+  k.B = r.B;
+  k.H = r.H;
+  k.W = r.W;
+  k.Pin = plane_pixels(r.H, r.W);
+  k.Ho = r.Ho;
+  k.Wo = r.Wo;
+  k.Pout = plane_pixels(r.Ho, r.Wo);
+  k.stride = r.sh;
+  k.pt = r.pt;
+  k.pl = r.pl;
+  k.s_in = r.C / 4;
+  k.n_chunks = s.n_chunks;
+  k.cout_pad = s.cout_pad;
+  k.s_out = slices(r.Co2);
+  k.n_split = s.n_split;
+  k.n_each = s.n_each;
+  k.n_img = s.n_img;
+  k.r_in = s.r_in;
+  k.r_out = s.r_out;
+  k.mt_in = s.mt_in;
+  k.mt_out = s.mt_out;
+  k.units = static_cast<int>(s.units);
+  k.Wp = s.Wp;
+  k.plane_words = s.plane_words;
+  k.n_bands = s.n_bands;
+  k.band_rows = s.band_rows;
+  k.stages = s.stages;
+  k.stage_bytes = s.stage_bytes;
+  k.we_bytes = s.we_bytes;
+  k.wp_bytes = s.wp_bytes;
+  k.x_bytes = s.x_bytes;
+  k.a2_bytes = s.a2_bytes;
+  k.h_bytes = s.h_bytes;
+  k.d2_col0 = 2u * static_cast<unsigned>(s.mt_in) * kNh;
+  k.act1 = r.ep.act_pre;
+  k.act2 = r.ep_mid.act_pre;
+  k.act3 = r.ep2.act_pre;
+  k.has_res = r.ep2.has_res;
+  k.act4 = r.ep2.act_post;
+  k.timeout_ns = 1000000000u;
+  static bool attr_done_dev[kMaxDevices] = {};
+  bool& attr_done = attr_done_dev[current_device_slot()];
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(inverted_residual_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(inverted_residual_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+    if (e != cudaSuccess) return static_cast<int>(e);
+    attr_done = true;
+  }
+  const int sms = device_sm_count();
+  const unsigned grid = static_cast<unsigned>(s.units < sms ? s.units : sms);
+  // the kernel reserves all of tensor memory: ask for enough shared memory that no second CTA shares the SM
+  size_t smem = s.smem;
+  if (smem < 120 * 1024) smem = 120 * 1024;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (r.sh == 1) launch_pdl(inverted_residual_kernel<1>, grid, kThreads, smem, st, k);
+  else launch_pdl(inverted_residual_kernel<2>, grid, kThreads, smem, st, k);
+  return static_cast<int>(cudaGetLastError());
+}
+
+unsigned int inverted_residual_error_word(int* cuda_err) {
+  unsigned int v = 0;
+  const cudaError_t e = cudaMemcpyFromSymbol(&v, g_ir_error, sizeof v);
+  if (cuda_err) *cuda_err = static_cast<int>(e);
+  return v;
+}
+
+}  // namespace gi

@@ -76,4 +76,13 @@ void depthwise_pointwise_pack(const float* w, const float* bias, int cin, int co
 int launch_depthwise_pointwise(const LaunchRec& r, const Ptrs& p, void* stream);
 unsigned int depthwise_pointwise_error_word(int* cuda_err);
 
+// One inverted-residual block (1x1 expansion -> depthwise 3x3 -> 1x1 projection, + residual) as one kernel (fp16
+// storage, planes of at most 256 pixels): neither hidden tensor leaves the SM.  `units` receives the kernel's parallelism.
+bool inverted_residual_supported(int B, int H, int W, int Ho, int Wo, int stride, int dil, int pt, int pl, int cin, int chid,
+                                 int cout, long long* units);
+void inverted_residual_pack(const float* we, const float* be, const float* wd, const float* bd, const float* wp, const float* bp,
+                            int cin, int chid, int cout, std::vector<uint8_t>* blob, LaunchRec* r);
+int launch_inverted_residual(const LaunchRec& r, const Ptrs& p, void* stream);
+unsigned int inverted_residual_error_word(int* cuda_err);
+
 }  // namespace gi

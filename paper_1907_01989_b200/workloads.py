@@ -327,6 +327,27 @@ def depthwise_then_pointwise(batch: int, h: int, w: int, c: int, cout: int, stri
     return b.finish()
 
 
+def inverted_residual_block(batch: int, h: int, w: int, cin: int, hidden: int, cout: int, stride: int = 1,
+                            act: str = ACT_RELU6, out_act: Optional[str] = None) -> GraphSpec:
+    """One inverted-residual block of MobileNetV2 on its own: 1x1 expansion + activation, depthwise 3x3 + activation,
+    linear 1x1 projection, and the residual sum where the block keeps shape (stride 1, cin == cout)."""
+    b = GraphBuilder(f"block_{batch}x{h}x{w}_{cin}_{hidden}_{cout}_s{stride}", batch, 14)
+    x = b.input(h, w, cin)
+    y = b.conv2d(x, hidden, 1)
+    if act != ACT_NONE:
+        y = b.activation(y, act)
+    y = b.depthwise(y, 3, stride, 1)
+    if act != ACT_NONE:
+        y = b.activation(y, act)
+    y = b.conv2d(y, cout, 1)
+    if stride == 1 and cin == cout:
+        y = b.add(x, y)
+    if out_act is not None:
+        y = b.activation(y, out_act)
+    b.output(y)
+    return b.finish()
+
+
 # ----------------------------------------------------------------------------------------
 # Workload 10: a network of "fire" modules - squeeze 1x1, then a 1x1 and a 3x3 expansion whose outputs are
 # concatenated - with a 2x2 stride-2 stem and a 3x3 stride-3 reduction: the operators and the kernel sizes /

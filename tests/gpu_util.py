@@ -33,7 +33,8 @@ class DeviceRun:
         self.graph, _ = api.graph_from_spec(spec, storage)
         self.ex = self.graph.compile(planner=planner, fuse=fuse, pointwise=pointwise, cross_op=cross_op)
         # tensors that stay on chip: the input of an op that runs inside the previous op's kernel
-        self.on_chip = {o.inputs[0] for o in self.ex.ops() if api.KERNEL_NAMES[o.kernel] == "none" and o.kind == api.GI_OP_CONV2D}
+        self.on_chip = {o.inputs[0] for o in self.ex.ops() if api.KERNEL_NAMES[o.kernel] == "none" and
+                        o.kind in (api.GI_OP_CONV2D, api.GI_OP_DEPTHWISE_CONV2D)}
         # ... and the converted copy of an NHWC input that the first convolution reads in the caller's layout itself
         self.on_chip |= {o.output for o in self.ex.ops() if api.KERNEL_NAMES[o.kernel] == "none" and o.kind == api.GI_EXEC_PACK}
         dev = "cuda:0"

@@ -753,3 +753,49 @@ def test_two_threads_run_one_executable_with_their_own_arenas():
         torch.cuda.synchronize()
         assert np.array_equal(outs[k % 2].float().cpu().numpy(), first)
     assert api.gi_device_status() == 0
+
+
+# ---------------------------------------------------------------------- a whole inverted-residual block as one kernel
+# (batch, H, W, Cin, hidden, Cout, stride): the block shapes of MobileNetV2 on 14x14 and 7x7 planes, small and odd
+# planes, hidden widths that are not a multiple of the 64-channel chunk, a batch that leaves the last unit half empty
+IR_CASES = [(3, 14, 14, 64, 384, 64, 1), (2, 14, 14, 64, 384, 96, 1), (2, 14, 14, 96, 576, 96, 1), (3, 14, 14, 96, 576, 160, 2),
+            (5, 7, 7, 160, 960, 160, 1), (4, 7, 7, 160, 960, 320, 1), (1, 7, 7, 16, 64, 16, 1), (3, 9, 5, 32, 100, 24, 1),
+            (2, 10, 12, 16, 72, 20, 2), (7, 3, 3, 48, 128, 48, 1), (2, 16, 16, 32, 192, 32, 1), (3, 11, 13, 16, 40, 16, 1)]
+
+
+@pytest.mark.parametrize("case", IR_CASES, ids=lambda c: "b%d_%dx%d_%d_%d_%d_s%d" % c)
+def test_inverted_residual_block_one_kernel(case):
+    b, h, w, cin, hidden, cout, stride = case
+    spec = wl.inverted_residual_block(b, h, w, cin, hidden, cout, stride)
+    run, xs, outs = check_outputs(spec, api.GI_F16, cross_op=api.GI_XOP_ON)
+    names = [api.KERNEL_NAMES[o.kernel] for o in run.ex.ops()]
+    assert names.count("inverted_residual") == 1 and names.count("none") == 2, names
+    again = run.run(xs)
+    for t in spec.outputs:
+        assert np.array_equal(outs[t], again[t])
+    assert api.gi_device_status() == 0
+
+
+@pytest.mark.parametrize("act,out_act", [(wl.ACT_RELU, None), (wl.ACT_NONE, wl.ACT_RELU6), (wl.ACT_RELU6, wl.ACT_RELU)])
+def test_inverted_residual_block_epilogues(act, out_act):
+    spec = wl.inverted_residual_block(3, 7, 7, 32, 96, 32, 1, act=act, out_act=out_act)
+    run, _, _ = check_outputs(spec, api.GI_F16, cross_op=api.GI_XOP_ON)
+    assert "inverted_residual" in [api.KERNEL_NAMES[o.kernel] for o in run.ex.ops()]
+
+
+def test_mobilenet_v2_batch32_blocks_as_one_kernel_every_tensor():
+    """Every stored tensor of the network with the ten 14x14 / 7x7 blocks as one kernel each (the hidden tensors of
+    those blocks are never stored: they are covered through the block outputs computed from them)."""
+    spec = wl.mobilenet_v2(4, size=224)
+    xs = [wl.make_input(spec)]
+    ref = og.run(spec, xs, storage="f16", fused=True, keep_all=True)
+    run = DeviceRun(spec, api.GI_F16, planner=api.GI_PLAN_NAIVE, guard_bytes=4096, cross_op=api.GI_XOP_ON)
+    names = [api.KERNEL_NAMES[o.kernel] for o in run.ex.ops()]
+    assert names.count("inverted_residual") == 10, names
+    outs = run.run(xs)
+    assert run.guard_intact()
+    for t, r in ref.items():
+        if t in run.on_chip:
+            continue
+        assert_close(outs[t] if t in outs else run.fetch(t), r, api.GI_F16, f"tensor {t}")
+    assert api.gi_device_status() == 0
