@@ -299,6 +299,9 @@ def run_sweep(args):
     elif args.sweep == "dwpw":  # the depthwise -> projection pairs of MobileNetV2 that have at least one tile per SM
         points = [(256, 112, 32, 16, 1), (256, 112, 96, 24, 2), (256, 56, 144, 24, 1), (256, 56, 144, 32, 2), (256, 28, 192, 32, 1),
                   (256, 28, 192, 64, 2), (256, 14, 384, 64, 1), (256, 14, 576, 96, 1)]
+    elif args.sweep == "block":  # the inverted-residual blocks of MobileNetV2 on 14x14 and 7x7 planes
+        points = [(256, 14, 64, 384, 64, 1), (256, 14, 64, 384, 96, 1), (256, 14, 96, 576, 96, 1), (256, 14, 96, 576, 160, 2),
+                  (256, 7, 160, 960, 160, 1), (256, 7, 160, 960, 320, 1)]
     elif args.sweep == "dw":
         points = [(b, hw, c, s) for b in (64, 256) for hw, c in ((112, 32), (112, 96), (56, 144), (28, 192), (14, 384),
                                                                  (14, 576), (7, 960)) for s in (1, 2)]
@@ -319,6 +322,10 @@ def run_sweep(args):
             b, hw, cin, cout, stride = pt
             spec = wl.single_conv3x3(b, hw, cin, cout, stride)
             name = f"conv3x3 b{b} {hw}x{hw} {cin}->{cout} s{stride}"
+        elif args.sweep == "block":
+            b, hw, cin, hidden, cout, stride = pt
+            spec = wl.inverted_residual_block(b, hw, hw, cin, hidden, cout, stride)
+            name = f"block b{b} {hw}x{hw} {cin}->{hidden}->{cout} s{stride}"
         elif args.sweep == "dwpw":
             b, hw, c, cout, stride = pt
             spec = wl.depthwise_then_pointwise(b, hw, hw, c, cout, stride, residual=args.residual)
@@ -335,7 +342,7 @@ def run_sweep(args):
         ex = g.compile(pointwise=PW_MODES[args.pointwise], cross_op=XOP_MODES[args.cross_op])
         ex.bind(dev)
         ops = ex.ops()
-        assert len(ops) == (2 if args.sweep in ("dwpw", "stem") else 1)
+        assert len(ops) == {"dwpw": 2, "stem": 2, "block": 3}.get(args.sweep, 1)
         # seeded images (the workload recipe), at most 8 distinct ones: image k of the batch is drawn image k % 8
         n_img = min(b, 8)
         xs_np = [wl.make_input(spec, images=list(range(n_img)), index=i) for i in range(len(spec.inputs))]
@@ -455,11 +462,12 @@ def main():
     ap.add_argument("--per-op", default=None, help="write the per-op timing table to this file")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-batch1", action="store_true", help="skip the batch-1 latency leg (keeps profiler runs short)")
-    ap.add_argument("--sweep", default=None, choices=["pw", "dw", "conv3", "dwpw", "stem"],
+    ap.add_argument("--sweep", default=None, choices=["pw", "dw", "conv3", "dwpw", "stem", "block"],
                     help="time single fused operators instead of a network")
     ap.add_argument("--points", default=None, help="sweep points 'B,HW,Cin,Cout;...' (pw), 'B,HW,C,stride;...' (dw), "
                     "'B,HW,Cin,Cout,stride;...' (conv3), 'B,HW,C,Cout,stride;...' (dwpw: depthwise then 1x1, see --cross-op), "
-                    "'B,HW,Cout;...' (stem: 3x3 stride-2 convolution of a 3-channel NHWC input, read in that layout)")
+                    "'B,HW,Cout;...' (stem: 3x3 stride-2 convolution of a 3-channel NHWC input, read in that layout), "
+                    "'B,HW,Cin,hidden,Cout,stride;...' (block: one inverted-residual block, see --cross-op)")
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--residual", action="store_true")
     ap.add_argument("--no-check", action="store_true", help="sweep: skip the comparison of sampled images with the CPU oracle")

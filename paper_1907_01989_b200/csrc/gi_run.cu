@@ -202,9 +202,10 @@ gi_status gi_run_timed(gi_exec* e, const void* const* dev_inputs, void* const* d
 namespace gi {
 int pointwise_ts_trace(unsigned long long* dst, int n);
 int depthwise_pointwise_trace(unsigned long long* dst, int n);
+int inverted_residual_trace(unsigned long long* dst, int n);
 }
 // debug builds only: copy the timeline table of the lane-per-pixel kernel's last launch
 extern "C" GI_API int gi_debug_trace(int which, unsigned long long* dst, int n) {
-  return which == 1 ? gi::depthwise_pointwise_trace(dst, n) : gi::pointwise_ts_trace(dst, n);
+  return which == 2 ? gi::inverted_residual_trace(dst, n) : which == 1 ? gi::depthwise_pointwise_trace(dst, n) : gi::pointwise_ts_trace(dst, n);
 }
 #endif

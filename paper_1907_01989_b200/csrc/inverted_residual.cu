@@ -53,6 +53,19 @@ constexpr int kSmemMax = 227 * 1024;
 constexpr int kDwBytes = (9 * kNh + kNh + kNh) * 4;  // depthwise taps, depthwise bias, expansion bias of a chunk
 
 __device__ unsigned int g_ir_error = 0;
+#ifdef GI_TRACE
+__device__ unsigned long long g_ir_trace[256 * 64];
+#define IR_EV(idx)                                           \
+  do {                                                       \
+    if (blockIdx.x < 256 && (idx) < 64) {                    \
+      unsigned long long t_;                                 \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); \
+      g_ir_trace[blockIdx.x * 64 + (idx)] = t_;              \
+    }                                                        \
+  } while (0)
+#else
+#define IR_EV(idx) ((void)0)
+#endif
 enum : unsigned { kErrCopy = 1u, kErrMma = 2u, kErrCompute = 4u, kErrDrain = 8u };
 
 struct IrParams {
@@ -74,7 +87,8 @@ struct IrParams {
   int n_bands, band_rows;
   int stages;
   unsigned stage_bytes, we_bytes, wp_bytes;
-  unsigned x_bytes, a2_bytes, h_bytes;
+  unsigned x_bytes, a2_bytes, h_bytes;  // h_bytes: ONE hidden tile (there are two)
+  unsigned x_pitch, a2_pitch;           // byte distance between the K groups (8 channels) of X / A2: rows x 16
   unsigned d2_col0;
   int act1, act2, act3, has_res, act4;  // after expansion, after depthwise, after projection, residual, after the sum
   unsigned timeout_ns;
@@ -96,14 +110,10 @@ __device__ __forceinline__ float act1f(float v, int kind) {
 // two floats -> fp16 pair with the activation applied: clamping the rounded value equals rounding the clamped
 // one because 0 and 6 are fp16 values
 __device__ __forceinline__ unsigned pack_act(float x, float y, int kind) {
-  unsigned d = pack_f16x2<false>(x, y);
-  if (kind != GI_ACT_NONE) {
-    __half2 h = *reinterpret_cast<__half2*>(&d);
-    h = __hmax2(h, __float2half2_rn(0.f));
-    if (kind == GI_ACT_RELU6) h = __hmin2(h, __float2half2_rn(6.f));
-    d = *reinterpret_cast<unsigned*>(&h);
-  }
-  return d;
+  if (kind == GI_ACT_NONE) return pack_f16x2<false>(x, y);
+  const unsigned d = pack_f16x2<true>(x, y);  // the conversion clamps at zero itself
+  // non-negative fp16 values order like 16-bit integers: the clamp at 6 is an integer minimum
+  return kind == GI_ACT_RELU6 ? __vmins2(d, 0x46004600u) : d;
 }
 __device__ __forceinline__ uint2 lds64(unsigned addr) {
   uint2 v;
@@ -136,6 +146,18 @@ __device__ __forceinline__ Tap tap_of(uint2 v) {
   return t;
 }
 
+// 16 accumulator columns (four 4-channel slices of one pixel) -> bias, activation, fp16 -> the pixel's place in the
+// four slices' planes of the hidden tile (`pitch` bytes apart); `bias` is the shared-memory address of the 16 biases
+__device__ __forceinline__ void store_hidden(const unsigned (&r)[16], unsigned bias, unsigned at, unsigned pitch, bool valid, int act) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float4 b = lds128f(bias + static_cast<unsigned>(i) * 16u);
+    const float2 v0 = __fadd2_rn(make_float2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), make_float2(b.x, b.y));
+    const float2 v1 = __fadd2_rn(make_float2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), make_float2(b.z, b.w));
+    if (valid) sts64(at + static_cast<unsigned>(i) * pitch, pack_act(v0.x, v0.y, act), pack_act(v1.x, v1.y, act));
+  }
+}
+
 template <int STRIDE>
 __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const IrParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
@@ -144,8 +166,8 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
   volatile unsigned* abort_flag = &hdr->abort_flag;
   const unsigned x0 = smem_u32(smem + kHeader);
   const unsigned a20 = x0 + p.x_bytes;
-  const unsigned h0 = a20 + p.a2_bytes;
-  const unsigned st0 = h0 + p.h_bytes;
+  const unsigned h0 = a20 + p.a2_bytes;           // two hidden tiles of h_bytes each
+  const unsigned st0 = h0 + 2u * p.h_bytes;
   const unsigned d1_cols = static_cast<unsigned>(p.mt_in) * kNh;  // one D1 buffer
 
   if (threadIdx.x == 0) {
@@ -182,7 +204,7 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
       for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
         for (int c = 0; c < p.n_chunks; ++c, ++g) {
           const unsigned stage = g % p.stages, phase = (g / p.stages) & 1u;
-          if (!mbar_wait(smem_u32(&hdr->w_empty[stage]), phase ^ 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCopy)) {
+          if (!mbar_wait_parked(smem_u32(&hdr->w_empty[stage]), phase ^ 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCopy)) {
             ok = false;
             break;
           }
@@ -210,68 +232,78 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
     if (lane == 0) {
       const unsigned idesc1 = (1u << 4) | ((static_cast<unsigned>(kNh) >> 3) << 17) | ((128u >> 4) << 24);
       const unsigned idesc2 = (1u << 4) | ((static_cast<unsigned>(p.n_each) >> 3) << 17) | ((128u >> 4) << 24);
-      const unsigned x_lbo = static_cast<unsigned>(p.mt_in) * 2048u;    // K group pitch of X: rows x 16 bytes
-      const unsigned a2_lbo = static_cast<unsigned>(p.mt_out) * 2048u;  // of A2
       const unsigned we_lbo = kNh * 16u, wp_lbo = static_cast<unsigned>(p.cout_pad) * 16u;
       const int k_steps1 = p.s_in / 4;  // 16 input channels per MMA
       unsigned g = 0, ul = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++ul) {
-        if (!mbar_wait(smem_u32(&hdr->x_full), ul & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma)) break;
+      // expansion of chunk c of the current unit (global chunk number gc) into D1[gc & 1]
+      auto expand = [&](unsigned gc) -> bool {
+        const unsigned stage = gc % p.stages, buf = gc & 1u;
+        if (!mbar_wait_parked(smem_u32(&hdr->w_full[stage]), (gc / p.stages) & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma) ||
+            !mbar_wait_parked(smem_u32(&hdr->d1_empty[buf]), ((gc >> 1) & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma))
+          return false;
         tc_fence_after();
-        for (int c = 0; c <= p.n_chunks && ok; ++c) {
-          if (c < p.n_chunks) {
-            const unsigned gc = g + c, stage = gc % p.stages, buf = gc & 1u;
-            if (!mbar_wait(smem_u32(&hdr->w_full[stage]), (gc / p.stages) & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma) ||
-                !mbar_wait(smem_u32(&hdr->d1_empty[buf]), ((gc >> 1) & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma)) {
-              ok = false;
-              break;
-            }
-            tc_fence_after();
-            const unsigned we = st0 + stage * p.stage_bytes;
-            for (int t = 0; t < p.mt_in; ++t) {
-              const unsigned d = tmem_base + buf * d1_cols + static_cast<unsigned>(t) * kNh;
-              unsigned long long ad = smem_desc(x0 + static_cast<unsigned>(t) * 2048u, x_lbo, 128);
-              unsigned long long bd = smem_desc(we, we_lbo, 128);
-              const unsigned long long ad_step = static_cast<unsigned long long>((2u * x_lbo) >> 4);
-              const unsigned long long bd_step = static_cast<unsigned long long>((2u * we_lbo) >> 4);
-              for (int ks = 0; ks < k_steps1; ++ks) {
-                umma_f16(d, ad, bd, idesc1, ks > 0 ? 1u : 0u);
+        const unsigned we = st0 + stage * p.stage_bytes;
+        for (int t = 0; t < p.mt_in; ++t) {
+          const unsigned d = tmem_base + buf * d1_cols + static_cast<unsigned>(t) * kNh;
+          unsigned long long ad = smem_desc(x0 + static_cast<unsigned>(t) * 2048u, p.x_pitch, 128);
+          unsigned long long bd = smem_desc(we, we_lbo, 128);
+          const unsigned long long ad_step = static_cast<unsigned long long>((2u * p.x_pitch) >> 4);
+          const unsigned long long bd_step = static_cast<unsigned long long>((2u * we_lbo) >> 4);
+          for (int ks = 0; ks < k_steps1; ++ks) {
+            umma_f16(d, ad, bd, idesc1, ks > 0 ? 1u : 0u);
+            ad += ad_step;
+            bd += bd_step;
+          }
+        }
+        umma_commit(smem_u32(&hdr->d1_full[buf]));
+        return true;
+      };
+      for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++ul) {
+        if (!mbar_wait_parked(smem_u32(&hdr->x_full), ul & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma)) break;
+        tc_fence_after();
+        // the expansions run two chunks ahead of the projections: their accumulators are drained one chunk early
+        ok = expand(g);
+        if (ok && p.n_chunks > 1) ok = expand(g + 1);
+        if (ok && ul == 0) IR_EV(6);
+        for (int c = 0; c < p.n_chunks && ok; ++c) {
+          const unsigned gp = g + c, stage = gp % p.stages;
+          // with three stages the weights of chunk c + 2 arrive while chunk c is being worked on; with two, its stage
+          // is the one projection(c) frees, so that expansion can only follow the projection
+          const bool early = p.stages >= 3 && c + 2 < p.n_chunks;
+          if (early) {
+            ok = expand(gp + 2);
+            if (!ok) break;
+            if (ul == 0) IR_EV(8 * (c + 2) + 6);
+          }
+          if (c == 0 && !mbar_wait_parked(smem_u32(&hdr->d2_empty), (ul & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma)) {
+            ok = false;
+            break;
+          }
+          if (!mbar_wait_parked(smem_u32(&hdr->a2_full), gp & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const unsigned wp = st0 + stage * p.stage_bytes + p.we_bytes;
+          for (int t = 0; t < p.mt_out; ++t)
+            for (int h = 0; h < p.n_split; ++h) {
+              const unsigned d = tmem_base + p.d2_col0 + static_cast<unsigned>(t * p.cout_pad + h * p.n_each);
+              unsigned long long ad = smem_desc(a20 + static_cast<unsigned>(t) * 2048u, p.a2_pitch, 128);
+              unsigned long long bd = smem_desc(wp + static_cast<unsigned>(h * p.n_each) * 16u, wp_lbo, 128);
+              const unsigned long long ad_step = static_cast<unsigned long long>((2u * p.a2_pitch) >> 4);
+              const unsigned long long bd_step = static_cast<unsigned long long>((2u * wp_lbo) >> 4);
+              for (int ks = 0; ks < kNh / 16; ++ks) {
+                umma_f16(d, ad, bd, idesc2, (c > 0 || ks > 0) ? 1u : 0u);
                 ad += ad_step;
                 bd += bd_step;
               }
             }
-            umma_commit(smem_u32(&hdr->d1_full[buf]));
-          }
-          if (c >= 1) {
-            const unsigned gp = g + c - 1, stage = gp % p.stages;
-            if (c == 1 && !mbar_wait(smem_u32(&hdr->d2_empty), (ul & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma)) {
-              ok = false;
-              break;
-            }
-            if (!mbar_wait(smem_u32(&hdr->a2_full), gp & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma)) {
-              ok = false;
-              break;
-            }
-            tc_fence_after();
-            const unsigned wp = st0 + stage * p.stage_bytes + p.we_bytes;
-            for (int t = 0; t < p.mt_out; ++t)
-              for (int h = 0; h < p.n_split; ++h) {
-                const unsigned d = tmem_base + p.d2_col0 + static_cast<unsigned>(t * p.cout_pad + h * p.n_each);
-                unsigned long long ad = smem_desc(a20 + static_cast<unsigned>(t) * 2048u, a2_lbo, 128);
-                unsigned long long bd = smem_desc(wp + static_cast<unsigned>(h * p.n_each) * 16u, wp_lbo, 128);
-                const unsigned long long ad_step = static_cast<unsigned long long>((2u * a2_lbo) >> 4);
-                const unsigned long long bd_step = static_cast<unsigned long long>((2u * wp_lbo) >> 4);
-                for (int ks = 0; ks < kNh / 16; ++ks) {
-                  umma_f16(d, ad, bd, idesc2, (c > 1 || ks > 0) ? 1u : 0u);
-                  ad += ad_step;
-                  bd += bd_step;
-                }
-              }
-            umma_commit(smem_u32(&hdr->a2_empty));
-            umma_commit(smem_u32(&hdr->w_empty[stage]));
-            if (c == p.n_chunks) umma_commit(smem_u32(&hdr->d2_full));
-          }
+          umma_commit(smem_u32(&hdr->a2_empty));
+          umma_commit(smem_u32(&hdr->w_empty[stage]));
+          if (c == p.n_chunks - 1) umma_commit(smem_u32(&hdr->d2_full));
+          if (ul == 0) IR_EV(8 * c + 7);
+          if (!early && p.stages < 3 && c + 2 < p.n_chunks) ok = expand(gp + 2);
         }
         g += p.n_chunks;
       }
@@ -294,15 +326,26 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
         const int img = r / p.r_in, q = r - img * p.r_in;
         if (b0 + img >= p.B) continue;
         const __half* src = p.in + ((static_cast<size_t>(s) * p.B + b0 + img) * p.Pin + q) * 4;
-        cp_async8(x0 + static_cast<unsigned>(s >> 1) * (static_cast<unsigned>(p.mt_in) * 2048u) + static_cast<unsigned>(r) * 16u +
-                      static_cast<unsigned>(s & 1) * 8u,
-                  src);
+        cp_async8(x0 + static_cast<unsigned>(s >> 1) * p.x_pitch + static_cast<unsigned>(r) * 16u + static_cast<unsigned>(s & 1) * 8u, src);
       }
     };
 
-    // the hidden tile's border is the zero padding of the depthwise convolution: cleared once, never written again
-    for (unsigned i = ctid; i < p.h_bytes / 16u; i += kComputeThreads)
+    // the hidden tiles' borders are the zero padding of the depthwise convolution: cleared once, never written again
+    for (unsigned i = ctid; i < 2u * p.h_bytes / 16u; i += kComputeThreads)
       asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(h0 + i * 16u), "r"(0u) : "memory");
+
+    // where this thread's accumulator rows go in a hidden tile (its rows are fixed: lane of the quarter, per 128-row tile)
+    unsigned dr_off[2];
+    bool dr_valid[2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      const int row = t * 128 + quarter * 32 + lane;
+      const int img = row / p.r_in, q = row - img * p.r_in;
+      const int y = q / p.W, x = q - y * p.W;
+      dr_valid[t] = t < p.mt_in && row < rows_in;
+      dr_off[t] = (static_cast<unsigned>(img) * p.plane_words + static_cast<unsigned>((y + 1) * p.Wp + x + 1)) * 8u;
+    }
+    const unsigned slice_pitch = static_cast<unsigned>(p.n_img) * p.plane_words * 8u;  // planes of one slice: one per image
 
     // this thread's place in the stencil: (band, plane = slice of the chunk x image, output column)
     const int planes = (kNh / 4) * p.n_img;
@@ -313,56 +356,68 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
     const int st_plane = st_rem / p.Wo, st_ox = st_rem - st_plane * p.Wo;
     const int st_slice = st_plane / p.n_img, st_img = st_plane - st_slice * p.n_img;
     const int st_r0 = band * p.band_rows, st_r1 = min(p.Ho, st_r0 + p.band_rows);
-    const unsigned st_h = h0 + static_cast<unsigned>(st_plane) * p.plane_words * 8u;
-    const unsigned st_a2 = a20 + static_cast<unsigned>(st_slice >> 1) * (static_cast<unsigned>(p.mt_out) * 2048u) +
-                           static_cast<unsigned>(st_img * p.r_out) * 16u + static_cast<unsigned>(st_slice & 1) * 8u;
+    const unsigned st_hoff = static_cast<unsigned>(st_plane) * p.plane_words * 8u;
+    const unsigned st_a2 = a20 + static_cast<unsigned>(st_slice >> 1) * p.a2_pitch + static_cast<unsigned>(st_img * p.r_out) * 16u +
+                           static_cast<unsigned>(st_slice & 1) * 8u;
 
-    pdl_wait();  // activations are read and written only below
     bool ok = true;
+    // ---- drain D1 of global chunk gc: 16 hidden channels of one pixel per tcgen05.ld; bias, activation, fp16 -> hidden tile gc & 1
+    auto drain = [&](unsigned gc, int ev) {
+      const unsigned stage = gc % p.stages, buf = gc & 1u;
+      const unsigned eb0 = st0 + stage * p.stage_bytes + p.we_bytes + p.wp_bytes + 10u * kNh * 4u;  // expansion bias of the chunk
+      const unsigned hb = h0 + buf * p.h_bytes;
+      if (ev >= 0 && ctid == 0 && ev / 8 < 6) IR_EV(48 + 2 * (ev / 8));
+      ok = ok && mbar_wait_warp(smem_u32(&hdr->w_full[stage]), (gc / p.stages) & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
+      if (ev >= 0 && ctid == 0 && ev / 8 < 6) IR_EV(49 + 2 * (ev / 8));
+      ok = ok && mbar_wait_warp(smem_u32(&hdr->d1_full[buf]), (gc >> 1) & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
+      if (ev >= 0 && ctid == 0) IR_EV(ev);
+      if (ok) {
+        tc_fence_after();
+        // a warp takes 16 columns (j = its index among the four warps of its lane quarter) of each tile; both tiles'
+        // loads are issued before either is used
+        const int j = qsub;
+        unsigned r0[16], r1[16];
+        tmem_ld16(tmem_base + lane_bits + buf * d1_cols + static_cast<unsigned>(j * 16), r0);
+        if (p.mt_in > 1) tmem_ld16(tmem_base + lane_bits + buf * d1_cols + static_cast<unsigned>(kNh + j * 16), r1);
+        const unsigned dst = hb + static_cast<unsigned>(j * 4) * slice_pitch;
+        tmem_ld_wait16(r0);
+        store_hidden(r0, eb0 + static_cast<unsigned>(j) * 64u, dst + dr_off[0], slice_pitch, dr_valid[0], p.act1);
+        if (p.mt_in > 1) {
+          tmem_ld_wait16(r1);
+          store_hidden(r1, eb0 + static_cast<unsigned>(j) * 64u, dst + dr_off[1], slice_pitch, dr_valid[1], p.act1);
+        }
+        tc_fence_before();
+      }
+      __syncwarp();
+      if (lane == 0 && ok) mbar_arrive(smem_u32(&hdr->d1_empty[buf]));
+    };
+
+    if (ctid == 0) IR_EV(60);
+    pdl_wait();  // activations are read and written only below
+    if (ctid == 0) IR_EV(61);
     if (static_cast<int>(blockIdx.x) < p.units) issue_x(blockIdx.x);
     cp_async_wait_all();
     fence_async_proxy();
     bar_compute();
     if (ctid == 0 && static_cast<int>(blockIdx.x) < p.units) mbar_arrive(smem_u32(&hdr->x_full));
+    if (ctid == 0) IR_EV(62);
 
     unsigned g = 0, ul = 0;
     for (int u = blockIdx.x; u < p.units; u += gridDim.x, ++ul) {
       const int b0 = u * p.n_img;
+      const bool more = u + static_cast<int>(gridDim.x) < p.units;
+      drain(g, -1);
+      bar_compute();  // hidden tile of chunk 0 complete
       for (int c = 0; c < p.n_chunks; ++c) {
-        const unsigned gc = g + c, stage = gc % p.stages, buf = gc & 1u;
-        const unsigned stg = st0 + stage * p.stage_bytes;
-        const unsigned dw0 = stg + p.we_bytes + p.wp_bytes;  // depthwise taps [9][64], depthwise bias [64], expansion bias [64]
-        ok = ok && mbar_wait_warp(smem_u32(&hdr->w_full[stage]), (gc / p.stages) & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
-        ok = ok && mbar_wait_warp(smem_u32(&hdr->d1_full[buf]), (gc >> 1) & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
-        if (ok) {
-          tc_fence_after();
-          // ---- drain D1: 16 hidden channels of one pixel per tcgen05.ld; bias, activation, fp16 -> hidden tile
-          for (int e = qsub; e < p.mt_in * 4; e += 4) {
-            const int t = e >> 2, j = e & 3;
-            unsigned r[16];
-            tmem_ld16(tmem_base + lane_bits + buf * d1_cols + static_cast<unsigned>(t * kNh + j * 16), r);
-            const int row = t * 128 + quarter * 32 + lane;
-            const int img = row / p.r_in, q = row - img * p.r_in;
-            const int y = q / p.W, x = q - y * p.W;
-            const bool valid = row < rows_in;
-            tmem_ld_wait16(r);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const int sl = j * 4 + i;
-              const float4 b = lds128f(dw0 + (10 * kNh + sl * 4) * 4u);
-              const unsigned w0 = pack_act(__uint_as_float(r[4 * i]) + b.x, __uint_as_float(r[4 * i + 1]) + b.y, p.act1);
-              const unsigned w1 = pack_act(__uint_as_float(r[4 * i + 2]) + b.z, __uint_as_float(r[4 * i + 3]) + b.w, p.act1);
-              if (valid)
-                sts64(h0 + (static_cast<unsigned>(sl * p.n_img + img) * p.plane_words + static_cast<unsigned>((y + 1) * p.Wp + x + 1)) * 8u, w0, w1);
-            }
-          }
-          tc_fence_before();
-        }
-        __syncwarp();
-        if (lane == 0 && ok) mbar_arrive(smem_u32(&hdr->d1_empty[buf]));
-        // the last expansion of this unit is complete (its accumulator was just read): X may be overwritten
-        if (c == p.n_chunks - 1 && u + static_cast<int>(gridDim.x) < p.units && ok) issue_x(u + gridDim.x);
-        bar_compute();  // the hidden tile is complete
+        const unsigned gc = g + c, stage = gc % p.stages;
+        const unsigned dw0 = st0 + stage * p.stage_bytes + p.we_bytes + p.wp_bytes;  // depthwise taps [9][64], depthwise bias [64]
+        if (ctid == 0 && ul == 0) IR_EV(8 * c + 0);
+        // the next chunk's expansion has long finished: drain it into the other hidden tile while the projection of the
+        // previous chunk, which still reads A2, completes
+        if (c + 1 < p.n_chunks) drain(gc + 1, ul == 0 ? 8 * c + 2 : -1);
+        // the last expansion of this unit is complete (its accumulator has been read): X may be overwritten
+        else if (more && ok) issue_x(u + gridDim.x);
+        if (ctid == 0 && ul == 0) IR_EV(8 * c + 1);
 
         // ---- this thread's depthwise weights (its slice of the chunk) into registers, then the stage is released
         float2 wlo[9], whi[9];
@@ -381,12 +436,13 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
         __syncwarp();
         if (lane == 0 && ok) mbar_arrive(smem_u32(&hdr->w_empty[stage]));
         ok = ok && mbar_wait_warp(smem_u32(&hdr->a2_empty), (gc & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
+        if (ctid == 0 && ul == 0) IR_EV(8 * c + 3);
 
         // ---- depthwise 3x3 from the hidden tile -> A operand of the projection
         if (ok && st_active) {
+          const unsigned st_h = h0 + (gc & 1u) * p.h_bytes + st_hoff;
           auto emit = [&](const Tap& a, int oy) {
-            const unsigned w0 = pack_act(a.lo.x, a.lo.y, p.act2), w1 = pack_act(a.hi.x, a.hi.y, p.act2);
-            sts64(st_a2 + static_cast<unsigned>(oy * p.Wo + st_ox) * 16u, w0, w1);
+            sts64(st_a2 + static_cast<unsigned>(oy * p.Wo + st_ox) * 16u, pack_act(a.lo.x, a.lo.y, p.act2), pack_act(a.hi.x, a.hi.y, p.act2));
           };
           if (STRIDE == 1) {
             // padded row iy (image row iy - 1) is tap row 0 of output row iy, row 1 of iy - 1, row 2 of iy - 2
@@ -441,61 +497,90 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
             }
           }
         }
+        if (ctid == 0 && ul == 0) IR_EV(8 * c + 4);
         fence_async_proxy();  // the A operand was written with ordinary stores; the MMA reads it through the async proxy
-        bar_compute();        // A2 complete; nobody reads the hidden tile any more
+        bar_compute();        // A2 and the next hidden tile are complete; nobody reads this chunk's hidden tile any more
         if (ctid == 0 && ok) mbar_arrive(smem_u32(&hdr->a2_full));
+        if (ctid == 0 && ul == 0) IR_EV(8 * c + 5);
       }
       g += p.n_chunks;
 
-      // ---- the next unit's X has been on its way since the last drain: publish it, then drain this unit's D2
-      const bool more = u + static_cast<int>(gridDim.x) < p.units;
+      // ---- the next unit's X has been on its way since the last chunk began: publish it, then drain this unit's D2
       if (more) {
         cp_async_wait_all();
         fence_async_proxy();
         bar_compute();
         if (ctid == 0 && ok) mbar_arrive(smem_u32(&hdr->x_full));
       }
+      // the residual does not depend on the accumulator: the first item's is fetched before waiting for the last
+      // projection, each further item's while the one before it is processed
+      const int groups = p.cout_pad >> 4, n_items = p.mt_out * groups;
+      auto item_px = [&](int e, int* t, int* j, size_t* px, bool* valid) {
+        *t = e / groups;
+        *j = e - *t * groups;
+        const int row = *t * 128 + quarter * 32 + lane;
+        const int img = row / p.r_out, q = row - img * p.r_out;
+        *valid = e < n_items && row < rows_out && b0 + img < p.B;
+        *px = static_cast<size_t>(b0 + img) * p.Pout + q;
+      };
+      auto fetch_res = [&](uint2* dstq, int e) {
+        int t, j;
+        size_t px;
+        bool valid;
+        item_px(e, &t, &j, &px, &valid);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int so = j * 4 + i;
+          dstq[i] = make_uint2(0u, 0u);
+          if (p.has_res && valid && so < p.s_out)
+            dstq[i] = __ldg(reinterpret_cast<const uint2*>(p.res + (static_cast<size_t>(so) * p.B * p.Pout + px) * 4));
+        }
+      };
+      uint2 res_cur[4], res_nxt[4];
+      fetch_res(res_cur, qsub);
       ok = ok && mbar_wait_warp(smem_u32(&hdr->d2_full), ul & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
       if (ok) {
         tc_fence_after();
-        const int groups = p.cout_pad >> 4;
-        for (int e = qsub; e < p.mt_out * groups; e += 4) {
-          const int t = e / groups, j = e - t * groups;
+        for (int e = qsub; e < n_items; e += 4) {
+          int t, j;
+          size_t px;
+          bool valid;
+          item_px(e, &t, &j, &px, &valid);
           unsigned r[16];
           tmem_ld16(tmem_base + lane_bits + p.d2_col0 + static_cast<unsigned>(t * p.cout_pad + j * 16), r);
-          const int row = t * 128 + quarter * 32 + lane;
-          const int img = row / p.r_out, q = row - img * p.r_out;
-          const bool valid = row < rows_out && b0 + img < p.B;
+          fetch_res(res_nxt, e + 4);
           tmem_ld_wait16(r);
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const int so = j * 4 + i;
             if (so >= p.s_out || !valid) continue;
             const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias2) + so);
-            const size_t off = ((static_cast<size_t>(so) * p.B + b0 + img) * p.Pout + q) * 4;  // in halves
+            const size_t off = (static_cast<size_t>(so) * p.B * p.Pout + px) * 4;  // in halves
             float v0 = act1f(__uint_as_float(r[4 * i]) + b.x, p.act3), v1 = act1f(__uint_as_float(r[4 * i + 1]) + b.y, p.act3);
             float v2 = act1f(__uint_as_float(r[4 * i + 2]) + b.z, p.act3), v3 = act1f(__uint_as_float(r[4 * i + 3]) + b.w, p.act3);
             if (p.has_res) {
-              const uint2 rq = __ldg(reinterpret_cast<const uint2*>(p.res + off));
-              const float2 r0 = __half22float2(*reinterpret_cast<const __half2*>(&rq.x));
-              const float2 r1 = __half22float2(*reinterpret_cast<const __half2*>(&rq.y));
-              v0 += r0.x;
-              v1 += r0.y;
-              v2 += r1.x;
-              v3 += r1.y;
+              const float2 q0 = __half22float2(*reinterpret_cast<const __half2*>(&res_cur[i].x));
+              const float2 q1 = __half22float2(*reinterpret_cast<const __half2*>(&res_cur[i].y));
+              v0 += q0.x;
+              v1 += q0.y;
+              v2 += q1.x;
+              v3 += q1.y;
             }
             uint2 o;
             o.x = pack_f16x2<false>(act1f(v0, p.act4), act1f(v1, p.act4));
             o.y = pack_f16x2<false>(act1f(v2, p.act4), act1f(v3, p.act4));
             *reinterpret_cast<uint2*>(p.out + off) = o;
             // an odd plane is stored with one extra pixel, which readers expect to be finite: zero it
-            if (q == p.r_out - 1 && p.Pout > p.r_out) *reinterpret_cast<uint2*>(p.out + off + 4) = make_uint2(0u, 0u);
+            if (p.Pout > p.r_out && (px + 1) % p.Pout == static_cast<size_t>(p.r_out)) *reinterpret_cast<uint2*>(p.out + off + 4) = make_uint2(0u, 0u);
           }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) res_cur[i] = res_nxt[i];
         }
         tc_fence_before();
       }
       __syncwarp();
       if (lane == 0 && ok) mbar_arrive(smem_u32(&hdr->d2_empty));
+      if (ctid == 0 && ul == 0) IR_EV(63);
     }
   }
 
@@ -510,7 +595,7 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
 
 struct Shape {
   int n_img, mt_in, mt_out, r_in, r_out, n_chunks, cout_pad, n_split, n_each, Wp, plane_words, n_bands, band_rows, stages;
-  unsigned we_bytes, wp_bytes, stage_bytes, x_bytes, a2_bytes, h_bytes;
+  unsigned we_bytes, wp_bytes, stage_bytes, x_bytes, a2_bytes, h_bytes, x_pitch, a2_pitch;
   size_t smem;
   long long units;
   bool ok;
@@ -548,10 +633,16 @@ Shape shape_of(int B, int H, int W, int Ho, int Wo, int stride, int cin, int chi
   s.we_bytes = static_cast<unsigned>(kNh) * cin * 2u;
   s.wp_bytes = static_cast<unsigned>(s.cout_pad) * kNh * 2u;
   s.stage_bytes = s.we_bytes + s.wp_bytes + kDwBytes;
-  s.x_bytes = static_cast<unsigned>(cin / 8) * s.mt_in * 2048u;
-  s.a2_bytes = static_cast<unsigned>(kNh / 8) * s.mt_out * 2048u;
-  s.h_bytes = (static_cast<unsigned>(planes) * s.plane_words * 8u + 15u) / 16u * 16u;
-  const long long fixed = kHeader + static_cast<long long>(s.x_bytes) + s.a2_bytes + s.h_bytes;
+  // The K groups of an operand lie `rows x 16 bytes` apart, rows = the unit's real pixel count.  An MMA reads 128
+  // rows per tile, so the tail of the last tile reads on into the next K group (and, for the last group, into the
+  // region behind the operand): rows that hold no pixel, whose results are never stored.
+  s.x_pitch = static_cast<unsigned>(s.n_img * s.r_in) * 16u;
+  s.a2_pitch = static_cast<unsigned>(s.n_img * s.r_out) * 16u;
+  s.x_bytes = (static_cast<unsigned>(cin / 8) * s.x_pitch + 127u) / 128u * 128u;
+  s.a2_bytes = (static_cast<unsigned>(kNh / 8) * s.a2_pitch + 127u) / 128u * 128u;
+  s.h_bytes = (static_cast<unsigned>(planes) * s.plane_words * 8u + 127u) / 128u * 128u;
+  // (the tail reads of A2's last K group land in the hidden tiles, 2 x h_bytes >= 2 KB, those of X in A2 or behind)
+  const long long fixed = kHeader + static_cast<long long>(s.x_bytes) + s.a2_bytes + 2ll * s.h_bytes;
   long long stages = (kSmemMax - fixed) / s.stage_bytes;
   if (stages < 2) return s;
   s.stages = stages > kMaxStages ? kMaxStages : static_cast<int>(stages);
@@ -669,6 +760,8 @@ int launch_inverted_residual(const LaunchRec& r, const Ptrs& p, void* stream) {
   k.x_bytes = s.x_bytes;
   k.a2_bytes = s.a2_bytes;
   k.h_bytes = s.h_bytes;
+  k.x_pitch = s.x_pitch;
+  k.a2_pitch = s.a2_pitch;
   k.d2_col0 = 2u * static_cast<unsigned>(s.mt_in) * kNh;
   k.act1 = r.ep.act_pre;
   k.act2 = r.ep_mid.act_pre;
@@ -694,6 +787,13 @@ int launch_inverted_residual(const LaunchRec& r, const Ptrs& p, void* stream) {
   else launch_pdl(inverted_residual_kernel<2>, grid, kThreads, smem, st, k);
   return static_cast<int>(cudaGetLastError());
 }
+
+#ifdef GI_TRACE
+int inverted_residual_trace(unsigned long long* dst, int n) {
+  const size_t bytes = sizeof(unsigned long long) * (n < 256 * 64 ? n : 256 * 64);
+  return static_cast<int>(cudaMemcpyFromSymbol(dst, g_ir_trace, bytes));
+}
+#endif
 
 unsigned int inverted_residual_error_word(int* cuda_err) {
   unsigned int v = 0;

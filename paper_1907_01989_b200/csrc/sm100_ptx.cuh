@@ -91,10 +91,14 @@ static __device__ __noinline__ bool mbar_wait_parked(unsigned bar, unsigned pari
 // The same wait for a whole warp that goes on to warp-collective instructions (tcgen05.ld / .st / .wait are
 // .sync.aligned: all 32 lanes must execute them together).  Lanes leave the polling loop at different
 // iterations; the vote brings them back together and gives every lane the same answer, so that the warp
-// also gives up as one.
+// also gives up as one.  A phase that has already completed - the common case for a consumer that runs behind
+// its producer - is recognised by one inline poll, without the call into the bounded-wait routine.
+// (Letting one lane poll for the warp, with a warp barrier and a shuffle behind it, measured slower: +1 us per
+// kernel at batch 1.)
 __device__ __forceinline__ bool mbar_wait_warp(unsigned bar, unsigned parity, volatile unsigned* abort_flag, unsigned timeout_ns,
                                                unsigned* error_word, unsigned code) {
-  const bool ok = mbar_wait(bar, parity, abort_flag, timeout_ns, error_word, code);
+  bool ok = mbar_try_wait(bar, parity);
+  if (!ok) ok = mbar_wait(bar, parity, abort_flag, timeout_ns, error_word, code);
   return __all_sync(0xffffffffu, ok) != 0;
 }
 
