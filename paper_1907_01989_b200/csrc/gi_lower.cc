@@ -304,7 +304,7 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
             const TensorDesc& dd = e->tensors[fd.out];
             if (inverted_residual_supported(e->batch, din->h, din->w, dd.h, dd.w, dwn.d.stride_h, dwn.d.dilation_h, dwn.d.pad_t,
                                             dwn.d.pad_l, din->c, op.d.cout, pwn.d.cout, &ir_units) &&
-                (e->opt.cross_op == GI_XOP_ON || ir_units >= 96)) {
+                (e->opt.cross_op == GI_XOP_ON || (ir_units >= 96 && din->h * din->w <= 64))) {
               const TensorDesc& d2 = e->tensors[fp.out];
               r.kernel = GI_KERNEL_INVERTED_RESIDUAL;
               r.Ho = dd.h;

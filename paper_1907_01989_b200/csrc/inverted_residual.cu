@@ -47,6 +47,7 @@ constexpr int kNh = 64;  // hidden channels per chunk
 constexpr int kComputeWarps = 16;
 constexpr int kComputeThreads = 32 * kComputeWarps;
 constexpr int kThreads = 64 + kComputeThreads;
+constexpr int kTeamWarps = kComputeWarps / 2, kTeamThreads = 32 * kTeamWarps;  // two teams take alternate chunks
 constexpr int kMaxStages = 3;
 constexpr int kHeader = 1024;
 constexpr int kSmemMax = 227 * 1024;
@@ -97,7 +98,7 @@ struct IrParams {
 struct Header {
   unsigned long long w_full[kMaxStages], w_empty[kMaxStages];
   unsigned long long d1_full[2], d1_empty[2];
-  unsigned long long a2_full, a2_empty, d2_full, d2_empty, x_full;
+  unsigned long long a2_full[2], a2_empty[2], d2_full, d2_empty, x_full;
   unsigned tmem_addr, abort_flag;
 };
 static_assert(sizeof(Header) <= kHeader, "header too large");
@@ -112,8 +113,9 @@ __device__ __forceinline__ float act1f(float v, int kind) {
 __device__ __forceinline__ unsigned pack_act(float x, float y, int kind) {
   if (kind == GI_ACT_NONE) return pack_f16x2<false>(x, y);
   const unsigned d = pack_f16x2<true>(x, y);  // the conversion clamps at zero itself
-  // non-negative fp16 values order like 16-bit integers: the clamp at 6 is an integer minimum
-  return kind == GI_ACT_RELU6 ? __vmins2(d, 0x46004600u) : d;
+  if (kind != GI_ACT_RELU6) return d;
+  const __half2 h = __hmin2(*reinterpret_cast<const __half2*>(&d), __float2half2_rn(6.f));
+  return *reinterpret_cast<const unsigned*>(&h);
 }
 __device__ __forceinline__ uint2 lds64(unsigned addr) {
   uint2 v;
@@ -135,6 +137,8 @@ __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wai
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 // barrier of the compute warps only (id 1); the copy and MMA warps never join it
 __device__ __forceinline__ void bar_compute() { asm volatile("bar.sync 1, %0;" ::"n"(kComputeThreads) : "memory"); }
+// barrier of one team of compute warps (ids 2 and 3)
+__device__ __forceinline__ void bar_team(int team) { asm volatile("bar.sync %0, %1;" ::"r"(2 + team), "n"(kTeamThreads) : "memory"); }
 
 struct Tap {
   float2 lo, hi;
@@ -147,18 +151,64 @@ __device__ __forceinline__ Tap tap_of(uint2 v) {
 }
 
 // 16 accumulator columns (four 4-channel slices of one pixel) -> bias, activation, fp16 -> the pixel's place in the
-// four slices' planes of the hidden tile (`pitch` bytes apart); `bias` is the shared-memory address of the 16 biases
-__device__ __forceinline__ void store_hidden(const unsigned (&r)[16], unsigned bias, unsigned at, unsigned pitch, bool valid, int act) {
+// four slices' planes of the hidden tile (`pitch` bytes apart)
+__device__ __forceinline__ void store_hidden(const unsigned (&r)[16], const float4 (&b)[4], unsigned at, unsigned pitch, bool valid, int act) {
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const float4 b = lds128f(bias + static_cast<unsigned>(i) * 16u);
-    const float2 v0 = __fadd2_rn(make_float2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), make_float2(b.x, b.y));
-    const float2 v1 = __fadd2_rn(make_float2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), make_float2(b.z, b.w));
+    const float2 v0 = __fadd2_rn(make_float2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), make_float2(b[i].x, b[i].y));
+    const float2 v1 = __fadd2_rn(make_float2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), make_float2(b[i].z, b[i].w));
     if (valid) sts64(at + static_cast<unsigned>(i) * pitch, pack_act(v0.x, v0.y, act), pack_act(v1.x, v1.y, act));
   }
 }
 
-template <int STRIDE>
+// Stride-1 stencil of one thread over a whole plane column of compile-time height, as straight-line code: `h` is
+// the shared-memory address of the thread's column in padded row 0 of its plane (row pitch WP pixel-slices), `a2` the
+// address of its channels in A2 for output row 0.  Padded row iy is tap row 0 of output row iy, row 1 of output row
+// iy - 1 and row 2 of iy - 2, so three accumulators rotate; with the trip count and the pitches known at compile time
+// the rotation costs no register moves and every address is an immediate offset.
+template <int ROWS, int WP>
+__device__ __forceinline__ void stencil_column(unsigned h, unsigned a2, const float2 (&wlo)[9], const float2 (&whi)[9], const Tap& bias,
+                                               int act) {
+  constexpr int WO = WP - 2;
+  Tap acc[3] = {bias, bias, bias};
+#pragma unroll
+  for (int iy = 0; iy < ROWS + 2; ++iy) {
+    const unsigned at = h + static_cast<unsigned>(iy * WP) * 8u;
+    const Tap t0 = tap_of(lds64(at)), t1 = tap_of(lds64(at + 8u)), t2 = tap_of(lds64(at + 16u));
+    Tap& done = acc[(iy + 1) % 3];  // output row iy - 2
+    Tap& mid = acc[(iy + 2) % 3];   // output row iy - 1
+    Tap& fresh = acc[iy % 3];       // output row iy
+    if (iy >= 2) {
+      done.lo = __ffma2_rn(t0.lo, wlo[6], done.lo);
+      done.hi = __ffma2_rn(t0.hi, whi[6], done.hi);
+      done.lo = __ffma2_rn(t1.lo, wlo[7], done.lo);
+      done.hi = __ffma2_rn(t1.hi, whi[7], done.hi);
+      done.lo = __ffma2_rn(t2.lo, wlo[8], done.lo);
+      done.hi = __ffma2_rn(t2.hi, whi[8], done.hi);
+      sts64(a2 + static_cast<unsigned>((iy - 2) * WO) * 16u, pack_act(done.lo.x, done.lo.y, act), pack_act(done.hi.x, done.hi.y, act));
+    }
+    if (iy >= 1 && iy <= ROWS) {
+      mid.lo = __ffma2_rn(t0.lo, wlo[3], mid.lo);
+      mid.hi = __ffma2_rn(t0.hi, whi[3], mid.hi);
+      mid.lo = __ffma2_rn(t1.lo, wlo[4], mid.lo);
+      mid.hi = __ffma2_rn(t1.hi, whi[4], mid.hi);
+      mid.lo = __ffma2_rn(t2.lo, wlo[5], mid.lo);
+      mid.hi = __ffma2_rn(t2.hi, whi[5], mid.hi);
+    }
+    if (iy < ROWS) {
+      fresh.lo = __ffma2_rn(t0.lo, wlo[0], bias.lo);
+      fresh.hi = __ffma2_rn(t0.hi, whi[0], bias.hi);
+      fresh.lo = __ffma2_rn(t1.lo, wlo[1], fresh.lo);
+      fresh.hi = __ffma2_rn(t1.hi, whi[1], fresh.hi);
+      fresh.lo = __ffma2_rn(t2.lo, wlo[2], fresh.lo);
+      fresh.hi = __ffma2_rn(t2.hi, whi[2], fresh.hi);
+    }
+  }
+}
+
+// STRIDE: of the depthwise convolution; PLANE: 14 or 7 = the hidden planes are 14x14 / 7x7 and a thread walks a whole
+// column (straight-line stencil); 0 = any supported plane (loops)
+template <int STRIDE, int PLANE>
 __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const IrParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   Header* hdr = reinterpret_cast<Header*>(smem);
@@ -166,21 +216,21 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
   volatile unsigned* abort_flag = &hdr->abort_flag;
   const unsigned x0 = smem_u32(smem + kHeader);
   const unsigned a20 = x0 + p.x_bytes;
-  const unsigned h0 = a20 + p.a2_bytes;           // two hidden tiles of h_bytes each
+  const unsigned h0 = a20 + 2u * p.a2_bytes;      // two A2 buffers, then two hidden tiles of h_bytes each: one per team
   const unsigned st0 = h0 + 2u * p.h_bytes;
   const unsigned d1_cols = static_cast<unsigned>(p.mt_in) * kNh;  // one D1 buffer
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < p.stages; ++i) {
       mbar_init(smem_u32(&hdr->w_full[i]), 1);
-      mbar_init(smem_u32(&hdr->w_empty[i]), 1 + kComputeWarps);
+      mbar_init(smem_u32(&hdr->w_empty[i]), 1 + kTeamWarps);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&hdr->d1_full[i]), 1);
-      mbar_init(smem_u32(&hdr->d1_empty[i]), kComputeWarps);
+      mbar_init(smem_u32(&hdr->d1_empty[i]), kTeamWarps);
+      mbar_init(smem_u32(&hdr->a2_full[i]), 1);
+      mbar_init(smem_u32(&hdr->a2_empty[i]), 1);
     }
-    mbar_init(smem_u32(&hdr->a2_full), 1);
-    mbar_init(smem_u32(&hdr->a2_empty), 1);
     mbar_init(smem_u32(&hdr->d2_full), 1);
     mbar_init(smem_u32(&hdr->d2_empty), kComputeWarps);
     mbar_init(smem_u32(&hdr->x_full), 1);
@@ -235,13 +285,15 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
       const unsigned we_lbo = kNh * 16u, wp_lbo = static_cast<unsigned>(p.cout_pad) * 16u;
       const int k_steps1 = p.s_in / 4;  // 16 input channels per MMA
       unsigned g = 0, ul = 0;
+      unsigned n_exp[2] = {0u, 0u}, n_prj[2] = {0u, 0u};  // expansions issued into D1[k], projections issued from A2[k]
       bool ok = true;
-      // expansion of chunk c of the current unit (global chunk number gc) into D1[gc & 1]
-      auto expand = [&](unsigned gc) -> bool {
-        const unsigned stage = gc % p.stages, buf = gc & 1u;
+      // expansion of chunk c of the current unit (its weights are chunk number gc of the copy warp's sequence) into D1[c & 1]
+      auto expand = [&](unsigned gc, int c) -> bool {
+        const unsigned stage = gc % p.stages, buf = static_cast<unsigned>(c) & 1u;
         if (!mbar_wait_parked(smem_u32(&hdr->w_full[stage]), (gc / p.stages) & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma) ||
-            !mbar_wait_parked(smem_u32(&hdr->d1_empty[buf]), ((gc >> 1) & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma))
+            !mbar_wait_parked(smem_u32(&hdr->d1_empty[buf]), (n_exp[buf] & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma))
           return false;
+        ++n_exp[buf];
         tc_fence_after();
         const unsigned we = st0 + stage * p.stage_bytes;
         for (int t = 0; t < p.mt_in; ++t) {
@@ -262,66 +314,76 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
       for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++ul) {
         if (!mbar_wait_parked(smem_u32(&hdr->x_full), ul & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma)) break;
         tc_fence_after();
-        // the expansions run two chunks ahead of the projections: their accumulators are drained one chunk early
-        ok = expand(g);
-        if (ok && p.n_chunks > 1) ok = expand(g + 1);
-        if (ok && ul == 0) IR_EV(6);
+        // one expansion per team is in flight ahead of the projections
+        ok = expand(g, 0);
+        if (ok && p.n_chunks > 1) ok = expand(g + 1, 1);
         for (int c = 0; c < p.n_chunks && ok; ++c) {
-          const unsigned gp = g + c, stage = gp % p.stages;
+          const unsigned gp = g + c, stage = gp % p.stages, k = static_cast<unsigned>(c) & 1u;
           // with three stages the weights of chunk c + 2 arrive while chunk c is being worked on; with two, its stage
           // is the one projection(c) frees, so that expansion can only follow the projection
           const bool early = p.stages >= 3 && c + 2 < p.n_chunks;
           if (early) {
-            ok = expand(gp + 2);
+            ok = expand(gp + 2, c + 2);
             if (!ok) break;
-            if (ul == 0) IR_EV(8 * (c + 2) + 6);
           }
           if (c == 0 && !mbar_wait_parked(smem_u32(&hdr->d2_empty), (ul & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma)) {
             ok = false;
             break;
           }
-          if (!mbar_wait_parked(smem_u32(&hdr->a2_full), gp & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma)) {
+          if (!mbar_wait_parked(smem_u32(&hdr->a2_full[k]), n_prj[k] & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrMma)) {
             ok = false;
             break;
           }
+          ++n_prj[k];
           tc_fence_after();
           const unsigned wp = st0 + stage * p.stage_bytes + p.we_bytes;
+          const unsigned a2 = a20 + k * p.a2_bytes;
           for (int t = 0; t < p.mt_out; ++t)
             for (int h = 0; h < p.n_split; ++h) {
               const unsigned d = tmem_base + p.d2_col0 + static_cast<unsigned>(t * p.cout_pad + h * p.n_each);
-              unsigned long long ad = smem_desc(a20 + static_cast<unsigned>(t) * 2048u, p.a2_pitch, 128);
+              unsigned long long ad = smem_desc(a2 + static_cast<unsigned>(t) * 2048u, p.a2_pitch, 128);
               unsigned long long bd = smem_desc(wp + static_cast<unsigned>(h * p.n_each) * 16u, wp_lbo, 128);
               const unsigned long long ad_step = static_cast<unsigned long long>((2u * p.a2_pitch) >> 4);
               const unsigned long long bd_step = static_cast<unsigned long long>((2u * wp_lbo) >> 4);
+#pragma unroll
               for (int ks = 0; ks < kNh / 16; ++ks) {
                 umma_f16(d, ad, bd, idesc2, (c > 0 || ks > 0) ? 1u : 0u);
                 ad += ad_step;
                 bd += bd_step;
               }
             }
-          umma_commit(smem_u32(&hdr->a2_empty));
+          umma_commit(smem_u32(&hdr->a2_empty[k]));
           umma_commit(smem_u32(&hdr->w_empty[stage]));
           if (c == p.n_chunks - 1) umma_commit(smem_u32(&hdr->d2_full));
           if (ul == 0) IR_EV(8 * c + 7);
-          if (!early && p.stages < 3 && c + 2 < p.n_chunks) ok = expand(gp + 2);
+          if (!early && p.stages < 3 && c + 2 < p.n_chunks) ok = expand(gp + 2, c + 2);
         }
         g += p.n_chunks;
       }
     }
   } else {
     // ------------------------------------------------------------ compute warps
+    // Two teams of eight warps take alternate chunks of a unit (team = chunk parity), each with its own expansion
+    // accumulator, hidden tile and A2 buffer: while one team waits for tensor memory or a barrier, the other one's
+    // stencil keeps the FMA pipe busy.  Warps 0-3 and 8-11 of the sixteen form team 0, so each team has two warps on
+    // every TMEM lane quarter (and on every scheduler).
     const int cw = warp - 2, ctid = threadIdx.x - 64;
-    const int quarter = warp & 3, qsub = cw >> 2;  // TMEM lane quarter of this warp; its index among the four warps sharing it
+    const int team = (cw >> 2) & 1;
+    const int ttid = ((cw & 3) | ((cw >> 3) << 2)) * 32 + lane;  // 0 .. 255 within the team
+    const int quarter = warp & 3, qsub = cw >> 3;                // TMEM lane quarter; index among the team's two warps on it
+    const int qall = cw >> 2;                                    // index among all four warps on the quarter (epilogue)
     const unsigned lane_bits = static_cast<unsigned>(quarter * 32) << 16;
     const int rows_in = p.n_img * p.r_in, rows_out = p.n_img * p.r_out;
+    const unsigned hb = h0 + static_cast<unsigned>(team) * p.h_bytes;    // this team's hidden tile
+    const unsigned a2b = a20 + static_cast<unsigned>(team) * p.a2_bytes; // ... and A2 buffer
 
-    // copies of a unit's X: thread i takes (slice, row) pairs i, i + 512, ...; consecutive threads take consecutive
-    // pixels of one slice (coalesced 8-byte reads); rows of images beyond the batch are left as they are (their
-    // results are never stored)
-    auto issue_x = [&](int u) {
+    // copies of a unit's X by `nthr` threads (index `tid`): thread i takes (slice, row) pairs i, i + nthr, ...; consecutive
+    // threads take consecutive pixels of one slice (coalesced 8-byte reads); rows of images beyond the batch are left as
+    // they are (their results are never stored)
+    auto issue_x = [&](int u, int tid, int nthr) {
       const int b0 = u * p.n_img;
       const int total = p.s_in * rows_in;
-      for (int i = ctid; i < total; i += kComputeThreads) {
+      for (int i = tid; i < total; i += nthr) {
         const int s = i / rows_in, r = i - s * rows_in;
         const int img = r / p.r_in, q = r - img * p.r_in;
         if (b0 + img >= p.B) continue;
@@ -347,77 +409,66 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
     }
     const unsigned slice_pitch = static_cast<unsigned>(p.n_img) * p.plane_words * 8u;  // planes of one slice: one per image
 
-    // this thread's place in the stencil: (band, plane = slice of the chunk x image, output column)
+    // this thread's place in its team's stencil: (band, plane = slice of the chunk x image, output column)
     const int planes = (kNh / 4) * p.n_img;
     const int per_band = planes * p.Wo;
-    const int band = ctid / per_band;
+    const int band = ttid / per_band;
     const bool st_active = band < p.n_bands;
-    const int st_rem = ctid - band * per_band;
+    const int st_rem = ttid - band * per_band;
     const int st_plane = st_rem / p.Wo, st_ox = st_rem - st_plane * p.Wo;
     const int st_slice = st_plane / p.n_img, st_img = st_plane - st_slice * p.n_img;
     const int st_r0 = band * p.band_rows, st_r1 = min(p.Ho, st_r0 + p.band_rows);
-    const unsigned st_hoff = static_cast<unsigned>(st_plane) * p.plane_words * 8u;
-    const unsigned st_a2 = a20 + static_cast<unsigned>(st_slice >> 1) * p.a2_pitch + static_cast<unsigned>(st_img * p.r_out) * 16u +
+    const unsigned st_h = hb + static_cast<unsigned>(st_plane) * p.plane_words * 8u;
+    const unsigned st_a2 = a2b + static_cast<unsigned>(st_slice >> 1) * p.a2_pitch + static_cast<unsigned>(st_img * p.r_out) * 16u +
                            static_cast<unsigned>(st_slice & 1) * 8u;
 
     bool ok = true;
-    // ---- drain D1 of global chunk gc: 16 hidden channels of one pixel per tcgen05.ld; bias, activation, fp16 -> hidden tile gc & 1
-    auto drain = [&](unsigned gc, int ev) {
-      const unsigned stage = gc % p.stages, buf = gc & 1u;
-      const unsigned eb0 = st0 + stage * p.stage_bytes + p.we_bytes + p.wp_bytes + 10u * kNh * 4u;  // expansion bias of the chunk
-      const unsigned hb = h0 + buf * p.h_bytes;
-      if (ev >= 0 && ctid == 0 && ev / 8 < 6) IR_EV(48 + 2 * (ev / 8));
-      ok = ok && mbar_wait_warp(smem_u32(&hdr->w_full[stage]), (gc / p.stages) & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
-      if (ev >= 0 && ctid == 0 && ev / 8 < 6) IR_EV(49 + 2 * (ev / 8));
-      ok = ok && mbar_wait_warp(smem_u32(&hdr->d1_full[buf]), (gc >> 1) & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
-      if (ev >= 0 && ctid == 0) IR_EV(ev);
-      if (ok) {
-        tc_fence_after();
-        // a warp takes 16 columns (j = its index among the four warps of its lane quarter) of each tile; both tiles'
-        // loads are issued before either is used
-        const int j = qsub;
-        unsigned r0[16], r1[16];
-        tmem_ld16(tmem_base + lane_bits + buf * d1_cols + static_cast<unsigned>(j * 16), r0);
-        if (p.mt_in > 1) tmem_ld16(tmem_base + lane_bits + buf * d1_cols + static_cast<unsigned>(kNh + j * 16), r1);
-        const unsigned dst = hb + static_cast<unsigned>(j * 4) * slice_pitch;
-        tmem_ld_wait16(r0);
-        store_hidden(r0, eb0 + static_cast<unsigned>(j) * 64u, dst + dr_off[0], slice_pitch, dr_valid[0], p.act1);
-        if (p.mt_in > 1) {
-          tmem_ld_wait16(r1);
-          store_hidden(r1, eb0 + static_cast<unsigned>(j) * 64u, dst + dr_off[1], slice_pitch, dr_valid[1], p.act1);
-        }
-        tc_fence_before();
-      }
-      __syncwarp();
-      if (lane == 0 && ok) mbar_arrive(smem_u32(&hdr->d1_empty[buf]));
-    };
-
     if (ctid == 0) IR_EV(60);
     pdl_wait();  // activations are read and written only below
     if (ctid == 0) IR_EV(61);
-    if (static_cast<int>(blockIdx.x) < p.units) issue_x(blockIdx.x);
+    if (static_cast<int>(blockIdx.x) < p.units) issue_x(blockIdx.x, ctid, kComputeThreads);
     cp_async_wait_all();
     fence_async_proxy();
     bar_compute();
     if (ctid == 0 && static_cast<int>(blockIdx.x) < p.units) mbar_arrive(smem_u32(&hdr->x_full));
     if (ctid == 0) IR_EV(62);
 
-    unsigned g = 0, ul = 0;
+    unsigned g = 0, ul = 0, uses = 0;  // uses: chunks this team has worked on (the phase of its barriers)
     for (int u = blockIdx.x; u < p.units; u += gridDim.x, ++ul) {
       const int b0 = u * p.n_img;
       const bool more = u + static_cast<int>(gridDim.x) < p.units;
-      drain(g, -1);
-      bar_compute();  // hidden tile of chunk 0 complete
-      for (int c = 0; c < p.n_chunks; ++c) {
+      for (int c = team; c < p.n_chunks; c += 2, ++uses) {
         const unsigned gc = g + c, stage = gc % p.stages;
-        const unsigned dw0 = st0 + stage * p.stage_bytes + p.we_bytes + p.wp_bytes;  // depthwise taps [9][64], depthwise bias [64]
-        if (ctid == 0 && ul == 0) IR_EV(8 * c + 0);
-        // the next chunk's expansion has long finished: drain it into the other hidden tile while the projection of the
-        // previous chunk, which still reads A2, completes
-        if (c + 1 < p.n_chunks) drain(gc + 1, ul == 0 ? 8 * c + 2 : -1);
-        // the last expansion of this unit is complete (its accumulator has been read): X may be overwritten
-        else if (more && ok) issue_x(u + gridDim.x);
-        if (ctid == 0 && ul == 0) IR_EV(8 * c + 1);
+        const unsigned dw0 = st0 + stage * p.stage_bytes + p.we_bytes + p.wp_bytes;  // depthwise taps [9][64], depthwise bias [64], expansion bias [64]
+        if (ttid == 0 && ul == 0) IR_EV(8 * c + 0);
+        // ---- drain this chunk's expansion: 16 hidden channels of one pixel per tcgen05.ld; bias, activation, fp16 -> hidden tile
+        ok = ok && mbar_wait_warp(smem_u32(&hdr->w_full[stage]), (gc / p.stages) & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
+        ok = ok && mbar_wait_warp(smem_u32(&hdr->d1_full[team]), uses & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
+        if (ttid == 0 && ul == 0) IR_EV(8 * c + 2);
+        if (ok) {
+          tc_fence_after();
+          // a team warp takes two of the four 16-column groups of its lane quarter, in both 128-row tiles; a group's 16
+          // biases are requested together with the accumulator columns
+          for (int e = 0; e < 2 * p.mt_in; ++e) {
+            const int t = e >> 1, j = qsub * 2 + (e & 1);
+            unsigned r[16];
+            tmem_ld16(tmem_base + lane_bits + static_cast<unsigned>(team) * d1_cols + static_cast<unsigned>(t * kNh + j * 16), r);
+            float4 b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) b[i] = lds128f(dw0 + 10u * kNh * 4u + static_cast<unsigned>(j * 4 + i) * 16u);
+            tmem_ld_wait16(r);
+            store_hidden(r, b, hb + static_cast<unsigned>(j * 4) * slice_pitch + (t ? dr_off[1] : dr_off[0]), slice_pitch,
+                         t ? dr_valid[1] : dr_valid[0], p.act1);
+          }
+          tc_fence_before();
+        }
+        __syncwarp();
+        if (lane == 0 && ok) mbar_arrive(smem_u32(&hdr->d1_empty[team]));
+        // the unit's last expansion is complete (its accumulator has just been read, and MMAs finish in order): X may
+        // be overwritten with the next unit's
+        if (c == p.n_chunks - 1 && more && ok) issue_x(u + gridDim.x, ttid, kTeamThreads);
+        if (ttid == 0 && ul == 0) IR_EV(8 * c + 1);
+        bar_team(team);  // the hidden tile is complete
 
         // ---- this thread's depthwise weights (its slice of the chunk) into registers, then the stage is released
         float2 wlo[9], whi[9];
@@ -435,16 +486,19 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
         }
         __syncwarp();
         if (lane == 0 && ok) mbar_arrive(smem_u32(&hdr->w_empty[stage]));
-        ok = ok && mbar_wait_warp(smem_u32(&hdr->a2_empty), (gc & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
-        if (ctid == 0 && ul == 0) IR_EV(8 * c + 3);
+        ok = ok && mbar_wait_warp(smem_u32(&hdr->a2_empty[team]), (uses & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
+        if (ttid == 0 && ul == 0) IR_EV(8 * c + 3);
 
         // ---- depthwise 3x3 from the hidden tile -> A operand of the projection
         if (ok && st_active) {
-          const unsigned st_h = h0 + (gc & 1u) * p.h_bytes + st_hoff;
           auto emit = [&](const Tap& a, int oy) {
             sts64(st_a2 + static_cast<unsigned>(oy * p.Wo + st_ox) * 16u, pack_act(a.lo.x, a.lo.y, p.act2), pack_act(a.hi.x, a.hi.y, p.act2));
           };
-          if (STRIDE == 1) {
+          if (STRIDE == 1 && PLANE == 14) {
+            stencil_column<14, 16>(st_h + static_cast<unsigned>(st_ox) * 8u, st_a2 + static_cast<unsigned>(st_ox) * 16u, wlo, whi, bias, p.act2);
+          } else if (STRIDE == 1 && PLANE == 7) {
+            stencil_column<7, 9>(st_h + static_cast<unsigned>(st_ox) * 8u, st_a2 + static_cast<unsigned>(st_ox) * 16u, wlo, whi, bias, p.act2);
+          } else if (STRIDE == 1) {
             // padded row iy (image row iy - 1) is tap row 0 of output row iy, row 1 of iy - 1, row 2 of iy - 2
             Tap a0 = bias, a1 = bias, a2 = bias;
             auto step = [&](Tap& done, Tap& mid, Tap& fresh, int iy) {
@@ -497,37 +551,37 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
             }
           }
         }
-        if (ctid == 0 && ul == 0) IR_EV(8 * c + 4);
+        if (ttid == 0 && ul == 0) IR_EV(8 * c + 4);
         fence_async_proxy();  // the A operand was written with ordinary stores; the MMA reads it through the async proxy
-        bar_compute();        // A2 and the next hidden tile are complete; nobody reads this chunk's hidden tile any more
-        if (ctid == 0 && ok) mbar_arrive(smem_u32(&hdr->a2_full));
-        if (ctid == 0 && ul == 0) IR_EV(8 * c + 5);
+        bar_team(team);       // A2 is complete; nobody in the team reads this hidden tile any more
+        if (ttid == 0 && ok) mbar_arrive(smem_u32(&hdr->a2_full[team]));
+        if (ttid == 0 && ul == 0) IR_EV(8 * c + 5);
       }
       g += p.n_chunks;
 
-      // ---- the next unit's X has been on its way since the last chunk began: publish it, then drain this unit's D2
-      if (more) {
-        cp_async_wait_all();
-        fence_async_proxy();
-        bar_compute();
-        if (ctid == 0 && ok) mbar_arrive(smem_u32(&hdr->x_full));
-      }
+      // ---- unit end: the teams meet; the next unit's X (on its way since the last chunk's drain) is published, then
+      // all sixteen warps drain D2
+      cp_async_wait_all();
+      fence_async_proxy();
+      bar_compute();
+      if (more && ctid == 0 && ok) mbar_arrive(smem_u32(&hdr->x_full));
       // the residual does not depend on the accumulator: the first item's is fetched before waiting for the last
       // projection, each further item's while the one before it is processed
       const int groups = p.cout_pad >> 4, n_items = p.mt_out * groups;
-      auto item_px = [&](int e, int* t, int* j, size_t* px, bool* valid) {
+      auto item_px = [&](int e, int* t, int* j, size_t* px, bool* valid, bool* last_px) {
         *t = e / groups;
         *j = e - *t * groups;
         const int row = *t * 128 + quarter * 32 + lane;
         const int img = row / p.r_out, q = row - img * p.r_out;
         *valid = e < n_items && row < rows_out && b0 + img < p.B;
         *px = static_cast<size_t>(b0 + img) * p.Pout + q;
+        *last_px = q == p.r_out - 1;
       };
       auto fetch_res = [&](uint2* dstq, int e) {
         int t, j;
         size_t px;
-        bool valid;
-        item_px(e, &t, &j, &px, &valid);
+        bool valid, last_px;
+        item_px(e, &t, &j, &px, &valid, &last_px);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int so = j * 4 + i;
@@ -537,15 +591,15 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
         }
       };
       uint2 res_cur[4], res_nxt[4];
-      fetch_res(res_cur, qsub);
+      fetch_res(res_cur, qall);
       ok = ok && mbar_wait_warp(smem_u32(&hdr->d2_full), ul & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
       if (ok) {
         tc_fence_after();
-        for (int e = qsub; e < n_items; e += 4) {
+        for (int e = qall; e < n_items; e += 4) {
           int t, j;
           size_t px;
-          bool valid;
-          item_px(e, &t, &j, &px, &valid);
+          bool valid, last_px;
+          item_px(e, &t, &j, &px, &valid, &last_px);
           unsigned r[16];
           tmem_ld16(tmem_base + lane_bits + p.d2_col0 + static_cast<unsigned>(t * p.cout_pad + j * 16), r);
           fetch_res(res_nxt, e + 4);
@@ -571,7 +625,7 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
             o.y = pack_f16x2<false>(act1f(v2, p.act4), act1f(v3, p.act4));
             *reinterpret_cast<uint2*>(p.out + off) = o;
             // an odd plane is stored with one extra pixel, which readers expect to be finite: zero it
-            if (p.Pout > p.r_out && (px + 1) % p.Pout == static_cast<size_t>(p.r_out)) *reinterpret_cast<uint2*>(p.out + off + 4) = make_uint2(0u, 0u);
+            if (p.Pout > p.r_out && last_px) *reinterpret_cast<uint2*>(p.out + off + 4) = make_uint2(0u, 0u);
           }
 #pragma unroll
           for (int i = 0; i < 4; ++i) res_cur[i] = res_nxt[i];
@@ -625,7 +679,7 @@ Shape shape_of(int B, int H, int W, int Ho, int Wo, int stride, int cin, int chi
   s.plane_words = (H + 2) * s.Wp;
   while (s.plane_words % 16 != W % 16) ++s.plane_words;  // consecutive planes start W words apart (mod 16): no bank conflicts
   const int planes = (kNh / 4) * s.n_img;
-  int bands = kComputeThreads / (planes * Wo);
+  int bands = kTeamThreads / (planes * Wo);
   if (bands < 1) return s;
   if (bands > Ho) bands = Ho;
   s.band_rows = (Ho + bands - 1) / bands;
@@ -642,7 +696,7 @@ Shape shape_of(int B, int H, int W, int Ho, int Wo, int stride, int cin, int chi
   s.a2_bytes = (static_cast<unsigned>(kNh / 8) * s.a2_pitch + 127u) / 128u * 128u;
   s.h_bytes = (static_cast<unsigned>(planes) * s.plane_words * 8u + 127u) / 128u * 128u;
   // (the tail reads of A2's last K group land in the hidden tiles, 2 x h_bytes >= 2 KB, those of X in A2 or behind)
-  const long long fixed = kHeader + static_cast<long long>(s.x_bytes) + s.a2_bytes + 2ll * s.h_bytes;
+  const long long fixed = kHeader + static_cast<long long>(s.x_bytes) + 2ll * s.a2_bytes + 2ll * s.h_bytes;
   long long stages = (kSmemMax - fixed) / s.stage_bytes;
   if (stages < 2) return s;
   s.stages = stages > kMaxStages ? kMaxStages : static_cast<int>(stages);
@@ -772,8 +826,10 @@ int launch_inverted_residual(const LaunchRec& r, const Ptrs& p, void* stream) {
   static bool attr_done_dev[kMaxDevices] = {};
   bool& attr_done = attr_done_dev[current_device_slot()];
   if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(inverted_residual_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(inverted_residual_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+    cudaError_t e = cudaFuncSetAttribute(inverted_residual_kernel<1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(inverted_residual_kernel<1, 14>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(inverted_residual_kernel<1, 7>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(inverted_residual_kernel<2, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
     if (e != cudaSuccess) return static_cast<int>(e);
     attr_done = true;
   }
@@ -783,8 +839,11 @@ int launch_inverted_residual(const LaunchRec& r, const Ptrs& p, void* stream) {
   size_t smem = s.smem;
   if (smem < 120 * 1024) smem = 120 * 1024;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (r.sh == 1) launch_pdl(inverted_residual_kernel<1>, grid, kThreads, smem, st, k);
-  else launch_pdl(inverted_residual_kernel<2>, grid, kThreads, smem, st, k);
+  const bool whole_column = r.sh == 1 && s.n_bands == 1 && r.H == r.W;  // a thread walks a whole column of its plane
+  if (whole_column && r.H == 14) launch_pdl(inverted_residual_kernel<1, 14>, grid, kThreads, smem, st, k);
+  else if (whole_column && r.H == 7) launch_pdl(inverted_residual_kernel<1, 7>, grid, kThreads, smem, st, k);
+  else if (r.sh == 1) launch_pdl(inverted_residual_kernel<1, 0>, grid, kThreads, smem, st, k);
+  else launch_pdl(inverted_residual_kernel<2, 0>, grid, kThreads, smem, st, k);
   return static_cast<int>(cudaGetLastError());
 }
 
