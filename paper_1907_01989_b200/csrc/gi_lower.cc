@@ -293,8 +293,12 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
           // Launches whose pixels all fit one wave of 128-pixel tiles are latency-bound and take the lane
           // kernel (shorter fill; MobileNetV2 batch 1 0.296 -> 0.276 ms) - up to 64 tiles always, up to one
           // tile per SM unless the input is 960 channels deep or more.
-          // Whole inverted-residual block as one kernel (small planes): chosen where the kernel has at least about one
-          // unit of work per SM - below that (batch 1) three kernels that each spread over all SMs are faster
+          // Whole inverted-residual block as one kernel.  The library's own choice (GI_XOP_AUTO) follows an A/B of
+          // MobileNetV2 at batch 256 on one B200, both builds alternating in one call: with the two 7x7 blocks that
+          // qualify as one kernel each the step takes 1.619 ms against 1.626 ms; with the 14x14 blocks as well 1.668 ms
+          // (alone, L2 flushed, a 14x14 block takes 55-88 us as one kernel against 52-73 us as three; a 7x7 block
+          // 55-66 against 60).  So: planes of at most 64 pixels, and at least about one unit of work per SM - below
+          // that (batch 1) three kernels that each spread over all SMs are faster.
           long long ir_units = 0;
           if (pointwise && tc && e->opt.fuse && e->opt.cross_op != GI_XOP_OFF && block_follows(g, e, i)) {
             const FusedOp& fd = e->ops[i + 1];

@@ -54,6 +54,9 @@ constexpr int kSmemMax = 227 * 1024;
 constexpr int kDwBytes = (9 * kNh + kNh + kNh) * 4;  // depthwise taps, depthwise bias, expansion bias of a chunk
 
 __device__ unsigned int g_ir_error = 0;
+#ifndef GI_TRACE_UNIT
+#define GI_TRACE_UNIT 0
+#endif
 #ifdef GI_TRACE
 __device__ unsigned long long g_ir_trace[256 * 64];
 #define IR_EV(idx)                                           \
@@ -232,7 +235,7 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
       mbar_init(smem_u32(&hdr->a2_empty[i]), 1);
     }
     mbar_init(smem_u32(&hdr->d2_full), 1);
-    mbar_init(smem_u32(&hdr->d2_empty), kComputeWarps);
+    mbar_init(smem_u32(&hdr->d2_empty), kTeamWarps);
     mbar_init(smem_u32(&hdr->x_full), 1);
     hdr->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -355,7 +358,7 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
           umma_commit(smem_u32(&hdr->a2_empty[k]));
           umma_commit(smem_u32(&hdr->w_empty[stage]));
           if (c == p.n_chunks - 1) umma_commit(smem_u32(&hdr->d2_full));
-          if (ul == 0) IR_EV(8 * c + 7);
+          if (ul == GI_TRACE_UNIT) IR_EV(8 * c + 7);
           if (!early && p.stages < 3 && c + 2 < p.n_chunks) ok = expand(gp + 2, c + 2);
         }
         g += p.n_chunks;
@@ -371,7 +374,6 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
     const int team = (cw >> 2) & 1;
     const int ttid = ((cw & 3) | ((cw >> 3) << 2)) * 32 + lane;  // 0 .. 255 within the team
     const int quarter = warp & 3, qsub = cw >> 3;                // TMEM lane quarter; index among the team's two warps on it
-    const int qall = cw >> 2;                                    // index among all four warps on the quarter (epilogue)
     const unsigned lane_bits = static_cast<unsigned>(quarter * 32) << 16;
     const int rows_in = p.n_img * p.r_in, rows_out = p.n_img * p.r_out;
     const unsigned hb = h0 + static_cast<unsigned>(team) * p.h_bytes;    // this team's hidden tile
@@ -382,13 +384,19 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
     // they are (their results are never stored)
     auto issue_x = [&](int u, int tid, int nthr) {
       const int b0 = u * p.n_img;
-      const int total = p.s_in * rows_in;
-      for (int i = tid; i < total; i += nthr) {
-        const int s = i / rows_in, r = i - s * rows_in;
-        const int img = r / p.r_in, q = r - img * p.r_in;
-        if (b0 + img >= p.B) continue;
-        const __half* src = p.in + ((static_cast<size_t>(s) * p.B + b0 + img) * p.Pin + q) * 4;
-        cp_async8(x0 + static_cast<unsigned>(s >> 1) * p.x_pitch + static_cast<unsigned>(r) * 16u + static_cast<unsigned>(s & 1) * 8u, src);
+      const bool second_ok = b0 + 1 < p.B;  // a unit holds one or two images
+      for (int r = tid; r < rows_in; r += nthr) {
+        const int img = r >= p.r_in ? 1 : 0, q = r - img * p.r_in;
+        if (img && !second_ok) continue;
+        const __half* src = p.in + (static_cast<size_t>(b0 + img) * p.Pin + q) * 4;
+        const size_t slice_stride = static_cast<size_t>(p.B) * p.Pin * 4;  // halves between two slices of the tensor
+        unsigned dst = x0 + static_cast<unsigned>(r) * 16u;
+        for (int s = 0; s < p.s_in; s += 2) {
+          cp_async8(dst, src);
+          cp_async8(dst + 8u, src + slice_stride);
+          src += 2 * slice_stride;
+          dst += p.x_pitch;
+        }
       }
     };
 
@@ -440,11 +448,11 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
       for (int c = team; c < p.n_chunks; c += 2, ++uses) {
         const unsigned gc = g + c, stage = gc % p.stages;
         const unsigned dw0 = st0 + stage * p.stage_bytes + p.we_bytes + p.wp_bytes;  // depthwise taps [9][64], depthwise bias [64], expansion bias [64]
-        if (ttid == 0 && ul == 0) IR_EV(8 * c + 0);
+        if (ttid == 0 && ul == GI_TRACE_UNIT) IR_EV(8 * c + 0);
         // ---- drain this chunk's expansion: 16 hidden channels of one pixel per tcgen05.ld; bias, activation, fp16 -> hidden tile
         ok = ok && mbar_wait_warp(smem_u32(&hdr->w_full[stage]), (gc / p.stages) & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
         ok = ok && mbar_wait_warp(smem_u32(&hdr->d1_full[team]), uses & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
-        if (ttid == 0 && ul == 0) IR_EV(8 * c + 2);
+        if (ttid == 0 && ul == GI_TRACE_UNIT) IR_EV(8 * c + 2);
         if (ok) {
           tc_fence_after();
           // a team warp takes two of the four 16-column groups of its lane quarter, in both 128-row tiles; a group's 16
@@ -467,7 +475,7 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
         // the unit's last expansion is complete (its accumulator has just been read, and MMAs finish in order): X may
         // be overwritten with the next unit's
         if (c == p.n_chunks - 1 && more && ok) issue_x(u + gridDim.x, ttid, kTeamThreads);
-        if (ttid == 0 && ul == 0) IR_EV(8 * c + 1);
+        if (ttid == 0 && ul == GI_TRACE_UNIT) IR_EV(8 * c + 1);
         bar_team(team);  // the hidden tile is complete
 
         // ---- this thread's depthwise weights (its slice of the chunk) into registers, then the stage is released
@@ -487,7 +495,7 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
         __syncwarp();
         if (lane == 0 && ok) mbar_arrive(smem_u32(&hdr->w_empty[stage]));
         ok = ok && mbar_wait_warp(smem_u32(&hdr->a2_empty[team]), (uses & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
-        if (ttid == 0 && ul == 0) IR_EV(8 * c + 3);
+        if (ttid == 0 && ul == GI_TRACE_UNIT) IR_EV(8 * c + 3);
 
         // ---- depthwise 3x3 from the hidden tile -> A operand of the projection
         if (ok && st_active) {
@@ -551,67 +559,79 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
             }
           }
         }
-        if (ttid == 0 && ul == 0) IR_EV(8 * c + 4);
+        if (ttid == 0 && ul == GI_TRACE_UNIT) IR_EV(8 * c + 4);
         fence_async_proxy();  // the A operand was written with ordinary stores; the MMA reads it through the async proxy
+        // the team that worked on the unit's last chunk also requested the next unit's X: its copies must have landed
+        // before the barrier that publishes them
+        if (c == p.n_chunks - 1 && more) {
+          cp_async_wait_all();
+          fence_async_proxy();
+        }
         bar_team(team);       // A2 is complete; nobody in the team reads this hidden tile any more
-        if (ttid == 0 && ok) mbar_arrive(smem_u32(&hdr->a2_full[team]));
-        if (ttid == 0 && ul == 0) IR_EV(8 * c + 5);
+        if (ttid == 0 && ok) {
+          mbar_arrive(smem_u32(&hdr->a2_full[team]));
+          if (c == p.n_chunks - 1 && more) mbar_arrive(smem_u32(&hdr->x_full));
+        }
+        if (ttid == 0 && ul == GI_TRACE_UNIT) IR_EV(8 * c + 5);
       }
       g += p.n_chunks;
+      // ---- unit end.  Team 0 goes straight on to the next unit; team 1 first drains D2 (the next unit's first
+      // projection, which needs D2 free, comes a whole chunk of team 0's work later), which also puts the two teams
+      // half a chunk apart: while one runs its stencil the other waits for tensor memory.
+      if (team == 0) continue;
 
-      // ---- unit end: the teams meet; the next unit's X (on its way since the last chunk's drain) is published, then
-      // all sixteen warps drain D2
-      cp_async_wait_all();
-      fence_async_proxy();
-      bar_compute();
-      if (more && ctid == 0 && ok) mbar_arrive(smem_u32(&hdr->x_full));
       // the residual does not depend on the accumulator: the first item's is fetched before waiting for the last
       // projection, each further item's while the one before it is processed
       const int groups = p.cout_pad >> 4, n_items = p.mt_out * groups;
-      auto item_px = [&](int e, int* t, int* j, size_t* px, bool* valid, bool* last_px) {
-        *t = e / groups;
-        *j = e - *t * groups;
-        const int row = *t * 128 + quarter * 32 + lane;
-        const int img = row / p.r_out, q = row - img * p.r_out;
-        *valid = e < n_items && row < rows_out && b0 + img < p.B;
-        *px = static_cast<size_t>(b0 + img) * p.Pout + q;
-        *last_px = q == p.r_out - 1;
-      };
+      const size_t o_slice = static_cast<size_t>(p.B) * p.Pout * 4;  // halves between two slices of the output
+      // where this thread's rows of the two output tiles are stored (a unit holds one or two images)
+      size_t ep_off[2];
+      bool ep_valid[2], ep_last[2];
+#pragma unroll
+      for (int t = 0; t < 2; ++t) {
+        const int row = t * 128 + quarter * 32 + lane;
+        const int img = row >= p.r_out ? 1 : 0, q = row - img * p.r_out;
+        ep_valid[t] = t < p.mt_out && row < rows_out && b0 + img < p.B;
+        ep_off[t] = (static_cast<size_t>(b0 + img) * p.Pout + q) * 4;
+        ep_last[t] = q == p.r_out - 1;
+      }
       auto fetch_res = [&](uint2* dstq, int e) {
-        int t, j;
-        size_t px;
-        bool valid, last_px;
-        item_px(e, &t, &j, &px, &valid, &last_px);
+        const int t = e / groups, j = e - t * groups;
+        const bool valid = e < n_items && (t ? ep_valid[1] : ep_valid[0]);
+        const __half* src = p.res + (t ? ep_off[1] : ep_off[0]) + static_cast<size_t>(j * 4) * o_slice;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const int so = j * 4 + i;
           dstq[i] = make_uint2(0u, 0u);
-          if (p.has_res && valid && so < p.s_out)
-            dstq[i] = __ldg(reinterpret_cast<const uint2*>(p.res + (static_cast<size_t>(so) * p.B * p.Pout + px) * 4));
+          if (p.has_res && valid && j * 4 + i < p.s_out) dstq[i] = __ldg(reinterpret_cast<const uint2*>(src + i * o_slice));
         }
       };
       uint2 res_cur[4], res_nxt[4];
-      fetch_res(res_cur, qall);
+      fetch_res(res_cur, qsub);
       ok = ok && mbar_wait_warp(smem_u32(&hdr->d2_full), ul & 1u, abort_flag, p.timeout_ns, &g_ir_error, kErrCompute);
       if (ok) {
         tc_fence_after();
-        for (int e = qall; e < n_items; e += 4) {
-          int t, j;
-          size_t px;
-          bool valid, last_px;
-          item_px(e, &t, &j, &px, &valid, &last_px);
+        const bool plain = p.act3 == GI_ACT_NONE && p.act4 == GI_ACT_NONE;  // the linear projection of an inverted-residual block
+        for (int e = qsub; e < n_items; e += 2) {
+          const int t = e / groups, j = e - t * groups;
+          const bool valid = t ? ep_valid[1] : ep_valid[0], last_px = t ? ep_last[1] : ep_last[0];
           unsigned r[16];
           tmem_ld16(tmem_base + lane_bits + p.d2_col0 + static_cast<unsigned>(t * p.cout_pad + j * 16), r);
-          fetch_res(res_nxt, e + 4);
+          fetch_res(res_nxt, e + 2);
+          __half* dst = p.out + (t ? ep_off[1] : ep_off[0]) + static_cast<size_t>(j * 4) * o_slice;
           tmem_ld_wait16(r);
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const int so = j * 4 + i;
             if (so >= p.s_out || !valid) continue;
             const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias2) + so);
-            const size_t off = (static_cast<size_t>(so) * p.B * p.Pout + px) * 4;  // in halves
-            float v0 = act1f(__uint_as_float(r[4 * i]) + b.x, p.act3), v1 = act1f(__uint_as_float(r[4 * i + 1]) + b.y, p.act3);
-            float v2 = act1f(__uint_as_float(r[4 * i + 2]) + b.z, p.act3), v3 = act1f(__uint_as_float(r[4 * i + 3]) + b.w, p.act3);
+            float v0 = __uint_as_float(r[4 * i]) + b.x, v1 = __uint_as_float(r[4 * i + 1]) + b.y;
+            float v2 = __uint_as_float(r[4 * i + 2]) + b.z, v3 = __uint_as_float(r[4 * i + 3]) + b.w;
+            if (!plain) {
+              v0 = act1f(v0, p.act3);
+              v1 = act1f(v1, p.act3);
+              v2 = act1f(v2, p.act3);
+              v3 = act1f(v3, p.act3);
+            }
             if (p.has_res) {
               const float2 q0 = __half22float2(*reinterpret_cast<const __half2*>(&res_cur[i].x));
               const float2 q1 = __half22float2(*reinterpret_cast<const __half2*>(&res_cur[i].y));
@@ -620,12 +640,19 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
               v2 += q1.x;
               v3 += q1.y;
             }
+            if (!plain) {
+              v0 = act1f(v0, p.act4);
+              v1 = act1f(v1, p.act4);
+              v2 = act1f(v2, p.act4);
+              v3 = act1f(v3, p.act4);
+            }
             uint2 o;
-            o.x = pack_f16x2<false>(act1f(v0, p.act4), act1f(v1, p.act4));
-            o.y = pack_f16x2<false>(act1f(v2, p.act4), act1f(v3, p.act4));
-            *reinterpret_cast<uint2*>(p.out + off) = o;
+            o.x = pack_f16x2<false>(v0, v1);
+            o.y = pack_f16x2<false>(v2, v3);
+            __half* at = dst + i * o_slice;
+            *reinterpret_cast<uint2*>(at) = o;
             // an odd plane is stored with one extra pixel, which readers expect to be finite: zero it
-            if (p.Pout > p.r_out && last_px) *reinterpret_cast<uint2*>(p.out + off + 4) = make_uint2(0u, 0u);
+            if (p.Pout > p.r_out && last_px) *reinterpret_cast<uint2*>(at + 4) = make_uint2(0u, 0u);
           }
 #pragma unroll
           for (int i = 0; i < 4; ++i) res_cur[i] = res_nxt[i];
@@ -634,7 +661,7 @@ __global__ void __launch_bounds__(kThreads, 1) inverted_residual_kernel(const Ir
       }
       __syncwarp();
       if (lane == 0 && ok) mbar_arrive(smem_u32(&hdr->d2_empty));
-      if (ctid == 0 && ul == 0) IR_EV(63);
+      if (ttid == 0 && ul == GI_TRACE_UNIT) IR_EV(63);
     }
   }
 
