@@ -92,7 +92,9 @@ enum {
   GI_PW_AUTO = 0,      /* tensor-core kernels for fp16 storage, CUDA-core kernel for fp32 storage */
   GI_PW_SIMT = 1,      /* force the plain CUDA-core kernel for every full convolution (validation) */
   GI_PW_TC_PAIR = 2,   /* 1x1: always the pixel-pair tensor-core kernel (operands by TMA) */
-  GI_PW_TC_LANE = 3    /* 1x1: always the lane-per-pixel tensor-core kernel (activations through tensor memory) */
+  GI_PW_TC_LANE = 3,   /* 1x1: always the lane-per-pixel tensor-core kernel (activations through tensor memory) */
+  GI_PW_TC_WIDE = 4    /* 1x1: always the wide-tile tensor-core kernel built for tensor-bound shapes (256 pixels x up to
+                          256 output channels per CTA, both operands streamed) */
 };
 
 /* Cross-operator kernels: a depthwise 3x3 convolution whose only consumer is a 1x1 convolution runs
@@ -188,7 +190,8 @@ enum {
   GI_KERNEL_NONE = 12,                /* no launch: the op ran inside the previous op's kernel */
   GI_KERNEL_CONCAT = 13,
   GI_KERNEL_CONV_TC = 14,             /* k x k convolution, any number of input channels, on the tensor cores */
-  GI_KERNEL_INVERTED_RESIDUAL = 15    /* this op (1x1 expansion) and the next two (depthwise 3x3, 1x1 projection) as one kernel */
+  GI_KERNEL_INVERTED_RESIDUAL = 15,   /* this op (1x1 expansion) and the next two (depthwise 3x3, 1x1 projection) as one kernel */
+  GI_KERNEL_POINTWISE_MM = 16         /* 1x1 convolution, wide tiles for tensor-bound shapes */
 };
 
 /* ---- graph construction (Section 3.1, "Initialization": the sub-graph given to the GPU backend) ---- */

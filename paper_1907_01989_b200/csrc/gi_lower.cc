@@ -118,6 +118,11 @@ static bool pointwise_follows(const gi_graph& g, const gi_exec* e, size_t i) {
          d.pad_r == 0;
 }
 
+// pixels of a 1x1 convolution's input as the kernels count them: batch x stored plane
+static long long m_px_all_for_mm(const gi_exec* e, const TensorDesc* t) {
+  return static_cast<long long>(e->batch) * plane_pixels(t->h, t->w);
+}
+
 static bool is_plain_pointwise(const gi_op_desc& d) {
   return d.kh == 1 && d.kw == 1 && d.stride_h == 1 && d.stride_w == 1 && d.pad_t == 0 && d.pad_l == 0 && d.pad_b == 0 && d.pad_r == 0;
 }
@@ -343,7 +348,21 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
           const bool lane_rule = op.d.cout >= 96 && din->c >= 64 && din->c < 960 && !(din->c <= 96 && op.d.cout >= 4 * din->c);
           const bool lane_auto = one_wave || lane_rule;
           const bool lane_kernel = e->opt.pointwise == GI_PW_TC_LANE || (e->opt.pointwise == GI_PW_AUTO && lane_auto);
-          if (pointwise && tc && lane_kernel && pointwise_ts_supported(din->c, op.d.cout)) {
+          // The wide-tile kernel (256 pixels x up to 256 output channels per CTA) is for the shapes bound by the tensor
+          // pipe: at least 512 input and 512 output channels.  Measured against the library's previous choice at batch
+          // 256 (time wide / time before): 14x14 1280->1280 0.57, 960->960 0.72, 576->576 0.76, 7x7 1024->1024 0.83,
+          // 14x14 512->512 0.96; but 7x7 512->1024 1.07 and 14x14 512->512 at batch 64 1.10, where the 256 x 256 tiles
+          // leave the last wave of CTAs two thirds empty - with 512 input channels it therefore needs well-filled waves
+          // (148 SMs).  Narrower layers lose 10-25 % to it: their tiles are short and its drain is not overlapped.
+          const long long mm_units = ((m_px_all_for_mm(e, din) + 255) / 256) * ((slices(op.d.cout) * 4 + 255) / 256);
+          const long long mm_waves = (mm_units + 147) / 148;
+          const bool mm_auto = din->c >= 512 && op.d.cout >= 512 && mm_units >= 64 &&
+                               (din->c >= 576 || mm_units * 100 >= mm_waves * 148 * 85);
+          const bool wide_kernel = e->opt.pointwise == GI_PW_TC_WIDE || (e->opt.pointwise == GI_PW_AUTO && mm_auto);
+          if (pointwise && tc && wide_kernel && pointwise_mm_supported(din->c, op.d.cout)) {
+            r.kernel = GI_KERNEL_POINTWISE_MM;
+            pointwise_mm_pack(op.weights.data(), op.bias.data(), din->c, op.d.cout, &e->weight_blob, &r);
+          } else if (pointwise && tc && lane_kernel && pointwise_ts_supported(din->c, op.d.cout)) {
             r.kernel = GI_KERNEL_POINTWISE_TS;
             pointwise_ts_pack(op.weights.data(), op.bias.data(), din->c, op.d.cout, &e->weight_blob, &r);
           } else if (pointwise && tc && pointwise_tc_supported(din->c, op.d.cout)) {

@@ -104,6 +104,7 @@ static gi_status run_impl(gi_exec* e, const void* const* dev_inputs, void* const
       case GI_KERNEL_DEPTHWISE: err = launch_depthwise(r, p, e->storage, stream); break;
       case GI_KERNEL_DEPTHWISE_POINTWISE: err = launch_depthwise_pointwise(r, p, stream); break;
       case GI_KERNEL_INVERTED_RESIDUAL: err = launch_inverted_residual(r, p, stream); break;
+      case GI_KERNEL_POINTWISE_MM: err = launch_pointwise_mm(r, p, stream); break;
       case GI_KERNEL_NONE: break;  // computed by the previous launch
       case GI_KERNEL_ELTWISE:
         if (r.ep.has_res && !p.in1) p.in1 = p.res;
@@ -134,6 +135,7 @@ gi_status gi_device_status(uint32_t* flags) {
   if (err == 0) *flags |= pointwise_ts_error_word(&err) << 24;
   if (err == 0) *flags |= depthwise_pointwise_error_word(&err) << 28;
   if (err == 0) *flags |= inverted_residual_error_word(&err) << 4;
+  if (err == 0) *flags |= pointwise_mm_error_word(&err) << 8;
   if (err != 0) return fail(GI_E_CUDA, std::string("gi_device_status: ") + cudaGetErrorString(static_cast<cudaError_t>(err)));
   return GI_OK;
 }

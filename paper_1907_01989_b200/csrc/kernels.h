@@ -76,6 +76,13 @@ void depthwise_pointwise_pack(const float* w, const float* bias, int cin, int co
 int launch_depthwise_pointwise(const LaunchRec& r, const Ptrs& p, void* stream);
 unsigned int depthwise_pointwise_error_word(int* cuda_err);
 
+// Pointwise convolution for tensor-bound shapes (many input and output channels): 256 x 256 CTA tiles, both operands
+// streamed (pointwise_mm.cu; fp16 storage)
+bool pointwise_mm_supported(int cin, int cout);
+void pointwise_mm_pack(const float* w, const float* bias, int cin, int cout, std::vector<uint8_t>* blob, LaunchRec* r);
+int launch_pointwise_mm(const LaunchRec& r, const Ptrs& p, void* stream);
+unsigned int pointwise_mm_error_word(int* cuda_err);
+
 // One inverted-residual block (1x1 expansion -> depthwise 3x3 -> 1x1 projection, + residual) as one kernel (fp16
 // storage, planes of at most 256 pixels): neither hidden tensor leaves the SM.  `units` receives the kernel's parallelism.
 bool inverted_residual_supported(int B, int H, int W, int Ho, int Wo, int stride, int dil, int pt, int pl, int cin, int chid,

@@ -1,0 +1,434 @@
+// Pointwise (1x1) convolution for the shapes that are bound by the tensor pipe, not by HBM: many input AND
+// output channels (512 -> 512, 960 -> 960, 1280 -> 1280 on 14x14 planes at batch 256).  The other two 1x1
+// kernels give a CTA a tile of 128 pixels x 64-192 output channels; per byte fetched from L2 that is 64-77
+// flops, and at the rate the tensor pipe could run L2 cannot deliver.  This kernel is built around flops per L2
+// byte instead: a CTA tile is 256 pixels x up to 256 output channels (128 flops per byte), every weight chunk
+// fetched is used for two 128-row MMAs, and the K axis streams through a ring of stages:
+//
+//   A chunk  256 pixels x 32 channels, copied straight from the channel-sliced tensor into the canonical K-major
+//            operand layout by 8-byte cp.async (two 4-channel slices interleave into one 16-byte operand row):
+//            exactly 2*M*N*K flops, nothing padded or duplicated
+//   B chunk  up to 256 output channels x 32 input channels of the dense weight matrix, packed at compile time,
+//            one bulk copy
+//   MMA      2 x 2 tcgen05.mma (M = 128, N = tile width, K = 16) per chunk into two accumulators that together fill
+//            tensor memory; tcgen05.commit hands the stage back
+//   drain    sixteen warps: bias, activation, residual, fp16, 8-byte stores (256 contiguous bytes per warp)
+//
+// Tiles are numbered so that CTAs running at the same time work on the output-channel tiles of the same pixels:
+// the activations come from HBM once, the re-reads hit L2.  The accumulators are single-buffered (they fill tensor
+// memory), so a tile's drain is not overlapped with the next tile's MMAs; with K >= 512 the drain is a tenth of a tile.
+// All waits are bounded.
+#include <cuda.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include "kernels.h"
+#include "pdl.cuh"
+#include "sm100_ptx.cuh"
+
+namespace gi {
+namespace {
+
+using namespace ptx;
+
+constexpr int kRows = 256;        // pixels per CTA tile: two MMAs of 128 rows
+constexpr int kKc = 8;            // input slices (32 channels) per chunk: small chunks, many stages in flight
+constexpr int kLoadWarps = 4, kDrainWarps = 16;
+constexpr int kLoadThreads = 32 * kLoadWarps;
+constexpr int kMmaWarps = 2;      // one issuing thread per 128-row accumulator: the issue stream, not the pipe, bounds a chunk
+constexpr int kFirstLoad = 1 + kMmaWarps, kFirstDrain = kFirstLoad + kLoadWarps;
+constexpr int kThreads = 32 * (kFirstDrain + kDrainWarps);
+constexpr int kMaxStages = 8;
+constexpr int kHeader = 1024;
+constexpr int kABytes = (kKc / 2) * kRows * 16;  // 16 KB
+constexpr int kSmemMax = 227 * 1024;
+constexpr int kAhead = 3;         // chunks a loader thread keeps in flight before it waits for the oldest
+
+__device__ unsigned int g_mm_error = 0;
+enum : unsigned { kErrCopy = 1u, kErrMma = 2u, kErrLoad = 4u, kErrDrain = 8u };
+
+struct MmParams {
+  const __half* in;
+  const __half* res;
+  __half* out;
+  const unsigned char* wts;  // [n_tiles][n_chunks] blocks of b_bytes
+  const float* bias;
+  unsigned int m_total;      // pixels (batch x stored plane)
+  int s_in, s_out;
+  int n_chunks, n_tile, n_tiles, m_tiles;
+  int stages;
+  unsigned b_bytes, stage_bytes;
+  int act_pre, has_res, act_post;
+  unsigned timeout_ns;
+};
+
+struct Header {
+  unsigned long long full[kMaxStages], empty[kMaxStages];  // full: the load threads' arrivals and the weight copy's bytes
+  unsigned long long acc_full, acc_empty;
+  unsigned tmem_addr, abort_flag;
+};
+static_assert(sizeof(Header) <= kHeader, "header too large");
+
+__device__ __forceinline__ float act1(float v, int kind) {
+  if (kind == GI_ACT_RELU) return fmaxf(v, 0.0f);
+  if (kind == GI_ACT_RELU6) return fminf(fmaxf(v, 0.0f), 6.0f);
+  return v;
+}
+// 8-byte asynchronous copy; with `bytes` = 0 nothing is read and the destination is filled with zeros
+__device__ __forceinline__ void cp_async8_zfill(unsigned dst, const void* src, unsigned bytes) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait_pending() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// ACT: activation right after the bias; TAIL: a residual add and / or a second activation follow
+template <int ACT, bool TAIL>
+__global__ void __launch_bounds__(kThreads, 1) pointwise_mm_kernel(const MmParams p) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  Header* hdr = reinterpret_cast<Header*>(smem);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile unsigned* abort_flag = &hdr->abort_flag;
+  const unsigned st0 = smem_u32(smem + kHeader);  // stage: A chunk (16 KB), then B chunk
+  const int n_units = p.m_tiles * p.n_tiles;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < p.stages; ++i) {
+      mbar_init(smem_u32(&hdr->full[i]), kLoadThreads + 1);
+      mbar_init(smem_u32(&hdr->empty[i]), kMmaWarps);
+    }
+    mbar_init(smem_u32(&hdr->acc_full), kMmaWarps);
+    mbar_init(smem_u32(&hdr->acc_empty), kDrainWarps);
+    hdr->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32(&hdr->tmem_addr), 512u);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const unsigned tmem_base = hdr->tmem_addr;
+  pdl_launch_dependents();
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ weight chunks (never change: no wait for the previous kernel)
+    if (lane == 0) {
+      unsigned it = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+        const int nt = u % p.n_tiles;
+        for (int c = 0; c < p.n_chunks; ++c, ++it) {
+          const unsigned stage = it % p.stages, phase = (it / p.stages) & 1u;
+          if (!mbar_wait_parked(smem_u32(&hdr->empty[stage]), phase ^ 1u, abort_flag, p.timeout_ns, &g_mm_error, kErrCopy)) {
+            ok = false;
+            break;
+          }
+          const unsigned full = smem_u32(&hdr->full[stage]);
+          mbar_expect_tx(full, p.b_bytes);
+          bulk_load(st0 + stage * p.stage_bytes + kABytes, p.wts + (static_cast<size_t>(nt) * p.n_chunks + c) * p.b_bytes, p.b_bytes, full);
+        }
+      }
+      if (!ok) {
+        const unsigned first = it > static_cast<unsigned>(p.stages) ? it - p.stages : 0u;
+        for (unsigned j = first; j < it; ++j) {
+          const unsigned long long t0 = global_timer_ns();
+          while (!mbar_try_wait(smem_u32(&hdr->full[j % p.stages]), (j / p.stages) & 1u)) {
+            if (global_timer_ns() - t0 > p.timeout_ns) {
+              atomicOr(&g_mm_error, kErrDrain);
+              break;
+            }
+          }
+        }
+      }
+    }
+  } else if (warp < kFirstLoad) {
+    // ------------------------------------------------------------ MMA issuers: warp 1 owns accumulator 0 (rows 0-127 of
+    // the tile), warp 2 accumulator 1; both read the same stages and each hands a stage back with its own commit
+    if (lane == 0) {
+      const int t = warp - 1;
+      const unsigned n_cols = static_cast<unsigned>(p.n_tile);
+      const unsigned idesc = (1u << 4) | ((n_cols >> 3) << 17) | ((128u >> 4) << 24);
+      const unsigned a_lbo = kRows * 16u, b_lbo = n_cols * 16u;
+      unsigned it = 0, tile = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++tile) {
+        // the first MMA of a tile overwrites the accumulators: the tile before must have been drained
+        if (!mbar_wait(smem_u32(&hdr->acc_empty), (tile & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_mm_error, kErrMma)) break;
+        tc_fence_after();
+        for (int c = 0; c < p.n_chunks; ++c, ++it) {
+          const unsigned stage = it % p.stages, phase = (it / p.stages) & 1u;
+          // the issuing thread's own instruction stream bounds the chunk rate: one barrier per stage for both operands,
+          // and a completed phase is recognised without the call into the bounded-wait routine
+          if (!mbar_try_wait(smem_u32(&hdr->full[stage]), phase) &&
+              !mbar_wait(smem_u32(&hdr->full[stage]), phase, abort_flag, p.timeout_ns, &g_mm_error, kErrMma)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const unsigned a_base = st0 + stage * p.stage_bytes, b_base = a_base + kABytes;
+          unsigned long long ad = smem_desc(a_base + static_cast<unsigned>(t) * 2048u, a_lbo, 128);
+          unsigned long long bd = smem_desc(b_base, b_lbo, 128);
+          const unsigned long long ad_step = static_cast<unsigned long long>((2u * a_lbo) >> 4);
+          const unsigned long long bd_step = static_cast<unsigned long long>((2u * b_lbo) >> 4);
+#pragma unroll
+          for (int ks = 0; ks < kKc / 4; ++ks) {
+            umma_f16(tmem_base + static_cast<unsigned>(t) * n_cols, ad, bd, idesc, (c > 0 || ks > 0) ? 1u : 0u);
+            ad += ad_step;
+            bd += bd_step;
+          }
+          umma_commit(smem_u32(&hdr->empty[stage]));
+        }
+        if (ok) umma_commit(smem_u32(&hdr->acc_full));
+      }
+    }
+  } else if (warp < kFirstDrain) {
+    // ------------------------------------------------------------ activation chunks: 8-byte cp.async into the operand layout
+    const int tid = threadIdx.x - 32 * kFirstLoad;  // 0 .. 127: rows tid and tid + 128 of the tile
+    pdl_wait();  // activations are read only below
+    unsigned it = 0, signalled = 0;
+    bool ok = true;
+    // chunk number j (of this CTA's sequence) has landed for this thread: make it visible to the tensor core's
+    // proxy and count this thread in
+    auto publish = [&](unsigned j) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_arrive(smem_u32(&hdr->full[j % p.stages]));
+    };
+    for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+      const int mt = u / p.n_tiles;
+      const unsigned px0 = static_cast<unsigned>(mt) * kRows + static_cast<unsigned>(tid);
+      for (int c = 0; c < p.n_chunks; ++c, ++it) {
+        const unsigned stage = it % p.stages, phase = (it / p.stages) & 1u;
+        if (!mbar_try_wait(smem_u32(&hdr->empty[stage]), phase ^ 1u) &&
+            !mbar_wait(smem_u32(&hdr->empty[stage]), phase ^ 1u, abort_flag, p.timeout_ns, &g_mm_error, kErrLoad)) {
+          ok = false;
+          break;
+        }
+        const unsigned dst0 = st0 + stage * p.stage_bytes + static_cast<unsigned>(tid) * 16u;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const unsigned px = px0 + static_cast<unsigned>(h) * 128u;
+          const bool px_ok = px < p.m_total;
+          const __half* src = p.in + (static_cast<size_t>(c * kKc) * p.m_total + (px_ok ? px : 0u)) * 4;
+          const unsigned dst = dst0 + static_cast<unsigned>(h) * 2048u;
+#pragma unroll
+          for (int s = 0; s < kKc; ++s) {
+            // slices beyond the tensor's last one and pixels beyond its end read nothing and are filled with zeros
+            const bool live = px_ok && c * kKc + s < p.s_in;
+            cp_async8_zfill(dst + static_cast<unsigned>(s >> 1) * (kRows * 16u) + static_cast<unsigned>(s & 1) * 8u,
+                            live ? static_cast<const void*>(src + static_cast<size_t>(s) * p.m_total * 4) : static_cast<const void*>(p.in),
+                            live ? 8u : 0u);
+          }
+        }
+        cp_async_commit();
+        if (it >= static_cast<unsigned>(kAhead)) {
+          cp_async_wait_pending<kAhead>();
+          publish(signalled++);
+        }
+      }
+    }
+    // the last chunks in flight
+    cp_async_wait_pending<0>();
+    if (ok)
+      while (signalled < it) publish(signalled++);
+  } else {
+    // ------------------------------------------------------------ drain: accumulators -> global memory
+    const int dw = warp - kFirstDrain;
+    const int quarter = warp & 3, sub = dw >> 2;  // TMEM lane quarter; index among the four warps sharing it
+    const unsigned lane_bits = static_cast<unsigned>(quarter * 32) << 16;
+    const int groups = p.n_tile >> 4;
+    pdl_wait();  // the residual is read and the output written only below
+    unsigned tile = 0;
+    for (int u = blockIdx.x; u < n_units; u += gridDim.x, ++tile) {
+      const int mt = u / p.n_tiles, nt = u - mt * p.n_tiles;
+      if (!mbar_wait_warp(smem_u32(&hdr->acc_full), tile & 1u, abort_flag, p.timeout_ns, &g_mm_error, kErrDrain)) break;
+      tc_fence_after();
+      for (int e = sub; e < 2 * groups; e += kDrainWarps / 4) {
+        const int t = e / groups, g = e - t * groups;
+        const unsigned pixel = static_cast<unsigned>(mt) * kRows + static_cast<unsigned>(t * 128 + quarter * 32 + lane);
+        const bool px_ok = pixel < p.m_total;
+        unsigned r[16];
+        tmem_ld16(tmem_base + lane_bits + static_cast<unsigned>(t * p.n_tile + g * 16), r);
+        const int so0 = (nt * p.n_tile) / 4 + g * 4;
+        // the drain of a 256 x 256 tile is 512 warp-wide slice stores that nothing overlaps (the accumulators fill
+        // tensor memory): every instruction here is paid in full, so the common tail-less case is kept to packed adds,
+        // the clamping conversion and one store
+        uint2 rq[4];
+        if (TAIL) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            rq[j] = make_uint2(0u, 0u);
+            if (p.has_res && px_ok && so0 + j < p.s_out)
+              rq[j] = __ldg(reinterpret_cast<const uint2*>(p.res + (static_cast<size_t>(so0 + j) * p.m_total + pixel) * 4));
+          }
+        }
+        __half* dst = p.out + (static_cast<size_t>(so0) * p.m_total + pixel) * 4;
+        const size_t slice_stride = static_cast<size_t>(p.m_total) * 4;
+        tmem_ld_wait16(r);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (so0 + j >= p.s_out || !px_ok) continue;
+          const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias) + so0 + j);
+          const float2 v0 = __fadd2_rn(make_float2(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1])), make_float2(b.x, b.y));
+          const float2 v1 = __fadd2_rn(make_float2(__uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3])), make_float2(b.z, b.w));
+          uint2 o;
+          if (!TAIL) {
+            // the conversion clamps at zero itself; clamping at 6 after the rounding equals rounding after the clamp
+            o.x = pack_f16x2<ACT != GI_ACT_NONE>(v0.x, v0.y);
+            o.y = pack_f16x2<ACT != GI_ACT_NONE>(v1.x, v1.y);
+            if (ACT == GI_ACT_RELU6) {
+              const __half2 six = __float2half2_rn(6.f);
+              const __half2 h0 = __hmin2(*reinterpret_cast<const __half2*>(&o.x), six), h1 = __hmin2(*reinterpret_cast<const __half2*>(&o.y), six);
+              o.x = *reinterpret_cast<const unsigned*>(&h0);
+              o.y = *reinterpret_cast<const unsigned*>(&h1);
+            }
+          } else {
+            const float2 q0 = __half22float2(*reinterpret_cast<const __half2*>(&rq[j].x));
+            const float2 q1 = __half22float2(*reinterpret_cast<const __half2*>(&rq[j].y));
+            o.x = pack_f16x2<false>(act1(act1(v0.x, ACT) + q0.x, p.act_post), act1(act1(v0.y, ACT) + q0.y, p.act_post));
+            o.y = pack_f16x2<false>(act1(act1(v1.x, ACT) + q1.x, p.act_post), act1(act1(v1.y, ACT) + q1.y, p.act_post));
+          }
+          *reinterpret_cast<uint2*>(dst + j * slice_stride) = o;
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&hdr->acc_empty));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512u);
+  }
+}
+
+struct Tiling {
+  int s_in, s_out, n_chunks, n_tiles, n_tile, stages;
+  unsigned b_bytes, stage_bytes;
+  size_t smem;
+};
+
+Tiling choose_tiling(int cin, int cout) {
+  Tiling t;
+  t.s_in = slices(cin);
+  t.s_out = slices(cout);
+  t.n_chunks = (t.s_in + kKc - 1) / kKc;
+  const int n_pad = (cout + 15) / 16 * 16;
+  t.n_tiles = (n_pad + 255) / 256;
+  t.n_tile = ((n_pad + t.n_tiles - 1) / t.n_tiles + 15) / 16 * 16;
+  t.b_bytes = static_cast<unsigned>(t.n_tile) * kKc * 8u;  // n_tile rows x 32 channels x 2 bytes
+  t.stage_bytes = kABytes + t.b_bytes;
+  int stages = (kSmemMax - kHeader) / static_cast<int>(t.stage_bytes);
+  t.stages = stages > kMaxStages ? kMaxStages : stages;
+  t.smem = kHeader + static_cast<size_t>(t.stages) * t.stage_bytes;
+  return t;
+}
+
+}  // namespace
+
+bool pointwise_mm_supported(int cin, int cout) {
+  if (cin <= 0 || cout <= 0) return false;
+  return choose_tiling(cin, cout).stages > kAhead;  // the loaders keep kAhead chunks in flight behind the one they fill
+}
+
+// Dense weights as the B operand, per (output tile, K chunk): [4 K groups][n_tile rows][8 halves]; entries beyond
+// the real channels are zero.
+void pointwise_mm_pack(const float* w, const float* bias, int cin, int cout, std::vector<uint8_t>* blob, LaunchRec* r) {
+  const Tiling t = choose_tiling(cin, cout);
+  const size_t wbytes = static_cast<size_t>(t.n_tiles) * t.n_chunks * t.b_bytes;
+  const uint64_t woff = round_up_u64(blob->size(), 256);
+  blob->resize(woff + wbytes, 0);
+  const uint64_t boff = round_up_u64(blob->size(), 256);
+  blob->resize(boff + static_cast<size_t>(t.n_tiles) * t.n_tile * sizeof(float), 0);
+  uint16_t* wp = reinterpret_cast<uint16_t*>(blob->data() + woff);
+  float* bp = reinterpret_cast<float*>(blob->data() + boff);
+  for (int co = 0; co < cout; ++co) {
+    const int nt = co / t.n_tile, row = co % t.n_tile;
+    bp[co] = bias[co];
+    for (int ci = 0; ci < cin; ++ci) {
+      const int chunk = ci / (kKc * 4), k = ci % (kKc * 4);
+      uint16_t* base = wp + (static_cast<size_t>(nt) * t.n_chunks + chunk) * (t.b_bytes / 2);
+      base[(static_cast<size_t>(k / 8) * t.n_tile + row) * 8 + k % 8] = f32_to_f16_rne(w[static_cast<size_t>(co) * cin + ci]);
+    }
+  }
+  r->wts = Loc{W_WEIGHTS, 0, woff};
+  r->bias = Loc{W_WEIGHTS, 0, boff};
+  r->wts_bytes = wbytes;
+  r->tc_nt = t.n_tile;
+  r->tc_kc = kKc;
+  r->tc_stages = t.stages;
+}
+
+int launch_pointwise_mm(const LaunchRec& r, const Ptrs& p, void* stream) {
+  const Tiling t = choose_tiling(r.C, r.Co);
+  MmParams k{};
+  k.in = static_cast<const __half*>(p.in0);
+  k.res = static_cast<const __half*>(p.res);
+  k.out = static_cast<__half*>(p.out);
+  k.wts = static_cast<const unsigned char*>(p.wts);
+  k.bias = static_cast<const float*>(p.bias);
+  k.m_total = static_cast<unsigned>(r.B) * static_cast<unsigned>(plane_pixels(r.H, r.W));
+  k.s_in = t.s_in;
+  k.s_out = t.s_out;
+  k.n_chunks = t.n_chunks;
+  k.n_tile = t.n_tile;
+  k.n_tiles = t.n_tiles;
+  k.m_tiles = static_cast<int>((k.m_total + kRows - 1) / kRows);
+  k.stages = t.stages;
+  k.b_bytes = t.b_bytes;
+  k.stage_bytes = t.stage_bytes;
+  k.act_pre = r.ep.act_pre;
+  k.has_res = r.ep.has_res;
+  k.act_post = r.ep.act_post;
+  k.timeout_ns = 1000000000u;
+  static bool attr_done_dev[kMaxDevices] = {};
+  bool& attr_done = attr_done_dev[current_device_slot()];
+  if (!attr_done) {
+    cudaError_t e = cudaSuccess;
+#define GI_MM_ATTR(A, T) \
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(pointwise_mm_kernel<A, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax)
+    GI_MM_ATTR(GI_ACT_NONE, false);
+    GI_MM_ATTR(GI_ACT_RELU, false);
+    GI_MM_ATTR(GI_ACT_RELU6, false);
+    GI_MM_ATTR(GI_ACT_NONE, true);
+    GI_MM_ATTR(GI_ACT_RELU, true);
+    GI_MM_ATTR(GI_ACT_RELU6, true);
+#undef GI_MM_ATTR
+    if (e != cudaSuccess) return static_cast<int>(e);
+    attr_done = true;
+  }
+  const long long units = static_cast<long long>(k.m_tiles) * k.n_tiles;
+  const int sms = device_sm_count();
+  const unsigned grid = static_cast<unsigned>(units < sms ? units : sms);
+  // the kernel reserves all of tensor memory: ask for enough shared memory that no second CTA shares the SM
+  size_t smem = t.smem;
+  if (smem < 120 * 1024) smem = 120 * 1024;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const bool tail = k.has_res || k.act_post != GI_ACT_NONE;
+#define GI_MM_LAUNCH(A, T) launch_pdl(pointwise_mm_kernel<A, T>, grid, kThreads, smem, st, k)
+  if (tail) {
+    if (k.act_pre == GI_ACT_RELU6) GI_MM_LAUNCH(GI_ACT_RELU6, true);
+    else if (k.act_pre == GI_ACT_RELU) GI_MM_LAUNCH(GI_ACT_RELU, true);
+    else GI_MM_LAUNCH(GI_ACT_NONE, true);
+  } else {
+    if (k.act_pre == GI_ACT_RELU6) GI_MM_LAUNCH(GI_ACT_RELU6, false);
+    else if (k.act_pre == GI_ACT_RELU) GI_MM_LAUNCH(GI_ACT_RELU, false);
+    else GI_MM_LAUNCH(GI_ACT_NONE, false);
+  }
+#undef GI_MM_LAUNCH
+  return static_cast<int>(cudaGetLastError());
+}
+
+unsigned int pointwise_mm_error_word(int* cuda_err) {
+  unsigned int v = 0;
+  const cudaError_t e = cudaMemcpyFromSymbol(&v, g_mm_error, sizeof v);
+  if (cuda_err) *cuda_err = static_cast<int>(e);
+  return v;
+}
+
+}  // namespace gi

@@ -99,8 +99,9 @@ def test_pointwise_fp32(case):
     assert "conv_simt" in kernels  # fp32 storage always takes the CUDA-core kernel
 
 
-@pytest.mark.parametrize("mode,kernel", [(api.GI_PW_TC_PAIR, "pointwise_tc"), (api.GI_PW_TC_LANE, "pointwise_ts")],
-                         ids=["pair", "lane"])
+@pytest.mark.parametrize("mode,kernel", [(api.GI_PW_TC_PAIR, "pointwise_tc"), (api.GI_PW_TC_LANE, "pointwise_ts"),
+                                         (api.GI_PW_TC_WIDE, "pointwise_mm")],
+                         ids=["pair", "lane", "wide"])
 @pytest.mark.parametrize("case", PW_CASES)
 def test_pointwise_tensor_core(case, mode, kernel):
     """Both tensor-core variants on every case: operands by TMA (pixel pairs) and through tensor memory."""
@@ -686,11 +687,11 @@ def test_sweep_pointwise_points_at_full_size(case):
     b, hw, cin, cout, res = case
     spec = wl.single_pointwise(b, hw, cin, cout, residual=res)
     run, _, _ = check_outputs(spec, api.GI_F16, images=[0, b // 2 + 1, b - 1])
-    assert any(api.KERNEL_NAMES[o.kernel] in ("pointwise_tc", "pointwise_ts") for o in run.ex.ops())
+    assert any(api.KERNEL_NAMES[o.kernel] in ("pointwise_tc", "pointwise_ts", "pointwise_mm") for o in run.ex.ops())
     assert api.gi_device_status() == 0
 
 
-@pytest.mark.parametrize("mode", [api.GI_PW_TC_PAIR, api.GI_PW_TC_LANE], ids=["pair", "lane"])
+@pytest.mark.parametrize("mode", [api.GI_PW_TC_PAIR, api.GI_PW_TC_LANE, api.GI_PW_TC_WIDE], ids=["pair", "lane", "wide"])
 @pytest.mark.parametrize("case", [(256, 14, 576, 576), (64, 14, 1280, 1280)], ids=["576", "1280"])
 def test_sweep_tensor_bound_points_both_variants(case, mode):
     b, hw, cin, cout = case
