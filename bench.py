@@ -44,7 +44,7 @@ import numpy as np  # noqa: E402
 
 NETS = {"v2": ("mobilenet_v2", "MobileNetV2-224"), "v1": ("mobilenet_v1", "MobileNetV1-224"),
         "seg": ("mobilenet_v2_segmentation", "MobileNetV2-513-OS16-seg"), "fire": ("fire_network", "fire-module-network-96")}
-PW_MODES = {"auto": 0, "simt": 1, "pair": 2, "lane": 3, "wide": 4}
+PW_MODES = {"auto": 0, "simt": 1, "pair": 2, "lane": 3, "wide": 4, "rule": 5}
 XOP_MODES = {"auto": 0, "off": 1, "on": 2}
 # dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes, from the ncu captures summarised
 # under profiles/ (depthwise: batch 128, 112x112x96, stride 1: 560.3 MB over 616.6 MB; pointwise_tc:
@@ -456,7 +456,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--net", default="v2", choices=sorted(NETS))
     ap.add_argument("--batch", type=int, default=None)
-    ap.add_argument("--pointwise", default="auto", choices=["auto", "simt", "pair", "lane", "wide"])
+    ap.add_argument("--pointwise", default="auto", choices=["auto", "simt", "pair", "lane", "wide", "rule"])
     ap.add_argument("--cross-op", default="auto", choices=["auto", "off", "on"],
                     help="depthwise + 1x1 convolution as one kernel: where the library chooses it, never, wherever supported")
     ap.add_argument("--per-op", default=None, help="write the per-op timing table to this file")

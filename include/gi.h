@@ -89,12 +89,15 @@ enum {
 
 /* Kernel choice for full convolutions. */
 enum {
-  GI_PW_AUTO = 0,      /* tensor-core kernels for fp16 storage, CUDA-core kernel for fp32 storage */
+  GI_PW_AUTO = 0,      /* tensor-core kernels for fp16 storage (which one: the measured launch table, else a rule), CUDA-core
+                          kernel for fp32 storage */
   GI_PW_SIMT = 1,      /* force the plain CUDA-core kernel for every full convolution (validation) */
   GI_PW_TC_PAIR = 2,   /* 1x1: always the pixel-pair tensor-core kernel (operands by TMA) */
   GI_PW_TC_LANE = 3,   /* 1x1: always the lane-per-pixel tensor-core kernel (activations through tensor memory) */
-  GI_PW_TC_WIDE = 4    /* 1x1: always the wide-tile tensor-core kernel built for tensor-bound shapes (256 pixels x up to
+  GI_PW_TC_WIDE = 4,   /* 1x1: always the wide-tile tensor-core kernel built for tensor-bound shapes (256 pixels x up to
                           256 output channels per CTA, both operands streamed) */
+  GI_PW_RULE = 5       /* like GI_PW_AUTO, but by the selection rule alone: the table of measured choices (the counterpart of
+                          the paper's work-group table, Section 4) is not consulted */
 };
 
 /* Cross-operator kernels: a depthwise 3x3 convolution whose only consumer is a 1x1 convolution runs

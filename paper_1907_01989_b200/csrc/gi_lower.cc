@@ -118,6 +118,24 @@ static bool pointwise_follows(const gi_graph& g, const gi_exec* e, size_t i) {
          d.pad_r == 0;
 }
 
+// Launch table: the fastest 1x1 kernel per shape as measured on the device (generated; the analogue of the paper's
+// table of optimal work-group sizes, Section 4).  Consulted before the rule below; shapes that are not in it - any
+// network other than the benchmark ones - take the rule.
+struct LaunchChoice {
+  long long px;
+  int cin, cout, kernel;
+  float ms_pair, ms_lane, ms_wide;
+};
+static const LaunchChoice kLaunchTable[] = {
+    {0, 0, 0, 0, 0.f, 0.f, 0.f},  // keeps the array non-empty when the table has not been generated
+#include "launch_table.inc"
+};
+static const LaunchChoice* launch_table_lookup(long long px, int cin, int cout) {
+  for (const LaunchChoice& c : kLaunchTable)
+    if (c.px == px && c.cin == cin && c.cout == cout && c.kernel != 0) return &c;
+  return nullptr;
+}
+
 // pixels of a 1x1 convolution's input as the kernels count them: batch x stored plane
 static long long m_px_all_for_mm(const gi_exec* e, const TensorDesc* t) {
   return static_cast<long long>(e->batch) * plane_pixels(t->h, t->w);
@@ -347,7 +365,7 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
           const bool one_wave = m_px_all <= 64LL * 128 || (m_px_all <= 148LL * 128 && din->c < 960);
           const bool lane_rule = op.d.cout >= 96 && din->c >= 64 && din->c < 960 && !(din->c <= 96 && op.d.cout >= 4 * din->c);
           const bool lane_auto = one_wave || lane_rule;
-          const bool lane_kernel = e->opt.pointwise == GI_PW_TC_LANE || (e->opt.pointwise == GI_PW_AUTO && lane_auto);
+          const bool lane_kernel = e->opt.pointwise == GI_PW_TC_LANE || ((e->opt.pointwise == GI_PW_AUTO || e->opt.pointwise == GI_PW_RULE) && lane_auto);
           // The wide-tile kernel (256 pixels x up to 256 output channels per CTA) is for the shapes bound by the tensor
           // pipe: at least 512 input and 512 output channels.  Measured against the library's previous choice at batch
           // 256 (time wide / time before): 14x14 1280->1280 0.57, 960->960 0.72, 576->576 0.76, 7x7 1024->1024 0.83,
@@ -358,11 +376,19 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
           const long long mm_waves = (mm_units + 147) / 148;
           const bool mm_auto = din->c >= 512 && op.d.cout >= 512 && mm_units >= 64 &&
                                (din->c >= 576 || mm_units * 100 >= mm_waves * 148 * 85);
-          const bool wide_kernel = e->opt.pointwise == GI_PW_TC_WIDE || (e->opt.pointwise == GI_PW_AUTO && mm_auto);
+          bool wide_kernel = e->opt.pointwise == GI_PW_TC_WIDE || ((e->opt.pointwise == GI_PW_AUTO || e->opt.pointwise == GI_PW_RULE) && mm_auto);
+          bool lane_tab = false, pair_tab = false;
+          if (e->opt.pointwise == GI_PW_AUTO && pointwise && tc) {
+            if (const LaunchChoice* lc = launch_table_lookup(m_px_all_for_mm(e, din), din->c, op.d.cout)) {
+              wide_kernel = lc->kernel == GI_KERNEL_POINTWISE_MM;
+              lane_tab = lc->kernel == GI_KERNEL_POINTWISE_TS;
+              pair_tab = lc->kernel == GI_KERNEL_POINTWISE_TC;
+            }
+          }
           if (pointwise && tc && wide_kernel && pointwise_mm_supported(din->c, op.d.cout)) {
             r.kernel = GI_KERNEL_POINTWISE_MM;
             pointwise_mm_pack(op.weights.data(), op.bias.data(), din->c, op.d.cout, &e->weight_blob, &r);
-          } else if (pointwise && tc && lane_kernel && pointwise_ts_supported(din->c, op.d.cout)) {
+          } else if (pointwise && tc && (lane_tab || (lane_kernel && !pair_tab)) && pointwise_ts_supported(din->c, op.d.cout)) {
             r.kernel = GI_KERNEL_POINTWISE_TS;
             pointwise_ts_pack(op.weights.data(), op.bias.data(), din->c, op.d.cout, &e->weight_blob, &r);
           } else if (pointwise && tc && pointwise_tc_supported(din->c, op.d.cout)) {

@@ -279,9 +279,13 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_tc_kernel(const __grid_
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
                 const float2 f = __half22float2(rh[i]);  // zero when there is no residual
-                const float x = act1(act1(v[i].x, ACT) + f.x, p.act_post);
-                const float y = act1(act1(v[i].y, ACT) + f.y, p.act_post);
-                oh[i] = __floats2half2_rn(x, y);
+                // the usual tail is the residual sum of a linear projection: no activation on either side of it
+                float2 s2 = __fadd2_rn(make_float2(act1(v[i].x, ACT), act1(v[i].y, ACT)), f);
+                if (p.act_post != GI_ACT_NONE) {
+                  s2.x = act1(s2.x, p.act_post);
+                  s2.y = act1(s2.y, p.act_post);
+                }
+                oh[i] = __floats2half2_rn(s2.x, s2.y);
               }
             }
             *reinterpret_cast<uint4*>(p.out + off) = o;

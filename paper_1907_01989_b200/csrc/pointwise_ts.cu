@@ -350,8 +350,15 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
             const uint2 q = res_cur[j];
             const float2 r0 = __half22float2(*reinterpret_cast<const __half2*>(&q.x));
             const float2 r1 = __half22float2(*reinterpret_cast<const __half2*>(&q.y));
-            h0 = __floats2half2_rn(act1(act1(v0.x, ACT) + r0.x, p.act_post), act1(act1(v0.y, ACT) + r0.y, p.act_post));
-            h1 = __floats2half2_rn(act1(act1(v1.x, ACT) + r1.x, p.act_post), act1(act1(v1.y, ACT) + r1.y, p.act_post));
+            // the usual tail is the residual sum of a linear projection: no activation on either side of it
+            float2 s0 = __fadd2_rn(make_float2(act1(v0.x, ACT), act1(v0.y, ACT)), r0);
+            float2 s1 = __fadd2_rn(make_float2(act1(v1.x, ACT), act1(v1.y, ACT)), r1);
+            if (p.act_post != GI_ACT_NONE) {
+              s0 = make_float2(act1(s0.x, p.act_post), act1(s0.y, p.act_post));
+              s1 = make_float2(act1(s1.x, p.act_post), act1(s1.y, p.act_post));
+            }
+            h0 = __floats2half2_rn(s0.x, s0.y);
+            h1 = __floats2half2_rn(s1.x, s1.y);
           }
           uint2 o;
           o.x = *reinterpret_cast<const unsigned*>(&h0);

@@ -338,20 +338,31 @@ def test_cross_op_option():
     g = api.graph_from_spec(pair, api.GI_F16)[0]
     a, c = g.compile(cross_op=api.GI_XOP_OFF, planner=api.GI_PLAN_NAIVE), g.compile(cross_op=api.GI_XOP_ON, planner=api.GI_PLAN_NAIVE)
     assert a.info.arena_bytes == c.info.arena_bytes and a.info.n_ops == c.info.n_ops
-    # whole network at batch 256: 13 pairs qualify; one kernel reads the pair's input while it writes its output, so a
-    # pair whose input and output share arena bytes (legal for two ops: their lifetimes do not meet) stays two kernels
+    # whole network at batch 256: the ten blocks on 14x14 and 7x7 planes run as one kernel each (expansion, depthwise
+    # and projection: two ops without a launch per block); of the seven blocks on larger planes the depthwise ->
+    # projection pair runs as one kernel (one op without a launch each).  One kernel reads the pair's / block's input
+    # while it writes its output, so where input and output share arena bytes (legal for separate ops: their
+    # lifetimes do not meet) the ops stay separate kernels - never under the naive plan
     v2 = kernels(wl.mobilenet_v2(256), cross_op=api.GI_XOP_ON, planner=api.GI_PLAN_NAIVE)
-    # (the 14th op without a launch is the layout conversion of the input, which the stem reads as NHWC itself)
-    assert v2.count("depthwise_pointwise") == 13 and v2.count("none") == 14 and v2[0] == "none" and v2[1] == "conv3x3_tc"
+    # (one more op without a launch: the layout conversion of the input, which the stem reads as NHWC itself)
+    assert v2.count("inverted_residual") == 10 and v2.count("depthwise_pointwise") == 7 and v2.count("none") == 28
+    assert v2[0] == "none" and v2[1] == "conv3x3_tc"
+    # the library's own choice: the blocks on 7x7 planes only (measured: the 14x14 blocks are not faster as one kernel),
+    # and none at batch 1, where a block would be a single CTA
+    auto = kernels(wl.mobilenet_v2(256), planner=api.GI_PLAN_NAIVE)
+    assert auto.count("inverted_residual") == 3 and auto.count("depthwise_pointwise") == 0
+    assert "inverted_residual" not in kernels(wl.mobilenet_v2(1))
     gv2 = api.graph_from_spec(wl.mobilenet_v2(256), api.GI_F16)[0]
     for planner in (api.GI_PLAN_GREEDY_BY_SIZE, api.GI_PLAN_GREEDY_SHARED_OBJECTS, api.GI_PLAN_MIN_COST_FLOW):
         ex = gv2.compile(cross_op=api.GI_XOP_ON, planner=planner)
         ops = ex.ops()
         for i, o in enumerate(ops):
-            if api.KERNEL_NAMES[o.kernel] == "depthwise_pointwise":
-                tin, tout = ex.tensor(o.inputs[0]), ex.tensor(ops[i + 1].output)
+            name = api.KERNEL_NAMES[o.kernel]
+            if name in ("depthwise_pointwise", "inverted_residual"):
+                tin, tout = ex.tensor(o.inputs[0]), ex.tensor(ops[i + (1 if name == "depthwise_pointwise" else 2)].output)
                 assert tin.offset + tin.bytes <= tout.offset or tout.offset + tout.bytes <= tin.offset
-    assert [api.KERNEL_NAMES[o.kernel] for o in gv2.compile(cross_op=api.GI_XOP_ON).ops()].count("depthwise_pointwise") == 11
+    names = [api.KERNEL_NAMES[o.kernel] for o in gv2.compile(cross_op=api.GI_XOP_ON).ops()]
+    assert names.count("depthwise_pointwise") == 5 and names.count("inverted_residual") == 9
     with pytest.raises(api.GiError):
         g.compile(cross_op=7)
 
@@ -475,3 +486,58 @@ def test_concat_view_eligibility_rules():
         b.output(b.conv2d(b.add(b.add(c1, c2), c3), 4, 1))
     spec, v = fused_and_views(same_twice_and_reused)
     assert v == {1: (4, 0), 2: (4, 2)}
+
+
+# ---------------------------------------------------------------------- launch table vs selection rule
+def _launch_table():
+    """Rows of csrc/launch_table.inc: (pixels, cin, cout, kernel id, ms pair, ms lane, ms wide)."""
+    import re
+    path = os.path.join(os.path.dirname(api.LIB_PATH), "csrc", "launch_table.inc")
+    rows = []
+    with open(path) as fh:
+        for line in fh:
+            m = re.match(r"\{(\d+)LL, (\d+), (\d+), (\d+), ([\d.]+)f, ([\d.]+)f, ([\d.]+)f\},", line.strip())
+            if m:
+                rows.append((int(m.group(1)), int(m.group(2)), int(m.group(3)), int(m.group(4)),
+                             float(m.group(5)), float(m.group(6)), float(m.group(7))))
+    return rows
+
+
+def test_launch_table_and_rule_agree_where_both_apply():
+    """The generated table of measured 1x1 kernel choices (the counterpart of the paper's work-group table,
+    Section 4) is consulted before the selection rule.  Where a shape is in the table, either both name the same
+    kernel, or the table's own measurements show the rule's kernel more than 3 % slower - and the executable
+    follows the table.  Shapes outside the table take the rule."""
+    rows = _launch_table()
+    assert len(rows) >= 60
+    col = {4: 4, 10: 5, 16: 6}  # kernel id -> column of its time
+    overrides = 0
+    for px, cin, cout, kern, *ms in rows:
+        # a square plane with that many stored pixels at one of the tuned batches
+        shape = None
+        for b in (256, 64, 16):
+            if px % b:
+                continue
+            for hw in (7, 14, 28, 56, 112, 33, 65, 129, 257):
+                if (hw * hw + 1) // 2 * 2 == px // b:
+                    shape = (b, hw)
+        assert shape, (px, cin, cout)
+        spec = wl.single_pointwise(shape[0], shape[1], cin, cout)
+        pick = {}
+        for mode in (api.GI_PW_AUTO, api.GI_PW_RULE):
+            g, _ = api.graph_from_spec(spec, api.GI_F16, io_layout=api.GI_PHWC4)
+            pick[mode] = g.compile(pointwise=mode).ops()[0].kernel
+        assert pick[api.GI_PW_AUTO] == kern, (px, cin, cout)
+        if pick[api.GI_PW_RULE] != kern:
+            overrides += 1
+            row = (px, cin, cout, kern) + tuple(ms)
+            t_table, t_rule = row[col[kern]], row[col[pick[api.GI_PW_RULE]]]
+            assert t_table > 0 and t_rule > 1.03 * t_table, (px, cin, cout, t_table, t_rule)
+    assert overrides <= len(rows) // 10  # the rule was distilled from these measurements: it rarely loses
+    # a shape that is not in the table takes the rule
+    spec = wl.single_pointwise(3, 10, 40, 72)
+    kernels = []
+    for mode in (api.GI_PW_AUTO, api.GI_PW_RULE):
+        g, _ = api.graph_from_spec(spec, api.GI_F16, io_layout=api.GI_PHWC4)
+        kernels.append(g.compile(pointwise=mode).ops()[0].kernel)
+    assert kernels[0] == kernels[1]
