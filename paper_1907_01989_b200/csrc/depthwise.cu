@@ -108,7 +108,12 @@ __device__ __forceinline__ Row widen(const uint2* u) {
 // needs are fetched with three loads and converted once (16 conversions for two outputs instead of 24), and
 // the pair is stored with one 16-byte store: the kernel is bound by the FMA pipe (packed FMAs, the fp16 ->
 // fp32 conversions and integer multiply-adds all issue there) as much as by HBM.
-template <int MODE, int ACT, bool TAIL, bool PACKED, bool PAIR>
+// PLANE (mode 0, PACKED, one column per thread; 14 or 7, else 0): the planes are PLANE x PLANE with one padding row and
+// column on every side, and a thread walks a whole column.  With the trip count and the row pitch known at compile
+// time the walk is straight-line code: the three running accumulators rotate without register moves, every address is
+// an immediate offset from one base and the tests for rows outside the plane disappear (measured in the kernel that
+// runs a whole inverted-residual block: 36 % less time in the same stencil).
+template <int MODE, int ACT, bool TAIL, bool PACKED, bool PAIR, int PLANE>
 __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __restrict__ in, const float* __restrict__ w,
                                                                 const float* __restrict__ bias, const __half* __restrict__ res,
                                                                 __half* __restrict__ out, const DwGeom g, const Epilogue ep) {
@@ -459,6 +464,53 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
           fma2(a0, 1);
           start2(a1);
         }
+      } else if (MODE == 0 && PACKED && PLANE > 0) {
+        const unsigned col = data + static_cast<unsigned>(x) * 8u;
+        const bool vl = x >= 1, vr = x + 1 < PLANE;
+        Acc acc[3];
+        acc[0] = bias_acc;
+#pragma unroll
+        for (int iy = 0; iy < PLANE; ++iy) {
+          // input row iy is kernel row 2 of output row iy - 1 (now complete), row 1 of output row iy, row 0 of iy + 1
+          uint2 u[3];
+          u[0] = make_uint2(0u, 0u);
+          u[2] = make_uint2(0u, 0u);
+          if (vl) u[0] = lds64(col + static_cast<unsigned>((iy * PLANE - 1) * 8));
+          u[1] = lds64(col + static_cast<unsigned>(iy * PLANE * 8));
+          if (vr) u[2] = lds64(col + static_cast<unsigned>((iy * PLANE + 1) * 8));
+          const Row r = widen(u);
+          if (iy >= 1) {
+            fma_row(acc[(iy + 2) % 3], r, wlo + 6, whi + 6);
+            emit(acc[(iy + 2) % 3]);
+          }
+          fma_row(acc[iy % 3], r, wlo + 3, whi + 3);
+          if (iy + 1 < PLANE) acc[(iy + 1) % 3] = fma_row_from(bias_acc, r, wlo, whi);
+        }
+        emit(acc[(PLANE - 1) % 3]);
+      } else if (MODE == 0 && !PACKED && PLANE == 28) {
+        // the same straight-line walk for 28-wide planes cut into bands of 14 output rows: the band's 16 input rows are
+        // staged with zero rows above the first and below the last row of the image, so every row is simply read
+        constexpr int kRowsOut = 14, kW = 28;
+        const unsigned col = data + static_cast<unsigned>(((ya - 1) * kW + x) * 8);
+        const bool vl = x >= 1, vr = x + 1 < kW;
+        Acc acc[3];
+#pragma unroll
+        for (int j = 0; j < kRowsOut + 2; ++j) {
+          // staged row j of the band is kernel row 2 of output row j - 2 (now complete), row 1 of j - 1, row 0 of j
+          uint2 u[3];
+          u[0] = make_uint2(0u, 0u);
+          u[2] = make_uint2(0u, 0u);
+          if (vl) u[0] = lds64(col + static_cast<unsigned>((j * kW - 1) * 8));
+          u[1] = lds64(col + static_cast<unsigned>(j * kW * 8));
+          if (vr) u[2] = lds64(col + static_cast<unsigned>((j * kW + 1) * 8));
+          const Row r = widen(u);
+          if (j >= 2) {
+            fma_row(acc[(j + 1) % 3], r, wlo + 6, whi + 6);
+            emit(acc[(j + 1) % 3]);
+          }
+          if (j >= 1 && j <= kRowsOut) fma_row(acc[(j + 2) % 3], r, wlo + 3, whi + 3);
+          if (j < kRowsOut) acc[j % 3] = fma_row_from(bias_acc, r, wlo, whi);
+        }
       } else if (MODE != 2) {
         // one pointer per tap column, walking down the staged rows; a column outside the image
         // stays on a zero pixel
@@ -686,18 +738,35 @@ static int depthwise_f16_impl(const LaunchRec& r, const Ptrs& p, void* stream, b
   const float* b = static_cast<const float*>(p.bias);
   const __half* res = static_cast<const __half*>(p.res);
   __half* out = static_cast<__half*>(p.out);
-  static bool attr_done_dev[kMaxDevices][3][3][2][2][2] = {};
-  bool(&attr_done)[3][3][2][2][2] = attr_done_dev[current_device_slot()];
+  static bool attr_done_dev[kMaxDevices][3][3][2][2][2][4] = {};
+  bool(&attr_done)[3][3][2][2][2][4] = attr_done_dev[current_device_slot()];
+  // small square planes, stride 1, one padding row / column on every side, a thread per whole column: straight-line stencil
+  const bool whole_plane = packed && mode == 0 && !pair && g.H == g.W && g.pt == 1 && g.pl == 1 && g.Ho == g.H && g.Wo == g.W;
+  // ... and 28-wide planes in bands of 14 rows per thread (staged with zero rows: not the one-copy mode)
+  const bool band28 = !packed && mode == 0 && !pair && g.W == 28 && g.Wo == 28 && g.Ho == g.H && g.H % 14 == 0 && g.tr == 14 && g.pt == 1 && g.pl == 1;
+  const int plane = whole_plane && g.H == 14 ? 14 : whole_plane && g.H == 7 ? 7 : band28 ? 28 : 0;
   const bool tail = r.ep.has_res || r.ep.act_post != GI_ACT_NONE;
-#define GI_DW_LAUNCH2(M, A, T, P, Q)                                                                                          \
+#define GI_DW_LAUNCH3(M, A, T, P, Q, PL, PLI)                                                                                 \
   do {                                                                                                                        \
-    if (!attr_done[M][A][T][P][Q]) {                                                                                          \
+    if (!attr_done[M][A][T][P][Q][PLI]) {                                                                                     \
       const cudaError_t e =                                                                                                   \
-          cudaFuncSetAttribute(depthwise_f16_kernel<M, A, T, P, Q>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);   \
+          cudaFuncSetAttribute(depthwise_f16_kernel<M, A, T, P, Q, PL>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem); \
       if (e != cudaSuccess) return static_cast<int>(e);                                                                       \
-      attr_done[M][A][T][P][Q] = true;                                                                                        \
+      attr_done[M][A][T][P][Q][PLI] = true;                                                                                   \
     }                                                                                                                         \
-    launch_pdl(depthwise_f16_kernel<M, A, T, P, Q>, static_cast<unsigned>(grid), threads, smem, st, in, w, b, res, out, g, r.ep); \
+    launch_pdl(depthwise_f16_kernel<M, A, T, P, Q, PL>, static_cast<unsigned>(grid), threads, smem, st, in, w, b, res, out, g, r.ep); \
+  } while (0)
+#define GI_DW_LAUNCH2(M, A, T, P, Q)                  \
+  do {                                                \
+    if (M == 0 && P == 1 && Q == 0 && plane == 14) {  \
+      GI_DW_LAUNCH3(0, A, T, 1, 0, 14, 1);            \
+    } else if (M == 0 && P == 1 && Q == 0 && plane == 7) { \
+      GI_DW_LAUNCH3(0, A, T, 1, 0, 7, 2);             \
+    } else if (M == 0 && P == 0 && Q == 0 && plane == 28) { \
+      GI_DW_LAUNCH3(0, A, T, 0, 0, 28, 3);            \
+    } else {                                          \
+      GI_DW_LAUNCH3(M, A, T, P, Q, 0, 0);             \
+    }                                                 \
   } while (0)
 #define GI_DW_LAUNCH(M, A, T, P)            \
   do {                                      \
@@ -740,6 +809,7 @@ static int depthwise_f16_impl(const LaunchRec& r, const Ptrs& p, void* stream, b
 #undef GI_DW_ACT
 #undef GI_DW_LAUNCH
 #undef GI_DW_LAUNCH2
+#undef GI_DW_LAUNCH3
   return static_cast<int>(cudaGetLastError());
 }
 
