@@ -439,6 +439,35 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
           *reinterpret_cast<uint4*>(op) = make_uint4(u0.x, u0.y, u1.x, u1.y);
           op += out_stride;
         };
+        if (PLANE == 112 || PLANE == 56) {
+          // sub-bands of exactly 14 output rows of a PLANE-wide image: the 16 staged rows as straight-line code (the
+          // accumulators rotate at compile time, the row offsets are immediates, columns outside the image are predicated)
+          constexpr int kRowsOut = 14;
+          Acc acc[3][2];
+#pragma unroll
+          for (int j = 0; j < kRowsOut + 2; ++j) {
+            uint4 m;
+            uint2 a = make_uint2(0u, 0u), d = make_uint2(0u, 0u);
+            if (vl) a = lds64(mid0 + static_cast<unsigned>(j * PLANE * 8 - 8));
+            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(m.x), "=r"(m.y), "=r"(m.z), "=r"(m.w) : "r"(mid0 + static_cast<unsigned>(j * PLANE * 8)));
+            if (vr) d = lds64(mid0 + static_cast<unsigned>(j * PLANE * 8 + 16));
+            plo[0] = __half22float2(*reinterpret_cast<const __half2*>(&a.x));
+            phi[0] = __half22float2(*reinterpret_cast<const __half2*>(&a.y));
+            plo[1] = __half22float2(*reinterpret_cast<const __half2*>(&m.x));
+            phi[1] = __half22float2(*reinterpret_cast<const __half2*>(&m.y));
+            plo[2] = __half22float2(*reinterpret_cast<const __half2*>(&m.z));
+            phi[2] = __half22float2(*reinterpret_cast<const __half2*>(&m.w));
+            plo[3] = __half22float2(*reinterpret_cast<const __half2*>(&d.x));
+            phi[3] = __half22float2(*reinterpret_cast<const __half2*>(&d.y));
+            if (j >= 2) {
+              fma2(acc[(j + 1) % 3], 2);
+              emit2(acc[(j + 1) % 3]);
+            }
+            if (j >= 1 && j <= kRowsOut) fma2(acc[(j + 2) % 3], 1);
+            if (j < kRowsOut) start2(acc[j % 3]);
+          }
+          continue;
+        }
         Acc a0[2], a1[2], a2[2];
         next4();
         start2(a0);
@@ -738,13 +767,15 @@ static int depthwise_f16_impl(const LaunchRec& r, const Ptrs& p, void* stream, b
   const float* b = static_cast<const float*>(p.bias);
   const __half* res = static_cast<const __half*>(p.res);
   __half* out = static_cast<__half*>(p.out);
-  static bool attr_done_dev[kMaxDevices][3][3][2][2][2][4] = {};
-  bool(&attr_done)[3][3][2][2][2][4] = attr_done_dev[current_device_slot()];
+  static bool attr_done_dev[kMaxDevices][3][3][2][2][2][6] = {};
+  bool(&attr_done)[3][3][2][2][2][6] = attr_done_dev[current_device_slot()];
   // small square planes, stride 1, one padding row / column on every side, a thread per whole column: straight-line stencil
   const bool whole_plane = packed && mode == 0 && !pair && g.H == g.W && g.pt == 1 && g.pl == 1 && g.Ho == g.H && g.Wo == g.W;
   // ... and 28-wide planes in bands of 14 rows per thread (staged with zero rows: not the one-copy mode)
   const bool band28 = !packed && mode == 0 && !pair && g.W == 28 && g.Wo == 28 && g.Ho == g.H && g.H % 14 == 0 && g.tr == 14 && g.pt == 1 && g.pl == 1;
-  const int plane = whole_plane && g.H == 14 ? 14 : whole_plane && g.H == 7 ? 7 : band28 ? 28 : 0;
+  // ... and the two-columns-per-thread mode on 112- and 56-wide planes whose sub-bands are exactly 14 rows
+  const bool pair14 = pair && mode == 0 && g.pt == 1 && g.tr == 14 && g.Ho % 14 == 0 && (g.W == 112 || g.W == 56);
+  const int plane = whole_plane && g.H == 14 ? 14 : whole_plane && g.H == 7 ? 7 : band28 ? 28 : pair14 ? g.W : 0;
   const bool tail = r.ep.has_res || r.ep.act_post != GI_ACT_NONE;
 #define GI_DW_LAUNCH3(M, A, T, P, Q, PL, PLI)                                                                                 \
   do {                                                                                                                        \
@@ -758,7 +789,11 @@ static int depthwise_f16_impl(const LaunchRec& r, const Ptrs& p, void* stream, b
   } while (0)
 #define GI_DW_LAUNCH2(M, A, T, P, Q)                  \
   do {                                                \
-    if (M == 0 && P == 1 && Q == 0 && plane == 14) {  \
+    if (M == 0 && P == 0 && Q == 1 && plane == 112) { \
+      GI_DW_LAUNCH3(0, A, T, 0, 1, 112, 4);           \
+    } else if (M == 0 && P == 0 && Q == 1 && plane == 56) { \
+      GI_DW_LAUNCH3(0, A, T, 0, 1, 56, 5);            \
+    } else if (M == 0 && P == 1 && Q == 0 && plane == 14) {  \
       GI_DW_LAUNCH3(0, A, T, 1, 0, 14, 1);            \
     } else if (M == 0 && P == 1 && Q == 0 && plane == 7) { \
       GI_DW_LAUNCH3(0, A, T, 1, 0, 7, 2);             \
