@@ -159,10 +159,8 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_mm_kernel(const MmParam
         tc_fence_after();
         for (int c = 0; c < p.n_chunks; ++c, ++it) {
           const unsigned stage = it % p.stages, phase = (it / p.stages) & 1u;
-          // the issuing thread's own instruction stream bounds the chunk rate: one barrier per stage for both operands,
-          // and a completed phase is recognised without the call into the bounded-wait routine
-          if (!mbar_try_wait(smem_u32(&hdr->full[stage]), phase) &&
-              !mbar_wait(smem_u32(&hdr->full[stage]), phase, abort_flag, p.timeout_ns, &g_mm_error, kErrMma)) {
+          // the issuing thread's own instruction stream bounds the chunk rate: one barrier per stage for both operands
+          if (!mbar_wait(smem_u32(&hdr->full[stage]), phase, abort_flag, p.timeout_ns, &g_mm_error, kErrMma)) {
             ok = false;
             break;
           }
@@ -200,8 +198,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_mm_kernel(const MmParam
       const unsigned px0 = static_cast<unsigned>(mt) * kRows + static_cast<unsigned>(tid);
       for (int c = 0; c < p.n_chunks; ++c, ++it) {
         const unsigned stage = it % p.stages, phase = (it / p.stages) & 1u;
-        if (!mbar_try_wait(smem_u32(&hdr->empty[stage]), phase ^ 1u) &&
-            !mbar_wait(smem_u32(&hdr->empty[stage]), phase ^ 1u, abort_flag, p.timeout_ns, &g_mm_error, kErrLoad)) {
+        if (!mbar_wait(smem_u32(&hdr->empty[stage]), phase ^ 1u, abort_flag, p.timeout_ns, &g_mm_error, kErrLoad)) {
           ok = false;
           break;
         }
