@@ -302,6 +302,15 @@ GI_API gi_status gi_run_timed(gi_exec* e, const void* const* dev_inputs, void* c
  * the word from the current device. */
 GI_API gi_status gi_device_status(uint32_t* flags);
 
+/* Self-test of the give-up path of the device-side waits.  Launches one warp that waits, with the library's own
+ * bounded-wait routine and a limit of `limit_us` microseconds (1 .. 100000), on a barrier that nothing ever
+ * completes; the wait must run out, raise the kernel's abort flag and error bit, and the kernel must return
+ * normally.  Synchronises `stream`.  *waited_us receives how long the wait lasted on the device, *gave_up 1 if it
+ * ended by running out (0 would mean the barrier completed, which cannot happen).  The error bit it sets lives in a
+ * word of its own: gi_device_status() is not affected and the CUDA context stays usable.  (The paper has no
+ * counterpart; its engine has no device-side waits.) */
+GI_API gi_status gi_selftest_bounded_wait(uint32_t limit_us, uint32_t* waited_us, int32_t* gave_up, void* stream);
+
 GI_API void gi_exec_destroy(gi_exec* e);
 
 /* ---- helpers ---- */

@@ -70,7 +70,7 @@ class gi_op_info(C.Structure):
 
 
 EXPORTS = ["gi_graph_create", "gi_graph_input", "gi_add_op", "gi_graph_output", "gi_graph_destroy", "gi_compile",
-           "gi_exec_query", "gi_exec_tensor", "gi_exec_op", "gi_exec_bind", "gi_run", "gi_run_static", "gi_run_timed", "gi_device_status", "gi_exec_destroy",
+           "gi_exec_query", "gi_exec_tensor", "gi_exec_op", "gi_exec_bind", "gi_run", "gi_run_static", "gi_run_timed", "gi_device_status", "gi_selftest_bounded_wait", "gi_exec_destroy",
            "gi_status_str", "gi_last_error", "gi_tensor_bytes", "gi_f32_to_f16"]
 
 _lib = None
@@ -109,6 +109,8 @@ def lib() -> C.CDLL:
     L.gi_run_timed.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp, C.c_size_t, vp, C.POINTER(C.c_float), C.c_int32]
     L.gi_device_status.argtypes = [C.POINTER(C.c_uint32)]
     L.gi_device_status.restype = C.c_int32
+    L.gi_selftest_bounded_wait.argtypes = [C.c_uint32, C.POINTER(C.c_uint32), C.POINTER(C.c_int32), vp]
+    L.gi_selftest_bounded_wait.restype = C.c_int32
     L.gi_exec_destroy.argtypes = [vp]
     L.gi_exec_destroy.restype = None
     L.gi_status_str.argtypes = [C.c_int32]
@@ -147,6 +149,13 @@ def gi_device_status() -> int:
     flags = C.c_uint32(0)
     _check(lib().gi_device_status(C.byref(flags)), "gi_device_status")
     return int(flags.value)
+
+
+def gi_selftest_bounded_wait(limit_us: int, stream=None):
+    """-> (microseconds the wait lasted on the device, True if it ended by running out)."""
+    waited, gave_up = C.c_uint32(0), C.c_int32(0)
+    _check(lib().gi_selftest_bounded_wait(limit_us, C.byref(waited), C.byref(gave_up), _stream_ptr(stream)), "gi_selftest_bounded_wait")
+    return int(waited.value), bool(gave_up.value)
 
 
 class Graph:

@@ -9,6 +9,7 @@
 
 #include "gi_internal.h"
 #include "kernels.h"
+#include "sm100_ptx.cuh"
 
 namespace gi {
 
@@ -174,6 +175,58 @@ gi_status gi_run_static(gi_exec* e, const void* const* dev_inputs, void* const* 
     arena = g_static_ptr[dev];
   }
   return run_impl(e, dev_inputs, dev_outputs, arena, GI_STATIC_ARENA_BYTES, stream, nullptr);
+}
+
+// ---------------------------------------------------------------- self-test of the bounded wait
+namespace {
+__device__ unsigned int g_selftest_error = 0;
+__global__ void bounded_wait_selftest_kernel(unsigned timeout_ns, unsigned long long* result) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ unsigned abort_flag;
+  if (threadIdx.x == 0) {
+    gi::ptx::mbar_init(gi::ptx::smem_u32(&bar), 1);  // one arrival expected; nobody arrives
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  const unsigned long long t0 = gi::ptx::global_timer_ns();
+  // the whole warp waits, as the drain warps of the tensor-core kernels do; one lane's limit ends it for all
+  const bool ok = gi::ptx::mbar_wait_warp(gi::ptx::smem_u32(&bar), 0u, &abort_flag, timeout_ns, &g_selftest_error, 1u);
+  const unsigned long long t1 = gi::ptx::global_timer_ns();
+  if (threadIdx.x == 0) {
+    result[0] = t1 - t0;
+    result[1] = ok ? 0ull : 1ull;
+    result[2] = abort_flag;
+    result[3] = g_selftest_error;
+  }
+}
+}  // namespace
+
+gi_status gi_selftest_bounded_wait(uint32_t limit_us, uint32_t* waited_us, int32_t* gave_up, void* stream) {
+  if (!waited_us || !gave_up) return fail(GI_E_INVALID, "gi_selftest_bounded_wait: null argument");
+  if (limit_us < 1 || limit_us > 100000) return fail(GI_E_INVALID, "gi_selftest_bounded_wait: limit_us must be 1 .. 100000");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // pinned, device-visible host memory for the four result words: the library allocates no device memory
+  unsigned long long* host = nullptr;
+  cudaError_t err = cudaHostAlloc(reinterpret_cast<void**>(&host), 4 * sizeof(unsigned long long), cudaHostAllocMapped);
+  if (err != cudaSuccess) return fail(GI_E_CUDA, std::string("gi_selftest_bounded_wait: ") + cudaGetErrorString(err));
+  for (int i = 0; i < 4; ++i) host[i] = ~0ull;
+  unsigned long long* dev = nullptr;
+  err = cudaHostGetDevicePointer(reinterpret_cast<void**>(&dev), host, 0);
+  if (err == cudaSuccess) {
+    bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(limit_us * 1000u, dev);
+    err = cudaGetLastError();
+  }
+  if (err == cudaSuccess) err = cudaStreamSynchronize(st);
+  gi_status status = GI_OK;
+  if (err != cudaSuccess) {
+    status = fail(GI_E_CUDA, std::string("gi_selftest_bounded_wait: ") + cudaGetErrorString(err));
+  } else {
+    *waited_us = static_cast<uint32_t>(host[0] / 1000ull);
+    *gave_up = (host[1] == 1ull && host[2] == 1ull && (host[3] & 1ull)) ? 1 : 0;
+  }
+  cudaFreeHost(host);
+  return status;
 }
 
 gi_status gi_run_timed(gi_exec* e, const void* const* dev_inputs, void* const* dev_outputs, void* dev_arena,

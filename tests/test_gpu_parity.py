@@ -801,3 +801,21 @@ def test_mobilenet_v2_batch32_blocks_as_one_kernel_every_tensor():
             continue
         assert_close(outs[t] if t in outs else run.fetch(t), r, api.GI_F16, f"tensor {t}")
     assert api.gi_device_status() == 0
+
+
+# ---------------------------------------------------------------------- the give-up path of the device-side waits
+def test_bounded_wait_runs_out_and_the_context_survives():
+    """Every wait in the kernels is bounded; here one is made to run out on purpose and safely: a warp waits on a
+    barrier that nothing completes, with a limit of a few milliseconds.  The wait must end by its limit (not hang,
+    not trap), report it, and leave the context healthy: a real inference afterwards still matches the oracle and the
+    kernels' own status word stays clean."""
+    waited_us, gave_up = api.gi_selftest_bounded_wait(3000)
+    assert gave_up
+    assert 2500 <= waited_us <= 50000, waited_us
+    waited_us, gave_up = api.gi_selftest_bounded_wait(200)
+    assert gave_up and 100 <= waited_us <= 20000, waited_us
+    with pytest.raises(api.GiError):
+        api.gi_selftest_bounded_wait(0)
+    assert api.gi_device_status() == 0
+    check_outputs(wl.separable_block(2), api.GI_F16)
+    assert api.gi_device_status() == 0
