@@ -100,17 +100,20 @@ enum {
                           the paper's work-group table, Section 4) is not consulted */
 };
 
-/* Cross-operator kernels: a depthwise 3x3 convolution whose only consumer is a 1x1 convolution runs
- * with it as one kernel, so the tensor between them never reaches memory (fp16 storage; the "Shader Program
- * Optimization" paragraph of Section 3.2 folds element-wise operators into their producer, this folds a whole operator).  Results are
- * those of the two operators run one after the other: the tensor between them is still rounded to
- * fp16.  The memory plan is not affected: the tensor keeps its place in the arena, unused; a pair whose input
- * and output the planner placed on the same bytes (legal for two ops, not for one kernel) stays two kernels. */
+/* Cross-operator kernels (fp16 storage).  The "Shader Program Optimization" paragraph of Section 3.2 folds element-wise
+ * operators into their producer; these fold whole operators, so that the tensors between them never reach memory:
+ *   (1) an inverted-residual block - 1x1 expansion, depthwise 3x3 (stride 1 or 2), 1x1 projection, optional residual
+ *       add - on planes of at most 256 pixels with a multiple of 16 input channels runs as ONE kernel;
+ *   (2) a depthwise 3x3 convolution whose only consumer is a 1x1 convolution runs with it as one kernel.
+ * Results are those of the operators run one after the other: the tensors in between are still rounded to fp16.  The
+ * memory plan is not affected: those tensors keep their place in the arena, unused; operators whose input and output the
+ * planner placed on the same bytes (legal for separate kernels, not for one that reads while it writes) stay separate. */
 enum {
-  GI_XOP_AUTO = 0,  /* the library's choice: at present the same as GI_XOP_OFF, the single kernel has not measured
-                       faster than the two kernels on any layer of the benchmark networks (default) */
+  GI_XOP_AUTO = 0,  /* the library's choice, from whole-network measurements (default): (1) for blocks on planes of at most
+                       64 pixels (7x7) when the batch gives at least 96 work units; never (2), which has not measured
+                       faster than the two kernels on any layer of the benchmark networks */
   GI_XOP_OFF = 1,   /* one kernel per fused op */
-  GI_XOP_ON = 2     /* wherever the kernel supports the pair */
+  GI_XOP_ON = 2     /* (1) wherever the block kernel supports the three ops, else (2) wherever the pair kernel does */
 };
 
 /*

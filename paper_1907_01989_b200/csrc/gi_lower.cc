@@ -318,9 +318,9 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
           // tile per SM unless the input is 960 channels deep or more.
           // Whole inverted-residual block as one kernel.  The library's own choice (GI_XOP_AUTO) follows an A/B of
           // MobileNetV2 at batch 256 on one B200, both builds alternating in one call: with the two 7x7 blocks that
-          // qualify as one kernel each the step takes 1.619 ms against 1.626 ms; with the 14x14 blocks as well 1.668 ms
-          // (alone, L2 flushed, a 14x14 block takes 55-88 us as one kernel against 52-73 us as three; a 7x7 block
-          // 55-66 against 60).  So: planes of at most 64 pixels, and at least about one unit of work per SM - below
+          // qualify as one kernel each the step takes 1.549 ms against 1.552 ms; with the 14x14 blocks as well it is 2.5 %
+          // slower (alone, L2 flushed, a 14x14 block takes 55-88 us as one kernel against 48-65 us as three; a 7x7
+          // block 55-66 against 56).  So: planes of at most 64 pixels, and at least about one unit of work per SM - below
           // that (batch 1) three kernels that each spread over all SMs are faster.
           long long ir_units = 0;
           if (pointwise && tc && e->opt.fuse && e->opt.cross_op != GI_XOP_OFF && block_follows(g, e, i)) {
