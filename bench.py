@@ -45,7 +45,7 @@ import numpy as np  # noqa: E402
 NETS = {"v2": ("mobilenet_v2", "MobileNetV2-224"), "v1": ("mobilenet_v1", "MobileNetV1-224"),
         "seg": ("mobilenet_v2_segmentation", "MobileNetV2-513-OS16-seg"), "fire": ("fire_network", "fire-module-network-96")}
 PW_MODES = {"auto": 0, "simt": 1, "pair": 2, "lane": 3, "wide": 4, "rule": 5}
-XOP_MODES = {"auto": 0, "off": 1, "on": 2}
+XOP_MODES = {"auto": 0, "off": 1, "on": 2, "chain": 3}
 # dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes, from the ncu captures summarised
 # under profiles/ (depthwise: batch 128, 112x112x96, stride 1: 560.3 MB over 616.6 MB; pointwise_tc:
 # batch 64, 112x112, 16->96: 119.6 MB over 179.8 MB, the tail of the output still being in L2)
@@ -302,6 +302,10 @@ def run_sweep(args):
     elif args.sweep == "block":  # the inverted-residual blocks of MobileNetV2 on 14x14 and 7x7 planes
         points = [(256, 14, 64, 384, 64, 1), (256, 14, 64, 384, 96, 1), (256, 14, 96, 576, 96, 1), (256, 14, 96, 576, 160, 2),
                   (256, 7, 160, 960, 160, 1), (256, 7, 160, 960, 320, 1)]
+    elif args.sweep == "pair":  # the projection -> expansion seams of MobileNetV2 (B, HW, Cin, Cmid, Cout)
+        points = [(256, 112, 32, 16, 96), (256, 56, 96, 24, 144), (256, 56, 144, 24, 144), (256, 28, 144, 32, 192),
+                  (256, 28, 192, 32, 192), (256, 14, 192, 64, 384), (256, 14, 384, 64, 384), (256, 14, 384, 96, 576),
+                  (256, 14, 576, 96, 576), (256, 7, 576, 160, 960), (256, 7, 960, 160, 960)]
     elif args.sweep == "dw":
         points = [(b, hw, c, s) for b in (64, 256) for hw, c in ((112, 32), (112, 96), (56, 144), (28, 192), (14, 384),
                                                                  (14, 576), (7, 960)) for s in (1, 2)]
@@ -326,6 +330,10 @@ def run_sweep(args):
             b, hw, cin, hidden, cout, stride = pt
             spec = wl.inverted_residual_block(b, hw, hw, cin, hidden, cout, stride)
             name = f"block b{b} {hw}x{hw} {cin}->{hidden}->{cout} s{stride}"
+        elif args.sweep == "pair":
+            b, hw, cin, cmid, cout = pt
+            spec = wl.pointwise_pair(b, hw, hw, cin, cmid, cout, residual=args.residual)
+            name = f"pw1x1+pw1x1 b{b} {hw}x{hw} {cin}->{cmid}->{cout}"
         elif args.sweep == "dwpw":
             b, hw, c, cout, stride = pt
             spec = wl.depthwise_then_pointwise(b, hw, hw, c, cout, stride, residual=args.residual)
@@ -342,7 +350,7 @@ def run_sweep(args):
         ex = g.compile(pointwise=PW_MODES[args.pointwise], cross_op=XOP_MODES[args.cross_op])
         ex.bind(dev)
         ops = ex.ops()
-        assert len(ops) == {"dwpw": 2, "stem": 2, "block": 3}.get(args.sweep, 1)
+        assert len(ops) == {"dwpw": 2, "stem": 2, "block": 3, "pair": 2}.get(args.sweep, 1)
         # seeded images (the workload recipe), at most 8 distinct ones: image k of the batch is drawn image k % 8
         n_img = min(b, 8)
         xs_np = [wl.make_input(spec, images=list(range(n_img)), index=i) for i in range(len(spec.inputs))]
@@ -457,12 +465,12 @@ def main():
     ap.add_argument("--net", default="v2", choices=sorted(NETS))
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--pointwise", default="auto", choices=["auto", "simt", "pair", "lane", "wide", "rule"])
-    ap.add_argument("--cross-op", default="auto", choices=["auto", "off", "on"],
-                    help="depthwise + 1x1 convolution as one kernel: where the library chooses it, never, wherever supported")
+    ap.add_argument("--cross-op", default="auto", choices=["auto", "off", "on", "chain"],
+                    help="cross-operator kernels: the library's choice, none, blocks and depthwise + 1x1 pairs wherever supported, 1x1 -> 1x1 pairs wherever supported")
     ap.add_argument("--per-op", default=None, help="write the per-op timing table to this file")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-batch1", action="store_true", help="skip the batch-1 latency leg (keeps profiler runs short)")
-    ap.add_argument("--sweep", default=None, choices=["pw", "dw", "conv3", "dwpw", "stem", "block"],
+    ap.add_argument("--sweep", default=None, choices=["pw", "dw", "conv3", "dwpw", "stem", "block", "pair"],
                     help="time single fused operators instead of a network")
     ap.add_argument("--points", default=None, help="sweep points 'B,HW,Cin,Cout;...' (pw), 'B,HW,C,stride;...' (dw), "
                     "'B,HW,Cin,Cout,stride;...' (conv3), 'B,HW,C,Cout,stride;...' (dwpw: depthwise then 1x1, see --cross-op), "

@@ -104,7 +104,9 @@ enum {
  * operators into their producer; these fold whole operators, so that the tensors between them never reach memory:
  *   (1) an inverted-residual block - 1x1 expansion, depthwise 3x3 (stride 1 or 2), 1x1 projection, optional residual
  *       add - on planes of at most 256 pixels with a multiple of 16 input channels runs as ONE kernel;
- *   (2) a depthwise 3x3 convolution whose only consumer is a 1x1 convolution runs with it as one kernel.
+ *   (2) a depthwise 3x3 convolution whose only consumer is a 1x1 convolution runs with it as one kernel;
+ *   (3) two consecutive 1x1 convolutions - a block's projection and the next block's expansion - run as one kernel
+ *       that stores both outputs and never reads the tensor between them back.
  * Results are those of the operators run one after the other: the tensors in between are still rounded to fp16.  The
  * memory plan is not affected: those tensors keep their place in the arena, unused; operators whose input and output the
  * planner placed on the same bytes (legal for separate kernels, not for one that reads while it writes) stay separate. */
@@ -113,7 +115,8 @@ enum {
                        64 pixels (7x7) when the batch gives at least 96 work units; never (2), which has not measured
                        faster than the two kernels on any layer of the benchmark networks */
   GI_XOP_OFF = 1,   /* one kernel per fused op */
-  GI_XOP_ON = 2     /* (1) wherever the block kernel supports the three ops, else (2) wherever the pair kernel does */
+  GI_XOP_ON = 2,    /* (1) wherever the block kernel supports the three ops, else (2) wherever the pair kernel does */
+  GI_XOP_CHAIN = 3  /* (3) wherever that kernel supports the two ops; neither (1) nor (2) */
 };
 
 /*
@@ -197,7 +200,8 @@ enum {
   GI_KERNEL_CONCAT = 13,
   GI_KERNEL_CONV_TC = 14,             /* k x k convolution, any number of input channels, on the tensor cores */
   GI_KERNEL_INVERTED_RESIDUAL = 15,   /* this op (1x1 expansion) and the next two (depthwise 3x3, 1x1 projection) as one kernel */
-  GI_KERNEL_POINTWISE_MM = 16         /* 1x1 convolution, wide tiles for tensor-bound shapes */
+  GI_KERNEL_POINTWISE_MM = 16,        /* 1x1 convolution, wide tiles for tensor-bound shapes */
+  GI_KERNEL_POINTWISE_CHAIN = 17      /* this op (1x1) and the next one (1x1) as one kernel; both outputs are stored */
 };
 
 /* ---- graph construction (Section 3.1, "Initialization": the sub-graph given to the GPU backend) ---- */

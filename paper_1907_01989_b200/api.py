@@ -27,10 +27,10 @@ GI_EXEC_PACK, GI_EXEC_UNPACK = 100, 101
 GI_ACT_NONE, GI_ACT_RELU, GI_ACT_RELU6 = 0, 1, 2
 GI_PLAN_GREEDY_BY_SIZE, GI_PLAN_GREEDY_SHARED_OBJECTS, GI_PLAN_NAIVE, GI_PLAN_MIN_COST_FLOW = 0, 1, 2, 3
 GI_PW_AUTO, GI_PW_SIMT, GI_PW_TC_PAIR, GI_PW_TC_LANE, GI_PW_TC_WIDE, GI_PW_RULE = 0, 1, 2, 3, 4, 5
-GI_XOP_AUTO, GI_XOP_OFF, GI_XOP_ON = 0, 1, 2
+GI_XOP_AUTO, GI_XOP_OFF, GI_XOP_ON, GI_XOP_CHAIN = 0, 1, 2, 3
 GI_STATIC_ARENA_BYTES = 16 << 20
 KERNEL_NAMES = {1: "pack", 2: "unpack", 3: "conv_simt", 4: "pointwise_tc", 5: "depthwise", 6: "eltwise", 7: "pool",
-                8: "resize", 9: "conv3x3_tc", 10: "pointwise_ts", 11: "depthwise_pointwise", 12: "none", 13: "concat", 14: "conv_tc", 15: "inverted_residual", 16: "pointwise_mm"}
+                8: "resize", 9: "conv3x3_tc", 10: "pointwise_ts", 11: "depthwise_pointwise", 12: "none", 13: "concat", 14: "conv_tc", 15: "inverted_residual", 16: "pointwise_mm", 17: "pointwise_chain"}
 
 _KIND = {wl.CONV2D: GI_OP_CONV2D, wl.DEPTHWISE: GI_OP_DEPTHWISE_CONV2D, wl.ADD: GI_OP_ADD,
          wl.ACTIVATION: GI_OP_ACTIVATION, wl.GLOBAL_AVG_POOL: GI_OP_GLOBAL_AVG_POOL,

@@ -8,7 +8,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgi.so")
 SOURCES = ["gi_graph.cc", "gi_compile.cc", "gi_lower.cc", "gi_run.cu", "kernels_simt.cu", "pointwise_tc.cu", "depthwise.cu", "conv3x3_tc.cu",
-           "pointwise_ts.cu", "depthwise_pointwise.cu", "conv_tc.cu", "inverted_residual.cu", "pointwise_mm.cu"]
+           "pointwise_ts.cu", "depthwise_pointwise.cu", "conv_tc.cu", "inverted_residual.cu", "pointwise_mm.cu", "pointwise_chain.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "--use_fast_math=false",
               "-Xcompiler", "-fPIC,-O2,-Wall,-fvisibility=hidden", "-cudart", "static"]
 

@@ -463,7 +463,7 @@ gi_status gi_compile(const gi_graph* g, const gi_compile_options* opt, gi_exec**
   }
   if (o.align < 256 || (o.align & (o.align - 1))) return fail(GI_E_INVALID, "gi_compile: align must be a power of two >= 256");
   if (o.pointwise < GI_PW_AUTO || o.pointwise > GI_PW_RULE) return fail(GI_E_INVALID, "gi_compile: unknown pointwise option");
-  if (o.cross_op < GI_XOP_AUTO || o.cross_op > GI_XOP_ON) return fail(GI_E_INVALID, "gi_compile: unknown cross_op option");
+  if (o.cross_op < GI_XOP_AUTO || o.cross_op > GI_XOP_CHAIN) return fail(GI_E_INVALID, "gi_compile: unknown cross_op option");
   gi_exec* e = nullptr;
   try {
     e = new gi_exec();

@@ -82,6 +82,9 @@ struct LaunchRec {
   // `ep2` the projection's; Cmid the hidden channels; the stride / pads are the depthwise op's, (Ho, Wo) its output
   int Cmid = 0;
   Epilogue ep_mid;
+  // two consecutive 1x1 convolutions as one kernel: `out` / `res` / `ep` / `wts` are the first one's (Cmid its output
+  // channels), `out2` / `ep2` / `wts2` / Co2 the second one's; `bias` holds both bias vectors
+  Loc out2;
 };
 
 struct FusedOp {

@@ -179,6 +179,30 @@ static bool block_follows(const gi_graph& g, const gi_exec* e, size_t i) {
   return true;
 }
 
+// Two tensors that both live in the arena and share at least one byte.
+static bool arena_overlap(const gi_exec* e, int t1, int t2) {
+  if (t1 < 0 || t2 < 0) return false;
+  const Loc a = loc_of(e, t1), b = loc_of(e, t2);
+  if (a.where != W_ARENA || b.where != W_ARENA) return false;
+  return a.offset < b.offset + e->plan[t2].bytes && b.offset < a.offset + e->plan[t1].bytes;
+}
+
+// Executed ops i and i + 1 are plain 1x1 convolutions, the second reads the first one's output and has neither a
+// residual nor a second activation: one kernel may run both, storing both outputs (the first output may have any
+// number of other readers).  As separate ops the first op's input and residual may die before the second op's output is
+// born, so the planner may have put that output on their bytes; one kernel reads them while it writes it - such a
+// pair stays two kernels.
+static bool chain_follows(const gi_graph& g, const gi_exec* e, size_t i) {
+  if (i + 1 >= e->ops.size()) return false;
+  const FusedOp& a = e->ops[i];
+  const FusedOp& b = e->ops[i + 1];
+  if (a.kind != GI_OP_CONV2D || b.kind != GI_OP_CONV2D || a.out < 0 || b.out < 0) return false;
+  if (b.in0 != a.out || b.residual >= 0 || b.act_post != GI_ACT_NONE) return false;
+  if (!is_plain_pointwise(g.ops[a.graph_op].d) || !is_plain_pointwise(g.ops[b.graph_op].d)) return false;
+  if (arena_overlap(e, a.in0, b.out) || arena_overlap(e, a.residual, b.out)) return false;
+  return true;
+}
+
 // The executed op that converts graph input `t` from NHWC, if executed op `reader` is the only op that reads
 // the converted tensor (and it is not also a graph output); else -1.
 static int nhwc_pack_feeding_only(const gi_exec* e, int t, size_t reader) {
@@ -360,6 +384,35 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
               e->op_info.push_back(info);
               continue;
             }
+          }
+          // Projection + the next block's expansion as one kernel (the expansion must not be the start of a block that
+          // runs as one kernel itself).
+          // GI_XOP_AUTO takes it where it measured faster inside MobileNetV2 at batch 256 than the two kernels: 14x14
+          // planes with at most 64 channels in the middle and at least two tiles per SM.
+          const long long pc_tiles = (m_px_all_for_mm(e, din) + 127) / 128;
+          const bool chain_auto = din->h * din->w > 64 && din->h * din->w <= 256 && op.d.cout <= 64 && din->c >= 192 && pc_tiles >= 2 * 148;
+          if (pointwise && tc && e->opt.fuse && (e->opt.cross_op == GI_XOP_CHAIN || (e->opt.cross_op == GI_XOP_AUTO && chain_auto)) &&
+              chain_follows(g, e, i) &&
+              pointwise_chain_supported(din->c, op.d.cout, g.ops[e->ops[i + 1].graph_op].d.cout, f.residual >= 0)) {
+            const FusedOp& fb = e->ops[i + 1];
+            const OpNode& nb = g.ops[fb.graph_op];
+            const TensorDesc& d2 = e->tensors[fb.out];
+            r.kernel = GI_KERNEL_POINTWISE_CHAIN;
+            r.Cmid = op.d.cout;
+            r.Co2 = nb.d.cout;
+            r.ep2.act_pre = fb.act_pre;
+            r.out2 = loc_of(e, fb.out);
+            pointwise_chain_pack(op.weights.data(), op.bias.data(), nb.weights.data(), nb.bias.data(), din->c, op.d.cout, nb.d.cout,
+                                 &e->weight_blob, &r);
+            const uint64_t c42 = slices(d2.c) * 4;
+            info.bytes = (in_px * in_c4 + out_px * out_c4 * (r.ep.has_res ? 2 : 1) + out_px * c42 +
+                          static_cast<uint64_t>(din->c) * op.d.cout + static_cast<uint64_t>(op.d.cout) * nb.d.cout) * eb;
+            info.flops = 2 * out_px * din->c * op.d.cout + 2 * out_px * op.d.cout * nb.d.cout;
+            absorbed = 1;
+            info.kernel = r.kernel;
+            e->launches.push_back(r);
+            e->op_info.push_back(info);
+            continue;
           }
           const long long m_px_all = static_cast<long long>(e->batch) * din->h * din->w;
           const bool one_wave = m_px_all <= 64LL * 128 || (m_px_all <= 148LL * 128 && din->c < 960);

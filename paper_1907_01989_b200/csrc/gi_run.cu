@@ -94,6 +94,7 @@ static gi_status run_impl(gi_exec* e, const void* const* dev_inputs, void* const
     p.bias = resolve(r.bias);
     p.wts2 = resolve(r.wts2);
     p.bias2 = resolve(r.bias2);
+    p.out2 = resolve(r.out2);
     int err = 0;
     switch (r.kernel) {
       case GI_KERNEL_PACK: err = launch_pack(r, p, e->storage, stream); break;
@@ -106,6 +107,7 @@ static gi_status run_impl(gi_exec* e, const void* const* dev_inputs, void* const
       case GI_KERNEL_DEPTHWISE_POINTWISE: err = launch_depthwise_pointwise(r, p, stream); break;
       case GI_KERNEL_INVERTED_RESIDUAL: err = launch_inverted_residual(r, p, stream); break;
       case GI_KERNEL_POINTWISE_MM: err = launch_pointwise_mm(r, p, stream); break;
+      case GI_KERNEL_POINTWISE_CHAIN: err = launch_pointwise_chain(r, p, &e->tc_state, static_cast<int>(i), stream); break;
       case GI_KERNEL_NONE: break;  // computed by the previous launch
       case GI_KERNEL_ELTWISE:
         if (r.ep.has_res && !p.in1) p.in1 = p.res;
@@ -137,6 +139,7 @@ gi_status gi_device_status(uint32_t* flags) {
   if (err == 0) *flags |= depthwise_pointwise_error_word(&err) << 28;
   if (err == 0) *flags |= inverted_residual_error_word(&err) << 4;
   if (err == 0) *flags |= pointwise_mm_error_word(&err) << 8;
+  if (err == 0) *flags |= pointwise_chain_error_word(&err) << 12;
   if (err != 0) return fail(GI_E_CUDA, std::string("gi_device_status: ") + cudaGetErrorString(static_cast<cudaError_t>(err)));
   return GI_OK;
 }
@@ -258,9 +261,10 @@ namespace gi {
 int pointwise_ts_trace(unsigned long long* dst, int n);
 int depthwise_pointwise_trace(unsigned long long* dst, int n);
 int inverted_residual_trace(unsigned long long* dst, int n);
+int pointwise_chain_trace(unsigned long long* dst, int n);
 }
 // debug builds only: copy the timeline table of the lane-per-pixel kernel's last launch
 extern "C" GI_API int gi_debug_trace(int which, unsigned long long* dst, int n) {
-  return which == 2 ? gi::inverted_residual_trace(dst, n) : which == 1 ? gi::depthwise_pointwise_trace(dst, n) : gi::pointwise_ts_trace(dst, n);
+  return which == 3 ? gi::pointwise_chain_trace(dst, n) : which == 2 ? gi::inverted_residual_trace(dst, n) : which == 1 ? gi::depthwise_pointwise_trace(dst, n) : gi::pointwise_ts_trace(dst, n);
 }
 #endif

@@ -24,6 +24,7 @@ struct Ptrs {
   const void* bias = nullptr;
   const void* wts2 = nullptr;   // second operator of a two-operator kernel
   const void* bias2 = nullptr;
+  void* out2 = nullptr;         // second output of a kernel that stores two tensors
 };
 
 int launch_pack(const LaunchRec& r, const Ptrs& p, int storage, void* stream);
@@ -82,6 +83,14 @@ bool pointwise_mm_supported(int cin, int cout);
 void pointwise_mm_pack(const float* w, const float* bias, int cin, int cout, std::vector<uint8_t>* blob, LaunchRec* r);
 int launch_pointwise_mm(const LaunchRec& r, const Ptrs& p, void* stream);
 unsigned int pointwise_mm_error_word(int* cuda_err);
+
+// Two consecutive 1x1 convolutions (a block's projection and the next block's expansion) as one kernel (fp16 storage):
+// both outputs are stored, the tensor between them is not read back (pointwise_chain.cu)
+bool pointwise_chain_supported(int cin, int cmid, int cout, bool has_res);
+void pointwise_chain_pack(const float* w1, const float* b1, const float* w2, const float* b2, int cin, int cmid, int cout,
+                          std::vector<uint8_t>* blob, LaunchRec* r);
+int launch_pointwise_chain(const LaunchRec& r, const Ptrs& p, void** state, int launch_index, void* stream);
+unsigned int pointwise_chain_error_word(int* cuda_err);
 
 // One inverted-residual block (1x1 expansion -> depthwise 3x3 -> 1x1 projection, + residual) as one kernel (fp16
 // storage, planes of at most 256 pixels): neither hidden tensor leaves the SM.  `units` receives the kernel's parallelism.

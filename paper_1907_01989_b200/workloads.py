@@ -348,6 +348,26 @@ def inverted_residual_block(batch: int, h: int, w: int, cin: int, hidden: int, c
     return b.finish()
 
 
+def pointwise_pair(batch: int, h: int, w: int, cin: int, cmid: int, cout: int, residual: bool = True,
+                   mid_act: str = ACT_NONE, act: str = ACT_RELU6) -> GraphSpec:
+    """The seam between two inverted-residual blocks on its own: the linear 1x1 projection of one block (plus the
+    residual sum, the residual being a second graph input) followed by the 1x1 expansion + activation of the next.
+    Both tensors are graph outputs: the narrow one is what the next block's residual sum would read."""
+    b = GraphBuilder(f"pair_{batch}x{h}x{w}_{cin}_{cmid}_{cout}_{int(residual)}", batch, 15)
+    x = b.input(h, w, cin)
+    y = b.conv2d(x, cmid, 1)
+    if mid_act != ACT_NONE:
+        y = b.activation(y, mid_act)
+    if residual:
+        y = b.add(b.input(h, w, cmid), y)
+    z = b.conv2d(y, cout, 1)
+    if act != ACT_NONE:
+        z = b.activation(z, act)
+    b.output(y)
+    b.output(z)
+    return b.finish()
+
+
 # ----------------------------------------------------------------------------------------
 # Workload 10: a network of "fire" modules - squeeze 1x1, then a 1x1 and a 3x3 expansion whose outputs are
 # concatenated - with a 2x2 stride-2 stem and a 3x3 stride-3 reduction: the operators and the kernel sizes /

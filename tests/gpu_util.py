@@ -32,9 +32,15 @@ class DeviceRun:
         self.spec, self.storage = spec, storage
         self.graph, _ = api.graph_from_spec(spec, storage)
         self.ex = self.graph.compile(planner=planner, fuse=fuse, pointwise=pointwise, cross_op=cross_op)
-        # tensors that stay on chip: the input of an op that runs inside the previous op's kernel
-        self.on_chip = {o.inputs[0] for o in self.ex.ops() if api.KERNEL_NAMES[o.kernel] == "none" and
-                        o.kind in (api.GI_OP_CONV2D, api.GI_OP_DEPTHWISE_CONV2D)}
+        # tensors that stay on chip: the input of an op that runs inside the previous op's kernel (the kernel that runs
+        # two 1x1 convolutions stores the tensor between them as well, so there it is compared like any other)
+        self.on_chip, launcher = set(), None
+        for o in self.ex.ops():
+            name = api.KERNEL_NAMES[o.kernel]
+            if name != "none":
+                launcher = name
+            elif o.kind in (api.GI_OP_CONV2D, api.GI_OP_DEPTHWISE_CONV2D) and launcher != "pointwise_chain":
+                self.on_chip.add(o.inputs[0])
         # ... and the converted copy of an NHWC input that the first convolution reads in the caller's layout itself
         self.on_chip |= {o.output for o in self.ex.ops() if api.KERNEL_NAMES[o.kernel] == "none" and o.kind == api.GI_EXEC_PACK}
         dev = "cuda:0"

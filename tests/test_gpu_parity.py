@@ -803,6 +803,69 @@ def test_mobilenet_v2_batch32_blocks_as_one_kernel_every_tensor():
     assert api.gi_device_status() == 0
 
 
+# ---------------------------------------------------------------------- 1x1 -> 1x1 as one kernel
+# (batch, H, W, Cin, Cmid, Cout, residual): the projection -> expansion seams of MobileNetV2 (every plane size), a
+# middle width that is not a multiple of 16 (24, 20), one that is not a multiple of 4 (10), input widths that leave the
+# last 32-channel chunk ragged, odd planes, a single pixel, more tiles than one wave of SMs
+PC_CASES = [(3, 14, 14, 384, 64, 384, True), (2, 14, 14, 384, 96, 576, False), (2, 14, 14, 576, 96, 576, True),
+            (3, 7, 7, 576, 112, 672, False), (5, 7, 7, 960, 80, 480, True), (2, 28, 28, 192, 32, 192, True),
+            (2, 28, 28, 144, 32, 192, False), (1, 56, 56, 144, 24, 144, True), (1, 56, 56, 96, 24, 144, False),
+            (1, 112, 112, 32, 16, 96, False), (3, 9, 5, 40, 20, 70, True), (2, 3, 3, 17, 10, 33, True), (4, 1, 1, 64, 16, 64, False),
+            (40, 28, 28, 48, 16, 48, True), (2, 6, 6, 100, 112, 130, False)]
+
+
+@pytest.mark.parametrize("case", PC_CASES, ids=lambda c: "b%d_%dx%d_%d_%d_%d_r%d" % c)
+def test_pointwise_pair_one_kernel(case):
+    b, h, w, cin, cmid, cout, residual = case
+    spec = wl.pointwise_pair(b, h, w, cin, cmid, cout, residual)
+    # every tensor its own memory: under a sharing plan the second output may lie on the first input's bytes, and the
+    # pair then stays two kernels (covered by the host tests)
+    run, xs, outs = check_outputs(spec, api.GI_F16, cross_op=api.GI_XOP_CHAIN, planner=api.GI_PLAN_NAIVE)
+    names = [api.KERNEL_NAMES[o.kernel] for o in run.ex.ops()]
+    assert names.count("pointwise_chain") == 1 and names.count("none") == 1, names
+    again = run.run(xs)
+    for t in spec.outputs:
+        assert np.array_equal(outs[t], again[t])
+    # the same two tensors from two kernels: identical bits (same products, same fp32 sums per output, same rounding)
+    two = DeviceRun(spec, api.GI_F16, cross_op=api.GI_XOP_OFF, planner=api.GI_PLAN_NAIVE).run(xs)
+    for t in spec.outputs:
+        assert_close(outs[t], two[t], api.GI_F16, f"{spec.name} output {t} against the two-kernel path")
+    assert api.gi_device_status() == 0
+
+
+def test_pointwise_pair_too_wide_for_one_kernel_stays_two():
+    """160 channels in the middle: the two weight rings, the operand tile and the residual strips no longer fit shared
+    memory together; the pair must fall back to two kernels and still be right."""
+    spec = wl.pointwise_pair(3, 7, 7, 960, 160, 960, True)
+    run, _, _ = check_outputs(spec, api.GI_F16, cross_op=api.GI_XOP_CHAIN, planner=api.GI_PLAN_NAIVE)
+    names = [api.KERNEL_NAMES[o.kernel] for o in run.ex.ops()]
+    assert "pointwise_chain" not in names and "none" not in names, names
+
+
+@pytest.mark.parametrize("mid_act,act", [(wl.ACT_RELU, wl.ACT_NONE), (wl.ACT_RELU6, wl.ACT_RELU), (wl.ACT_NONE, wl.ACT_RELU6)])
+def test_pointwise_pair_epilogues(mid_act, act):
+    spec = wl.pointwise_pair(3, 10, 10, 48, 32, 80, True, mid_act=mid_act, act=act)
+    run, _, _ = check_outputs(spec, api.GI_F16, cross_op=api.GI_XOP_CHAIN, planner=api.GI_PLAN_NAIVE)
+    assert "pointwise_chain" in [api.KERNEL_NAMES[o.kernel] for o in run.ex.ops()]
+
+
+def test_mobilenet_v2_seams_as_one_kernel_every_tensor():
+    """Every stored tensor of the network with each projection -> expansion seam as one kernel."""
+    spec = wl.mobilenet_v2(4, size=224)
+    xs = [wl.make_input(spec)]
+    ref = og.run(spec, xs, storage="f16", fused=True, keep_all=True)
+    run = DeviceRun(spec, api.GI_F16, planner=api.GI_PLAN_NAIVE, guard_bytes=4096, cross_op=api.GI_XOP_CHAIN)
+    names = [api.KERNEL_NAMES[o.kernel] for o in run.ex.ops()]
+    assert names.count("pointwise_chain") == 13, names  # all seams but the three with 160 channels in the middle
+    outs = run.run(xs)
+    assert run.guard_intact()
+    for t, r in ref.items():
+        if t in run.on_chip:
+            continue
+        assert_close(outs[t] if t in outs else run.fetch(t), r, api.GI_F16, f"tensor {t}")
+    assert api.gi_device_status() == 0
+
+
 # ---------------------------------------------------------------------- the give-up path of the device-side waits
 def test_bounded_wait_runs_out_and_the_context_survives():
     """Every wait in the kernels is bounded; here one is made to run out on purpose and safely: a warp waits on a

@@ -367,6 +367,60 @@ def test_cross_op_option():
         g.compile(cross_op=7)
 
 
+def test_pointwise_pair_option():
+    """Two consecutive 1x1 convolutions as one kernel: chosen at compile time, only where pattern, kernel and memory plan allow."""
+    def compiled(spec, storage=api.GI_F16, **kw):
+        return api.graph_from_spec(spec, storage)[0].compile(**kw)
+
+    def kernels(spec, storage=api.GI_F16, **kw):
+        return [api.KERNEL_NAMES[o.kernel] for o in compiled(spec, storage, **kw).ops()]
+
+    pair = wl.pointwise_pair(4, 14, 14, 384, 64, 384, True)
+    on = kernels(pair, cross_op=api.GI_XOP_CHAIN, planner=api.GI_PLAN_NAIVE)
+    assert on.count("pointwise_chain") == 1 and on.index("none") == on.index("pointwise_chain") + 1
+    assert "pointwise_chain" not in kernels(pair, cross_op=api.GI_XOP_OFF) and "pointwise_chain" not in kernels(pair, cross_op=api.GI_XOP_ON)
+    # fp32 storage, a second operator with a residual of its own, a strided second operator, too many channels in the middle
+    assert "pointwise_chain" not in kernels(pair, api.GI_F32, cross_op=api.GI_XOP_CHAIN, planner=api.GI_PLAN_NAIVE)
+    b = wl.GraphBuilder("pair_second_residual", 2, 15)
+    x = b.input(8, 8, 32)
+    y = b.conv2d(x, 32, 1)
+    b.output(b.add(x, b.conv2d(y, 32, 1)))
+    assert "pointwise_chain" not in kernels(b.finish(), cross_op=api.GI_XOP_CHAIN, planner=api.GI_PLAN_NAIVE)
+    b = wl.GraphBuilder("pair_strided", 2, 15)
+    b.output(b.conv2d(b.conv2d(b.input(8, 8, 32), 16, 1), 32, 1, 2))
+    assert "pointwise_chain" not in kernels(b.finish(), cross_op=api.GI_XOP_CHAIN, planner=api.GI_PLAN_NAIVE)
+    assert "pointwise_chain" not in kernels(wl.pointwise_pair(2, 7, 7, 960, 160, 960, True), cross_op=api.GI_XOP_CHAIN, planner=api.GI_PLAN_NAIVE)
+    # the plan is not affected
+    a, c = compiled(pair, cross_op=api.GI_XOP_OFF), compiled(pair, cross_op=api.GI_XOP_CHAIN)
+    assert a.info.arena_bytes == c.info.arena_bytes and a.info.n_ops == c.info.n_ops
+    # whole network: every projection -> expansion seam with at most 128 channels in the middle under the naive plan;
+    # under the sharing plans the second output may lie on the bytes of the first operator's input or residual (their
+    # lifetimes do not meet as separate ops): one kernel would read them while it writes it, so those stay two kernels
+    gv2 = api.graph_from_spec(wl.mobilenet_v2(256), api.GI_F16)[0]
+    assert [api.KERNEL_NAMES[o.kernel] for o in gv2.compile(cross_op=api.GI_XOP_CHAIN, planner=api.GI_PLAN_NAIVE).ops()].count("pointwise_chain") == 13
+    # (Algorithm 1 hands every hidden tensor the shared object its predecessor has just left: no seam qualifies there)
+    for planner, expect in ((api.GI_PLAN_GREEDY_BY_SIZE, 11), (api.GI_PLAN_GREEDY_SHARED_OBJECTS, 0), (api.GI_PLAN_MIN_COST_FLOW, 12)):
+        ex = gv2.compile(cross_op=api.GI_XOP_CHAIN, planner=planner)
+        ops = ex.ops()
+        n = 0
+        for i, o in enumerate(ops):
+            if api.KERNEL_NAMES[o.kernel] != "pointwise_chain":
+                continue
+            n += 1
+            tout = ex.tensor(ops[i + 1].output)
+            for t in (o.inputs[0], o.residual):
+                if t >= 0:
+                    tin = ex.tensor(t)
+                    assert tin.offset + tin.bytes <= tout.offset or tout.offset + tout.bytes <= tin.offset
+        assert n == expect
+    # the library's own choice at batch 256: the four seams on 14x14 planes with 64 channels in the middle (measured);
+    # none at batch 1 or 64, where the tiles would not fill the SMs twice
+    auto = [api.KERNEL_NAMES[o.kernel] for o in gv2.compile().ops()]
+    assert auto.count("pointwise_chain") == 4
+    for batch in (1, 64):
+        assert "pointwise_chain" not in kernels(wl.mobilenet_v2(batch))
+
+
 def test_identity_resize_removed_like_the_oracle():
     """Graph clean-up (Section 3.1): the library drops the same identity ops as the oracle; plan and op list agree."""
     for extra in (False, True):
