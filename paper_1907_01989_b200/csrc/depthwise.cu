@@ -108,7 +108,8 @@ __device__ __forceinline__ Row widen(const uint2* u) {
 // needs are fetched with three loads and converted once (16 conversions for two outputs instead of 24), and
 // the pair is stored with one 16-byte store: the kernel is bound by the FMA pipe (packed FMAs, the fp16 ->
 // fp32 conversions and integer multiply-adds all issue there) as much as by HBM.
-// PLANE (mode 0, PACKED, one column per thread; 14 or 7, else 0): the planes are PLANE x PLANE with one padding row and
+// PLANE (0 = none; mode 0: 14 / 7 whole packed planes, 28 in bands of 14 rows, 112 / 56 with PAIR in sub-bands of 14 rows; mode 1:
+// 112 / 56 / 28 wide planes in bands of 8 / 7 / 7 output rows).  For the packed case: the planes are PLANE x PLANE with one padding row and
 // column on every side, and a thread walks a whole column.  With the trip count and the row pitch known at compile
 // time the walk is straight-line code: the three running accumulators rotate without register moves, every address is
 // an immediate offset from one base and the tests for rows outside the plane disappear (measured in the kernel that
@@ -540,6 +541,35 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
           if (j >= 1 && j <= kRowsOut) fma_row(acc[(j + 2) % 3], r, wlo + 3, whi + 3);
           if (j < kRowsOut) acc[j % 3] = fma_row_from(bias_acc, r, wlo, whi);
         }
+      } else if (MODE == 1 && !PACKED && PLANE > 0) {
+        // stride 2 without padding above / left on PLANE-wide planes, bands of exactly kRowsOut output rows: the band's
+        // 2 * kRowsOut + 1 staged rows as straight-line code.  Window columns 2x and 2x + 1 are one aligned 16-byte
+        // load; column 2x + 2 lies outside the image only for the last output column.  An even staged row is kernel
+        // row 2 of the output row above it and row 0 of the one below; an odd one is kernel row 1.
+        constexpr int kRowsOut = PLANE == 112 ? 8 : 7, kW = PLANE;
+        const unsigned col = data + static_cast<unsigned>((2 * ya * kW + 2 * x) * 8);
+        const bool vr = 2 * x + 2 < kW;
+        Acc cur = bias_acc;
+#pragma unroll
+        for (int j = 0; j <= 2 * kRowsOut; ++j) {
+          uint4 m;
+          uint2 u[3];
+          asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(m.x), "=r"(m.y), "=r"(m.z), "=r"(m.w) : "r"(col + static_cast<unsigned>(j * kW * 8)));
+          u[0] = make_uint2(m.x, m.y);
+          u[1] = make_uint2(m.z, m.w);
+          u[2] = make_uint2(0u, 0u);
+          if (vr) u[2] = lds64(col + static_cast<unsigned>((j * kW + 2) * 8));
+          const Row r = widen(u);
+          if (j & 1) {
+            fma_row(cur, r, wlo + 3, whi + 3);
+          } else {
+            if (j > 0) {
+              fma_row(cur, r, wlo + 6, whi + 6);
+              emit(cur);
+            }
+            if (j < 2 * kRowsOut) cur = fma_row_from(bias_acc, r, wlo, whi);
+          }
+        }
       } else if (MODE != 2) {
         // one pointer per tap column, walking down the staged rows; a column outside the image
         // stays on a zero pixel
@@ -767,15 +797,18 @@ static int depthwise_f16_impl(const LaunchRec& r, const Ptrs& p, void* stream, b
   const float* b = static_cast<const float*>(p.bias);
   const __half* res = static_cast<const __half*>(p.res);
   __half* out = static_cast<__half*>(p.out);
-  static bool attr_done_dev[kMaxDevices][3][3][2][2][2][6] = {};
-  bool(&attr_done)[3][3][2][2][2][6] = attr_done_dev[current_device_slot()];
+  static bool attr_done_dev[kMaxDevices][3][3][2][2][2][9] = {};
+  bool(&attr_done)[3][3][2][2][2][9] = attr_done_dev[current_device_slot()];
   // small square planes, stride 1, one padding row / column on every side, a thread per whole column: straight-line stencil
   const bool whole_plane = packed && mode == 0 && !pair && g.H == g.W && g.pt == 1 && g.pl == 1 && g.Ho == g.H && g.Wo == g.W;
   // ... and 28-wide planes in bands of 14 rows per thread (staged with zero rows: not the one-copy mode)
   const bool band28 = !packed && mode == 0 && !pair && g.W == 28 && g.Wo == 28 && g.Ho == g.H && g.H % 14 == 0 && g.tr == 14 && g.pt == 1 && g.pl == 1;
   // ... and the two-columns-per-thread mode on 112- and 56-wide planes whose sub-bands are exactly 14 rows
   const bool pair14 = pair && mode == 0 && g.pt == 1 && g.tr == 14 && g.Ho % 14 == 0 && (g.W == 112 || g.W == 56);
-  const int plane = whole_plane && g.H == 14 ? 14 : whole_plane && g.H == 7 ? 7 : band28 ? 28 : pair14 ? g.W : 0;
+  // ... and stride 2 without padding above / left on 112-, 56- and 28-wide planes whose bands are exactly 8 / 7 / 7 output rows
+  const bool down = !packed && mode == 1 && g.pt == 0 && g.pl == 0 && (g.W == 112 || g.W == 56 || g.W == 28) && g.Wo == g.W / 2 &&
+                    g.Ho == g.H / 2 && g.H % 2 == 0 && g.sub == 1 && g.tr == (g.W == 112 ? 8 : 7) && g.Ho % g.tr == 0;
+  const int plane = whole_plane && g.H == 14 ? 14 : whole_plane && g.H == 7 ? 7 : band28 ? 28 : pair14 ? g.W : down ? g.W : 0;
   const bool tail = r.ep.has_res || r.ep.act_post != GI_ACT_NONE;
 #define GI_DW_LAUNCH3(M, A, T, P, Q, PL, PLI)                                                                                 \
   do {                                                                                                                        \
@@ -799,6 +832,12 @@ static int depthwise_f16_impl(const LaunchRec& r, const Ptrs& p, void* stream, b
       GI_DW_LAUNCH3(0, A, T, 1, 0, 7, 2);             \
     } else if (M == 0 && P == 0 && Q == 0 && plane == 28) { \
       GI_DW_LAUNCH3(0, A, T, 0, 0, 28, 3);            \
+    } else if (M == 1 && P == 0 && Q == 0 && plane == 112) { \
+      GI_DW_LAUNCH3(1, A, T, 0, 0, 112, 6);           \
+    } else if (M == 1 && P == 0 && Q == 0 && plane == 56) { \
+      GI_DW_LAUNCH3(1, A, T, 0, 0, 56, 7);            \
+    } else if (M == 1 && P == 0 && Q == 0 && plane == 28) { \
+      GI_DW_LAUNCH3(1, A, T, 0, 0, 28, 8);            \
     } else {                                          \
       GI_DW_LAUNCH3(M, A, T, P, Q, 0, 0);             \
     }                                                 \
