@@ -109,7 +109,7 @@ __device__ __forceinline__ Row widen(const uint2* u) {
 // the pair is stored with one 16-byte store: the kernel is bound by the FMA pipe (packed FMAs, the fp16 ->
 // fp32 conversions and integer multiply-adds all issue there) as much as by HBM.
 // PLANE (0 = none; mode 0: 14 / 7 whole packed planes, 28 in bands of 14 rows, 112 / 56 with PAIR in sub-bands of 14 rows; mode 1:
-// 112 / 56 / 28 wide planes in bands of 8 / 7 / 7 output rows).  For the packed case: the planes are PLANE x PLANE with one padding row and
+// 112 / 56 / 28 wide planes in bands of 8 / 7 / 7 output rows, 14 whole packed planes).  For the packed case: the planes are PLANE x PLANE with one padding row and
 // column on every side, and a thread walks a whole column.  With the trip count and the row pitch known at compile
 // time the walk is straight-line code: the three running accumulators rotate without register moves, every address is
 // an immediate offset from one base and the tests for rows outside the plane disappear (measured in the kernel that
@@ -570,6 +570,34 @@ __global__ void __launch_bounds__(256, 2) depthwise_f16_kernel(const __half* __r
             if (j < 2 * kRowsOut) cur = fma_row_from(bias_acc, r, wlo, whi);
           }
         }
+      } else if (MODE == 1 && PACKED && PLANE == 14) {
+        // the same for whole 14 x 14 planes staged back to back (7 output rows): row 14 lies outside the plane and
+        // contributes nothing, so the last output row is complete after row 13
+        constexpr int kW = 14;
+        const unsigned col = data + static_cast<unsigned>(2 * x * 8);
+        const bool vr = 2 * x + 2 < kW;
+        Acc cur = bias_acc;
+#pragma unroll
+        for (int j = 0; j < kW; ++j) {
+          uint4 m;
+          uint2 u[3];
+          asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(m.x), "=r"(m.y), "=r"(m.z), "=r"(m.w) : "r"(col + static_cast<unsigned>(j * kW * 8)));
+          u[0] = make_uint2(m.x, m.y);
+          u[1] = make_uint2(m.z, m.w);
+          u[2] = make_uint2(0u, 0u);
+          if (vr) u[2] = lds64(col + static_cast<unsigned>((j * kW + 2) * 8));
+          const Row r = widen(u);
+          if (j & 1) {
+            fma_row(cur, r, wlo + 3, whi + 3);
+            if (j == kW - 1) emit(cur);
+          } else {
+            if (j > 0) {
+              fma_row(cur, r, wlo + 6, whi + 6);
+              emit(cur);
+            }
+            cur = fma_row_from(bias_acc, r, wlo, whi);
+          }
+        }
       } else if (MODE != 2) {
         // one pointer per tap column, walking down the staged rows; a column outside the image
         // stays on a zero pixel
@@ -797,8 +825,8 @@ static int depthwise_f16_impl(const LaunchRec& r, const Ptrs& p, void* stream, b
   const float* b = static_cast<const float*>(p.bias);
   const __half* res = static_cast<const __half*>(p.res);
   __half* out = static_cast<__half*>(p.out);
-  static bool attr_done_dev[kMaxDevices][3][3][2][2][2][9] = {};
-  bool(&attr_done)[3][3][2][2][2][9] = attr_done_dev[current_device_slot()];
+  static bool attr_done_dev[kMaxDevices][3][3][2][2][2][10] = {};
+  bool(&attr_done)[3][3][2][2][2][10] = attr_done_dev[current_device_slot()];
   // small square planes, stride 1, one padding row / column on every side, a thread per whole column: straight-line stencil
   const bool whole_plane = packed && mode == 0 && !pair && g.H == g.W && g.pt == 1 && g.pl == 1 && g.Ho == g.H && g.Wo == g.W;
   // ... and 28-wide planes in bands of 14 rows per thread (staged with zero rows: not the one-copy mode)
@@ -808,7 +836,9 @@ static int depthwise_f16_impl(const LaunchRec& r, const Ptrs& p, void* stream, b
   // ... and stride 2 without padding above / left on 112-, 56- and 28-wide planes whose bands are exactly 8 / 7 / 7 output rows
   const bool down = !packed && mode == 1 && g.pt == 0 && g.pl == 0 && (g.W == 112 || g.W == 56 || g.W == 28) && g.Wo == g.W / 2 &&
                     g.Ho == g.H / 2 && g.H % 2 == 0 && g.sub == 1 && g.tr == (g.W == 112 ? 8 : 7) && g.Ho % g.tr == 0;
-  const int plane = whole_plane && g.H == 14 ? 14 : whole_plane && g.H == 7 ? 7 : band28 ? 28 : pair14 ? g.W : down ? g.W : 0;
+  // ... and on whole 14 x 14 planes staged by one copy
+  const bool down14 = packed && mode == 1 && g.pt == 0 && g.pl == 0 && g.W == 14 && g.H == 14 && g.Wo == 7 && g.Ho == 7;
+  const int plane = whole_plane && g.H == 14 ? 14 : whole_plane && g.H == 7 ? 7 : band28 ? 28 : pair14 ? g.W : down ? g.W : down14 ? 14 : 0;
   const bool tail = r.ep.has_res || r.ep.act_post != GI_ACT_NONE;
 #define GI_DW_LAUNCH3(M, A, T, P, Q, PL, PLI)                                                                                 \
   do {                                                                                                                        \
@@ -838,6 +868,8 @@ static int depthwise_f16_impl(const LaunchRec& r, const Ptrs& p, void* stream, b
       GI_DW_LAUNCH3(1, A, T, 0, 0, 56, 7);            \
     } else if (M == 1 && P == 0 && Q == 0 && plane == 28) { \
       GI_DW_LAUNCH3(1, A, T, 0, 0, 28, 8);            \
+    } else if (M == 1 && P == 1 && Q == 0 && plane == 14) { \
+      GI_DW_LAUNCH3(1, A, T, 1, 0, 14, 9);            \
     } else {                                          \
       GI_DW_LAUNCH3(M, A, T, P, Q, 0, 0);             \
     }                                                 \
