@@ -773,7 +773,8 @@ static int depthwise_f16_impl(const LaunchRec& r, const Ptrs& p, void* stream, b
     return q.head_px + ((px + 1) & ~1) + ((q.W + 3) & ~1);  // zero head, staged rows, zero row behind
   };
   g.plane_stride_px = smem_for(g);
-  const long long budget = 64 * 1024;  // per staging buffer: two buffers per CTA, two or three CTAs per SM
+  // per staging buffer: two buffers per CTA, two or three CTAs per SM - unless the measured table says otherwise
+  const long long budget = (r.dw_buf_kb > 0 ? r.dw_buf_kb : 64) * 1024LL;
   while (static_cast<long long>(g.plane_stride_px) * 8 * g.nb > budget && (g.nb > 1 || g.sub > 1 || g.tr > 1)) {
     if (g.nb > 1) {
       g.nb = (g.nb + 1) / 2;
@@ -796,7 +797,8 @@ static int depthwise_f16_impl(const LaunchRec& r, const Ptrs& p, void* stream, b
   const size_t buf_bytes = packed ? static_cast<size_t>(g.Pin) * 8 * g.nb + 16 : static_cast<size_t>(g.plane_stride_px) * 8 * g.nb;
   // bytes in flight hide the HBM latency: two CTAs per SM (the register file allows no more),
   // each with up to three items requested ahead of the one it computes
-  int nbuf = static_cast<int>(static_cast<size_t>(kSmemPerCta) / buf_bytes);
+  const size_t per_cta = r.dw_cta_kb > 0 ? static_cast<size_t>(r.dw_cta_kb) * 1024 : static_cast<size_t>(kSmemPerCta);
+  int nbuf = static_cast<int>(per_cta / buf_bytes);
   g.nbuf = nbuf > 4 ? 4 : nbuf < 2 ? 2 : nbuf;
   const size_t smem = buf_bytes * g.nbuf;
   if (smem > static_cast<size_t>(kMaxSmem)) return static_cast<int>(cudaErrorInvalidConfiguration);

@@ -71,6 +71,9 @@ struct LaunchRec {
   int in0_dead = 0;
   // depthwise: 1 = the shared-memory staged fp16 stencil runs this op, 0 = the plain one-thread-per-pixel kernel
   int dw_staged = 0;
+  // staged stencil: size limit of one staging buffer and shared memory of one CTA in KB, from the measured table of
+  // staging choices (0 = the kernel's defaults, 64 and 110)
+  int dw_buf_kb = 0, dw_cta_kb = 0;
   // the stem convolution reads the caller's NHWC input itself; the layout conversion in front of it launches nothing
   int nhwc_in = 0;
   // depthwise + pointwise as one kernel: the 1x1 convolution's weights, bias, output channels and epilogue

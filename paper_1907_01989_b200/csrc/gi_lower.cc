@@ -1,6 +1,7 @@
 // Lowering: choose a kernel per executed op, pack its weights into the kernel's operand
 // layout (fp16 storage: weights rounded to fp16 once, biases stay fp32) and record the
 // launch geometry.  Host work only.
+#include <cstdlib>
 #include <cstring>
 
 #include "gi_internal.h"
@@ -133,6 +134,23 @@ static const LaunchChoice kLaunchTable[] = {
 static const LaunchChoice* launch_table_lookup(long long px, int cin, int cout) {
   for (const LaunchChoice& c : kLaunchTable)
     if (c.px == px && c.cin == cin && c.cout == cout && c.kernel != 0) return &c;
+  return nullptr;
+}
+
+// The same for the staged depthwise stencil: how large a staging buffer may be and how much shared memory a CTA takes
+// (which together decide planes per work item, buffers in flight and CTAs per SM), per depthwise shape of the
+// benchmark networks, as measured by the tuner.  Shapes that are not in the table run with the kernel's defaults.
+struct DwChoice {
+  int batch, h, w, c, stride, buf_kb, cta_kb;
+  float ms_default, ms_best;
+};
+static const DwChoice kDwTable[] = {
+    {0, 0, 0, 0, 0, 0, 0, 0.f, 0.f},  // keeps the array non-empty when the table has not been generated
+#include "dw_table.inc"
+};
+static const DwChoice* dw_table_lookup(int batch, int h, int w, int c, int stride) {
+  for (const DwChoice& d : kDwTable)
+    if (d.batch == batch && d.h == h && d.w == w && d.c == c && d.stride == stride && d.batch != 0) return &d;
   return nullptr;
 }
 
@@ -297,7 +315,24 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
         } else if (f.kind == GI_OP_DEPTHWISE_CONV2D) {
           r.kernel = GI_KERNEL_DEPTHWISE;
           r.C = din->c;
+          if (op.d.dilation_h == 1 && op.d.stride_h == op.d.stride_w) {
+            // (GI_DW_BUF_KB / GI_DW_CTA_KB in the environment of gi_compile override the table: the tuner's hook)
+            const char* ebuf = getenv("GI_DW_BUF_KB");
+            const char* ecta = getenv("GI_DW_CTA_KB");
+            if (ebuf || ecta) {
+              r.dw_buf_kb = ebuf ? atoi(ebuf) : 0;
+              r.dw_cta_kb = ecta ? atoi(ecta) : 0;
+            } else if (const DwChoice* dc = dw_table_lookup(e->batch, din->h, din->w, din->c, op.d.stride_h)) {
+              r.dw_buf_kb = dc->buf_kb;
+              r.dw_cta_kb = dc->cta_kb;
+            }
+          }
           r.dw_staged = e->storage == GI_F16 && depthwise_f16_supported(r);
+          if (!r.dw_staged && (r.dw_buf_kb || r.dw_cta_kb)) {
+            // not with these sizes: the kernel's own
+            r.dw_buf_kb = r.dw_cta_kb = 0;
+            r.dw_staged = e->storage == GI_F16 && depthwise_f16_supported(r);
+          }
           if (!r.dw_staged && e->batch > 65535)
             return fail(GI_E_UNSUPPORTED, "gi_compile: depthwise convolution: batch above 65535 with a shape only the plain kernel runs");
           pack_depthwise(op, din->c, e->storage, &e->weight_blob, &r);

@@ -595,3 +595,29 @@ def test_launch_table_and_rule_agree_where_both_apply():
         g, _ = api.graph_from_spec(spec, api.GI_F16, io_layout=api.GI_PHWC4)
         kernels.append(g.compile(pointwise=mode).ops()[0].kernel)
     assert kernels[0] == kernels[1]
+
+
+def test_depthwise_staging_table_is_sane_and_compiles():
+    """The generated table of staging sizes for the depthwise stencil: an entry keeps the kernel's defaults (0, 0) unless
+    its own measurements show another setting more than 3 % faster, every size is one the tuner tries, and every shape in
+    it still compiles to the staged kernel (a setting the kernel cannot run falls back to the defaults)."""
+    import re
+    path = os.path.join(ROOT, "paper_1907_01989_b200", "csrc", "dw_table.inc")
+    rows = [tuple(float(v.rstrip("f")) for v in m.group(1).split(",")) for m in re.finditer(r"^\{([^}]*)\},", open(path).read(), re.M)]
+    assert len(rows) >= 30
+    for b, h, w, c, stride, buf_kb, cta_kb, t0, t1 in rows:
+        assert buf_kb in (0, 16, 24, 36, 48, 64) and cta_kb in (0, 56, 75, 110)
+        assert (buf_kb, cta_kb) == (0, 0) or t1 * 1.03 < t0
+        assert t1 <= t0
+    for b, h, w, c, stride, *_ in rows[:12]:
+        spec = wl.single_depthwise(int(b), int(h), int(c), int(stride), 1)
+        g, _ = api.graph_from_spec(spec, api.GI_F16, io_layout=api.GI_PHWC4)
+        assert [api.KERNEL_NAMES[o.kernel] for o in g.compile().ops()] == ["depthwise"]
+    # the override used by the tuner: sizes from the environment at compile time, nonsense falls back to the defaults
+    os.environ["GI_DW_BUF_KB"], os.environ["GI_DW_CTA_KB"] = "1", "1"
+    try:
+        g, _ = api.graph_from_spec(wl.single_depthwise(4, 56, 32, 1, 1), api.GI_F16, io_layout=api.GI_PHWC4)
+        assert [api.KERNEL_NAMES[o.kernel] for o in g.compile().ops()] == ["depthwise"]
+    finally:
+        del os.environ["GI_DW_BUF_KB"], os.environ["GI_DW_CTA_KB"]
+
