@@ -7,12 +7,12 @@
 // One launch, one fill and one drain replace two, and the second operator's input costs no memory traffic.
 //
 // Per tile of 128 pixels (row r of every MMA = pixel r of the tile):
-//   G1   D1[128 x N1] = X[128 x K1] * W1^T       X streamed in 32-channel chunks: one TMA box (128 pixels x 8 slices) per
+//   G1   D1[128 x N1] = X[128 x K1] * W1^T       X streamed in 64-channel chunks: one TMA box (128 pixels x 16 slices) per
 //                                                chunk lands in a deep ring; four warps rearrange it IN PLACE into the
 //                                                canonical K-major operand layout (two 4-channel slices interleave into
-//                                                one 16-byte operand row: every thread reads its pixel's eight pixel-slices,
+//                                                one 16-byte operand row: every thread reads its pixel's sixteen pixel-slices,
 //                                                the 128 threads meet at a named barrier, every thread writes its pixel's
-//                                                four rows); the chunk's W1 rows (bulk copy) have a ring of their own.  (8-byte
+//                                                eight rows); the chunk's W1 rows (bulk copy) have a ring of their own.  (8-byte
 //                                                cp.async straight into the operand layout was the first version: each copy
 //                                                holds an L1 line while in flight, and the little L1 left beside 200 KB of
 //                                                shared memory capped a CTA at 14 GB/s.)
@@ -21,8 +21,8 @@
 //   G2   D2[128 x n2_blk] = A2[128 x N1] * W2[block]^T     for each block of output channels; W2 blocks by bulk copy,
 //                                                resident when all of them fit
 //   T2   bias, activation, fp16 -> global memory (the second operator's output)
-// D1 and A2 are double-buffered where tensor memory allows, D2 always: the MMA thread issues G1 of tile t+1 before G2
-// of tile t, so loads, both MMAs and both drains of neighbouring tiles overlap.
+// D1 and A2 are double-buffered where tensor memory allows, D2 always: the MMA thread issues G1 of tile t+1 and keeps G2 of
+// tile t as pending work that its waits poll for, so loads, both MMAs and both drains of neighbouring tiles overlap.
 //
 // Warps: 0 = X copies, 1 = MMA issuer and TMEM owner, 2..5 = X repack, 6..9 = T1, 10..21 = T2, 22 = W2 copies, 23 = W1 copies.
 // All waits are bounded; a wait that runs out raises the abort flag and every role leaves its loop.
@@ -48,7 +48,7 @@ constexpr int kW2Warp = kFirstT2 + kT2Warps, kW1Warp = kW2Warp + 1;
 constexpr int kThreads = 32 * (kW1Warp + 1);
 constexpr int kMaxLand = 16, kMaxW1 = 8, kMaxW2Slots = 12;
 constexpr int kHeader = 1024;
-constexpr int kABytes = (kKc / 2) * kRows * 16;  // 8 KB: one chunk of X
+constexpr int kABytes = (kKc / 2) * kRows * 16;  // 16 KB: one chunk of X
 constexpr int kSmemMax = 227 * 1024;
 constexpr int kMinLand = 3;  // landing stages: the launches this kernel is for are bound by bytes in flight per SM
 
@@ -395,7 +395,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_chain_kernel(const __gr
     }
   } else if (warp < kFirstT1) {
     // ------------------------------------------------------------ X chunks: landing layout -> operand layout, in place
-    // landed: [slice][pixel] 8-byte pixel-slices; operand: [K group of 8 channels][pixel] 16-byte rows.  Both are 8 KB;
+    // landed: [slice][pixel] 8-byte pixel-slices; operand: [K group of 8 channels][pixel] 16-byte rows.  Both are 16 KB;
     // a thread's four rows lie where other threads' pixel-slices landed, so all 128 threads read before any writes.
     const int row = threadIdx.x - 32 * kFirstLoad;  // 0 .. 127: row of the tile
     unsigned it = 0;
@@ -627,7 +627,7 @@ Tiling try_tiling(int cin, int cmid, int cout, bool has_res, int d_bufs) {
   t.n2_blocks = (n2_pad + max_blk - 1) / max_blk;
   t.n2_blk = ((n2_pad + t.n2_blocks - 1) / t.n2_blocks + 15) / 16 * 16;
   t.d2_col0 = static_cast<unsigned>(t.d_bufs * t.n1_pad);
-  t.w1_bytes = static_cast<unsigned>(t.n1_pad) * kKc * 8u;  // n1_pad rows x 32 channels x 2 bytes
+  t.w1_bytes = static_cast<unsigned>(t.n1_pad) * kKc * 8u;  // n1_pad rows x 64 channels x 2 bytes
   t.w2_bytes = static_cast<unsigned>(t.n2_blk) * static_cast<unsigned>(t.n1_pad) * 2u;
   t.w2_pitch = (t.w2_bytes + 1023u) / 1024u * 1024u;
   t.a2_bytes = static_cast<unsigned>(kRows) * static_cast<unsigned>(t.n1_pad) * 2u;
@@ -675,7 +675,7 @@ Tiling choose_tiling(int cin, int cmid, int cout, bool has_res) {
 
 bool pointwise_chain_supported(int cin, int cmid, int cout, bool has_res) { return choose_tiling(cin, cmid, cout, has_res).ok; }
 
-// First operator: dense weights as the B operand per K chunk, [4 K groups][n1_pad rows][8 halves].  Second operator:
+// First operator: dense weights as the B operand per K chunk, [8 K groups][n1_pad rows][8 halves].  Second operator:
 // per block of output channels [n1_pad / 8 K groups][n2_blk rows][8 halves].  Entries beyond the real channels are
 // zero, and so are the padded biases, so padded columns of both accumulators hold exact zeros.
 void pointwise_chain_pack(const float* w1, const float* b1, const float* w2, const float* b2, int cin, int cmid, int cout,
