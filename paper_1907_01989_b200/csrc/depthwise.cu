@@ -98,6 +98,11 @@ __device__ __forceinline__ Row widen(const uint2* u) {
 // MODE 1: stride 2, dilation 1, same padding limit - the last row of an output is the first row
 //         of the next
 // MODE 2: anything else - three rows fetched per output row, each tap tested
+// MODE 3: stride 1, dilation d > 1, padding d on every side (the dilated blocks of a segmentation backbone), whole planes
+//         staged by one copy: the rows of one residue class modulo d form an ordinary 3-row stencil among themselves
+//         (output row y reads rows y - d, y, y + d), so a thread owns (plane, residue, column) and walks its class
+//         with the three running accumulators of mode 0 - every staged pixel is fetched and widened three times, as in
+//         mode 0, instead of nine times as in mode 2
 // PACKED (modes 0/1, small planes): a work item is a run of whole planes, which are contiguous in
 //         memory, so ONE bulk copy stages them back to back (many small copies are slow); the
 //         rows above and below a plane are then its neighbours' rows, so row validity is tested
@@ -307,7 +312,8 @@ __global__ void __launch_bounds__(256, (PLANE > 0 && !PAIR) ? 3 : 2) depthwise_f
         sb = vp - pi * g.sub;
       }
       if (PAIR) x *= 2;
-      const int ya = oy0 + sb * g.tr, yb = min(oy1, ya + g.tr);
+      // (mode 3: `sb` is the residue class, whose first row is row sb)
+      const int ya = MODE == 3 ? sb : oy0 + sb * g.tr, yb = MODE == 3 ? H : min(oy1, ya + g.tr);
       if (ya >= yb) continue;
       // plane_zero: a pixel of the zero head; data: where pixel (0,0) of the plane would be staged
       const unsigned plane_zero = PACKED ? buf_addr : buf_addr + static_cast<unsigned>(pi) * g.plane_stride_px * 8u;
@@ -316,7 +322,7 @@ __global__ void __launch_bounds__(256, (PLANE > 0 && !PAIR) ? 3 : 2) depthwise_f
       const size_t out_off = ((static_cast<size_t>(s) * g.B + b0 + pi) * g.Pout + static_cast<size_t>(ya) * Wo + x) * 4;
       __half* op = out + out_off;
       const ptrdiff_t res_minus_out = res - out;  // only used when TAIL
-      const int out_stride = Wo * 4;
+      const int out_stride = MODE == 3 ? g.dil * Wo * 4 : Wo * 4;  // halves from one output row of this thread to its next
       auto emit = [&](const Acc& a) {
         uint2 u;
         if (!TAIL) {
@@ -540,6 +546,56 @@ __global__ void __launch_bounds__(256, (PLANE > 0 && !PAIR) ? 3 : 2) depthwise_f
           }
           if (j >= 1 && j <= kRowsOut) fma_row(acc[(j + 2) % 3], r, wlo + 3, whi + 3);
           if (j < kRowsOut) acc[j % 3] = fma_row_from(bias_acc, r, wlo, whi);
+        }
+      } else if (MODE == 3) {
+        const int d = g.dil;
+        const bool vl = x - d >= 0, vr = x + d < W;
+        unsigned at = data + static_cast<unsigned>((ya * W + x) * 8);
+        const unsigned row_step = static_cast<unsigned>(d * W) * 8u, dx = static_cast<unsigned>(d) * 8u;
+        auto next_row = [&]() {
+          uint2 u[3];
+          u[0] = make_uint2(0u, 0u);
+          u[2] = make_uint2(0u, 0u);
+          if (vl) u[0] = lds64(at - dx);
+          u[1] = lds64(at);
+          if (vr) u[2] = lds64(at + dx);
+          at += row_step;
+          return widen(u);
+        };
+        const int n = (H - ya + d - 1) / d;  // rows of this residue class
+        // class row k is kernel row 2 of the class's output row k - 1, row 1 of output row k, row 0 of output row k + 1
+        Acc a0 = bias_acc, a1, a2;
+        Row r = next_row();
+        fma_row(a0, r, wlo + 3, whi + 3);
+        a1 = fma_row_from(bias_acc, r, wlo, whi);
+        for (int k = 1;; k += 3) {
+          if (k >= n) {
+            emit(a0);
+            break;
+          }
+          r = next_row();
+          fma_row(a0, r, wlo + 6, whi + 6);
+          emit(a0);
+          fma_row(a1, r, wlo + 3, whi + 3);
+          a2 = fma_row_from(bias_acc, r, wlo, whi);
+          if (k + 1 >= n) {
+            emit(a1);
+            break;
+          }
+          r = next_row();
+          fma_row(a1, r, wlo + 6, whi + 6);
+          emit(a1);
+          fma_row(a2, r, wlo + 3, whi + 3);
+          a0 = fma_row_from(bias_acc, r, wlo, whi);
+          if (k + 2 >= n) {
+            emit(a2);
+            break;
+          }
+          r = next_row();
+          fma_row(a2, r, wlo + 6, whi + 6);
+          emit(a2);
+          fma_row(a0, r, wlo + 3, whi + 3);
+          a1 = fma_row_from(bias_acc, r, wlo, whi);
         }
       } else if (MODE == 1 && !PACKED && PLANE > 0) {
         // stride 2 without padding above / left on PLANE-wide planes, bands of exactly kRowsOut output rows: the band's
@@ -789,12 +845,24 @@ static int depthwise_f16_impl(const LaunchRec& r, const Ptrs& p, void* stream, b
     g.bands = (total_sub + g.sub - 1) / g.sub;
     g.plane_stride_px = smem_for(g);
   }
+  // dilated, stride 1, padded by the dilation, planes small enough to stage a few whole: the residue-class walk
+  const bool dilated = g.stride == 1 && g.dil > 1 && g.pt == g.dil && g.pl == g.dil && g.Ho == g.H && g.Wo == g.W && g.dil <= g.H &&
+                       static_cast<long long>(g.Pin) * 8 <= budget;
+  if (dilated) {
+    g.sub = g.dil;                          // residue classes
+    g.tr = (g.H + g.dil - 1) / g.dil;       // rows of the longest class
+    g.bands = 1;
+    long long planes = budget / (static_cast<long long>(g.Pin) * 8);
+    if (planes > 8) planes = 8;
+    g.nb = planes < g.B ? static_cast<int>(planes) : g.B;
+    g.plane_stride_px = smem_for(g);
+  }
   // the fast paths need the rows above and below the image to be at most one (zero rows in the buffer)
   const int overshoot = (g.Ho - 1) * g.stride - g.pt + 2 - (g.H - 1);
   const bool edge_ok = g.dil == 1 && g.pt <= 1 && overshoot <= 1;
-  const int mode = (edge_ok && g.stride == 1) ? 0 : (edge_ok && g.stride == 2) ? 1 : 2;
+  const int mode = dilated ? 3 : (edge_ok && g.stride == 1) ? 0 : (edge_ok && g.stride == 2) ? 1 : 2;
   // small planes, several per item, each walked top to bottom by its threads: stage them with one copy
-  const bool packed = mode != 2 && g.bands == 1 && g.sub == 1 && g.nb > 4 && !pair;
+  const bool packed = mode == 3 || (mode != 2 && g.bands == 1 && g.sub == 1 && g.nb > 4 && !pair);
   g.packed = packed ? 1 : 0;
   const size_t buf_bytes = packed ? static_cast<size_t>(g.Pin) * 8 * g.nb + 16 : static_cast<size_t>(g.plane_stride_px) * 8 * g.nb;
   // bytes in flight hide the HBM latency: two CTAs per SM (the register file allows no more),
@@ -844,8 +912,8 @@ static int depthwise_f16_impl(const LaunchRec& r, const Ptrs& p, void* stream, b
   const float* b = static_cast<const float*>(p.bias);
   const __half* res = static_cast<const __half*>(p.res);
   __half* out = static_cast<__half*>(p.out);
-  static bool attr_done_dev[kMaxDevices][3][3][2][2][2][11] = {};
-  bool(&attr_done)[3][3][2][2][2][11] = attr_done_dev[current_device_slot()];
+  static bool attr_done_dev[kMaxDevices][4][3][2][2][2][11] = {};
+  bool(&attr_done)[4][3][2][2][2][11] = attr_done_dev[current_device_slot()];
   const bool tail = r.ep.has_res || r.ep.act_post != GI_ACT_NONE;
 #define GI_DW_LAUNCH3(M, A, T, P, Q, PL, PLI)                                                                                 \
   do {                                                                                                                        \
@@ -917,6 +985,8 @@ static int depthwise_f16_impl(const LaunchRec& r, const Ptrs& p, void* stream, b
     GI_DW_MODE(0);
   } else if (mode == 1) {
     GI_DW_MODE(1);
+  } else if (mode == 3) {
+    GI_DW_MODE(3);
   } else {
     GI_DW_MODE(2);
   }

@@ -123,6 +123,9 @@ DW_CASES = [  # batch, hw, c, stride, dilation, residual
     (1, 7, 32, 1, 1, False), (2, 14, 96, 2, 1, False), (1, 33, 24, 1, 2, False), (1, 33, 8, 1, 4, True),
     (3, 9, 10, 2, 1, False), (1, 56, 144, 1, 1, True), (2, 112, 32, 2, 1, False), (1, 65, 12, 2, 1, False),
     (2, 3, 5, 1, 1, False), (1, 1, 7, 1, 1, False), (2, 2, 4, 2, 1, False),
+    # dilated: even and odd planes, classes of unequal length, several planes per work item, a dilation larger than the plane
+    (5, 20, 40, 1, 2, False), (3, 20, 12, 1, 4, True), (2, 10, 8, 1, 3, False), (2, 5, 4, 1, 4, False), (1, 3, 8, 1, 4, False),
+    (16, 33, 96, 1, 2, False),
 ]
 
 
