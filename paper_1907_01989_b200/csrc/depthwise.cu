@@ -809,9 +809,13 @@ static int depthwise_f16_impl(const LaunchRec& r, const Ptrs& p, void* stream, b
   if (g.sub < 1) g.sub = 1;
   // rows walked by a thread: 16 (stride 1) or 8; pairs: 14, which divides the usual plane heights - bands of
   // equal height measured better than taller ones with a short last band (16 rows: 10-20 % slower on 112 / 56)
-  // 28 x 28 planes are walked whole as well (28 rows per thread): whole planes are contiguous, so one copy stages an
-  // item instead of one per plane, and no halo row is read twice (batch 256, 192 channels: 0.0430 -> 0.0389 ms)
-  const int tr_target = g.stride == 1 ? (pair ? 14 : (g.W == 28 && g.H == 28 ? 28 : 16)) : 8;
+  // planes of up to about 33 x 33 pixels are walked whole as well (28 or 33 rows per thread): whole planes are contiguous,
+  // so one copy stages an item instead of one per plane, and no halo row is read twice (28 x 28, batch 256, 192 channels:
+  // 0.0430 -> 0.0389 ms)
+  // - where that still leaves at least one work item per SM (at batch 1 the bands are the parallelism)
+  const int whole_nb = g.nb < 1 ? 1 : g.nb;
+  const bool whole = g.H > 16 && g.H * g.W <= 1100 && static_cast<long long>(g.S) * ((g.B + whole_nb - 1) / whole_nb) >= 148;
+  const int tr_target = g.stride == 1 ? (pair ? 14 : (whole ? g.H : 16)) : 8;
   int total_sub = (g.Ho + tr_target - 1) / tr_target;
   if (pair) {
     // up to four sub-bands of one plane (they share halo rows), two passes of the threads per item; the
