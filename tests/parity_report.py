@@ -32,6 +32,8 @@ def main():
         outs = run.run(xs)
         rows = []
         for t, r in sorted(ref.items()):
+            if t in run.on_chip:  # never stored (the converted copy of an NHWC input the stem reads itself, a fused block's hidden tensors)
+                continue
             got = outs[t] if t in outs else run.fetch(t)
             worst, q999 = error_report(got, r, storage)
             rows.append((t, tuple(spec.shapes[t]), worst, q999))
