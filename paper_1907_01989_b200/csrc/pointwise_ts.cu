@@ -7,15 +7,17 @@
 // and the weight operand is the dense [Cout][Cin] matrix, small enough to stay in shared memory
 // for the whole kernel (each CTA keeps the rows of its share of the output channels).  What
 // streams is the activation only: TMA boxes of 128 pixels x ks slices land in a ring of shared
-// memory stages, four transfer warps move a stage into tensor memory (8-byte ld.shared per lane,
+// memory stages, eight transfer warps move a stage into tensor memory (8-byte ld.shared per lane,
 // tcgen05.st), and every byte of shared memory that is not weights is activation in flight -
 // which is what a layer bound by HBM latency x bandwidth needs.  The pixel-pair variant
 // (pointwise_tc.cu) keeps the layers with few input channels and large planes; this one takes
 // the layers where that variant's 4x expanded weight tile crowded the activations out of shared
 // memory.
 //
-// CTA = 22 warps: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-5 transfer
-// (one TMEM lane quarter each), warps 6-21 drain the accumulator (four per quarter: bias,
+// CTA = 26 warps: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-9 transfer
+// (two per TMEM lane quarter, taking alternate groups of 8 slices: with deep inputs and a single tile per CTA - batch 1 - the
+// transfer of K through four warps was a third of a launch; MobileNetV2 batch 1 0.240 -> 0.2375 ms, 0.2215 -> 0.218 ms as a
+// CUDA graph), warps 10-25 drain the accumulator (four per quarter: bias,
 // activation, residual, fp16 pack, 8-byte stores, 256 contiguous bytes per warp).  Accumulators
 // and A chunks are double-buffered in the 512 TMEM columns.  If a CTA's weight share does not
 // fit, the weights stream through the same stages instead.  All waits are bounded.
@@ -35,7 +37,7 @@ namespace {
 using namespace ptx;
 
 constexpr int kRows = 128;
-constexpr int kTransferWarps = 4;
+constexpr int kTransferWarps = 8;  // two per TMEM lane quarter: each moves every other group of 8 slices of a chunk
 constexpr int kDrainWarps = 16;
 constexpr int kThreads = 32 * (2 + kTransferWarps + kDrainWarps);
 constexpr int kMaxStages = 8;
@@ -256,6 +258,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, +32)
     const unsigned lane_bits = static_cast<unsigned>(quarter * 32) << 16;
     const unsigned row_off = static_cast<unsigned>(quarter * 32 + lane) * 8u;
+    const int part = (warp - 2) >> 2;  // which of the quarter's two transfer warps
     unsigned it = 0;
     bool ok = true;
     for (int m = m_first; m < p.m_tiles && ok; m += m_step) {
@@ -272,7 +275,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
         const unsigned t_addr = tmem_base + lane_bits + a_col0 + abuf * a_cols;
         // a box narrower than 128 pixels leaves the upper lane quarters without data: their rows of the
         // accumulator are never stored, so their lanes of the A operand may hold anything
-        for (int j = 0; j < p.ks && quarter * 32 < p.box_px; j += 8) {
+        for (int j = 8 * part; j < p.ks && quarter * 32 < p.box_px; j += 8 * (kTransferWarps / 4)) {
           unsigned r[16];
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
