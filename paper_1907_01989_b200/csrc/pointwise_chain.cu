@@ -409,7 +409,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_chain_kernel(const __gr
 #pragma unroll
         for (int sl = 0; sl < kKc; ++sl)
           asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(v[sl][0]), "=r"(v[sl][1]) : "r"(base + static_cast<unsigned>(sl) * (kRows * 8u) + static_cast<unsigned>(row) * 8u) : "memory");
-        // the barrier also carries the verdict of the wait, so that all four warps leave together if one gave up
+        // the barrier also carries the outcome of the wait, so that all four warps leave together if one gave up
         unsigned all_ok;
         asm volatile(
             "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred p, 1, %2, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
