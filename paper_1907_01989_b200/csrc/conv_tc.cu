@@ -11,9 +11,10 @@
 // window's first pixel is the same for every pixel and comes from a small table in shared memory) and write
 // them, two per 16-byte unit, straight into the canonical K-major shared-memory operand layout; the weights
 // sit in shared memory for the whole kernel.
-// Operand buffers are double-buffered against the MMAs (a buffer is handed back by tcgen05.commit), the
-// accumulators against the epilogue: the gather of tile i+1 runs while the MMAs of tile i finish, and the
-// same 128 threads then drain tile i (bias, fused element-wise tail, 8 bytes per output slice).  Waits are
+// Three operand buffers (handed back by tcgen05.commit) and two accumulators decouple three roles: four gather warps,
+// the MMA warp, and four epilogue warps that drain a tile (bias, fused element-wise tail, 8 bytes per output slice).
+// (First version: the same 128 threads gathered tile i+1 and then drained tile i; a gather thread waits for its loads
+// most of the time, an epilogue thread for tensor memory, and in one thread neither wait hides the other.)  Waits are
 // bounded like in the other tensor-core kernels.  The 3 x 3 kernel for a single input slice (the stem of the
 // MobileNets) is the special case with one chunk and no hand-back; it keeps its own file.
 #include <cuda.h>
@@ -34,8 +35,9 @@ constexpr int kRows = 128;             // output pixels per tile
 // the smaller operand buffers and register footprint let six CTAs instead of four share an SM (measured:
 // the fire network 0.296 -> 0.284 ms with 8, while 3x3 32 -> 32 and 64 -> 64 lose 8-18 % with 8)
 constexpr int kMaxUnits = 16;
-constexpr int kGatherThreads = 128;
-constexpr int kThreads = kGatherThreads + 32;
+constexpr int kGatherThreads = 128, kEpilogueWarps = 4;
+constexpr int kThreads = kGatherThreads + 32 + 32 * kEpilogueWarps;  // warps 0-3 gather, 4 issues the MMAs, 5-8 drain
+constexpr int kABufs = 3;
 constexpr int kMaxN = 256;
 constexpr int kHeaderBytes = 1024;
 constexpr int kMaxWeightBytes = 150 * 1024;
@@ -58,14 +60,15 @@ struct ConvParams {
   int step_b, step_q;        // (gridDim.x / n_groups) * 128 pixels = step_b planes + step_q pixels
   unsigned m_total;          // B * Pout (< 2^31)
   int has_res, act_post;
+  int a_bufs;                // operand buffers in the ring: 3, or 2 where the third would cost a CTA per SM
   unsigned tmem_cols;
   unsigned timeout_ns;
 };
 
 struct Header {
-  unsigned long long a_full[2];
-  unsigned long long a_empty[2];
-  unsigned long long acc_full[2];
+  unsigned long long a_full[kABufs];
+  unsigned long long a_empty[kABufs];
+  unsigned long long acc_full[2], acc_empty[2];
   unsigned tmem_addr;
   unsigned abort_flag;
 };
@@ -79,14 +82,14 @@ __device__ __forceinline__ float act1(float v, int kind) {
 // UNITS: pixel-slices per K chunk; ACT: activation right after the bias; TAIL: a residual add and / or a second
 // activation follow
 template <int UNITS, int ACT, bool TAIL>
-__global__ void __launch_bounds__(kThreads, UNITS == 8 ? 6 : 4) conv_kxk_tc_kernel(const ConvParams p) {
+__global__ void __launch_bounds__(kThreads, UNITS == 8 ? 4 : 3) conv_kxk_tc_kernel(const ConvParams p) {
   constexpr int kUnits = UNITS;
   constexpr int kKCores = kUnits / 2;  // 16-byte K units per row and chunk
   constexpr int kABytes = kKCores * kRows * 16;
   extern __shared__ __align__(1024) unsigned char smem[];
   Header* hdr = reinterpret_cast<Header*>(smem);
-  unsigned char* a_tiles = smem + kHeaderBytes;         // 2 x kABytes
-  unsigned char* b_tile = a_tiles + 2 * kABytes;        // n_chunks * 8 * n_pad * 16
+  unsigned char* a_tiles = smem + kHeaderBytes;         // kABufs x kABytes
+  unsigned char* b_tile = a_tiles + p.a_bufs * kABytes;  // n_chunks * 8 * n_pad * 16
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile unsigned* abort_flag = &hdr->abort_flag;
   // CTA group g computes output channels [g * n_pad, (g + 1) * n_pad) of every pixel tile it walks; the CTAs of
@@ -98,10 +101,13 @@ __global__ void __launch_bounds__(kThreads, UNITS == 8 ? 6 : 4) conv_kxk_tc_kern
   const unsigned char* wts = p.wts + (one_group ? 0 : static_cast<size_t>(blockIdx.x % p.n_groups) * p.n_chunks * kKCores * p.n_pad * 16);
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < kABufs; ++i) {
       mbar_init(smem_u32(&hdr->a_full[i]), kGatherThreads);
       mbar_init(smem_u32(&hdr->a_empty[i]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&hdr->acc_full[i]), 1);
+      mbar_init(smem_u32(&hdr->acc_empty[i]), kEpilogueWarps);
     }
     hdr->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -159,13 +165,15 @@ __global__ void __launch_bounds__(kThreads, UNITS == 8 ? 6 : 4) conv_kxk_tc_kern
               tap_ok |= 1u << (ky * p.k + kx);
       }
       for (int c = 0; c < p.n_chunks; ++c, ++it) {
-        const int buf = static_cast<int>(it & 1u);
+        // (two constant divisors instead of a division by a run-time value in every chunk)
+        const int buf = static_cast<int>(p.a_bufs == 3 ? it % 3u : it & 1u);
+        const unsigned e_phase = ((p.a_bufs == 3 ? it / 3u : it >> 1) & 1u) ^ 1u;
         // The loads do not touch the operand buffer: with 16-unit chunks they are issued before the wait for it
         // (3x3 64 -> 64 on 56x56 0.260 -> 0.246 ms, 128 -> 128 on 28x28 0.399 -> 0.358 ms); with 8-unit chunks
         // and their 64-register budget that order spills and measured 2-5 % slower, so there the wait comes first.
         constexpr bool kLoadsFirst = kUnits == 16;
         if (!kLoadsFirst &&
-            !mbar_wait_warp(smem_u32(&hdr->a_empty[buf]), ((it >> 1) & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_conv_kxk_error, 1u))
+            !mbar_wait_warp(smem_u32(&hdr->a_empty[buf]), e_phase, abort_flag, p.timeout_ns, &g_conv_kxk_error, 1u))
           return false;
         uint2 unit[kUnits];
         const int4* off4 = reinterpret_cast<const int4*>(unit_off + c * kUnits);
@@ -178,7 +186,7 @@ __global__ void __launch_bounds__(kThreads, UNITS == 8 ? 6 : 4) conv_kxk_tc_kern
           for (int e = 0; e < 4; ++e) unit[4 * j4 + e] = ((tap_ok >> tn[e]) & 1u) ? __ldg(base + of[e]) : make_uint2(0u, 0u);
         }
         if (kLoadsFirst &&
-            !mbar_wait_warp(smem_u32(&hdr->a_empty[buf]), ((it >> 1) & 1u) ^ 1u, abort_flag, p.timeout_ns, &g_conv_kxk_error, 1u))
+            !mbar_wait_warp(smem_u32(&hdr->a_empty[buf]), e_phase, abort_flag, p.timeout_ns, &g_conv_kxk_error, 1u))
           return false;
         uint4* dst = reinterpret_cast<uint4*>(a_tiles + buf * kABytes) + t;
 #pragma unroll
@@ -190,11 +198,64 @@ __global__ void __launch_bounds__(kThreads, UNITS == 8 ? 6 : 4) conv_kxk_tc_kern
       }
       return true;
     };
+    // this thread's pixel advances by a fixed number of planes and pixels per tile: no divisions by the plane size in the loop
+    const unsigned gp0 = static_cast<unsigned>(cta) * kRows + t;
+    int b = static_cast<int>(gp0 / static_cast<unsigned>(p.Pout));
+    int q = static_cast<int>(gp0 - static_cast<unsigned>(b) * p.Pout);
+    unsigned gp = gp0;
+    const unsigned gp_step = static_cast<unsigned>(ctas) * kRows;
+    for (int tile = cta; tile < p.tiles; tile += ctas) {
+      if (!gather_tile(b, q, gp < p.m_total)) break;
+      gp += gp_step;
+      b += p.step_b;
+      q += p.step_q;
+      if (q >= p.Pout) {
+        q -= p.Pout;
+        ++b;
+      }
+    }
+  } else if (warp == 4) {
+    // ---- MMA issuer
+    if (lane == 0) {
+      // instruction descriptor: fp32 accumulator, fp16 A and B, both K-major, M = 128, N = n_pad
+      const unsigned idesc = (1u << 4) | ((n_cols >> 3) << 17) | ((kRows >> 4) << 24);
+      const unsigned b_base = smem_u32(b_tile), b_lbo = n_cols * 16u;
+      unsigned it = 0;
+      int n = 0;
+      bool ok = true;
+      for (int tile = cta; tile < p.tiles && ok; tile += ctas, ++n) {
+        const unsigned d_tmem = tmem_base + static_cast<unsigned>(n & 1) * n_cols;
+        // the accumulator must have been read out by the epilogue of the tile that used it last
+        if (!mbar_wait(smem_u32(&hdr->acc_empty[n & 1]), ((n >> 1) & 1) ^ 1, abort_flag, p.timeout_ns, &g_conv_kxk_error, 2u)) break;
+        for (int c = 0; c < p.n_chunks; ++c, ++it) {
+          const int buf = static_cast<int>(p.a_bufs == 3 ? it % 3u : it & 1u);
+          if (!mbar_wait(smem_u32(&hdr->a_full[buf]), (p.a_bufs == 3 ? it / 3u : it >> 1) & 1u, abort_flag, p.timeout_ns, &g_conv_kxk_error, 2u)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const unsigned a_base = smem_u32(a_tiles + buf * kABytes);
+          const unsigned bc_base = b_base + static_cast<unsigned>(c) * kKCores * b_lbo;
+#pragma unroll
+          for (int ks = 0; ks < kKCores / 2; ++ks) {
+            const unsigned long long ad = smem_desc(a_base + ks * 2 * kRows * 16, kRows * 16, 128);
+            const unsigned long long bd = smem_desc(bc_base + ks * 2 * b_lbo, b_lbo, 128);
+            umma_f16(d_tmem, ad, bd, idesc, (c > 0 || ks > 0) ? 1u : 0u);
+          }
+          umma_commit(smem_u32(&hdr->a_empty[buf]));  // the buffer is free once these MMAs have read it
+        }
+        // the accumulator's barrier, the one the epilogue waits on, is committed last
+        if (ok) umma_commit(smem_u32(&hdr->acc_full[n & 1]));
+      }
+    }
+  } else {
+    // ---- epilogue warps: lane quarter = warp index modulo 4
+    const int real_px = p.Ho * p.Wo;
     // ---- epilogue of one tile from accumulator `buf`; gp = this thread's pixel in the whole tensor
     auto epilogue = [&](int buf, unsigned phase, unsigned gp, bool in_tensor, bool real) -> bool {
       if (!mbar_wait_warp(smem_u32(&hdr->acc_full[buf]), phase, abort_flag, p.timeout_ns, &g_conv_kxk_error, 4u)) return false;
       tc_fence_after();
-      const unsigned t_addr = tmem_base + buf * n_cols + (static_cast<unsigned>(warp * 32) << 16);
+      const unsigned t_addr = tmem_base + buf * n_cols + (static_cast<unsigned>((warp & 3) * 32) << 16);
       const int grp = p.n_groups == 1 ? 0 : static_cast<int>(blockIdx.x) % p.n_groups, so0 = grp * (p.n_pad / 4);
       const float* bias = p.bias + grp * p.n_pad;
       auto finish = [&](const unsigned* r, unsigned c0) {
@@ -247,75 +308,19 @@ __global__ void __launch_bounds__(kThreads, UNITS == 8 ? 6 : 4) conv_kxk_tc_kern
       return true;
     };
 
-    // software pipeline over this CTA's tiles: the gather of tile n is issued before the epilogue of tile
-    // n - 1.  The pixel of this thread advances by a fixed number of planes and pixels per step: no
-    // divisions by the plane size in the loop
-    const unsigned gp0 = static_cast<unsigned>(cta) * kRows + t;
-    int b = static_cast<int>(gp0 / static_cast<unsigned>(p.Pout));
-    int q = static_cast<int>(gp0 - static_cast<unsigned>(b) * p.Pout);
+    const unsigned gp0 = static_cast<unsigned>(cta) * kRows + static_cast<unsigned>((warp & 3) * 32 + lane);
+    int q = static_cast<int>(gp0 % static_cast<unsigned>(p.Pout));
     unsigned gp = gp0;
     const unsigned gp_step = static_cast<unsigned>(ctas) * kRows;
     int n = 0;
-    bool have_prev = false, prev_in = false, prev_real = false;
-    unsigned prev_gp = 0;
     for (int tile = cta; tile < p.tiles; tile += ctas, ++n) {
-      // accumulator n & 1 was drained by the epilogue of tile n - 2, which these threads ran before
-      // this gather: their arrivals for the first chunk also order the accumulator's reuse
       const bool in_tensor = gp < p.m_total;
-      if (!gather_tile(b, q, in_tensor)) {
-        have_prev = false;
-        break;
-      }
-      if (have_prev && !epilogue((n - 1) & 1, ((n - 1) >> 1) & 1, prev_gp, prev_in, prev_real)) {
-        have_prev = false;
-        break;
-      }
-      have_prev = true;
-      prev_gp = gp;
-      prev_in = in_tensor;
-      prev_real = in_tensor && q < real_px;
+      if (!epilogue(n & 1, (n >> 1) & 1, gp, in_tensor, in_tensor && q < real_px)) break;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&hdr->acc_empty[n & 1]));
       gp += gp_step;
-      b += p.step_b;
       q += p.step_q;
-      if (q >= p.Pout) {
-        q -= p.Pout;
-        ++b;
-      }
-    }
-    if (have_prev) epilogue((n - 1) & 1, ((n - 1) >> 1) & 1, prev_gp, prev_in, prev_real);
-  } else if (lane == 0) {
-    // ---- MMA issuer
-    // instruction descriptor: fp32 accumulator, fp16 A and B, both K-major, M = 128, N = n_pad
-    const unsigned idesc = (1u << 4) | ((n_cols >> 3) << 17) | ((kRows >> 4) << 24);
-    const unsigned b_base = smem_u32(b_tile), b_lbo = n_cols * 16u;
-    unsigned it = 0;
-    int n = 0;
-    bool ok = true;
-    for (int tile = cta; tile < p.tiles && ok; tile += ctas, ++n) {
-      const unsigned d_tmem = tmem_base + static_cast<unsigned>(n & 1) * n_cols;
-      for (int c = 0; c < p.n_chunks; ++c, ++it) {
-        const int buf = static_cast<int>(it & 1u);
-        if (!mbar_wait(smem_u32(&hdr->a_full[buf]), (it >> 1) & 1u, abort_flag, p.timeout_ns, &g_conv_kxk_error, 2u)) {
-          ok = false;
-          break;
-        }
-        tc_fence_after();
-        const unsigned a_base = smem_u32(a_tiles + buf * kABytes);
-        const unsigned bc_base = b_base + static_cast<unsigned>(c) * kKCores * b_lbo;
-#pragma unroll
-        for (int ks = 0; ks < kKCores / 2; ++ks) {
-          const unsigned long long ad = smem_desc(a_base + ks * 2 * kRows * 16, kRows * 16, 128);
-          const unsigned long long bd = smem_desc(bc_base + ks * 2 * b_lbo, b_lbo, 128);
-          umma_f16(d_tmem, ad, bd, idesc, (c > 0 || ks > 0) ? 1u : 0u);
-        }
-        if (c + 1 < p.n_chunks) umma_commit(smem_u32(&hdr->a_empty[buf]));  // the buffer is free once these MMAs have read it
-      }
-      if (ok) {
-        // the last chunk's buffer and the accumulator complete together; the accumulator's barrier, the
-        // one the epilogue waits on, is committed last
-        umma_commit(smem_u32(&hdr->a_empty[(it - 1u) & 1u]));
-        umma_commit(smem_u32(&hdr->acc_full[n & 1]));
-      }
+      if (q >= p.Pout) q -= p.Pout;
     }
   }
 
@@ -430,12 +435,23 @@ int launch_conv_kxk_tc(const LaunchRec& r, const Ptrs& p, void* stream) {
   bool& attr_set = attr_set_dev[current_device_slot()];
   const int sms = device_sm_count();
   const int units = units_of(r.kh, r.C);
-  const size_t smem = kHeaderBytes + 2 * static_cast<size_t>(units / 2) * kRows * 16 + static_cast<size_t>(cores_of(r.kh, r.C)) * k.n_pad * 16 +
-                      static_cast<size_t>(k.n_chunks) * units * 8;  // + the two per-unit tables
+  auto smem_with = [&](int bufs) {
+    return kHeaderBytes + bufs * static_cast<size_t>(units / 2) * kRows * 16 + static_cast<size_t>(cores_of(r.kh, r.C)) * k.n_pad * 16 +
+           static_cast<size_t>(k.n_chunks) * units * 8;  // + the two per-unit tables
+  };
+  auto ctas_with = [&](int bufs) {
+    int n = static_cast<int>((227 * 1024) / (smem_with(bufs) + 1024));
+    const int cap = units == 8 ? 4 : 3;  // the register file
+    return n > cap ? cap : n;
+  };
+  // a third operand buffer lets the gather run further ahead, unless it costs a resident CTA (3 x 3 64 -> 64 on 56 x 56:
+  // 0.227 ms with two buffers and two CTAs per SM, 0.256 ms with three and one)
+  k.a_bufs = ctas_with(kABufs) >= ctas_with(2) ? kABufs : 2;
+  const size_t smem = smem_with(k.a_bufs);
   if (!attr_set) {
     cudaError_t e = cudaSuccess;
     // tables: at most 1/16 of the weights (n_pad >= 16)
-    const int bytes = kHeaderBytes + 2 * (kMaxUnits / 2) * kRows * 16 + kMaxWeightBytes + kMaxWeightBytes / 16;
+    const int bytes = kHeaderBytes + kABufs * (kMaxUnits / 2) * kRows * 16 + kMaxWeightBytes + kMaxWeightBytes / 16;
 #define GI_CK_ATTR(A, T)                                                                                                             \
   do {                                                                                                                               \
     if (e == cudaSuccess) e = cudaFuncSetAttribute(conv_kxk_tc_kernel<8, A, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);  \
@@ -451,12 +467,12 @@ int launch_conv_kxk_tc(const LaunchRec& r, const Ptrs& p, void* stream) {
     if (e != cudaSuccess) return static_cast<int>(e);
     attr_set = true;
   }
-  // a few CTAs per SM: one CTA's gather latency hides behind another's epilogue; tensor memory allows
-  // 512 / tmem_cols of them, shared memory 227 KB / smem, the register file four (six with 8-unit chunks)
+  // a few CTAs per SM: tensor memory allows 512 / tmem_cols of them, shared memory 227 KB / smem, the register file
+  // three (four with 8-unit chunks)
   int per_sm = static_cast<int>(512u / cols);
   const int by_smem = static_cast<int>((227 * 1024) / (smem + 1024));
   if (per_sm > by_smem) per_sm = by_smem;
-  if (per_sm > (units == 8 ? 6 : 4)) per_sm = units == 8 ? 6 : 4;
+  if (per_sm > (units == 8 ? 4 : 3)) per_sm = units == 8 ? 4 : 3;
   if (per_sm < 1) per_sm = 1;
   // the grid is a whole number of CTAs per group
   long long per_group = static_cast<long long>(sms) * per_sm / k.n_groups;
