@@ -240,7 +240,11 @@ GI_API void gi_graph_destroy(gi_graph* g);
  * no copy: its inputs are placed inside its output (the slices of a tensor follow one another in memory,
  * Section 4), their producers write there, and the CONCAT launches nothing (GI_KERNEL_NONE).
  * Host work only; no CUDA call is made.
- * `opt` may be NULL for defaults.  The graph stays valid and may be compiled again. */
+ * `opt` may be NULL for defaults.  The graph stays valid and may be compiled again.
+ * Two tables generated from measurements on the device (the counterpart of the paper's table of optimal work-group sizes,
+ * Section 4) are consulted: which 1x1 kernel runs a shape, and how much the depthwise stencil stages at a time.  The
+ * environment variables GI_DW_BUF_KB and GI_DW_CTA_KB, read here, override the second table for every depthwise operator of
+ * the graph (largest staging buffer and shared memory of one CTA, in KB); they exist for the tuner that generates it. */
 GI_API gi_status gi_compile(const gi_graph* g, const gi_compile_options* opt, gi_exec** out);
 
 GI_API gi_status gi_exec_query(const gi_exec* e, gi_exec_info* info);
