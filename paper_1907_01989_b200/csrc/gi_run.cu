@@ -106,7 +106,7 @@ static gi_status run_impl(gi_exec* e, const void* const* dev_inputs, void* const
       case GI_KERNEL_DEPTHWISE: err = launch_depthwise(r, p, e->storage, stream); break;
       case GI_KERNEL_DEPTHWISE_POINTWISE: err = launch_depthwise_pointwise(r, p, stream); break;
       case GI_KERNEL_INVERTED_RESIDUAL: err = launch_inverted_residual(r, p, stream); break;
-      case GI_KERNEL_POINTWISE_MM: err = launch_pointwise_mm(r, p, stream); break;
+      case GI_KERNEL_POINTWISE_MM: err = launch_pointwise_mm(r, p, &e->tc_state, static_cast<int>(i), stream); break;
       case GI_KERNEL_POINTWISE_CHAIN: err = launch_pointwise_chain(r, p, &e->tc_state, static_cast<int>(i), stream); break;
       case GI_KERNEL_NONE: break;  // computed by the previous launch
       case GI_KERNEL_ELTWISE:

@@ -81,7 +81,7 @@ unsigned int depthwise_pointwise_error_word(int* cuda_err);
 // streamed (pointwise_mm.cu; fp16 storage)
 bool pointwise_mm_supported(int cin, int cout);
 void pointwise_mm_pack(const float* w, const float* bias, int cin, int cout, std::vector<uint8_t>* blob, LaunchRec* r);
-int launch_pointwise_mm(const LaunchRec& r, const Ptrs& p, void* stream);
+int launch_pointwise_mm(const LaunchRec& r, const Ptrs& p, void** state, int launch_index, void* stream);
 unsigned int pointwise_mm_error_word(int* cuda_err);
 
 // Two consecutive 1x1 convolutions (a block's projection and the next block's expansion) as one kernel (fp16 storage):

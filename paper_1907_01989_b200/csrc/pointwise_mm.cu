@@ -5,9 +5,13 @@
 // byte instead: a CTA tile is 256 pixels x up to 256 output channels (128 flops per byte), every weight chunk
 // fetched is used for two 128-row MMAs, and the K axis streams through a ring of stages:
 //
-//   A chunk  256 pixels x 32 channels, copied straight from the channel-sliced tensor into the canonical K-major
-//            operand layout by 8-byte cp.async (two 4-channel slices interleave into one 16-byte operand row):
-//            exactly 2*M*N*K flops, nothing padded or duplicated
+//   A chunk  256 pixels x 32 channels: one tiled TMA copy lands the eight 4-channel slices as they lie in memory
+//            ([slice][pixel] 8-byte pixel-slices); eight warps then interleave pairs of slices into the canonical
+//            K-major operand rows (16 bytes = 8 channels of one pixel) in place - a K group's 4 KB of operand rows
+//            lie exactly where its two slices landed, so one warp owns a K group and needs no barrier but its own.
+//            Exactly 2*M*N*K flops, nothing padded or duplicated.  (Gathering the rows with 8-byte cp.async
+//            instead - every copy holds a first-level cache line while in flight - fed a chunk in twice the time
+//            its four MMAs take: 892 TFLOP/s on 1280 -> 1280 where this path does better than 1300.)
 //   B chunk  up to 256 output channels x 32 input channels of the dense weight matrix, packed at compile time,
 //            one bulk copy
 //   MMA      2 x 2 tcgen05.mma (M = 128, N = tile width, K = 16) per chunk into two accumulators that together fill
@@ -25,6 +29,7 @@
 #include "kernels.h"
 #include "pdl.cuh"
 #include "sm100_ptx.cuh"
+#include "tma_host.h"
 
 namespace gi {
 namespace {
@@ -33,19 +38,19 @@ using namespace ptx;
 
 constexpr int kRows = 256;        // pixels per CTA tile: two MMAs of 128 rows
 constexpr int kKc = 8;            // input slices (32 channels) per chunk: small chunks, many stages in flight
-constexpr int kLoadWarps = 4, kDrainWarps = 16;
-constexpr int kLoadThreads = 32 * kLoadWarps;
-constexpr int kMmaWarps = 2;      // one issuing thread per 128-row accumulator: the issue stream, not the pipe, bounds a chunk
-constexpr int kFirstLoad = 1 + kMmaWarps, kFirstDrain = kFirstLoad + kLoadWarps;
+constexpr int kRepackWarps = 8, kDrainWarps = 16;  // repack: four warps (one per K group) on even chunks, four on odd ones
+constexpr int kMmaWarps = 2;      // one issuing thread per 128-row accumulator
+constexpr int kTmaWarp = 1 + kMmaWarps;  // activation copies
+constexpr int kFirstRepack = kTmaWarp + 1, kFirstDrain = kFirstRepack + kRepackWarps;
+static_assert(kFirstDrain % 4 == 0, "a drain warp's TMEM lane quarter is its warp index modulo 4");
 constexpr int kThreads = 32 * (kFirstDrain + kDrainWarps);
 constexpr int kMaxStages = 8;
 constexpr int kHeader = 1024;
 constexpr int kABytes = (kKc / 2) * kRows * 16;  // 16 KB
 constexpr int kSmemMax = 227 * 1024;
-constexpr int kAhead = 3;         // chunks a loader thread keeps in flight before it waits for the oldest
 
 __device__ unsigned int g_mm_error = 0;
-enum : unsigned { kErrCopy = 1u, kErrMma = 2u, kErrLoad = 4u, kErrDrain = 8u };
+enum : unsigned { kErrCopy = 1u, kErrMma = 2u, kErrLoad = 4u, kErrDrain = 8u, kErrRepack = 16u };
 
 struct MmParams {
   const __half* in;
@@ -63,7 +68,8 @@ struct MmParams {
 };
 
 struct Header {
-  unsigned long long full[kMaxStages], empty[kMaxStages];  // full: the load threads' arrivals and the weight copy's bytes
+  unsigned long long landed[kMaxStages];  // both copies of a stage (activations as they lie in memory, weights) have arrived
+  unsigned long long full[kMaxStages], empty[kMaxStages];  // full: the four repack warps of the chunk are done
   unsigned long long acc_full, acc_empty;
   unsigned tmem_addr, abort_flag;
 };
@@ -74,19 +80,13 @@ __device__ __forceinline__ float act1(float v, int kind) {
   if (kind == GI_ACT_RELU6) return fminf(fmaxf(v, 0.0f), 6.0f);
   return v;
 }
-// 8-byte asynchronous copy; with `bytes` = 0 nothing is read and the destination is filled with zeros
-__device__ __forceinline__ void cp_async8_zfill(unsigned dst, const void* src, unsigned bytes) {
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait_pending() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+__device__ __forceinline__ void st_shared_v4(unsigned addr, unsigned a, unsigned b, unsigned c, unsigned d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
 // ACT: activation right after the bias; TAIL: a residual add and / or a second activation follow
 template <int ACT, bool TAIL>
-__global__ void __launch_bounds__(kThreads, 1) pointwise_mm_kernel(const MmParams p) {
+__global__ void __launch_bounds__(kThreads, 1) pointwise_mm_kernel(const __grid_constant__ CUtensorMap tmap_a, const MmParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   Header* hdr = reinterpret_cast<Header*>(smem);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -96,7 +96,8 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_mm_kernel(const MmParam
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < p.stages; ++i) {
-      mbar_init(smem_u32(&hdr->full[i]), kLoadThreads + 1);
+      mbar_init(smem_u32(&hdr->landed[i]), 2);
+      mbar_init(smem_u32(&hdr->full[i]), kRepackWarps / 2);
       mbar_init(smem_u32(&hdr->empty[i]), kMmaWarps);
     }
     mbar_init(smem_u32(&hdr->acc_full), kMmaWarps);
@@ -106,6 +107,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_mm_kernel(const MmParam
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) tmem_alloc(smem_u32(&hdr->tmem_addr), 512u);
+  if (warp == kTmaWarp && lane == 0) prefetch_tensormap(&tmap_a);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -125,16 +127,16 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_mm_kernel(const MmParam
             ok = false;
             break;
           }
-          const unsigned full = smem_u32(&hdr->full[stage]);
-          mbar_expect_tx(full, p.b_bytes);
-          bulk_load(st0 + stage * p.stage_bytes + kABytes, p.wts + (static_cast<size_t>(nt) * p.n_chunks + c) * p.b_bytes, p.b_bytes, full);
+          const unsigned landed = smem_u32(&hdr->landed[stage]);
+          mbar_expect_tx(landed, p.b_bytes);
+          bulk_load(st0 + stage * p.stage_bytes + kABytes, p.wts + (static_cast<size_t>(nt) * p.n_chunks + c) * p.b_bytes, p.b_bytes, landed);
         }
       }
       if (!ok) {
         const unsigned first = it > static_cast<unsigned>(p.stages) ? it - p.stages : 0u;
         for (unsigned j = first; j < it; ++j) {
           const unsigned long long t0 = global_timer_ns();
-          while (!mbar_try_wait(smem_u32(&hdr->full[j % p.stages]), (j / p.stages) & 1u)) {
+          while (!mbar_try_wait(smem_u32(&hdr->landed[j % p.stages]), (j / p.stages) & 1u)) {
             if (global_timer_ns() - t0 > p.timeout_ns) {
               atomicOr(&g_mm_error, kErrDrain);
               break;
@@ -143,7 +145,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_mm_kernel(const MmParam
         }
       }
     }
-  } else if (warp < kFirstLoad) {
+  } else if (warp < kTmaWarp) {
     // ------------------------------------------------------------ MMA issuers: warp 1 owns accumulator 0 (rows 0-127 of
     // the tile), warp 2 accumulator 1; both read the same stages and each hands a stage back with its own commit
     if (lane == 0) {
@@ -181,54 +183,75 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_mm_kernel(const MmParam
         if (ok) umma_commit(smem_u32(&hdr->acc_full));
       }
     }
-  } else if (warp < kFirstDrain) {
-    // ------------------------------------------------------------ activation chunks: 8-byte cp.async into the operand layout
-    const int tid = threadIdx.x - 32 * kFirstLoad;  // 0 .. 127: rows tid and tid + 128 of the tile
-    pdl_wait();  // activations are read only below
-    unsigned it = 0, signalled = 0;
-    bool ok = true;
-    // chunk number j (of this CTA's sequence) has landed for this thread: make it visible to the tensor core's
-    // proxy and count this thread in
-    auto publish = [&](unsigned j) {
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      mbar_arrive(smem_u32(&hdr->full[j % p.stages]));
-    };
-    for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-      const int mt = u / p.n_tiles;
-      const unsigned px0 = static_cast<unsigned>(mt) * kRows + static_cast<unsigned>(tid);
-      for (int c = 0; c < p.n_chunks; ++c, ++it) {
-        const unsigned stage = it % p.stages, phase = (it / p.stages) & 1u;
-        if (!mbar_wait(smem_u32(&hdr->empty[stage]), phase ^ 1u, abort_flag, p.timeout_ns, &g_mm_error, kErrLoad)) {
-          ok = false;
-          break;
-        }
-        const unsigned dst0 = st0 + stage * p.stage_bytes + static_cast<unsigned>(tid) * 16u;
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const unsigned px = px0 + static_cast<unsigned>(h) * 128u;
-          const bool px_ok = px < p.m_total;
-          const __half* src = p.in + (static_cast<size_t>(c * kKc) * p.m_total + (px_ok ? px : 0u)) * 4;
-          const unsigned dst = dst0 + static_cast<unsigned>(h) * 2048u;
-#pragma unroll
-          for (int s = 0; s < kKc; ++s) {
-            // slices beyond the tensor's last one and pixels beyond its end read nothing and are filled with zeros
-            const bool live = px_ok && c * kKc + s < p.s_in;
-            cp_async8_zfill(dst + static_cast<unsigned>(s >> 1) * (kRows * 16u) + static_cast<unsigned>(s & 1) * 8u,
-                            live ? static_cast<const void*>(src + static_cast<size_t>(s) * p.m_total * 4) : static_cast<const void*>(p.in),
-                            live ? 8u : 0u);
+  } else if (warp == kTmaWarp) {
+    // ------------------------------------------------------------ activation chunks: one tiled copy of 256 pixels x 8 slices
+    // each; pixels beyond the tensor's end and slices beyond its last one read as zeros
+    if (lane == 0) {
+      pdl_wait();  // the activations are the previous kernel's output
+      unsigned it = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+        const int mt = u / p.n_tiles;
+        for (int c = 0; c < p.n_chunks; ++c, ++it) {
+          const unsigned stage = it % p.stages, phase = (it / p.stages) & 1u;
+          if (!mbar_wait_parked(smem_u32(&hdr->empty[stage]), phase ^ 1u, abort_flag, p.timeout_ns, &g_mm_error, kErrLoad)) {
+            ok = false;
+            break;
           }
+          const unsigned landed = smem_u32(&hdr->landed[stage]);
+          mbar_expect_tx(landed, kABytes);
+          tma_load_2d(st0 + stage * p.stage_bytes, &tmap_a, mt * kRows, c * kKc, landed);
         }
-        cp_async_commit();
-        if (it >= static_cast<unsigned>(kAhead)) {
-          cp_async_wait_pending<kAhead>();
-          publish(signalled++);
+      }
+      if (!ok) {
+        // copies in flight must land before the CTA leaves
+        const unsigned first = it > static_cast<unsigned>(p.stages) ? it - p.stages : 0u;
+        for (unsigned j = first; j < it; ++j) {
+          const unsigned long long t0 = global_timer_ns();
+          while (!mbar_try_wait(smem_u32(&hdr->landed[j % p.stages]), (j / p.stages) & 1u)) {
+            if (global_timer_ns() - t0 > p.timeout_ns) {
+              atomicOr(&g_mm_error, kErrDrain);
+              break;
+            }
+          }
         }
       }
     }
-    // the last chunks in flight
-    cp_async_wait_pending<0>();
-    if (ok)
-      while (signalled < it) publish(signalled++);
+  } else if (warp < kFirstDrain) {
+    // ------------------------------------------------------------ landing layout -> operand layout, in place.  Landed:
+    // [slice][pixel] 8-byte pixel-slices (2 KB per slice); operand: [K group of 8 channels][pixel] 16-byte rows (4 KB
+    // per K group) - K group g takes the place of slices 2g and 2g+1.  A warp owns one K group of every second chunk:
+    // it reads the group's 512 pixel-slices into registers, and only then writes its 256 rows.
+    const int rw = warp - kFirstRepack;
+    const unsigned kg = static_cast<unsigned>(rw & 3), parity = static_cast<unsigned>(rw >> 2);
+    unsigned it = 0;
+    bool ok = true;
+    for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+      for (int c = 0; c < p.n_chunks; ++c, ++it) {
+        if ((it & 1u) != parity) continue;
+        const unsigned stage = it % p.stages, phase = (it / p.stages) & 1u;
+        if (!mbar_wait_warp(smem_u32(&hdr->landed[stage]), phase, abort_flag, p.timeout_ns, &g_mm_error, kErrRepack)) {
+          ok = false;
+          break;
+        }
+        const unsigned base = st0 + stage * p.stage_bytes + kg * 4096u;
+        unsigned lo[8][2], hi[8][2];  // pixel-slices of the even and of the odd slice, pixels lane, lane + 32, ...
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const unsigned px = static_cast<unsigned>(lane + 32 * j);
+          asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(lo[j][0]), "=r"(lo[j][1]) : "r"(base + px * 8u) : "memory");
+          asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(hi[j][0]), "=r"(hi[j][1]) : "r"(base + 2048u + px * 8u) : "memory");
+        }
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          st_shared_v4(base + static_cast<unsigned>(lane + 32 * j) * 16u, lo[j][0], lo[j][1], hi[j][0], hi[j][1]);
+        // visible to the tensor core's proxy, then count this warp in
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&hdr->full[stage]));
+      }
+    }
   } else {
     // ------------------------------------------------------------ drain: accumulators -> global memory
     const int dw = warp - kFirstDrain;
@@ -330,7 +353,7 @@ Tiling choose_tiling(int cin, int cout) {
 
 bool pointwise_mm_supported(int cin, int cout) {
   if (cin <= 0 || cout <= 0) return false;
-  return choose_tiling(cin, cout).stages > kAhead;  // the loaders keep kAhead chunks in flight behind the one they fill
+  return choose_tiling(cin, cout).stages >= 3;
 }
 
 // Dense weights as the B operand, per (output tile, K chunk): [4 K groups][n_tile rows][8 halves]; entries beyond
@@ -361,7 +384,7 @@ void pointwise_mm_pack(const float* w, const float* bias, int cin, int cout, std
   r->tc_stages = t.stages;
 }
 
-int launch_pointwise_mm(const LaunchRec& r, const Ptrs& p, void* stream) {
+int launch_pointwise_mm(const LaunchRec& r, const Ptrs& p, void** state, int launch_index, void* stream) {
   const Tiling t = choose_tiling(r.C, r.Co);
   MmParams k{};
   k.in = static_cast<const __half*>(p.in0);
@@ -399,6 +422,13 @@ int launch_pointwise_mm(const LaunchRec& r, const Ptrs& p, void* stream) {
     if (e != cudaSuccess) return static_cast<int>(e);
     attr_done = true;
   }
+  CUtensorMap tmap;
+  {
+    const int err = map_cache_lookup(state, launch_index, p.in0, &tmap, [&](CUtensorMap* m) {
+      return encode_plane_map(m, p.in0, k.m_total, t.s_in, kRows, kKc);
+    });
+    if (err != 0) return err;
+  }
   const long long units = static_cast<long long>(k.m_tiles) * k.n_tiles;
   const int sms = device_sm_count();
   const unsigned grid = static_cast<unsigned>(units < sms ? units : sms);
@@ -407,7 +437,7 @@ int launch_pointwise_mm(const LaunchRec& r, const Ptrs& p, void* stream) {
   if (smem < 120 * 1024) smem = 120 * 1024;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool tail = k.has_res || k.act_post != GI_ACT_NONE;
-#define GI_MM_LAUNCH(A, T) launch_pdl(pointwise_mm_kernel<A, T>, grid, kThreads, smem, st, k)
+#define GI_MM_LAUNCH(A, T) launch_pdl(pointwise_mm_kernel<A, T>, grid, kThreads, smem, st, tmap, k)
   if (tail) {
     if (k.act_pre == GI_ACT_RELU6) GI_MM_LAUNCH(GI_ACT_RELU6, true);
     else if (k.act_pre == GI_ACT_RELU) GI_MM_LAUNCH(GI_ACT_RELU, true);
