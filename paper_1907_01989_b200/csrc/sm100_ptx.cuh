@@ -206,6 +206,166 @@ __device__ __forceinline__ void tmem_ld_wait16(unsigned* r) {
                : "memory");
 }
 
+// true in exactly one lane of a converged warp
+__device__ __forceinline__ bool elect_one() {
+  unsigned pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
+
+// ---- CTA pairs (a cluster of two CTAs on the two SMs that share one tensor-core pair) -------------------------
+__device__ __forceinline__ unsigned cluster_ctarank() {
+  unsigned r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// hardware barrier over all threads of the cluster; every thread of both CTAs must reach it
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// the address of `addr` (a shared-memory address of this CTA) in CTA `rank` of the cluster
+__device__ __forceinline__ unsigned mapa_shared(unsigned addr, unsigned rank) {
+  unsigned r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+// arrive on an mbarrier of any CTA of the cluster; what this thread wrote before is visible to the waiter
+__device__ __forceinline__ void mbar_arrive_cluster(unsigned cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// poll an mbarrier of this CTA that the other CTA of the pair arrives on
+__device__ __forceinline__ bool mbar_try_wait_cluster(unsigned bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Non-blocking tests of a phase (try_wait may suspend the thread for a while when the phase is not complete):
+// for a thread that has other work to issue first and looks at the answer later.
+__device__ __forceinline__ bool mbar_test_wait(unsigned bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_test_wait_cluster(unsigned bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// bounded wait on such a barrier (same contract as mbar_wait)
+static __device__ __noinline__ bool mbar_wait_cluster_slow(unsigned bar, unsigned parity, volatile unsigned* abort_flag, unsigned timeout_ns,
+                                                    unsigned* error_word, unsigned code) {
+  unsigned long long t0 = 0;
+  for (unsigned spin = 0;; ++spin) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    if ((spin & 255u) == 255u) {
+      if (*abort_flag) return false;
+      const unsigned long long now = global_timer_ns();
+      if (t0 == 0) {
+        t0 = now;
+      } else if (now - t0 > timeout_ns) {
+        *abort_flag = 1;
+        atomicOr(error_word, code);
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ bool mbar_wait_cluster(unsigned bar, unsigned parity, volatile unsigned* abort_flag, unsigned timeout_ns,
+                                                  unsigned* error_word, unsigned code) {
+  if (mbar_try_wait_cluster(bar, parity)) return true;
+  return mbar_wait_cluster_slow(bar, parity, abort_flag, timeout_ns, error_word, code);
+}
+__device__ __forceinline__ bool mbar_wait_cluster_warp(unsigned bar, unsigned parity, volatile unsigned* abort_flag, unsigned timeout_ns,
+                                                       unsigned* error_word, unsigned code) {
+  const bool ok = mbar_wait_cluster(bar, parity, abort_flag, timeout_ns, error_word, code);
+  return __all_sync(0xffffffffu, ok) != 0;
+}
+// The parked form of that wait (see mbar_wait_parked): each poll may sleep in hardware for up to a microsecond
+// and returns as soon as the phase completes.  For roles that wait most of the time - a warp that spins on a
+// barrier floods the shared-memory pipeline that also feeds the tensor core its operands.
+static __device__ __noinline__ bool mbar_wait_cluster_parked(unsigned bar, unsigned parity, volatile unsigned* abort_flag, unsigned timeout_ns,
+                                                      unsigned* error_word, unsigned code) {
+  unsigned long long t0 = 0;
+  for (unsigned spin = 0;; ++spin) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(1000u)
+        : "memory");
+    if (ok) return true;
+    if ((spin & 15u) == 15u) {
+      if (*abort_flag) return false;
+      const unsigned long long now = global_timer_ns();
+      if (t0 == 0) {
+        t0 = now;
+      } else if (now - t0 > timeout_ns) {
+        *abort_flag = 1;
+        atomicOr(error_word, code);
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ bool mbar_wait_cluster_parked_warp(unsigned bar, unsigned parity, volatile unsigned* abort_flag,
+                                                              unsigned timeout_ns, unsigned* error_word, unsigned code) {
+  const bool ok = mbar_wait_cluster_parked(bar, parity, abort_flag, timeout_ns, error_word, code);
+  return __all_sync(0xffffffffu, ok) != 0;
+}
+__device__ __forceinline__ bool mbar_wait_parked_warp(unsigned bar, unsigned parity, volatile unsigned* abort_flag, unsigned timeout_ns,
+                                                      unsigned* error_word, unsigned code) {
+  const bool ok = mbar_wait_parked(bar, parity, abort_flag, timeout_ns, error_word, code);
+  return __all_sync(0xffffffffu, ok) != 0;
+}
+// Tensor memory of both CTAs of a pair, same columns in each: one warp of EACH CTA executes these
+__device__ __forceinline__ void tmem_alloc_pair(unsigned smem_dst, unsigned cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(unsigned taddr, unsigned cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// D (+)= A * B^T over the pair, 256 x N x 16: each CTA supplies 128 rows of A and N/2 rows of B from its own shared
+// memory (same offsets in both) and receives its 128 rows of D in its own tensor memory.  Issued by one thread of
+// the pair's first CTA.
+__device__ __forceinline__ void umma_pair_f16(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc, unsigned idesc,
+                                              unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrive on an mbarrier of either CTA (cluster address) once every pair MMA issued so far by this thread has completed
+__device__ __forceinline__ void umma_pair_commit(unsigned cluster_addr) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_addr) : "memory");
+}
 
 }  // namespace ptx
 }  // namespace gi
