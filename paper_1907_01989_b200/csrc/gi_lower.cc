@@ -454,16 +454,16 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
           const bool lane_rule = op.d.cout >= 96 && din->c >= 64 && din->c < 960 && !(din->c <= 96 && op.d.cout >= 4 * din->c);
           const bool lane_auto = one_wave || lane_rule;
           const bool lane_kernel = e->opt.pointwise == GI_PW_TC_LANE || ((e->opt.pointwise == GI_PW_AUTO || e->opt.pointwise == GI_PW_RULE) && lane_auto);
-          // The wide-tile kernel (256 pixels x up to 256 output channels per CTA) is for the shapes bound by the tensor
-          // pipe: at least 512 input and 512 output channels.  Measured against the library's previous choice at batch
-          // 256 (time wide / time before): 14x14 1280->1280 0.57, 960->960 0.72, 576->576 0.76, 7x7 1024->1024 0.83,
-          // 14x14 512->512 0.96; but 7x7 512->1024 1.07 and 14x14 512->512 at batch 64 1.10, where the 256 x 256 tiles
-          // leave the last wave of CTAs two thirds empty - with 512 input channels it therefore needs well-filled waves
-          // (148 SMs).  Narrower layers lose 10-25 % to it: their tiles are short and its drain is not overlapped.
+          // The wide-tile kernel (a CTA pair per tile of 256 pixels x up to 256 output channels) is for the layers with many
+          // input channels: at least 512.  Measured against the better of the other two kernels at batch 256 (time wide /
+          // time other): 7x7 1024->1024 0.56, 14x14 512->512 0.76, 7x7 512->1024 0.80, 960->160 0.82, 960->320 0.95,
+          // 576->160 0.93; batch 64: 14x14 512->512 0.90, 576->96 0.88, 7x7 1024->1024 0.72.  It loses where a launch has
+          // too few tiles to fill the 74 pairs' pipelines (batch 64 7x7 960->160, 13 tiles: 1.14) and where many tiles
+          // meet a narrow output (batch 256 14x14 576->96, 196 tiles: 1.09 - an MMA takes the same 128 cycles for 96
+          // output channels as for 256).  From 256 input and 256 output channels on it is 4-14 % ahead (28x28 256->256,
+          // 7x7 320->1280); with fewer channels it wins or loses by a few per cent: the table decides.
           const long long mm_units = ((m_px_all_for_mm(e, din) + 255) / 256) * ((slices(op.d.cout) * 4 + 255) / 256);
-          const long long mm_waves = (mm_units + 147) / 148;
-          const bool mm_auto = din->c >= 512 && op.d.cout >= 512 && mm_units >= 64 &&
-                               (din->c >= 576 || mm_units * 100 >= mm_waves * 148 * 85);
+          const bool mm_auto = mm_units >= 40 && ((din->c >= 512 && (op.d.cout >= 160 || mm_units <= 74)) || (din->c >= 256 && op.d.cout >= 256));
           bool wide_kernel = e->opt.pointwise == GI_PW_TC_WIDE || ((e->opt.pointwise == GI_PW_AUTO || e->opt.pointwise == GI_PW_RULE) && mm_auto);
           bool lane_tab = false, pair_tab = false;
           if (e->opt.pointwise == GI_PW_AUTO && pointwise && tc) {

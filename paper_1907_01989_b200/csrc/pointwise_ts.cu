@@ -39,6 +39,7 @@ using namespace ptx;
 constexpr int kRows = 128;
 constexpr int kTransferWarps = 8;  // two per TMEM lane quarter: each moves every other group of 8 slices of a chunk
 constexpr int kDrainWarps = 16;
+constexpr int kMaxNCta = 256;  // output channels per CTA: two accumulators and the A buffers share the 512 TMEM columns
 constexpr int kThreads = 32 * (2 + kTransferWarps + kDrainWarps);
 constexpr int kMaxStages = 8;
 constexpr int kSmemHeader = 1024;
@@ -301,6 +302,16 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
     const int part_id = (warp - (2 + kTransferWarps)) >> 2;     // takes every kParts-th 16-column group
     const unsigned lane_bits = static_cast<unsigned>(quarter * 32) << 16;
     const int groups = p.n_cta >> 4;
+    // This CTA's output channels are the same for every tile: lane l keeps the bias of column l % 16 of each of this
+    // warp's 16-column groups and the epilogue broadcasts from there.  (A load from global memory per slice inside the
+    // epilogue queues behind the barrier polls and shared-memory traffic of the other warps.)
+    constexpr int kGroupsPerWarp = (kMaxNCta / 16 + kParts - 1) / kParts;
+    float bpre[kGroupsPerWarp];
+#pragma unroll
+    for (int k = 0; k < kGroupsPerWarp; ++k) {
+      const int g = part_id + k * kParts;
+      bpre[k] = g < groups ? __ldg(p.bias + n_part * p.n_cta + g * 16 + (lane & 15)) : 0.f;
+    }
     unsigned tile = 0;
     for (int m = m_first; m < p.m_tiles; m += m_step, ++tile) {
       const unsigned acc = tile & 1u, acc_phase = (tile >> 1) & 1u;
@@ -323,7 +334,10 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
       tc_fence_after();
       if (tile == 0 && threadIdx.x == 32 * (2 + kTransferWarps)) GI_TRACE_EVENT(g_ts_trace, 6);
       const unsigned t_addr = tmem_base + lane_bits + acc * acc_cols;
-      for (int g = part_id; g < groups; g += kParts) {
+#pragma unroll
+      for (int k = 0; k < kGroupsPerWarp; ++k) {
+        const int g = part_id + k * kParts;
+        if (g >= groups) break;
         if (TAIL) fetch_res(res_next, g + kParts);
         unsigned r[16];
         tmem_ld16(t_addr + g * 16, r);
@@ -331,8 +345,12 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int so = (n_part * p.n_cta) / 4 + g * 4 + j;
+          float4 b;
+          b.x = __shfl_sync(0xffffffffu, bpre[k], 4 * j);
+          b.y = __shfl_sync(0xffffffffu, bpre[k], 4 * j + 1);
+          b.z = __shfl_sync(0xffffffffu, bpre[k], 4 * j + 2);
+          b.w = __shfl_sync(0xffffffffu, bpre[k], 4 * j + 3);
           if (so >= p.s_out || !px_ok) continue;
-          const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias) + so);
           const size_t off = (static_cast<size_t>(so) * p.m_total_px + pixel) * 4;  // in halves
           const float2 v0 = __fadd2_rn(make_float2(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1])), make_float2(b.x, b.y));
           const float2 v1 = __fadd2_rn(make_float2(__uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3])), make_float2(b.z, b.w));
