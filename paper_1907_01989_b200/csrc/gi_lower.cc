@@ -375,12 +375,13 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
           // Launches whose pixels all fit one wave of 128-pixel tiles are latency-bound and take the lane
           // kernel (shorter fill; MobileNetV2 batch 1 0.296 -> 0.276 ms) - up to 64 tiles always, up to one
           // tile per SM unless the input is 960 channels deep or more.
-          // Whole inverted-residual block as one kernel.  The library's own choice (GI_XOP_AUTO) follows an A/B of
-          // MobileNetV2 at batch 256 on one B200, both builds alternating in one call: with the two 7x7 blocks that
-          // qualify as one kernel each the step takes 1.549 ms against 1.552 ms; with the 14x14 blocks as well it is 2.5 %
-          // slower (alone, L2 flushed, a 14x14 block takes 55-88 us as one kernel against 48-65 us as three; a 7x7
-          // block 55-66 against 56).  So: planes of at most 64 pixels, and at least about one unit of work per SM - below
-          // that (batch 1) three kernels that each spread over all SMs are faster.
+          // Whole inverted-residual block as one kernel: only on request (GI_XOP_ON).  The library's own choice
+          // (GI_XOP_AUTO) follows A/Bs of MobileNetV2 at batch 256 on one B200.  With the 14x14 blocks as one kernel each
+          // the step is 2.5 % slower (alone, L2 flushed, a 14x14 block takes 55-88 us as one kernel against 48-65 us as
+          // three).  The two 7x7 blocks that qualify were a tie (1.549 against 1.552 ms) until the 1x1 kernels around
+          // them got faster - the CTA-pair kernel on 960 -> 160, the lane-per-pixel kernel's drain on 160 -> 960; now
+          // three kernels per block win: 1.450 ms against 1.469 ms with the blocks fused (55 us each, bound by their own
+          // instruction stream).
           long long ir_units = 0;
           if (pointwise && tc && e->opt.fuse && e->opt.cross_op != GI_XOP_OFF && block_follows(g, e, i)) {
             const FusedOp& fd = e->ops[i + 1];
@@ -390,7 +391,7 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
             const TensorDesc& dd = e->tensors[fd.out];
             if (inverted_residual_supported(e->batch, din->h, din->w, dd.h, dd.w, dwn.d.stride_h, dwn.d.dilation_h, dwn.d.pad_t,
                                             dwn.d.pad_l, din->c, op.d.cout, pwn.d.cout, &ir_units) &&
-                (e->opt.cross_op == GI_XOP_ON || (ir_units >= 96 && din->h * din->w <= 64))) {
+                e->opt.cross_op == GI_XOP_ON) {
               const TensorDesc& d2 = e->tensors[fp.out];
               r.kernel = GI_KERNEL_INVERTED_RESIDUAL;
               r.Ho = dd.h;
