@@ -111,9 +111,10 @@ enum {
  * memory plan is not affected: those tensors keep their place in the arena, unused; operators whose input and output the
  * planner placed on the same bytes (legal for separate kernels, not for one that reads while it writes) stay separate. */
 enum {
-  GI_XOP_AUTO = 0,  /* the library's choice, from whole-network measurements (default): (1) for blocks on planes of at most
-                       64 pixels (7x7) when the batch gives at least 96 work units; never (2), which has not measured
-                       faster than the two kernels on any layer of the benchmark networks */
+  GI_XOP_AUTO = 0,  /* the library's choice, from whole-network measurements (default): (3) for seams on planes of 65 to 256
+                       pixels with at most 64 channels between the two convolutions, at least 192 into the first and two
+                       pixel tiles per SM; never (1) or (2), which have not measured faster than separate kernels inside
+                       the benchmark networks */
   GI_XOP_OFF = 1,   /* one kernel per fused op */
   GI_XOP_ON = 2,    /* (1) wherever the block kernel supports the three ops, else (2) wherever the pair kernel does */
   GI_XOP_CHAIN = 3  /* (3) wherever that kernel supports the two ops; neither (1) nor (2) */
