@@ -433,6 +433,89 @@ def run_sweep(args):
                          f"{r['frac_of_roofline']}\n")
 
 
+def run_slice8_sweep(args):
+    """The layout comparison (slices of 8 channels against the library's slices of 4) on single 1x1 layers: the same
+    seeded layer and images through (a) the library's own kernel choice on PHWC4 tensors, (b) the wide-tile kernel on
+    PHWC4 tensors (tiled copy + rearrangement in shared memory), (c) the wide-tile kernel on tensors stored in slices of
+    8 channels (gi_slice8_pointwise_run: the tiled copy lands operand rows directly).  Timing and checking as in
+    run_sweep: CUDA event pair per launch, L2 flushed before each, sampled images against the oracle."""
+    import torch
+    from paper_1907_01989_b200 import api
+    from paper_1907_01989_b200 import workloads as wl
+    from oracle import graph as og
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+    points = ([tuple(int(v) for v in pt.split(",")) for pt in args.points.split(";") if pt] if args.points else
+              [(256, 14, 512, 512), (256, 14, 1280, 1280), (256, 28, 256, 256), (256, 7, 960, 320)])
+
+    def sliced(x, width, total_halves):  # layout only: [B,H,W,C] -> [S][B][plane][width], zero filled
+        B_, H_, W_, C_ = x.shape
+        S_, P_ = (C_ + width - 1) // width, (H_ * W_ + 1) // 2 * 2
+        x = torch.nn.functional.pad(x.reshape(B_, H_ * W_, C_), (0, S_ * width - C_, 0, P_ - H_ * W_))
+        flat = x.reshape(B_, P_, S_, width).permute(2, 0, 1, 3).contiguous().reshape(-1)
+        full = torch.zeros(total_halves, dtype=torch.float16, device=dev)
+        full[: flat.numel()] = flat
+        return full
+
+    def image_of(raw, width, b, hw, c, img):  # one image back as [1,H,W,C] fp32 on the host
+        S_, P_ = (c + width - 1) // width, (hw * hw + 1) // 2 * 2
+        a = raw[: S_ * b * P_ * width].reshape(S_, b, P_, width)[:, img, : hw * hw, :]
+        return a.permute(1, 0, 2).reshape(1, hw, hw, S_ * width)[..., :c].float().cpu().numpy()
+
+    def timed(launch):
+        for _ in range(3):
+            launch()
+        ms = []
+        for _ in range(args.iters):
+            flush.zero_()
+            a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            launch()
+            z.record(stream)
+            z.synchronize()
+            ms.append(a.elapsed_time(z))
+        return statistics.median(ms)
+
+    for b, hw, cin, cout in points:
+        spec = wl.single_pointwise(b, hw, cin, cout)
+        n_img = min(b, 8)
+        x_np = wl.make_input(spec, images=list(range(n_img)))
+        x = torch.from_numpy(x_np).to(dev).half().repeat((b + n_img - 1) // n_img, 1, 1, 1)[:b].contiguous()
+        sel = sorted({0, b - 1})
+        ref = og.run(spec, [x_np[[i % n_img for i in sel]]], storage="f16", fused=True)[spec.outputs[0]]
+        flops = 2.0 * b * hw * hw * cin * cout
+
+        def report(layout, kernel, ms, raw, width):
+            worst = 0.0
+            for k, img in enumerate(sel):
+                got, want = image_of(raw, width, b, hw, cout, img), ref[k:k + 1]
+                assert np.isfinite(got).all(), f"{layout}: non-finite output"
+                worst = max(worst, float((np.abs(got - want) / (1e-2 + 1e-2 * np.abs(want))).max()))
+            assert worst <= 1.0, f"{layout}: disagrees with the oracle (normalised error {worst:.3f})"
+            print(json.dumps({"op": f"pw1x1 b{b} {hw}x{hw} {cin}->{cout}", "layout": layout, "kernel": kernel, "ms": round(ms, 5),
+                              "tflops": round(flops / ms / 1e9, 1), "checked": True, "max_error_over_tolerance": round(worst, 4)}), flush=True)
+
+        for mode in ("auto", "wide"):
+            g, _ = api.graph_from_spec(spec, api.GI_F16, io_layout=api.GI_PHWC4, out_layout=api.GI_PHWC4)
+            ex = g.compile(pointwise=PW_MODES[mode])
+            ex.bind(dev)
+            ins = [sliced(x, 4, api.gi_tensor_bytes(b, hw, hw, cin) // 2)]
+            outs = [torch.full((api.gi_tensor_bytes(b, hw, hw, cout) // 2,), float("nan"), dtype=torch.float16, device=dev)]
+            ms = timed(lambda: ex.run(ins, outs, stream))
+            kernel = "+".join(api.KERNEL_NAMES[q.kernel] for q in ex.ops())
+            report("slices of 4 channels, " + ("the library's choice" if mode == "auto" else "wide-tile kernel"), kernel, ms, outs[0], 4)
+        conv = [o for o in spec.ops if o.kind == wl.CONV2D][0]
+        blob = torch.from_numpy(api.gi_slice8_pointwise_pack(conv.weights.reshape(cout, cin), conv.bias)).to(dev)
+        x8 = sliced(x, 8, api.gi_slice8_tensor_bytes(b, hw, hw, cin) // 2)
+        out8 = torch.full((api.gi_slice8_tensor_bytes(b, hw, hw, cout) // 2,), float("nan"), dtype=torch.float16, device=dev)
+        act = {wl.ACT_NONE: api.GI_ACT_NONE, wl.ACT_RELU: api.GI_ACT_RELU, wl.ACT_RELU6: api.GI_ACT_RELU6}[
+            [o for o in spec.ops if o.kind == wl.ACTIVATION][0].act if any(o.kind == wl.ACTIVATION for o in spec.ops) else wl.ACT_NONE]
+        ms = timed(lambda: api.gi_slice8_pointwise_run(x8.data_ptr(), out8.data_ptr(), blob.data_ptr(), b, hw, hw, cin, cout, act, stream))
+        report("slices of 8 channels, wide-tile kernel", "pointwise_mm", ms, out8, 8)
+
+
 def run_host_check(args):
     """The multi-rank plumbing without a GPU: rank and world size from the launcher's environment, a gloo group,
     the batch shard of this rank, and the whole-job throughput from the slowest rank's (synthetic) time."""
@@ -470,8 +553,8 @@ def main():
     ap.add_argument("--per-op", default=None, help="write the per-op timing table to this file")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-batch1", action="store_true", help="skip the batch-1 latency leg (keeps profiler runs short)")
-    ap.add_argument("--sweep", default=None, choices=["pw", "dw", "conv3", "dwpw", "stem", "block", "pair"],
-                    help="time single fused operators instead of a network")
+    ap.add_argument("--sweep", default=None, choices=["pw", "dw", "conv3", "dwpw", "stem", "block", "pair", "slice8"],
+                    help="time single fused operators instead of a network (slice8: the layout comparison on 1x1 layers, points 'B,HW,Cin,Cout;...')")
     ap.add_argument("--points", default=None, help="sweep points 'B,HW,Cin,Cout;...' (pw), 'B,HW,C,stride;...' (dw), "
                     "'B,HW,Cin,Cout,stride;...' (conv3), 'B,HW,C,Cout,stride;...' (dwpw: depthwise then 1x1, see --cross-op), "
                     "'B,HW,Cout;...' (stem: 3x3 stride-2 convolution of a 3-channel NHWC input, read in that layout), "
@@ -493,6 +576,9 @@ def main():
 
     if args.fp16_peak:
         measure_fp16_peak()
+        return
+    if args.sweep == "slice8":
+        run_slice8_sweep(args)
         return
     if args.sweep:
         run_sweep(args)

@@ -323,6 +323,28 @@ GI_API gi_status gi_device_status(uint32_t* flags);
  * counterpart; its engine has no device-side waits.) */
 GI_API gi_status gi_selftest_bounded_wait(uint32_t limit_us, uint32_t* waited_us, int32_t* gave_up, void* stream);
 
+
+/* Layout experiment (not on the inference path): a 1x1 convolution + bias + activation on tensors stored in slices of
+ * EIGHT channels instead of four - [ceil(C/8)][batch][plane][8] fp16, plane = H*W rounded up to even, channels beyond
+ * C and the padding pixel zero.  Section 4, "Data Layout", fixes 4 channels per slice because a texel is 4 values; at
+ * fp16 a 4-channel pixel-slice is 8 bytes, half of the 16 bytes the tensor core reads as one operand row, so the
+ * library's 1x1 kernels either pair pixels or rearrange slices in shared memory.  With 8 channels a pixel-slice IS an
+ * operand row and a tiled copy lands a tile where the MMA reads it.  These three calls run the wide-tile 1x1 kernel
+ * that way, so that the two layouts can be compared on the same layer (bench.py --sweep slice8):
+ *   gi_slice8_pointwise_blob_bytes  bytes of the packed weights + bias of a layer
+ *   gi_slice8_pointwise_pack        packs w[cout][cin] and bias[cout] (host, fp32; weights are rounded to fp16 as in
+ *                                   gi_add_op) into `host_blob`, which the caller copies to the device (256-byte aligned)
+ *   gi_slice8_pointwise_run         enqueues out = act(conv1x1(in) + bias) on `stream`; `dev_in` / `dev_out` are device
+ *                                   tensors in the layout above (16-byte aligned, gi_slice8_tensor_bytes each), `act`
+ *                                   a GI_ACT_* value.  Needs the wide-tile kernel's support for (cin, cout).
+ * The library allocates nothing; errors as everywhere else (GI_E_INVALID, GI_E_UNSUPPORTED, GI_E_CUDA). */
+GI_API uint64_t gi_slice8_tensor_bytes(int32_t batch, int32_t H, int32_t W, int32_t C);
+GI_API gi_status gi_slice8_pointwise_blob_bytes(int32_t cin, int32_t cout, uint64_t* bytes);
+GI_API gi_status gi_slice8_pointwise_pack(const float* w, const float* bias, int32_t cin, int32_t cout, void* host_blob,
+                                          uint64_t blob_bytes);
+GI_API gi_status gi_slice8_pointwise_run(const void* dev_in, void* dev_out, const void* dev_blob, int32_t batch, int32_t H,
+                                         int32_t W, int32_t cin, int32_t cout, int32_t act, void* stream);
+
 GI_API void gi_exec_destroy(gi_exec* e);
 
 /* ---- helpers ---- */

@@ -71,6 +71,7 @@ class gi_op_info(C.Structure):
 
 EXPORTS = ["gi_graph_create", "gi_graph_input", "gi_add_op", "gi_graph_output", "gi_graph_destroy", "gi_compile",
            "gi_exec_query", "gi_exec_tensor", "gi_exec_op", "gi_exec_bind", "gi_run", "gi_run_static", "gi_run_timed", "gi_device_status", "gi_selftest_bounded_wait", "gi_exec_destroy",
+           "gi_slice8_tensor_bytes", "gi_slice8_pointwise_blob_bytes", "gi_slice8_pointwise_pack", "gi_slice8_pointwise_run",
            "gi_status_str", "gi_last_error", "gi_tensor_bytes", "gi_f32_to_f16"]
 
 _lib = None
@@ -113,6 +114,14 @@ def lib() -> C.CDLL:
     L.gi_selftest_bounded_wait.restype = C.c_int32
     L.gi_exec_destroy.argtypes = [vp]
     L.gi_exec_destroy.restype = None
+    L.gi_slice8_tensor_bytes.argtypes = [C.c_int32] * 4
+    L.gi_slice8_tensor_bytes.restype = C.c_uint64
+    L.gi_slice8_pointwise_blob_bytes.argtypes = [C.c_int32, C.c_int32, C.POINTER(C.c_uint64)]
+    L.gi_slice8_pointwise_blob_bytes.restype = C.c_int32
+    L.gi_slice8_pointwise_pack.argtypes = [vp, vp, C.c_int32, C.c_int32, vp, C.c_uint64]
+    L.gi_slice8_pointwise_pack.restype = C.c_int32
+    L.gi_slice8_pointwise_run.argtypes = [vp, vp, vp] + [C.c_int32] * 6 + [vp]
+    L.gi_slice8_pointwise_run.restype = C.c_int32
     L.gi_status_str.argtypes = [C.c_int32]
     L.gi_status_str.restype = C.c_char_p
     L.gi_last_error.argtypes = []
@@ -156,6 +165,27 @@ def gi_selftest_bounded_wait(limit_us: int, stream=None):
     waited, gave_up = C.c_uint32(0), C.c_int32(0)
     _check(lib().gi_selftest_bounded_wait(limit_us, C.byref(waited), C.byref(gave_up), _stream_ptr(stream)), "gi_selftest_bounded_wait")
     return int(waited.value), bool(gave_up.value)
+
+
+def gi_slice8_tensor_bytes(batch, H, W, Cc) -> int:
+    return int(lib().gi_slice8_tensor_bytes(batch, H, W, Cc))
+
+
+def gi_slice8_pointwise_pack(w: np.ndarray, bias: np.ndarray) -> np.ndarray:
+    """Packed weights + bias (uint8 array) of a 1x1 layer w[cout, cin] for gi_slice8_pointwise_run."""
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    bias = np.ascontiguousarray(bias, dtype=np.float32)
+    cout, cin = w.shape
+    n = C.c_uint64(0)
+    _check(lib().gi_slice8_pointwise_blob_bytes(cin, cout, C.byref(n)), "gi_slice8_pointwise_blob_bytes")
+    blob = np.zeros(int(n.value), dtype=np.uint8)
+    _check(lib().gi_slice8_pointwise_pack(w.ctypes.data, bias.ctypes.data, cin, cout, blob.ctypes.data, blob.size), "gi_slice8_pointwise_pack")
+    return blob
+
+
+def gi_slice8_pointwise_run(dev_in: int, dev_out: int, dev_blob: int, batch, H, W, cin, cout, act, stream=None) -> None:
+    """Argument marshalling only: the three pointers are device addresses (torch tensors' data_ptr())."""
+    _check(lib().gi_slice8_pointwise_run(dev_in, dev_out, dev_blob, batch, H, W, cin, cout, act, _stream_ptr(stream)), "gi_slice8_pointwise_run")
 
 
 class Graph:

@@ -3,7 +3,9 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <cstring>
 #include <mutex>
+#include <new>
 #include <string>
 #include <vector>
 
@@ -252,6 +254,66 @@ gi_status gi_run_timed(gi_exec* e, const void* const* dev_inputs, void* const* d
   for (cudaEvent_t x : ev)
     if (x) cudaEventDestroy(x);
   return st;
+}
+
+// ---- layout experiment: 1x1 convolution on tensors in slices of eight channels
+uint64_t gi_slice8_tensor_bytes(int32_t batch, int32_t H, int32_t W, int32_t C) {
+  if (batch <= 0 || H <= 0 || W <= 0 || C <= 0) return 0;
+  return static_cast<uint64_t>((C + 7) / 8) * batch * plane_pixels(H, W) * 16u;
+}
+
+namespace {
+gi_status slice8_shape(const char* who, int32_t cin, int32_t cout) {
+  if (cin <= 0 || cout <= 0) return fail(GI_E_INVALID, std::string(who) + ": cin and cout must be positive");
+  if (!pointwise_mm_supported(cin, cout)) return fail(GI_E_UNSUPPORTED, std::string(who) + ": shape not supported by the wide-tile kernel");
+  return GI_OK;
+}
+}  // namespace
+
+// the blob: packed weights at offset 0, bias behind them (256-byte aligned), exactly as pointwise_mm_pack lays them out
+gi_status gi_slice8_pointwise_blob_bytes(int32_t cin, int32_t cout, uint64_t* bytes) {
+  if (!bytes) return fail(GI_E_INVALID, "gi_slice8_pointwise_blob_bytes: null argument");
+  const gi_status st = slice8_shape("gi_slice8_pointwise_blob_bytes", cin, cout);
+  if (st != GI_OK) return st;
+  uint64_t boff = 0;
+  pointwise_mm_blob_layout(cin, cout, &boff, bytes);
+  return GI_OK;
+}
+
+gi_status gi_slice8_pointwise_pack(const float* w, const float* bias, int32_t cin, int32_t cout, void* host_blob, uint64_t blob_bytes) {
+  if (!w || !bias || !host_blob) return fail(GI_E_INVALID, "gi_slice8_pointwise_pack: null argument");
+  const gi_status st = slice8_shape("gi_slice8_pointwise_pack", cin, cout);
+  if (st != GI_OK) return st;
+  try {
+    std::vector<uint8_t> blob;
+    LaunchRec r{};
+    pointwise_mm_pack(w, bias, cin, cout, &blob, &r);
+    if (blob_bytes < blob.size()) return fail(GI_E_INVALID, "gi_slice8_pointwise_pack: host_blob too small");
+    std::memcpy(host_blob, blob.data(), blob.size());
+    return GI_OK;
+  } catch (const std::bad_alloc&) {
+    return fail(GI_E_NOMEM, "gi_slice8_pointwise_pack: out of memory");
+  }
+}
+
+gi_status gi_slice8_pointwise_run(const void* dev_in, void* dev_out, const void* dev_blob, int32_t batch, int32_t H, int32_t W,
+                                  int32_t cin, int32_t cout, int32_t act, void* stream) {
+  if (!dev_in || !dev_out || !dev_blob) return fail(GI_E_INVALID, "gi_slice8_pointwise_run: null argument");
+  if (batch <= 0 || H <= 0 || W <= 0 || cin <= 0 || cout <= 0) return fail(GI_E_INVALID, "gi_slice8_pointwise_run: sizes must be positive");
+  if (act != GI_ACT_NONE && act != GI_ACT_RELU && act != GI_ACT_RELU6) return fail(GI_E_INVALID, "gi_slice8_pointwise_run: unknown activation");
+  if ((reinterpret_cast<uintptr_t>(dev_in) | reinterpret_cast<uintptr_t>(dev_out)) & 15u)
+    return fail(GI_E_INVALID, "gi_slice8_pointwise_run: tensors must be 16-byte aligned");
+  if (reinterpret_cast<uintptr_t>(dev_blob) & 255u) return fail(GI_E_INVALID, "gi_slice8_pointwise_run: the blob must be 256-byte aligned");
+  if (!pointwise_mm_supported(cin, cout)) return fail(GI_E_UNSUPPORTED, "gi_slice8_pointwise_run: shape not supported by the wide-tile kernel");
+  const uint64_t m_total = static_cast<uint64_t>(batch) * plane_pixels(H, W);
+  if (m_total >= (1ull << 31)) return fail(GI_E_UNSUPPORTED, "gi_slice8_pointwise_run: tensor too large");
+  uint64_t boff = 0, total = 0;
+  pointwise_mm_blob_layout(cin, cout, &boff, &total);
+  const unsigned char* blob = static_cast<const unsigned char*>(dev_blob);
+  const int err = launch_pointwise_mm_slice8(dev_in, dev_out, blob, reinterpret_cast<const float*>(blob + boff),
+                                             static_cast<unsigned>(m_total), cin, cout, act, stream);
+  if (err != 0) return fail(GI_E_CUDA, std::string("gi_slice8_pointwise_run: ") + cudaGetErrorString(static_cast<cudaError_t>(err)));
+  return GI_OK;
 }
 
 }  // extern "C"

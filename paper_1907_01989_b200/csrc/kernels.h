@@ -81,7 +81,10 @@ unsigned int depthwise_pointwise_error_word(int* cuda_err);
 // streamed (pointwise_mm.cu; fp16 storage)
 bool pointwise_mm_supported(int cin, int cout);
 void pointwise_mm_pack(const float* w, const float* bias, int cin, int cout, std::vector<uint8_t>* blob, LaunchRec* r);
+void pointwise_mm_blob_layout(int cin, int cout, uint64_t* bias_off, uint64_t* total);
 int launch_pointwise_mm(const LaunchRec& r, const Ptrs& p, void** state, int launch_index, void* stream);
+int launch_pointwise_mm_slice8(const void* in, void* out, const void* wts, const float* bias, unsigned m_total, int cin, int cout,
+                               int act, void* stream);
 unsigned int pointwise_mm_error_word(int* cuda_err);
 
 // Two consecutive 1x1 convolutions (a block's projection and the next block's expansion) as one kernel (fp16 storage):

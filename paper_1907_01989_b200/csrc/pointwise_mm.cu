@@ -94,12 +94,21 @@ __device__ __forceinline__ float act1(float v, int kind) {
   if (kind == GI_ACT_RELU6) return fminf(fmaxf(v, 0.0f), 6.0f);
   return v;
 }
+// offset (in halves) of the 4 channels [4 so, 4 so + 4) of a pixel: slices of 4 channels, or - S8 - of 8
+template <bool S8>
+__device__ __forceinline__ size_t slice_offset(int so, unsigned m_total, unsigned pixel) {
+  if (S8) return (static_cast<size_t>(so >> 1) * m_total + pixel) * 8 + static_cast<size_t>(so & 1) * 4;
+  return (static_cast<size_t>(so) * m_total + pixel) * 4;
+}
 __device__ __forceinline__ void st_shared_v4(unsigned addr, unsigned a, unsigned b, unsigned c, unsigned d) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
-// ACT: activation right after the bias; TAIL: a residual add and / or a second activation follow
-template <int ACT, bool TAIL>
+// ACT: activation right after the bias; TAIL: a residual add and / or a second activation follow; S8: input and output
+// are stored in slices of 8 channels (16 bytes per pixel-slice) instead of 4 - the layout experiment of
+// gi_slice8_pointwise_*: a pixel-slice is then an operand row, the tiled copy lands the rows where the MMA reads
+// them and nothing is rearranged
+template <int ACT, bool TAIL, bool S8>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
     pointwise_mm_kernel(const __grid_constant__ CUtensorMap tmap_a, const MmParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
@@ -256,7 +265,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
           }
           const unsigned landed = smem_u32(&hdr->landed[stage]);
           mbar_expect_tx(landed, kABytes);
-          tma_load_2d(st0 + stage * p.stage_bytes, &tmap_a, px0, c * kKc, landed);
+          // (8-channel slices: the map counts 8-byte halves of the 16-byte pixel-slices)
+          if (S8) tma_load_2d(st0 + stage * p.stage_bytes, &tmap_a, 2 * px0, c * (kKc / 2), landed);
+          else tma_load_2d(st0 + stage * p.stage_bytes, &tmap_a, px0, c * kKc, landed);
         }
       }
       if (!ok) {
@@ -293,21 +304,23 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
           ok = false;
           break;
         }
-        const unsigned base = st0 + stage * p.stage_bytes + kg * 2048u;
-        unsigned lo[4][2], hi[4][2];  // pixel-slices of the even and of the odd slice, pixels lane, lane + 32, ...
+        if (!S8) {
+          const unsigned base = st0 + stage * p.stage_bytes + kg * 2048u;
+          unsigned lo[4][2], hi[4][2];  // pixel-slices of the even and of the odd slice, pixels lane, lane + 32, ...
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const unsigned px = static_cast<unsigned>(lane + 32 * j);
-          asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(lo[j][0]), "=r"(lo[j][1]) : "r"(base + px * 8u) : "memory");
-          asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(hi[j][0]), "=r"(hi[j][1]) : "r"(base + 1024u + px * 8u) : "memory");
-        }
-        __syncwarp();
+          for (int j = 0; j < 4; ++j) {
+            const unsigned px = static_cast<unsigned>(lane + 32 * j);
+            asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(lo[j][0]), "=r"(lo[j][1]) : "r"(base + px * 8u) : "memory");
+            asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(hi[j][0]), "=r"(hi[j][1]) : "r"(base + 1024u + px * 8u) : "memory");
+          }
+          __syncwarp();
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-          st_shared_v4(base + static_cast<unsigned>(lane + 32 * j) * 16u, lo[j][0], lo[j][1], hi[j][0], hi[j][1]);
-        // visible to the tensor core's proxy, then count this warp in
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        __syncwarp();
+          for (int j = 0; j < 4; ++j)
+            st_shared_v4(base + static_cast<unsigned>(lane + 32 * j) * 16u, lo[j][0], lo[j][1], hi[j][0], hi[j][1]);
+          // visible to the tensor core's proxy, then count this warp in
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+        }  // with 8-channel slices the copy itself wrote the operand rows: the warp only passes the arrival on
         if (lane == 0) {
           if (rank == 0) mbar_arrive(smem_u32(&hdr->full[stage]));
           else asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(peer_full0 + stage * 8u) : "memory");
@@ -362,11 +375,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
           for (int j = 0; j < 4; ++j) {
             rq[j] = make_uint2(0u, 0u);
             if (p.has_res && px_ok && so0 + j < p.s_out)
-              rq[j] = __ldg(reinterpret_cast<const uint2*>(p.res + (static_cast<size_t>(so0 + j) * p.m_total + pixel) * 4));
+              rq[j] = __ldg(reinterpret_cast<const uint2*>(p.res + slice_offset<S8>(so0 + j, p.m_total, pixel)));
           }
         }
-        __half* dst = p.out + (static_cast<size_t>(so0) * p.m_total + pixel) * 4;
-        const size_t slice_stride = static_cast<size_t>(p.m_total) * 4;
         tmem_ld_wait16(r);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -395,7 +406,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
             o.x = pack_f16x2<false>(act1(act1(v0.x, ACT) + q0.x, p.act_post), act1(act1(v0.y, ACT) + q0.y, p.act_post));
             o.y = pack_f16x2<false>(act1(act1(v1.x, ACT) + q1.x, p.act_post), act1(act1(v1.y, ACT) + q1.y, p.act_post));
           }
-          *reinterpret_cast<uint2*>(dst + j * slice_stride) = o;
+          *reinterpret_cast<uint2*>(p.out + slice_offset<S8>(so0 + j, p.m_total, pixel)) = o;
         }
       }
       // every tensor-memory load of this warp has completed (the wait above): a relaxed arrival is enough to let the
@@ -448,6 +459,14 @@ Tiling choose_tiling(int cin, int cout) {
 bool pointwise_mm_supported(int cin, int cout) {
   if (cin <= 0 || cout <= 0) return false;
   return choose_tiling(cin, cout).stages >= 4;
+}
+
+// Where pointwise_mm_pack puts things in an empty blob: weights at 0, bias behind them; total size.
+void pointwise_mm_blob_layout(int cin, int cout, uint64_t* bias_off, uint64_t* total) {
+  const Tiling t = choose_tiling(cin, cout);
+  const uint64_t wbytes = static_cast<uint64_t>(t.n_tiles) * t.n_chunks * 2 * t.b_bytes;
+  *bias_off = round_up_u64(wbytes, 256);
+  *total = *bias_off + static_cast<uint64_t>(t.n_tiles) * t.n_tile * sizeof(float);
 }
 
 // Dense weights as the B operand, per (output tile, K chunk, half of the tile's rows): [4 K groups][n_tile / 2 rows]
@@ -505,7 +524,7 @@ int launch_pointwise_mm(const LaunchRec& r, const Ptrs& p, void** state, int lau
   if (!attr_done) {
     cudaError_t e = cudaSuccess;
 #define GI_MM_ATTR(A, T) \
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(pointwise_mm_kernel<A, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax)
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(pointwise_mm_kernel<A, T, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax)
     GI_MM_ATTR(GI_ACT_NONE, false);
     GI_MM_ATTR(GI_ACT_RELU, false);
     GI_MM_ATTR(GI_ACT_RELU6, false);
@@ -531,7 +550,7 @@ int launch_pointwise_mm(const LaunchRec& r, const Ptrs& p, void** state, int lau
   if (smem < 120 * 1024) smem = 120 * 1024;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool tail = k.has_res || k.act_post != GI_ACT_NONE;
-#define GI_MM_LAUNCH(A, T) launch_pdl(pointwise_mm_kernel<A, T>, grid, kThreads, smem, st, tmap, k)
+#define GI_MM_LAUNCH(A, T) launch_pdl(pointwise_mm_kernel<A, T, false>, grid, kThreads, smem, st, tmap, k)
   if (tail) {
     if (k.act_pre == GI_ACT_RELU6) GI_MM_LAUNCH(GI_ACT_RELU6, true);
     else if (k.act_pre == GI_ACT_RELU) GI_MM_LAUNCH(GI_ACT_RELU, true);
@@ -542,6 +561,59 @@ int launch_pointwise_mm(const LaunchRec& r, const Ptrs& p, void** state, int lau
     else GI_MM_LAUNCH(GI_ACT_NONE, false);
   }
 #undef GI_MM_LAUNCH
+  return static_cast<int>(cudaGetLastError());
+}
+
+// The layout experiment: the same kernel on tensors stored in slices of 8 channels.  `wts` / `bias` are device copies of
+// what pointwise_mm_pack wrote (the packed weights do not depend on the activations' slice width).
+int launch_pointwise_mm_slice8(const void* in, void* out, const void* wts, const float* bias, unsigned m_total, int cin, int cout,
+                               int act, void* stream) {
+  const Tiling t = choose_tiling(cin, cout);
+  MmParams k{};
+  k.res = nullptr;
+  k.out = static_cast<__half*>(out);
+  k.wts = static_cast<const unsigned char*>(wts);
+  k.bias = bias;
+  k.m_total = m_total;
+  k.s_out = 2 * ((cout + 7) / 8);  // in 4-channel groups: the whole last 8-channel slice is written (zeros beyond cout)
+  k.n_chunks = t.n_chunks;
+  k.n_tile = t.n_tile;
+  k.n_tiles = t.n_tiles;
+  k.m_tiles = static_cast<int>((m_total + kPairRows - 1) / kPairRows);
+  k.stages = t.stages;
+  k.b_bytes = t.b_bytes;
+  k.stage_bytes = t.stage_bytes;
+  k.act_pre = act;
+  k.timeout_ns = 1000000000u;
+  static bool attr_done_dev[kMaxDevices] = {};
+  bool& attr_done = attr_done_dev[current_device_slot()];
+  if (!attr_done) {
+    cudaError_t e = cudaSuccess;
+#define GI_MM_ATTR(A) \
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(pointwise_mm_kernel<A, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax)
+    GI_MM_ATTR(GI_ACT_NONE);
+    GI_MM_ATTR(GI_ACT_RELU);
+    GI_MM_ATTR(GI_ACT_RELU6);
+#undef GI_MM_ATTR
+    if (e != cudaSuccess) return static_cast<int>(e);
+    attr_done = true;
+  }
+  CUtensorMap tmap;
+  {
+    // [slices of 8][pixels][16 bytes] as rows of 8-byte elements: a box of 128 pixels x 8 slices lands as 8 blocks of
+    // 128 16-byte rows - the canonical K-major operand layout as it is
+    const int err = encode_plane_map(&tmap, in, 2ull * m_total, (cin + 7) / 8, 2 * kRows, kKc / 2);
+    if (err != 0) return err;
+  }
+  const long long units = static_cast<long long>(k.m_tiles) * k.n_tiles;
+  const int pairs_max = device_sm_count() / 2;
+  const unsigned grid = 2u * static_cast<unsigned>(units < pairs_max ? units : pairs_max);
+  size_t smem = t.smem;
+  if (smem < 120 * 1024) smem = 120 * 1024;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (act == GI_ACT_RELU6) launch_pdl(pointwise_mm_kernel<GI_ACT_RELU6, false, true>, grid, kThreads, smem, st, tmap, k);
+  else if (act == GI_ACT_RELU) launch_pdl(pointwise_mm_kernel<GI_ACT_RELU, false, true>, grid, kThreads, smem, st, tmap, k);
+  else launch_pdl(pointwise_mm_kernel<GI_ACT_NONE, false, true>, grid, kThreads, smem, st, tmap, k);
   return static_cast<int>(cudaGetLastError());
 }
 

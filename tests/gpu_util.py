@@ -17,6 +17,21 @@ def unpack_phwc4(raw: np.ndarray, B: int, H: int, W: int, Cc: int) -> np.ndarray
     return np.ascontiguousarray(a.transpose(1, 2, 0, 3).reshape(B, H, W, S * 4)[..., :Cc])
 
 
+def pack_slice8(x: np.ndarray) -> np.ndarray:
+    """NHWC -> [ceil(C/8)][B][plane][8] (the 8-channel-slice layout of include/gi.h's layout experiment), zero padded."""
+    B, H, W, Cc = x.shape
+    S, P = (Cc + 7) // 8, (H * W + 1) // 2 * 2
+    a = np.zeros((B, P, S * 8), dtype=x.dtype)
+    a[:, : H * W, :Cc] = x.reshape(B, H * W, Cc)
+    return np.ascontiguousarray(a.reshape(B, P, S, 8).transpose(2, 0, 1, 3))
+
+
+def unpack_slice8(raw: np.ndarray, B: int, H: int, W: int, Cc: int) -> np.ndarray:
+    S, P = (Cc + 7) // 8, (H * W + 1) // 2 * 2
+    a = raw[: S * B * P * 8].reshape(S, B, P, 8)[:, :, : H * W, :]
+    return np.ascontiguousarray(a.transpose(1, 2, 0, 3).reshape(B, H, W, S * 8)[..., :Cc])
+
+
 # Every byte of the arena (and of the output buffers) starts as 0xFF: in fp16 and in fp32 storage that is a NaN.
 # The 1x1 tensor-core kernels multiply neighbouring pixels and padding lanes by structural zeros, and
 # 0 x NaN = NaN, so a kernel that leaves a padding lane or the padding pixel of an odd plane unwritten - harmless

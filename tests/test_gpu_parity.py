@@ -869,6 +869,44 @@ def test_mobilenet_v2_seams_as_one_kernel_every_tensor():
     assert api.gi_device_status() == 0
 
 
+# ---------------------------------------------------------------------- layout experiment: slices of eight channels
+S8_CASES = [  # batch, hw, cin, cout, act: ragged channels and planes, one CTA pair half empty, many output tiles, long K
+    (2, 9, 10, 22, wl.ACT_RELU), (3, 14, 144, 32, wl.ACT_NONE), (1, 33, 320, 256, wl.ACT_RELU6),
+    (4, 1, 1280, 1001, wl.ACT_NONE), (16, 14, 512, 512, wl.ACT_RELU6), (5, 7, 960, 320, wl.ACT_NONE),
+]
+
+
+@pytest.mark.parametrize("case", S8_CASES)
+def test_slice8_pointwise_matches_the_oracle(case):
+    """The wide-tile 1x1 kernel on tensors stored in slices of 8 channels (gi_slice8_pointwise_*): the tiled copy lands
+    operand rows directly.  Same seeded layer and input as the PHWC4 path, every output element against the oracle; the
+    output buffer starts as NaN bytes, so padding lanes and the padding pixel must be written (as zeros)."""
+    import torch
+    from tests.gpu_util import pack_slice8, unpack_slice8, POISON
+    batch, hw, cin, cout, act = case
+    spec = wl.single_pointwise(batch, hw, cin, cout, False, act)
+    x = wl.make_input(spec)
+    ref = og.run(spec, [x], storage="f16", fused=True)[spec.outputs[0]]
+    conv = [o for o in spec.ops if o.kind == wl.CONV2D][0]
+    blob = torch.from_numpy(api.gi_slice8_pointwise_pack(conv.weights.reshape(cout, cin), conv.bias)).to("cuda:0")
+    x_dev = torch.from_numpy(pack_slice8(x.astype(np.float16))).to("cuda:0")
+    assert x_dev.numel() * 2 == api.gi_slice8_tensor_bytes(batch, hw, hw, cin)
+    out_bytes = api.gi_slice8_tensor_bytes(batch, hw, hw, cout)
+    out_dev = torch.full((out_bytes,), POISON, dtype=torch.uint8, device="cuda:0")
+    api.gi_slice8_pointwise_run(x_dev.data_ptr(), out_dev.data_ptr(), blob.data_ptr(), batch, hw, hw, cin, cout, api._ACT[act])
+    torch.cuda.synchronize()
+    assert api.gi_device_status() == 0
+    raw = out_dev.cpu().numpy().view(np.float16).astype(np.float32)
+    assert_close(unpack_slice8(raw, batch, hw, hw, cout), ref, api.GI_F16, f"slice8 {case}")
+    # every stored value is finite (a later 1x1 layer multiplies padding lanes and the padding pixel by zero weights,
+    # and 0 x NaN = NaN), and the lanes beyond the last channel hold zeros
+    S, P = (cout + 7) // 8, (hw * hw + 1) // 2 * 2
+    phys = raw[: S * batch * P * 8].reshape(S, batch, P, 8)
+    assert np.isfinite(phys).all()
+    if cout % 8:
+        assert np.all(phys[S - 1, :, : hw * hw, cout % 8:] == 0)
+
+
 # ---------------------------------------------------------------------- the give-up path of the device-side waits
 def test_bounded_wait_runs_out_and_the_context_survives():
     """Every wait in the kernels is bounded; here one is made to run out on purpose and safely: a warp waits on a
