@@ -8,12 +8,13 @@
 //             x up to 256 output channels with tcgen05.mma.cta_group::2 (M = 256): each CTA stages its own 128
 //             pixels of the activations and its own half of the weight tile - 128 flops per fetched byte, the
 //             hardware exchanges the weight halves - and receives its 128 rows of the accumulator in its own
-//             tensor memory.  An accumulator is 256 of the 512 columns, so there are two: the sixteen drain warps
+//             tensor memory.  An accumulator is 256 of the 512 columns, so there are two: the twelve drain warps
 //             of each CTA write tile t out while the MMAs of tile t+1 run.  (One CTA per tile with the same
 //             fetch ratio needs a 256 x 256 accumulator that fills tensor memory; its drain, 5 us a tile, could
-//             not be overlapped: 641 TFLOP/s on 512 -> 512 where the pair does better than 1000.)
+//             not be overlapped: 641 TFLOP/s on 512 -> 512 and 1147 on 1280 -> 1280 where the pair does 713 and 1274.)
 //   A chunk   128 pixels x 64 channels per CTA: one tiled TMA copy lands the sixteen 4-channel slices as they lie in
-//             memory ([slice][pixel] 8-byte pixel-slices); eight warps then interleave pairs of slices into the
+//             memory ([slice][pixel] 8-byte pixel-slices); eight warps (of sixteen: even and odd chunks) then interleave pairs
+//             of slices into the
 //             canonical K-major operand rows (16 bytes = 8 channels of one pixel) in place - a K group's 2 KB of
 //             operand rows lie exactly where its two slices landed, so one warp owns a K group and needs no
 //             barrier but its own.  Exactly 2*M*N*K flops, nothing padded or duplicated.  (Gathering the rows
@@ -24,7 +25,8 @@
 //   MMA       4 tcgen05.mma (256 x N x 16) per chunk, issued by one thread of the pair's first CTA once its own
 //             repack warps and the other CTA's - they arrive on a barrier of the first CTA - have finished the
 //             chunk; a tcgen05.commit per CTA hands the stage back to both
-//   drain     bias, activation, residual, fp16, 8-byte stores (256 contiguous bytes per warp)
+//   drain     bias (fetched a tile ahead, kept in registers, broadcast by shuffle), activation, residual, fp16, 8-byte
+//             stores (256 contiguous bytes per warp)
 //
 // Tiles are numbered so that pairs running at the same time work on the output-channel tiles of the same pixels:
 // the activations come from HBM once, the re-reads hit L2.  No copy is multicast; every wait is bounded, and both
