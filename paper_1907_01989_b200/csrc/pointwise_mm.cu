@@ -13,13 +13,12 @@
 //             fetch ratio needs a 256 x 256 accumulator that fills tensor memory; its drain, 5 us a tile, could
 //             not be overlapped: 641 TFLOP/s on 512 -> 512 and 1147 on 1280 -> 1280 where the pair does 713 and 1274.)
 //   A chunk   128 pixels x 64 channels per CTA: one tiled TMA copy lands the sixteen 4-channel slices as they lie in
-//             memory ([slice][pixel] 8-byte pixel-slices); eight warps (of sixteen: even and odd chunks) then interleave pairs
-//             of slices into the
-//             canonical K-major operand rows (16 bytes = 8 channels of one pixel) in place - a K group's 2 KB of
-//             operand rows lie exactly where its two slices landed, so one warp owns a K group and needs no
-//             barrier but its own.  Exactly 2*M*N*K flops, nothing padded or duplicated.  (Gathering the rows
-//             with 8-byte cp.async instead - every copy holds a first-level cache line while in flight - fed a
-//             chunk in twice the time its MMAs take.)
+//             memory ([slice][pixel] 8-byte pixel-slices); eight warps (of sixteen: eight for the even chunks, eight
+//             for the odd ones) then interleave pairs of slices into the canonical K-major operand rows (16 bytes =
+//             8 channels of one pixel) in place - a K group's 2 KB of operand rows lie exactly where its two slices
+//             landed, so one warp owns a K group and needs no barrier but its own.  Exactly 2*M*N*K flops, nothing
+//             padded or duplicated.  (Gathering the rows with 8-byte cp.async instead - every copy holds a
+//             first-level cache line while in flight - fed a chunk in twice the time its MMAs take.)
 //   B chunk   this CTA's half of up to 256 output channels x 64 input channels of the dense weight matrix, packed
 //             at compile time, one bulk copy
 //   MMA       4 tcgen05.mma (256 x N x 16) per chunk, issued by one thread of the pair's first CTA once its own
