@@ -621,3 +621,43 @@ def test_depthwise_staging_table_is_sane_and_compiles():
     finally:
         del os.environ["GI_DW_BUF_KB"], os.environ["GI_DW_CTA_KB"]
 
+
+
+# ---------------------------------------------------------------------- layout experiment: host side
+def test_slice8_host_side():
+    """The host half of gi_slice8_pointwise_*: tensor sizes, argument checks, and where the packed weights of the
+    CTA-pair kernel put each value (the first CTA of a pair gets the first half of a tile's output channels)."""
+    import ctypes as C
+    # [ceil(C/8)][batch][plane rounded up to even][8] halves
+    assert api.gi_slice8_tensor_bytes(3, 7, 7, 20) == 3 * 3 * 50 * 16
+    assert api.gi_slice8_tensor_bytes(1, 2, 2, 8) == 1 * 1 * 4 * 16
+    assert api.gi_slice8_tensor_bytes(0, 2, 2, 8) == 0
+    rng = np.random.default_rng(11)
+    cin, cout = 72, 40  # two K chunks of 64 channels (the second one ragged), one output tile of 48 rows (two halves of 24)
+    w = (rng.integers(-64, 64, size=(cout, cin)) / 64.0).astype(np.float32)  # exactly representable in fp16
+    bias = rng.standard_normal(cout).astype(np.float32)
+    blob = api.gi_slice8_pointwise_pack(w, bias)
+    n_tile, half_rows, n_chunks = 48, 24, 2
+    b_bytes = half_rows * 64 * 2
+    assert blob.size == (n_chunks * 2 * b_bytes + 255) // 256 * 256 + n_tile * 4
+    halves = blob[: n_chunks * 2 * b_bytes].view(np.float16).astype(np.float32).reshape(n_chunks, 2, 8, half_rows, 8)
+    want = np.zeros((n_chunks, 2, 8, half_rows, 8), dtype=np.float32)
+    for co in range(cout):
+        for ci in range(cin):
+            want[ci // 64, co // half_rows, (ci % 64) // 8, co % half_rows, ci % 8] = w[co, ci]
+    assert np.array_equal(halves, want)
+    off = (n_chunks * 2 * b_bytes + 255) // 256 * 256
+    assert np.array_equal(blob[off: off + cout * 4].view(np.float32), bias)
+    assert not blob[off + cout * 4:].any()
+    # argument checks need no device
+    L = api.lib()
+    n = C.c_uint64(0)
+    assert L.gi_slice8_pointwise_blob_bytes(0, 8, C.byref(n)) == api.GI_E_INVALID
+    assert L.gi_slice8_pointwise_blob_bytes(8, 8, None) == api.GI_E_INVALID
+    assert L.gi_slice8_pointwise_pack(None, None, 8, 8, None, 0) == api.GI_E_INVALID
+    small = np.zeros(16, dtype=np.uint8)
+    assert L.gi_slice8_pointwise_pack(w.ctypes.data, bias.ctypes.data, cin, cout, small.ctypes.data, small.size) == api.GI_E_INVALID
+    assert L.gi_slice8_pointwise_run(None, None, None, 1, 2, 2, 8, 8, 0, None) == api.GI_E_INVALID
+    assert L.gi_slice8_pointwise_run(16, 32, 256, 1, 2, 2, 8, 8, 7, None) == api.GI_E_INVALID   # unknown activation
+    assert L.gi_slice8_pointwise_run(16, 40, 256, 1, 2, 2, 8, 8, 0, None) == api.GI_E_INVALID   # output not 16-byte aligned
+    assert L.gi_slice8_pointwise_run(16, 32, 128, 1, 2, 2, 8, 8, 0, None) == api.GI_E_INVALID   # blob not 256-byte aligned
