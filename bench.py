@@ -642,6 +642,10 @@ def main():
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()  # started before the warm-up so that it is sampling when the timed region begins
+    # no garbage-collection pause between two launches of a timed step: the host only enqueues work here
+    import gc
+    gc.collect()
+    gc.disable()
     for _ in range(args.warmup):
         flush.zero_()
         step_resident()
@@ -877,6 +881,7 @@ def main():
                 graph_ms = f"capture failed: {type(exc).__name__}"
             b1_launches = sum(1 for o in ex1.ops() if api.KERNEL_NAMES[o.kernel] != "none")
 
+        gc.enable()
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
             v, cores, sample, _, _ = oracle_images_per_s(spec_fn)
