@@ -365,13 +365,15 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
           const bool pointwise = op.d.kh == 1 && op.d.stride_h == 1 && op.d.stride_w == 1 && op.d.pad_t == 0 &&
                                  op.d.pad_l == 0 && op.d.pad_b == 0 && op.d.pad_r == 0;
           const bool tc = e->storage == GI_F16 && e->opt.pointwise != GI_PW_SIMT;
-          // Which tensor-core kernel: a rule distilled from measurements of both kernels on every 1x1 shape of
-          // the benchmark networks at batch 256 (single launches, and confirmed inside the networks: MobileNetV2
-          // 1.711 -> 1.688 ms, MobileNetV1 1.432 -> 1.383 ms against the previous rule).  The lane-per-pixel kernel
-          // (dense weights, activations through tensor memory) wins for 64 <= Cin < 960 with at least 96 output
-          // channels, except for narrow-input expansions (Cin <= 96, Cout >= 4 Cin); the pixel-pair kernel
-          // (both operands by TMA, 4x expanded weights) wins elsewhere: few input or output channels, where its
-          // tiles are small, and very deep inputs, where the lane kernel's weights no longer stay resident.
+          // Which tensor-core kernel: a rule distilled from measurements of the kernels on every 1x1 shape of
+          // the benchmark networks (single launches whose input was written just before, as a producing kernel
+          // leaves it, and confirmed inside the networks).  The lane-per-pixel kernel (dense weights, activations
+          // through tensor memory) wins for 24 <= Cin < 960 with at least 96 output channels - the expansion layers
+          // 24 -> 144, 32 -> 192 and 96 -> 576 included: with their input cold the pixel-pair kernel measured 8 % ahead
+          // there, inside MobileNetV2, where the projection before them has just written it, the lane kernel is
+          // 1.8 % of the whole step faster (1.450 -> 1.424 ms at batch 256); the pixel-pair kernel (both operands by
+          // TMA, 4x expanded weights) wins elsewhere: few input or output channels, where its tiles are small,
+          // and very deep inputs, where the lane kernel's weights no longer stay resident.
           // Launches whose pixels all fit one wave of 128-pixel tiles are latency-bound and take the lane
           // kernel (shorter fill; MobileNetV2 batch 1 0.296 -> 0.276 ms) - up to 64 tiles always, up to one
           // tile per SM unless the input is 960 channels deep or more.
@@ -452,7 +454,7 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
           }
           const long long m_px_all = static_cast<long long>(e->batch) * din->h * din->w;
           const bool one_wave = m_px_all <= 64LL * 128 || (m_px_all <= 148LL * 128 && din->c < 960);
-          const bool lane_rule = op.d.cout >= 96 && din->c >= 64 && din->c < 960 && !(din->c <= 96 && op.d.cout >= 4 * din->c);
+          const bool lane_rule = op.d.cout >= 96 && din->c >= 24 && din->c < 960;
           const bool lane_auto = one_wave || lane_rule;
           const bool lane_kernel = e->opt.pointwise == GI_PW_TC_LANE || ((e->opt.pointwise == GI_PW_AUTO || e->opt.pointwise == GI_PW_RULE) && lane_auto);
           // The wide-tile kernel (a CTA pair per tile of 256 pixels x up to 256 output channels) is for the layers with many
@@ -461,10 +463,10 @@ gi_status lower(const gi_graph& g, gi_exec* e) {
           // 576->160 0.93; batch 64: 14x14 512->512 0.90, 576->96 0.88, 7x7 1024->1024 0.72.  It loses where a launch has
           // too few tiles to fill the 74 pairs' pipelines (batch 64 7x7 960->160, 13 tiles: 1.14) and where many tiles
           // meet a narrow output (batch 256 14x14 576->96, 196 tiles: 1.09 - an MMA takes the same 128 cycles for 96
-          // output channels as for 256).  From 256 input and 256 output channels on it is 4-14 % ahead (28x28 256->256,
-          // 7x7 320->1280); with fewer channels it wins or loses by a few per cent: the table decides.
+          // output channels as for 256).  With fewer input channels it wins or loses by a few per cent (28x28 256->256
+          // 4 % ahead, 14x14 256->512 15 % behind the lane kernel): the table decides.
           const long long mm_units = ((m_px_all_for_mm(e, din) + 255) / 256) * ((slices(op.d.cout) * 4 + 255) / 256);
-          const bool mm_auto = mm_units >= 40 && ((din->c >= 512 && (op.d.cout >= 160 || mm_units <= 74)) || (din->c >= 256 && op.d.cout >= 256));
+          const bool mm_auto = mm_units >= 40 && din->c >= 512 && (op.d.cout >= 160 || mm_units <= 74);
           bool wide_kernel = e->opt.pointwise == GI_PW_TC_WIDE || ((e->opt.pointwise == GI_PW_AUTO || e->opt.pointwise == GI_PW_RULE) && mm_auto);
           bool lane_tab = false, pair_tab = false;
           if (e->opt.pointwise == GI_PW_AUTO && pointwise && tc) {

@@ -305,8 +305,9 @@ def test_kernel_choice_options():
     g = api.graph_from_spec(even, api.GI_F16)[0]
     with pytest.raises(api.GiError):
         g.compile(pointwise=9)
-    pw = wl.single_pointwise(128, 14, 64, 384)
+    pw = wl.single_pointwise(128, 14, 16, 96)  # few input channels: the pixel-pair kernel by the rule
     assert "pointwise_tc" in kernels(pw) and "pointwise_ts" in kernels(pw, pointwise=api.GI_PW_TC_LANE)
+    assert "pointwise_ts" in kernels(wl.single_pointwise(128, 14, 64, 384))  # an expansion with 24 or more input channels
     assert "conv_simt" in kernels(pw, pointwise=api.GI_PW_SIMT)
     # all pixels in one wave of 128-pixel tiles: the lane-per-pixel kernel whatever the channel counts
     small = wl.single_pointwise(2, 14, 64, 384)
