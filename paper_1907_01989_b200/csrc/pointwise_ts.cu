@@ -39,7 +39,6 @@ using namespace ptx;
 constexpr int kRows = 128;
 constexpr int kTransferWarps = 8;  // two per TMEM lane quarter: each moves every other group of 8 slices of a chunk
 constexpr int kDrainWarps = 16;
-constexpr int kMaxNCta = 256;  // output channels per CTA: two accumulators and the A buffers share the 512 TMEM columns
 constexpr int kThreads = 32 * (2 + kTransferWarps + kDrainWarps);
 constexpr int kMaxStages = 8;
 constexpr int kSmemHeader = 1024;
@@ -79,7 +78,8 @@ struct Header {
   unsigned tmem_addr;
   unsigned abort_flag;
 };
-static_assert(sizeof(Header) <= kSmemHeader, "header too large");
+constexpr int kBiasOffset = 256;  // the CTA's bias values (at most kMaxNcta floats) follow the barriers in the header
+static_assert(sizeof(Header) <= kBiasOffset && kBiasOffset + kMaxNcta * sizeof(float) <= kSmemHeader, "header too large");
 
 __device__ __forceinline__ void tmem_st16(unsigned taddr, const unsigned* r) {
   asm volatile(
@@ -153,6 +153,10 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) tmem_alloc(smem_u32(&hdr->tmem_addr), 512u);
+  // this CTA's bias (its output channels are the same for every tile) in shared memory, behind the barriers: the
+  // epilogue reads it per slice, and a load from global memory there queues behind everything the SM has in flight
+  float* bias_s = reinterpret_cast<float*>(smem + kBiasOffset);
+  for (int i = threadIdx.x; i < p.n_cta; i += kThreads) bias_s[i] = __ldg(p.bias + n_part * p.n_cta + i);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -302,16 +306,6 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
     const int part_id = (warp - (2 + kTransferWarps)) >> 2;     // takes every kParts-th 16-column group
     const unsigned lane_bits = static_cast<unsigned>(quarter * 32) << 16;
     const int groups = p.n_cta >> 4;
-    // This CTA's output channels are the same for every tile: lane l keeps the bias of column l % 16 of each of this
-    // warp's 16-column groups and the epilogue broadcasts from there.  (A load from global memory per slice inside the
-    // epilogue queues behind the barrier polls and shared-memory traffic of the other warps.)
-    constexpr int kGroupsPerWarp = (kMaxNCta / 16 + kParts - 1) / kParts;
-    float bpre[kGroupsPerWarp];
-#pragma unroll
-    for (int k = 0; k < kGroupsPerWarp; ++k) {
-      const int g = part_id + k * kParts;
-      bpre[k] = g < groups ? __ldg(p.bias + n_part * p.n_cta + g * 16 + (lane & 15)) : 0.f;
-    }
     unsigned tile = 0;
     for (int m = m_first; m < p.m_tiles; m += m_step, ++tile) {
       const unsigned acc = tile & 1u, acc_phase = (tile >> 1) & 1u;
@@ -334,10 +328,7 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
       tc_fence_after();
       if (tile == 0 && threadIdx.x == 32 * (2 + kTransferWarps)) GI_TRACE_EVENT(g_ts_trace, 6);
       const unsigned t_addr = tmem_base + lane_bits + acc * acc_cols;
-#pragma unroll
-      for (int k = 0; k < kGroupsPerWarp; ++k) {
-        const int g = part_id + k * kParts;
-        if (g >= groups) break;
+      for (int g = part_id; g < groups; g += kParts) {
         if (TAIL) fetch_res(res_next, g + kParts);
         unsigned r[16];
         tmem_ld16(t_addr + g * 16, r);
@@ -345,24 +336,17 @@ __global__ void __launch_bounds__(kThreads, 1) pointwise_ts_kernel(const __grid_
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int so = (n_part * p.n_cta) / 4 + g * 4 + j;
-          float4 b;
-          b.x = __shfl_sync(0xffffffffu, bpre[k], 4 * j);
-          b.y = __shfl_sync(0xffffffffu, bpre[k], 4 * j + 1);
-          b.z = __shfl_sync(0xffffffffu, bpre[k], 4 * j + 2);
-          b.w = __shfl_sync(0xffffffffu, bpre[k], 4 * j + 3);
           if (so >= p.s_out || !px_ok) continue;
+          const float4 b = *reinterpret_cast<const float4*>(bias_s + g * 16 + 4 * j);
           const size_t off = (static_cast<size_t>(so) * p.m_total_px + pixel) * 4;  // in halves
           const float2 v0 = __fadd2_rn(make_float2(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1])), make_float2(b.x, b.y));
           const float2 v1 = __fadd2_rn(make_float2(__uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3])), make_float2(b.z, b.w));
           __half2 h0, h1;
           if (!TAIL) {
-            // clamping after the rounding equals rounding after the clamp: 0 and 6 are fp16 values
-            h0 = __floats2half2_rn(v0.x, v0.y);
-            h1 = __floats2half2_rn(v1.x, v1.y);
-            if (ACT != GI_ACT_NONE) {
-              h0 = __hmax2(h0, __float2half2_rn(0.f));
-              h1 = __hmax2(h1, __float2half2_rn(0.f));
-            }
+            // the conversion clamps at zero itself; clamping at 6 after the rounding equals rounding after the clamp
+            const unsigned u0 = pack_f16x2<ACT != GI_ACT_NONE>(v0.x, v0.y), u1 = pack_f16x2<ACT != GI_ACT_NONE>(v1.x, v1.y);
+            h0 = *reinterpret_cast<const __half2*>(&u0);
+            h1 = *reinterpret_cast<const __half2*>(&u1);
             if (ACT == GI_ACT_RELU6) {
               h0 = __hmin2(h0, __float2half2_rn(6.f));
               h1 = __hmin2(h1, __float2half2_rn(6.f));
