@@ -28,8 +28,8 @@
 //             stores (256 contiguous bytes per warp)
 //
 // Tiles are numbered so that pairs running at the same time work on the output-channel tiles of the same pixels:
-// the activations come from HBM once, the re-reads hit L2.  No copy is multicast; every wait is bounded, and both
-// CTAs of a pair meet at a cluster barrier before either releases tensor memory or leaves.
+// the activations come from HBM once, the re-reads hit L2.  Every copy goes to the one CTA that issued it; every wait
+// is bounded, and both CTAs of a pair meet at a cluster barrier before either releases tensor memory or leaves.
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
