@@ -202,6 +202,33 @@ def test_expected_fused_counts_and_arena():
         assert ex.info.arena_bytes == ex.info.lower_bound_bytes
 
 
+def test_kernels_of_the_benchmark_step():
+    """Which kernel runs which layer of MobileNetV2-224 at batch 256 (the bench configuration): the generated launch
+    table and the cross-operator rule decide at compile time, so the mix is checked without a GPU.  The expansion
+    layers from 24 input channels on and the 14x14 / 7x7 projections run on the lane-per-pixel kernel, the 112x112
+    layers and the 56x56 / 28x28 projections on the pixel-pair kernel, the 7x7 layers with 576 or more input channels on
+    the CTA-pair kernel, four 14x14 seams as one kernel each; no block runs as one kernel."""
+    from collections import Counter
+    ex = api.graph_from_spec(wl.mobilenet_v2(256), api.GI_F16)[0].compile()
+    ops = ex.ops()
+    mix = Counter(api.KERNEL_NAMES[o.kernel] for o in ops)
+    assert mix["depthwise"] == 17 and mix["conv3x3_tc"] == 1 and mix["pool"] == 1 and mix["unpack"] == 1
+    assert mix["pointwise_chain"] == 4 and mix["inverted_residual"] == 0 and mix["depthwise_pointwise"] == 0
+    assert mix["pointwise_ts"] + mix["pointwise_tc"] + mix["pointwise_mm"] == 27
+    assert mix["pointwise_mm"] >= 3 and mix["pointwise_ts"] >= 12
+    assert sum(v for k, v in mix.items() if k != "none") == 51
+    for o in ops:
+        name = api.KERNEL_NAMES[o.kernel]
+        if name in ("pointwise_ts", "pointwise_tc", "pointwise_mm"):
+            tin, tout = ex.tensor(o.inputs[0]), ex.tensor(o.output)
+            if tin.h == 7 and tin.c >= 576:
+                assert name == "pointwise_mm", (tin.h, tin.c, tout.c)
+            if tout.c >= 4 * tin.c and tin.c >= 24:
+                assert name == "pointwise_ts", (tin.h, tin.c, tout.c)  # an expansion layer
+            if tin.h == 112:
+                assert name == "pointwise_tc", (tin.h, tin.c, tout.c)
+
+
 # ---------------------------------------------------------------------- error behaviour
 def _conv_desc(x, cout=8, k=1, **kw):
     d = api.gi_op_desc()
